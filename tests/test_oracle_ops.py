@@ -1,0 +1,271 @@
+"""Pins for the oracle's compute operators and whole blocks: closed forms, invariants,
+textbook special cases and brute force on tiny inputs.  CPU only."""
+import itertools
+import math
+
+import numpy as np
+import pytest
+
+from oracle import layout, llama, ops, swin
+
+rng = np.random.default_rng(11)
+
+
+# ---------------------------------------------------------------- normalisation / linear
+def test_layernorm_invariants():
+    x = rng.standard_normal((6, 32)) * 3 + 1.5
+    eps = 1e-5
+    y = ops.layernorm(x, np.ones(32), np.zeros(32), eps)
+    assert np.allclose(y.mean(-1), 0, atol=1e-12)
+    var = x.var(-1)                                  # biased
+    assert np.allclose(y.var(-1), var / (var + eps), rtol=1e-12)
+    assert np.allclose(ops.layernorm(x + 7.0, np.ones(32), np.zeros(32), eps), y, atol=1e-9)
+    g, b = rng.standard_normal(32), rng.standard_normal(32)
+    assert np.allclose(ops.layernorm(x, g, b, eps), y * g + b, atol=1e-12)
+    # brute force on one row
+    r = x[0]
+    mu = sum(r) / 32
+    v = sum((t - mu) ** 2 for t in r) / 32
+    assert np.allclose(y[0], [(t - mu) / math.sqrt(v + eps) for t in r], atol=1e-12)
+
+
+def test_rmsnorm_invariants():
+    x = rng.standard_normal((5, 64))
+    y = ops.rmsnorm(x, np.ones(64), 1e-5)
+    assert np.allclose(np.sqrt((y * y).mean(-1)), 1.0, atol=1e-4)
+    assert np.allclose(ops.rmsnorm(3.0 * x, np.ones(64), 0.0), ops.rmsnorm(x, np.ones(64), 0.0), atol=1e-12)
+    r = x[1]
+    ms = sum(t * t for t in r) / 64
+    g = rng.standard_normal(64)
+    assert np.allclose(ops.rmsnorm(x, g, 1e-5)[1], [t * gg / math.sqrt(ms + 1e-5) for t, gg in zip(r, g)], atol=1e-12)
+
+
+def test_linear_identity_and_bruteforce():
+    x = rng.standard_normal((4, 6))
+    assert np.array_equal(ops.linear(x, np.eye(6)), x)
+    w, b = rng.standard_normal((3, 6)), rng.standard_normal(3)
+    y = ops.linear(x, w, b)
+    for m, n in itertools.product(range(4), range(3)):
+        assert abs(y[m, n] - (sum(x[m, k] * w[n, k] for k in range(6)) + b[n])) < 1e-12
+
+
+def test_gelu_pins():
+    assert ops.gelu(np.array([0.0]))[0] == 0.0
+    u = rng.standard_normal(50) * 3
+    assert np.allclose(ops.gelu(u) - ops.gelu(-u), u, atol=1e-12)
+    assert abs(ops.gelu(np.array([1.0]))[0] - 0.8413447460685429) < 1e-12     # Phi(1)
+    assert abs(ops.gelu(np.array([-1.0]))[0] + 0.15865525393145707) < 1e-12
+    assert np.allclose(ops.gelu(u), [0.5 * t * (1 + math.erf(t / math.sqrt(2))) for t in u], atol=1e-14)
+
+
+def test_softmax_pins():
+    s = rng.standard_normal((3, 4, 9)) * 5
+    p = ops.softmax(s)
+    assert np.allclose(p.sum(-1), 1.0, atol=1e-13)
+    assert np.allclose(ops.softmax(s + 100.0), p, atol=1e-13)
+    assert np.allclose(ops.softmax(np.full((2, 5), 3.3)), 0.2)
+    r = s[0, 0]
+    e = [math.exp(t - max(r)) for t in r]
+    assert np.allclose(p[0, 0], [t / sum(e) for t in e], atol=1e-14)
+
+
+# ---------------------------------------------------------------- bias / mask / rope
+def test_rel_pos_index_pins():
+    idx = ops.rel_pos_index(7)
+    assert idx.min() == 0 and idx.max() == 168 and len(np.unique(idx)) == 169
+    assert (np.diag(idx) == 84).all()
+    ws = 7
+    for i, j, k, l in [(0, 8, 10, 18), (3, 48, 0, 45), (20, 6, 34, 20)]:
+        di = (i // ws - j // ws, i % ws - j % ws)
+        dk = (k // ws - l // ws, k % ws - l % ws)
+        assert (di == dk) == (idx[i, j] == idx[k, l])
+    # equal displacement <=> equal index, exhaustively
+    disp = {}
+    for i in range(49):
+        for j in range(49):
+            key = (i // ws - j // ws, i % ws - j % ws)
+            assert disp.setdefault(key, idx[i, j]) == idx[i, j]
+    assert len(disp) == 169
+    idx4 = ops.rel_pos_index(4)
+    assert idx4.max() == 48 and (np.diag(idx4) == 24).all()
+
+
+@pytest.mark.parametrize("H,W,ws,s,nontrivial", [(8, 8, 4, 2, 3), (14, 14, 7, 3, 3), (56, 56, 7, 3, 15), (21, 21, 7, 3, 5)])
+def test_shift_mask_no_wrap_characterisation(H, W, ws, s, nontrivial):
+    """Two tokens of one shifted window may attend iff, in ORIGINAL coordinates, they are
+    not separated by the image seam: |dh| < ws and |dw| < ws."""
+    mask = ops.shifted_window_mask(H, W, ws, s)
+    nWh, nWw = H // ws, W // ws
+    assert mask.shape == (nWh * nWw, ws * ws, ws * ws)
+    assert set(np.unique(mask).tolist()) <= {0.0, -100.0}
+    assert sum(1 for m in mask if (m != 0).any()) == nontrivial
+    for wy, wx in itertools.product(range(nWh), range(nWw)):
+        coords = [((wy * ws + ty + s) % H, (wx * ws + tx + s) % W) for ty in range(ws) for tx in range(ws)]
+        m = mask[wy * nWw + wx]
+        for i, (hi, wi) in enumerate(coords):
+            for j, (hj, wj) in enumerate(coords):
+                ok = abs(hi - hj) < ws and abs(wi - wj) < ws
+                assert (m[i, j] == 0.0) == ok
+
+
+def test_rope_pins():
+    S, D = 9, 16
+    q, k = rng.standard_normal((S, D)), rng.standard_normal((S, D))
+    rq = ops.rope(q, 10000.0)
+    assert np.allclose(rq[0], q[0])                                         # position 0 is identity
+    half = D // 2
+    assert np.allclose(rq[:, :half] ** 2 + rq[:, half:] ** 2, q[:, :half] ** 2 + q[:, half:] ** 2)
+    # <RoPE(q,m), RoPE(k,n)> depends only on m - n: place the same vectors at other positions
+    qq, kk = np.tile(q[0], (S, 1)), np.tile(k[0], (S, 1))
+    a, b = ops.rope(qq, 10000.0), ops.rope(kk, 10000.0)
+    assert abs(a[5] @ b[3] - a[7] @ b[5]) < 1e-12 and abs(a[2] @ b[2] - a[8] @ b[8]) < 1e-12
+    # brute force of one element pair
+    p, i = 4, 3
+    phi = p * 10000.0 ** (-(2 * i) / D)
+    assert abs(rq[p, i] - (q[p, i] * math.cos(phi) - q[p, i + half] * math.sin(phi))) < 1e-12
+    assert abs(rq[p, i + half] - (q[p, i + half] * math.cos(phi) + q[p, i] * math.sin(phi))) < 1e-12
+
+
+# ---------------------------------------------------------------- attention
+def _attention_bruteforce(q, k, v, allowed):
+    T, d = q.shape
+    out = np.zeros((T, v.shape[1]))
+    for i in range(T):
+        sc = [sum(q[i, e] * k[j, e] for e in range(d)) / math.sqrt(d) if allowed(i, j) else None for j in range(T)]
+        m = max(t for t in sc if t is not None)
+        w = [math.exp(t - m) if t is not None else 0.0 for t in sc]
+        for j in range(T):
+            out[i] += w[j] / sum(w) * v[j]
+    return out
+
+
+def test_window_attention_reduces_to_plain_attention():
+    # ws = H = W, no shift, zero bias table  =>  textbook multi-head attention over all tokens
+    ws, heads, d = 3, 2, 4
+    T = ws * ws
+    q, k, v = (rng.standard_normal((1, heads, T, d)) for _ in range(3))
+    o = swin.window_attention(q, k, v, np.zeros(((2 * ws - 1) ** 2, heads)), ws)
+    for h in range(heads):
+        assert np.allclose(o[0, h], _attention_bruteforce(q[0, h], k[0, h], v[0, h], lambda i, j: True), atol=1e-12)
+
+
+def test_window_attention_bias_is_added_per_head():
+    ws, heads, d = 2, 2, 4
+    T = 4
+    q = np.zeros((1, heads, T, d))
+    k = np.zeros((1, heads, T, d))
+    v = rng.standard_normal((1, heads, T, d))
+    table = np.zeros((9, heads))
+    table[4, 1] = 50.0            # centre of the table = zero displacement, head 1 only
+    o = swin.window_attention(q, k, v, table, ws)
+    assert np.allclose(o[0, 0], v[0, 0].mean(0, keepdims=True).repeat(T, 0))   # head 0 uniform
+    assert np.allclose(o[0, 1], v[0, 1], atol=1e-12)                            # head 1: diagonal dominates
+
+
+def test_causal_attention_pins():
+    H, S, D = 2, 7, 4
+    q, k, v = (rng.standard_normal((H, S, D)) for _ in range(3))
+    o = llama.causal_attention(q, k, v)
+    assert np.allclose(o[:, 0], v[:, 0])
+    for h in range(H):
+        assert np.allclose(o[h], _attention_bruteforce(q[h], k[h], v[h], lambda i, j: j <= i), atol=1e-12)
+    o0 = llama.causal_attention(np.zeros_like(q), k, v)
+    for i in range(S):
+        assert np.allclose(o0[:, i], v[:, : i + 1].mean(1))
+
+
+# ---------------------------------------------------------------- whole blocks
+def _params(C, heads, ws, mlp_ratio, scale=0.2):
+    p = {"ln1_g": 1 + 0.1 * rng.standard_normal(C), "ln1_b": 0.1 * rng.standard_normal(C),
+         "w_qkv": scale * rng.standard_normal((3 * C, C)), "b_qkv": 0.1 * rng.standard_normal(3 * C),
+         "rel_bias_table": 0.3 * rng.standard_normal(((2 * ws - 1) ** 2, heads)),
+         "w_proj": scale * rng.standard_normal((C, C)), "b_proj": 0.1 * rng.standard_normal(C)}
+    if mlp_ratio:
+        p.update({"ln2_g": 1 + 0.1 * rng.standard_normal(C), "ln2_b": 0.1 * rng.standard_normal(C),
+                  "w_fc1": scale * rng.standard_normal((C * mlp_ratio, C)), "b_fc1": 0.1 * rng.standard_normal(C * mlp_ratio),
+                  "w_fc2": scale * rng.standard_normal((C, C * mlp_ratio)), "b_fc2": 0.1 * rng.standard_normal(C)})
+    return p
+
+
+def test_swin_block_uniform_attention_closed_form():
+    """w_q = w_k = 0 and a zero bias table make the softmax uniform over allowed keys, so
+    each token's attention output is the mean of v over the tokens of its shifted window
+    that are not across the seam -- computed here token by token in ORIGINAL coordinates,
+    with no partition or roll code."""
+    B, H, W, C, heads, ws, s = 2, 8, 8, 8, 2, 4, 2
+    p = _params(C, heads, ws, 0)
+    p["w_qkv"][: 2 * C] = 0.0
+    p["b_qkv"][: 2 * C] = 0.0
+    p["rel_bias_table"][:] = 0.0
+    x = rng.standard_normal((B, H, W, C))
+    y = swin.swin_block(x, p, heads=heads, window=ws, shift=s, mlp_ratio=0)
+    xn = ops.layernorm(x, p["ln1_g"], p["ln1_b"], 1e-5)
+    vfull = xn @ p["w_qkv"][2 * C:].T + p["b_qkv"][2 * C:]                 # [B,H,W,C]
+    exp = np.zeros_like(x)
+    for b, h, w in itertools.product(range(B), range(H), range(W)):
+        # shifted coordinates decide the window; original coordinates decide the seam
+        hs, wsft = (h - s) % H, (w - s) % W
+        members = []
+        for h2, w2 in itertools.product(range(H), range(W)):
+            h2s, w2s = (h2 - s) % H, (w2 - s) % W
+            if h2s // ws == hs // ws and w2s // ws == wsft // ws and abs(h2 - h) < ws and abs(w2 - w) < ws:
+                members.append(vfull[b, h2, w2])
+        exp[b, h, w] = x[b, h, w] + np.mean(members, axis=0) @ p["w_proj"].T + p["b_proj"]
+    assert np.allclose(y, exp, atol=1e-10)
+
+
+def test_swin_block_special_cases():
+    B, H, W, C, heads, ws = 1, 8, 8, 8, 2, 4
+    x = rng.standard_normal((B, H, W, C))
+    p = _params(C, heads, ws, 2)
+    # all linear weights and biases zero => y = x (both halves)
+    z = {k: (np.zeros_like(v) if k.startswith(("w_", "b_")) else v) for k, v in p.items()}
+    assert np.allclose(swin.swin_block(x, z, heads=heads, window=ws, shift=2, mlp_ratio=2), x)
+    # a block is equivariant to a cyclic translation by a whole window when unshifted
+    y0 = swin.swin_block(x, p, heads=heads, window=ws, shift=0, mlp_ratio=2)
+    xt = layout.roll(layout.roll(x, ws, 1), ws, 2)
+    yt = swin.swin_block(xt, p, heads=heads, window=ws, shift=0, mlp_ratio=2)
+    assert np.allclose(layout.roll(layout.roll(y0, ws, 1), ws, 2), yt, atol=1e-12)
+    # shift changes the result (the shifted path is not a no-op)
+    y2 = swin.swin_block(x, p, heads=heads, window=ws, shift=2, mlp_ratio=2)
+    assert np.abs(y2 - y0).max() > 1e-3
+    # single window covering the image, no shift: block == plain MHA + MLP written directly
+    ws2 = 8
+    p2 = _params(C, heads, ws2, 2)
+    p2["rel_bias_table"][:] = 0.0
+    y = swin.swin_block(x, p2, heads=heads, window=ws2, shift=0, mlp_ratio=2)
+    xn = ops.layernorm(x, p2["ln1_g"], p2["ln1_b"], 1e-5).reshape(H * W, C)
+    qkv = xn @ p2["w_qkv"].T + p2["b_qkv"]
+    d = C // heads
+    att = np.zeros((H * W, C))
+    for h in range(heads):
+        q, k, v = (qkv[:, i * C + h * d: i * C + (h + 1) * d] for i in range(3))
+        att[:, h * d:(h + 1) * d] = _attention_bruteforce(q, k, v, lambda i, j: True)
+    y1 = x.reshape(H * W, C) + att @ p2["w_proj"].T + p2["b_proj"]
+    yn = ops.layernorm(y1, p2["ln2_g"], p2["ln2_b"], 1e-5)
+    zz = y1 + ops.gelu(yn @ p2["w_fc1"].T + p2["b_fc1"]) @ p2["w_fc2"].T + p2["b_fc2"]
+    assert np.allclose(y.reshape(H * W, C), zz, atol=1e-10)
+
+
+def test_attn_layer_against_direct_restatement():
+    S, heads, D = 6, 2, 8
+    hidden = heads * D
+    x = rng.standard_normal((1, S, hidden))
+    p = {"rms_g": 1 + 0.1 * rng.standard_normal(hidden), "w_qkv": 0.3 * rng.standard_normal((3 * hidden, hidden)),
+         "w_o": 0.3 * rng.standard_normal((hidden, hidden))}
+    y = llama.attn_layer(x, p, heads=heads, head_dim=D, add_residual=True)
+    xn = x[0] * p["rms_g"] / np.sqrt((x[0] ** 2).mean(-1, keepdims=True) + 1e-5)
+    qkv = xn @ p["w_qkv"].T
+    att = np.zeros((S, hidden))
+    for h in range(heads):
+        q, k, v = (qkv[:, i * hidden + h * D: i * hidden + (h + 1) * D] for i in range(3))
+        att[:, h * D:(h + 1) * D] = _attention_bruteforce(ops.rope(q, 10000.0), ops.rope(k, 10000.0), v, lambda i, j: j <= i)
+    assert np.allclose(y[0], x[0] + att @ p["w_o"].T, atol=1e-10)
+    # q = k = 0 => prefix means of v pass through w_o
+    p0 = dict(p)
+    p0["w_qkv"] = p["w_qkv"].copy()
+    p0["w_qkv"][: 2 * hidden] = 0
+    y0 = llama.attn_layer(x, p0, heads=heads, head_dim=D)
+    v = (xn @ p["w_qkv"].T)[:, 2 * hidden:]
+    pm = np.cumsum(v, 0) / np.arange(1, S + 1)[:, None]
+    assert np.allclose(y0[0], pm @ p["w_o"].T, atol=1e-10)
