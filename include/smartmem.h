@@ -1,0 +1,204 @@
+/*
+ * smartmem.h -- C ABI of the layout-transformation-elimination hot path.
+ *
+ * The method (SmartMem, ASPLOS '24) removes Reshape / Transpose / Slice / Gather-class
+ * operators ("Fixed output" operators, Table 3) from a transformer operator chain by
+ * replacing them with index computation inside the operator they are fused with
+ * (Section 3.2.1, "Operator Elimination based on Index Comprehension"), after reducing the
+ * index arithmetic to its cheapest form (Section 3.2.1, "Strength reduction on index
+ * computation").  This library does that for linear operator chains on one B200:
+ *
+ *   smartmem_plan        host-only planner: operator chain + tensor layouts -> kernel steps,
+ *                        each with composed, strength-reduced index maps
+ *   smartmem_run_chain   runs a planned chain on a CUDA stream
+ *   smartmem_swin_block  one Swin Transformer block (shifted-window attention + MLP)
+ *   smartmem_attn_layer  one decoder attention layer (RMSNorm, QKV, RoPE, causal attention, o_proj)
+ *
+ * Every entry point takes a `mode`: SMARTMEM_ELIMINATE folds all layout operators into the
+ * operand loads / result stores of the compute kernels; SMARTMEM_EXPLICIT runs the same
+ * compute kernels but materialises every data-moving layout operator with a copy kernel, so
+ * the gain from elimination can be measured.
+ *
+ * Conventions
+ *   - All data pointers are DEVICE pointers owned by the caller unless a comment says "host".
+ *     The library never allocates device memory; scratch comes from the caller's workspace.
+ *   - Tensors are row-major (last dimension contiguous) unless strides are given.  Linear
+ *     weights are [out_features, in_features]: the reduction dimension is the contiguous
+ *     one for both GEMM operands (Section 3.2.2, reduction-dimension layout rule).
+ *   - Calls validate on the host, enqueue work on the given stream and return without
+ *     synchronising.  The return value is a smartmem_status_t.  Nothing aborts or prints.
+ *   - Device-side waits are bounded; a wait that runs out sets a device status word that
+ *     smartmem_last_device_status() reads back.
+ *   - There is no CPU fallback: without a CUDA device the run entry points return
+ *     SMARTMEM_ERR_CUDA.
+ */
+#ifndef SMARTMEM_H_
+#define SMARTMEM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  SMARTMEM_OK = 0,
+  SMARTMEM_ERR_INVALID_ARG = -1, /* null pointer, bad enum, bad count                    */
+  SMARTMEM_ERR_SHAPE = -2,       /* shapes inconsistent with the operator                */
+  SMARTMEM_ERR_UNSUPPORTED = -3, /* valid request the kernels do not cover               */
+  SMARTMEM_ERR_WORKSPACE = -4,   /* workspace too small                                  */
+  SMARTMEM_ERR_ALIGNMENT = -5,   /* a base pointer is not 16-byte aligned                */
+  SMARTMEM_ERR_CUDA = -6,        /* a CUDA runtime/driver call failed (or no device)     */
+  SMARTMEM_ERR_TIMEOUT = -7,     /* a bounded device-side wait ran out                   */
+  SMARTMEM_ERR_BOUNDS = -8       /* debug bounds check tripped                           */
+} smartmem_status_t;
+
+typedef enum { SMARTMEM_F32 = 0, SMARTMEM_BF16 = 1 } smartmem_dtype_t;
+typedef enum { SMARTMEM_ELIMINATE = 0, SMARTMEM_EXPLICIT = 1 } smartmem_mode_t;
+
+/* Operator vocabulary of a chain.  Layout operators have a Fixed output layout (Table 3,
+ * right column) and are the ones elimination removes; compute operators are kept. */
+typedef enum {
+  SMARTMEM_OP_RESHAPE = 0,          /* shape[] = new shape                                 */
+  SMARTMEM_OP_TRANSPOSE = 1,        /* perm[]: out.shape[k] = in.shape[perm[k]]            */
+  SMARTMEM_OP_ROLL = 2,             /* axis, shift[0]: out[j] = in[(j - shift) mod N]      */
+  SMARTMEM_OP_SLICE = 3,            /* start[], shape[] = extent                           */
+  SMARTMEM_OP_WINDOW_PARTITION = 4, /* [B,H,W,C] -> [B*H/ws*W/ws, ws*ws, C]; window = ws   */
+  SMARTMEM_OP_WINDOW_REVERSE = 5,   /* inverse; shape[0..2] = B,H,W                        */
+  SMARTMEM_OP_COPY = 16,            /* consumer: writes the current tensor contiguously    */
+  SMARTMEM_OP_LINEAR = 17,          /* consumer: out[M,N] = A[M,K] W[N,K]^T, W = side_input[0] */
+  SMARTMEM_OP_BMM_NT = 18           /* consumer: out[..,i,j] = sum_e A[..,i,e] B[..,j,e]; B is the
+                                       result of running the same layout run on side_input[0] */
+} smartmem_op_kind_t;
+
+#define SMARTMEM_MAX_DIMS 8
+#define SMARTMEM_MAX_ATOMS 16
+#define SMARTMEM_MAX_ROLLS 4
+
+typedef struct {
+  int32_t kind;                      /* smartmem_op_kind_t                                  */
+  int32_t ndim;                      /* entries used in shape / perm / start                */
+  int64_t shape[SMARTMEM_MAX_DIMS];  /* reshape target, slice extent, window_reverse B,H,W  */
+  int32_t perm[SMARTMEM_MAX_DIMS];   /* transpose                                           */
+  int64_t start[SMARTMEM_MAX_DIMS];  /* slice                                               */
+  int64_t shift;                     /* roll                                                */
+  int32_t axis;                      /* roll                                                */
+  int32_t window;                    /* window partition / reverse                          */
+  int32_t side_input[2];             /* index into the plan's inputs[] (weights, 2nd operand) */
+} smartmem_op_t;
+
+typedef struct {
+  int32_t dtype;                     /* smartmem_dtype_t                                    */
+  int32_t ndim;
+  int64_t shape[SMARTMEM_MAX_DIMS];
+  int64_t stride[SMARTMEM_MAX_DIMS]; /* in elements; all zero = contiguous row-major        */
+} smartmem_tensor_desc_t;
+
+/* A composed index map in canonical form (Section 3.2.1: identity / split / merge index
+ * dependencies derived from static shapes, then strength-reduced).  The consumer's linear
+ * index i (row-major over its logical shape) is written in mixed radix over `extent[]`
+ * (atom 0 is the most significant digit); the source offset in elements is
+ *
+ *     base + sum_{a : roll_of[a] < 0} digit_a * src_stride[a]
+ *          + sum_r ((sum_{a : roll_of[a] == r} digit_a * roll_weight[a] + roll_shift[r]) mod roll_mod[r]) * roll_stride[r]
+ *
+ * i.e. no division or modulo by tensor extents survives except one modulo per rolled
+ * dimension.  klass: 0 identity (the chain vanishes), 1 affine (no roll; a TMA tensor map or
+ * a tiled transpose can express it), 2 strided gather with rolls, 3 not canonicalisable
+ * (the split points of the shapes do not refine each other): only the sequential
+ * divide/modulo program -- the unoptimised form of Fig. 4 -- can evaluate it. */
+typedef struct {
+  int32_t n_atoms;
+  int64_t extent[SMARTMEM_MAX_ATOMS];
+  int64_t src_stride[SMARTMEM_MAX_ATOMS];
+  int32_t roll_of[SMARTMEM_MAX_ATOMS];
+  int64_t roll_weight[SMARTMEM_MAX_ATOMS];
+  int32_t n_rolls;
+  int64_t roll_shift[SMARTMEM_MAX_ROLLS];
+  int64_t roll_mod[SMARTMEM_MAX_ROLLS];
+  int64_t roll_stride[SMARTMEM_MAX_ROLLS];
+  int64_t base;
+  int64_t n_elements;                /* number of consumer elements                         */
+  int32_t vec_elems;                 /* widest power-of-two run (<= 16 bytes) that is contiguous
+                                        in both source and consumer and never straddles a wrap */
+  int32_t klass;
+} smartmem_index_map_t;
+
+typedef struct smartmem_plan smartmem_plan_t; /* opaque, library-owned, host memory */
+
+/* Operator classification (Table 3) and the pairwise decisions of Tables 5 and 6.
+ * quadrant: 0 ILD&Variable, 1 ILI&Variable, 2 ILD&Fixed, 3 ILI&Fixed.
+ * action  : 0 keep both, 1 try fuse, 2 eliminate 1st, 3 eliminate 2nd, 4 eliminate both.
+ * result  : resulting quadrant, or -1 where the table says N/A.
+ * search  : 0 no search, 1 search both, 2 search fused, 3 search 1st, 4 search 2nd. */
+int smartmem_op_quadrant(int32_t op_kind, int32_t* quadrant);
+int smartmem_pair_decision(int32_t first_quadrant, int32_t second_quadrant, int32_t* action,
+                           int32_t* result, int32_t* search);
+
+/* Host only (no CUDA call).  Walks the chain, splits it at compute operators, and for each
+ * maximal run of layout operators composes the index map (ELIMINATE) or emits one copy
+ * step per data-moving layout operator (EXPLICIT; a Reshape of a contiguous tensor stays
+ * metadata).  inputs[0] is the chain's input, other entries are side inputs.
+ * Errors: INVALID_ARG, SHAPE (operator/shape mismatch), UNSUPPORTED. */
+int smartmem_plan(const smartmem_op_t* ops, int32_t n_ops, const smartmem_tensor_desc_t* inputs,
+                  int32_t n_inputs, int32_t mode, smartmem_plan_t** out_plan);
+int smartmem_plan_destroy(smartmem_plan_t* plan);
+/* Number of kernel steps in total and how many of them are layout copies. */
+int smartmem_plan_num_steps(const smartmem_plan_t* plan, int32_t* n_steps, int32_t* n_copies);
+/* Index map of operand `operand` (0 = first/A operand, 1 = second/B operand) of step `step`. */
+int smartmem_plan_get_map(const smartmem_plan_t* plan, int32_t step, int32_t operand,
+                          smartmem_index_map_t* out);
+/* Logical shape of the chain's result. */
+int smartmem_plan_output_desc(const smartmem_plan_t* plan, smartmem_tensor_desc_t* out);
+/* Bytes of device workspace smartmem_run_chain needs (intermediate copies in EXPLICIT mode). */
+int smartmem_plan_workspace_bytes(const smartmem_plan_t* plan, size_t* bytes);
+/* Host evaluators, for tests: source offset of consumer element i through the canonical map,
+ * and through the sequential divide/modulo program of the same run (the unoptimised form). */
+int64_t smartmem_map_eval(const smartmem_index_map_t* map, int64_t consumer_linear_index);
+int64_t smartmem_plan_eval_sequential(const smartmem_plan_t* plan, int32_t step, int32_t operand,
+                                      int64_t consumer_linear_index);
+
+/* Enqueues the plan's kernels.  inputs[i] matches the planner's inputs[i]; outputs[0] receives
+ * the result (contiguous, bf16 or f32 as the input dtype).  `cuda_stream` is a cudaStream_t. */
+int smartmem_run_chain(const smartmem_plan_t* plan, const void* const* inputs, void* const* outputs,
+                       void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* One Swin block.  x, y: [B,H,W,C]; y = x + proj(window_attention(LN1(x))) and, when
+ * mlp_ratio > 0, then y += fc2(GELU(fc1(LN2(y)))).  rel_bias_table is [(2*window-1)^2, heads].
+ * Requirements: window divides H and W; 0 <= shift < window; C = heads * head_dim with
+ * head_dim in {16, 32}; window*window <= 64; x and y must not alias.
+ * dtype F32 runs plain-FMA kernels (a 10-bit-mantissa tensor-core path cannot meet 1e-4);
+ * dtype BF16 runs the tensor-core kernels with fp32 accumulation, statistics and softmax. */
+typedef struct {
+  int32_t dtype, B, H, W, C, heads, window, shift, mlp_ratio;
+  float ln_eps;
+  const void *ln1_g, *ln1_b, *w_qkv, *b_qkv, *rel_bias_table, *w_proj, *b_proj;
+  const void *ln2_g, *ln2_b, *w_fc1, *b_fc1, *w_fc2, *b_fc2;
+} smartmem_swin_params_t;
+int smartmem_swin_block_workspace_bytes(const smartmem_swin_params_t* p, int32_t mode, size_t* bytes);
+int smartmem_swin_block(const smartmem_swin_params_t* p, const void* x, void* y, void* workspace,
+                        size_t workspace_bytes, int32_t mode, void* cuda_stream);
+
+/* One decoder attention layer, prefill.  x, y: [B,S,hidden], bf16.  w_qkv is [3*hidden, hidden]
+ * with output columns ordered (q|k|v, head, head_dim); RoPE pairs (i, i + head_dim/2). */
+typedef struct {
+  int32_t dtype, B, S, hidden, heads, head_dim, causal, add_residual;
+  float rms_eps, rope_theta;
+  const void *rms_g, *w_qkv, *w_o;
+} smartmem_attn_params_t;
+int smartmem_attn_layer_workspace_bytes(const smartmem_attn_params_t* p, int32_t mode, size_t* bytes);
+int smartmem_attn_layer(const smartmem_attn_params_t* p, const void* x, void* y, void* workspace,
+                        size_t workspace_bytes, int32_t mode, void* cuda_stream);
+
+/* Synchronises the stream and returns the device status word (SMARTMEM_OK, _TIMEOUT or _BOUNDS)
+ * in *status, then clears it. */
+int smartmem_last_device_status(void* cuda_stream, int32_t* status);
+/* Number of kernels this library has launched since it was loaded (for benchmark accounting). */
+int64_t smartmem_launch_count(void);
+const char* smartmem_status_string(int32_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SMARTMEM_H_ */

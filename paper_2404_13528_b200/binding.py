@@ -1,0 +1,245 @@
+"""ctypes binding of the C ABI in include/smartmem.h.
+
+Argument marshalling only: every step of the hot path runs inside the CUDA library.  The
+functions keep the C names.  Device buffers are passed as integers (``tensor.data_ptr()``),
+streams as ``torch.cuda.current_stream().cuda_stream``.  If the shared library is missing
+the import of any entry point raises -- there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsmartmem.so")
+
+MAX_DIMS, MAX_ATOMS, MAX_ROLLS = 8, 16, 4
+OK = 0
+ERR_INVALID_ARG, ERR_SHAPE, ERR_UNSUPPORTED, ERR_WORKSPACE = -1, -2, -3, -4
+ERR_ALIGNMENT, ERR_CUDA, ERR_TIMEOUT, ERR_BOUNDS = -5, -6, -7, -8
+F32, BF16 = 0, 1
+ELIMINATE, EXPLICIT = 0, 1
+OP_RESHAPE, OP_TRANSPOSE, OP_ROLL, OP_SLICE, OP_WINDOW_PARTITION, OP_WINDOW_REVERSE = 0, 1, 2, 3, 4, 5
+OP_COPY, OP_LINEAR, OP_BMM_NT = 16, 17, 18
+
+
+class Op(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("ndim", C.c_int32), ("shape", C.c_int64 * MAX_DIMS),
+                ("perm", C.c_int32 * MAX_DIMS), ("start", C.c_int64 * MAX_DIMS), ("shift", C.c_int64),
+                ("axis", C.c_int32), ("window", C.c_int32), ("side_input", C.c_int32 * 2)]
+
+
+class TensorDesc(C.Structure):
+    _fields_ = [("dtype", C.c_int32), ("ndim", C.c_int32), ("shape", C.c_int64 * MAX_DIMS),
+                ("stride", C.c_int64 * MAX_DIMS)]
+
+
+class IndexMap(C.Structure):
+    _fields_ = [("n_atoms", C.c_int32), ("extent", C.c_int64 * MAX_ATOMS), ("src_stride", C.c_int64 * MAX_ATOMS),
+                ("roll_of", C.c_int32 * MAX_ATOMS), ("roll_weight", C.c_int64 * MAX_ATOMS), ("n_rolls", C.c_int32),
+                ("roll_shift", C.c_int64 * MAX_ROLLS), ("roll_mod", C.c_int64 * MAX_ROLLS),
+                ("roll_stride", C.c_int64 * MAX_ROLLS), ("base", C.c_int64), ("n_elements", C.c_int64),
+                ("vec_elems", C.c_int32), ("klass", C.c_int32)]
+
+
+class SwinParams(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("dtype", "B", "H", "W", "C", "heads", "window", "shift", "mlp_ratio")] + \
+               [("ln_eps", C.c_float)] + \
+               [(n, C.c_void_p) for n in ("ln1_g", "ln1_b", "w_qkv", "b_qkv", "rel_bias_table", "w_proj", "b_proj",
+                                          "ln2_g", "ln2_b", "w_fc1", "b_fc1", "w_fc2", "b_fc2")]
+
+
+class AttnParams(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("dtype", "B", "S", "hidden", "heads", "head_dim", "causal", "add_residual")] + \
+               [("rms_eps", C.c_float), ("rope_theta", C.c_float)] + \
+               [(n, C.c_void_p) for n in ("rms_g", "w_qkv", "w_o")]
+
+
+EXPORTED = [
+    "smartmem_op_quadrant", "smartmem_pair_decision", "smartmem_plan", "smartmem_plan_destroy",
+    "smartmem_plan_num_steps", "smartmem_plan_get_map", "smartmem_plan_output_desc",
+    "smartmem_plan_workspace_bytes", "smartmem_map_eval", "smartmem_plan_eval_sequential", "smartmem_run_chain",
+    "smartmem_swin_block_workspace_bytes", "smartmem_swin_block", "smartmem_attn_layer_workspace_bytes",
+    "smartmem_attn_layer", "smartmem_last_device_status", "smartmem_launch_count", "smartmem_status_string",
+]
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Loads libsmartmem.so (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2404_13528_b200.build` "
+                           "(the hot path has no CPU fallback)")
+    L = C.CDLL(LIB_PATH)
+    P = C.POINTER
+    vp, i32, i64 = C.c_void_p, C.c_int32, C.c_int64
+    sig = {
+        "smartmem_op_quadrant": (C.c_int, [i32, P(i32)]),
+        "smartmem_pair_decision": (C.c_int, [i32, i32, P(i32), P(i32), P(i32)]),
+        "smartmem_plan": (C.c_int, [P(Op), i32, P(TensorDesc), i32, i32, P(vp)]),
+        "smartmem_plan_destroy": (C.c_int, [vp]),
+        "smartmem_plan_num_steps": (C.c_int, [vp, P(i32), P(i32)]),
+        "smartmem_plan_get_map": (C.c_int, [vp, i32, i32, P(IndexMap)]),
+        "smartmem_plan_output_desc": (C.c_int, [vp, P(TensorDesc)]),
+        "smartmem_plan_workspace_bytes": (C.c_int, [vp, P(C.c_size_t)]),
+        "smartmem_map_eval": (i64, [P(IndexMap), i64]),
+        "smartmem_plan_eval_sequential": (i64, [vp, i32, i32, i64]),
+        "smartmem_run_chain": (C.c_int, [vp, P(vp), P(vp), vp, C.c_size_t, vp]),
+        "smartmem_swin_block_workspace_bytes": (C.c_int, [P(SwinParams), i32, P(C.c_size_t)]),
+        "smartmem_swin_block": (C.c_int, [P(SwinParams), vp, vp, vp, C.c_size_t, i32, vp]),
+        "smartmem_attn_layer_workspace_bytes": (C.c_int, [P(AttnParams), i32, P(C.c_size_t)]),
+        "smartmem_attn_layer": (C.c_int, [P(AttnParams), vp, vp, vp, C.c_size_t, i32, vp]),
+        "smartmem_last_device_status": (C.c_int, [vp, P(i32)]),
+        "smartmem_launch_count": (i64, []),
+        "smartmem_status_string": (C.c_char_p, [i32]),
+    }
+    for name, (res, args) in sig.items():
+        f = getattr(L, name)
+        f.restype, f.argtypes = res, args
+    _lib = L
+    return L
+
+
+class SmartmemError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {smartmem_status_string(code)} ({code})")
+
+
+def _check(rc: int, where: str):
+    if rc != OK:
+        raise SmartmemError(rc, where)
+
+
+# ---------------------------------------------------------------------------------------------
+# helpers to build the C structures
+# ---------------------------------------------------------------------------------------------
+def make_op(kind: int, *, shape=(), perm=(), start=(), shift=0, axis=0, window=0, side_input=(0, 0)) -> Op:
+    o = Op()
+    o.kind = kind
+    o.ndim = max(len(shape), len(perm), len(start))
+    for i, v in enumerate(shape):
+        o.shape[i] = int(v)
+    for i, v in enumerate(perm):
+        o.perm[i] = int(v)
+    for i, v in enumerate(start):
+        o.start[i] = int(v)
+    o.shift, o.axis, o.window = int(shift), int(axis), int(window)
+    o.side_input[0], o.side_input[1] = int(side_input[0]), int(side_input[1])
+    return o
+
+
+def make_desc(shape, dtype: int = BF16, stride=None) -> TensorDesc:
+    d = TensorDesc()
+    d.dtype, d.ndim = dtype, len(shape)
+    for i, v in enumerate(shape):
+        d.shape[i] = int(v)
+    if stride is not None:
+        for i, v in enumerate(stride):
+            d.stride[i] = int(v)
+    return d
+
+
+# ---------------------------------------------------------------------------------------------
+# entry points (same names as the C ABI)
+# ---------------------------------------------------------------------------------------------
+def smartmem_status_string(code: int) -> str:
+    return lib().smartmem_status_string(code).decode()
+
+
+def smartmem_op_quadrant(kind: int) -> int:
+    q = C.c_int32()
+    _check(lib().smartmem_op_quadrant(kind, C.byref(q)), "smartmem_op_quadrant")
+    return q.value
+
+
+def smartmem_pair_decision(first: int, second: int):
+    a, r, s = C.c_int32(), C.c_int32(), C.c_int32()
+    _check(lib().smartmem_pair_decision(first, second, C.byref(a), C.byref(r), C.byref(s)), "smartmem_pair_decision")
+    return a.value, r.value, s.value
+
+
+def smartmem_plan(ops, inputs, mode: int) -> int:
+    """ops: list of Op; inputs: list of TensorDesc.  Returns an opaque plan handle."""
+    arr_o = (Op * len(ops))(*ops)
+    arr_i = (TensorDesc * len(inputs))(*inputs)
+    h = C.c_void_p()
+    _check(lib().smartmem_plan(arr_o, len(ops), arr_i, len(inputs), mode, C.byref(h)), "smartmem_plan")
+    return h.value
+
+
+def smartmem_plan_destroy(plan: int):
+    _check(lib().smartmem_plan_destroy(plan), "smartmem_plan_destroy")
+
+
+def smartmem_plan_num_steps(plan: int):
+    a, b = C.c_int32(), C.c_int32()
+    _check(lib().smartmem_plan_num_steps(plan, C.byref(a), C.byref(b)), "smartmem_plan_num_steps")
+    return a.value, b.value
+
+
+def smartmem_plan_get_map(plan: int, step: int, operand: int = 0) -> IndexMap:
+    m = IndexMap()
+    _check(lib().smartmem_plan_get_map(plan, step, operand, C.byref(m)), "smartmem_plan_get_map")
+    return m
+
+
+def smartmem_plan_output_desc(plan: int) -> TensorDesc:
+    d = TensorDesc()
+    _check(lib().smartmem_plan_output_desc(plan, C.byref(d)), "smartmem_plan_output_desc")
+    return d
+
+
+def smartmem_plan_workspace_bytes(plan: int) -> int:
+    n = C.c_size_t()
+    _check(lib().smartmem_plan_workspace_bytes(plan, C.byref(n)), "smartmem_plan_workspace_bytes")
+    return n.value
+
+
+def smartmem_map_eval(m: IndexMap, i: int) -> int:
+    return lib().smartmem_map_eval(C.byref(m), i)
+
+
+def smartmem_plan_eval_sequential(plan: int, step: int, operand: int, i: int) -> int:
+    return lib().smartmem_plan_eval_sequential(plan, step, operand, i)
+
+
+def smartmem_run_chain(plan: int, inputs, outputs, workspace: int, workspace_bytes: int, stream: int):
+    """inputs / outputs: lists of device pointers (ints)."""
+    ai = (C.c_void_p * len(inputs))(*inputs)
+    ao = (C.c_void_p * len(outputs))(*outputs)
+    _check(lib().smartmem_run_chain(plan, ai, ao, workspace, workspace_bytes, stream), "smartmem_run_chain")
+
+
+def smartmem_swin_block_workspace_bytes(p: SwinParams, mode: int) -> int:
+    n = C.c_size_t()
+    _check(lib().smartmem_swin_block_workspace_bytes(C.byref(p), mode, C.byref(n)), "smartmem_swin_block_workspace_bytes")
+    return n.value
+
+
+def smartmem_swin_block(p: SwinParams, x: int, y: int, workspace: int, workspace_bytes: int, mode: int, stream: int):
+    _check(lib().smartmem_swin_block(C.byref(p), x, y, workspace, workspace_bytes, mode, stream), "smartmem_swin_block")
+
+
+def smartmem_attn_layer_workspace_bytes(p: AttnParams, mode: int) -> int:
+    n = C.c_size_t()
+    _check(lib().smartmem_attn_layer_workspace_bytes(C.byref(p), mode, C.byref(n)), "smartmem_attn_layer_workspace_bytes")
+    return n.value
+
+
+def smartmem_attn_layer(p: AttnParams, x: int, y: int, workspace: int, workspace_bytes: int, mode: int, stream: int):
+    _check(lib().smartmem_attn_layer(C.byref(p), x, y, workspace, workspace_bytes, mode, stream), "smartmem_attn_layer")
+
+
+def smartmem_last_device_status(stream: int) -> int:
+    s = C.c_int32()
+    _check(lib().smartmem_last_device_status(stream, C.byref(s)), "smartmem_last_device_status")
+    return s.value
+
+
+def smartmem_launch_count() -> int:
+    return lib().smartmem_launch_count()

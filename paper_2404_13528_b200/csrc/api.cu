@@ -1,0 +1,117 @@
+// C-ABI entry points (see include/smartmem.h).
+#include <atomic>
+#include <mutex>
+#include <vector>
+
+#include "common.cuh"
+#include "gemm_tc.cuh"
+#include "plan.hpp"
+
+#define EXPORT extern "C" __attribute__((visibility("default")))
+
+namespace smartmem {
+
+static std::atomic<long long> g_launches{0};
+void count_launch(int n) { g_launches += n; }
+
+__device__ int g_status_word;
+
+int* device_status_ptr() {
+  static int* p = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* q = nullptr;
+    if (cudaGetSymbolAddress(&q, g_status_word) == cudaSuccess) {
+      p = (int*)q;
+      cudaMemset(p, 0, sizeof(int));
+    }
+  });
+  return p;
+}
+
+}  // namespace smartmem
+
+using namespace smartmem;
+
+EXPORT int64_t smartmem_launch_count(void) { return g_launches.load(); }
+
+EXPORT int smartmem_last_device_status(void* cuda_stream, int32_t* status) {
+  if (!status) return SMARTMEM_ERR_INVALID_ARG;
+  int* p = device_status_ptr();
+  if (!p) return SMARTMEM_ERR_CUDA;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  int v = 0;
+  if (cudaMemcpyAsync(&v, p, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return SMARTMEM_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return SMARTMEM_ERR_CUDA;
+  if (v != 0) cudaMemsetAsync(p, 0, sizeof(int), st);
+  *status = v;
+  return SMARTMEM_OK;
+}
+
+namespace {
+
+bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
+
+}  // namespace
+
+EXPORT int smartmem_run_chain(const smartmem_plan_t* plan, const void* const* inputs, void* const* outputs,
+                              void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!plan || !inputs || !outputs || !outputs[0]) return SMARTMEM_ERR_INVALID_ARG;
+  for (int i = 0; i < plan->n_inputs; ++i) {
+    if (!inputs[i]) return SMARTMEM_ERR_INVALID_ARG;
+    if (!aligned16(inputs[i])) return SMARTMEM_ERR_ALIGNMENT;
+  }
+  if (!aligned16(outputs[0]) || !aligned16(workspace)) return SMARTMEM_ERR_ALIGNMENT;
+  if (plan->workspace_bytes > workspace_bytes || (plan->workspace_bytes && !workspace)) return SMARTMEM_ERR_WORKSPACE;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) return SMARTMEM_ERR_CUDA;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  auto buf = [&](int ref) -> void* {
+    if (ref >= 0) return const_cast<void*>(inputs[ref]);
+    if (ref == -1) return outputs[0];
+    return (char*)workspace + plan->slot_offset[-2 - ref];
+  };
+  for (const Step& s : plan->steps) {
+    const int esz = s.dtype == SMARTMEM_F32 ? 4 : 2;
+    int rc = SMARTMEM_OK;
+    if (s.kind == STEP_COPY) {
+      rc = launch_copy_map(s.map[0], esz, buf(s.src[0]), buf(s.dst), st);
+    } else if (s.kind == STEP_LINEAR || s.kind == STEP_BMM_NT) {
+      if (s.dtype != SMARTMEM_BF16) return SMARTMEM_ERR_UNSUPPORTED;
+      TcOperand A, B;
+      rc = tc_operand_from_map(s.map[0], s.n_batch_atoms[0], s.n_row_atoms[0], buf(s.src[0]), &A);
+      if (rc != SMARTMEM_OK) return rc;
+      if (s.kind == STEP_LINEAR) {
+        B = tc_operand_plain(inputs[s.weight], s.N, s.K, s.K);
+      } else {
+        rc = tc_operand_from_map(s.map[1], s.n_batch_atoms[1], s.n_row_atoms[1], buf(s.src[1]), &B);
+        if (rc != SMARTMEM_OK) return rc;
+      }
+      TcEpilogue ep;
+      memset(&ep, 0, sizeof(ep));
+      ep.out = buf(s.dst);
+      ep.ldc = s.N;
+      ep.out_batch_stride = s.M * s.N;
+      rc = launch_gemm_tc(A, B, ep, s.batch, s.M, s.N, s.K, st);
+    } else {
+      rc = SMARTMEM_ERR_UNSUPPORTED;
+    }
+    if (rc != SMARTMEM_OK) return rc;
+  }
+  return SMARTMEM_OK;
+}
+
+EXPORT int smartmem_attn_layer_workspace_bytes(const smartmem_attn_params_t* p, int32_t mode, size_t* bytes) {
+  return SMARTMEM_ERR_UNSUPPORTED;
+}
+EXPORT int smartmem_attn_layer(const smartmem_attn_params_t* p, const void* x, void* y, void* workspace,
+                               size_t workspace_bytes, int32_t mode, void* cuda_stream) {
+  return SMARTMEM_ERR_UNSUPPORTED;
+}
+EXPORT int smartmem_swin_block_workspace_bytes(const smartmem_swin_params_t* p, int32_t mode, size_t* bytes) {
+  return SMARTMEM_ERR_UNSUPPORTED;
+}
+EXPORT int smartmem_swin_block(const smartmem_swin_params_t* p, const void* x, void* y, void* workspace,
+                               size_t workspace_bytes, int32_t mode, void* cuda_stream) {
+  return SMARTMEM_ERR_UNSUPPORTED;
+}

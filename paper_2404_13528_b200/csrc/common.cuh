@@ -1,0 +1,145 @@
+// Shared device/host helpers of the CUDA path.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "smartmem.h"
+
+namespace smartmem {
+
+// ---------------------------------------------------------------------------------------
+// Device status word (bounded waits / debug bounds) and launch accounting.
+// ---------------------------------------------------------------------------------------
+int* device_status_ptr();                 // device address of the status word (per process)
+void count_launch(int n = 1);
+
+// ---------------------------------------------------------------------------------------
+// Division by a run-time constant without a divide instruction: q = umulhi(n, mul) >> shr
+// for 0 <= n < 2^31 (round-up reciprocal).  Extents are plan-time constants, so the
+// reciprocals are computed once on the host.
+// ---------------------------------------------------------------------------------------
+struct FastDiv {
+  uint32_t d, mul, shr;
+};
+
+inline FastDiv make_fastdiv(uint32_t d) {
+  FastDiv f{d, 0u, 0u};
+  if (d > 1) {
+    uint32_t l = 0;
+    while ((1ull << l) < d) ++l;        // ceil(log2 d)
+    uint32_t p = 31 + l;
+    f.mul = (uint32_t)(((1ull << p) + d - 1) / d);
+    f.shr = p - 32;
+  }
+  return f;
+}
+
+__device__ __forceinline__ uint32_t fd_div(uint32_t n, const FastDiv& f) {
+  return f.d == 1 ? n : (__umulhi(n, f.mul) >> f.shr);
+}
+
+// ---------------------------------------------------------------------------------------
+// Device form of a canonical index map (see smartmem_index_map_t).  `unit` elements of the
+// innermost atom are handled as one vector, so extent[n-1] is in vectors and offsets are
+// returned in elements.
+// ---------------------------------------------------------------------------------------
+constexpr int kMaxDevAtoms = 10;
+struct DevMap {
+  int n_atoms, n_rolls;
+  FastDiv ext[kMaxDevAtoms];
+  long long stride[kMaxDevAtoms];       // elements; for the (vectorised) innermost atom: unit
+  int roll_of[kMaxDevAtoms];
+  int weight[kMaxDevAtoms];
+  int roll_shift[SMARTMEM_MAX_ROLLS], roll_mod[SMARTMEM_MAX_ROLLS];
+  long long roll_stride[SMARTMEM_MAX_ROLLS];
+  long long base;
+};
+
+// Source offset (elements) of consumer unit `i`.
+__device__ __forceinline__ long long devmap_eval(const DevMap& m, uint32_t i) {
+  long long off = m.base;
+  int u[SMARTMEM_MAX_ROLLS] = {0, 0, 0, 0};
+#pragma unroll 1
+  for (int a = m.n_atoms - 1; a >= 0; --a) {
+    uint32_t q = fd_div(i, m.ext[a]);
+    uint32_t digit = i - q * m.ext[a].d;
+    i = q;
+    int r = m.roll_of[a];
+    if (r < 0) off += (long long)digit * m.stride[a];
+    else u[r] += (int)digit * m.weight[a];
+  }
+#pragma unroll
+  for (int r = 0; r < SMARTMEM_MAX_ROLLS; ++r)
+    if (r < m.n_rolls) {
+      int v = u[r] + m.roll_shift[r];
+      if (v >= m.roll_mod[r]) v -= m.roll_mod[r];     // u < mod and shift < mod: one conditional subtract
+      off += (long long)v * m.roll_stride[r];
+    }
+  return off;
+}
+
+// Host: builds a DevMap over atoms [a0, a1) of a public map, treating `unit` elements of the
+// innermost selected atom as one unit (unit must divide its extent; its stride must be 1 when
+// unit > 1).  `with_base` adds the map's base.  Returns false if it does not fit.
+bool make_devmap(const smartmem_index_map_t& m, int a0, int a1, int unit, bool with_base, DevMap* out);
+
+// ---------------------------------------------------------------------------------------
+// Small numeric helpers.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ float bf16_bits_to_float(uint16_t b) { return __uint_as_float((uint32_t)b << 16); }
+__device__ __forceinline__ float2 bf16x2_to_float2(uint32_t w) {
+  return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u));
+}
+__device__ __forceinline__ uint32_t float2_to_bf16x2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ float gelu_erf(float u) { return 0.5f * u * (1.0f + erff(u * 0.70710678118654752f)); }
+
+template <typename T> struct ElemIO;
+template <> struct ElemIO<float> {
+  static constexpr int kVec = 4;          // elements per 16 bytes
+  __device__ static void load(const float* p, float* v) {
+    float4 t = *reinterpret_cast<const float4*>(p);
+    v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+  }
+  __device__ static void store(float* p, const float* v) {
+    *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
+  }
+  __device__ static float ld1(const float* p) { return *p; }
+  __device__ static void st1(float* p, float v) { *p = v; }
+};
+template <> struct ElemIO<__nv_bfloat16> {
+  static constexpr int kVec = 8;
+  __device__ static void load(const __nv_bfloat16* p, float* v) {
+    uint4 t = *reinterpret_cast<const uint4*>(p);
+    float2 a = bf16x2_to_float2(t.x), b = bf16x2_to_float2(t.y), c = bf16x2_to_float2(t.z), d = bf16x2_to_float2(t.w);
+    v[0] = a.x; v[1] = a.y; v[2] = b.x; v[3] = b.y; v[4] = c.x; v[5] = c.y; v[6] = d.x; v[7] = d.y;
+  }
+  __device__ static void store(__nv_bfloat16* p, const float* v) {
+    uint4 t;
+    t.x = float2_to_bf16x2(v[0], v[1]); t.y = float2_to_bf16x2(v[2], v[3]);
+    t.z = float2_to_bf16x2(v[4], v[5]); t.w = float2_to_bf16x2(v[6], v[7]);
+    *reinterpret_cast<uint4*>(p) = t;
+  }
+  __device__ static float ld1(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+  __device__ static void st1(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
+};
+
+// ---------------------------------------------------------------------------------------
+// Launchers (defined in the .cu files).  All return a smartmem_status_t.
+// ---------------------------------------------------------------------------------------
+// Map-driven copy: out (contiguous) <- src through `map`.
+int launch_copy_map(const smartmem_index_map_t& map, int elem_size, const void* src, void* dst, cudaStream_t st);
+
+// LayerNorm / RMSNorm over rows of length C.  Row r of the output (row-major [rows, C]) is
+// read from src at element offset rowmap(r) (rowmap == nullptr: r * C).
+int launch_norm(int dtype, bool rms, const void* src, void* dst, const void* gamma, const void* beta, float eps,
+                long long rows, int C, const DevMap* rowmap, cudaStream_t st);
+
+// Elementwise helpers of the EXPLICIT path.
+int launch_rope_inplace(void* qk, long long rows, int row_stride, int heads2, int head_dim, float theta, int S,
+                        cudaStream_t st);
+
+}  // namespace smartmem

@@ -1,0 +1,177 @@
+// Map-driven copy kernels: the consumer is the identity, so the kernel is exactly the
+// composed index map of an eliminated layout run (Section 3.2.1) applied on the load side.
+// They serve the copy-only chains and every materialised layout operator of EXPLICIT mode.
+#include <vector>
+
+#include "common.cuh"
+
+namespace smartmem {
+
+bool make_devmap(const smartmem_index_map_t& m, int a0, int a1, int unit, bool with_base, DevMap* out) {
+  if (a1 - a0 > kMaxDevAtoms || a0 < 0 || a1 > m.n_atoms) return false;
+  DevMap d;
+  memset(&d, 0, sizeof(d));
+  d.n_atoms = a1 - a0;
+  d.n_rolls = m.n_rolls;
+  d.base = with_base ? m.base : 0;
+  for (int r = 0; r < m.n_rolls; ++r) {
+    if (m.roll_mod[r] >= (1ll << 30)) return false;
+    d.roll_shift[r] = (int)m.roll_shift[r];
+    d.roll_mod[r] = (int)m.roll_mod[r];
+    d.roll_stride[r] = m.roll_stride[r];
+  }
+  for (int a = a0; a < a1; ++a) {
+    int64_t e = m.extent[a];
+    long long s = m.src_stride[a];
+    if (a == a1 - 1 && unit > 1) {
+      if (m.roll_of[a] >= 0 || s != 1 || e % unit) return false;
+      e /= unit;
+      s = unit;
+    }
+    if (e >= (1ll << 31) || m.roll_weight[a] >= (1ll << 30)) return false;
+    d.ext[a - a0] = make_fastdiv((uint32_t)e);
+    d.stride[a - a0] = s;
+    d.roll_of[a - a0] = m.roll_of[a];
+    d.weight[a - a0] = (int)m.roll_weight[a];
+  }
+  *out = d;
+  return true;
+}
+
+namespace {
+
+template <int VB> struct VecT;
+template <> struct VecT<16> { using type = uint4; };
+template <> struct VecT<8> { using type = uint2; };
+template <> struct VecT<4> { using type = uint32_t; };
+template <> struct VecT<2> { using type = uint16_t; };
+
+// One thread per output vector of VB bytes: decompose the vector index over the atoms,
+// load through the map, store contiguously (coalesced).
+template <int VB>
+__global__ void __launch_bounds__(256) copy_gather_kernel(const __grid_constant__ DevMap map, const char* __restrict__ src,
+                                                          char* __restrict__ dst, uint32_t n_units, int elem_size) {
+  using V = typename VecT<VB>::type;
+  uint32_t i = blockIdx.x * 256u + threadIdx.x;
+  if (i >= n_units) return;
+  long long off = devmap_eval(map, i);
+  V v = *reinterpret_cast<const V*>(src + off * elem_size);
+  *reinterpret_cast<V*>(dst + (size_t)i * VB) = v;
+}
+
+// Affine map whose consumer-innermost atom I is strided in the source while another atom J is
+// source-contiguous: a 64 x 64 tile transpose of 2-byte elements through shared memory.  Loads are
+// 16-byte vectors along J, stores 16-byte vectors along I.
+struct TransposeArgs {
+  int n_outer;
+  FastDiv outer_ext[kMaxDevAtoms];
+  long long outer_src[kMaxDevAtoms], outer_dst[kMaxDevAtoms];
+  long long src_stride_i, dst_stride_j, base;
+  int tiles_i, tiles_j;
+};
+
+__global__ void __launch_bounds__(256) copy_transpose16_kernel(const __grid_constant__ TransposeArgs a,
+                                                               const uint16_t* __restrict__ src, uint16_t* __restrict__ dst) {
+  __shared__ uint32_t tile[64][33];          // [j][i-pair]
+  uint32_t b = blockIdx.x;
+  uint32_t tj = b % a.tiles_j;
+  b /= a.tiles_j;
+  uint32_t ti = b % a.tiles_i;
+  b /= a.tiles_i;
+  long long so = a.base, dof = 0;
+  for (int k = a.n_outer - 1; k >= 0; --k) {
+    uint32_t q = fd_div(b, a.outer_ext[k]);
+    uint32_t digit = b - q * a.outer_ext[k].d;
+    b = q;
+    so += (long long)digit * a.outer_src[k];
+    dof += (long long)digit * a.outer_dst[k];
+  }
+  const int tid = threadIdx.x;
+  {
+    const int p = tid >> 3, jg = tid & 7;
+    const uint16_t* s0 = src + so + (long long)(ti * 64 + 2 * p) * a.src_stride_i + tj * 64 + jg * 8;
+    uint4 r0 = *reinterpret_cast<const uint4*>(s0);
+    uint4 r1 = *reinterpret_cast<const uint4*>(s0 + a.src_stride_i);
+    const uint32_t w0[4] = {r0.x, r0.y, r0.z, r0.w}, w1[4] = {r1.x, r1.y, r1.z, r1.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      tile[jg * 8 + 2 * e][p] = (w0[e] & 0xFFFFu) | (w1[e] << 16);
+      tile[jg * 8 + 2 * e + 1][p] = (w0[e] >> 16) | (w1[e] & 0xFFFF0000u);
+    }
+  }
+  __syncthreads();
+#pragma unroll
+  for (int pass = 0; pass < 2; ++pass) {
+    const int q = tid & 7, j = (tid >> 3) + 32 * pass;
+    uint4 v;
+    v.x = tile[j][4 * q + 0];
+    v.y = tile[j][4 * q + 1];
+    v.z = tile[j][4 * q + 2];
+    v.w = tile[j][4 * q + 3];
+    *reinterpret_cast<uint4*>(dst + dof + (long long)(tj * 64 + j) * a.dst_stride_j + ti * 64 + q * 8) = v;
+  }
+}
+
+}  // namespace
+
+int launch_copy_map(const smartmem_index_map_t& map, int elem_size, const void* src, void* dst, cudaStream_t st) {
+  if (map.klass == 3) return SMARTMEM_ERR_UNSUPPORTED;
+  if (map.n_elements == 0) return SMARTMEM_OK;
+  const int n = map.n_atoms;
+  // fast path: tiled transpose
+  if (map.klass == 1 && elem_size == 2 && n >= 2 && map.src_stride[n - 1] != 1) {
+    int J = -1;
+    for (int a = 0; a < n - 1; ++a)
+      if (map.src_stride[a] == 1) J = a;
+    if (J >= 0 && map.extent[n - 1] % 64 == 0 && map.extent[J] % 64 == 0 && n - 2 <= kMaxDevAtoms) {
+      TransposeArgs t;
+      memset(&t, 0, sizeof(t));
+      std::vector<long long> cstride(n);
+      long long run = 1;
+      for (int a = n - 1; a >= 0; --a) {
+        cstride[a] = run;
+        run *= map.extent[a];
+      }
+      bool ok = map.base % 8 == 0 && map.src_stride[n - 1] % 8 == 0 && cstride[J] % 8 == 0;
+      long long outer = 1;
+      for (int a = 0; a < n - 1; ++a) {
+        if (a == J) continue;
+        ok = ok && map.src_stride[a] % 8 == 0 && cstride[a] % 8 == 0 && map.extent[a] < (1ll << 31);
+        t.outer_ext[t.n_outer] = make_fastdiv((uint32_t)map.extent[a]);
+        t.outer_src[t.n_outer] = map.src_stride[a];
+        t.outer_dst[t.n_outer] = cstride[a];
+        ++t.n_outer;
+        outer *= map.extent[a];
+      }
+      t.src_stride_i = map.src_stride[n - 1];
+      t.dst_stride_j = cstride[J];
+      t.base = map.base;
+      t.tiles_i = (int)(map.extent[n - 1] / 64);
+      t.tiles_j = (int)(map.extent[J] / 64);
+      long long blocks = outer * t.tiles_i * t.tiles_j;
+      if (ok && blocks < (1ll << 31)) {
+        copy_transpose16_kernel<<<(unsigned)blocks, 256, 0, st>>>(t, (const uint16_t*)src, (uint16_t*)dst);
+        count_launch();
+        return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
+      }
+    }
+  }
+  const int v = map.vec_elems;
+  const int vb = v * elem_size;
+  DevMap d;
+  if (!make_devmap(map, 0, n, v, true, &d)) return SMARTMEM_ERR_UNSUPPORTED;
+  long long units = map.n_elements / v;
+  if (units >= (1ll << 31)) return SMARTMEM_ERR_UNSUPPORTED;
+  unsigned grid = (unsigned)((units + 255) / 256);
+  switch (vb) {
+    case 16: copy_gather_kernel<16><<<grid, 256, 0, st>>>(d, (const char*)src, (char*)dst, (uint32_t)units, elem_size); break;
+    case 8: copy_gather_kernel<8><<<grid, 256, 0, st>>>(d, (const char*)src, (char*)dst, (uint32_t)units, elem_size); break;
+    case 4: copy_gather_kernel<4><<<grid, 256, 0, st>>>(d, (const char*)src, (char*)dst, (uint32_t)units, elem_size); break;
+    case 2: copy_gather_kernel<2><<<grid, 256, 0, st>>>(d, (const char*)src, (char*)dst, (uint32_t)units, elem_size); break;
+    default: return SMARTMEM_ERR_UNSUPPORTED;
+  }
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
+}
+
+}  // namespace smartmem

@@ -1,0 +1,471 @@
+// bf16 GEMM on the 5th-generation tensor cores (tcgen05), fp32 accumulation in TMEM.
+//
+//   out[b, m, n] = epilogue( sum_k A[b, m, k] * B[b, n, k] )
+//
+// Both operands are read "reduction dimension contiguous" (Section 3.2.2) straight from the
+// producer's buffer: the composed index map of an eliminated layout run is affine here, so it
+// becomes a TMA tensor map (up to 5-D box) and costs nothing at run time.  An operand whose
+// rows -- not its reduction dimension -- are contiguous in the producer's buffer (the NCHW ->
+// NHWC case) is loaded as it lies and multiplied through the MN-major operand mode of the
+// tensor core, so that transpose disappears as well.
+//
+// CTA = 6 warps: warp 0 issues TMA loads into a STAGES-deep shared-memory ring, warp 1 owns the
+// TMEM allocation and issues tcgen05.mma (one thread), warps 2-5 run the epilogue
+// (TMEM -> registers -> bias / GELU / RoPE / residual -> bf16 -> global, optionally scattering
+// rows through an index map: window reverse + reverse cyclic shift folded into the store).
+#include <mutex>
+#include <unordered_map>
+#include <string>
+#include <vector>
+
+#include "gemm_tc.cuh"
+#include "ptx.cuh"
+
+namespace smartmem {
+namespace {
+
+constexpr int BM = 128;
+constexpr int BK = 64;                   // 64 bf16 = 128 bytes = one swizzle row
+constexpr int A_STAGE_BYTES = BM * BK * 2;
+
+struct OpCoord {
+  int rank, mn_major;
+  FastDiv tiles_inner;
+  int n_outer;                           // outer row atoms then batch atoms, innermost first
+  int n_outer_row;
+  FastDiv outer[3];
+};
+
+struct GemmArgs {
+  int M, N, K;
+  OpCoord ca, cb;
+  __nv_bfloat16* out;
+  long long ldc, out_batch_stride;
+  const __nv_bfloat16* bias;
+  const __nv_bfloat16* residual;
+  int gelu, has_rowmap;
+  int rope_cols, rope_S;                 // columns [0, rope_cols) are rotated; position = row % rope_S
+  const float2* rope_tab;                // [rope_S, 64] (cos, sin)
+  int* status;
+  DevMap rowmap;
+};
+
+__device__ __forceinline__ void op_coords(const OpCoord& oc, uint32_t tile, uint32_t batch, int tile_rows, int k0,
+                                          int* c) {
+  uint32_t q = fd_div(tile, oc.tiles_inner);
+  int row0 = (int)(tile - q * oc.tiles_inner.d) * tile_rows;
+  c[0] = oc.mn_major ? row0 : k0;
+  c[1] = oc.mn_major ? k0 : row0;
+  int n = 2;
+  for (int i = 0; i < oc.n_outer; ++i) {
+    uint32_t& src = (i < oc.n_outer_row) ? q : batch;
+    uint32_t qq = fd_div(src, oc.outer[i]);
+    c[n++] = (int)(src - qq * oc.outer[i].d);
+    src = qq;
+  }
+}
+
+// erf by the rational approximation 7.1.26 of Abramowitz & Stegun (|error| <= 1.5e-7), far
+// below bf16 resolution; one reciprocal and one exponential instead of erff's long polynomial.
+__device__ __forceinline__ float gelu_fast(float u) {
+  const float x = fabsf(u) * 0.70710678118654752f;
+  const float t = __frcp_rn(fmaf(0.3275911f, x, 1.0f));
+  float p = fmaf(1.061405429f, t, -1.453152027f);
+  p = fmaf(p, t, 1.421413741f);
+  p = fmaf(p, t, -0.284496736f);
+  p = fmaf(p, t, 0.254829592f);
+  const float e = 1.0f - p * t * __expf(-x * x);       // erf(|u| / sqrt 2)
+  return 0.5f * u * (1.0f + copysignf(e, u));
+}
+
+template <int BN, int STAGES, bool A_MN>
+__global__ void __launch_bounds__(192, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ GemmArgs g) {
+  constexpr int B_STAGE_BYTES = BN * BK * 2;
+  constexpr uint32_t TMEM_COLS = BN <= 32 ? 32 : BN <= 64 ? 64 : BN <= 128 ? 128 : 256;
+  constexpr uint32_t IDESC = ptx::make_idesc_bf16(BM, BN, A_MN, false);
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
+  uint8_t* sA = smem;
+  uint8_t* sB = smem + STAGES * A_STAGE_BYTES;
+  uint64_t* full = reinterpret_cast<uint64_t*>(sB + STAGES * B_STAGE_BYTES);
+  uint64_t* empty = full + STAGES;
+  uint64_t* tmem_full = empty + STAGES;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_full + 1);
+  int* abort_flag = reinterpret_cast<int*>(tmem_slot + 1);
+  float* bias_s = reinterpret_cast<float*>(tmem_slot + 2);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t tile_n = blockIdx.x, tile_m = blockIdx.y, batch = blockIdx.z;
+  const int nkb = (g.K + BK - 1) / BK;
+  const int last_ksteps = (g.K - (nkb - 1) * BK + 15) / 16;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      ptx::mbar_init(&full[s], 1);
+      ptx::mbar_init(&empty[s], 1);
+    }
+    ptx::mbar_init(tmem_full, 1);
+    *abort_flag = 0;
+    ptx::fence_barrier_init();
+    ptx::fence_proxy_async();
+  }
+  if (warp == 0 && lane == 0) {
+    ptx::prefetch_tensormap(&tmA);
+    ptx::prefetch_tensormap(&tmB);
+  }
+  if (warp == 1) ptx::tmem_alloc(tmem_slot, TMEM_COLS);
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int issued = 0;
+      for (int kb = 0; kb < nkb; ++kb) {
+        const int s = kb % STAGES;
+        const uint32_t ph = (kb / STAGES) & 1;
+        if (!ptx::mbar_wait(&empty[s], ph ^ 1, abort_flag, g.status)) break;
+        ptx::mbar_expect_tx(&full[s], A_STAGE_BYTES + B_STAGE_BYTES);
+        int c[5];
+        op_coords(g.ca, tile_m, batch, BM, kb * BK, c);
+        if (A_MN) {
+          ptx::tma_load_nd(g.ca.rank, sA + s * A_STAGE_BYTES, &tmA, &full[s], c);
+          c[0] += 64;
+          ptx::tma_load_nd(g.ca.rank, sA + s * A_STAGE_BYTES + A_STAGE_BYTES / 2, &tmA, &full[s], c);
+        } else {
+          ptx::tma_load_nd(g.ca.rank, sA + s * A_STAGE_BYTES, &tmA, &full[s], c);
+        }
+        op_coords(g.cb, tile_n, batch, BN, kb * BK, c);
+        ptx::tma_load_nd(g.cb.rank, sB + s * B_STAGE_BYTES, &tmB, &full[s], c);
+        issued = kb + 1;
+      }
+      if (*abort_flag) {
+        // unwinding: give copies already in flight a bounded chance to land before the CTA leaves
+        for (int kb = (issued > STAGES ? issued - STAGES : 0); kb < issued; ++kb) {
+          const unsigned long long t0 = ptx::globaltimer();
+          while (!ptx::mbar_try_wait(&full[kb % STAGES], (kb / STAGES) & 1) && ptx::globaltimer() - t0 < 2000000ull) {
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      bool ok = true;
+      for (int kb = 0; kb < nkb && ok; ++kb) {
+        const int s = kb % STAGES;
+        const uint32_t ph = (kb / STAGES) & 1;
+        ok = ptx::mbar_wait(&full[s], ph, abort_flag, g.status);
+        if (!ok) break;
+        ptx::tc_fence_after();
+        const uint32_t a0 = ptx::smem_u32(sA + s * A_STAGE_BYTES), b0 = ptx::smem_u32(sB + s * B_STAGE_BYTES);
+        const int ks = (kb == nkb - 1) ? last_ksteps : BK / 16;
+        for (int k = 0; k < ks; ++k) {
+          // K-major, 128-byte swizzle: 8-row groups are 1024 bytes apart; one k16 step is 32 bytes
+          // along the swizzled row.  MN-major: 64-row chunks are 8192 bytes apart (leading offset),
+          // 8-deep k groups 1024 bytes apart, one k16 step is 2048 bytes.
+          const uint64_t ad = A_MN ? ptx::make_smem_desc(a0 + k * 2048, A_STAGE_BYTES / 2, 1024)
+                                   : ptx::make_smem_desc(a0 + k * 32, 16, 1024);
+          const uint64_t bd = ptx::make_smem_desc(b0 + k * 32, 16, 1024);
+          ptx::tc_mma_bf16(tmem_base, ad, bd, IDESC, (kb | k) ? 1u : 0u);
+        }
+        ptx::tc_commit(&empty[s]);
+      }
+      if (ok) ptx::tc_commit(tmem_full);
+    }
+  } else {
+    const int et = threadIdx.x - 64;                     // 0..127
+    const int n0 = tile_n * BN;
+    for (int c = et; c < BN; c += 128)
+      bias_s[c] = (g.bias && n0 + c < g.N) ? __bfloat162float(g.bias[n0 + c]) : 0.f;
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    const bool ok = ptx::mbar_wait(tmem_full, 0, abort_flag, g.status);
+    ptx::tc_fence_after();
+    const int q = warp & 3;
+    const int row = tile_m * BM + q * 32 + lane;
+    if (ok) {
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+      const bool row_ok = row < g.M;
+      long long off = 0;
+      if (row_ok) off = g.has_rowmap ? devmap_eval(g.rowmap, (uint32_t)row) : (long long)row * g.ldc;
+      off += (long long)batch * g.out_batch_stride;
+      __nv_bfloat16* orow = g.out + off;
+      const __nv_bfloat16* rrow = g.residual ? g.residual + off : nullptr;
+
+      auto finish = [&](float* acc, int c0) {            // bias / GELU / residual / store of 32 columns
+        const int col0 = n0 + c0;
+        if (!row_ok || col0 >= g.N) return;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) acc[j] += bias_s[c0 + j];
+        if (g.gelu) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) acc[j] = gelu_fast(acc[j]);
+        }
+        if (col0 + 32 <= g.N) {
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            if (rrow) {
+              float r[8];
+              ElemIO<__nv_bfloat16>::load(rrow + col0 + v * 8, r);
+#pragma unroll
+              for (int e = 0; e < 8; ++e) acc[v * 8 + e] += r[e];
+            }
+            ElemIO<__nv_bfloat16>::store(orow + col0 + v * 8, acc + v * 8);
+          }
+        } else {
+          for (int j = 0; j < 32 && col0 + j < g.N; ++j) {
+            float r = rrow ? __bfloat162float(rrow[col0 + j]) : 0.f;
+            orow[col0 + j] = __float2bfloat16_rn(acc[j] + r);
+          }
+        }
+      };
+
+      for (int ch = 0; ch < BN / 32; ++ch) {
+        const int c0 = ch * 32;
+        const bool rope = g.rope_cols > 0 && n0 + c0 < g.rope_cols;
+        if (rope) {
+          if ((ch & 3) >= 2) continue;                   // done together with chunk ch - 2
+          uint32_t ra[32], rb[32];
+          ptx::tmem_ld32(taddr + c0, ra);
+          ptx::tmem_ld32(taddr + c0 + 64, rb);
+          ptx::tmem_ld_wait();
+          float x1[32], x2[32];
+          const float2* tab = g.rope_tab + (long long)(row_ok ? row % g.rope_S : 0) * 64 + (ch & 1) * 32;
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const float2 cs = tab[j];
+            const float a = __uint_as_float(ra[j]), b = __uint_as_float(rb[j]);
+            x1[j] = a * cs.x - b * cs.y;
+            x2[j] = b * cs.x + a * cs.y;
+          }
+          finish(x1, c0);
+          finish(x2, c0 + 64);
+        } else {
+          uint32_t r[32];
+          ptx::tmem_ld32(taddr + c0, r);
+          ptx::tmem_ld_wait();
+          float acc[32];
+#pragma unroll
+          for (int j = 0; j < 32; ++j) acc[j] = __uint_as_float(r[j]);
+          finish(acc, c0);
+        }
+      }
+    }
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Host side: tensor maps.
+// ---------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  });
+  return fn;
+}
+
+std::mutex g_tm_mu;
+std::unordered_map<std::string, CUtensorMap> g_tm_cache;
+
+int encode_cached(const void* ptr, int rank, const uint64_t* dims, const uint64_t* strides_b, const uint32_t* box,
+                  CUtensorMap* out) {
+  std::string key((const char*)&ptr, sizeof(ptr));
+  key.append((const char*)&rank, sizeof(rank));
+  key.append((const char*)dims, sizeof(uint64_t) * rank);
+  key.append((const char*)strides_b, sizeof(uint64_t) * (rank - 1));
+  key.append((const char*)box, sizeof(uint32_t) * rank);
+  {
+    std::lock_guard<std::mutex> lk(g_tm_mu);
+    auto it = g_tm_cache.find(key);
+    if (it != g_tm_cache.end()) {
+      *out = it->second;
+      return SMARTMEM_OK;
+    }
+  }
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return SMARTMEM_ERR_CUDA;
+  cuuint64_t d[5], s[4];
+  cuuint32_t b[5], es[5];
+  for (int i = 0; i < rank; ++i) {
+    d[i] = dims[i];
+    b[i] = box[i];
+    es[i] = 1;
+    if (i < rank - 1) s[i] = strides_b[i];
+  }
+  CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(ptr), d, s, b, es,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return SMARTMEM_ERR_CUDA;
+  std::lock_guard<std::mutex> lk(g_tm_mu);
+  if (g_tm_cache.size() > 4096) g_tm_cache.clear();
+  g_tm_cache[key] = *out;
+  return SMARTMEM_OK;
+}
+
+// Turns an operand description into a tensor map + the coordinate rule of the kernel.
+int build_operand(const TcOperand& op, int tile_rows, CUtensorMap* tm, OpCoord* oc) {
+  if (op.n_row_atoms < 1 || op.n_row_atoms + op.n_batch_atoms > 4) return SMARTMEM_ERR_UNSUPPORTED;
+  if (((uintptr_t)op.ptr & 15) != 0) return SMARTMEM_ERR_ALIGNMENT;
+  const int nr = op.n_row_atoms, nb = op.n_batch_atoms;
+  const long long in_ext = op.row_extent[nr - 1], in_str = op.row_stride[nr - 1];
+  const bool mn = op.k_stride != 1;
+  if (mn && in_str != 1) return SMARTMEM_ERR_UNSUPPORTED;
+  if (nr > 1 && in_ext % tile_rows) return SMARTMEM_ERR_UNSUPPORTED;
+  uint64_t dims[5], strides[4];
+  uint32_t box[5];
+  int rank = 0;
+  auto push = [&](long long ext, long long str_elems, uint32_t bx) -> bool {
+    if (rank > 0) {
+      if ((str_elems * 2) % 16 || str_elems <= 0) return false;
+      strides[rank - 1] = (uint64_t)str_elems * 2;
+    }
+    dims[rank] = (uint64_t)ext;
+    box[rank] = bx;
+    ++rank;
+    return true;
+  };
+  bool ok = true;
+  if (!mn) {
+    ok = ok && push(op.K, 1, BK) && push(in_ext, in_str, (uint32_t)tile_rows);
+  } else {
+    ok = ok && push(in_ext, 1, 64) && push(op.K, op.k_stride, BK);
+  }
+  memset(oc, 0, sizeof(*oc));
+  for (int i = nr - 2; i >= 0 && ok; --i) {
+    ok = push(op.row_extent[i], op.row_stride[i], 1);
+    oc->outer[oc->n_outer++] = make_fastdiv((uint32_t)op.row_extent[i]);
+    oc->n_outer_row++;
+  }
+  for (int i = nb - 1; i >= 0 && ok; --i) {
+    ok = push(op.batch_extent[i], op.batch_stride[i], 1);
+    oc->outer[oc->n_outer++] = make_fastdiv((uint32_t)op.batch_extent[i]);
+  }
+  if (!ok) return SMARTMEM_ERR_UNSUPPORTED;
+  if (rank < 2) return SMARTMEM_ERR_UNSUPPORTED;
+  oc->rank = rank;
+  oc->mn_major = mn ? 1 : 0;
+  oc->tiles_inner = make_fastdiv((uint32_t)((in_ext + tile_rows - 1) / tile_rows));
+  return encode_cached(op.ptr, rank, dims, strides, box, tm);
+}
+
+template <int BN, int STAGES, bool A_MN>
+int launch_t(const CUtensorMap& ta, const CUtensorMap& tb, const GemmArgs& g, dim3 grid, cudaStream_t st) {
+  constexpr size_t smem = 1024 + STAGES * (A_STAGE_BYTES + BN * BK * 2) + (2 * STAGES + 1) * 8 + 16 + BN * 4;
+  static bool configured = false;
+  if (!configured) {
+    if (cudaFuncSetAttribute(gemm_tc_kernel<BN, STAGES, A_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+        cudaSuccess)
+      return SMARTMEM_ERR_CUDA;
+    configured = true;
+  }
+  gemm_tc_kernel<BN, STAGES, A_MN><<<grid, 192, smem, st>>>(ta, tb, g);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
+}
+
+}  // namespace
+
+int tc_operand_from_map(const smartmem_index_map_t& m, int n_batch_atoms, int n_row_atoms, const void* ptr,
+                        TcOperand* op) {
+  if (m.klass == 3 || m.n_rolls > 0) return SMARTMEM_ERR_UNSUPPORTED;
+  const int nk = m.n_atoms - n_batch_atoms - n_row_atoms;
+  if (nk != 1 || n_row_atoms < 1 || n_row_atoms > 3 || n_batch_atoms > 3) return SMARTMEM_ERR_UNSUPPORTED;
+  memset(op, 0, sizeof(*op));
+  op->ptr = (const char*)ptr + m.base * 2;
+  op->n_batch_atoms = n_batch_atoms;
+  op->n_row_atoms = n_row_atoms;
+  for (int i = 0; i < n_batch_atoms; ++i) {
+    op->batch_extent[i] = m.extent[i];
+    op->batch_stride[i] = m.src_stride[i];
+  }
+  for (int i = 0; i < n_row_atoms; ++i) {
+    op->row_extent[i] = m.extent[n_batch_atoms + i];
+    op->row_stride[i] = m.src_stride[n_batch_atoms + i];
+  }
+  op->K = m.extent[m.n_atoms - 1];
+  op->k_stride = m.src_stride[m.n_atoms - 1];
+  return SMARTMEM_OK;
+}
+
+TcOperand tc_operand_plain(const void* ptr, long long rows, long long K, long long ld) {
+  TcOperand op;
+  memset(&op, 0, sizeof(op));
+  op.ptr = ptr;
+  op.n_row_atoms = 1;
+  op.row_extent[0] = rows;
+  op.row_stride[0] = ld;
+  op.K = K;
+  op.k_stride = 1;
+  return op;
+}
+
+int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep, long long batch, long long M,
+                   long long N, long long K, cudaStream_t st) {
+  if (M < 1 || N < 1 || K < 1 || batch < 1 || batch > 65535 || M >= (1ll << 31) || N >= (1ll << 31))
+    return SMARTMEM_ERR_UNSUPPORTED;
+  if (A.K != K || B.K != K) return SMARTMEM_ERR_SHAPE;
+  if (((uintptr_t)ep.out & 15) || ((uintptr_t)ep.residual & 15) || ep.ldc % 8) return SMARTMEM_ERR_ALIGNMENT;
+  const bool a_mn = A.k_stride != 1;
+  if (B.k_stride != 1) return SMARTMEM_ERR_UNSUPPORTED;
+  // tile width: the widest of {256, 128, 96, 64} that divides N (fewest wasted columns), else 128
+  int bn = 128;
+  if (ep.rope_cols > 0) bn = 256;
+  else if (N % 256 == 0) bn = 256;
+  else if (N % 128 == 0) bn = 128;
+  else if (N % 96 == 0) bn = 96;
+  else if (N % 64 == 0) bn = 64;
+  if (ep.rope_cols > 0 && (N % 256 || ep.rope_cols % 128 || !ep.rope_tab || ep.rope_S < 1)) return SMARTMEM_ERR_UNSUPPORTED;
+  const int nkb = (int)((K + BK - 1) / BK);
+  const int stages = nkb <= 2 ? 2 : 4;
+  GemmArgs g;
+  memset(&g, 0, sizeof(g));
+  CUtensorMap ta, tb;
+  int rc = build_operand(A, BM, &ta, &g.ca);
+  if (rc != SMARTMEM_OK) return rc;
+  rc = build_operand(B, bn, &tb, &g.cb);
+  if (rc != SMARTMEM_OK) return rc;
+  g.M = (int)M; g.N = (int)N; g.K = (int)K;
+  g.out = (__nv_bfloat16*)ep.out;
+  g.ldc = ep.ldc;
+  g.out_batch_stride = ep.out_batch_stride;
+  g.bias = (const __nv_bfloat16*)ep.bias;
+  g.residual = (const __nv_bfloat16*)ep.residual;
+  g.gelu = ep.gelu;
+  g.has_rowmap = ep.rowmap ? 1 : 0;
+  if (ep.rowmap) g.rowmap = *ep.rowmap;
+  g.rope_cols = ep.rope_cols;
+  g.rope_S = ep.rope_S;
+  g.rope_tab = (const float2*)ep.rope_tab;
+  g.status = device_status_ptr();
+  if (!g.status) return SMARTMEM_ERR_CUDA;
+  dim3 grid((unsigned)((N + bn - 1) / bn), (unsigned)((M + BM - 1) / BM), (unsigned)batch);
+  if (grid.y > 65535) return SMARTMEM_ERR_UNSUPPORTED;
+#define SM_CASE(BN_, ST_, MN_)                                                                  \
+  if (bn == BN_ && stages == ST_ && a_mn == MN_) return launch_t<BN_, ST_, MN_>(ta, tb, g, grid, st);
+  SM_CASE(256, 4, false) SM_CASE(256, 2, false) SM_CASE(128, 4, false) SM_CASE(128, 2, false)
+  SM_CASE(96, 4, false) SM_CASE(96, 2, false) SM_CASE(64, 4, false) SM_CASE(64, 2, false)
+  SM_CASE(256, 4, true) SM_CASE(128, 4, true) SM_CASE(256, 2, true) SM_CASE(128, 2, true)
+#undef SM_CASE
+  return SMARTMEM_ERR_UNSUPPORTED;
+}
+
+}  // namespace smartmem

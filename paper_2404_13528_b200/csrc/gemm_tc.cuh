@@ -1,0 +1,37 @@
+// Host-side interface of the tcgen05 GEMM.
+#pragma once
+#include "common.cuh"
+
+namespace smartmem {
+
+// A [rows, K] bf16 operand as it lies in the producer's buffer: its rows are indexed by up
+// to 3 "row atoms" (mixed radix, outermost first) below up to 3 batch atoms; strides are in
+// elements.  k_stride == 1: reduction-dim contiguous (K-major).  Otherwise the innermost row
+// atom must be contiguous (MN-major operand).
+struct TcOperand {
+  const void* ptr;
+  int n_batch_atoms, n_row_atoms;
+  long long batch_extent[3], batch_stride[3];
+  long long row_extent[3], row_stride[3];
+  long long K, k_stride;
+};
+
+struct TcEpilogue {
+  void* out;                 // bf16
+  long long ldc;             // row pitch in elements (ignored for rows placed by rowmap)
+  long long out_batch_stride;
+  const void* bias;          // [N] bf16 or null
+  const void* residual;      // same addressing as out, or null
+  int gelu;
+  const DevMap* rowmap;      // output row -> element offset, or null
+  int rope_cols, rope_S;     // rotate columns [0, rope_cols) in 128-wide heads; position = row % rope_S
+  const void* rope_tab;      // float2 [rope_S, 64]
+};
+
+int tc_operand_from_map(const smartmem_index_map_t& m, int n_batch_atoms, int n_row_atoms, const void* ptr,
+                        TcOperand* op);
+TcOperand tc_operand_plain(const void* ptr, long long rows, long long K, long long ld);
+int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep, long long batch, long long M,
+                   long long N, long long K, cudaStream_t st);
+
+}  // namespace smartmem

@@ -1,0 +1,152 @@
+// LayerNorm / RMSNorm over the last dimension (kept operators: ILD & Variable, Table 3).
+// The rows may be fetched through a composed index map (cyclic shift + window partition
+// folded into the loads), so the normalised rows come out in the consumer's order with no
+// layout copy in between.  Statistics are fp32 and two-pass (mean, then centred variance);
+// reductions use warp shuffles.
+#include "common.cuh"
+
+namespace smartmem {
+namespace {
+
+template <int LPR>
+__device__ __forceinline__ float group_sum(float v) {
+#pragma unroll
+  for (int o = LPR / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+  return v;
+}
+
+// LPR lanes cooperate on one row; VPL 16-byte vectors per lane are kept in registers
+// (VPL == 0: any row length, the row is re-read from L1/L2 for each pass).
+template <typename T, int LPR, int VPL, bool RMS>
+__global__ void __launch_bounds__(256) norm_kernel(const T* __restrict__ src, T* __restrict__ dst,
+                                                   const T* __restrict__ gamma, const T* __restrict__ beta, float eps,
+                                                   long long rows, int C, const __grid_constant__ DevMap rowmap,
+                                                   int has_map) {
+  constexpr int KV = ElemIO<T>::kVec;
+  constexpr int NV = VPL > 0 ? VPL : 1;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int sub = lane % LPR, rsub = lane / LPR;
+  const long long row = ((long long)blockIdx.x * 8 + warp) * (32 / LPR) + rsub;
+  const bool active = row < rows;
+  const long long soff = active ? (has_map ? devmap_eval(rowmap, (uint32_t)row) : row * (long long)C) : 0;
+  const T* s = src + soff;
+  const int nvec = C / KV;
+  const float invC = 1.0f / (float)C;
+  float v[NV][KV];
+  float sum = 0.f;
+  if constexpr (VPL > 0) {
+#pragma unroll
+    for (int k = 0; k < VPL; ++k) {
+      const int vi = sub + k * LPR;
+      if (active && vi < nvec) {
+        ElemIO<T>::load(s + vi * KV, v[k]);
+      } else {
+#pragma unroll
+        for (int e = 0; e < KV; ++e) v[k][e] = 0.f;
+      }
+#pragma unroll
+      for (int e = 0; e < KV; ++e) sum += RMS ? v[k][e] * v[k][e] : v[k][e];
+    }
+  } else {
+    for (int vi = sub; vi < nvec && active; vi += LPR) {
+      ElemIO<T>::load(s + vi * KV, v[0]);
+#pragma unroll
+      for (int e = 0; e < KV; ++e) sum += RMS ? v[0][e] * v[0][e] : v[0][e];
+    }
+  }
+  sum = group_sum<LPR>(sum);
+  float mean = 0.f, rstd;
+  if constexpr (RMS) {
+    rstd = rsqrtf(sum * invC + eps);
+  } else {
+    mean = sum * invC;
+    float sq = 0.f;
+    if constexpr (VPL > 0) {
+#pragma unroll
+      for (int k = 0; k < VPL; ++k) {
+        const int vi = sub + k * LPR;
+        if (active && vi < nvec) {
+#pragma unroll
+          for (int e = 0; e < KV; ++e) sq += (v[k][e] - mean) * (v[k][e] - mean);
+        }
+      }
+    } else {
+      for (int vi = sub; vi < nvec && active; vi += LPR) {
+        ElemIO<T>::load(s + vi * KV, v[0]);
+#pragma unroll
+        for (int e = 0; e < KV; ++e) sq += (v[0][e] - mean) * (v[0][e] - mean);
+      }
+    }
+    sq = group_sum<LPR>(sq);
+    rstd = rsqrtf(sq * invC + eps);
+  }
+  if (!active) return;
+  T* d = dst + row * (long long)C;
+  auto emit = [&](int vi, float* x) {
+    float g[KV], b[KV], y[KV];
+    ElemIO<T>::load(gamma + vi * KV, g);
+    if constexpr (!RMS) ElemIO<T>::load(beta + vi * KV, b);
+#pragma unroll
+    for (int e = 0; e < KV; ++e) y[e] = RMS ? x[e] * rstd * g[e] : (x[e] - mean) * rstd * g[e] + b[e];
+    ElemIO<T>::store(d + vi * KV, y);
+  };
+  if constexpr (VPL > 0) {
+#pragma unroll
+    for (int k = 0; k < VPL; ++k) {
+      const int vi = sub + k * LPR;
+      if (vi < nvec) emit(vi, v[k]);
+    }
+  } else {
+    for (int vi = sub; vi < nvec; vi += LPR) {
+      ElemIO<T>::load(s + vi * KV, v[0]);
+      emit(vi, v[0]);
+    }
+  }
+}
+
+template <typename T, bool RMS>
+int launch_norm_t(const void* src, void* dst, const void* gamma, const void* beta, float eps, long long rows, int C,
+                  const DevMap* rowmap, cudaStream_t st) {
+  constexpr int KV = ElemIO<T>::kVec;
+  if (C % KV) return SMARTMEM_ERR_UNSUPPORTED;
+  if (rows >= (1ll << 31)) return SMARTMEM_ERR_UNSUPPORTED;
+  const int nvec = C / KV;
+  DevMap dm;
+  memset(&dm, 0, sizeof(dm));
+  if (rowmap) dm = *rowmap;
+  const int has = rowmap ? 1 : 0;
+  const T* s = (const T*)src;
+  T* d = (T*)dst;
+  const T* g = (const T*)gamma;
+  const T* b = (const T*)beta;
+#define SM_LAUNCH(LPR, VPL)                                                                      \
+  {                                                                                              \
+    long long rpb = 8 * (32 / LPR);                                                              \
+    unsigned grid = (unsigned)((rows + rpb - 1) / rpb);                                          \
+    norm_kernel<T, LPR, VPL, RMS><<<grid, 256, 0, st>>>(s, d, g, b, eps, rows, C, dm, has);      \
+  }
+  if (nvec <= 4) SM_LAUNCH(4, 1)
+  else if (nvec <= 8) SM_LAUNCH(8, 1)
+  else if (nvec <= 16) SM_LAUNCH(16, 1)
+  else if (nvec <= 32) SM_LAUNCH(32, 1)
+  else if (nvec <= 64) SM_LAUNCH(32, 2)
+  else if (nvec <= 128) SM_LAUNCH(32, 4)
+  else SM_LAUNCH(32, 0)
+#undef SM_LAUNCH
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
+}
+
+}  // namespace
+
+int launch_norm(int dtype, bool rms, const void* src, void* dst, const void* gamma, const void* beta, float eps,
+                long long rows, int C, const DevMap* rowmap, cudaStream_t st) {
+  if (rows == 0) return SMARTMEM_OK;
+  if (dtype == SMARTMEM_F32)
+    return rms ? launch_norm_t<float, true>(src, dst, gamma, beta, eps, rows, C, rowmap, st)
+               : launch_norm_t<float, false>(src, dst, gamma, beta, eps, rows, C, rowmap, st);
+  return rms ? launch_norm_t<__nv_bfloat16, true>(src, dst, gamma, beta, eps, rows, C, rowmap, st)
+             : launch_norm_t<__nv_bfloat16, false>(src, dst, gamma, beta, eps, rows, C, rowmap, st);
+}
+
+}  // namespace smartmem
