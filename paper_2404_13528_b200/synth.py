@@ -156,7 +156,7 @@ def chain_inputs(config_id: int, which: str, dtype: str = "bf16", small: bool = 
         return {"xq": normal(seed, 0, (B, S, H * D), 1.0, 0.0, dtype),
                 "xk": normal(seed, 1, (B, S, H * D), 1.0, 0.0, dtype), "dims": (B, S, H, D)}
     if which == "2b":
-        B, C, Hh, Ww, N = (2, 64, 8, 24, 64) if small else (8, 256, 64, 64, 256)
+        B, C, Hh, Ww, N = (2, 64, 8, 32, 128) if small else (8, 256, 64, 64, 256)
         return {"x": normal(seed, 2, (B, C, Hh, Ww), 1.0, 0.0, dtype),
                 "w": normal(seed, 3, (N, C), 0.02, 0.0, dtype), "dims": (B, C, Hh, Ww, N)}
     raise ValueError(which)

@@ -1,0 +1,126 @@
+"""GPU parity of smartmem_run_chain: copy-only layout chains are bit-exact against the
+oracle's materialised tensors; GEMM consumers are bit-identical between ELIMINATE and
+EXPLICIT and within the bf16 tolerance of the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import chains
+from paper_2404_13528_b200 import binding as sm
+from paper_2404_13528_b200 import synth
+from tests.gpu_util import assert_close_bf16, check_status, stream, to_dev, to_host_bits, to_host_f64
+from tests.test_planner import _ops_from_chain
+
+pytestmark = pytest.mark.gpu
+
+
+def run_plan(ops, descs, mode, inputs, out_shape, dtype=torch.bfloat16):
+    plan = sm.smartmem_plan(ops, descs, mode)
+    try:
+        wsb = sm.smartmem_plan_workspace_bytes(plan)
+        ws = torch.empty(max(wsb, 16), dtype=torch.uint8, device="cuda")
+        out = torch.full(out_shape, float("nan"), dtype=dtype, device="cuda")
+        sm.smartmem_run_chain(plan, [t.data_ptr() for t in inputs], [out.data_ptr()], ws.data_ptr(), wsb, stream())
+        check_status()
+        return out
+    finally:
+        sm.smartmem_plan_destroy(plan)
+
+
+def copy_chain_case(shape, chain, dtype="bf16"):
+    x = synth.normal(77, 0, shape, dtype=dtype)
+    ref = chains.apply_layout_chain(x, chain)           # moves the raw storage values: exact
+    xd = to_dev(x)
+    ops = _ops_from_chain(chain) + [sm.make_op(sm.OP_COPY)]
+    desc = [sm.make_desc(shape, sm.BF16 if dtype == "bf16" else sm.F32)]
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    for mode in (sm.ELIMINATE, sm.EXPLICIT):
+        out = run_plan(ops, desc, mode, [xd], ref.shape, tdt)
+        assert np.array_equal(to_host_bits(out), ref), f"mode {mode}"
+
+
+CH2A = lambda B, S, H, D: [{"op": "reshape", "shape": (B, S, H, D)}, {"op": "transpose", "perm": (0, 2, 1, 3)}]
+CH2B = lambda B, C, H, W: [{"op": "transpose", "perm": (0, 2, 3, 1)}, {"op": "reshape", "shape": (B, H * W, C)}]
+
+
+def swin_e1(s, ws):
+    return [{"op": "roll", "shift": -s, "axis": 1}, {"op": "roll", "shift": -s, "axis": 2},
+            {"op": "window_partition", "window": ws}]
+
+
+@pytest.mark.parametrize("shape,chain", [
+    ((2, 96, 4 * 64), CH2A(2, 96, 4, 64)),
+    ((8, 1024, 16 * 64), CH2A(8, 1024, 16, 64)),                    # full size of the benchmark chain
+    ((2, 64, 8, 24), CH2B(2, 64, 8, 24)),                           # ragged tiles -> gather path
+    ((2, 128, 16, 16), CH2B(2, 128, 16, 16)),                       # tiled transpose path
+    ((8, 256, 64, 64), CH2B(8, 256, 64, 64)),                       # full size
+    ((1, 8, 8, 32), swin_e1(2, 4)),
+    ((3, 14, 14, 96), swin_e1(3, 7)),
+    ((2, 56, 56, 96), swin_e1(3, 7)),
+    ((5, 5, 5), [{"op": "reshape", "shape": (5, 25)}, {"op": "transpose", "perm": (1, 0)}]),
+    ((4, 6, 10), [{"op": "slice", "start": (1, 0, 2), "extent": (2, 6, 8)}, {"op": "transpose", "perm": (2, 0, 1)}]),
+])
+def test_copy_only_chains_bit_exact(shape, chain):
+    copy_chain_case(shape, chain)
+
+
+def test_copy_only_chain_fp32():
+    copy_chain_case((1, 8, 8, 32), swin_e1(2, 4), dtype="f32")
+    copy_chain_case((3, 7, 20), [{"op": "transpose", "perm": (1, 2, 0)}], dtype="f32")
+
+
+@pytest.mark.parametrize("small", [True, False])
+def test_chain_2a_qkt(small):
+    inp = synth.chain_inputs(2, "2a", small=small)
+    B, S, H, D = inp["dims"]
+    xq, xk = to_dev(inp["xq"]), to_dev(inp["xk"])
+    ops = _ops_from_chain(CH2A(B, S, H, D)) + [sm.make_op(sm.OP_BMM_NT, side_input=(1, 0))]
+    descs = [sm.make_desc((B, S, H * D)), sm.make_desc((B, S, H * D))]
+    outs = [run_plan(ops, descs, mode, [xq, xk], (B, H, S, S)) for mode in (sm.ELIMINATE, sm.EXPLICIT)]
+    assert torch.equal(outs[0], outs[1])                 # same kernel, only the load path differs
+    got = to_host_f64(outs[0])
+    if small:
+        ref = chains.chain_2a_scores(synth.to_f64(inp["xq"]), synth.to_f64(inp["xk"]), H)
+        assert_close_bf16(got, ref, "2a scores")
+    else:                                                # sampled (b, h) slices at full size
+        q = synth.to_f64(inp["xq"]).reshape(B, S, H, D)
+        k = synth.to_f64(inp["xk"]).reshape(B, S, H, D)
+        for b, h in [(0, 0), (3, 7), (7, 15)]:
+            assert_close_bf16(got[b, h], q[b, :, h] @ k[b, :, h].T, f"2a scores[{b},{h}]")
+
+
+@pytest.mark.parametrize("small", [True, False])
+def test_chain_2b_gemm(small):
+    inp = synth.chain_inputs(2, "2b", small=small)
+    B, C, Hh, Ww, N = inp["dims"]
+    x, w = to_dev(inp["x"]), to_dev(inp["w"])
+    ops = _ops_from_chain(CH2B(B, C, Hh, Ww)) + [sm.make_op(sm.OP_LINEAR, side_input=(1, 0))]
+    descs = [sm.make_desc((B, C, Hh, Ww)), sm.make_desc((N, C))]
+    outs = [run_plan(ops, descs, mode, [x, w], (B, Hh * Ww, N)) for mode in (sm.ELIMINATE, sm.EXPLICIT)]
+    assert torch.equal(outs[0], outs[1])
+    ref = chains.chain_2b_gemm(synth.to_f64(inp["x"]), synth.to_f64(inp["w"])).reshape(B, Hh * Ww, N)
+    assert_close_bf16(to_host_f64(outs[0]), ref, "2b gemm")
+
+
+def test_plain_linear_shapes():
+    """Plain [M,K] x [N,K]^T with ragged M, several tile widths and a K tail."""
+    for M, N, K in [(200, 96, 96), (128, 288, 96), (300, 384, 96), (130, 96, 384), (257, 512, 512), (64, 64, 64)]:
+        a = synth.normal(5, M * 7 + N, (M, K), dtype="bf16")
+        w = synth.normal(5, K * 3 + N + 1, (N, K), std=0.05, dtype="bf16")
+        out = run_plan([sm.make_op(sm.OP_LINEAR, side_input=(1, 0))], [sm.make_desc((M, K)), sm.make_desc((N, K))],
+                       sm.ELIMINATE, [to_dev(a), to_dev(w)], (M, N))
+        assert_close_bf16(to_host_f64(out), synth.to_f64(a) @ synth.to_f64(w).T, f"linear {M}x{N}x{K}")
+
+
+def test_run_chain_rejects_bad_arguments():
+    plan = sm.smartmem_plan([sm.make_op(sm.OP_TRANSPOSE, perm=(1, 0)), sm.make_op(sm.OP_COPY)],
+                            [sm.make_desc((64, 64))], sm.EXPLICIT)
+    x = torch.zeros(64 * 64 + 8, dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros(64, 64, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(sm.SmartmemError) as e:
+        sm.smartmem_run_chain(plan, [x.data_ptr() + 2], [out.data_ptr()], 0, 0, stream())
+    assert e.value.code == sm.ERR_ALIGNMENT
+    with pytest.raises(sm.SmartmemError) as e:
+        sm.smartmem_run_chain(plan, [x.data_ptr()], [out.data_ptr()], 0, 0, stream())
+    assert e.value.code == sm.ERR_WORKSPACE
+    sm.smartmem_plan_destroy(plan)
