@@ -108,10 +108,3 @@ EXPORT int smartmem_attn_layer(const smartmem_attn_params_t* p, const void* x, v
                                size_t workspace_bytes, int32_t mode, void* cuda_stream) {
   return SMARTMEM_ERR_UNSUPPORTED;
 }
-EXPORT int smartmem_swin_block_workspace_bytes(const smartmem_swin_params_t* p, int32_t mode, size_t* bytes) {
-  return SMARTMEM_ERR_UNSUPPORTED;
-}
-EXPORT int smartmem_swin_block(const smartmem_swin_params_t* p, const void* x, void* y, void* workspace,
-                               size_t workspace_bytes, int32_t mode, void* cuda_stream) {
-  return SMARTMEM_ERR_UNSUPPORTED;
-}

@@ -1,0 +1,41 @@
+// Host-side interface of the attention kernels and the fp32 plain-FMA GEMM.
+#pragma once
+#include "common.cuh"
+
+namespace smartmem {
+
+// An attention operand x[n, h, t, e] addressed as ptr + n*sn + h*sh + t*st + e*se (elements).
+struct AttnOperand {
+  const void* ptr;
+  long long sn, sh, st, se;
+};
+
+struct WinAttnArgs {
+  AttnOperand q, k, v, o;
+  const void* table;        // [(2ws-1)^2, heads]
+  int table_f32;
+  int heads, T, ws, d, shift, H, W, nWw, win_per_img;
+  float scale;
+};
+int launch_window_attention(const WinAttnArgs& a, int dtype, long long n_windows, cudaStream_t st);
+
+// Causal attention over [S] positions for `heads` heads of dimension 128 (bf16).
+struct CausalAttnArgs {
+  AttnOperand q, k, v, o;   // n = batch, h = head
+  int S, heads, batch;
+  float scale;
+};
+int launch_causal_attention(const CausalAttnArgs& a, cudaStream_t st);
+
+// out[M,N] = A[M,K] W[N,K]^T (+bias)(GELU)(+residual), fp32 with plain FMAs.  Rows of A may be
+// gathered through `amap`, rows of out scattered through `omap` (residual uses the same offsets).
+struct SimtGemmArgs {
+  const float* A; const float* W; const float* bias; const float* residual; float* out;
+  int M, N, K;
+  long long lda, ldc;
+  int gelu, has_amap, has_omap;
+  DevMap amap, omap;
+};
+int launch_gemm_simt_f32(const SimtGemmArgs& a, cudaStream_t st);
+
+}  // namespace smartmem

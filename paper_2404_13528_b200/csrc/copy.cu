@@ -112,12 +112,65 @@ __global__ void __launch_bounds__(256) copy_transpose16_kernel(const __grid_cons
   }
 }
 
+
+// Batched transpose of small contiguous blocks: the last two consumer atoms are (J, I) of a
+// source block [I][J] that is contiguous (stride of I == extent of J), e.g. a materialised K^T of
+// one (window, head).  One CTA per block: coalesced 16-byte loads of the whole block into shared
+// memory, coalesced 4-byte stores of the transposed block.
+__global__ void __launch_bounds__(256) copy_block_transpose16_kernel(const __grid_constant__ DevMap outer,
+                                                                     const uint16_t* __restrict__ src,
+                                                                     uint16_t* __restrict__ dst, int EI, int EJ) {
+  extern __shared__ uint16_t blk[];
+  const int RS = EJ + 2;
+  const int E = EI * EJ;
+  const long long so = devmap_eval(outer, blockIdx.x);
+  const uint16_t* sp = src + so;
+  uint16_t* dp = dst + (long long)blockIdx.x * E;
+  if ((so & 7) == 0 && (EJ & 7) == 0) {
+    for (int l = threadIdx.x * 8; l < E; l += 256 * 8) {
+      const uint4 v = *reinterpret_cast<const uint4*>(sp + l);
+      const int i = l / EJ, j = l - i * EJ;
+      uint32_t* d32 = reinterpret_cast<uint32_t*>(blk + i * RS + j);
+      d32[0] = v.x; d32[1] = v.y; d32[2] = v.z; d32[3] = v.w;
+    }
+  } else {
+    for (int l = threadIdx.x; l < E; l += 256) {
+      const int i = l / EJ, j = l - i * EJ;
+      blk[i * RS + j] = sp[l];
+    }
+  }
+  __syncthreads();
+  for (int q = threadIdx.x * 2; q < E; q += 512) {        // E is even (checked by the launcher)
+    int j0 = q / EI, i0 = q - j0 * EI;
+    int i1 = i0 + 1, j1 = j0;
+    if (i1 == EI) { i1 = 0; ++j1; }
+    const uint32_t v = (uint32_t)blk[i0 * RS + j0] | ((uint32_t)blk[i1 * RS + j1] << 16);
+    *reinterpret_cast<uint32_t*>(dp + q) = v;
+  }
+}
+
 }  // namespace
 
 int launch_copy_map(const smartmem_index_map_t& map, int elem_size, const void* src, void* dst, cudaStream_t st) {
   if (map.klass == 3) return SMARTMEM_ERR_UNSUPPORTED;
   if (map.n_elements == 0) return SMARTMEM_OK;
   const int n = map.n_atoms;
+  // fast path: batched transpose of small contiguous blocks
+  if (map.klass == 1 && elem_size == 2 && n >= 2 && map.src_stride[n - 1] != 1 && map.src_stride[n - 2] == 1 &&
+      map.src_stride[n - 1] == map.extent[n - 2] && map.extent[n - 1] * map.extent[n - 2] <= 16384 &&
+      (map.extent[n - 1] * map.extent[n - 2]) % 2 == 0) {
+    DevMap outer;
+    long long blocks = map.n_elements / (map.extent[n - 1] * map.extent[n - 2]);
+    if (make_devmap(map, 0, n - 2, 1, true, &outer) && blocks < (1ll << 31)) {
+      const int EI = (int)map.extent[n - 1], EJ = (int)map.extent[n - 2];
+      const size_t smem = (size_t)EI * (EJ + 2) * 2;
+      if (smem <= 40000) {
+      copy_block_transpose16_kernel<<<(unsigned)blocks, 256, smem, st>>>(outer, (const uint16_t*)src, (uint16_t*)dst, EI, EJ);
+      count_launch();
+      return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
+      }
+    }
+  }
   // fast path: tiled transpose
   if (map.klass == 1 && elem_size == 2 && n >= 2 && map.src_stride[n - 1] != 1) {
     int J = -1;

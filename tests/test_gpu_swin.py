@@ -1,0 +1,116 @@
+"""GPU parity of smartmem_swin_block against the fp64 oracle, both modes."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import swin as oswin
+from paper_2404_13528_b200 import binding as sm
+from paper_2404_13528_b200 import synth
+from tests.gpu_util import assert_close_bf16, assert_close_f32, check_status, stream, to_dev, to_host_f64
+
+pytestmark = pytest.mark.gpu
+
+PARAM_NAMES = ["ln1_g", "ln1_b", "w_qkv", "b_qkv", "rel_bias_table", "w_proj", "b_proj",
+               "ln2_g", "ln2_b", "w_fc1", "b_fc1", "w_fc2", "b_fc2"]
+
+
+def run_block(inp, dev, *, B, H, W, C, heads, window, shift, mlp_ratio, dtype, mode, x_dev=None):
+    p = sm.SwinParams()
+    p.dtype = sm.F32 if dtype == "f32" else sm.BF16
+    p.B, p.H, p.W, p.C, p.heads, p.window, p.shift, p.mlp_ratio = B, H, W, C, heads, window, shift, mlp_ratio
+    p.ln_eps = 1e-5
+    for n in PARAM_NAMES:
+        if n in dev:
+            setattr(p, n, dev[n].data_ptr())
+    x = dev["x"] if x_dev is None else x_dev
+    y = torch.full_like(x, float("nan"))
+    wsb = sm.smartmem_swin_block_workspace_bytes(p, mode)
+    ws = torch.empty(wsb, dtype=torch.uint8, device="cuda")
+    sm.smartmem_swin_block(p, x.data_ptr(), y.data_ptr(), ws.data_ptr(), wsb, mode, stream())
+    check_status()
+    return y
+
+
+def oracle_block(inp, images, *, heads, window, shift, mlp_ratio, x=None):
+    pf = {k: synth.to_f64(v) for k, v in inp.items() if k != "x"}
+    xf = synth.to_f64(inp["x"] if x is None else x)[images]
+    return oswin.swin_block(xf, pf, heads=heads, window=window, shift=shift, mlp_ratio=mlp_ratio)
+
+
+def case(config_id, *, B, H, W, C, heads, window, shift, mlp_ratio, dtype, images=None, **kw):
+    inp = synth.swin_inputs(config_id, B, H, W, C, heads, window, mlp_ratio, dtype, **kw)
+    dev = {k: to_dev(v) for k, v in inp.items()}
+    images = list(range(B)) if images is None else images
+    ref = oracle_block(inp, images, heads=heads, window=window, shift=shift, mlp_ratio=mlp_ratio)
+    outs = []
+    for mode in (sm.ELIMINATE, sm.EXPLICIT):
+        y = run_block(inp, dev, B=B, H=H, W=W, C=C, heads=heads, window=window, shift=shift, mlp_ratio=mlp_ratio,
+                      dtype=dtype, mode=mode)
+        got = to_host_f64(y)[images]
+        (assert_close_f32 if dtype == "f32" else assert_close_bf16)(got, ref, f"mode {mode}")
+        outs.append(y)
+    # both modes run the same arithmetic in the same order: only the data movement differs
+    assert torch.equal(outs[0], outs[1])
+
+
+def test_config1_tiny_swin_fp32():
+    """B=1, 8x8 tokens, C=32, 2 heads of 16, window 4, shift 2, attention half only."""
+    cfg = dict(B=1, H=8, W=8, C=32, heads=2, window=4, shift=2, mlp_ratio=0, dtype="f32")
+    case(1, perturbed_affine=False, zero_bias=True, **cfg)      # gamma = 1, beta = 0, b = 0 as stated
+    case(1, perturbed_affine=True, zero_bias=False, **cfg)      # an indexing error in gamma/beta/bias would show
+
+
+def test_fp32_with_mlp_and_no_shift():
+    case(11, B=2, H=8, W=12, C=32, heads=2, window=4, shift=0, mlp_ratio=2, dtype="f32")
+    case(12, B=1, H=14, W=14, C=64, heads=2, window=7, shift=3, mlp_ratio=4, dtype="f32")
+
+
+@pytest.mark.parametrize("cfg", [
+    dict(B=2, H=14, W=14, C=64, heads=2, window=7, shift=3, mlp_ratio=4),
+    dict(B=3, H=14, W=21, C=96, heads=3, window=7, shift=0, mlp_ratio=4),
+    dict(B=1, H=8, W=8, C=32, heads=2, window=4, shift=2, mlp_ratio=0),       # head_dim 16, T = 16
+    dict(B=2, H=16, W=16, C=64, heads=2, window=8, shift=5, mlp_ratio=2),     # T = 64 exactly
+    dict(B=5, H=7, W=7, C=32, heads=1, window=7, shift=0, mlp_ratio=1),       # one window per image, ragged M
+])
+def test_small_bf16_blocks(cfg):
+    case(20, dtype="bf16", **cfg)
+
+
+def test_config3_swin_t_stage1_full_size():
+    """B=32, 56x56, C=96, 3 heads, window 7, shift 3, MLP x4 at full size; the oracle checks two images."""
+    case(3, B=32, H=56, W=56, C=96, heads=3, window=7, shift=3, mlp_ratio=4, dtype="bf16", images=[0, 31])
+
+
+def test_config4_swin_b_stage3_block_pair():
+    """B=64, 14x14, C=512, 16 heads: a regular block then a shifted block with independent weights."""
+    B, H, W, C, heads, ws = 64, 14, 14, 512, 16, 7
+    images = [0, 63]
+    a = synth.swin_inputs(4, B, H, W, C, heads, ws, 4, "bf16", weight_set=0)
+    b = synth.swin_inputs(4, B, H, W, C, heads, ws, 4, "bf16", weight_set=1)
+    da, db = {k: to_dev(v) for k, v in a.items()}, {k: to_dev(v) for k, v in b.items()}
+    outs = []
+    for mode in (sm.ELIMINATE, sm.EXPLICIT):
+        y1 = run_block(a, da, B=B, H=H, W=W, C=C, heads=heads, window=ws, shift=0, mlp_ratio=4, dtype="bf16", mode=mode)
+        y2 = run_block(b, db, B=B, H=H, W=W, C=C, heads=heads, window=ws, shift=3, mlp_ratio=4, dtype="bf16", mode=mode,
+                       x_dev=y1)
+        outs.append((y1, y2))
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
+    y1, y2 = outs[0]
+    ref1 = oracle_block(a, images, heads=heads, window=ws, shift=0, mlp_ratio=4)
+    assert_close_bf16(to_host_f64(y1)[images], ref1, "block A")
+    # block B is checked on the GPU's own (bf16) block-A output, so that each block is compared
+    # with the oracle on identical inputs
+    y1_bits = y1.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+    ref2 = oracle_block(b, images, heads=heads, window=ws, shift=3, mlp_ratio=4, x=y1_bits)
+    assert_close_bf16(to_host_f64(y2)[images], ref2, "block B")
+
+
+def test_swin_block_rejects_bad_arguments():
+    inp = synth.swin_inputs(1, 1, 8, 8, 32, 2, 4, 0, "f32")
+    dev = {k: to_dev(v) for k, v in inp.items()}
+    base = dict(B=1, H=8, W=8, C=32, heads=2, window=4, shift=2, mlp_ratio=0, dtype="f32", mode=sm.ELIMINATE)
+    for bad, code in [(dict(window=3), sm.ERR_SHAPE), (dict(shift=4), sm.ERR_SHAPE), (dict(heads=3), sm.ERR_SHAPE),
+                      (dict(heads=4), sm.ERR_UNSUPPORTED), (dict(mode=5), sm.ERR_INVALID_ARG)]:
+        with pytest.raises(sm.SmartmemError) as e:
+            run_block(inp, dev, **{**base, **bad})
+        assert e.value.code == code, bad
