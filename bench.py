@@ -1,0 +1,328 @@
+#!/usr/bin/env python
+"""Benchmark of the layout-elimination hot path: one Swin block per step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+A step is one pass of the whole hot path (LayerNorm -> shifted-window attention -> projection
+-> MLP, every layout operator folded into the kernels) over one batch of synthetic input of the
+Swin-T stage-1 shape (B=32, 56x56 tokens, C=96, 3 heads, window 7, shift 3, MLP x4, bf16).
+`value` is tokens/s with inputs resident in HBM; `e2e` is the same metric through the C ABI
+with host buffers (pinned host -> device copy of x and device -> host copy of y inside the timed
+region).  The explicit-layout variant of the same kernels is timed beside it, the dominant
+kernel is placed on the HBM roofline from per-kernel CUDA-event timings, and the CPU oracle is
+timed on the host cores as a reported baseline.  With N > 1 every rank runs its own batch
+(weak scaling, no collective on the data path).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+WORKLOAD = dict(name="swin_t_stage1_block", config_id=3, B=32, H=56, W=56, C=96, heads=3, window=7, shift=3,
+                mlp_ratio=4, dtype="bf16")
+METRIC = "swin_block_tokens_per_s"
+UNIT = "tokens/s"
+N_SETS = 4          # rotating buffer sets: > 1 GB touched between reuses of a set (L2 is 126 MB)
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "source": "measured (MEASURED_PEAKS.json)"}
+    return {"hbm_gbs": 6650.0, "source": "fallback (earlier measurement on this pool)"}
+
+
+def algorithmic_bytes(w):
+    """Compulsory HBM bytes of each kernel of the ELIMINATE chain: every input once, every output once."""
+    U = w["B"] * w["H"] * w["W"] * w["C"] * 2          # one [M, C] bf16 tensor
+    C, r = w["C"], w["mlp_ratio"]
+    wq, wp, w1 = 3 * C * C * 2, C * C * 2, r * C * C * 2
+    return {
+        "ln1_gather": 2 * U, "qkv_gemm": U + wq + 3 * U, "window_attention": 3 * U + U,
+        "proj_gemm_scatter_residual": U + wp + U + U, "ln2": 2 * U, "fc1_gemm_gelu": U + w1 + r * U,
+        "fc2_gemm_residual": r * U + w1 + U + U,
+        # explicit-layout variant: each copy reads and writes its tensor once
+        "ln1": 2 * U, "copy_shift": 2 * U, "copy_partition": 2 * U, "copy_head_split": 6 * U, "copy_k_transpose": 2 * U,
+        "copy_head_merge": 2 * U, "copy_window_reverse": 2 * U, "copy_unshift": 2 * U, "proj_gemm_residual": 3 * U + wp,
+    }
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the GPU is under load."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "50", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([t.strip() for t in line.split(",")])
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        busy = [c for c in sm if c > 0.5 * max(sm)] or sm
+        return {"sm_mhz": statistics.median(busy), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_tokens_per_s(n_images, repeats=1):
+    """The CPU oracle, as it stands, on `n_images` images of the workload.  Returns (tokens/s, seconds)."""
+    import numpy as np
+    from oracle import swin as oswin
+    from paper_2404_13528_b200 import synth
+    w = WORKLOAD
+    inp = synth.swin_inputs(w["config_id"], n_images, w["H"], w["W"], w["C"], w["heads"], w["window"], w["mlp_ratio"], w["dtype"])
+    pf = {k: synth.to_f64(v) for k, v in inp.items() if k != "x"}
+    x = synth.to_f64(inp["x"])
+    best = float("inf")
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        y = oswin.swin_block(x, pf, heads=w["heads"], window=w["window"], shift=w["shift"], mlp_ratio=w["mlp_ratio"])
+        best = min(best, time.perf_counter() - t0)
+    assert np.isfinite(y).all()
+    return n_images * w["H"] * w["W"] / best, best
+
+
+def host_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info()]
+        return max(n) if n else (os.cpu_count() or 1)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args):
+    """Reference arm: the CPU oracle timed on the host cores, each step a bounded sample (2 images)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy  # noqa: F401  (loads the BLAS threadpool before counting its threads)
+    n_img = 2
+    for _ in range(args.warmup):
+        oracle_tokens_per_s(n_img)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_tokens_per_s(n_img)
+    dt = time.perf_counter() - t0
+    w = WORKLOAD
+    val = n_img * w["H"] * w["W"] * args.steps / dt
+    sample = f"{n_img} of {w['B']} images of the workload per step (the images of a batch are independent)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w["name"], "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": host_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=500)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="smartmem", choices=["smartmem", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    args.warmup = max(args.warmup, 3)
+
+    import torch
+    from paper_2404_13528_b200 import binding as sm
+    from paper_2404_13528_b200 import synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    sm.lib()
+
+    w = WORKLOAD
+    M = w["B"] * w["H"] * w["W"]
+    inp = synth.swin_inputs(w["config_id"] + 1000 * rank, w["B"], w["H"], w["W"], w["C"], w["heads"], w["window"],
+                            w["mlp_ratio"], w["dtype"])
+
+    def dev(a):
+        return torch.from_numpy(a.view("int16").copy()).cuda().view(torch.bfloat16)
+
+    params = {k: dev(v) for k, v in inp.items() if k != "x"}
+    x_host = torch.from_numpy(inp["x"].view("int16").copy()).view(torch.bfloat16).pin_memory()
+    y_host = torch.empty_like(x_host).pin_memory()
+    xs = [x_host.cuda() for _ in range(N_SETS)]
+    ys = [torch.empty_like(xs[0]) for _ in range(N_SETS)]
+    p = sm.SwinParams()
+    p.dtype = sm.BF16
+    p.B, p.H, p.W, p.C, p.heads, p.window, p.shift, p.mlp_ratio = (w["B"], w["H"], w["W"], w["C"], w["heads"], w["window"],
+                                                                   w["shift"], w["mlp_ratio"])
+    p.ln_eps = 1e-5
+    for k, t in params.items():
+        setattr(p, k, t.data_ptr())
+    wsb = {m: sm.smartmem_swin_block_workspace_bytes(p, m) for m in (sm.ELIMINATE, sm.EXPLICIT)}
+    wss = [torch.empty(wsb[sm.EXPLICIT], dtype=torch.uint8, device="cuda") for _ in range(N_SETS)]
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def step(i, mode):
+        j = i % N_SETS
+        sm.smartmem_swin_block(p, xs[j].data_ptr(), ys[j].data_ptr(), wss[j].data_ptr(), wsb[mode], mode, stream)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(mode, steps):
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n0 = sm.smartmem_launch_count()
+        e0.record()
+        for i in range(steps):
+            step(i, mode)
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1)
+        launches = sm.smartmem_launch_count() - n0
+        if dist is not None:
+            t = torch.tensor([ms], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms, launches
+
+    sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ else
+                           os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local])
+    sampler.start()
+    for i in range(args.warmup):
+        step(i, sm.ELIMINATE)
+        step(i, sm.EXPLICIT)
+    ms_elim, launches = timed(sm.ELIMINATE, args.steps)
+    ms_expl, _ = timed(sm.EXPLICIT, args.steps)
+    st = sm.smartmem_last_device_status(stream)
+    if st != sm.OK:
+        raise SystemExit(f"device status {st}: {sm.smartmem_status_string(st)}")
+
+    # per-kernel durations (CUDA events recorded on the launching stream around every launch)
+    per = {sm.ELIMINATE: {}, sm.EXPLICIT: {}}
+    reps = min(args.steps, 30)
+    for mode in per:
+        for i in range(reps):
+            j = i % N_SETS
+            for name, ms in sm.smartmem_swin_block_timed(p, xs[j].data_ptr(), ys[j].data_ptr(), wss[j].data_ptr(), wsb[mode],
+                                                         mode, stream):
+                per[mode].setdefault(name, []).append(ms)
+    peaks = measured_peaks()
+    ab = algorithmic_bytes(w)
+    kernels = {}
+    for mode, tag in ((sm.ELIMINATE, "eliminate"), (sm.EXPLICIT, "explicit")):
+        kernels[tag] = []
+        for name, v in per[mode].items():
+            ms = statistics.median(v)
+            gbs = ab[name] / (ms * 1e-3) / 1e9 if ms > 0 else None
+            kernels[tag].append({"kernel": name, "ms": round(ms, 5), "algorithmic_bytes": ab[name],
+                                 "gbs": gbs and round(gbs, 1), "frac_of_hbm_peak": gbs and round(gbs / peaks["hbm_gbs"], 4)})
+    dom = max(kernels["eliminate"], key=lambda k: k["ms"])
+
+    # end to end through the C ABI with host buffers
+    e2e_steps = min(args.steps, 30)
+    for i in range(3):
+        xs[0].copy_(x_host, non_blocking=True); step(0, sm.ELIMINATE); y_host.copy_(ys[0], non_blocking=True)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(e2e_steps):
+        j = i % N_SETS
+        xs[j].copy_(x_host, non_blocking=True)
+        step(i, sm.ELIMINATE)
+        y_host.copy_(ys[j], non_blocking=True)
+    e1.record()
+    barrier()
+    ms_e2e = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([ms_e2e], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_e2e = float(t.item())
+    clocks = sampler.stop()
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, secs = oracle_tokens_per_s(w["B"])
+        cpu = {"value": v, "unit": UNIT, "cores": host_threads(), "kind": "oracle",
+               "sample": f"the whole workload once ({w['B']} images, {secs:.1f} s)"}
+
+    if rank == 0:
+        tokens = M * world
+        value = tokens * args.steps / (ms_elim * 1e-3)
+        traffic = None
+        tpath = os.path.join(ROOT, "profiles", "traffic.json")      # per-launch DRAM bytes from an ncu capture
+        if os.path.exists(tpath):
+            with open(tpath) as f:
+                traffic = json.load(f).get(dom["kernel"])
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_elim / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": w["name"], "B_per_gpu": w["B"], "H": w["H"], "W": w["W"], "C": w["C"], "heads": w["heads"],
+                       "window": w["window"], "shift": w["shift"], "mlp_ratio": w["mlp_ratio"], "mode": "eliminate",
+                       "l2": f"{N_SETS} rotating buffer sets (> 1 GB touched between reuses of a set)",
+                       "parallelism": f"replicas x{world}" if world > 1 else "single gpu"},
+            "explicit_variant": {"value": tokens * args.steps / (ms_expl * 1e-3), "unit": UNIT,
+                                 "ms_per_step": ms_expl / args.steps, "speedup_of_eliminate": ms_expl / ms_elim},
+            "e2e": {"value": tokens * e2e_steps / (ms_e2e * 1e-3), "unit": UNIT,
+                    "h2d_bytes_per_step": x_host.numel() * 2, "d2h_bytes_per_step": y_host.numel() * 2},
+            "gpu_launches": launches,
+            "clocks": clocks,
+            "roofline": {"bound": "hbm", "kernel": dom["kernel"], "achieved": dom["gbs"], "peak": peaks["hbm_gbs"],
+                         "unit": "GB/s", "frac": dom["frac_of_hbm_peak"], "traffic": traffic, "peak_source": peaks["source"]},
+            "kernels": kernels,
+        }
+        if cpu is not None:
+            out["cpu_baseline"] = cpu
+        print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -180,6 +180,15 @@ int smartmem_swin_block_workspace_bytes(const smartmem_swin_params_t* p, int32_t
 int smartmem_swin_block(const smartmem_swin_params_t* p, const void* x, void* y, void* workspace,
                         size_t workspace_bytes, int32_t mode, void* cuda_stream);
 
+/* Measurement aid (no counterpart in the paper): the same block, with a CUDA event recorded on
+ * `cuda_stream` before every kernel launch.  Synchronises the stream, then writes the duration of
+ * each kernel in milliseconds to kernel_ms[i] (host) and its label, NUL-terminated, to
+ * kernel_names + i * names_stride (host); *n_kernels receives the count (at most max_kernels). */
+int smartmem_swin_block_timed(const smartmem_swin_params_t* p, const void* x, void* y, void* workspace,
+                              size_t workspace_bytes, int32_t mode, void* cuda_stream, float* kernel_ms,
+                              char* kernel_names, int32_t names_stride, int32_t max_kernels,
+                              int32_t* n_kernels);
+
 /* One decoder attention layer, prefill.  x, y: [B,S,hidden], bf16.  w_qkv is [3*hidden, hidden]
  * with output columns ordered (q|k|v, head, head_dim); RoPE pairs (i, i + head_dim/2). */
 typedef struct {

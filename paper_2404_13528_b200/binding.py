@@ -60,7 +60,7 @@ EXPORTED = [
     "smartmem_plan_num_steps", "smartmem_plan_get_map", "smartmem_plan_output_desc",
     "smartmem_plan_workspace_bytes", "smartmem_map_eval", "smartmem_plan_eval_sequential", "smartmem_run_chain",
     "smartmem_swin_block_workspace_bytes", "smartmem_swin_block", "smartmem_attn_layer_workspace_bytes",
-    "smartmem_attn_layer", "smartmem_last_device_status", "smartmem_launch_count", "smartmem_status_string",
+    "smartmem_attn_layer", "smartmem_swin_block_timed", "smartmem_last_device_status", "smartmem_launch_count", "smartmem_status_string",
 ]
 
 _lib = None
@@ -91,6 +91,8 @@ def lib() -> C.CDLL:
         "smartmem_run_chain": (C.c_int, [vp, P(vp), P(vp), vp, C.c_size_t, vp]),
         "smartmem_swin_block_workspace_bytes": (C.c_int, [P(SwinParams), i32, P(C.c_size_t)]),
         "smartmem_swin_block": (C.c_int, [P(SwinParams), vp, vp, vp, C.c_size_t, i32, vp]),
+        "smartmem_swin_block_timed": (C.c_int, [P(SwinParams), vp, vp, vp, C.c_size_t, i32, vp, P(C.c_float), C.c_char_p,
+                                      i32, i32, P(i32)]),
         "smartmem_attn_layer_workspace_bytes": (C.c_int, [P(AttnParams), i32, P(C.c_size_t)]),
         "smartmem_attn_layer": (C.c_int, [P(AttnParams), vp, vp, vp, C.c_size_t, i32, vp]),
         "smartmem_last_device_status": (C.c_int, [vp, P(i32)]),
@@ -223,6 +225,18 @@ def smartmem_swin_block_workspace_bytes(p: SwinParams, mode: int) -> int:
 
 def smartmem_swin_block(p: SwinParams, x: int, y: int, workspace: int, workspace_bytes: int, mode: int, stream: int):
     _check(lib().smartmem_swin_block(C.byref(p), x, y, workspace, workspace_bytes, mode, stream), "smartmem_swin_block")
+
+
+def smartmem_swin_block_timed(p: SwinParams, x: int, y: int, workspace: int, workspace_bytes: int, mode: int, stream: int):
+    """Runs the block with an event before every kernel; returns [(label, milliseconds), ...]."""
+    maxk, stride = 32, 48
+    ms = (C.c_float * maxk)()
+    names = C.create_string_buffer(maxk * stride)
+    n = C.c_int32()
+    _check(lib().smartmem_swin_block_timed(C.byref(p), x, y, workspace, workspace_bytes, mode, stream, ms, names, stride,
+                                           maxk, C.byref(n)), "smartmem_swin_block_timed")
+    raw = names.raw
+    return [(raw[i * stride:(i + 1) * stride].split(b"\0", 1)[0].decode(), float(ms[i])) for i in range(n.value)]
 
 
 def smartmem_attn_layer_workspace_bytes(p: AttnParams, mode: int) -> int:
