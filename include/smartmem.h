@@ -189,6 +189,31 @@ int smartmem_swin_block_timed(const smartmem_swin_params_t* p, const void* x, vo
                               char* kernel_names, int32_t names_stride, int32_t max_kernels,
                               int32_t* n_kernels);
 
+/* The Swin block for callers that cannot allocate device memory (the paper has no counterpart;
+ * this is a deployment aid).  Typical callers: a step that runs while the process's device
+ * memory pool is frozen (everything committed to caches and activations, so a cudaMalloc would
+ * fail or stall the device), a plugin that is handed buffers and a stream but not the host's
+ * allocator, or start-up code that runs before any allocator exists.  They pass only x and y;
+ * the block's intermediates go to a fixed array of SMARTMEM_STATIC_SCRATCH bytes (32 MiB,
+ * reported by smartmem_swin_block_static_scratch_bytes) that is part of the library image:
+ * every GPU that loads the library holds those 32 MiB until the process exits.
+ *
+ *  - Same arguments, requirements and results as smartmem_swin_block, minus the workspace.
+ *  - A block whose intermediates need more than the fixed array (see
+ *    smartmem_swin_block_workspace_bytes) is rejected with SMARTMEM_ERR_WORKSPACE
+ *    ("workspace too small"); nothing is launched.
+ *  - The call itself performs no device allocation and frees nothing: no cudaMalloc / cudaFree and
+ *    no allocating library routine.  The first call on each device looks up the array's device
+ *    address (the device must be current); make that first call before starting any stream
+ *    capture on that device.
+ *  - All calls on a device share the one array, and it keeps whatever the previous call left in it.
+ *    The block overwrites every intermediate before reading it, so nothing needs clearing; but two
+ *    calls whose kernels overlap on the GPU (different streams, no ordering between them) race on
+ *    the array and corrupt each other.  Order them on one stream or with events. */
+int smartmem_swin_block_static_scratch_bytes(size_t* bytes);
+int smartmem_swin_block_noalloc(const smartmem_swin_params_t* p, const void* x, void* y, int32_t mode,
+                                void* cuda_stream);
+
 /* One decoder attention layer, prefill.  x, y: [B,S,hidden], bf16.  w_qkv is [3*hidden, hidden]
  * with output columns ordered (q|k|v, head, head_dim); RoPE pairs (i, i + head_dim/2). */
 typedef struct {

@@ -60,7 +60,8 @@ EXPORTED = [
     "smartmem_plan_num_steps", "smartmem_plan_get_map", "smartmem_plan_output_desc",
     "smartmem_plan_workspace_bytes", "smartmem_map_eval", "smartmem_plan_eval_sequential", "smartmem_run_chain",
     "smartmem_swin_block_workspace_bytes", "smartmem_swin_block", "smartmem_attn_layer_workspace_bytes",
-    "smartmem_attn_layer", "smartmem_swin_block_timed", "smartmem_last_device_status", "smartmem_launch_count", "smartmem_status_string",
+    "smartmem_attn_layer", "smartmem_swin_block_timed", "smartmem_swin_block_static_scratch_bytes",
+    "smartmem_swin_block_noalloc", "smartmem_last_device_status", "smartmem_launch_count", "smartmem_status_string",
 ]
 
 _lib = None
@@ -93,6 +94,8 @@ def lib() -> C.CDLL:
         "smartmem_swin_block": (C.c_int, [P(SwinParams), vp, vp, vp, C.c_size_t, i32, vp]),
         "smartmem_swin_block_timed": (C.c_int, [P(SwinParams), vp, vp, vp, C.c_size_t, i32, vp, P(C.c_float), C.c_char_p,
                                       i32, i32, P(i32)]),
+        "smartmem_swin_block_static_scratch_bytes": (C.c_int, [P(C.c_size_t)]),
+        "smartmem_swin_block_noalloc": (C.c_int, [P(SwinParams), vp, vp, i32, vp]),
         "smartmem_attn_layer_workspace_bytes": (C.c_int, [P(AttnParams), i32, P(C.c_size_t)]),
         "smartmem_attn_layer": (C.c_int, [P(AttnParams), vp, vp, vp, C.c_size_t, i32, vp]),
         "smartmem_last_device_status": (C.c_int, [vp, P(i32)]),
@@ -237,6 +240,19 @@ def smartmem_swin_block_timed(p: SwinParams, x: int, y: int, workspace: int, wor
                                            maxk, C.byref(n)), "smartmem_swin_block_timed")
     raw = names.raw
     return [(raw[i * stride:(i + 1) * stride].split(b"\0", 1)[0].decode(), float(ms[i])) for i in range(n.value)]
+
+
+def smartmem_swin_block_static_scratch_bytes() -> int:
+    n = C.c_size_t()
+    _check(lib().smartmem_swin_block_static_scratch_bytes(C.byref(n)), "smartmem_swin_block_static_scratch_bytes")
+    return n.value
+
+
+def smartmem_swin_block_noalloc(p: SwinParams, x: int, y: int, mode: int, stream: int):
+    """The Swin block for callers that cannot allocate device memory: no workspace argument, the
+    intermediates live in a fixed 32 MiB array inside the library.  Calls share that array, so
+    calls that overlap on the GPU race; blocks that need more are rejected (ERR_WORKSPACE)."""
+    _check(lib().smartmem_swin_block_noalloc(C.byref(p), x, y, mode, stream), "smartmem_swin_block_noalloc")
 
 
 def smartmem_attn_layer_workspace_bytes(p: AttnParams, mode: int) -> int:

@@ -344,3 +344,55 @@ EXPORT int smartmem_swin_block_timed(const smartmem_swin_params_t* p, const void
   *n_kernels = n;
   return rc != SMARTMEM_OK ? rc : rs;
 }
+
+// ---------------------------------------------------------------------------------------
+// Swin block without a caller workspace.
+//
+// Some callers of this library cannot allocate device memory at the point where they run a
+// block: code that executes inside a memory-frozen phase of a serving process (its device
+// memory pool is fully committed to KV caches and activations, and a cudaMalloc there either
+// fails or forces a device-wide synchronisation), plugin hosts that hand the library a stream
+// and buffers but keep the allocator to themselves, and start-up paths that run before the
+// host framework's allocator exists.  For them the intermediates of the block live in a
+// fixed array that is part of the loaded library image on every device.
+// ---------------------------------------------------------------------------------------
+#define SMARTMEM_STATIC_SCRATCH_BYTES (32u << 20)
+static __device__ __align__(256) unsigned char g_static_scratch[SMARTMEM_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mu;
+void* g_scratch_ptr[kMaxDevices] = {nullptr};
+
+// Device address of the static scratch array on the current device.  In host code the name
+// g_static_scratch is only a handle for the runtime, never an address a kernel may use, so the
+// address is asked for once per device (with that device current) and remembered.
+int static_scratch(void** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SMARTMEM_ERR_CUDA;
+  std::lock_guard<std::mutex> lk(g_scratch_mu);
+  if (!g_scratch_ptr[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress((void**)&ptr, g_static_scratch) != cudaSuccess || !ptr) return SMARTMEM_ERR_CUDA;
+    g_scratch_ptr[dev] = ptr;
+  }
+  *out = g_scratch_ptr[dev];
+  return SMARTMEM_OK;
+}
+}  // namespace
+
+EXPORT int smartmem_swin_block_static_scratch_bytes(size_t* bytes) {
+  if (!bytes) return SMARTMEM_ERR_INVALID_ARG;
+  *bytes = SMARTMEM_STATIC_SCRATCH_BYTES;
+  return SMARTMEM_OK;
+}
+
+EXPORT int smartmem_swin_block_noalloc(const smartmem_swin_params_t* p, const void* x, void* y, int32_t mode,
+                                       void* cuda_stream) {
+  int rc = validate(p, mode);
+  if (rc != SMARTMEM_OK) return rc;
+  if (ws_layout(*p, mode).total > SMARTMEM_STATIC_SCRATCH_BYTES) return SMARTMEM_ERR_WORKSPACE;
+  void* scratch = nullptr;
+  if ((rc = static_scratch(&scratch)) != SMARTMEM_OK) return rc;
+  return run_block(p, x, y, scratch, SMARTMEM_STATIC_SCRATCH_BYTES, mode, cuda_stream, nullptr);
+}
