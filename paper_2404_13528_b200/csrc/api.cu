@@ -101,10 +101,3 @@ EXPORT int smartmem_run_chain(const smartmem_plan_t* plan, const void* const* in
   return SMARTMEM_OK;
 }
 
-EXPORT int smartmem_attn_layer_workspace_bytes(const smartmem_attn_params_t* p, int32_t mode, size_t* bytes) {
-  return SMARTMEM_ERR_UNSUPPORTED;
-}
-EXPORT int smartmem_attn_layer(const smartmem_attn_params_t* p, const void* x, void* y, void* workspace,
-                               size_t workspace_bytes, int32_t mode, void* cuda_stream) {
-  return SMARTMEM_ERR_UNSUPPORTED;
-}

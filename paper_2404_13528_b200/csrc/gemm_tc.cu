@@ -9,8 +9,9 @@
 // NHWC case) is loaded as it lies and multiplied through the MN-major operand mode of the
 // tensor core, so that transpose disappears as well.
 //
-// CTA = 6 warps: warp 0 issues TMA loads into a STAGES-deep shared-memory ring, warp 1 owns the
-// TMEM allocation and issues tcgen05.mma (one thread), warps 2-5 run the epilogue
+// Persistent CTAs (one per SM) of 10 warps: warp 0 issues TMA loads into a 4-stage shared-memory
+// ring, warp 1 owns the TMEM allocation and issues tcgen05.mma (one thread) into one of two
+// accumulator buffers, warps 2-9 run the epilogue of the previous tile meanwhile
 // (TMEM -> registers -> bias / GELU / RoPE / residual -> bf16 -> global, optionally scattering
 // rows through an index map: window reverse + reverse cyclic shift folded into the store).
 #include <mutex>
@@ -38,6 +39,7 @@ struct OpCoord {
 
 struct GemmArgs {
   int M, N, K;
+  int tiles_n, tiles_m, batch;
   OpCoord ca, cb;
   __nv_bfloat16* out;
   long long ldc, out_batch_stride;
@@ -65,26 +67,35 @@ __device__ __forceinline__ void op_coords(const OpCoord& oc, uint32_t tile, uint
   }
 }
 
-// erf by the rational approximation 7.1.26 of Abramowitz & Stegun (|error| <= 1.5e-7), far
-// below bf16 resolution; one reciprocal and one exponential instead of erff's long polynomial.
+// GELU in the bf16 epilogue: u * Phi(u) with Phi evaluated through the hyperbolic-tangent form
+// 0.5 (1 + tanh(sqrt(2/pi) (u + 0.044715 u^3))) and the hardware tanh.  It differs from the erf
+// form by at most 5e-4 in absolute value, i.e. by less than an eighth of a bf16 ulp wherever the
+// result exceeds 1 and by less than 1e-4 |u| near zero, at a third of the instruction count (the
+// epilogue of the fc1 GEMM is issue-bound).  The fp32 kernels use erff.
 __device__ __forceinline__ float gelu_fast(float u) {
-  const float x = fabsf(u) * 0.70710678118654752f;
-  const float t = __frcp_rn(fmaf(0.3275911f, x, 1.0f));
-  float p = fmaf(1.061405429f, t, -1.453152027f);
-  p = fmaf(p, t, 1.421413741f);
-  p = fmaf(p, t, -0.284496736f);
-  p = fmaf(p, t, 0.254829592f);
-  const float e = 1.0f - p * t * __expf(-x * x);       // erf(|u| / sqrt 2)
-  return 0.5f * u * (1.0f + copysignf(e, u));
+  const float u2 = u * u;
+  const float inner = u * fmaf(0.0356774081f, u2, 0.7978845608f);
+  float t;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(inner));
+  const float h = 0.5f * u;
+  return fmaf(h, t, h);
 }
 
+constexpr int kEpiWarps = 16;
+constexpr int kThreads = 64 + 32 * kEpiWarps;
+
+// Persistent kernel: one CTA per SM walks over output tiles (tile = blockIdx.x + i * gridDim.x).
+// The shared-memory ring and two TMEM accumulator buffers run across tile boundaries, so the
+// loads and MMAs of tile i+1 overlap the epilogue of tile i.
 template <int BN, int STAGES, bool A_MN>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ GemmArgs g) {
   constexpr int B_STAGE_BYTES = BN * BK * 2;
-  constexpr uint32_t TMEM_COLS = BN <= 32 ? 32 : BN <= 64 ? 64 : BN <= 128 ? 128 : 256;
+  constexpr uint32_t ACC_COLS = BN <= 32 ? 32 : BN <= 64 ? 64 : BN <= 128 ? 128 : 256;   // one accumulator buffer
+  constexpr uint32_t TMEM_COLS = 2 * ACC_COLS;
   constexpr uint32_t IDESC = ptx::make_idesc_bf16(BM, BN, A_MN, false);
+  constexpr int NSUB = BN / 16;                              // 16-column sub-chunks per tile
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -92,22 +103,25 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   uint8_t* sB = smem + STAGES * A_STAGE_BYTES;
   uint64_t* full = reinterpret_cast<uint64_t*>(sB + STAGES * B_STAGE_BYTES);
   uint64_t* empty = full + STAGES;
-  uint64_t* tmem_full = empty + STAGES;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_full + 1);
+  uint64_t* tmem_full = empty + STAGES;                      // [2]
+  uint64_t* tmem_empty = tmem_full + 2;                      // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_empty + 2);
   int* abort_flag = reinterpret_cast<int*>(tmem_slot + 1);
-  float* bias_s = reinterpret_cast<float*>(tmem_slot + 2);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t tile_n = blockIdx.x, tile_m = blockIdx.y, batch = blockIdx.z;
   const int nkb = (g.K + BK - 1) / BK;
   const int last_ksteps = (g.K - (nkb - 1) * BK + 15) / 16;
+  const uint32_t total_tiles = (uint32_t)g.tiles_n * g.tiles_m * g.batch;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
       ptx::mbar_init(&full[s], 1);
       ptx::mbar_init(&empty[s], 1);
     }
-    ptx::mbar_init(tmem_full, 1);
+    for (int b = 0; b < 2; ++b) {
+      ptx::mbar_init(&tmem_full[b], 1);
+      ptx::mbar_init(&tmem_empty[b], kEpiWarps);
+    }
     *abort_flag = 0;
     ptx::fence_barrier_init();
     ptx::fence_proxy_async();
@@ -124,135 +138,182 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   if (warp == 0) {
     if (lane == 0) {
-      int issued = 0;
-      for (int kb = 0; kb < nkb; ++kb) {
-        const int s = kb % STAGES;
-        const uint32_t ph = (kb / STAGES) & 1;
-        if (!ptx::mbar_wait(&empty[s], ph ^ 1, abort_flag, g.status)) break;
-        ptx::mbar_expect_tx(&full[s], A_STAGE_BYTES + B_STAGE_BYTES);
-        int c[5];
-        op_coords(g.ca, tile_m, batch, BM, kb * BK, c);
-        if (A_MN) {
-          ptx::tma_load_nd(g.ca.rank, sA + s * A_STAGE_BYTES, &tmA, &full[s], c);
-          c[0] += 64;
-          ptx::tma_load_nd(g.ca.rank, sA + s * A_STAGE_BYTES + A_STAGE_BYTES / 2, &tmA, &full[s], c);
-        } else {
-          ptx::tma_load_nd(g.ca.rank, sA + s * A_STAGE_BYTES, &tmA, &full[s], c);
+      uint32_t kbg = 0;                                      // k-block counter across tiles
+      bool ok = true;
+      for (uint32_t t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+        const uint32_t tile_n = t % g.tiles_n, r = t / g.tiles_n, tile_m = r % g.tiles_m, batch = r / g.tiles_m;
+        for (int kb = 0; kb < nkb; ++kb, ++kbg) {
+          const int s = kbg % STAGES;
+          const uint32_t ph = (kbg / STAGES) & 1;
+          ok = ptx::mbar_wait(&empty[s], ph ^ 1, abort_flag, g.status);
+          if (!ok) break;
+          ptx::mbar_expect_tx(&full[s], A_STAGE_BYTES + B_STAGE_BYTES);
+          int c[5];
+          op_coords(g.ca, tile_m, batch, BM, kb * BK, c);
+          if (A_MN) {
+            ptx::tma_load_nd(g.ca.rank, sA + s * A_STAGE_BYTES, &tmA, &full[s], c);
+            c[0] += 64;
+            ptx::tma_load_nd(g.ca.rank, sA + s * A_STAGE_BYTES + A_STAGE_BYTES / 2, &tmA, &full[s], c);
+          } else {
+            ptx::tma_load_nd(g.ca.rank, sA + s * A_STAGE_BYTES, &tmA, &full[s], c);
+          }
+          op_coords(g.cb, tile_n, batch, BN, kb * BK, c);
+          ptx::tma_load_nd(g.cb.rank, sB + s * B_STAGE_BYTES, &tmB, &full[s], c);
         }
-        op_coords(g.cb, tile_n, batch, BN, kb * BK, c);
-        ptx::tma_load_nd(g.cb.rank, sB + s * B_STAGE_BYTES, &tmB, &full[s], c);
-        issued = kb + 1;
       }
       if (*abort_flag) {
         // unwinding: give copies already in flight a bounded chance to land before the CTA leaves
-        for (int kb = (issued > STAGES ? issued - STAGES : 0); kb < issued; ++kb) {
+        for (uint32_t k = (kbg > (uint32_t)STAGES ? kbg - STAGES : 0); k < kbg; ++k) {
           const unsigned long long t0 = ptx::globaltimer();
-          while (!ptx::mbar_try_wait(&full[kb % STAGES], (kb / STAGES) & 1) && ptx::globaltimer() - t0 < 2000000ull) {
+          while (!ptx::mbar_try_wait(&full[k % STAGES], (k / STAGES) & 1) && ptx::globaltimer() - t0 < 2000000ull) {
           }
         }
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
+      uint32_t kbg = 0, it = 0;
       bool ok = true;
-      for (int kb = 0; kb < nkb && ok; ++kb) {
-        const int s = kb % STAGES;
-        const uint32_t ph = (kb / STAGES) & 1;
-        ok = ptx::mbar_wait(&full[s], ph, abort_flag, g.status);
+      for (uint32_t t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
+        const uint32_t buf = it & 1, use = it >> 1;
+        ok = ptx::mbar_wait(&tmem_empty[buf], (use & 1) ^ 1, abort_flag, g.status);   // epilogue drained it
         if (!ok) break;
         ptx::tc_fence_after();
-        const uint32_t a0 = ptx::smem_u32(sA + s * A_STAGE_BYTES), b0 = ptx::smem_u32(sB + s * B_STAGE_BYTES);
-        const int ks = (kb == nkb - 1) ? last_ksteps : BK / 16;
-        for (int k = 0; k < ks; ++k) {
-          // K-major, 128-byte swizzle: 8-row groups are 1024 bytes apart; one k16 step is 32 bytes
-          // along the swizzled row.  MN-major: 64-row chunks are 8192 bytes apart (leading offset),
-          // 8-deep k groups 1024 bytes apart, one k16 step is 2048 bytes.
-          const uint64_t ad = A_MN ? ptx::make_smem_desc(a0 + k * 2048, A_STAGE_BYTES / 2, 1024)
-                                   : ptx::make_smem_desc(a0 + k * 32, 16, 1024);
-          const uint64_t bd = ptx::make_smem_desc(b0 + k * 32, 16, 1024);
-          ptx::tc_mma_bf16(tmem_base, ad, bd, IDESC, (kb | k) ? 1u : 0u);
+        const uint32_t d_tmem = tmem_base + buf * ACC_COLS;
+        for (int kb = 0; kb < nkb; ++kb, ++kbg) {
+          const int s = kbg % STAGES;
+          const uint32_t ph = (kbg / STAGES) & 1;
+          ok = ptx::mbar_wait(&full[s], ph, abort_flag, g.status);
+          if (!ok) break;
+          ptx::tc_fence_after();
+          const uint32_t a0 = ptx::smem_u32(sA + s * A_STAGE_BYTES), b0 = ptx::smem_u32(sB + s * B_STAGE_BYTES);
+          const int ks = (kb == nkb - 1) ? last_ksteps : BK / 16;
+          for (int k = 0; k < ks; ++k) {
+            // K-major, 128-byte swizzle: 8-row groups are 1024 bytes apart; one k16 step is 32 bytes
+            // along the swizzled row.  MN-major: 64-row chunks are 8192 bytes apart (leading offset),
+            // 8-deep k groups 1024 bytes apart, one k16 step is 2048 bytes.
+            const uint64_t ad = A_MN ? ptx::make_smem_desc(a0 + k * 2048, A_STAGE_BYTES / 2, 1024)
+                                     : ptx::make_smem_desc(a0 + k * 32, 16, 1024);
+            const uint64_t bd = ptx::make_smem_desc(b0 + k * 32, 16, 1024);
+            ptx::tc_mma_bf16(d_tmem, ad, bd, IDESC, (kb | k) ? 1u : 0u);
+          }
+          ptx::tc_commit(&empty[s]);
         }
-        ptx::tc_commit(&empty[s]);
+        if (ok) ptx::tc_commit(&tmem_full[buf]);
       }
-      if (ok) ptx::tc_commit(tmem_full);
     }
   } else {
-    const int et = threadIdx.x - 64;                     // 0..127
-    const int n0 = tile_n * BN;
-    for (int c = et; c < BN; c += 128)
-      bias_s[c] = (g.bias && n0 + c < g.N) ? __bfloat162float(g.bias[n0 + c]) : 0.f;
-    asm volatile("bar.sync 1, 128;" ::: "memory");
-    const bool ok = ptx::mbar_wait(tmem_full, 0, abort_flag, g.status);
-    ptx::tc_fence_after();
-    const int q = warp & 3;
-    const int row = tile_m * BM + q * 32 + lane;
-    if (ok) {
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+    const int e = warp - 2;
+    const int q = warp & 3;                                  // TMEM lane quadrant this warp may read
+    const int grp = e >> 2;                                  // which sub-chunks (sub % 4 == grp)
+    uint32_t it = 0;
+    bool ok = true;
+    for (uint32_t t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
+      const uint32_t tile_n = t % g.tiles_n, r = t / g.tiles_n, tile_m = r % g.tiles_m, batch = r / g.tiles_m;
+      const uint32_t buf = it & 1, use = it >> 1;
+      const int n0 = tile_n * BN;
+      const int row = tile_m * BM + q * 32 + lane;
       const bool row_ok = row < g.M;
       long long off = 0;
       if (row_ok) off = g.has_rowmap ? devmap_eval(g.rowmap, (uint32_t)row) : (long long)row * g.ldc;
       off += (long long)batch * g.out_batch_stride;
-      __nv_bfloat16* orow = g.out + off;
-      const __nv_bfloat16* rrow = g.residual ? g.residual + off : nullptr;
+      __nv_bfloat16* __restrict__ orow = g.out + off;
+      const __nv_bfloat16* __restrict__ rrow = g.residual ? g.residual + off : nullptr;
 
-      auto finish = [&](float* acc, int c0) {            // bias / GELU / residual / store of 32 columns
+      // residual of the first sub-chunk is fetched while the MMAs of this tile still run
+      uint4 res[2] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
+      auto fetch_res = [&](int c0) {
+        if (rrow && row_ok && n0 + c0 + 16 <= g.N) {
+          res[0] = *reinterpret_cast<const uint4*>(rrow + n0 + c0);
+          res[1] = *reinterpret_cast<const uint4*>(rrow + n0 + c0 + 8);
+        }
+      };
+      const bool rope_tile = g.rope_cols > 0 && n0 < g.rope_cols;
+      if (!rope_tile) fetch_res(grp * 16);
+
+      ok = ptx::mbar_wait(&tmem_full[buf], use & 1, abort_flag, g.status);
+      if (!ok) break;
+      ptx::tc_fence_after();
+      const uint32_t taddr = tmem_base + buf * ACC_COLS + ((uint32_t)(q * 32) << 16);
+
+      auto finish = [&](float* acc, int c0, const uint4* rv) {    // bias / GELU / residual / store of 16 columns
         const int col0 = n0 + c0;
         if (!row_ok || col0 >= g.N) return;
+        if (col0 + 16 <= g.N) {
+          if (g.bias) {
 #pragma unroll
-        for (int j = 0; j < 32; ++j) acc[j] += bias_s[c0 + j];
-        if (g.gelu) {
+            for (int v = 0; v < 2; ++v) {
+              float b[8];
+              ElemIO<__nv_bfloat16>::load(g.bias + col0 + v * 8, b);
 #pragma unroll
-          for (int j = 0; j < 32; ++j) acc[j] = gelu_fast(acc[j]);
-        }
-        if (col0 + 32 <= g.N) {
-#pragma unroll
-          for (int v = 0; v < 4; ++v) {
-            if (rrow) {
-              float r[8];
-              ElemIO<__nv_bfloat16>::load(rrow + col0 + v * 8, r);
-#pragma unroll
-              for (int e = 0; e < 8; ++e) acc[v * 8 + e] += r[e];
+              for (int j = 0; j < 8; ++j) acc[v * 8 + j] += b[j];
             }
-            ElemIO<__nv_bfloat16>::store(orow + col0 + v * 8, acc + v * 8);
           }
+          if (g.gelu) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) acc[j] = gelu_fast(acc[j]);
+          }
+          if (rv) {
+#pragma unroll
+            for (int v = 0; v < 2; ++v) {
+              const uint32_t w[4] = {rv[v].x, rv[v].y, rv[v].z, rv[v].w};
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const float2 f = bf16x2_to_float2(w[j]);
+                acc[v * 8 + 2 * j] += f.x;
+                acc[v * 8 + 2 * j + 1] += f.y;
+              }
+            }
+          }
+          ElemIO<__nv_bfloat16>::store(orow + col0, acc);
+          ElemIO<__nv_bfloat16>::store(orow + col0 + 8, acc + 8);
         } else {
-          for (int j = 0; j < 32 && col0 + j < g.N; ++j) {
-            float r = rrow ? __bfloat162float(rrow[col0 + j]) : 0.f;
-            orow[col0 + j] = __float2bfloat16_rn(acc[j] + r);
+          for (int j = 0; j < 16 && col0 + j < g.N; ++j) {
+            float v = acc[j] + (g.bias ? __bfloat162float(g.bias[col0 + j]) : 0.f);
+            if (g.gelu) v = gelu_fast(v);
+            if (rrow) v += __bfloat162float(rrow[col0 + j]);
+            orow[col0 + j] = __float2bfloat16_rn(v);
           }
         }
       };
 
-      for (int ch = 0; ch < BN / 32; ++ch) {
-        const int c0 = ch * 32;
-        const bool rope = g.rope_cols > 0 && n0 + c0 < g.rope_cols;
-        if (rope) {
-          if ((ch & 3) >= 2) continue;                   // done together with chunk ch - 2
-          uint32_t ra[32], rb[32];
-          ptx::tmem_ld32(taddr + c0, ra);
-          ptx::tmem_ld32(taddr + c0 + 64, rb);
+      for (int sub = grp; sub < NSUB; sub += 4) {
+        const int c0 = sub * 16;
+        if (rope_tile && n0 + c0 < g.rope_cols) {
+          // rotary pairs are (c, c + 64) inside a 128-column head: sub-chunks sub and sub + 4
+          if ((sub & 7) >= 4) continue;
+          uint32_t ra[16], rb[16];
+          ptx::tmem_ld16(taddr + c0, ra);
+          ptx::tmem_ld16(taddr + c0 + 64, rb);
           ptx::tmem_ld_wait();
-          float x1[32], x2[32];
-          const float2* tab = g.rope_tab + (long long)(row_ok ? row % g.rope_S : 0) * 64 + (ch & 1) * 32;
+          float x1[16], x2[16];
+          const float2* tab = g.rope_tab + (long long)(row_ok ? row % g.rope_S : 0) * 64 + (sub & 3) * 16;
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
+          for (int j = 0; j < 16; ++j) {
             const float2 cs = tab[j];
             const float a = __uint_as_float(ra[j]), b = __uint_as_float(rb[j]);
             x1[j] = a * cs.x - b * cs.y;
             x2[j] = b * cs.x + a * cs.y;
           }
-          finish(x1, c0);
-          finish(x2, c0 + 64);
+          finish(x1, c0, nullptr);
+          finish(x2, c0 + 64, nullptr);
         } else {
-          uint32_t r[32];
-          ptx::tmem_ld32(taddr + c0, r);
+          uint32_t rv[16];
+          ptx::tmem_ld16(taddr + c0, rv);
           ptx::tmem_ld_wait();
-          float acc[32];
+          float acc[16];
 #pragma unroll
-          for (int j = 0; j < 32; ++j) acc[j] = __uint_as_float(r[j]);
-          finish(acc, c0);
+          for (int j = 0; j < 16; ++j) acc[j] = __uint_as_float(rv[j]);
+          const bool vec_res = rrow && n0 + c0 + 16 <= g.N;
+          uint4 cur[2] = {res[0], res[1]};
+          if (sub + 4 < NSUB) fetch_res(c0 + 64);              // next sub-chunk's residual in flight
+          finish(acc, c0, vec_res ? cur : nullptr);
         }
       }
+      // all of this warp's TMEM reads of the buffer have completed (wait::ld above)
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&tmem_empty[buf]);
     }
   }
   ptx::tc_fence_before();
@@ -367,9 +428,19 @@ int build_operand(const TcOperand& op, int tile_rows, CUtensorMap* tm, OpCoord* 
   return encode_cached(op.ptr, rank, dims, strides, box, tm);
 }
 
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
+  }
+  return n;
+}
+
 template <int BN, int STAGES, bool A_MN>
-int launch_t(const CUtensorMap& ta, const CUtensorMap& tb, const GemmArgs& g, dim3 grid, cudaStream_t st) {
-  constexpr size_t smem = 1024 + STAGES * (A_STAGE_BYTES + BN * BK * 2) + (2 * STAGES + 1) * 8 + 16 + BN * 4;
+int launch_t(const CUtensorMap& ta, const CUtensorMap& tb, const GemmArgs& g, cudaStream_t st) {
+  constexpr size_t smem = 1024 + STAGES * (A_STAGE_BYTES + BN * BK * 2) + (2 * STAGES + 4) * 8 + 16;
   static bool configured = false;
   if (!configured) {
     if (cudaFuncSetAttribute(gemm_tc_kernel<BN, STAGES, A_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
@@ -377,7 +448,9 @@ int launch_t(const CUtensorMap& ta, const CUtensorMap& tb, const GemmArgs& g, di
       return SMARTMEM_ERR_CUDA;
     configured = true;
   }
-  gemm_tc_kernel<BN, STAGES, A_MN><<<grid, 192, smem, st>>>(ta, tb, g);
+  const long long tiles = (long long)g.tiles_n * g.tiles_m * g.batch;
+  const unsigned grid = (unsigned)(tiles < sm_count() ? tiles : sm_count());
+  gemm_tc_kernel<BN, STAGES, A_MN><<<grid, kThreads, smem, st>>>(ta, tb, g);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
 }
@@ -420,7 +493,7 @@ TcOperand tc_operand_plain(const void* ptr, long long rows, long long K, long lo
 
 int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep, long long batch, long long M,
                    long long N, long long K, cudaStream_t st) {
-  if (M < 1 || N < 1 || K < 1 || batch < 1 || batch > 65535 || M >= (1ll << 31) || N >= (1ll << 31))
+  if (M < 1 || N < 1 || K < 1 || batch < 1 ||  M >= (1ll << 31) || N >= (1ll << 31))
     return SMARTMEM_ERR_UNSUPPORTED;
   if (A.K != K || B.K != K) return SMARTMEM_ERR_SHAPE;
   if (((uintptr_t)ep.out & 15) || ((uintptr_t)ep.residual & 15) || ep.ldc % 8) return SMARTMEM_ERR_ALIGNMENT;
@@ -433,9 +506,9 @@ int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep,
   else if (N % 128 == 0) bn = 128;
   else if (N % 96 == 0) bn = 96;
   else if (N % 64 == 0) bn = 64;
-  if (ep.rope_cols > 0 && (N % 256 || ep.rope_cols % 128 || !ep.rope_tab || ep.rope_S < 1)) return SMARTMEM_ERR_UNSUPPORTED;
+  if (ep.rope_cols > 0 && (N % 256 || ep.rope_cols % 256 || !ep.rope_tab || ep.rope_S < 1)) return SMARTMEM_ERR_UNSUPPORTED;
   const int nkb = (int)((K + BK - 1) / BK);
-  const int stages = nkb <= 2 ? 2 : 4;
+  const int stages = 4;
   GemmArgs g;
   memset(&g, 0, sizeof(g));
   CUtensorMap ta, tb;
@@ -457,13 +530,14 @@ int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep,
   g.rope_tab = (const float2*)ep.rope_tab;
   g.status = device_status_ptr();
   if (!g.status) return SMARTMEM_ERR_CUDA;
-  dim3 grid((unsigned)((N + bn - 1) / bn), (unsigned)((M + BM - 1) / BM), (unsigned)batch);
-  if (grid.y > 65535) return SMARTMEM_ERR_UNSUPPORTED;
+  g.tiles_n = (int)((N + bn - 1) / bn);
+  g.tiles_m = (int)((M + BM - 1) / BM);
+  g.batch = (int)batch;
+  if ((long long)g.tiles_n * g.tiles_m * g.batch >= (1ll << 31)) return SMARTMEM_ERR_UNSUPPORTED;
 #define SM_CASE(BN_, ST_, MN_)                                                                  \
-  if (bn == BN_ && stages == ST_ && a_mn == MN_) return launch_t<BN_, ST_, MN_>(ta, tb, g, grid, st);
-  SM_CASE(256, 4, false) SM_CASE(256, 2, false) SM_CASE(128, 4, false) SM_CASE(128, 2, false)
-  SM_CASE(96, 4, false) SM_CASE(96, 2, false) SM_CASE(64, 4, false) SM_CASE(64, 2, false)
-  SM_CASE(256, 4, true) SM_CASE(128, 4, true) SM_CASE(256, 2, true) SM_CASE(128, 2, true)
+  if (bn == BN_ && stages == ST_ && a_mn == MN_) return launch_t<BN_, ST_, MN_>(ta, tb, g, st);
+  SM_CASE(256, 4, false) SM_CASE(128, 4, false) SM_CASE(96, 4, false) SM_CASE(64, 4, false)
+  SM_CASE(256, 4, true) SM_CASE(128, 4, true)
 #undef SM_CASE
   return SMARTMEM_ERR_UNSUPPORTED;
 }

@@ -1,0 +1,55 @@
+"""GPU parity of smartmem_attn_layer (RMSNorm, QKV, RoPE, causal attention, o_proj) against the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import llama as ollama
+from paper_2404_13528_b200 import binding as sm
+from paper_2404_13528_b200 import synth
+from tests.gpu_util import assert_close_bf16, check_status, stream, to_dev, to_host_f64
+
+pytestmark = pytest.mark.gpu
+
+
+def run_layer(dev, *, B, S, hidden, heads, add_residual, mode):
+    p = sm.AttnParams()
+    p.dtype, p.B, p.S, p.hidden, p.heads, p.head_dim, p.causal, p.add_residual = sm.BF16, B, S, hidden, heads, hidden // heads, 1, add_residual
+    p.rms_eps, p.rope_theta = 1e-5, 10000.0
+    p.rms_g, p.w_qkv, p.w_o = dev["rms_g"].data_ptr(), dev["w_qkv"].data_ptr(), dev["w_o"].data_ptr()
+    y = torch.full_like(dev["x"], float("nan"))
+    n = sm.smartmem_attn_layer_workspace_bytes(p, mode)
+    ws = torch.empty(n, dtype=torch.uint8, device="cuda")
+    sm.smartmem_attn_layer(p, dev["x"].data_ptr(), y.data_ptr(), ws.data_ptr(), n, mode, stream())
+    check_status()
+    return y
+
+
+def case(config_id, B, S, hidden, heads, add_residual):
+    inp = synth.attn_layer_inputs(config_id, S, hidden, B=B)
+    dev = {k: to_dev(v) for k, v in inp.items()}
+    pf = {k: synth.to_f64(v) for k, v in inp.items() if k != "x"}
+    ref = ollama.attn_layer(synth.to_f64(inp["x"]), pf, heads=heads, head_dim=hidden // heads, add_residual=bool(add_residual))
+    for mode in (sm.ELIMINATE, sm.EXPLICIT):
+        y = run_layer(dev, B=B, S=S, hidden=hidden, heads=heads, add_residual=add_residual, mode=mode)
+        assert_close_bf16(to_host_f64(y), ref, f"mode {mode}")
+
+
+@pytest.mark.parametrize("B,S,hidden,heads,res", [(1, 64, 256, 2, 0), (2, 200, 256, 2, 1), (1, 333, 512, 4, 0)])
+def test_small_attention_layers(B, S, hidden, heads, res):
+    case(30, B, S, hidden, heads, res)
+
+
+def test_config5_llama_style_layer_full_size():
+    """B=1, S=2048, hidden 4096, 32 heads x 128."""
+    case(5, 1, 2048, 4096, 32, 0)
+
+
+def test_attn_layer_rejects_bad_arguments():
+    inp = synth.attn_layer_inputs(31, 64, 256)
+    dev = {k: to_dev(v) for k, v in inp.items()}
+    with pytest.raises(sm.SmartmemError) as e:
+        run_layer(dev, B=1, S=64, hidden=256, heads=4, add_residual=0, mode=sm.ELIMINATE)     # head_dim 64
+    assert e.value.code == sm.ERR_UNSUPPORTED
+    with pytest.raises(sm.SmartmemError) as e:
+        run_layer(dev, B=1, S=64, hidden=256, heads=3, add_residual=0, mode=sm.ELIMINATE)
+    assert e.value.code == sm.ERR_SHAPE
