@@ -153,6 +153,183 @@ def run_reference(args):
     }))
 
 
+
+# ------------------------------------------------------------------------------------------------
+# The other configurations (parity-test cases): timed on request with --workload, same protocol.
+# ------------------------------------------------------------------------------------------------
+OTHER_WORKLOADS = ["swin_b_stage3_block_pair", "llama_attention_layer", "chain_2a_qkt", "chain_2b_gemm",
+                   "chain_2a_copy", "chain_2b_copy"]
+
+
+def _peaks_all():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), float(d["bf16_tflops"]), "measured (MEASURED_PEAKS.json; bf16 burst)"
+    return 6650.0, 1590.0, "fallback (earlier measurement on this pool)"
+
+
+def run_other(args):
+    """Times one of the other configurations: K steps per variant, per-kernel CUDA-event durations through
+    smartmem_profile_begin/_end, and the roofline position of every kernel of the ELIMINATE variant."""
+    import numpy as np
+    import torch
+    from paper_2404_13528_b200 import binding as sm
+    from paper_2404_13528_b200 import synth
+
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    stream = torch.cuda.current_stream().cuda_stream
+    name = args.workload
+
+    def dev(a):
+        return torch.from_numpy(a.view("int16").copy()).cuda().view(torch.bfloat16)
+
+    sets = 3
+    steps = {}
+    if name == "swin_b_stage3_block_pair":
+        B, H, W, C, heads, ws = 64, 14, 14, 512, 16, 7
+        M = B * H * W
+        U = M * C * 2
+        blocks = []
+        for wset, shift in ((0, 0), (1, 3)):
+            inp = synth.swin_inputs(4, B, H, W, C, heads, ws, 4, "bf16", weight_set=wset)
+            d = {k: dev(v) for k, v in inp.items()}
+            p = sm.SwinParams()
+            p.dtype = sm.BF16
+            p.B, p.H, p.W, p.C, p.heads, p.window, p.shift, p.mlp_ratio = B, H, W, C, heads, ws, shift, 4
+            p.ln_eps = 1e-5
+            for k, t in d.items():
+                if k != "x":
+                    setattr(p, k, t.data_ptr())
+            blocks.append((p, d))
+        xs = [blocks[0][1]["x"].clone() for _ in range(sets)]
+        mid = [torch.empty_like(xs[0]) for _ in range(sets)]
+        ys = [torch.empty_like(xs[0]) for _ in range(sets)]
+        wsb = {m: sm.smartmem_swin_block_workspace_bytes(blocks[0][0], m) for m in (sm.ELIMINATE, sm.EXPLICIT)}
+        wss = [torch.empty(wsb[sm.EXPLICIT], dtype=torch.uint8, device="cuda") for _ in range(sets)]
+
+        def step(i, mode):
+            j = i % sets
+            sm.smartmem_swin_block(blocks[0][0], xs[j].data_ptr(), mid[j].data_ptr(), wss[j].data_ptr(), wsb[mode], mode, stream)
+            sm.smartmem_swin_block(blocks[1][0], mid[j].data_ptr(), ys[j].data_ptr(), wss[j].data_ptr(), wsb[mode], mode, stream)
+        tokens = M
+        wq, wp, w1 = 3 * C * C * 2, C * C * 2, 4 * C * C * 2
+        one = [("ln1_gather", 2 * U, 0), ("qkv_gemm", 4 * U + wq, 2 * M * C * 3 * C), ("window_attention", 4 * U, 4 * M * 49 * C),
+               ("proj_gemm_scatter_residual", 3 * U + wp, 2 * M * C * C), ("ln2", 2 * U, 0),
+               ("fc1_gemm_gelu", 5 * U + w1, 2 * M * C * 4 * C), ("fc2_gemm_residual", 6 * U + w1, 2 * M * C * 4 * C)]
+        model = one + one
+    elif name == "llama_attention_layer":
+        S, hidden, heads = 2048, 4096, 32
+        inp = synth.attn_layer_inputs(5, S, hidden)
+        d = {k: dev(v) for k, v in inp.items()}
+        p = sm.AttnParams()
+        p.dtype, p.B, p.S, p.hidden, p.heads, p.head_dim, p.causal, p.add_residual = sm.BF16, 1, S, hidden, heads, 128, 1, 0
+        p.rms_eps, p.rope_theta = 1e-5, 10000.0
+        p.rms_g, p.w_qkv, p.w_o = d["rms_g"].data_ptr(), d["w_qkv"].data_ptr(), d["w_o"].data_ptr()
+        xs = [d["x"].clone() for _ in range(sets)]
+        ys = [torch.empty_like(xs[0]) for _ in range(sets)]
+        wsb = {m: sm.smartmem_attn_layer_workspace_bytes(p, m) for m in (sm.ELIMINATE, sm.EXPLICIT)}
+        wss = [torch.empty(wsb[sm.EXPLICIT], dtype=torch.uint8, device="cuda") for _ in range(sets)]
+
+        def step(i, mode):
+            j = i % sets
+            sm.smartmem_attn_layer(p, xs[j].data_ptr(), ys[j].data_ptr(), wss[j].data_ptr(), wsb[mode], mode, stream)
+        tokens = S
+        X = S * hidden * 2
+        model = [("rope_table", S * 64 * 8, 0), ("rmsnorm", 2 * X, 0), ("qkv_gemm_rope", 4 * X + 3 * hidden * hidden * 2, 2 * S * hidden * 3 * hidden),
+                 ("causal_attention", 4 * X, 4 * heads * 128 * S * (S + 1) // 2), ("o_proj_gemm", 2 * X + hidden * hidden * 2, 2 * S * hidden * hidden)]
+    else:
+        which = "2a" if "2a" in name else "2b"
+        inp = synth.chain_inputs(2, which)
+        if which == "2a":
+            B, S, Hh, D = inp["dims"]
+            layout = [sm.make_op(sm.OP_RESHAPE, shape=(B, S, Hh, D)), sm.make_op(sm.OP_TRANSPOSE, perm=(0, 2, 1, 3))]
+            srcs = [dev(inp["xq"]), dev(inp["xk"])]
+            descs = [sm.make_desc((B, S, Hh * D)), sm.make_desc((B, S, Hh * D))]
+            if name.endswith("copy"):
+                ops, oshape, srcs, descs = layout + [sm.make_op(sm.OP_COPY)], (B, Hh, S, D), srcs[:1], descs[:1]
+                model = [("copy_map", 2 * B * S * Hh * D * 2, 0)]
+            else:
+                ops, oshape = layout + [sm.make_op(sm.OP_BMM_NT, side_input=(1, 0))], (B, Hh, S, S)
+                model = [("qkt_gemm", 2 * B * S * Hh * D * 2 + B * Hh * S * S * 2, 2 * B * Hh * S * S * D)]
+            tokens = B * S
+        else:
+            B, C, Hh, Ww, N = inp["dims"]
+            layout = [sm.make_op(sm.OP_TRANSPOSE, perm=(0, 2, 3, 1)), sm.make_op(sm.OP_RESHAPE, shape=(B, Hh * Ww, C))]
+            srcs = [dev(inp["x"]), dev(inp["w"])]
+            descs = [sm.make_desc((B, C, Hh, Ww)), sm.make_desc((N, C))]
+            if name.endswith("copy"):
+                ops, oshape, srcs, descs = layout + [sm.make_op(sm.OP_COPY)], (B, Hh * Ww, C), srcs[:1], descs[:1]
+                model = [("copy_map", 2 * B * C * Hh * Ww * 2, 0)]
+            else:
+                ops, oshape = layout + [sm.make_op(sm.OP_LINEAR, side_input=(1, 0))], (B, Hh * Ww, N)
+                model = [("gemm_mn_major_operand", B * C * Hh * Ww * 2 + N * C * 2 + B * Hh * Ww * N * 2, 2 * B * Hh * Ww * N * C)]
+            tokens = B * Hh * Ww
+        sets = 8
+        plans = {m: sm.smartmem_plan(ops, descs, m) for m in (sm.ELIMINATE, sm.EXPLICIT)}
+        wsb = {m: sm.smartmem_plan_workspace_bytes(plans[m]) for m in plans}
+        ins = [[t.clone() for t in srcs] for _ in range(sets)]
+        outs = [torch.empty(oshape, dtype=torch.bfloat16, device="cuda") for _ in range(sets)]
+        wss = [torch.empty(max(wsb[sm.EXPLICIT], 16), dtype=torch.uint8, device="cuda") for _ in range(sets)]
+
+        def step(i, mode):
+            j = i % sets
+            sm.smartmem_run_chain(plans[mode], [t.data_ptr() for t in ins[j]], [outs[j].data_ptr()], wss[j].data_ptr(), wsb[mode], stream)
+
+    def timed(mode, k):
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(k):
+            step(i, mode)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1)
+
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    for i in range(args.warmup):
+        step(i, sm.ELIMINATE)
+        step(i, sm.EXPLICIT)
+    ms = {m: timed(m, args.steps) for m in (sm.ELIMINATE, sm.EXPLICIT)}
+    per = {}
+    for mode, tag in ((sm.ELIMINATE, "eliminate"), (sm.EXPLICIT, "explicit")):
+        acc = None
+        reps = min(args.steps, 20)
+        for i in range(reps):
+            sm.smartmem_profile_begin()
+            step(i, mode)
+            r = sm.smartmem_profile_end(stream)
+            acc = [[n, [t]] for n, t in r] if acc is None else [[a[0], a[1] + [t]] for a, (n, t) in zip(acc, r)]
+        per[tag] = [(n, statistics.median(v)) for n, v in acc]
+    clocks = sampler.stop()
+    st = sm.smartmem_last_device_status(stream)
+    if st != sm.OK:
+        raise SystemExit(f"device status {st}")
+    hbm, tf, src = _peaks_all()
+    kern = []
+    for (label, nbytes, flops), (kname, t) in zip(model, per["eliminate"]):
+        t_s = t * 1e-3
+        bound = "tensor" if flops / (tf * 1e12) > nbytes / (hbm * 1e9) else "hbm"
+        ach = flops / t_s / 1e12 if bound == "tensor" else nbytes / t_s / 1e9
+        kern.append({"kernel": label, "launched_as": kname, "ms": round(t, 5), "bound": bound, "achieved": round(ach, 1),
+                     "unit": "TFLOP/s" if bound == "tensor" else "GB/s", "frac": round(ach / (tf if bound == "tensor" else hbm), 4)})
+    dom = max(kern, key=lambda k: k["ms"])
+    print(json.dumps({
+        "metric": name + "_tokens_per_s", "value": tokens * args.steps / (ms[sm.ELIMINATE] * 1e-3), "unit": UNIT, "n_gpus": 1,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms[sm.ELIMINATE] / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": name, "mode": "eliminate", "l2": f"{sets} rotating buffer sets"},
+        "explicit_variant": {"ms_per_step": ms[sm.EXPLICIT] / args.steps, "speedup_of_eliminate": ms[sm.EXPLICIT] / ms[sm.ELIMINATE],
+                             "kernels": [{"launched_as": n, "ms": round(t, 5)} for n, t in per["explicit"]]},
+        "clocks": clocks,
+        "roofline": {"bound": dom["bound"], "kernel": dom["kernel"], "achieved": dom["achieved"], "unit": dom["unit"],
+                     "peak": tf if dom["bound"] == "tensor" else hbm, "frac": dom["frac"], "traffic": None, "peak_source": src},
+        "kernels": kern,
+    }))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -160,10 +337,14 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="smartmem", choices=["smartmem", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default=WORKLOAD["name"],
+                    help="swin_t_stage1_block (default, the benchmark line) or one of: " + ", ".join(OTHER_WORKLOADS))
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
     args.warmup = max(args.warmup, 3)
+    if args.workload != WORKLOAD["name"]:
+        return run_other(args)
 
     import torch
     from paper_2404_13528_b200 import binding as sm

@@ -189,6 +189,15 @@ int smartmem_swin_block_timed(const smartmem_swin_params_t* p, const void* x, vo
                               char* kernel_names, int32_t names_stride, int32_t max_kernels,
                               int32_t* n_kernels);
 
+/* Measurement aid for any entry point (no counterpart in the paper): between smartmem_profile_begin()
+ * and smartmem_profile_end() every kernel launch of the library is preceded by a CUDA event on
+ * its stream.  _end records a last event on `cuda_stream`, synchronises it and writes each
+ * kernel's duration (ms) and label as smartmem_swin_block_timed does.  Not thread-safe against
+ * concurrent launches from other host threads; meant for benchmarks. */
+int smartmem_profile_begin(void);
+int smartmem_profile_end(void* cuda_stream, float* kernel_ms, char* kernel_names, int32_t names_stride,
+                         int32_t max_kernels, int32_t* n_kernels);
+
 /* The Swin block for callers that cannot allocate device memory (the paper has no counterpart;
  * this is a deployment aid).  Typical callers: a step that runs while the process's device
  * memory pool is frozen (everything committed to caches and activations, so a cudaMalloc would

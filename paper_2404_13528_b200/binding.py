@@ -61,7 +61,7 @@ EXPORTED = [
     "smartmem_plan_workspace_bytes", "smartmem_map_eval", "smartmem_plan_eval_sequential", "smartmem_run_chain",
     "smartmem_swin_block_workspace_bytes", "smartmem_swin_block", "smartmem_attn_layer_workspace_bytes",
     "smartmem_attn_layer", "smartmem_swin_block_timed", "smartmem_swin_block_static_scratch_bytes",
-    "smartmem_swin_block_noalloc", "smartmem_last_device_status", "smartmem_launch_count", "smartmem_status_string",
+    "smartmem_swin_block_noalloc", "smartmem_profile_begin", "smartmem_profile_end", "smartmem_last_device_status", "smartmem_launch_count", "smartmem_status_string",
 ]
 
 _lib = None
@@ -98,6 +98,8 @@ def lib() -> C.CDLL:
         "smartmem_swin_block_noalloc": (C.c_int, [P(SwinParams), vp, vp, i32, vp]),
         "smartmem_attn_layer_workspace_bytes": (C.c_int, [P(AttnParams), i32, P(C.c_size_t)]),
         "smartmem_attn_layer": (C.c_int, [P(AttnParams), vp, vp, vp, C.c_size_t, i32, vp]),
+        "smartmem_profile_begin": (C.c_int, []),
+        "smartmem_profile_end": (C.c_int, [vp, P(C.c_float), C.c_char_p, i32, i32, P(i32)]),
         "smartmem_last_device_status": (C.c_int, [vp, P(i32)]),
         "smartmem_launch_count": (i64, []),
         "smartmem_status_string": (C.c_char_p, [i32]),
@@ -263,6 +265,21 @@ def smartmem_attn_layer_workspace_bytes(p: AttnParams, mode: int) -> int:
 
 def smartmem_attn_layer(p: AttnParams, x: int, y: int, workspace: int, workspace_bytes: int, mode: int, stream: int):
     _check(lib().smartmem_attn_layer(C.byref(p), x, y, workspace, workspace_bytes, mode, stream), "smartmem_attn_layer")
+
+
+def smartmem_profile_begin():
+    _check(lib().smartmem_profile_begin(), "smartmem_profile_begin")
+
+
+def smartmem_profile_end(stream: int):
+    """Returns [(label, milliseconds), ...] for every kernel launched since smartmem_profile_begin()."""
+    maxk, stride = 256, 32
+    ms = (C.c_float * maxk)()
+    names = C.create_string_buffer(maxk * stride)
+    n = C.c_int32()
+    _check(lib().smartmem_profile_end(stream, ms, names, stride, maxk, C.byref(n)), "smartmem_profile_end")
+    raw = names.raw
+    return [(raw[i * stride:(i + 1) * stride].split(b"\0", 1)[0].decode(), float(ms[i])) for i in range(n.value)]
 
 
 def smartmem_last_device_status(stream: int) -> int:

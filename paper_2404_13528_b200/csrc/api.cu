@@ -14,6 +14,20 @@ namespace smartmem {
 static std::atomic<long long> g_launches{0};
 void count_launch(int n) { g_launches += n; }
 
+static std::mutex g_prof_mu;
+static bool g_prof_on = false;
+static std::vector<cudaEvent_t> g_prof_ev;
+static std::vector<const char*> g_prof_names;
+void profile_tick(const char* name, cudaStream_t st) {
+  if (!g_prof_on) return;
+  std::lock_guard<std::mutex> lk(g_prof_mu);
+  cudaEvent_t e;
+  if (cudaEventCreate(&e) != cudaSuccess) return;
+  cudaEventRecord(e, st);
+  g_prof_ev.push_back(e);
+  g_prof_names.push_back(name);
+}
+
 __device__ int g_status_word;
 
 int* device_status_ptr() {
@@ -32,6 +46,40 @@ int* device_status_ptr() {
 }  // namespace smartmem
 
 using namespace smartmem;
+
+EXPORT int smartmem_profile_begin(void) {
+  std::lock_guard<std::mutex> lk(g_prof_mu);
+  for (cudaEvent_t e : g_prof_ev) cudaEventDestroy(e);
+  g_prof_ev.clear();
+  g_prof_names.clear();
+  g_prof_on = true;
+  return SMARTMEM_OK;
+}
+
+EXPORT int smartmem_profile_end(void* cuda_stream, float* kernel_ms, char* kernel_names, int32_t names_stride,
+                                int32_t max_kernels, int32_t* n_kernels) {
+  if (!kernel_ms || !kernel_names || !n_kernels || max_kernels < 1 || names_stride < 8) return SMARTMEM_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  profile_tick("end", st);
+  std::lock_guard<std::mutex> lk(g_prof_mu);
+  g_prof_on = false;
+  int rs = cudaStreamSynchronize(st) == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
+  int n = 0;
+  for (size_t i = 0; i + 1 < g_prof_ev.size() && n < max_kernels; ++i, ++n) {
+    float ms = 0.f;
+    if (rs == SMARTMEM_OK) cudaEventElapsedTime(&ms, g_prof_ev[i], g_prof_ev[i + 1]);
+    kernel_ms[n] = ms;
+    const char* nm = g_prof_names[i];
+    int k = 0;
+    while (nm[k] && k < names_stride - 1) { kernel_names[n * names_stride + k] = nm[k]; ++k; }
+    kernel_names[n * names_stride + k] = 0;
+  }
+  for (cudaEvent_t e : g_prof_ev) cudaEventDestroy(e);
+  g_prof_ev.clear();
+  g_prof_names.clear();
+  *n_kernels = n;
+  return rs;
+}
 
 EXPORT int64_t smartmem_launch_count(void) { return g_launches.load(); }
 

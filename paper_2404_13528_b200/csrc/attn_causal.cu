@@ -216,6 +216,7 @@ int launch_causal_attention(const CausalAttnArgs& a, cudaStream_t st) {
       return SMARTMEM_ERR_CUDA;
     configured = true;
   }
+  profile_tick("causal_attention", st);
   dim3 grid((a.S + BMQ - 1) / BMQ, a.heads, a.batch);
   causal_attn_kernel<<<grid, 128, smem, st>>>(a);
   count_launch();
@@ -224,6 +225,7 @@ int launch_causal_attention(const CausalAttnArgs& a, cudaStream_t st) {
 
 int launch_rope_table(float* tab, int S, int head_dim, float theta, cudaStream_t st) {
   const int n = S * (head_dim / 2);
+  profile_tick("rope_table", st);
   rope_table_kernel<<<(n + 255) / 256, 256, 0, st>>>((float2*)tab, S, head_dim / 2, (double)theta);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
@@ -231,6 +233,7 @@ int launch_rope_table(float* tab, int S, int head_dim, float theta, cudaStream_t
 
 int launch_rope_rows(void* x, long long rows, int S, int head_dim, const float* tab, cudaStream_t st) {
   const long long n = rows * (head_dim / 2);
+  profile_tick("rope_rows", st);
   rope_rows_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>((__nv_bfloat16*)x, rows, S, head_dim, (const float2*)tab);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;

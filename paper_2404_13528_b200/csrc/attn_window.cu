@@ -269,6 +269,7 @@ int launch_window_attention(const WinAttnArgs& a, int dtype, long long n_windows
   if (a.T < 1 || a.T > TP || a.ws * a.ws != a.T || (2 * a.ws - 1) * (2 * a.ws - 1) > 256) return SMARTMEM_ERR_UNSUPPORTED;
   long long units = n_windows * a.heads;
   if (units < 1 || units >= (1ll << 31)) return SMARTMEM_ERR_UNSUPPORTED;
+  profile_tick("window_attention", st);
   if (dtype == SMARTMEM_F32) {
     if (a.d > 32) return SMARTMEM_ERR_UNSUPPORTED;
     win_attn_f32_kernel<<<(unsigned)units, 128, 0, st>>>(a);

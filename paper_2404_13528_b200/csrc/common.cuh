@@ -13,6 +13,9 @@ namespace smartmem {
 // ---------------------------------------------------------------------------------------
 int* device_status_ptr();                 // device address of the status word (per process)
 void count_launch(int n = 1);
+// When a profiling session is open (smartmem_profile_begin), records a CUDA event on `st` labelled
+// `name`; every launcher calls it right before its kernel launch.
+void profile_tick(const char* name, cudaStream_t st);
 
 // ---------------------------------------------------------------------------------------
 // Division by a run-time constant without a divide instruction: q = umulhi(n, mul) >> shr
@@ -137,9 +140,5 @@ int launch_copy_map(const smartmem_index_map_t& map, int elem_size, const void* 
 // read from src at element offset rowmap(r) (rowmap == nullptr: r * C).
 int launch_norm(int dtype, bool rms, const void* src, void* dst, const void* gamma, const void* beta, float eps,
                 long long rows, int C, const DevMap* rowmap, cudaStream_t st);
-
-// Elementwise helpers of the EXPLICIT path.
-int launch_rope_inplace(void* qk, long long rows, int row_stride, int heads2, int head_dim, float theta, int S,
-                        cudaStream_t st);
 
 }  // namespace smartmem

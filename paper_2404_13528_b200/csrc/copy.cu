@@ -152,6 +152,7 @@ __global__ void __launch_bounds__(256) copy_block_transpose16_kernel(const __gri
 }  // namespace
 
 int launch_copy_map(const smartmem_index_map_t& map, int elem_size, const void* src, void* dst, cudaStream_t st) {
+  profile_tick("copy_map", st);
   if (map.klass == 3) return SMARTMEM_ERR_UNSUPPORTED;
   if (map.n_elements == 0) return SMARTMEM_OK;
   const int n = map.n_atoms;

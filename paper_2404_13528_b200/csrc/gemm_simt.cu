@@ -37,6 +37,7 @@ int launch_gemm_simt_f32(const SimtGemmArgs& a, cudaStream_t st) {
   if (a.M < 1 || a.N < 1 || a.K < 1) return SMARTMEM_ERR_UNSUPPORTED;
   dim3 grid((a.N + 15) / 16, (a.M + 15) / 16);
   if (grid.y > 65535) return SMARTMEM_ERR_UNSUPPORTED;
+  profile_tick("gemm_simt_f32", st);
   gemm_simt_f32_kernel<<<grid, 256, 0, st>>>(a);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;

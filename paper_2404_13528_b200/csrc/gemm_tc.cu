@@ -448,6 +448,7 @@ int launch_t(const CUtensorMap& ta, const CUtensorMap& tb, const GemmArgs& g, cu
       return SMARTMEM_ERR_CUDA;
     configured = true;
   }
+  profile_tick("gemm_tc", st);
   const long long tiles = (long long)g.tiles_n * g.tiles_m * g.batch;
   const unsigned grid = (unsigned)(tiles < sm_count() ? tiles : sm_count());
   gemm_tc_kernel<BN, STAGES, A_MN><<<grid, kThreads, smem, st>>>(ta, tb, g);

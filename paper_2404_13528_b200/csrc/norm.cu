@@ -141,6 +141,7 @@ int launch_norm_t(const void* src, void* dst, const void* gamma, const void* bet
 
 int launch_norm(int dtype, bool rms, const void* src, void* dst, const void* gamma, const void* beta, float eps,
                 long long rows, int C, const DevMap* rowmap, cudaStream_t st) {
+  profile_tick(rms ? "rmsnorm" : "layernorm", st);
   if (rows == 0) return SMARTMEM_OK;
   if (dtype == SMARTMEM_F32)
     return rms ? launch_norm_t<float, true>(src, dst, gamma, beta, eps, rows, C, rowmap, st)
