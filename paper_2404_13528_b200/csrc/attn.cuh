@@ -15,6 +15,7 @@ struct WinAttnArgs {
   const void* table;        // [(2ws-1)^2, heads]
   int table_f32;
   int heads, T, ws, d, shift, H, W, nWw, win_per_img;
+  int n_windows;            // set by the launcher
   float scale;
 };
 int launch_window_attention(const WinAttnArgs& a, int dtype, long long n_windows, cudaStream_t st);

@@ -95,7 +95,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   constexpr uint32_t ACC_COLS = BN <= 32 ? 32 : BN <= 64 ? 64 : BN <= 128 ? 128 : 256;   // one accumulator buffer
   constexpr uint32_t TMEM_COLS = 2 * ACC_COLS;
   constexpr uint32_t IDESC = ptx::make_idesc_bf16(BM, BN, A_MN, false);
-  constexpr int NSUB = BN / 16;                              // 16-column sub-chunks per tile
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -107,6 +106,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   uint64_t* tmem_empty = tmem_full + 2;                      // [2]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_empty + 2);
   int* abort_flag = reinterpret_cast<int*>(tmem_slot + 1);
+  uint8_t* stage_base = reinterpret_cast<uint8_t*>(tmem_slot + 4);                      // 16-byte aligned
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nkb = (g.K + BK - 1) / BK;
@@ -203,9 +203,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       }
     }
   } else {
+    // Epilogue.  Warp (quadrant q, column group grp) owns rows q*32..q*32+31 (one TMEM lane per
+    // thread) and CG = BN/4 columns, handled in rounds of RC <= 32 columns:
+    //   phase 1 (thread = row): TMEM -> fp32 -> [RoPE] -> +bias -> [GELU] -> [+residual] -> bf16 -> staging row
+    //   phase 2 (threads spread along the row): 16-byte stores, RC*2 contiguous bytes per row,
+    // so a store instruction writes whole 32-byte sectors and several sectors of one line at once.
+    constexpr int CG = BN / 4;
+    constexpr int RC = (BN == 256 && STAGES == 4) ? 16 : (CG > 32 ? 32 : CG);   // 4 stages leave less staging room
+    constexpr int ROUNDS = CG / RC;
+    constexpr int RH = ROUNDS > 1 ? ROUNDS / 2 : 1;          // BN == 256: rounds [0, RH) hold the first halves of rotary pairs
+    constexpr int VPR = RC / 8;                              // 16-byte vectors per row per round
+    constexpr int STG_ROW = RC * 2 + 16;                     // bytes; the pad keeps phase 1 conflict-free
     const int e = warp - 2;
     const int q = warp & 3;                                  // TMEM lane quadrant this warp may read
-    const int grp = e >> 2;                                  // which sub-chunks (sub % 4 == grp)
+    const int grp = e >> 2;
+    uint8_t* stage = stage_base + e * (32 * STG_ROW);
     uint32_t it = 0;
     bool ok = true;
     for (uint32_t t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
@@ -217,98 +229,105 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       long long off = 0;
       if (row_ok) off = g.has_rowmap ? devmap_eval(g.rowmap, (uint32_t)row) : (long long)row * g.ldc;
       off += (long long)batch * g.out_batch_stride;
-      __nv_bfloat16* __restrict__ orow = g.out + off;
       const __nv_bfloat16* __restrict__ rrow = g.residual ? g.residual + off : nullptr;
+      const bool rope_tile = BN == 256 && g.rope_cols > 0 && n0 < g.rope_cols;
+      auto col_of = [&](int rd) {
+        return BN == 256 ? 128 * (grp >> 1) + 32 * (grp & 1) + RC * (rd % RH) + 64 * (rd / RH) : grp * CG;
+      };
 
-      // residual of the first sub-chunk is fetched while the MMAs of this tile still run
-      uint4 res[2] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
+      uint4 res[VPR];
       auto fetch_res = [&](int c0) {
-        if (rrow && row_ok && n0 + c0 + 16 <= g.N) {
-          res[0] = *reinterpret_cast<const uint4*>(rrow + n0 + c0);
-          res[1] = *reinterpret_cast<const uint4*>(rrow + n0 + c0 + 8);
+#pragma unroll
+        for (int v = 0; v < VPR; ++v) {
+          res[v] = make_uint4(0, 0, 0, 0);
+          if (rrow && row_ok && n0 + c0 + v * 8 + 8 <= g.N) res[v] = *reinterpret_cast<const uint4*>(rrow + n0 + c0 + v * 8);
         }
       };
-      const bool rope_tile = g.rope_cols > 0 && n0 < g.rope_cols;
-      if (!rope_tile) fetch_res(grp * 16);
+      fetch_res(col_of(0));                                  // in flight while this tile's MMAs still run
 
       ok = ptx::mbar_wait(&tmem_full[buf], use & 1, abort_flag, g.status);
       if (!ok) break;
       ptx::tc_fence_after();
       const uint32_t taddr = tmem_base + buf * ACC_COLS + ((uint32_t)(q * 32) << 16);
 
-      auto finish = [&](float* acc, int c0, const uint4* rv) {    // bias / GELU / residual / store of 16 columns
-        const int col0 = n0 + c0;
-        if (!row_ok || col0 >= g.N) return;
-        if (col0 + 16 <= g.N) {
-          if (g.bias) {
 #pragma unroll
-            for (int v = 0; v < 2; ++v) {
-              float b[8];
-              ElemIO<__nv_bfloat16>::load(g.bias + col0 + v * 8, b);
+      for (int rd = 0; rd < ROUNDS; ++rd) {
+        const int c0 = col_of(rd);
+        float acc[RC];
+        {
+          uint32_t rv[RC];
+          ptx::tmem_ld_cols<RC>(taddr + c0, rv);
+          if (rope_tile) {
+            // rotary pairs are (c, c + 64) inside a 128-column head: round 0 holds the first half
+            // of the pair, round 1 the second; each round reads both halves from TMEM
+            uint32_t rw[RC];
+            ptx::tmem_ld_cols<RC>(taddr + (rd < RH ? c0 + 64 : c0 - 64), rw);
+            ptx::tmem_ld_wait();
+            // this thread's RC (cos, sin) pairs are contiguous: 16-byte loads, whole sectors used
+            const float4* tab4 = reinterpret_cast<const float4*>(g.rope_tab + (long long)(row_ok ? row % g.rope_S : 0) * 64 +
+                                                                 (grp & 1) * 32 + RC * (rd % RH));
 #pragma unroll
-              for (int j = 0; j < 8; ++j) acc[v * 8 + j] += b[j];
+            for (int j = 0; j < RC; j += 2) {
+              const float4 cs = __ldg(tab4 + j / 2);
+              const float x0 = __uint_as_float(rv[j]), y0 = __uint_as_float(rw[j]);
+              const float x1 = __uint_as_float(rv[j + 1]), y1 = __uint_as_float(rw[j + 1]);
+              acc[j] = rd < RH ? x0 * cs.x - y0 * cs.y : x0 * cs.x + y0 * cs.y;
+              acc[j + 1] = rd < RH ? x1 * cs.z - y1 * cs.w : x1 * cs.z + y1 * cs.w;
             }
-          }
-          if (g.gelu) {
+          } else {
+            ptx::tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 16; ++j) acc[j] = gelu_fast(acc[j]);
-          }
-          if (rv) {
-#pragma unroll
-            for (int v = 0; v < 2; ++v) {
-              const uint32_t w[4] = {rv[v].x, rv[v].y, rv[v].z, rv[v].w};
-#pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                const float2 f = bf16x2_to_float2(w[j]);
-                acc[v * 8 + 2 * j] += f.x;
-                acc[v * 8 + 2 * j + 1] += f.y;
-              }
-            }
-          }
-          ElemIO<__nv_bfloat16>::store(orow + col0, acc);
-          ElemIO<__nv_bfloat16>::store(orow + col0 + 8, acc + 8);
-        } else {
-          for (int j = 0; j < 16 && col0 + j < g.N; ++j) {
-            float v = acc[j] + (g.bias ? __bfloat162float(g.bias[col0 + j]) : 0.f);
-            if (g.gelu) v = gelu_fast(v);
-            if (rrow) v += __bfloat162float(rrow[col0 + j]);
-            orow[col0 + j] = __float2bfloat16_rn(v);
+            for (int j = 0; j < RC; ++j) acc[j] = __uint_as_float(rv[j]);
           }
         }
-      };
-
-      for (int sub = grp; sub < NSUB; sub += 4) {
-        const int c0 = sub * 16;
-        if (rope_tile && n0 + c0 < g.rope_cols) {
-          // rotary pairs are (c, c + 64) inside a 128-column head: sub-chunks sub and sub + 4
-          if ((sub & 7) >= 4) continue;
-          uint32_t ra[16], rb[16];
-          ptx::tmem_ld16(taddr + c0, ra);
-          ptx::tmem_ld16(taddr + c0 + 64, rb);
-          ptx::tmem_ld_wait();
-          float x1[16], x2[16];
-          const float2* tab = g.rope_tab + (long long)(row_ok ? row % g.rope_S : 0) * 64 + (sub & 3) * 16;
+        if (g.bias) {
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const float2 cs = tab[j];
-            const float a = __uint_as_float(ra[j]), b = __uint_as_float(rb[j]);
-            x1[j] = a * cs.x - b * cs.y;
-            x2[j] = b * cs.x + a * cs.y;
+          for (int v = 0; v < VPR; ++v) {
+            if (n0 + c0 + v * 8 + 8 <= g.N) {
+              float bb[8];
+              ElemIO<__nv_bfloat16>::load(g.bias + n0 + c0 + v * 8, bb);
+#pragma unroll
+              for (int j = 0; j < 8; ++j) acc[v * 8 + j] += bb[j];
+            }
           }
-          finish(x1, c0, nullptr);
-          finish(x2, c0 + 64, nullptr);
-        } else {
-          uint32_t rv[16];
-          ptx::tmem_ld16(taddr + c0, rv);
-          ptx::tmem_ld_wait();
-          float acc[16];
-#pragma unroll
-          for (int j = 0; j < 16; ++j) acc[j] = __uint_as_float(rv[j]);
-          const bool vec_res = rrow && n0 + c0 + 16 <= g.N;
-          uint4 cur[2] = {res[0], res[1]};
-          if (sub + 4 < NSUB) fetch_res(c0 + 64);              // next sub-chunk's residual in flight
-          finish(acc, c0, vec_res ? cur : nullptr);
         }
+        if (g.gelu) {
+#pragma unroll
+          for (int j = 0; j < RC; ++j) acc[j] = gelu_fast(acc[j]);
+        }
+        if (rrow) {
+#pragma unroll
+          for (int v = 0; v < VPR; ++v) {
+            const uint32_t w[4] = {res[v].x, res[v].y, res[v].z, res[v].w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const float2 f = bf16x2_to_float2(w[j]);
+              acc[v * 8 + 2 * j] += f.x;
+              acc[v * 8 + 2 * j + 1] += f.y;
+            }
+          }
+          if (rd + 1 < ROUNDS) fetch_res(col_of(rd + 1));
+        }
+#pragma unroll
+        for (int v = 0; v < VPR; ++v) {
+          uint4 pk;
+          pk.x = float2_to_bf16x2(acc[v * 8 + 0], acc[v * 8 + 1]);
+          pk.y = float2_to_bf16x2(acc[v * 8 + 2], acc[v * 8 + 3]);
+          pk.z = float2_to_bf16x2(acc[v * 8 + 4], acc[v * 8 + 5]);
+          pk.w = float2_to_bf16x2(acc[v * 8 + 6], acc[v * 8 + 7]);
+          *reinterpret_cast<uint4*>(stage + lane * STG_ROW + v * 16) = pk;
+        }
+        __syncwarp();
+#pragma unroll
+        for (int i = 0; i < VPR; ++i) {
+          const int v = lane + 32 * i;
+          const int rr = v / VPR, seg = v - rr * VPR;
+          const long long roff = __shfl_sync(0xFFFFFFFFu, off, rr);
+          const int rok = __shfl_sync(0xFFFFFFFFu, (int)row_ok, rr);
+          const uint4 pk = *reinterpret_cast<const uint4*>(stage + rr * STG_ROW + seg * 16);
+          if (rok && n0 + c0 + seg * 8 + 8 <= g.N) *reinterpret_cast<uint4*>(g.out + roff + n0 + c0 + seg * 8) = pk;
+        }
+        __syncwarp();
       }
       // all of this warp's TMEM reads of the buffer have completed (wait::ld above)
       ptx::tc_fence_before();
@@ -440,7 +459,9 @@ int sm_count() {
 
 template <int BN, int STAGES, bool A_MN>
 int launch_t(const CUtensorMap& ta, const CUtensorMap& tb, const GemmArgs& g, cudaStream_t st) {
-  constexpr size_t smem = 1024 + STAGES * (A_STAGE_BYTES + BN * BK * 2) + (2 * STAGES + 4) * 8 + 16;
+  constexpr int RCc = (BN == 256 && STAGES == 4) ? 16 : ((BN / 4) > 32 ? 32 : (BN / 4));
+  constexpr size_t smem = 1024 + STAGES * (A_STAGE_BYTES + BN * BK * 2) + (2 * STAGES + 4) * 8 + 16 +
+                          kEpiWarps * 32 * (RCc * 2 + 16);
   static bool configured = false;
   if (!configured) {
     if (cudaFuncSetAttribute(gemm_tc_kernel<BN, STAGES, A_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
@@ -497,7 +518,10 @@ int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep,
   if (M < 1 || N < 1 || K < 1 || batch < 1 ||  M >= (1ll << 31) || N >= (1ll << 31))
     return SMARTMEM_ERR_UNSUPPORTED;
   if (A.K != K || B.K != K) return SMARTMEM_ERR_SHAPE;
-  if (((uintptr_t)ep.out & 15) || ((uintptr_t)ep.residual & 15) || ep.ldc % 8) return SMARTMEM_ERR_ALIGNMENT;
+  if (((uintptr_t)ep.out & 15) || ((uintptr_t)ep.residual & 15) || ((uintptr_t)ep.bias & 15) || ep.ldc % 8 ||
+      ep.out_batch_stride % 8)
+    return SMARTMEM_ERR_ALIGNMENT;
+  if (N % 8) return SMARTMEM_ERR_UNSUPPORTED;
   const bool a_mn = A.k_stride != 1;
   if (B.k_stride != 1) return SMARTMEM_ERR_UNSUPPORTED;
   // tile width: the widest of {256, 128, 96, 64} that divides N (fewest wasted columns), else 128
@@ -509,7 +533,7 @@ int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep,
   else if (N % 64 == 0) bn = 64;
   if (ep.rope_cols > 0 && (N % 256 || ep.rope_cols % 256 || !ep.rope_tab || ep.rope_S < 1)) return SMARTMEM_ERR_UNSUPPORTED;
   const int nkb = (int)((K + BK - 1) / BK);
-  const int stages = 4;
+  const int stages = (bn == 256 && nkb <= 3) ? 3 : 4;   // short K: wider store rounds instead of a 4th stage
   GemmArgs g;
   memset(&g, 0, sizeof(g));
   CUtensorMap ta, tb;
@@ -537,8 +561,8 @@ int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep,
   if ((long long)g.tiles_n * g.tiles_m * g.batch >= (1ll << 31)) return SMARTMEM_ERR_UNSUPPORTED;
 #define SM_CASE(BN_, ST_, MN_)                                                                  \
   if (bn == BN_ && stages == ST_ && a_mn == MN_) return launch_t<BN_, ST_, MN_>(ta, tb, g, st);
-  SM_CASE(256, 4, false) SM_CASE(128, 4, false) SM_CASE(96, 4, false) SM_CASE(64, 4, false)
-  SM_CASE(256, 4, true) SM_CASE(128, 4, true)
+  SM_CASE(256, 3, false) SM_CASE(256, 4, false) SM_CASE(128, 4, false) SM_CASE(96, 4, false) SM_CASE(64, 4, false)
+  SM_CASE(256, 3, true) SM_CASE(256, 4, true) SM_CASE(128, 4, true)
 #undef SM_CASE
   return SMARTMEM_ERR_UNSUPPORTED;
 }

@@ -16,90 +16,123 @@ __device__ __forceinline__ float group_sum(float v) {
 }
 
 // LPR lanes cooperate on one row; VPL 16-byte vectors per lane are kept in registers
-// (VPL == 0: any row length, the row is re-read from L1/L2 for each pass).
-template <typename T, int LPR, int VPL, bool RMS>
+// (VPL == 0: any row length, the row is re-read from L1/L2 for each pass).  Each lane group
+// handles RPG rows at once so that RPG independent loads are in flight per lane.
+template <typename T, int LPR, int VPL, bool RMS, int RPG>
 __global__ void __launch_bounds__(256) norm_kernel(const T* __restrict__ src, T* __restrict__ dst,
                                                    const T* __restrict__ gamma, const T* __restrict__ beta, float eps,
                                                    long long rows, int C, const __grid_constant__ DevMap rowmap,
                                                    int has_map) {
   constexpr int KV = ElemIO<T>::kVec;
   constexpr int NV = VPL > 0 ? VPL : 1;
+  constexpr int GPB = 8 * (32 / LPR);                       // lane groups per block
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int sub = lane % LPR, rsub = lane / LPR;
-  const long long row = ((long long)blockIdx.x * 8 + warp) * (32 / LPR) + rsub;
-  const bool active = row < rows;
-  const long long soff = active ? (has_map ? devmap_eval(rowmap, (uint32_t)row) : row * (long long)C) : 0;
-  const T* s = src + soff;
+  const int sub = lane % LPR, grp = warp * (32 / LPR) + lane / LPR;
+  const long long row0 = (long long)blockIdx.x * (GPB * RPG) + grp;
   const int nvec = C / KV;
   const float invC = 1.0f / (float)C;
-  float v[NV][KV];
-  float sum = 0.f;
-  if constexpr (VPL > 0) {
+  float v[RPG][NV][KV];
+  const T* s[RPG];
+  bool active[RPG];
+  float sum[RPG];
 #pragma unroll
-    for (int k = 0; k < VPL; ++k) {
-      const int vi = sub + k * LPR;
-      if (active && vi < nvec) {
-        ElemIO<T>::load(s + vi * KV, v[k]);
-      } else {
-#pragma unroll
-        for (int e = 0; e < KV; ++e) v[k][e] = 0.f;
-      }
-#pragma unroll
-      for (int e = 0; e < KV; ++e) sum += RMS ? v[k][e] * v[k][e] : v[k][e];
-    }
-  } else {
-    for (int vi = sub; vi < nvec && active; vi += LPR) {
-      ElemIO<T>::load(s + vi * KV, v[0]);
-#pragma unroll
-      for (int e = 0; e < KV; ++e) sum += RMS ? v[0][e] * v[0][e] : v[0][e];
-    }
+  for (int r = 0; r < RPG; ++r) {
+    const long long row = row0 + (long long)r * GPB;
+    active[r] = row < rows;
+    const long long soff = active[r] ? (has_map ? devmap_eval(rowmap, (uint32_t)row) : row * (long long)C) : 0;
+    s[r] = src + soff;
   }
-  sum = group_sum<LPR>(sum);
-  float mean = 0.f, rstd;
-  if constexpr (RMS) {
-    rstd = rsqrtf(sum * invC + eps);
-  } else {
-    mean = sum * invC;
-    float sq = 0.f;
+#pragma unroll
+  for (int r = 0; r < RPG; ++r) {
+    sum[r] = 0.f;
     if constexpr (VPL > 0) {
 #pragma unroll
       for (int k = 0; k < VPL; ++k) {
         const int vi = sub + k * LPR;
-        if (active && vi < nvec) {
+        if (active[r] && vi < nvec) {
+          ElemIO<T>::load(s[r] + vi * KV, v[r][k]);
+        } else {
 #pragma unroll
-          for (int e = 0; e < KV; ++e) sq += (v[k][e] - mean) * (v[k][e] - mean);
+          for (int e = 0; e < KV; ++e) v[r][k][e] = 0.f;
         }
       }
-    } else {
-      for (int vi = sub; vi < nvec && active; vi += LPR) {
-        ElemIO<T>::load(s + vi * KV, v[0]);
+    }
+  }
 #pragma unroll
-        for (int e = 0; e < KV; ++e) sq += (v[0][e] - mean) * (v[0][e] - mean);
+  for (int r = 0; r < RPG; ++r) {
+    if constexpr (VPL > 0) {
+#pragma unroll
+      for (int k = 0; k < VPL; ++k)
+#pragma unroll
+        for (int e = 0; e < KV; ++e) sum[r] += RMS ? v[r][k][e] * v[r][k][e] : v[r][k][e];
+    } else {
+      for (int vi = sub; vi < nvec && active[r]; vi += LPR) {
+        ElemIO<T>::load(s[r] + vi * KV, v[r][0]);
+#pragma unroll
+        for (int e = 0; e < KV; ++e) sum[r] += RMS ? v[r][0][e] * v[r][0][e] : v[r][0][e];
       }
     }
-    sq = group_sum<LPR>(sq);
-    rstd = rsqrtf(sq * invC + eps);
+    sum[r] = group_sum<LPR>(sum[r]);
   }
-  if (!active) return;
-  T* d = dst + row * (long long)C;
-  auto emit = [&](int vi, float* x) {
-    float g[KV], b[KV], y[KV];
-    ElemIO<T>::load(gamma + vi * KV, g);
-    if constexpr (!RMS) ElemIO<T>::load(beta + vi * KV, b);
+  float mean[RPG], rstd[RPG];
 #pragma unroll
-    for (int e = 0; e < KV; ++e) y[e] = RMS ? x[e] * rstd * g[e] : (x[e] - mean) * rstd * g[e] + b[e];
-    ElemIO<T>::store(d + vi * KV, y);
+  for (int r = 0; r < RPG; ++r) {
+    mean[r] = 0.f;
+    if constexpr (RMS) {
+      rstd[r] = rsqrtf(sum[r] * invC + eps);
+    } else {
+      mean[r] = sum[r] * invC;
+      float sq = 0.f;
+      if constexpr (VPL > 0) {
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) {
+          const int vi = sub + k * LPR;
+          if (active[r] && vi < nvec) {
+#pragma unroll
+            for (int e = 0; e < KV; ++e) sq += (v[r][k][e] - mean[r]) * (v[r][k][e] - mean[r]);
+          }
+        }
+      } else {
+        for (int vi = sub; vi < nvec && active[r]; vi += LPR) {
+          ElemIO<T>::load(s[r] + vi * KV, v[r][0]);
+#pragma unroll
+          for (int e = 0; e < KV; ++e) sq += (v[r][0][e] - mean[r]) * (v[r][0][e] - mean[r]);
+        }
+      }
+      sq = group_sum<LPR>(sq);
+      rstd[r] = rsqrtf(sq * invC + eps);
+    }
+  }
+  auto emit = [&](int r, int vi, float* x, const float* g, const float* b) {
+    float y[KV];
+#pragma unroll
+    for (int e = 0; e < KV; ++e) y[e] = RMS ? x[e] * rstd[r] * g[e] : (x[e] - mean[r]) * rstd[r] * g[e] + b[e];
+    ElemIO<T>::store(dst + (row0 + (long long)r * GPB) * (long long)C + vi * KV, y);
   };
   if constexpr (VPL > 0) {
 #pragma unroll
     for (int k = 0; k < VPL; ++k) {
       const int vi = sub + k * LPR;
-      if (vi < nvec) emit(vi, v[k]);
+      if (vi < nvec) {
+        float g[KV], b[KV];
+        ElemIO<T>::load(gamma + vi * KV, g);
+        if constexpr (!RMS) ElemIO<T>::load(beta + vi * KV, b);
+#pragma unroll
+        for (int r = 0; r < RPG; ++r)
+          if (active[r]) emit(r, vi, v[r][k], g, b);
+      }
     }
   } else {
     for (int vi = sub; vi < nvec; vi += LPR) {
-      ElemIO<T>::load(s + vi * KV, v[0]);
-      emit(vi, v[0]);
+      float g[KV], b[KV];
+      ElemIO<T>::load(gamma + vi * KV, g);
+      if constexpr (!RMS) ElemIO<T>::load(beta + vi * KV, b);
+#pragma unroll
+      for (int r = 0; r < RPG; ++r)
+        if (active[r]) {
+          ElemIO<T>::load(s[r] + vi * KV, v[r][0]);
+          emit(r, vi, v[r][0], g, b);
+        }
     }
   }
 }
@@ -119,19 +152,19 @@ int launch_norm_t(const void* src, void* dst, const void* gamma, const void* bet
   T* d = (T*)dst;
   const T* g = (const T*)gamma;
   const T* b = (const T*)beta;
-#define SM_LAUNCH(LPR, VPL)                                                                      \
-  {                                                                                              \
-    long long rpb = 8 * (32 / LPR);                                                              \
-    unsigned grid = (unsigned)((rows + rpb - 1) / rpb);                                          \
-    norm_kernel<T, LPR, VPL, RMS><<<grid, 256, 0, st>>>(s, d, g, b, eps, rows, C, dm, has);      \
+#define SM_LAUNCH(LPR, VPL, RPG)                                                                  \
+  {                                                                                               \
+    long long rpb = 8 * (32 / LPR) * RPG;                                                         \
+    unsigned grid = (unsigned)((rows + rpb - 1) / rpb);                                           \
+    norm_kernel<T, LPR, VPL, RMS, RPG><<<grid, 256, 0, st>>>(s, d, g, b, eps, rows, C, dm, has);  \
   }
-  if (nvec <= 4) SM_LAUNCH(4, 1)
-  else if (nvec <= 8) SM_LAUNCH(8, 1)
-  else if (nvec <= 16) SM_LAUNCH(16, 1)
-  else if (nvec <= 32) SM_LAUNCH(32, 1)
-  else if (nvec <= 64) SM_LAUNCH(32, 2)
-  else if (nvec <= 128) SM_LAUNCH(32, 4)
-  else SM_LAUNCH(32, 0)
+  if (nvec <= 4) SM_LAUNCH(4, 1, 4)
+  else if (nvec <= 8) SM_LAUNCH(8, 1, 4)
+  else if (nvec <= 16) SM_LAUNCH(16, 1, 4)
+  else if (nvec <= 32) SM_LAUNCH(32, 1, 4)
+  else if (nvec <= 64) SM_LAUNCH(32, 2, 2)
+  else if (nvec <= 128) SM_LAUNCH(32, 4, 1)
+  else SM_LAUNCH(32, 0, 1)
 #undef SM_LAUNCH
   count_launch();
   return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
