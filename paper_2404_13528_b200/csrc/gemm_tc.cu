@@ -217,7 +217,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int e = warp - 2;
     const int q = warp & 3;                                  // TMEM lane quadrant this warp may read
     const int grp = e >> 2;
+    constexpr bool QSTAGE = !(BN == 256 && STAGES == 4);     // per-quadrant staging of whole rows
+    constexpr int QROW = BN * 2 + 16;                        // bytes; the pad keeps phase 1 conflict-free
     uint8_t* stage = stage_base + e * (32 * STG_ROW);
+    uint8_t* qstage = stage_base + q * (32 * QROW);
     uint32_t it = 0;
     bool ok = true;
     for (uint32_t t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
@@ -315,24 +318,43 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           pk.y = float2_to_bf16x2(acc[v * 8 + 2], acc[v * 8 + 3]);
           pk.z = float2_to_bf16x2(acc[v * 8 + 4], acc[v * 8 + 5]);
           pk.w = float2_to_bf16x2(acc[v * 8 + 6], acc[v * 8 + 7]);
-          *reinterpret_cast<uint4*>(stage + lane * STG_ROW + v * 16) = pk;
+          if constexpr (QSTAGE) *reinterpret_cast<uint4*>(qstage + lane * QROW + (c0 + v * 8) * 2) = pk;
+          else *reinterpret_cast<uint4*>(stage + lane * STG_ROW + v * 16) = pk;
         }
-        __syncwarp();
+        if constexpr (!QSTAGE) {
+          __syncwarp();
 #pragma unroll
-        for (int i = 0; i < VPR; ++i) {
-          const int v = lane + 32 * i;
-          const int rr = v / VPR, seg = v - rr * VPR;
-          const long long roff = __shfl_sync(0xFFFFFFFFu, off, rr);
-          const int rok = __shfl_sync(0xFFFFFFFFu, (int)row_ok, rr);
-          const uint4 pk = *reinterpret_cast<const uint4*>(stage + rr * STG_ROW + seg * 16);
-          if (rok && n0 + c0 + seg * 8 + 8 <= g.N) *reinterpret_cast<uint4*>(g.out + roff + n0 + c0 + seg * 8) = pk;
+          for (int i = 0; i < VPR; ++i) {
+            const int v = lane + 32 * i;
+            const int rr = v / VPR, seg = v - rr * VPR;
+            const long long roff = __shfl_sync(0xFFFFFFFFu, off, rr);
+            const int rok = __shfl_sync(0xFFFFFFFFu, (int)row_ok, rr);
+            const uint4 pk = *reinterpret_cast<const uint4*>(stage + rr * STG_ROW + seg * 16);
+            if (rok && n0 + c0 + seg * 8 + 8 <= g.N) *reinterpret_cast<uint4*>(g.out + roff + n0 + c0 + seg * 8) = pk;
+          }
+          __syncwarp();
         }
-        __syncwarp();
       }
       // all of this warp's TMEM reads of the buffer have completed (wait::ld above)
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&tmem_empty[buf]);
+      if constexpr (QSTAGE) {
+        // the four warps of the quadrant have filled a 32 x BN staging tile: store whole rows
+        constexpr int VR = BN / 8;                           // 16-byte vectors per row
+        asm volatile("bar.sync %0, 128;" ::"r"(1 + q) : "memory");
+        const int tq = grp * 32 + lane;
+#pragma unroll
+        for (int i = 0; i < VR / 4; ++i) {
+          const int v = tq + 128 * i;
+          const int rr = v / VR, seg = v - rr * VR;
+          const long long roff = __shfl_sync(0xFFFFFFFFu, off, rr);
+          const int rok = __shfl_sync(0xFFFFFFFFu, (int)row_ok, rr);
+          const uint4 pk = *reinterpret_cast<const uint4*>(qstage + rr * QROW + seg * 16);
+          if (rok && n0 + seg * 8 + 8 <= g.N) *reinterpret_cast<uint4*>(g.out + roff + n0 + seg * 8) = pk;
+        }
+        asm volatile("bar.sync %0, 128;" ::"r"(1 + q) : "memory");
+      }
     }
   }
   ptx::tc_fence_before();
@@ -461,7 +483,7 @@ template <int BN, int STAGES, bool A_MN>
 int launch_t(const CUtensorMap& ta, const CUtensorMap& tb, const GemmArgs& g, cudaStream_t st) {
   constexpr int RCc = (BN == 256 && STAGES == 4) ? 16 : ((BN / 4) > 32 ? 32 : (BN / 4));
   constexpr size_t smem = 1024 + STAGES * (A_STAGE_BYTES + BN * BK * 2) + (2 * STAGES + 4) * 8 + 16 +
-                          kEpiWarps * 32 * (RCc * 2 + 16);
+                          ((BN == 256 && STAGES == 4) ? kEpiWarps * 32 * (RCc * 2 + 16) : 4 * 32 * (BN * 2 + 16));
   static bool configured = false;
   if (!configured) {
     if (cudaFuncSetAttribute(gemm_tc_kernel<BN, STAGES, A_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
