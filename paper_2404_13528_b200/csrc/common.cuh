@@ -59,26 +59,36 @@ struct DevMap {
   long long base;
 };
 
-// Source offset (elements) of consumer unit `i`.
+// Source offset (elements) of consumer unit `i`.  Everything stays in registers: the rolled
+// coordinates are accumulated with selects instead of an indexed array.
 __device__ __forceinline__ long long devmap_eval(const DevMap& m, uint32_t i) {
   long long off = m.base;
-  int u[SMARTMEM_MAX_ROLLS] = {0, 0, 0, 0};
+  int u0 = 0, u1 = 0, u2 = 0, u3 = 0;
 #pragma unroll 1
   for (int a = m.n_atoms - 1; a >= 0; --a) {
-    uint32_t q = fd_div(i, m.ext[a]);
-    uint32_t digit = i - q * m.ext[a].d;
+    const uint32_t q = fd_div(i, m.ext[a]);
+    const int digit = (int)(i - q * m.ext[a].d);
     i = q;
-    int r = m.roll_of[a];
-    if (r < 0) off += (long long)digit * m.stride[a];
-    else u[r] += (int)digit * m.weight[a];
-  }
-#pragma unroll
-  for (int r = 0; r < SMARTMEM_MAX_ROLLS; ++r)
-    if (r < m.n_rolls) {
-      int v = u[r] + m.roll_shift[r];
-      if (v >= m.roll_mod[r]) v -= m.roll_mod[r];     // u < mod and shift < mod: one conditional subtract
-      off += (long long)v * m.roll_stride[r];
+    const int r = m.roll_of[a];
+    if (r < 0) {
+      off += (long long)digit * m.stride[a];
+    } else {
+      const int w = digit * m.weight[a];
+      u0 += r == 0 ? w : 0;
+      u1 += r == 1 ? w : 0;
+      u2 += r == 2 ? w : 0;
+      u3 += r == 3 ? w : 0;
     }
+  }
+  auto wrap = [&](int u, int r) {
+    int v = u + m.roll_shift[r];
+    if (v >= m.roll_mod[r]) v -= m.roll_mod[r];     // u < mod and shift < mod: one conditional subtract
+    off += (long long)v * m.roll_stride[r];
+  };
+  if (m.n_rolls > 0) wrap(u0, 0);
+  if (m.n_rolls > 1) wrap(u1, 1);
+  if (m.n_rolls > 2) wrap(u2, 2);
+  if (m.n_rolls > 3) wrap(u3, 3);
   return off;
 }
 

@@ -501,6 +501,17 @@ int launch_t(const CUtensorMap& ta, const CUtensorMap& tb, const GemmArgs& g, cu
 
 }  // namespace
 
+int tc_encode_2d(const void* ptr, long long inner, long long outer, long long pitch_elems, int box_inner, int box_outer,
+                 CUtensorMap* out) {
+  if (((uintptr_t)ptr & 15) || (pitch_elems * 2) % 16) return SMARTMEM_ERR_ALIGNMENT;
+  const uint64_t dims[2] = {(uint64_t)inner, (uint64_t)outer};
+  const uint64_t strides[1] = {(uint64_t)pitch_elems * 2};
+  const uint32_t box[2] = {(uint32_t)box_inner, (uint32_t)box_outer};
+  return encode_cached(ptr, 2, dims, strides, box, out);
+}
+
+int tc_sm_count() { return sm_count(); }
+
 int tc_operand_from_map(const smartmem_index_map_t& m, int n_batch_atoms, int n_row_atoms, const void* ptr,
                         TcOperand* op) {
   if (m.klass == 3 || m.n_rolls > 0) return SMARTMEM_ERR_UNSUPPORTED;

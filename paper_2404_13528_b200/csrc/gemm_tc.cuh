@@ -1,5 +1,7 @@
 // Host-side interface of the tcgen05 GEMM.
 #pragma once
+#include <cuda.h>
+
 #include "common.cuh"
 
 namespace smartmem {
@@ -33,5 +35,16 @@ int tc_operand_from_map(const smartmem_index_map_t& m, int n_batch_atoms, int n_
 TcOperand tc_operand_plain(const void* ptr, long long rows, long long K, long long ld);
 int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep, long long batch, long long M,
                    long long N, long long K, cudaStream_t st);
+
+// bf16 row-major [outer, inner] matrix as a 2-D tensor map with 128-byte swizzle (box_inner = 64).
+int tc_encode_2d(const void* ptr, long long inner, long long outer, long long pitch_elems, int box_inner, int box_outer,
+                 CUtensorMap* out);
+int tc_sm_count();
+
+// Fused MLP: out = residual + (GELU(A W1^T + b1)) W2^T + b2 with the hidden activation kept on chip.
+// A [M, C], W1 [hidden, C], W2 [C, hidden], C in {64, 96, 128}, hidden a multiple of 128.
+bool mlp_fused_supported(long long C, long long hidden);
+int launch_mlp_fused(const void* A, const void* W1, const void* b1, const void* W2, const void* b2, const void* residual,
+                     void* out, long long M, long long C, long long hidden, cudaStream_t st);
 
 }  // namespace smartmem

@@ -15,16 +15,17 @@ __device__ __forceinline__ float group_sum(float v) {
   return v;
 }
 
-// LPR lanes cooperate on one row; VPL 16-byte vectors per lane are kept in registers
-// (VPL == 0: any row length, the row is re-read from L1/L2 for each pass).  Each lane group
-// handles RPG rows at once so that RPG independent loads are in flight per lane.
-template <typename T, int LPR, int VPL, bool RMS, int RPG>
+// LPR lanes cooperate on one row and keep up to 4 16-byte vectors each in registers (vector k of
+// lane l is vector l + k * LPR of the row, so a warp-wide load covers 32 / LPR rows with runs of
+// LPR * 16 contiguous bytes).  RPG rows per lane group are in flight together.  GENERIC: any row
+// length; the row is re-read from L1/L2 for each pass instead of being kept.
+template <typename T, int LPR, bool RMS, int RPG, bool GENERIC>
 __global__ void __launch_bounds__(256) norm_kernel(const T* __restrict__ src, T* __restrict__ dst,
                                                    const T* __restrict__ gamma, const T* __restrict__ beta, float eps,
-                                                   long long rows, int C, const __grid_constant__ DevMap rowmap,
+                                                   long long rows, int C, int vpl, const __grid_constant__ DevMap rowmap,
                                                    int has_map) {
   constexpr int KV = ElemIO<T>::kVec;
-  constexpr int NV = VPL > 0 ? VPL : 1;
+  constexpr int NV = GENERIC ? 1 : 4;
   constexpr int GPB = 8 * (32 / LPR);                       // lane groups per block
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int sub = lane % LPR, grp = warp * (32 / LPR) + lane / LPR;
@@ -39,17 +40,23 @@ __global__ void __launch_bounds__(256) norm_kernel(const T* __restrict__ src, T*
   for (int r = 0; r < RPG; ++r) {
     const long long row = row0 + (long long)r * GPB;
     active[r] = row < rows;
-    const long long soff = active[r] ? (has_map ? devmap_eval(rowmap, (uint32_t)row) : row * (long long)C) : 0;
+    long long soff = 0;
+    if (has_map) {
+      if (sub == 0 && active[r]) soff = devmap_eval(rowmap, (uint32_t)row);   // one lane per row, then broadcast
+      soff = __shfl_sync(0xFFFFFFFFu, soff, lane - sub);
+    } else if (active[r]) {
+      soff = row * (long long)C;
+    }
     s[r] = src + soff;
   }
 #pragma unroll
   for (int r = 0; r < RPG; ++r) {
     sum[r] = 0.f;
-    if constexpr (VPL > 0) {
+    if constexpr (!GENERIC) {
 #pragma unroll
-      for (int k = 0; k < VPL; ++k) {
+      for (int k = 0; k < NV; ++k) {
         const int vi = sub + k * LPR;
-        if (active[r] && vi < nvec) {
+        if (k < vpl && active[r] && vi < nvec) {
           ElemIO<T>::load(s[r] + vi * KV, v[r][k]);
         } else {
 #pragma unroll
@@ -60,11 +67,13 @@ __global__ void __launch_bounds__(256) norm_kernel(const T* __restrict__ src, T*
   }
 #pragma unroll
   for (int r = 0; r < RPG; ++r) {
-    if constexpr (VPL > 0) {
+    if constexpr (!GENERIC) {
 #pragma unroll
-      for (int k = 0; k < VPL; ++k)
+      for (int k = 0; k < NV; ++k)
+        if (k < vpl) {
 #pragma unroll
-        for (int e = 0; e < KV; ++e) sum[r] += RMS ? v[r][k][e] * v[r][k][e] : v[r][k][e];
+          for (int e = 0; e < KV; ++e) sum[r] += RMS ? v[r][k][e] * v[r][k][e] : v[r][k][e];
+        }
     } else {
       for (int vi = sub; vi < nvec && active[r]; vi += LPR) {
         ElemIO<T>::load(s[r] + vi * KV, v[r][0]);
@@ -83,11 +92,11 @@ __global__ void __launch_bounds__(256) norm_kernel(const T* __restrict__ src, T*
     } else {
       mean[r] = sum[r] * invC;
       float sq = 0.f;
-      if constexpr (VPL > 0) {
+      if constexpr (!GENERIC) {
 #pragma unroll
-        for (int k = 0; k < VPL; ++k) {
+        for (int k = 0; k < NV; ++k) {
           const int vi = sub + k * LPR;
-          if (active[r] && vi < nvec) {
+          if (k < vpl && active[r] && vi < nvec) {
 #pragma unroll
             for (int e = 0; e < KV; ++e) sq += (v[r][k][e] - mean[r]) * (v[r][k][e] - mean[r]);
           }
@@ -103,17 +112,19 @@ __global__ void __launch_bounds__(256) norm_kernel(const T* __restrict__ src, T*
       rstd[r] = rsqrtf(sq * invC + eps);
     }
   }
+  // y = x * (rstd g) + (beta - mean rstd g): two fused multiply-adds per element
   auto emit = [&](int r, int vi, float* x, const float* g, const float* b) {
     float y[KV];
+    const float ms = -mean[r] * rstd[r];
 #pragma unroll
-    for (int e = 0; e < KV; ++e) y[e] = RMS ? x[e] * rstd[r] * g[e] : (x[e] - mean[r]) * rstd[r] * g[e] + b[e];
+    for (int e = 0; e < KV; ++e) y[e] = RMS ? x[e] * rstd[r] * g[e] : fmaf(fmaf(x[e], rstd[r], ms), g[e], b[e]);
     ElemIO<T>::store(dst + (row0 + (long long)r * GPB) * (long long)C + vi * KV, y);
   };
-  if constexpr (VPL > 0) {
+  if constexpr (!GENERIC) {
 #pragma unroll
-    for (int k = 0; k < VPL; ++k) {
+    for (int k = 0; k < NV; ++k) {
       const int vi = sub + k * LPR;
-      if (vi < nvec) {
+      if (k < vpl && vi < nvec) {
         float g[KV], b[KV];
         ElemIO<T>::load(gamma + vi * KV, g);
         if constexpr (!RMS) ElemIO<T>::load(beta + vi * KV, b);
@@ -152,19 +163,18 @@ int launch_norm_t(const void* src, void* dst, const void* gamma, const void* bet
   T* d = (T*)dst;
   const T* g = (const T*)gamma;
   const T* b = (const T*)beta;
-#define SM_LAUNCH(LPR, VPL, RPG)                                                                  \
-  {                                                                                               \
-    long long rpb = 8 * (32 / LPR) * RPG;                                                         \
-    unsigned grid = (unsigned)((rows + rpb - 1) / rpb);                                           \
-    norm_kernel<T, LPR, VPL, RMS, RPG><<<grid, 256, 0, st>>>(s, d, g, b, eps, rows, C, dm, has);  \
+#define SM_LAUNCH(LPR, RPG, GEN)                                                                          \
+  {                                                                                                       \
+    const int vpl = (nvec + LPR - 1) / LPR;                                                               \
+    long long rpb = 8 * (32 / LPR) * RPG;                                                                 \
+    unsigned grid = (unsigned)((rows + rpb - 1) / rpb);                                                   \
+    norm_kernel<T, LPR, RMS, RPG, GEN><<<grid, 256, 0, st>>>(s, d, g, b, eps, rows, C, vpl, dm, has);     \
   }
-  if (nvec <= 4) SM_LAUNCH(4, 1, 4)
-  else if (nvec <= 8) SM_LAUNCH(8, 1, 4)
-  else if (nvec <= 16) SM_LAUNCH(16, 1, 4)
-  else if (nvec <= 32) SM_LAUNCH(32, 1, 4)
-  else if (nvec <= 64) SM_LAUNCH(32, 2, 2)
-  else if (nvec <= 128) SM_LAUNCH(32, 4, 1)
-  else SM_LAUNCH(32, 0, 1)
+  if (nvec <= 16) SM_LAUNCH(4, 2, false)
+  else if (nvec <= 32) SM_LAUNCH(8, 2, false)
+  else if (nvec <= 64) SM_LAUNCH(16, 1, false)
+  else if (nvec <= 128) SM_LAUNCH(32, 1, false)
+  else SM_LAUNCH(32, 1, true)
 #undef SM_LAUNCH
   count_launch();
   return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
