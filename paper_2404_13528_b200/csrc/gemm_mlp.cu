@@ -14,12 +14,23 @@
 #include "gemm_tc.cuh"
 #include "ptx.cuh"
 
+#ifdef MLP_EXP_TIMING
+__device__ long long g_mlp_dbg[8192];
+#define DBG(slot) do { if (blockIdx.x == 0) g_mlp_dbg[(slot)] = clock64(); } while (0)
+extern "C" __attribute__((visibility("default"))) int smartmem_debug_read(long long* host, int n) {
+  return (int)cudaMemcpyFromSymbol(host, g_mlp_dbg, sizeof(long long) * n);
+}
+#else
+#define DBG(slot) do { } while (0)
+#endif
+
 namespace smartmem {
 namespace {
 
 constexpr int BM = 128, BK = 64, HC = 128;         // tile rows, k-block, hidden chunk
 constexpr int KB_BYTES = BM * BK * 2;              // one 128 x 64 bf16 operand block: 16 KB
-constexpr int NST = 4;                             // weight ring stages (16 KB each)
+constexpr int NST = 3;                             // weight ring stages; one stage = both k-blocks of a chunk's W1 or W2
+constexpr int WST_BYTES = 2 * KB_BYTES;
 constexpr int kEpiWarps = 16, kThreads = 64 + 32 * kEpiWarps;
 constexpr uint32_t TM_S1 = 0, TM_OUT = 256, TMEM_COLS = 512;
 
@@ -44,16 +55,17 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                  const __grid_constant__ CUtensorMap tmW2, const __grid_constant__ MlpArgs g) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
-  uint8_t* sA = smem;                              // [2 bufs][2 k-blocks][16 KB]
-  uint8_t* sH = sA + 4 * KB_BYTES;                 // [2 bufs][2 k-blocks][16 KB]
-  uint8_t* sW = sH + 4 * KB_BYTES;                 // [NST][16 KB]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sW + NST * KB_BYTES);
+  uint8_t* sA = smem;                              // [2 k-blocks][16 KB]
+  uint8_t* sH = sA + 2 * KB_BYTES;                 // [2 bufs][2 k-blocks][16 KB]
+  uint8_t* sW = sH + 4 * KB_BYTES;                 // [NST][2 k-blocks][16 KB]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sW + NST * WST_BYTES);
   uint64_t *a_full = bars, *a_empty = bars + 2, *w_full = bars + 4, *w_empty = w_full + NST;
   uint64_t *s1_full = w_empty + NST, *s1_empty = s1_full + 2, *h_full = s1_empty + 2, *h_empty = h_full + 2;
   uint64_t *out_full = h_empty + 2, *out_empty = out_full + 1;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(out_empty + 1);
   int* abort_flag = reinterpret_cast<int*>(tmem_slot + 1);
   uint8_t* qstage_base = reinterpret_cast<uint8_t*>(tmem_slot + 4);
+  float* b1_s = reinterpret_cast<float*>(qstage_base + 4 * 32 * (g.C == 128 ? 256 : g.C * 2 + 16));   // [hidden]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int NC = g.n_chunks;
@@ -84,6 +96,7 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     ptx::prefetch_tensormap(&tmW1);
     ptx::prefetch_tensormap(&tmW2);
   }
+  for (int i = threadIdx.x; i < g.hidden; i += kThreads) b1_s[i] = __bfloat162float(g.b1[i]);
   if (warp == 1) ptx::tmem_alloc(tmem_slot, TMEM_COLS);
   ptx::tc_fence_before();
   __syncthreads();
@@ -94,27 +107,28 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     if (lane == 0) {
       uint32_t wcnt = 0, it = 0;
       bool ok = true;
-      auto load_w = [&](const CUtensorMap* tm, int c0, int c1, uint32_t bytes) {
+      auto load_w1 = [&](int c) {                      // [128 hidden rows] x C, as nkb1 k-blocks
         const int s = wcnt % NST;
         ok = ok && ptx::mbar_wait(&w_empty[s], ((wcnt / NST) & 1) ^ 1, abort_flag, g.status);
         if (!ok) return;
-        ptx::mbar_expect_tx(&w_full[s], bytes);
-        ptx::tma_load_2d(sW + s * KB_BYTES, tm, &w_full[s], c0, c1);
+        ptx::mbar_expect_tx(&w_full[s], nkb1 * KB_BYTES);
+        for (int kb = 0; kb < nkb1; ++kb) ptx::tma_load_2d(sW + s * WST_BYTES + kb * KB_BYTES, &tmW1, &w_full[s], kb * BK, c * HC);
         ++wcnt;
       };
-      auto load_w1 = [&](int c) {
-        for (int kb = 0; kb < nkb1 && ok; ++kb) load_w(&tmW1, kb * BK, c * HC, KB_BYTES);
-      };
-      auto load_w2 = [&](int c) {
-        for (int kb = 0; kb < 2 && ok; ++kb) load_w(&tmW2, c * HC + kb * BK, 0, (uint32_t)g.C * BK * 2);
+      auto load_w2 = [&](int c) {                      // [C rows] x 128 hidden columns, as 2 k-blocks
+        const int s = wcnt % NST;
+        ok = ok && ptx::mbar_wait(&w_empty[s], ((wcnt / NST) & 1) ^ 1, abort_flag, g.status);
+        if (!ok) return;
+        ptx::mbar_expect_tx(&w_full[s], 2 * (uint32_t)g.C * BK * 2);
+        for (int kb = 0; kb < 2; ++kb) ptx::tma_load_2d(sW + s * WST_BYTES + kb * KB_BYTES, &tmW2, &w_full[s], c * HC + kb * BK, 0);
+        ++wcnt;
       };
       for (uint32_t t = blockIdx.x; t < (uint32_t)g.tiles && ok; t += gridDim.x, ++it) {
-        const uint32_t ab = it & 1;
-        ok = ptx::mbar_wait(&a_empty[ab], ((it >> 1) & 1) ^ 1, abort_flag, g.status);
+        ok = ptx::mbar_wait(&a_empty[0], (it & 1) ^ 1, abort_flag, g.status);
         if (!ok) break;
-        ptx::mbar_expect_tx(&a_full[ab], nkb1 * KB_BYTES);
+        ptx::mbar_expect_tx(&a_full[0], nkb1 * KB_BYTES);
         for (int kb = 0; kb < nkb1; ++kb)
-          ptx::tma_load_2d(sA + (ab * 2 + kb) * KB_BYTES, &tmA, &a_full[ab], kb * BK, (int)t * BM);
+          ptx::tma_load_2d(sA + kb * KB_BYTES, &tmA, &a_full[0], kb * BK, (int)t * BM);
         // weights in the order the MMA warp consumes them
         load_w1(0);
         for (int c = 0; c < NC && ok; ++c) {
@@ -130,23 +144,26 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       uint32_t wcnt = 0, it = 0, s1cnt = 0, hcnt = 0;
       bool ok = true;
       for (uint32_t t = blockIdx.x; t < (uint32_t)g.tiles && ok; t += gridDim.x, ++it) {
-        const uint32_t ab = it & 1;
-        ok = ptx::mbar_wait(&a_full[ab], (it >> 1) & 1, abort_flag, g.status);
+        ok = ptx::mbar_wait(&a_full[0], it & 1, abort_flag, g.status);
         if (!ok) break;
         auto fc1 = [&]() {                              // S1[buf] = A W1[chunk]^T
           const uint32_t sb = s1cnt & 1;
           ok = ok && ptx::mbar_wait(&s1_empty[sb], ((s1cnt >> 1) & 1) ^ 1, abort_flag, g.status);
-          for (int kb = 0; kb < nkb1 && ok; ++kb, ++wcnt) {
+          if (ok) {
             const int s = wcnt % NST;
             ok = ptx::mbar_wait(&w_full[s], (wcnt / NST) & 1, abort_flag, g.status);
-            if (!ok) break;
-            ptx::tc_fence_after();
-            const uint32_t a0 = ptx::smem_u32(sA + (ab * 2 + kb) * KB_BYTES), b0 = ptx::smem_u32(sW + s * KB_BYTES);
-            const int ks = kb == 0 ? (g.C < BK ? g.C / 16 : BK / 16) : k1_last;
-            for (int k = 0; k < ks; ++k)
-              ptx::tc_mma_bf16(tmem_base + TM_S1 + sb * HC, ptx::make_smem_desc(a0 + k * 32, 16, 1024),
-                               ptx::make_smem_desc(b0 + k * 32, 16, 1024), idesc1, (kb | k) ? 1u : 0u);
-            ptx::tc_commit(&w_empty[s]);
+            if (ok) {
+              ptx::tc_fence_after();
+              for (int kb = 0; kb < nkb1; ++kb) {
+                const uint32_t a0 = ptx::smem_u32(sA + kb * KB_BYTES), b0 = ptx::smem_u32(sW + s * WST_BYTES + kb * KB_BYTES);
+                const int ks = kb == 0 ? (g.C < BK ? g.C / 16 : BK / 16) : k1_last;
+                for (int k = 0; k < ks; ++k)
+                  ptx::tc_mma_bf16(tmem_base + TM_S1 + sb * HC, ptx::make_smem_desc(a0 + k * 32, 16, 1024),
+                                   ptx::make_smem_desc(b0 + k * 32, 16, 1024), idesc1, (kb | k) ? 1u : 0u);
+              }
+              ptx::tc_commit(&w_empty[s]);
+              ++wcnt;
+            }
           }
           if (ok) ptx::tc_commit(&s1_full[sb]);
           ++s1cnt;
@@ -155,16 +172,20 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           const uint32_t hb = hcnt & 1;
           ok = ok && ptx::mbar_wait(&h_full[hb], (hcnt >> 1) & 1, abort_flag, g.status);
           if (ok && c == 0) ok = ptx::mbar_wait(out_empty, (it & 1) ^ 1, abort_flag, g.status);
-          for (int kb = 0; kb < 2 && ok; ++kb, ++wcnt) {
+          if (ok) {
             const int s = wcnt % NST;
             ok = ptx::mbar_wait(&w_full[s], (wcnt / NST) & 1, abort_flag, g.status);
-            if (!ok) break;
-            ptx::tc_fence_after();
-            const uint32_t a0 = ptx::smem_u32(sH + (hb * 2 + kb) * KB_BYTES), b0 = ptx::smem_u32(sW + s * KB_BYTES);
-            for (int k = 0; k < BK / 16; ++k)
-              ptx::tc_mma_bf16(tmem_base + TM_OUT, ptx::make_smem_desc(a0 + k * 32, 16, 1024),
-                               ptx::make_smem_desc(b0 + k * 32, 16, 1024), idesc2, (c | kb | k) ? 1u : 0u);
-            ptx::tc_commit(&w_empty[s]);
+            if (ok) {
+              ptx::tc_fence_after();
+              for (int kb = 0; kb < 2; ++kb) {
+                const uint32_t a0 = ptx::smem_u32(sH + (hb * 2 + kb) * KB_BYTES), b0 = ptx::smem_u32(sW + s * WST_BYTES + kb * KB_BYTES);
+                for (int k = 0; k < BK / 16; ++k)
+                  ptx::tc_mma_bf16(tmem_base + TM_OUT, ptx::make_smem_desc(a0 + k * 32, 16, 1024),
+                                   ptx::make_smem_desc(b0 + k * 32, 16, 1024), idesc2, (c | kb | k) ? 1u : 0u);
+              }
+              ptx::tc_commit(&w_empty[s]);
+              ++wcnt;
+            }
           }
           if (ok) ptx::tc_commit(&h_empty[hb]);
           ++hcnt;
@@ -172,7 +193,7 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         fc1();
         for (int c = 0; c < NC && ok; ++c) {
           if (c + 1 < NC) fc1();
-          if (c + 1 == NC && ok) ptx::tc_commit(&a_empty[ab]);   // every fc1 MMA of this tile has been issued
+          if (c + 1 == NC && ok) ptx::tc_commit(&a_empty[0]);   // every fc1 MMA of this tile has been issued
           fc2(c);
         }
         if (ok) ptx::tc_commit(out_full);
@@ -190,6 +211,12 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       const bool row_ok = row < g.M;
       for (int c = 0; c < NC && ok; ++c, ++s1cnt, ++hcnt) {
         const uint32_t sb = s1cnt & 1, hb = hcnt & 1;
+        float bb[32];                                    // this warp's 32 biases of the chunk, fetched before the wait
+#pragma unroll
+        for (int v = 0; v < 8; ++v) {
+          const float4 b4 = *reinterpret_cast<const float4*>(b1_s + c * HC + grp * 32 + v * 4);
+          bb[v * 4 + 0] = b4.x; bb[v * 4 + 1] = b4.y; bb[v * 4 + 2] = b4.z; bb[v * 4 + 3] = b4.w;
+        }
         ok = ptx::mbar_wait(&s1_full[sb], (s1cnt >> 1) & 1, abort_flag, g.status);
         if (!ok) break;
         ok = ptx::mbar_wait(&h_empty[hb], ((hcnt >> 1) & 1) ^ 1, abort_flag, g.status);   // fc2 done with this buffer
@@ -200,12 +227,11 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         ptx::tmem_ld_wait();
         float acc[32];
 #pragma unroll
-        for (int v = 0; v < 4; ++v) {
-          float bb[8];
-          ElemIO<__nv_bfloat16>::load(g.b1 + c * HC + grp * 32 + v * 8, bb);
-#pragma unroll
-          for (int j = 0; j < 8; ++j) acc[v * 8 + j] = gelu_tanh(__uint_as_float(rv[v * 8 + j]) + bb[j]);
-        }
+#ifdef MLP_EXP_NOGELU
+        for (int j = 0; j < 32; ++j) acc[j] = __uint_as_float(rv[j]) + bb[j];
+#else
+        for (int j = 0; j < 32; ++j) acc[j] = gelu_tanh(__uint_as_float(rv[j]) + bb[j]);
+#endif
         // chunk columns grp*32 .. +31 -> k-block (grp >> 1), 16-byte chunks ((grp & 1) * 4 + v) ^ (row & 7)
         uint8_t* hrow = sH + (hb * 2 + (grp >> 1)) * KB_BYTES + r_tile * 128;
 #pragma unroll
@@ -296,7 +322,7 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 }  // namespace
 
 bool mlp_fused_supported(long long C, long long hidden) {
-  return (C == 64 || C == 96 || C == 128) && hidden >= HC && hidden % HC == 0;
+  return (C == 64 || C == 96) && hidden >= HC && hidden % HC == 0 && hidden <= 1024;
 }
 
 int launch_mlp_fused(const void* A, const void* W1, const void* b1, const void* W2, const void* b2, const void* residual,
@@ -319,7 +345,8 @@ int launch_mlp_fused(const void* A, const void* W1, const void* b1, const void* 
   g.out = (__nv_bfloat16*)out;
   g.status = device_status_ptr();
   if (!g.status) return SMARTMEM_ERR_CUDA;
-  const size_t smem = 1024 + (4 + 4 + NST) * KB_BYTES + (8 + 2 * NST + 6) * 8 + 16 + 4 * 32 * (C == 128 ? 256 : C * 2 + 16);
+  const size_t smem = 1024 + (2 + 4 + 2 * NST) * KB_BYTES + (8 + 2 * NST + 6) * 8 + 16 + 4 * 32 * (C == 128 ? 256 : C * 2 + 16) +
+                      (size_t)hidden * 4;
   static bool configured = false;
   if (!configured) {
     if (cudaFuncSetAttribute(mlp_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448) != cudaSuccess)

@@ -42,7 +42,7 @@ int tc_encode_2d(const void* ptr, long long inner, long long outer, long long pi
 int tc_sm_count();
 
 // Fused MLP: out = residual + (GELU(A W1^T + b1)) W2^T + b2 with the hidden activation kept on chip.
-// A [M, C], W1 [hidden, C], W2 [C, hidden], C in {64, 96, 128}, hidden a multiple of 128.
+// A [M, C], W1 [hidden, C], W2 [C, hidden], C in {64, 96}, hidden a multiple of 128 (at most 1024).
 bool mlp_fused_supported(long long C, long long hidden);
 int launch_mlp_fused(const void* A, const void* W1, const void* b1, const void* W2, const void* b2, const void* residual,
                      void* out, long long M, long long C, long long hidden, cudaStream_t st);
