@@ -15,7 +15,8 @@ struct WinAttnArgs {
   const void* table;        // [(2ws-1)^2, heads]
   int table_f32;
   int heads, T, ws, d, shift, H, W, nWw, win_per_img;
-  int n_windows;            // set by the launcher
+  int n_windows, nWh;       // set by the launcher
+  FastDiv fd_wpi, fd_nww;   // reciprocals of win_per_img and nWw (set by the launcher)
   float scale;
 };
 int launch_window_attention(const WinAttnArgs& a, int dtype, long long n_windows, cudaStream_t st);

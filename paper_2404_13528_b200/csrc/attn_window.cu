@@ -29,7 +29,13 @@ __device__ __forceinline__ const T* unit_ptr(const AttnOperand& o, int n, int h)
   return (const T*)o.ptr + (long long)n * o.sn + (long long)h * o.sh;
 }
 
-// Region label of token t of window (wy, wx) in shifted coordinates.
+// Region label of token (ty, tx) of window (wy, wx) in shifted coordinates.
+__device__ __forceinline__ int region_label2(int ty, int tx, int ws, int wy, int wx, int H, int W, int shift) {
+  const int hp = wy * ws + ty, wp = wx * ws + tx;
+  const int rh = hp < H - ws ? 0 : (hp < H - shift ? 1 : 2);
+  const int rw = wp < W - ws ? 0 : (wp < W - shift ? 1 : 2);
+  return 3 * rh + rw;
+}
 __device__ __forceinline__ int region_label(int t, int ws, int wy, int wx, int H, int W, int shift) {
   const int hp = wy * ws + t / ws, wp = wx * ws + t % ws;
   const int rh = hp < H - ws ? 0 : (hp < H - shift ? 1 : 2);
@@ -66,22 +72,32 @@ __global__ void __launch_bounds__(128) win_attn_bf16_kernel(const __grid_constan
   // rows >= T of every tile stay zero for the whole kernel
   for (int i = tid; i < 2 * 3 * TILE / 8; i += 128) reinterpret_cast<uint4*>(&bufs[0][0][0])[i] = make_uint4(0, 0, 0, 0);
 
+  // token coordinates: divisions by the (run-time) window size happen once per thread, here
+  __shared__ int code_s[TP];
+  const int my_ty = tid / ws, my_tx = tid - my_ty * ws;      // token `tid` of a window (tid < 64 used)
+  if (tid < TP) code_s[tid] = my_ty * (2 * ws - 1) + my_tx;
+  __syncthreads();
   // bias fragment of this head: element (row, col) <- table[(dy + ws - 1)(2ws - 1) + dx + ws - 1, h]
+  //                                                 = table[code(row) - code(col) + (ws - 1) 2 ws, h]
   float bias[8][4];
+  {
+    const int off = (ws - 1) * 2 * ws;
+    const int cr[2] = {code_s[r0] + off, code_s[r1] + off};
 #pragma unroll
-  for (int j = 0; j < 8; ++j) {
+    for (int j = 0; j < 8; ++j) {
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const int r = (e < 2) ? r0 : r1, c = j * 8 + 2 * t4 + (e & 1);
-      float v = 0.f;
-      if (r < T && c < T) {
-        const int idx = (r / ws - c / ws + ws - 1) * (2 * ws - 1) + (r % ws - c % ws + ws - 1);
-        v = a.table_f32 ? ((const float*)a.table)[idx * a.heads + h]
-                        : __bfloat162float(((const __nv_bfloat16*)a.table)[idx * a.heads + h]);
-      } else if (c >= T) {
-        v = -INFINITY;                          // padded key columns never contribute
+      for (int e = 0; e < 4; ++e) {
+        const int r = (e < 2) ? r0 : r1, c = j * 8 + 2 * t4 + (e & 1);
+        float v = 0.f;
+        if (r < T && c < T) {
+          const int idx = cr[e >> 1] - code_s[c];
+          v = a.table_f32 ? ((const float*)a.table)[idx * a.heads + h]
+                          : __bfloat162float(((const __nv_bfloat16*)a.table)[idx * a.heads + h]);
+        } else if (c >= T) {
+          v = -INFINITY;                          // padded key columns never contribute
+        }
+        bias[j][e] = v;
       }
-      bias[j][e] = v;
     }
   }
   __syncthreads();
@@ -107,8 +123,9 @@ __global__ void __launch_bounds__(128) win_attn_bf16_kernel(const __grid_constan
       }
     }
     if (a.shift > 0 && tid < TP) {
-      const int wl = n % a.win_per_img;
-      lab_s[b][tid] = region_label(tid, ws, wl / a.nWw, wl % a.nWw, a.H, a.W, a.shift);
+      const int wl = n - (int)fd_div((uint32_t)n, a.fd_wpi) * a.win_per_img;
+      const int wy = (int)fd_div((uint32_t)wl, a.fd_nww), wx = wl - wy * a.nWw;
+      lab_s[b][tid] = region_label2(my_ty, my_tx, ws, wy, wx, a.H, a.W, a.shift);
     }
   };
 
@@ -131,6 +148,9 @@ __global__ void __launch_bounds__(128) win_attn_bf16_kernel(const __grid_constan
       for (int j = 0; j < 8; ++j) s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
 #pragma unroll
       for (int kk = 0; kk < D / 16; ++kk) {
+#ifdef WA_EXP_NOQK
+        s[kk][0] = __uint_as_float(Qw[r0 * RW + t4]); break;
+#endif
         uint32_t af[4];
         af[0] = Qw[r0 * RW + kk * 8 + t4];
         af[1] = Qw[r1 * RW + kk * 8 + t4];
@@ -146,6 +166,7 @@ __global__ void __launch_bounds__(128) win_attn_bf16_kernel(const __grid_constan
         }
       }
       // ---- scale + bias (+ mask on the windows that touch the seam), softmax ------------------
+#ifndef WA_EXP_NOSOFTMAX
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
 #pragma unroll
@@ -153,8 +174,9 @@ __global__ void __launch_bounds__(128) win_attn_bf16_kernel(const __grid_constan
       }
       bool masked = false;
       if (a.shift > 0) {
-        const int wl = n % a.win_per_img;
-        masked = (wl / a.nWw == a.H / ws - 1) || (wl % a.nWw == a.nWw - 1);
+        const int wl = n - (int)fd_div((uint32_t)n, a.fd_wpi) * a.win_per_img;
+        const int wy = (int)fd_div((uint32_t)wl, a.fd_nww), wx = wl - wy * a.nWw;
+        masked = (wy == a.nWh - 1) || (wx == a.nWw - 1);
       }
       if (masked) {
         const int l0 = lab_s[b][r0], l1 = lab_s[b][r1];
@@ -183,7 +205,11 @@ __global__ void __launch_bounds__(128) win_attn_bf16_kernel(const __grid_constan
       for (int j = 0; j < 8; ++j) {
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
+#ifdef WA_EXP_NOEXP
+          const float p0 = s[j][e] - m0, p1 = s[j][2 + e] - m1;
+#else
           const float p0 = __expf(s[j][e] - m0), p1 = __expf(s[j][2 + e] - m1);
+#endif
           s[j][e] = p0;
           s[j][2 + e] = p1;
           sum0 += p0;
@@ -194,12 +220,21 @@ __global__ void __launch_bounds__(128) win_attn_bf16_kernel(const __grid_constan
       sum0 += __shfl_xor_sync(0xFFFFFFFFu, sum0, 2);
       sum1 += __shfl_xor_sync(0xFFFFFFFFu, sum1, 1);
       sum1 += __shfl_xor_sync(0xFFFFFFFFu, sum1, 2);
+#else
+      float sum0 = 1.f, sum1 = 1.f;
+#endif
       // ---- O = P V: the score fragments are the A fragments of the second MMA -----------------
       float o[D / 8][4];
 #pragma unroll
       for (int j = 0; j < D / 8; ++j) o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f;
+#ifdef WA_EXP_NOPV
+      for (int j = 0; j < D / 8; ++j) { o[j][0] = s[j][0]; o[j][1] = s[j][1]; o[j][2] = s[j][2]; o[j][3] = s[j][3]; }
+#endif
 #pragma unroll
       for (int kk = 0; kk < 4; ++kk) {
+#ifdef WA_EXP_NOPV
+        break;
+#endif
         if (kk * 16 < T) {
           uint32_t af[4];
           af[0] = float2_to_bf16x2(s[2 * kk][0], s[2 * kk][1]);
@@ -329,6 +364,9 @@ int launch_window_attention(const WinAttnArgs& a, int dtype, long long n_windows
     if (a.d != 16 && a.d != 32) return SMARTMEM_ERR_UNSUPPORTED;
     WinAttnArgs b = a;
     b.n_windows = (int)n_windows;
+    b.nWh = a.win_per_img / a.nWw;
+    b.fd_wpi = make_fastdiv((uint32_t)a.win_per_img);
+    b.fd_nww = make_fastdiv((uint32_t)a.nWw);
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) sms = 148;
