@@ -58,6 +58,26 @@ def algorithmic_bytes(w):
     }
 
 
+def shard_seed(config_id: int, rank: int) -> int:
+    """Each rank draws its own batch: the workload shards over images with no exchange step."""
+    return config_id + 1000 * rank
+
+
+def max_over_ranks(dist, value: float, device) -> float:
+    """The slowest rank's time bounds the job (no-op without a process group)."""
+    if dist is None:
+        return value
+    import torch
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tokens_per_s(tokens_per_rank: int, world: int, steps: int, ms: float) -> float:
+    """Aggregate throughput of `world` replicas that each did `steps` steps in `ms` (max over ranks)."""
+    return tokens_per_rank * world * steps / (ms * 1e-3)
+
+
 class ClockSampler:
     """Samples SM clock and throttle reasons with nvidia-smi while the GPU is under load."""
     Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
@@ -267,11 +287,13 @@ def run_other(args):
                 model = [("gemm_mn_major_operand", B * C * Hh * Ww * 2 + N * C * 2 + B * Hh * Ww * N * 2, 2 * B * Hh * Ww * N * C)]
             tokens = B * Hh * Ww
         sets = 8
-        plans = {m: sm.smartmem_plan(ops, descs, m) for m in (sm.ELIMINATE, sm.EXPLICIT)}
+        modes = (sm.ELIMINATE, sm.EXPLICIT) + ((sm.ELIMINATE_NAIVE,) if name.endswith("copy") else ())
+        plans = {m: sm.smartmem_plan(ops, descs, m) for m in modes}
         wsb = {m: sm.smartmem_plan_workspace_bytes(plans[m]) for m in plans}
         ins = [[t.clone() for t in srcs] for _ in range(sets)]
         outs = [torch.empty(oshape, dtype=torch.bfloat16, device="cuda") for _ in range(sets)]
         wss = [torch.empty(max(wsb[sm.EXPLICIT], 16), dtype=torch.uint8, device="cuda") for _ in range(sets)]
+        naive = sm.ELIMINATE_NAIVE in plans
 
         def step(i, mode):
             j = i % sets
@@ -293,6 +315,11 @@ def run_other(args):
         step(i, sm.ELIMINATE)
         step(i, sm.EXPLICIT)
     ms = {m: timed(m, args.steps) for m in (sm.ELIMINATE, sm.EXPLICIT)}
+    ms_naive = None
+    if name.endswith("copy"):
+        for i in range(args.warmup):
+            step(i, sm.ELIMINATE_NAIVE)
+        ms_naive = timed(sm.ELIMINATE_NAIVE, args.steps)
     per = {}
     for mode, tag in ((sm.ELIMINATE, "eliminate"), (sm.EXPLICIT, "explicit")):
         acc = None
@@ -323,6 +350,8 @@ def run_other(args):
         "config": {"workload": name, "mode": "eliminate", "l2": f"{sets} rotating buffer sets"},
         "explicit_variant": {"ms_per_step": ms[sm.EXPLICIT] / args.steps, "speedup_of_eliminate": ms[sm.EXPLICIT] / ms[sm.ELIMINATE],
                              "kernels": [{"launched_as": n, "ms": round(t, 5)} for n, t in per["explicit"]]},
+        "naive_index_variant": None if ms_naive is None else {"ms_per_step": ms_naive / args.steps,
+                                                                 "speedup_of_strength_reduced_map": ms_naive / ms[sm.ELIMINATE]},
         "clocks": clocks,
         "roofline": {"bound": dom["bound"], "kernel": dom["kernel"], "achieved": dom["achieved"], "unit": dom["unit"],
                      "peak": tf if dom["bound"] == "tensor" else hbm, "frac": dom["frac"], "traffic": None, "peak_source": src},
@@ -364,7 +393,7 @@ def main():
 
     w = WORKLOAD
     M = w["B"] * w["H"] * w["W"]
-    inp = synth.swin_inputs(w["config_id"] + 1000 * rank, w["B"], w["H"], w["W"], w["C"], w["heads"], w["window"],
+    inp = synth.swin_inputs(shard_seed(w["config_id"], rank), w["B"], w["H"], w["W"], w["C"], w["heads"], w["window"],
                             w["mlp_ratio"], w["dtype"])
 
     def dev(a):
@@ -404,12 +433,8 @@ def main():
             step(i, mode)
         e1.record()
         barrier()
-        ms = e0.elapsed_time(e1)
+        ms = max_over_ranks(dist, e0.elapsed_time(e1), "cuda")
         launches = sm.smartmem_launch_count() - n0
-        if dist is not None:
-            t = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
         return ms, launches
 
     sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ else
@@ -459,11 +484,7 @@ def main():
         y_host.copy_(ys[j], non_blocking=True)
     e1.record()
     barrier()
-    ms_e2e = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([ms_e2e], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item())
+    ms_e2e = max_over_ranks(dist, e0.elapsed_time(e1), "cuda")
     clocks = sampler.stop()
 
     cpu = None
@@ -474,7 +495,7 @@ def main():
 
     if rank == 0:
         tokens = M * world
-        value = tokens * args.steps / (ms_elim * 1e-3)
+        value = whole_job_tokens_per_s(M, world, args.steps, ms_elim)
         traffic = None
         tpath = os.path.join(ROOT, "profiles", "traffic.json")      # per-launch DRAM bytes from an ncu capture
         if os.path.exists(tpath):

@@ -55,7 +55,10 @@ typedef enum {
 } smartmem_status_t;
 
 typedef enum { SMARTMEM_F32 = 0, SMARTMEM_BF16 = 1 } smartmem_dtype_t;
-typedef enum { SMARTMEM_ELIMINATE = 0, SMARTMEM_EXPLICIT = 1 } smartmem_mode_t;
+/* ELIMINATE_NAIVE (smartmem_plan / smartmem_run_chain only): layout runs are eliminated, but copy
+ * consumers evaluate the sequential divide/modulo program instead of the strength-reduced map --
+ * the "index computation (no opt.)" form of Fig. 4, kept to measure what strength reduction buys. */
+typedef enum { SMARTMEM_ELIMINATE = 0, SMARTMEM_EXPLICIT = 1, SMARTMEM_ELIMINATE_NAIVE = 2 } smartmem_mode_t;
 
 /* Operator vocabulary of a chain.  Layout operators have a Fixed output layout (Table 3,
  * right column) and are the ones elimination removes; compute operators are kept. */
@@ -101,10 +104,14 @@ typedef struct {
  * (atom 0 is the most significant digit); the source offset in elements is
  *
  *     base + sum_{a : roll_of[a] < 0} digit_a * src_stride[a]
- *          + sum_r ((sum_{a : roll_of[a] == r} digit_a * roll_weight[a] + roll_shift[r]) mod roll_mod[r]) * roll_stride[r]
+ *          + sum_r place_r( (sum_{a : roll_of[a] == r} digit_a * roll_weight[a] + roll_shift[r]) mod roll_mod[r] )
  *
- * i.e. no division or modulo by tensor extents survives except one modulo per rolled
- * dimension.  klass: 0 identity (the chain vanishes), 1 affine (no roll; a TMA tensor map or
+ * where place_r(v) = v * roll_stride[r] when the rolled dimension is an affine coordinate of the
+ * producer's buffer (roll_n_parts[r] == 1), and otherwise v is written in mixed radix over
+ * roll_part_extent[r][] (part 0 most significant) and each digit is multiplied by
+ * roll_part_stride[r][] (a dimension rolled after it was merged from non-nesting factors, e.g.
+ * H after a window reverse).  No division or modulo by tensor extents survives except one
+ * modulo per rolled dimension (and the part digits of such merged dimensions).  klass: 0 identity (the chain vanishes), 1 affine (no roll; a TMA tensor map or
  * a tiled transpose can express it), 2 strided gather with rolls, 3 not canonicalisable
  * (the split points of the shapes do not refine each other): only the sequential
  * divide/modulo program -- the unoptimised form of Fig. 4 -- can evaluate it. */
@@ -118,6 +125,9 @@ typedef struct {
   int64_t roll_shift[SMARTMEM_MAX_ROLLS];
   int64_t roll_mod[SMARTMEM_MAX_ROLLS];
   int64_t roll_stride[SMARTMEM_MAX_ROLLS];
+  int32_t roll_n_parts[SMARTMEM_MAX_ROLLS];
+  int64_t roll_part_extent[SMARTMEM_MAX_ROLLS][SMARTMEM_MAX_ROLLS];
+  int64_t roll_part_stride[SMARTMEM_MAX_ROLLS][SMARTMEM_MAX_ROLLS];
   int64_t base;
   int64_t n_elements;                /* number of consumer elements                         */
   int32_t vec_elems;                 /* widest power-of-two run (<= 16 bytes) that is contiguous

@@ -18,7 +18,7 @@ OK = 0
 ERR_INVALID_ARG, ERR_SHAPE, ERR_UNSUPPORTED, ERR_WORKSPACE = -1, -2, -3, -4
 ERR_ALIGNMENT, ERR_CUDA, ERR_TIMEOUT, ERR_BOUNDS = -5, -6, -7, -8
 F32, BF16 = 0, 1
-ELIMINATE, EXPLICIT = 0, 1
+ELIMINATE, EXPLICIT, ELIMINATE_NAIVE = 0, 1, 2
 OP_RESHAPE, OP_TRANSPOSE, OP_ROLL, OP_SLICE, OP_WINDOW_PARTITION, OP_WINDOW_REVERSE = 0, 1, 2, 3, 4, 5
 OP_COPY, OP_LINEAR, OP_BMM_NT = 16, 17, 18
 
@@ -38,7 +38,9 @@ class IndexMap(C.Structure):
     _fields_ = [("n_atoms", C.c_int32), ("extent", C.c_int64 * MAX_ATOMS), ("src_stride", C.c_int64 * MAX_ATOMS),
                 ("roll_of", C.c_int32 * MAX_ATOMS), ("roll_weight", C.c_int64 * MAX_ATOMS), ("n_rolls", C.c_int32),
                 ("roll_shift", C.c_int64 * MAX_ROLLS), ("roll_mod", C.c_int64 * MAX_ROLLS),
-                ("roll_stride", C.c_int64 * MAX_ROLLS), ("base", C.c_int64), ("n_elements", C.c_int64),
+                ("roll_stride", C.c_int64 * MAX_ROLLS), ("roll_n_parts", C.c_int32 * MAX_ROLLS),
+                ("roll_part_extent", (C.c_int64 * MAX_ROLLS) * MAX_ROLLS),
+                ("roll_part_stride", (C.c_int64 * MAX_ROLLS) * MAX_ROLLS), ("base", C.c_int64), ("n_elements", C.c_int64),
                 ("vec_elems", C.c_int32), ("klass", C.c_int32)]
 
 

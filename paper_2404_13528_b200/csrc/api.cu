@@ -100,6 +100,31 @@ namespace {
 
 bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
 
+bool make_devseq(const SeqProgram& sp, DevSeq* out) {
+  if (sp.stages.size() > (size_t)kSeqMaxStages || sp.src_shape.size() > (size_t)kSeqMaxDims) return false;
+  memset(out, 0, sizeof(*out));
+  out->n_stages = (int)sp.stages.size();
+  out->n_src = (int)sp.src_shape.size();
+  for (int k = 0; k < out->n_src; ++k) {
+    out->src_shape[k] = sp.src_shape[k];
+    out->src_stride[k] = sp.src_stride[k];
+  }
+  for (int i = 0; i < out->n_stages; ++i) {
+    const SeqStage& a = sp.stages[i];
+    DevSeqStage& d = out->st[i];
+    if (a.in_shape.size() > (size_t)kSeqMaxDims || a.out_shape.size() > (size_t)kSeqMaxDims) return false;
+    d.kind = a.kind; d.n_in = (int)a.in_shape.size(); d.n_out = (int)a.out_shape.size();
+    d.axis = a.axis;
+    if (a.shift > (1ll << 30) || a.shift < -(1ll << 30)) return false;
+    d.shift = (int)a.shift;
+    for (int k = 0; k < d.n_in; ++k) { if (a.in_shape[k] >= (1ll << 31)) return false; d.in_shape[k] = (int)a.in_shape[k]; }
+    for (int k = 0; k < d.n_out; ++k) { if (a.out_shape[k] >= (1ll << 31)) return false; d.out_shape[k] = (int)a.out_shape[k]; }
+    for (size_t k = 0; k < a.perm.size(); ++k) d.aux[k] = a.perm[k];
+    for (size_t k = 0; k < a.start.size(); ++k) d.aux[k] = (int)a.start[k];
+  }
+  return true;
+}
+
 }  // namespace
 
 EXPORT int smartmem_run_chain(const smartmem_plan_t* plan, const void* const* inputs, void* const* outputs,
@@ -123,7 +148,13 @@ EXPORT int smartmem_run_chain(const smartmem_plan_t* plan, const void* const* in
     const int esz = s.dtype == SMARTMEM_F32 ? 4 : 2;
     int rc = SMARTMEM_OK;
     if (s.kind == STEP_COPY) {
-      rc = launch_copy_map(s.map[0], esz, buf(s.src[0]), buf(s.dst), st);
+      if (s.map[0].klass == 3 || (plan->mode == SMARTMEM_ELIMINATE_NAIVE && !s.is_layout_copy)) {
+        DevSeq q;
+        if (!make_devseq(s.seq[0], &q)) return SMARTMEM_ERR_UNSUPPORTED;
+        rc = launch_copy_seq(q, s.map[0].n_elements, esz, buf(s.src[0]), buf(s.dst), st);
+      } else {
+        rc = launch_copy_map(s.map[0], esz, buf(s.src[0]), buf(s.dst), st);
+      }
     } else if (s.kind == STEP_LINEAR || s.kind == STEP_BMM_NT) {
       if (s.dtype != SMARTMEM_BF16) return SMARTMEM_ERR_UNSUPPORTED;
       TcOperand A, B;

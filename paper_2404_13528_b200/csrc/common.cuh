@@ -56,6 +56,9 @@ struct DevMap {
   int weight[kMaxDevAtoms];
   int roll_shift[SMARTMEM_MAX_ROLLS], roll_mod[SMARTMEM_MAX_ROLLS];
   long long roll_stride[SMARTMEM_MAX_ROLLS];
+  int roll_n_parts[SMARTMEM_MAX_ROLLS];                     // > 1: decompose the wrapped coordinate again
+  FastDiv roll_part_ext[SMARTMEM_MAX_ROLLS][SMARTMEM_MAX_ROLLS];
+  long long roll_part_stride[SMARTMEM_MAX_ROLLS][SMARTMEM_MAX_ROLLS];
   long long base;
 };
 
@@ -83,7 +86,16 @@ __device__ __forceinline__ long long devmap_eval(const DevMap& m, uint32_t i) {
   auto wrap = [&](int u, int r) {
     int v = u + m.roll_shift[r];
     if (v >= m.roll_mod[r]) v -= m.roll_mod[r];     // u < mod and shift < mod: one conditional subtract
-    off += (long long)v * m.roll_stride[r];
+    if (m.roll_n_parts[r] <= 1) {
+      off += (long long)v * m.roll_stride[r];
+    } else {
+      uint32_t vv = (uint32_t)v;
+      for (int k = m.roll_n_parts[r] - 1; k >= 0; --k) {
+        const uint32_t q = fd_div(vv, m.roll_part_ext[r][k]);
+        off += (long long)(vv - q * m.roll_part_ext[r][k].d) * m.roll_part_stride[r][k];
+        vv = q;
+      }
+    }
   };
   if (m.n_rolls > 0) wrap(u0, 0);
   if (m.n_rolls > 1) wrap(u1, 1);
@@ -143,6 +155,21 @@ template <> struct ElemIO<__nv_bfloat16> {
 // ---------------------------------------------------------------------------------------
 // Launchers (defined in the .cu files).  All return a smartmem_status_t.
 // ---------------------------------------------------------------------------------------
+// The sequential ("no optimisation") index program of a layout run, for the device: the consumer
+// index is pushed backwards through the stages with one divide/modulo chain per stage.
+constexpr int kSeqMaxStages = 12, kSeqMaxDims = 8;
+struct DevSeqStage {
+  int kind, n_in, n_out, axis, shift;
+  int in_shape[kSeqMaxDims], out_shape[kSeqMaxDims], aux[kSeqMaxDims];   // aux: perm (transpose) or start (slice)
+};
+struct DevSeq {
+  int n_stages, n_src;
+  DevSeqStage st[kSeqMaxStages];
+  long long src_shape[kSeqMaxDims], src_stride[kSeqMaxDims];
+};
+// Copy through the sequential program (any chain; one thread per element, true div/mod).
+int launch_copy_seq(const DevSeq& seq, long long n_elements, int elem_size, const void* src, void* dst, cudaStream_t st);
+
 // Map-driven copy: out (contiguous) <- src through `map`.
 int launch_copy_map(const smartmem_index_map_t& map, int elem_size, const void* src, void* dst, cudaStream_t st);
 

@@ -19,6 +19,12 @@ bool make_devmap(const smartmem_index_map_t& m, int a0, int a1, int unit, bool w
     d.roll_shift[r] = (int)m.roll_shift[r];
     d.roll_mod[r] = (int)m.roll_mod[r];
     d.roll_stride[r] = m.roll_stride[r];
+    d.roll_n_parts[r] = m.roll_n_parts[r];
+    for (int k = 0; k < m.roll_n_parts[r] && k < SMARTMEM_MAX_ROLLS; ++k) {
+      if (m.roll_part_extent[r][k] >= (1ll << 31)) return false;
+      d.roll_part_ext[r][k] = make_fastdiv((uint32_t)m.roll_part_extent[r][k]);
+      d.roll_part_stride[r][k] = m.roll_part_stride[r][k];
+    }
   }
   for (int a = a0; a < a1; ++a) {
     int64_t e = m.extent[a];
@@ -149,7 +155,62 @@ __global__ void __launch_bounds__(256) copy_block_transpose16_kernel(const __gri
   }
 }
 
+// The unoptimised form of an eliminated run (Fig. 4, right): every stage delinearises the index
+// in its output shape and linearises it in its input shape with run-time divides and modulos.
+template <typename E>
+__global__ void __launch_bounds__(256) copy_seq_kernel(const __grid_constant__ DevSeq q, const E* __restrict__ src,
+                                                       E* __restrict__ dst, long long n) {
+  const long long i0 = (long long)blockIdx.x * 256 + threadIdx.x;
+  if (i0 >= n) return;
+  long long idx = i0;
+  for (int si = q.n_stages - 1; si >= 0; --si) {
+    const DevSeqStage& st = q.st[si];
+    long long c[kSeqMaxDims], in[kSeqMaxDims];
+    for (int k = st.n_out - 1; k >= 0; --k) {
+      c[k] = idx % st.out_shape[k];
+      idx /= st.out_shape[k];
+    }
+    if (st.kind == SMARTMEM_OP_RESHAPE) {
+      long long lin = 0;
+      for (int k = 0; k < st.n_out; ++k) lin = lin * st.out_shape[k] + c[k];
+      idx = lin;
+      continue;
+    }
+    for (int k = 0; k < st.n_in; ++k) in[k] = 0;
+    if (st.kind == SMARTMEM_OP_TRANSPOSE) {
+      for (int k = 0; k < st.n_out; ++k) in[st.aux[k]] = c[k];
+    } else if (st.kind == SMARTMEM_OP_ROLL) {
+      for (int k = 0; k < st.n_out; ++k) in[k] = c[k];
+      long long v = (c[st.axis] - st.shift) % st.in_shape[st.axis];
+      in[st.axis] = v < 0 ? v + st.in_shape[st.axis] : v;
+    } else {                                      // slice
+      for (int k = 0; k < st.n_out; ++k) in[k] = c[k] + st.aux[k];
+    }
+    long long lin = 0;
+    for (int k = 0; k < st.n_in; ++k) lin = lin * st.in_shape[k] + in[k];
+    idx = lin;
+  }
+  long long off = 0;
+  for (int k = q.n_src - 1; k >= 0; --k) {
+    off += (idx % q.src_shape[k]) * q.src_stride[k];
+    idx /= q.src_shape[k];
+  }
+  dst[i0] = src[off];
+}
+
 }  // namespace
+
+int launch_copy_seq(const DevSeq& seq, long long n, int elem_size, const void* src, void* dst, cudaStream_t st) {
+  profile_tick("copy_seq", st);
+  if (n == 0) return SMARTMEM_OK;
+  const long long blocks = (n + 255) / 256;
+  if (blocks >= (1ll << 31)) return SMARTMEM_ERR_UNSUPPORTED;
+  if (elem_size == 2) copy_seq_kernel<uint16_t><<<(unsigned)blocks, 256, 0, st>>>(seq, (const uint16_t*)src, (uint16_t*)dst, n);
+  else if (elem_size == 4) copy_seq_kernel<uint32_t><<<(unsigned)blocks, 256, 0, st>>>(seq, (const uint32_t*)src, (uint32_t*)dst, n);
+  else return SMARTMEM_ERR_UNSUPPORTED;
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
+}
 
 int launch_copy_map(const smartmem_index_map_t& map, int elem_size, const void* src, void* dst, cudaStream_t st) {
   profile_tick("copy_map", st);

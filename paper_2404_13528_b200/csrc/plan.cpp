@@ -29,6 +29,7 @@ struct Atom {
 };
 struct RollD {
   int64_t shift, mod, stride;
+  std::vector<int64_t> part_extent, part_stride;   // more than one part: the rolled dim is not affine in the source
 };
 
 struct TState {
@@ -142,7 +143,19 @@ void do_roll(TState& s, int axis, int64_t shift) {
   if (nested_weights(d, w)) {
     if ((int)s.rolls.size() >= SMARTMEM_MAX_ROLLS) { s.canonical = false; return; }
     int r = (int)s.rolls.size();
-    s.rolls.push_back({sp, N, d.back().stride});
+    s.rolls.push_back({sp, N, d.back().stride, {N}, {d.back().stride}});
+    for (size_t i = 0; i < d.size(); ++i) { d[i].roll = r; d[i].weight = w[i]; d[i].stride = 0; }
+    return;
+  }
+  bool all_plain = !d.empty();
+  for (auto& a : d) all_plain = all_plain && a.roll < 0;
+  if (all_plain && (int)d.size() <= SMARTMEM_MAX_ROLLS && (int)s.rolls.size() < SMARTMEM_MAX_ROLLS) {
+    // merged from factors that do not nest in the source: the rolled coordinate is decomposed
+    // again over these factors after the wrap
+    int r = (int)s.rolls.size();
+    RollD rd{sp, N, 0, {}, {}};
+    for (auto& a : d) { rd.part_extent.push_back(a.extent); rd.part_stride.push_back(a.stride); }
+    s.rolls.push_back(rd);
     for (size_t i = 0; i < d.size(); ++i) { d[i].roll = r; d[i].weight = w[i]; d[i].stride = 0; }
     return;
   }
@@ -303,7 +316,7 @@ int finalize_map(const TState& s, const std::vector<int>& group_end, int elem_si
     for (int k = dim0; k < group_end[g]; ++k)
       for (Atom a : s.dims[k]) {
         if (a.extent == 1) continue;
-        if (a.roll >= 0 && s.rolls[a.roll].shift == 0) {    // shifts cancelled: a plain affine atom again
+        if (a.roll >= 0 && s.rolls[a.roll].shift == 0 && s.rolls[a.roll].part_extent.size() == 1) {   // shifts cancelled: a plain affine atom again
           a.stride = a.weight * s.rolls[a.roll].stride;
           a.roll = -1;
           a.weight = 0;
@@ -336,9 +349,18 @@ int finalize_map(const TState& s, const std::vector<int>& group_end, int elem_si
       m->roll_shift[m->n_rolls] = s.rolls[r].shift;
       m->roll_mod[m->n_rolls] = s.rolls[r].mod;
       m->roll_stride[m->n_rolls] = s.rolls[r].stride;
+      m->roll_n_parts[m->n_rolls] = (int)s.rolls[r].part_extent.size();
+      for (size_t k = 0; k < s.rolls[r].part_extent.size(); ++k) {
+        m->roll_part_extent[m->n_rolls][k] = s.rolls[r].part_extent[k];
+        m->roll_part_stride[m->n_rolls][k] = s.rolls[r].part_stride[k];
+      }
       ++m->n_rolls;
     } else {
-      m->base += pmod(s.rolls[r].shift, s.rolls[r].mod) * s.rolls[r].stride;
+      int64_t v = pmod(s.rolls[r].shift, s.rolls[r].mod);
+      for (int k = (int)s.rolls[r].part_extent.size() - 1; k >= 0; --k) {
+        m->base += (v % s.rolls[r].part_extent[k]) * s.rolls[r].part_stride[k];
+        v /= s.rolls[r].part_extent[k];
+      }
     }
   }
   m->n_atoms = (int)out.size();
@@ -360,7 +382,8 @@ int finalize_map(const TState& s, const std::vector<int>& group_end, int elem_si
     shrink(m->base);
     for (int i = 0; i + 1 < m->n_atoms; ++i)
       if (m->roll_of[i] < 0) shrink(m->src_stride[i]);
-    for (int r = 0; r < m->n_rolls; ++r) shrink(m->roll_stride[r]);
+    for (int r = 0; r < m->n_rolls; ++r)
+      for (int k = 0; k < m->roll_n_parts[r]; ++k) shrink(m->roll_part_stride[r][k]);
   }
   m->vec_elems = v;
   if (m->n_rolls > 0) {
@@ -534,7 +557,8 @@ int smartmem_pair_decision(int32_t a, int32_t b, int32_t* action, int32_t* resul
 int smartmem_plan(const smartmem_op_t* ops, int32_t n_ops, const smartmem_tensor_desc_t* inputs, int32_t n_inputs,
                   int32_t mode, smartmem_plan_t** out_plan) {
   if (!ops || !inputs || !out_plan || n_ops < 1 || n_inputs < 1) return SMARTMEM_ERR_INVALID_ARG;
-  if (mode != SMARTMEM_ELIMINATE && mode != SMARTMEM_EXPLICIT) return SMARTMEM_ERR_INVALID_ARG;
+  if (mode != SMARTMEM_ELIMINATE && mode != SMARTMEM_EXPLICIT && mode != SMARTMEM_ELIMINATE_NAIVE)
+    return SMARTMEM_ERR_INVALID_ARG;
   for (int i = 0; i < n_inputs; ++i) {
     if (inputs[i].ndim < 1 || inputs[i].ndim > SMARTMEM_MAX_DIMS) return SMARTMEM_ERR_INVALID_ARG;
     if (inputs[i].dtype != SMARTMEM_F32 && inputs[i].dtype != SMARTMEM_BF16) return SMARTMEM_ERR_INVALID_ARG;
@@ -684,7 +708,13 @@ int64_t smartmem_map_eval(const smartmem_index_map_t* m, int64_t idx) {
     if (m->roll_of[a] < 0) off += digit * m->src_stride[a];
     else u[m->roll_of[a]] += digit * m->roll_weight[a];
   }
-  for (int r = 0; r < m->n_rolls; ++r) off += ((u[r] + m->roll_shift[r]) % m->roll_mod[r]) * m->roll_stride[r];
+  for (int r = 0; r < m->n_rolls; ++r) {
+    int64_t v = (u[r] + m->roll_shift[r]) % m->roll_mod[r];
+    for (int k = m->roll_n_parts[r] - 1; k >= 0; --k) {
+      off += (v % m->roll_part_extent[r][k]) * m->roll_part_stride[r][k];
+      v /= m->roll_part_extent[r][k];
+    }
+  }
   return off;
 }
 

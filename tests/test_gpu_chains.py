@@ -34,7 +34,7 @@ def copy_chain_case(shape, chain, dtype="bf16"):
     ops = _ops_from_chain(chain) + [sm.make_op(sm.OP_COPY)]
     desc = [sm.make_desc(shape, sm.BF16 if dtype == "bf16" else sm.F32)]
     tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
-    for mode in (sm.ELIMINATE, sm.EXPLICIT):
+    for mode in (sm.ELIMINATE, sm.EXPLICIT, sm.ELIMINATE_NAIVE):
         out = run_plan(ops, desc, mode, [xd], ref.shape, tdt)
         assert np.array_equal(to_host_bits(out), ref), f"mode {mode}"
 
@@ -57,8 +57,13 @@ def swin_e1(s, ws):
     ((1, 8, 8, 32), swin_e1(2, 4)),
     ((3, 14, 14, 96), swin_e1(3, 7)),
     ((2, 56, 56, 96), swin_e1(3, 7)),
+    ((2 * 8 * 8, 49, 96), [{"op": "window_reverse", "window": 7, "B": 2, "H": 56, "W": 56},
+                           {"op": "roll", "shift": 3, "axis": 1}, {"op": "roll", "shift": 3, "axis": 2}]),
     ((5, 5, 5), [{"op": "reshape", "shape": (5, 25)}, {"op": "transpose", "perm": (1, 0)}]),
     ((4, 6, 10), [{"op": "slice", "start": (1, 0, 2), "extent": (2, 6, 8)}, {"op": "transpose", "perm": (2, 0, 1)}]),
+    # split points that do not refine each other: only the sequential program can evaluate it
+    ((4, 6), [{"op": "transpose", "perm": (1, 0)}, {"op": "reshape", "shape": (8, 3)}]),
+    ((12, 10, 6), [{"op": "transpose", "perm": (2, 0, 1)}, {"op": "reshape", "shape": (8, 9, 10)}, {"op": "roll", "shift": 2, "axis": 1}]),
 ])
 def test_copy_only_chains_bit_exact(shape, chain):
     copy_chain_case(shape, chain)
