@@ -470,21 +470,53 @@ def main():
                                  "gbs": gbs and round(gbs, 1), "frac_of_hbm_peak": gbs and round(gbs / peaks["hbm_gbs"], 4)})
     dom = max(kernels["eliminate"], key=lambda k: k["ms"])
 
-    # end to end through the C ABI with host buffers
-    e2e_steps = min(args.steps, 30)
-    for i in range(3):
-        xs[0].copy_(x_host, non_blocking=True); step(0, sm.ELIMINATE); y_host.copy_(ys[0], non_blocking=True)
+    # end to end through the C ABI with host buffers: every step copies its input from pinned host
+    # memory and its result back.  Copies and compute run on three streams over the rotating buffer
+    # sets, so the PCIe transfers of neighbouring steps overlap the kernels (each step still has
+    # its own H2D copy, its own block call and its own D2H copy).
+    e2e_steps = min(max(args.steps, 8), 64)
+    y_hosts = [torch.empty_like(x_host).pin_memory() for _ in range(N_SETS)]
+    s_in, s_comp, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
+    ev_in = [torch.cuda.Event() for _ in range(N_SETS)]
+    ev_comp = [torch.cuda.Event() for _ in range(N_SETS)]
+    ev_out = [torch.cuda.Event() for _ in range(N_SETS)]
+
+    def e2e_loop(n):
+        for i in range(n):
+            j = i % N_SETS
+            with torch.cuda.stream(s_in):
+                if i >= N_SETS:
+                    s_in.wait_event(ev_comp[j])             # the block that last read xs[j] is done
+                xs[j].copy_(x_host, non_blocking=True)
+                ev_in[j].record(s_in)
+            with torch.cuda.stream(s_comp):
+                s_comp.wait_event(ev_in[j])
+                if i >= N_SETS:
+                    s_comp.wait_event(ev_out[j])            # ys[j] has been read back
+                sm.smartmem_swin_block(p, xs[j].data_ptr(), ys[j].data_ptr(), wss[j].data_ptr(), wsb[sm.ELIMINATE],
+                                       sm.ELIMINATE, s_comp.cuda_stream)
+                ev_comp[j].record(s_comp)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_comp[j])
+                y_hosts[j].copy_(ys[j], non_blocking=True)
+                ev_out[j].record(s_out)
+
+    e2e_loop(N_SETS)
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for i in range(e2e_steps):
-        j = i % N_SETS
-        xs[j].copy_(x_host, non_blocking=True)
-        step(i, sm.ELIMINATE)
-        y_host.copy_(ys[j], non_blocking=True)
-    e1.record()
+    cur = torch.cuda.current_stream()
+    e0.record(cur)
+    for st_ in (s_in, s_comp, s_out):
+        st_.wait_event(e0)
+    e2e_loop(e2e_steps)
+    for st_ in (s_in, s_comp, s_out):
+        done = torch.cuda.Event()
+        done.record(st_)
+        cur.wait_event(done)
+    e1.record(cur)
     barrier()
     ms_e2e = max_over_ranks(dist, e0.elapsed_time(e1), "cuda")
+    y_host = y_hosts[0]
     clocks = sampler.stop()
 
     cpu = None
