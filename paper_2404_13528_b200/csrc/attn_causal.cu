@@ -9,6 +9,8 @@
 // One CTA = 64 query rows of one head (4 warps x 16 rows); keys/values stream through shared
 // memory in 64-row tiles (cp.async, double buffered); scores never leave registers (online
 // softmax).  Contractions use warp-level mma.sync m16n8k16.
+#include <cstdlib>
+
 #include "attn.cuh"
 #include "ptx.cuh"
 
@@ -204,7 +206,15 @@ __global__ void rope_rows_kernel(__nv_bfloat16* x, long long rows, int S, int Dh
 
 }  // namespace
 
+int launch_causal_attention_tc(const CausalAttnArgs& a, cudaStream_t st);
+
 int launch_causal_attention(const CausalAttnArgs& a, cudaStream_t st) {
+  // tcgen05 path for the two operand layouts it knows; SMARTMEM_CAUSAL_LEGACY=1 keeps the warp-MMA kernel
+  static const bool legacy = [] { const char* e = getenv("SMARTMEM_CAUSAL_LEGACY"); return e && e[0] == '1'; }();
+  if (!legacy) {
+    const int rc = launch_causal_attention_tc(a, st);
+    if (rc != SMARTMEM_ERR_UNSUPPORTED) return rc;
+  }
   if (a.S < 1 || a.heads < 1 || a.batch < 1 || a.heads > 65535 || a.batch > 65535) return SMARTMEM_ERR_UNSUPPORTED;
   const AttnOperand* ops[4] = {&a.q, &a.k, &a.v, &a.o};
   for (auto* o : ops)

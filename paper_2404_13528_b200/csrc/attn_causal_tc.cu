@@ -1,0 +1,346 @@
+// Causal attention (prefill, head dimension 128) on the tcgen05 tensor cores.
+//
+// One CTA = 128 query positions of one head.  K and V stream through shared memory in tiles of
+// 128 keys (TMA, double buffered); S = Q K^T and O += P V are tcgen05.mma with the accumulators in
+// TMEM (two S buffers, one O); four softmax warps own one query row per thread (the TMEM lane),
+// so row maxima and sums need no shuffles.  P goes back to the tensor core through shared memory in
+// the K-major swizzled operand layout; V is consumed as it lies in memory ([key, d] rows) through
+// the MN-major operand mode, so no transpose of V exists anywhere.  The running maximum is only
+// refreshed when it grows by more than 2^8 (then O and the running sum are rescaled), which keeps
+// the TMEM read-modify-write of O off the common path.
+//
+// q, k, v are addressed as TMA boxes inside the buffer the QKV GEMM wrote ([B*S, 3*H*D], head split
+// eliminated) or inside materialised [B, H, S, D] tensors (explicit variant); the output tile is
+// stored at column h*D of [B*S, H*D] (head merge eliminated) or into [B, H, S, D].
+#include "attn.cuh"
+#include "gemm_tc.cuh"
+#include "ptx.cuh"
+
+namespace smartmem {
+namespace {
+
+constexpr int BQ = 128, BKV = 128, D = 128;
+constexpr int KB = 128 * 64 * 2;                      // one 128 x 64 bf16 block
+constexpr uint32_t TM_S = 0, TM_O = 256, TMEM_COLS = 512;
+constexpr int kThreads = 192;
+constexpr float kRescaleThreshold = 8.0f;             // log2 units
+
+struct TcAttnArgs {
+  int S, heads, batch, n_qt;
+  int q_col0, k_col0, v_col0, col_per_head;           // TMA column of (operand, head): col0 + h * col_per_head
+  long long row_per_batch, row_per_head;              // TMA row of (b, h, t): b * row_per_batch + h * row_per_head + t
+  __nv_bfloat16* out;
+  long long o_sn, o_sh, o_st;
+  float scale_log2;
+  int* status;
+};
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+      "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),
+      "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
+      "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__global__ void __launch_bounds__(kThreads, 1)
+causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                      const __grid_constant__ CUtensorMap tmV, const __grid_constant__ TcAttnArgs g) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
+  uint8_t* sQ = smem;                                  // [2 k-blocks][16 KB]
+  uint8_t* sK = sQ + 2 * KB;                           // [2 stages][2 k-blocks][16 KB]
+  uint8_t* sV = sK + 4 * KB;                           // [2 stages][2 d-chunks][16 KB]
+  uint8_t* sP = sV + 4 * KB;                           // [2 k-blocks][16 KB]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sP + 2 * KB);
+  uint64_t *q_full = bars, *k_full = bars + 1, *k_empty = bars + 3, *v_full = bars + 5, *v_empty = bars + 7;
+  uint64_t *s_full = bars + 9, *s_empty = bars + 11, *p_full = bars + 13, *p_empty = bars + 14, *o_done = bars + 15;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
+  int* abort_flag = reinterpret_cast<int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // heaviest units (last query tiles) first
+  const int bh_count = g.batch * g.heads;
+  const int qt = g.n_qt - 1 - (int)(blockIdx.x / bh_count);
+  const int bh = (int)(blockIdx.x % bh_count);
+  const int b = bh / g.heads, h = bh - b * g.heads;
+  const int n_kv = qt + 1;
+  const long long row_base = (long long)b * g.row_per_batch + (long long)h * g.row_per_head;
+
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(q_full, 1);
+    for (int i = 0; i < 2; ++i) {
+      ptx::mbar_init(&k_full[i], 1);
+      ptx::mbar_init(&k_empty[i], 1);
+      ptx::mbar_init(&v_full[i], 1);
+      ptx::mbar_init(&v_empty[i], 1);
+      ptx::mbar_init(&s_full[i], 1);
+      ptx::mbar_init(&s_empty[i], 4);
+    }
+    ptx::mbar_init(p_full, 4);
+    ptx::mbar_init(p_empty, 1);
+    ptx::mbar_init(o_done, 1);
+    *abort_flag = 0;
+    ptx::fence_barrier_init();
+    ptx::fence_proxy_async();
+  }
+  if (warp == 0 && lane == 0) {
+    ptx::prefetch_tensormap(&tmQ);
+    ptx::prefetch_tensormap(&tmK);
+    ptx::prefetch_tensormap(&tmV);
+  }
+  if (warp == 1) ptx::tmem_alloc(tmem_slot, TMEM_COLS);
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      const int qc = g.q_col0 + h * g.col_per_head, kc = g.k_col0 + h * g.col_per_head, vc = g.v_col0 + h * g.col_per_head;
+      ptx::mbar_expect_tx(q_full, 2 * KB);
+      for (int kb = 0; kb < 2; ++kb) ptx::tma_load_2d(sQ + kb * KB, &tmQ, q_full, qc + kb * 64, (int)(row_base + qt * BQ));
+      bool ok = true;
+      for (int j = 0; j < n_kv && ok; ++j) {
+        const int s = j & 1;
+        const uint32_t ph = (j >> 1) & 1;
+        const int krow = (int)(row_base + (long long)j * BKV);
+        ok = ptx::mbar_wait(&k_empty[s], ph ^ 1, abort_flag, g.status);
+        if (!ok) break;
+        ptx::mbar_expect_tx(&k_full[s], 2 * KB);
+        for (int kb = 0; kb < 2; ++kb) ptx::tma_load_2d(sK + (s * 2 + kb) * KB, &tmK, &k_full[s], kc + kb * 64, krow);
+        ok = ptx::mbar_wait(&v_empty[s], ph ^ 1, abort_flag, g.status);
+        if (!ok) break;
+        ptx::mbar_expect_tx(&v_full[s], 2 * KB);
+        for (int dc = 0; dc < 2; ++dc) ptx::tma_load_2d(sV + (s * 2 + dc) * KB, &tmV, &v_full[s], vc + dc * 64, krow);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc_s = ptx::make_idesc_bf16(BQ, BKV, false, false);
+      const uint32_t idesc_pv = ptx::make_idesc_bf16(BQ, D, false, true);      // V: MN-major B operand
+      bool ok = ptx::mbar_wait(q_full, 0, abort_flag, g.status);
+      auto issue_s = [&](int j) {
+        const int s = j & 1;
+        const uint32_t ph = (j >> 1) & 1;
+        ok = ok && ptx::mbar_wait(&s_empty[s], ph ^ 1, abort_flag, g.status);
+        ok = ok && ptx::mbar_wait(&k_full[s], ph, abort_flag, g.status);
+        if (!ok) return;
+        ptx::tc_fence_after();
+        for (int kb = 0; kb < 2; ++kb) {
+          const uint32_t a0 = ptx::smem_u32(sQ + kb * KB), b0 = ptx::smem_u32(sK + (s * 2 + kb) * KB);
+          for (int k = 0; k < 4; ++k)
+            ptx::tc_mma_bf16(tmem_base + TM_S + s * BKV, ptx::make_smem_desc(a0 + k * 32, 16, 1024),
+                             ptx::make_smem_desc(b0 + k * 32, 16, 1024), idesc_s, (kb | k) ? 1u : 0u);
+        }
+        ptx::tc_commit(&k_empty[s]);
+        ptx::tc_commit(&s_full[s]);
+      };
+      auto issue_pv = [&](int j) {
+        const int s = j & 1;
+        ok = ok && ptx::mbar_wait(p_full, j & 1, abort_flag, g.status);
+        ok = ok && ptx::mbar_wait(&v_full[s], (j >> 1) & 1, abort_flag, g.status);
+        if (!ok) return;
+        ptx::tc_fence_after();
+        const uint32_t p0 = ptx::smem_u32(sP), v0 = ptx::smem_u32(sV + s * 2 * KB);
+        for (int ks = 0; ks < 8; ++ks)                 // 16 keys per step
+          ptx::tc_mma_bf16(tmem_base + TM_O, ptx::make_smem_desc(p0 + (ks >> 2) * KB + (ks & 3) * 32, 16, 1024),
+                           ptx::make_smem_desc(v0 + ks * 2048, KB, 1024), idesc_pv, (j | ks) ? 1u : 0u);
+        ptx::tc_commit(&v_empty[s]);
+        ptx::tc_commit(p_empty);
+      };
+      issue_s(0);
+      for (int j = 0; j < n_kv && ok; ++j) {
+        if (j + 1 < n_kv) issue_s(j + 1);
+        issue_pv(j);
+      }
+      if (ok) ptx::tc_commit(o_done);
+    }
+  } else {
+    const int q = warp & 3;                            // TMEM lane quadrant
+    const int r = q * 32 + lane;                       // query row inside the tile
+    const int qi = qt * BQ + r;                        // position
+    const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
+    float m_used = -INFINITY, l = 0.f;
+    bool ok = true;
+    for (int j = 0; j < n_kv && ok; ++j) {
+      const int sb = j & 1;
+      ok = ptx::mbar_wait(&s_full[sb], (j >> 1) & 1, abort_flag, g.status);
+      if (!ok) break;
+      ptx::tc_fence_after();
+      const uint32_t ts = tmem_base + TM_S + sb * BKV + lane_addr;
+      const bool diag = (j == qt);
+      const int kj0 = j * BKV;
+      // pass 1: row maximum (log2 domain)
+      float mx = -INFINITY;
+#pragma unroll 1
+      for (int ch = 0; ch < 4; ++ch) {
+        uint32_t rv[32];
+        ptx::tmem_ld32(ts + ch * 32, rv);
+        ptx::tmem_ld_wait();
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+          const float v = __uint_as_float(rv[c]) * g.scale_log2;
+          if (!diag || kj0 + ch * 32 + c <= qi) mx = fmaxf(mx, v);
+        }
+      }
+      float corr = 1.f;
+      bool rescale = false;
+      if (mx > m_used + kRescaleThreshold) {           // (first tile: m_used = -inf)
+        corr = ex2(m_used - mx);                       // 0 on the first tile
+        l *= corr;
+        m_used = mx;
+        rescale = j > 0;
+      }
+      // pass 2: p = 2^(s - m), packed to bf16 for the second MMA
+      uint32_t pk[64];
+#pragma unroll
+      for (int ch = 0; ch < 4; ++ch) {
+        uint32_t rv[32];
+        ptx::tmem_ld32(ts + ch * 32, rv);
+        ptx::tmem_ld_wait();
+#pragma unroll
+        for (int c = 0; c < 32; c += 2) {
+          float p0 = ex2(fmaf(__uint_as_float(rv[c]), g.scale_log2, -m_used));
+          float p1 = ex2(fmaf(__uint_as_float(rv[c + 1]), g.scale_log2, -m_used));
+          if (diag) {
+            if (kj0 + ch * 32 + c > qi) p0 = 0.f;
+            if (kj0 + ch * 32 + c + 1 > qi) p1 = 0.f;
+          }
+          l += p0 + p1;
+          pk[ch * 16 + c / 2] = float2_to_bf16x2(p0, p1);
+        }
+      }
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&s_empty[sb]);   // this warp has read its part of the S buffer
+      // the previous P V must have completed before P is overwritten or O rescaled
+      ok = ptx::mbar_wait(p_empty, (j & 1) ^ 1, abort_flag, g.status);
+      if (!ok) break;
+      ptx::tc_fence_after();
+      if (__any_sync(0xFFFFFFFFu, rescale)) {
+        const uint32_t to = tmem_base + TM_O + lane_addr;
+#pragma unroll 1
+        for (int ch = 0; ch < 4; ++ch) {
+          uint32_t rv[32];
+          ptx::tmem_ld32(to + ch * 32, rv);
+          ptx::tmem_ld_wait();
+#pragma unroll
+          for (int c = 0; c < 32; ++c) rv[c] = __float_as_uint(__uint_as_float(rv[c]) * (rescale ? corr : 1.f));
+          tmem_st32(to + ch * 32, rv);
+        }
+        tmem_st_wait();
+      }
+      // P row r: 16 chunks of 8 keys; chunk c8 lives in k-block c8 / 8 at position (c8 % 8) ^ (r % 8)
+#pragma unroll
+      for (int c8 = 0; c8 < 16; ++c8) {
+        const uint4 v4 = make_uint4(pk[c8 * 4 + 0], pk[c8 * 4 + 1], pk[c8 * 4 + 2], pk[c8 * 4 + 3]);
+        *reinterpret_cast<uint4*>(sP + (c8 >> 3) * KB + r * 128 + (((c8 & 7) ^ (r & 7)) << 4)) = v4;
+      }
+      ptx::fence_proxy_async();
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(p_full);
+    }
+    if (ok) ok = ptx::mbar_wait(o_done, 0, abort_flag, g.status);
+    if (ok) {
+      ptx::tc_fence_after();
+      const float inv = 1.f / l;
+      __nv_bfloat16* orow = g.out + (long long)b * g.o_sn + (long long)h * g.o_sh + (long long)qi * g.o_st;
+      const uint32_t to = tmem_base + TM_O + lane_addr;
+#pragma unroll 1
+      for (int ch = 0; ch < 4; ++ch) {
+        uint32_t rv[32];
+        ptx::tmem_ld32(to + ch * 32, rv);
+        ptx::tmem_ld_wait();
+        if (qi < g.S) {
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            float o8[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) o8[e] = __uint_as_float(rv[v * 8 + e]) * inv;
+            ElemIO<__nv_bfloat16>::store(orow + ch * 32 + v * 8, o8);
+          }
+        }
+      }
+    }
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+}  // namespace
+
+// Returns SMARTMEM_ERR_UNSUPPORTED when the operand layout is neither of the two it knows.
+int launch_causal_attention_tc(const CausalAttnArgs& a, cudaStream_t st) {
+  const long long S = a.S, H = a.heads, B = a.batch;
+  if (S < 1 || H < 1 || B < 1) return SMARTMEM_ERR_UNSUPPORTED;
+  const AttnOperand* ops[3] = {&a.q, &a.k, &a.v};
+  for (auto* o : ops)
+    if (o->se != 1 || ((uintptr_t)o->ptr & 15)) return SMARTMEM_ERR_UNSUPPORTED;
+  if (a.o.se != 1 || a.o.st % 8 || a.o.sn % 8 || a.o.sh % 8 || ((uintptr_t)a.o.ptr & 15)) return SMARTMEM_ERR_UNSUPPORTED;
+  TcAttnArgs g;
+  memset(&g, 0, sizeof(g));
+  CUtensorMap tq, tk, tv;
+  int rc;
+  const long long st_ = a.q.st;
+  const bool interleaved = a.q.sh == D && a.k.sh == D && a.v.sh == D && a.k.st == st_ && a.v.st == st_ &&
+                           a.q.sn == S * st_ && a.k.sn == S * st_ && a.v.sn == S * st_ && st_ % 8 == 0;
+  const bool head_major = a.q.st == D && a.k.st == D && a.v.st == D && a.q.sh == S * D && a.k.sh == S * D &&
+                          a.v.sh == S * D && a.q.sn == H * S * D && a.k.sn == H * S * D && a.v.sn == H * S * D;
+  if (interleaved) {
+    // one [B*S, row pitch] matrix holds q, k and v side by side; columns are offsets from q
+    const long long kcol = ((const char*)a.k.ptr - (const char*)a.q.ptr) / 2, vcol = ((const char*)a.v.ptr - (const char*)a.q.ptr) / 2;
+    if (kcol < 0 || vcol < 0 || kcol + H * D > st_ || vcol + H * D > st_) return SMARTMEM_ERR_UNSUPPORTED;
+    if ((rc = tc_encode_2d(a.q.ptr, st_, B * S, st_, 64, 128, &tq)) != SMARTMEM_OK) return rc;
+    tk = tq;
+    tv = tq;
+    g.q_col0 = 0; g.k_col0 = (int)kcol; g.v_col0 = (int)vcol; g.col_per_head = D;
+    g.row_per_batch = S; g.row_per_head = 0;
+  } else if (head_major) {
+    if ((rc = tc_encode_2d(a.q.ptr, D, B * H * S, D, 64, 128, &tq)) != SMARTMEM_OK) return rc;
+    if ((rc = tc_encode_2d(a.k.ptr, D, B * H * S, D, 64, 128, &tk)) != SMARTMEM_OK) return rc;
+    if ((rc = tc_encode_2d(a.v.ptr, D, B * H * S, D, 64, 128, &tv)) != SMARTMEM_OK) return rc;
+    g.col_per_head = 0;
+    g.row_per_batch = H * S; g.row_per_head = S;
+  } else {
+    return SMARTMEM_ERR_UNSUPPORTED;
+  }
+  if (B * H * S >= (1ll << 31)) return SMARTMEM_ERR_UNSUPPORTED;
+  g.S = (int)S; g.heads = (int)H; g.batch = (int)B;
+  g.n_qt = (int)((S + BQ - 1) / BQ);
+  g.out = (__nv_bfloat16*)a.o.ptr;
+  g.o_sn = a.o.sn; g.o_sh = a.o.sh; g.o_st = a.o.st;
+  g.scale_log2 = a.scale * 1.4426950408889634f;
+  g.status = device_status_ptr();
+  if (!g.status) return SMARTMEM_ERR_CUDA;
+  const size_t smem = 1024 + 12 * KB + 16 * 8 + 16;
+  static bool configured = false;
+  if (!configured) {
+    if (cudaFuncSetAttribute(causal_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return SMARTMEM_ERR_CUDA;
+    configured = true;
+  }
+  const long long ctas = (long long)g.n_qt * B * H;
+  if (ctas >= (1ll << 31)) return SMARTMEM_ERR_UNSUPPORTED;
+  profile_tick("causal_attention_tc", st);
+  causal_attn_tc_kernel<<<(unsigned)ctas, kThreads, smem, st>>>(tq, tk, tv, g);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
+}
+
+}  // namespace smartmem
