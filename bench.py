@@ -257,7 +257,7 @@ def run_other(args):
             sm.smartmem_attn_layer(p, xs[j].data_ptr(), ys[j].data_ptr(), wss[j].data_ptr(), wsb[mode], mode, stream)
         tokens = S
         X = S * hidden * 2
-        model = [("rope_table", S * 64 * 8, 0), ("rmsnorm", 2 * X, 0), ("qkv_gemm_rope", 4 * X + 3 * hidden * hidden * 2, 2 * S * hidden * 3 * hidden),
+        model = [("rmsnorm", 2 * X, 0), ("qkv_gemm_rope", 4 * X + 3 * hidden * hidden * 2, 2 * S * hidden * 3 * hidden),
                  ("causal_attention", 4 * X, 4 * heads * 128 * S * (S + 1) // 2), ("o_proj_gemm", 2 * X + hidden * hidden * 2, 2 * S * hidden * hidden)]
     else:
         which = "2a" if "2a" in name else "2b"

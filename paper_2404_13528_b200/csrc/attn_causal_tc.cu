@@ -181,19 +181,21 @@ causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       const uint32_t ts = tmem_base + TM_S + sb * BKV + lane_addr;
       const bool diag = (j == qt);
       const int kj0 = j * BKV;
-      // pass 1: row maximum (log2 domain)
-      float mx = -INFINITY;
-#pragma unroll 1
-      for (int ch = 0; ch < 4; ++ch) {
-        uint32_t rv[32];
-        ptx::tmem_ld32(ts + ch * 32, rv);
-        ptx::tmem_ld_wait();
+      // the whole score row of this thread: four loads in flight, one wait
+      uint32_t rv[128];
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-          const float v = __uint_as_float(rv[c]) * g.scale_log2;
-          if (!diag || kj0 + ch * 32 + c <= qi) mx = fmaxf(mx, v);
-        }
+      for (int ch = 0; ch < 4; ++ch) ptx::tmem_ld32(ts + ch * 32, rv + ch * 32);
+      ptx::tmem_ld_wait();
+      float mx = -INFINITY;                            // row maximum (log2 domain)
+      if (diag) {
+#pragma unroll
+        for (int c = 0; c < 128; ++c)
+          if (kj0 + c <= qi) mx = fmaxf(mx, __uint_as_float(rv[c]));
+      } else {
+#pragma unroll
+        for (int c = 0; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(rv[c]));
       }
+      mx *= g.scale_log2;                              // the scale is positive
       float corr = 1.f;
       bool rescale = false;
       if (mx > m_used + kRescaleThreshold) {           // (first tile: m_used = -inf)
@@ -202,25 +204,22 @@ causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         m_used = mx;
         rescale = j > 0;
       }
-      // pass 2: p = 2^(s - m), packed to bf16 for the second MMA
+      // p = 2^(s - m), packed to bf16 for the second MMA
       uint32_t pk[64];
+      float l0 = 0.f, l1 = 0.f;
 #pragma unroll
-      for (int ch = 0; ch < 4; ++ch) {
-        uint32_t rv[32];
-        ptx::tmem_ld32(ts + ch * 32, rv);
-        ptx::tmem_ld_wait();
-#pragma unroll
-        for (int c = 0; c < 32; c += 2) {
-          float p0 = ex2(fmaf(__uint_as_float(rv[c]), g.scale_log2, -m_used));
-          float p1 = ex2(fmaf(__uint_as_float(rv[c + 1]), g.scale_log2, -m_used));
-          if (diag) {
-            if (kj0 + ch * 32 + c > qi) p0 = 0.f;
-            if (kj0 + ch * 32 + c + 1 > qi) p1 = 0.f;
-          }
-          l += p0 + p1;
-          pk[ch * 16 + c / 2] = float2_to_bf16x2(p0, p1);
+      for (int c = 0; c < 128; c += 2) {
+        float p0 = ex2(fmaf(__uint_as_float(rv[c]), g.scale_log2, -m_used));
+        float p1 = ex2(fmaf(__uint_as_float(rv[c + 1]), g.scale_log2, -m_used));
+        if (diag) {
+          if (kj0 + c > qi) p0 = 0.f;
+          if (kj0 + c + 1 > qi) p1 = 0.f;
         }
+        l0 += p0;
+        l1 += p1;
+        pk[c / 2] = float2_to_bf16x2(p0, p1);
       }
+      l += l0 + l1;
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&s_empty[sb]);   // this warp has read its part of the S buffer

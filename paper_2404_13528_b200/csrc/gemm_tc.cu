@@ -47,7 +47,7 @@ struct GemmArgs {
   const __nv_bfloat16* residual;
   int gelu, has_rowmap;
   int rope_cols, rope_S;                 // columns [0, rope_cols) are rotated; position = row % rope_S
-  const float2* rope_tab;                // [rope_S, 64] (cos, sin)
+  float rope_c;                          // log2(theta) / 64
   int* status;
   DevMap rowmap;
 };
@@ -266,16 +266,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             uint32_t rw[RC];
             ptx::tmem_ld_cols<RC>(taddr + (rd < RH ? c0 + 64 : c0 - 64), rw);
             ptx::tmem_ld_wait();
-            // this thread's RC (cos, sin) pairs are contiguous: 16-byte loads, whole sectors used
-            const float4* tab4 = reinterpret_cast<const float4*>(g.rope_tab + (long long)(row_ok ? row % g.rope_S : 0) * 64 +
-                                                                 (grp & 1) * 32 + RC * (rd % RH));
+            // angle = position * theta^(-i/64), reduced mod 2 pi in two steps, then the hardware
+            // sine / cosine: no table traffic (a [S, 64] table read 16 bytes per lane per row
+            // slowed the whole kernel by a fifth)
+            const float pos = (float)(row_ok ? row % g.rope_S : 0);
+            const int i0 = (grp & 1) * 32 + RC * (rd % RH);
 #pragma unroll
-            for (int j = 0; j < RC; j += 2) {
-              const float4 cs = __ldg(tab4 + j / 2);
-              const float x0 = __uint_as_float(rv[j]), y0 = __uint_as_float(rw[j]);
-              const float x1 = __uint_as_float(rv[j + 1]), y1 = __uint_as_float(rw[j + 1]);
-              acc[j] = rd < RH ? x0 * cs.x - y0 * cs.y : x0 * cs.x + y0 * cs.y;
-              acc[j + 1] = rd < RH ? x1 * cs.z - y1 * cs.w : x1 * cs.z + y1 * cs.w;
+            for (int j = 0; j < RC; ++j) {
+              float f;
+              asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(f) : "f"(-(float)(i0 + j) * g.rope_c));
+              const float ang = pos * f;
+              const float kk = rintf(ang * 0.15915494309189535f);
+              float red = fmaf(-kk, 6.2831854820251465f, ang);
+              red = fmaf(kk, 1.7484556e-7f, red);
+              const float sn = __sinf(red), cs = __cosf(red);
+              const float x = __uint_as_float(rv[j]), y = __uint_as_float(rw[j]);
+              acc[j] = rd < RH ? x * cs - y * sn : x * cs + y * sn;
             }
           } else {
             ptx::tmem_ld_wait();
@@ -564,7 +570,7 @@ int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep,
   else if (N % 128 == 0) bn = 128;
   else if (N % 96 == 0) bn = 96;
   else if (N % 64 == 0) bn = 64;
-  if (ep.rope_cols > 0 && (N % 256 || ep.rope_cols % 256 || !ep.rope_tab || ep.rope_S < 1)) return SMARTMEM_ERR_UNSUPPORTED;
+  if (ep.rope_cols > 0 && (N % 256 || ep.rope_cols % 256 || ep.rope_S < 1)) return SMARTMEM_ERR_UNSUPPORTED;
   const int nkb = (int)((K + BK - 1) / BK);
   const int stages = (bn == 256 && nkb <= 3) ? 3 : 4;   // short K: wider store rounds instead of a 4th stage
   GemmArgs g;
@@ -585,7 +591,7 @@ int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep,
   if (ep.rowmap) g.rowmap = *ep.rowmap;
   g.rope_cols = ep.rope_cols;
   g.rope_S = ep.rope_S;
-  g.rope_tab = (const float2*)ep.rope_tab;
+  g.rope_c = ep.rope_log2_theta / 64.0f;
   g.status = device_status_ptr();
   if (!g.status) return SMARTMEM_ERR_CUDA;
   g.tiles_n = (int)((N + bn - 1) / bn);

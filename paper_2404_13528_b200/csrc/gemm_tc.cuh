@@ -27,7 +27,7 @@ struct TcEpilogue {
   int gelu;
   const DevMap* rowmap;      // output row -> element offset, or null
   int rope_cols, rope_S;     // rotate columns [0, rope_cols) in 128-wide heads; position = row % rope_S
-  const void* rope_tab;      // float2 [rope_S, 64]
+  float rope_log2_theta;     // angle of pair i at position p: p * 2^(-i/64 * rope_log2_theta)
 };
 
 int tc_operand_from_map(const smartmem_index_map_t& m, int n_batch_atoms, int n_row_atoms, const void* ptr,

@@ -112,14 +112,14 @@ EXPORT int smartmem_attn_layer(const smartmem_attn_params_t* pp, const void* x, 
   float* tab = (float*)at(L.tab);
 
 #define SM_TRY(expr) do { rc = (expr); if (rc != SMARTMEM_OK) return rc; } while (0)
-  SM_TRY(launch_rope_table(tab, (int)S, (int)D, p.rope_theta, st));
+  if (!elim) SM_TRY(launch_rope_table(tab, (int)S, (int)D, p.rope_theta, st));   // only the stand-alone RoPE pass reads it
   SM_TRY(launch_norm(SMARTMEM_BF16, true, x, at(L.xn), p.rms_g, nullptr, p.rms_eps, M, (int)hid, nullptr, st));
   {
     TcEpilogue ep;
     memset(&ep, 0, sizeof(ep));
     ep.out = at(L.qkv);
     ep.ldc = 3 * hid;
-    if (elim) { ep.rope_cols = (int)(2 * hid); ep.rope_S = (int)S; ep.rope_tab = tab; }
+    if (elim) { ep.rope_cols = (int)(2 * hid); ep.rope_S = (int)S; ep.rope_log2_theta = log2f(p.rope_theta); }
     SM_TRY(launch_gemm_tc(tc_operand_plain(at(L.xn), M, hid, hid), tc_operand_plain(p.w_qkv, 3 * hid, hid, hid), ep, 1, M,
                           3 * hid, hid, st));
   }
