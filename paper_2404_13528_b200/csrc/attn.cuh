@@ -20,6 +20,18 @@ struct WinAttnArgs {
   float scale;
 };
 int launch_window_attention(const WinAttnArgs& a, int dtype, long long n_windows, cudaStream_t st);
+int launch_window_attention_tc(const WinAttnArgs& a, long long n_windows, cudaStream_t st);
+
+#ifdef __CUDACC__
+// Region label of token (ty, tx) of window (wy, wx) of a shifted block, in shifted coordinates:
+// 3 * r(row) + r(col) with r = 0 before the last window, 1 in its unwrapped part, 2 in the wrapped part.
+__device__ __forceinline__ int region_label2(int ty, int tx, int ws, int wy, int wx, int H, int W, int shift) {
+  const int hp = wy * ws + ty, wp = wx * ws + tx;
+  const int rh = hp < H - ws ? 0 : (hp < H - shift ? 1 : 2);
+  const int rw = wp < W - ws ? 0 : (wp < W - shift ? 1 : 2);
+  return 3 * rh + rw;
+}
+#endif
 
 // Causal attention over [S] positions for `heads` heads of dimension 128 (bf16).
 struct CausalAttnArgs {

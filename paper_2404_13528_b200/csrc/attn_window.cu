@@ -16,6 +16,8 @@
 // T = ws*ws <= 64 and d <= 32 make tiles far smaller than a tcgen05 instruction (128 x N), and the
 // kernel is bound by HBM traffic (it reads 3 M C and writes M C elements for 4 M T d flops), so the
 // contractions use warp-level mma.sync m16n8k16: four warps, 16 query rows each.
+#include <cstdlib>
+
 #include "attn.cuh"
 #include "ptx.cuh"
 
@@ -29,13 +31,6 @@ __device__ __forceinline__ const T* unit_ptr(const AttnOperand& o, int n, int h)
   return (const T*)o.ptr + (long long)n * o.sn + (long long)h * o.sh;
 }
 
-// Region label of token (ty, tx) of window (wy, wx) in shifted coordinates.
-__device__ __forceinline__ int region_label2(int ty, int tx, int ws, int wy, int wx, int H, int W, int shift) {
-  const int hp = wy * ws + ty, wp = wx * ws + tx;
-  const int rh = hp < H - ws ? 0 : (hp < H - shift ? 1 : 2);
-  const int rw = wp < W - ws ? 0 : (wp < W - shift ? 1 : 2);
-  return 3 * rh + rw;
-}
 __device__ __forceinline__ int region_label(int t, int ws, int wy, int wx, int H, int W, int shift) {
   const int hp = wy * ws + t / ws, wp = wx * ws + t % ws;
   const int rh = hp < H - ws ? 0 : (hp < H - shift ? 1 : 2);
@@ -351,9 +346,9 @@ int launch_window_attention(const WinAttnArgs& a, int dtype, long long n_windows
   if (a.T < 1 || a.T > TP || a.ws * a.ws != a.T || (2 * a.ws - 1) * (2 * a.ws - 1) > 256) return SMARTMEM_ERR_UNSUPPORTED;
   long long units = n_windows * a.heads;
   if (units < 1 || units >= (1ll << 31)) return SMARTMEM_ERR_UNSUPPORTED;
-  profile_tick("window_attention", st);
   if (dtype == SMARTMEM_F32) {
     if (a.d > 32) return SMARTMEM_ERR_UNSUPPORTED;
+    profile_tick("window_attention_f32", st);
     win_attn_f32_kernel<<<(unsigned)units, 128, 0, st>>>(a);
   } else {
     // vector loads need 16-byte aligned rows when the element stride is 1
@@ -362,6 +357,11 @@ int launch_window_attention(const WinAttnArgs& a, int dtype, long long n_windows
       if (o->se == 1 && (o->st % 8 || o->sn % 8 || o->sh % 8 || ((uintptr_t)o->ptr & 15))) return SMARTMEM_ERR_ALIGNMENT;
     if (a.o.se != 1 || a.o.st % 8 || a.o.sn % 8 || a.o.sh % 8 || ((uintptr_t)a.o.ptr & 15)) return SMARTMEM_ERR_ALIGNMENT;
     if (a.d != 16 && a.d != 32) return SMARTMEM_ERR_UNSUPPORTED;
+    static const bool legacy = [] { const char* e = getenv("SMARTMEM_WINDOW_LEGACY"); return e && e[0] == '1'; }();
+    if (!legacy) {
+      const int rc = launch_window_attention_tc(a, n_windows, st);
+      if (rc != SMARTMEM_ERR_UNSUPPORTED) return rc;
+    }
     WinAttnArgs b = a;
     b.n_windows = (int)n_windows;
     b.nWh = a.win_per_img / a.nWw;
@@ -374,6 +374,7 @@ int launch_window_attention(const WinAttnArgs& a, int dtype, long long n_windows
     if (per_head < 1) per_head = 1;
     if (per_head > n_windows) per_head = n_windows;
     const unsigned grid = (unsigned)(per_head * a.heads);
+    profile_tick("window_attention", st);
     if (a.d == 32) win_attn_bf16_kernel<32><<<grid, 128, 0, st>>>(b);
     else win_attn_bf16_kernel<16><<<grid, 128, 0, st>>>(b);
   }

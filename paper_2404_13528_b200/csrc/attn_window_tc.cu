@@ -1,0 +1,420 @@
+// Window attention (head dimension 32, T = ws*ws <= 64) on the tcgen05 tensor cores.
+//
+// Two windows of one head share a 128-row MMA tile: S = [Q0; Q1] [K0; K1]^T is computed as one
+// 128 x 128 x 32 product (only its two diagonal 64 x 64 blocks are used) and O = P [V0; V1] as one
+// 128 x 32 x 128 product with a block-diagonal P, so each window only sees its own keys.  The tensor
+// core has time to spare here; what the layout buys is that every query row belongs to exactly one
+// thread (its TMEM lane): bias, mask, maximum, exponentials and the row sum need no shuffles, no
+// fragment bookkeeping and no shared-memory fragment loads, which is what bounded the warp-MMA
+// version (it was instruction-issue bound).
+//
+// q, k, v are TMA boxes of 64 rows x 32 columns inside the [M, 3C] buffer of the QKV GEMM (head
+// split, K transpose eliminated); operands that TMA cannot address (the materialised K^T of the
+// explicit variant) are loaded by four helper warps into the same swizzled layout.  V is used as it
+// lies ([key, d] rows) through the MN-major operand mode.  Results are stored as whole 64-byte rows
+// at column h*32 of [M, C] (head merge eliminated) or into [nW, nH, T, d].
+//
+// Persistent CTAs keep one head (its relative-position bias sits in shared memory as a [T, T]
+// table) and stream window pairs through a 3-stage ring; S and O are double buffered in TMEM.
+#include "attn.cuh"
+#include "gemm_tc.cuh"
+#include "ptx.cuh"
+
+namespace smartmem {
+namespace {
+
+constexpr int D = 32, TP = 64;
+constexpr int OP_BYTES = 128 * 64;                    // one operand of a pair: 128 rows x 64 bytes
+constexpr int STAGE_BYTES = 3 * OP_BYTES;             // q, k, v
+constexpr int NSTAGE = 3;
+constexpr int P_BYTES = 2 * 128 * 128;                // P: 2 k-blocks of [128 rows x 128 bytes]
+constexpr uint32_t TM_S = 0, TM_O = 256, TMEM_COLS = 512;
+constexpr int kSoftmaxWarps = 4, kLoaderWarps = 4;
+constexpr int kThreads = 64 + 32 * (kSoftmaxWarps + kLoaderWarps);
+
+struct WinTcArgs {
+  WinAttnArgs a;
+  int n_pairs, tma_mask;                               // bit m set: operand m (q, k, v) comes through TMA
+  FastDiv fd_T;
+  int col0[3], col_per_head[3];                        // TMA column of (operand, head)
+  long long row_per_window[3], row_per_head[3];        // TMA row of (window, head): n * rpw + h * rph
+  int* status;
+};
+
+// Shared-memory matrix descriptor with 64-byte swizzle (rows of 64 bytes, 8-row groups 512 bytes apart).
+__device__ __forceinline__ uint64_t make_desc_sw64(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)4 << 61;
+  return d;
+}
+
+__device__ __forceinline__ float ex2f(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constant__ CUtensorMap tm1,
+                   const __grid_constant__ CUtensorMap tm2, const __grid_constant__ WinTcArgs g) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
+  uint8_t* sIn = smem;                                 // [NSTAGE][q, k, v][128 rows x 64 B]
+  uint8_t* sP = sIn + NSTAGE * STAGE_BYTES;            // [2 k-blocks][128 x 128 B]
+  float* bias_s = reinterpret_cast<float*>(sP + P_BYTES);        // [64][65], log2 domain
+  int* lab_s = reinterpret_cast<int*>(bias_s + TP * 65);         // [2][64]
+  int* tyx_s = lab_s + 2 * TP;                                   // [64]: ty << 8 | tx
+  uint64_t* bars = reinterpret_cast<uint64_t*>(tyx_s + TP);
+  uint64_t *in_full = bars, *in_empty = bars + NSTAGE, *s_full = bars + 2 * NSTAGE, *s_empty = s_full + 2;
+  uint64_t *p_full = s_empty + 2, *p_empty = p_full + 1, *o_full = p_empty + 1, *o_empty = o_full + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_empty + 2);
+  int* abort_flag = reinterpret_cast<int*>(tmem_slot + 1);
+
+  const WinAttnArgs& a = g.a;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
+  const int T = a.T, ws = a.ws;
+  const int h = blockIdx.x % a.heads;
+  const int cidx = blockIdx.x / a.heads, cstride = gridDim.x / a.heads;
+  const bool any_manual = g.tma_mask != 7;
+  const float LOG2E = 1.4426950408889634f;
+
+  if (tid == 0) {
+    for (int i = 0; i < NSTAGE; ++i) {
+      ptx::mbar_init(&in_full[i], 1 + (any_manual ? 32 * kLoaderWarps : 0));
+      ptx::mbar_init(&in_empty[i], 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      ptx::mbar_init(&s_full[i], 1);
+      ptx::mbar_init(&s_empty[i], kSoftmaxWarps);
+      ptx::mbar_init(&o_full[i], 1);
+      ptx::mbar_init(&o_empty[i], kSoftmaxWarps);
+    }
+    ptx::mbar_init(p_full, kSoftmaxWarps);
+    ptx::mbar_init(p_empty, 1);
+    *abort_flag = 0;
+    ptx::fence_barrier_init();
+    ptx::fence_proxy_async();
+  }
+  // one-time tables: token coordinates, the head's bias as a [T, T] table, zeroed staging
+  if (tid < TP) tyx_s[tid] = ((tid / ws) << 8) | (tid % ws);
+  for (int i = tid; i < TP * TP; i += kThreads) {
+    const int r = i / TP, c = i - r * TP;
+    float v = 0.f;
+    if (c >= T) {
+      v = -INFINITY;                                   // padded keys never contribute
+    } else if (r < T) {
+      const int idx = (r / ws - c / ws + ws - 1) * (2 * ws - 1) + (r % ws - c % ws + ws - 1);
+      v = LOG2E * (a.table_f32 ? ((const float*)a.table)[idx * a.heads + h]
+                               : __bfloat162float(((const __nv_bfloat16*)a.table)[idx * a.heads + h]));
+    }
+    bias_s[r * 65 + c] = v;
+  }
+  for (int i = tid; i < (NSTAGE * STAGE_BYTES + P_BYTES) / 16; i += kThreads)
+    reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
+  if (warp == 0 && lane == 0) {
+    ptx::prefetch_tensormap(&tm0);
+    ptx::prefetch_tensormap(&tm1);
+    ptx::prefetch_tensormap(&tm2);
+  }
+  if (warp == 1) ptx::tmem_alloc(tmem_slot, TMEM_COLS);
+  ptx::fence_proxy_async();
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const CUtensorMap* tms[3] = {&tm0, &tm1, &tm2};
+  const AttnOperand* ops[3] = {&a.q, &a.k, &a.v};
+
+  if (warp == 0) {
+    // ---- TMA producer ------------------------------------------------------------------------
+    if (lane == 0) {
+      int n_tma = 0;
+      for (int m = 0; m < 3; ++m) n_tma += (g.tma_mask >> m) & 1;
+      bool ok = true;
+      uint32_t it = 0;
+      for (int p = cidx; p < g.n_pairs && ok; p += cstride, ++it) {
+        const int s = it % NSTAGE;
+        ok = ptx::mbar_wait(&in_empty[s], ((it / NSTAGE) & 1) ^ 1, abort_flag, g.status);
+        if (!ok) break;
+        const int nwin = (2 * p + 1 < a.n_windows) ? 2 : 1;
+        ptx::mbar_expect_tx(&in_full[s], (uint32_t)(n_tma * nwin * TP * 64));
+        for (int m = 0; m < 3; ++m) {
+          if (!((g.tma_mask >> m) & 1)) continue;
+          for (int w = 0; w < nwin; ++w) {
+            const long long n = 2 * p + w;
+            ptx::tma_load_2d(sIn + s * STAGE_BYTES + m * OP_BYTES + w * (TP * 64), tms[m], &in_full[s],
+                             g.col0[m] + h * g.col_per_head[m], (int)(n * g.row_per_window[m] + h * g.row_per_head[m]));
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---- MMA issuer --------------------------------------------------------------------------
+    if (lane == 0) {
+      const uint32_t idesc_s = ptx::make_idesc_bf16(128, 128, false, false);
+      const uint32_t idesc_pv = ptx::make_idesc_bf16(128, D, false, true);     // V: MN-major B operand
+      bool ok = true;
+      const int my_units = cidx < g.n_pairs ? (g.n_pairs - cidx + cstride - 1) / cstride : 0;
+      auto issue_s = [&](int u) {
+        const int s = u % NSTAGE, sb = u & 1;
+        ok = ok && ptx::mbar_wait(&s_empty[sb], ((u >> 1) & 1) ^ 1, abort_flag, g.status);
+        ok = ok && ptx::mbar_wait(&in_full[s], (u / NSTAGE) & 1, abort_flag, g.status);
+        if (!ok) return;
+        ptx::tc_fence_after();
+        const uint32_t q0 = ptx::smem_u32(sIn + s * STAGE_BYTES), k0 = q0 + OP_BYTES;
+        for (int k = 0; k < D / 16; ++k)
+          ptx::tc_mma_bf16(tmem_base + TM_S + sb * 128, make_desc_sw64(q0 + k * 32, 16, 512),
+                           make_desc_sw64(k0 + k * 32, 16, 512), idesc_s, k ? 1u : 0u);
+        ptx::tc_commit(&s_full[sb]);
+      };
+      auto issue_pv = [&](int u) {
+        const int s = u % NSTAGE, ob = u & 1;
+        ok = ok && ptx::mbar_wait(p_full, u & 1, abort_flag, g.status);
+        ok = ok && ptx::mbar_wait(&o_empty[ob], ((u >> 1) & 1) ^ 1, abort_flag, g.status);
+        if (!ok) return;
+        ptx::tc_fence_after();
+        const uint32_t p0 = ptx::smem_u32(sP), v0 = ptx::smem_u32(sIn + s * STAGE_BYTES + 2 * OP_BYTES);
+        for (int ks = 0; ks < 8; ++ks)                 // 16 keys per step
+          ptx::tc_mma_bf16(tmem_base + TM_O + ob * D, ptx::make_smem_desc(p0 + (ks >> 2) * (128 * 128) + (ks & 3) * 32, 16, 1024),
+                           make_desc_sw64(v0 + ks * 1024, 16, 512), idesc_pv, ks ? 1u : 0u);
+        ptx::tc_commit(&in_empty[s]);
+        ptx::tc_commit(p_empty);
+        ptx::tc_commit(&o_full[ob]);
+      };
+      if (my_units > 0) issue_s(0);
+      for (int u = 0; u < my_units && ok; ++u) {
+        if (u + 1 < my_units) issue_s(u + 1);
+        issue_pv(u);
+      }
+    }
+  } else if (warp < 2 + kSoftmaxWarps) {
+    // ---- softmax + epilogue: one query row per thread -------------------------------------------
+    const int q = warp & 3;                            // TMEM lane quadrant
+    const int r = q * 32 + lane;                       // row of the pair tile
+    const int w = r >> 6, i = r & 63;                  // window of the pair, token
+    const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
+    const float scale2 = a.scale * LOG2E;
+    const int my_ty = tyx_s[i] >> 8, my_tx = tyx_s[i] & 255;
+    const float* brow = bias_s + i * 65;
+    float inv_prev = 0.f;
+    int n_prev = -1;
+    bool ok = true;
+    auto epilogue = [&](int u, float inv, int n) {     // O(u) -> global
+      const int ob = u & 1;
+      ok = ok && ptx::mbar_wait(&o_full[ob], (u >> 1) & 1, abort_flag, g.status);
+      if (!ok) return;
+      ptx::tc_fence_after();
+      uint32_t rv[32];
+      ptx::tmem_ld32(tmem_base + TM_O + ob * D + lane_addr, rv);
+      ptx::tmem_ld_wait();
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&o_empty[ob]);
+      if (i < T && n < a.n_windows) {
+        __nv_bfloat16* dst = (__nv_bfloat16*)a.o.ptr + (long long)n * a.o.sn + (long long)h * a.o.sh + (long long)i * a.o.st;
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+          float o8[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) o8[e] = __uint_as_float(rv[v * 8 + e]) * inv;
+          ElemIO<__nv_bfloat16>::store(dst + v * 8, o8);
+        }
+      }
+    };
+    int u = 0;
+    for (int p = cidx; p < g.n_pairs && ok; p += cstride, ++u) {
+      const int sb = u & 1;
+      const int n = 2 * p + w;
+      // region labels of this window (only windows on the seam of a shifted block are masked)
+      bool masked = false;
+      int my_lab = 0;
+      if (a.shift > 0 && n < a.n_windows) {
+        const int wl = n - (int)fd_div((uint32_t)n, a.fd_wpi) * a.win_per_img;
+        const int wy = (int)fd_div((uint32_t)wl, a.fd_nww), wx = wl - wy * a.nWw;
+        masked = (wy == a.nWh - 1) || (wx == a.nWw - 1);
+        if (masked) my_lab = region_label2(my_ty, my_tx, ws, wy, wx, a.H, a.W, a.shift);
+      }
+      if (masked) {                                    // uniform over the 64 threads of the window
+        lab_s[w * TP + i] = my_lab;
+        asm volatile("bar.sync %0, 64;" ::"r"(1 + w) : "memory");
+      }
+      ok = ptx::mbar_wait(&s_full[sb], (u >> 1) & 1, abort_flag, g.status);
+      if (!ok) break;
+      ptx::tc_fence_after();
+      uint32_t rv[64];
+      const uint32_t ts = tmem_base + TM_S + sb * 128 + lane_addr + w * 64;    // this window's 64 key columns
+      ptx::tmem_ld32(ts, rv);
+      ptx::tmem_ld32(ts + 32, rv + 32);
+      ptx::tmem_ld_wait();
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&s_empty[sb]);
+      float sc[64];
+      float mx = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < 64; ++c) {
+        float v = fmaf(__uint_as_float(rv[c]), scale2, brow[c]);
+        if (masked && c < T && lab_s[w * TP + c] != my_lab) v -= 100.f * LOG2E;
+        sc[c] = v;
+        mx = fmaxf(mx, v);
+      }
+      if (masked) asm volatile("bar.sync %0, 64;" ::"r"(1 + w) : "memory");      // labels may be overwritten next unit
+      float sum0 = 0.f, sum1 = 0.f;
+      uint32_t pk[32];
+#pragma unroll
+      for (int c = 0; c < 64; c += 2) {
+        const float p0 = ex2f(sc[c] - mx), p1 = ex2f(sc[c + 1] - mx);
+        sum0 += p0;
+        sum1 += p1;
+        pk[c / 2] = float2_to_bf16x2(p0, p1);
+      }
+      const float inv = 1.f / (sum0 + sum1);
+      // previous P V must have completed before P is overwritten
+      ok = ptx::mbar_wait(p_empty, (u & 1) ^ 1, abort_flag, g.status);
+      if (!ok) break;
+      // P row r: its window's keys are columns w*64 .. w*64+63 = k-block w; chunk c8 at (c8 ^ (r % 8))
+#pragma unroll
+      for (int c8 = 0; c8 < 8; ++c8) {
+        const uint4 v4 = make_uint4(pk[c8 * 4 + 0], pk[c8 * 4 + 1], pk[c8 * 4 + 2], pk[c8 * 4 + 3]);
+        *reinterpret_cast<uint4*>(sP + w * (128 * 128) + r * 128 + ((c8 ^ (r & 7)) << 4)) = v4;
+      }
+      ptx::fence_proxy_async();
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(p_full);
+      // the previous unit's output is drained while this unit's P V runs
+      if (u > 0) epilogue(u - 1, inv_prev, n_prev);
+      inv_prev = inv;
+      n_prev = n;
+    }
+    if (ok && u > 0) epilogue(u - 1, inv_prev, n_prev);
+  } else {
+    // ---- helper loaders for operands TMA cannot address (e.g. a materialised K^T) ----------------
+    if (any_manual) {
+      const int lt = tid - 32 * (2 + kSoftmaxWarps);   // 0 .. 63
+      bool ok = true;
+      uint32_t it = 0;
+      for (int p = cidx; p < g.n_pairs && ok; p += cstride, ++it) {
+        const int s = it % NSTAGE;
+        ok = ptx::mbar_wait(&in_empty[s], ((it / NSTAGE) & 1) ^ 1, abort_flag, g.status);
+        if (!ok) break;
+        for (int m = 0; m < 3; ++m) {
+          if ((g.tma_mask >> m) & 1) continue;
+          const AttnOperand& o = *ops[m];
+          uint8_t* dst = sIn + s * STAGE_BYTES + m * OP_BYTES;
+          // A window's operand is one contiguous block of T*D elements when it is a materialised
+          // [T, d] or [d, T] matrix: read it with 16-byte loads and scatter the 8 elements of a load
+          // to their (token, feature) slots of the swizzled tile.
+          const bool block_td = o.se == 1 && o.st == D, block_dt = o.st == 1 && o.se == T;
+          const bool vec_ok = (block_td || block_dt) && (T * D) % 8 == 0 && o.sn % 8 == 0 && o.sh % 8 == 0 &&
+                              ((uintptr_t)o.ptr & 15) == 0;
+          auto put = [&](int w, int t, int e, __nv_bfloat16 v) {
+            const int row = w * TP + t;                // 64-byte rows, 16-byte chunks swizzled by (row / 2) % 4
+            *reinterpret_cast<__nv_bfloat16*>(dst + row * 64 + ((((e >> 3) ^ ((row >> 1) & 3))) << 4) + (e & 7) * 2) = v;
+          };
+          if (vec_ok) {
+            const int nvec = T * D / 8;
+            for (int idx = lt; idx < 2 * nvec; idx += 32 * kLoaderWarps) {
+              const int w = idx >= nvec ? 1 : 0, vi = idx - w * nvec;
+              const long long n = 2 * p + w;
+              uint4 raw = make_uint4(0, 0, 0, 0);
+              if (n < a.n_windows)
+                raw = *reinterpret_cast<const uint4*>((const __nv_bfloat16*)o.ptr + n * o.sn + (long long)h * o.sh + vi * 8);
+              const __nv_bfloat16* ev = reinterpret_cast<const __nv_bfloat16*>(&raw);
+              // (token, feature) of the first element: one reciprocal division, then counting
+              int t, e;
+              if (block_td) { t = (vi * 8) >> 5; e = (vi * 8) & 31; }
+              else { e = (int)fd_div((uint32_t)(vi * 8), g.fd_T); t = vi * 8 - e * T; }
+#pragma unroll
+              for (int k = 0; k < 8; ++k) {
+                put(w, t, e, ev[k]);
+                if (block_td) { if (++e == D) { e = 0; ++t; } }
+                else { if (++t == T) { t = 0; ++e; } }
+              }
+            }
+          } else {
+            for (int idx = lt; idx < 2 * T * D; idx += 32 * kLoaderWarps) {
+              const int w = idx / (T * D), rem = idx - w * (T * D);
+              int t, e;
+              if (o.se == 1) { t = rem / D; e = rem - t * D; } else { e = rem / T; t = rem - e * T; }
+              const long long n = 2 * p + w;
+              __nv_bfloat16 v = __float2bfloat16_rn(0.f);
+              if (n < a.n_windows)
+                v = ((const __nv_bfloat16*)o.ptr)[n * o.sn + (long long)h * o.sh + (long long)t * o.st + (long long)e * o.se];
+              put(w, t, e, v);
+            }
+          }
+        }
+        ptx::fence_proxy_async();
+        ptx::mbar_arrive(&in_full[s]);
+      }
+    }
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+}  // namespace
+
+// Returns SMARTMEM_ERR_UNSUPPORTED for shapes the kernel does not cover (the caller then uses the
+// warp-MMA kernel).
+int launch_window_attention_tc(const WinAttnArgs& a_in, long long n_windows, cudaStream_t st) {
+  if (a_in.d != D || a_in.T > TP || a_in.T < 1 || n_windows < 1 || n_windows >= (1ll << 30)) return SMARTMEM_ERR_UNSUPPORTED;
+  if (a_in.o.se != 1 || a_in.o.st % 8 || a_in.o.sn % 8 || a_in.o.sh % 8 || ((uintptr_t)a_in.o.ptr & 15)) return SMARTMEM_ERR_UNSUPPORTED;
+  WinTcArgs g;
+  memset(&g, 0, sizeof(g));
+  g.a = a_in;
+  WinAttnArgs& a = g.a;
+  a.n_windows = (int)n_windows;
+  a.nWh = a.win_per_img / a.nWw;
+  a.fd_wpi = make_fastdiv((uint32_t)a.win_per_img);
+  a.fd_nww = make_fastdiv((uint32_t)a.nWw);
+  g.n_pairs = (int)((n_windows + 1) / 2);
+  g.fd_T = make_fastdiv((uint32_t)a.T);
+  g.status = device_status_ptr();
+  if (!g.status) return SMARTMEM_ERR_CUDA;
+  CUtensorMap tm[3];
+  memset(tm, 0, sizeof(tm));
+  const AttnOperand* ops[3] = {&a.q, &a.k, &a.v};
+  const long long T = a.T, H = a.heads;
+  for (int m = 0; m < 3; ++m) {
+    const AttnOperand& o = *ops[m];
+    // rows of 32 contiguous elements, 16-byte aligned pitch; two addressing patterns
+    const bool rows_ok = o.se == 1 && o.st % 8 == 0 && ((uintptr_t)o.ptr & 15) == 0;
+    if (rows_ok && o.sh == D && o.sn == T * o.st) {                 // [M, pitch] with heads side by side
+      if (tc_encode_2d_sw64(o.ptr, H * D, n_windows * T, o.st, D, TP, &tm[m]) != SMARTMEM_OK) continue;
+      g.col0[m] = 0; g.col_per_head[m] = D; g.row_per_window[m] = T; g.row_per_head[m] = 0;
+      g.tma_mask |= 1 << m;
+    } else if (rows_ok && o.st == D && o.sh == T * D && o.sn == H * T * D) {     // [nW, nH, T, d]
+      if (tc_encode_2d_sw64(o.ptr, D, n_windows * H * T, D, D, TP, &tm[m]) != SMARTMEM_OK) continue;
+      g.col0[m] = 0; g.col_per_head[m] = 0; g.row_per_window[m] = H * T; g.row_per_head[m] = T;
+      g.tma_mask |= 1 << m;
+    }
+  }
+  const size_t smem = 1024 + NSTAGE * STAGE_BYTES + P_BYTES + TP * 65 * 4 + 3 * TP * 4 + (2 * NSTAGE + 10) * 8 + 16;
+  static bool configured = false;
+  if (!configured) {
+    if (cudaFuncSetAttribute(win_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return SMARTMEM_ERR_CUDA;
+    configured = true;
+  }
+  const int sms = tc_sm_count();
+  long long per_head = (long long)sms / a.heads;
+  if (per_head < 1) per_head = 1;
+  if (per_head > g.n_pairs) per_head = g.n_pairs;
+  const unsigned grid = (unsigned)(per_head * a.heads);
+  profile_tick("window_attention_tc", st);
+  win_attn_tc_kernel<<<grid, kThreads, smem, st>>>(tm[0], tm[1], tm[2], g);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
+}
+
+}  // namespace smartmem

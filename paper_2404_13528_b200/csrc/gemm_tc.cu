@@ -395,12 +395,13 @@ std::mutex g_tm_mu;
 std::unordered_map<std::string, CUtensorMap> g_tm_cache;
 
 int encode_cached(const void* ptr, int rank, const uint64_t* dims, const uint64_t* strides_b, const uint32_t* box,
-                  CUtensorMap* out) {
+                  CUtensorMap* out, int swizzle_bytes = 128) {
   std::string key((const char*)&ptr, sizeof(ptr));
   key.append((const char*)&rank, sizeof(rank));
   key.append((const char*)dims, sizeof(uint64_t) * rank);
   key.append((const char*)strides_b, sizeof(uint64_t) * (rank - 1));
   key.append((const char*)box, sizeof(uint32_t) * rank);
+  key.append((const char*)&swizzle_bytes, sizeof(int));
   {
     std::lock_guard<std::mutex> lk(g_tm_mu);
     auto it = g_tm_cache.find(key);
@@ -420,7 +421,8 @@ int encode_cached(const void* ptr, int rank, const uint64_t* dims, const uint64_
     if (i < rank - 1) s[i] = strides_b[i];
   }
   CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(ptr), d, s, b, es,
-                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return SMARTMEM_ERR_CUDA;
   std::lock_guard<std::mutex> lk(g_tm_mu);
@@ -514,6 +516,15 @@ int tc_encode_2d(const void* ptr, long long inner, long long outer, long long pi
   const uint64_t strides[1] = {(uint64_t)pitch_elems * 2};
   const uint32_t box[2] = {(uint32_t)box_inner, (uint32_t)box_outer};
   return encode_cached(ptr, 2, dims, strides, box, out);
+}
+
+int tc_encode_2d_sw64(const void* ptr, long long inner, long long outer, long long pitch_elems, int box_inner,
+                      int box_outer, CUtensorMap* out) {
+  if (((uintptr_t)ptr & 15) || (pitch_elems * 2) % 16 || box_inner * 2 != 64) return SMARTMEM_ERR_ALIGNMENT;
+  const uint64_t dims[2] = {(uint64_t)inner, (uint64_t)outer};
+  const uint64_t strides[1] = {(uint64_t)pitch_elems * 2};
+  const uint32_t box[2] = {(uint32_t)box_inner, (uint32_t)box_outer};
+  return encode_cached(ptr, 2, dims, strides, box, out, 64);
 }
 
 int tc_sm_count() { return sm_count(); }

@@ -39,6 +39,9 @@ int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep,
 // bf16 row-major [outer, inner] matrix as a 2-D tensor map with 128-byte swizzle (box_inner = 64).
 int tc_encode_2d(const void* ptr, long long inner, long long outer, long long pitch_elems, int box_inner, int box_outer,
                  CUtensorMap* out);
+// Same with 64-byte swizzle: boxes of 32 bf16 columns (64-byte rows).
+int tc_encode_2d_sw64(const void* ptr, long long inner, long long outer, long long pitch_elems, int box_inner,
+                      int box_outer, CUtensorMap* out);
 int tc_sm_count();
 
 // Fused MLP: out = residual + (GELU(A W1^T + b1)) W2^T + b2 with the hidden activation kept on chip.
