@@ -15,7 +15,8 @@
 // at column h*32 of [M, C] (head merge eliminated) or into [nW, nH, T, d].
 //
 // Persistent CTAs keep one head (its relative-position bias sits in shared memory as a [T, T]
-// table) and stream window pairs through a 3-stage ring; S and O are double buffered in TMEM.
+// table) and stream window pairs through a 3-stage ring.  Two softmax groups of four warps
+// alternate over the units, each with its own S and O buffers in TMEM and its own P tile.
 #include "attn.cuh"
 #include "gemm_tc.cuh"
 #include "ptx.cuh"
@@ -27,10 +28,10 @@ constexpr int D = 32, TP = 64;
 constexpr int OP_BYTES = 128 * 64;                    // one operand of a pair: 128 rows x 64 bytes
 constexpr int STAGE_BYTES = 3 * OP_BYTES;             // q, k, v
 constexpr int NSTAGE = 3;
-constexpr int P_BYTES = 2 * 128 * 128;                // P: 2 k-blocks of [128 rows x 128 bytes]
+constexpr int P_BYTES = 2 * 128 * 128;                // P: 2 k-blocks of [128 rows x 128 bytes] (one per softmax group)
 constexpr uint32_t TM_S = 0, TM_O = 256, TMEM_COLS = 512;
-constexpr int kSoftmaxWarps = 4, kLoaderWarps = 4;
-constexpr int kThreads = 64 + 32 * (kSoftmaxWarps + kLoaderWarps);
+constexpr int kSoftmaxWarps = 4, kGroups = 2, kLoaderWarps = 4;   // two softmax groups alternate over the units
+constexpr int kThreads = 64 + 32 * (kGroups * kSoftmaxWarps + kLoaderWarps);
 
 struct WinTcArgs {
   WinAttnArgs a;
@@ -64,13 +65,13 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
   uint8_t* sIn = smem;                                 // [NSTAGE][q, k, v][128 rows x 64 B]
-  uint8_t* sP = sIn + NSTAGE * STAGE_BYTES;            // [2 k-blocks][128 x 128 B]
-  float* bias_s = reinterpret_cast<float*>(sP + P_BYTES);        // [64][65], log2 domain
-  int* lab_s = reinterpret_cast<int*>(bias_s + TP * 65);         // [2][64]
-  int* tyx_s = lab_s + 2 * TP;                                   // [64]: ty << 8 | tx
+  uint8_t* sP = sIn + NSTAGE * STAGE_BYTES;            // [kGroups][2 k-blocks][128 x 128 B]
+  float* bias_s = reinterpret_cast<float*>(sP + kGroups * P_BYTES);   // [64][65], log2 domain
+  int* lab_s = reinterpret_cast<int*>(bias_s + TP * 65);         // [kGroups][2][64]
+  int* tyx_s = lab_s + kGroups * 2 * TP;                         // [64]: ty << 8 | tx
   uint64_t* bars = reinterpret_cast<uint64_t*>(tyx_s + TP);
   uint64_t *in_full = bars, *in_empty = bars + NSTAGE, *s_full = bars + 2 * NSTAGE, *s_empty = s_full + 2;
-  uint64_t *p_full = s_empty + 2, *p_empty = p_full + 1, *o_full = p_empty + 1, *o_empty = o_full + 2;
+  uint64_t *p_full = s_empty + 2, *p_empty = p_full + 2, *o_full = p_empty + 2, *o_empty = o_full + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_empty + 2);
   int* abort_flag = reinterpret_cast<int*>(tmem_slot + 1);
 
@@ -93,8 +94,10 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
       ptx::mbar_init(&o_full[i], 1);
       ptx::mbar_init(&o_empty[i], kSoftmaxWarps);
     }
-    ptx::mbar_init(p_full, kSoftmaxWarps);
-    ptx::mbar_init(p_empty, 1);
+    for (int i = 0; i < 2; ++i) {
+      ptx::mbar_init(&p_full[i], kSoftmaxWarps);
+      ptx::mbar_init(&p_empty[i], 1);
+    }
     *abort_flag = 0;
     ptx::fence_barrier_init();
     ptx::fence_proxy_async();
@@ -113,7 +116,7 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
     }
     bias_s[r * 65 + c] = v;
   }
-  for (int i = tid; i < (NSTAGE * STAGE_BYTES + P_BYTES) / 16; i += kThreads)
+  for (int i = tid; i < (NSTAGE * STAGE_BYTES + kGroups * P_BYTES) / 16; i += kThreads)
     reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
   if (warp == 0 && lane == 0) {
     ptx::prefetch_tensormap(&tm0);
@@ -173,16 +176,16 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
       };
       auto issue_pv = [&](int u) {
         const int s = u % NSTAGE, ob = u & 1;
-        ok = ok && ptx::mbar_wait(p_full, u & 1, abort_flag, g.status);
+        ok = ok && ptx::mbar_wait(&p_full[ob], (u >> 1) & 1, abort_flag, g.status);
         ok = ok && ptx::mbar_wait(&o_empty[ob], ((u >> 1) & 1) ^ 1, abort_flag, g.status);
         if (!ok) return;
         ptx::tc_fence_after();
-        const uint32_t p0 = ptx::smem_u32(sP), v0 = ptx::smem_u32(sIn + s * STAGE_BYTES + 2 * OP_BYTES);
+        const uint32_t p0 = ptx::smem_u32(sP + ob * P_BYTES), v0 = ptx::smem_u32(sIn + s * STAGE_BYTES + 2 * OP_BYTES);
         for (int ks = 0; ks < 8; ++ks)                 // 16 keys per step
           ptx::tc_mma_bf16(tmem_base + TM_O + ob * D, ptx::make_smem_desc(p0 + (ks >> 2) * (128 * 128) + (ks & 3) * 32, 16, 1024),
                            make_desc_sw64(v0 + ks * 1024, 16, 512), idesc_pv, ks ? 1u : 0u);
         ptx::tc_commit(&in_empty[s]);
-        ptx::tc_commit(p_empty);
+        ptx::tc_commit(&p_empty[ob]);
         ptx::tc_commit(&o_full[ob]);
       };
       if (my_units > 0) issue_s(0);
@@ -191,8 +194,9 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
         issue_pv(u);
       }
     }
-  } else if (warp < 2 + kSoftmaxWarps) {
-    // ---- softmax + epilogue: one query row per thread -------------------------------------------
+  } else if (warp < 2 + kGroups * kSoftmaxWarps) {
+    // ---- softmax + epilogue: one query row per thread; group gi takes the units u = gi (mod 2) ----
+    const int gi = (warp - 2) / kSoftmaxWarps;
     const int q = warp & 3;                            // TMEM lane quadrant
     const int r = q * 32 + lane;                       // row of the pair tile
     const int w = r >> 6, i = r & 63;                  // window of the pair, token
@@ -204,7 +208,7 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
     int n_prev = -1;
     bool ok = true;
     auto epilogue = [&](int u, float inv, int n) {     // O(u) -> global
-      const int ob = u & 1;
+      const int ob = u & 1;                            // == gi
       ok = ok && ptx::mbar_wait(&o_full[ob], (u >> 1) & 1, abort_flag, g.status);
       if (!ok) return;
       ptx::tc_fence_after();
@@ -225,8 +229,9 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
         }
       }
     };
-    int u = 0;
-    for (int p = cidx; p < g.n_pairs && ok; p += cstride, ++u) {
+    int u = gi;
+    int done = 0;
+    for (int p = cidx + gi * cstride; p < g.n_pairs && ok; p += 2 * cstride, u += 2, ++done) {
       const int sb = u & 1;
       const int n = 2 * p + w;
       // region labels of this window (only windows on the seam of a shifted block are masked)
@@ -239,8 +244,8 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
         if (masked) my_lab = region_label2(my_ty, my_tx, ws, wy, wx, a.H, a.W, a.shift);
       }
       if (masked) {                                    // uniform over the 64 threads of the window
-        lab_s[w * TP + i] = my_lab;
-        asm volatile("bar.sync %0, 64;" ::"r"(1 + w) : "memory");
+        lab_s[(gi * 2 + w) * TP + i] = my_lab;
+        asm volatile("bar.sync %0, 64;" ::"r"(1 + gi * 2 + w) : "memory");
       }
       ok = ptx::mbar_wait(&s_full[sb], (u >> 1) & 1, abort_flag, g.status);
       if (!ok) break;
@@ -258,11 +263,11 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
 #pragma unroll
       for (int c = 0; c < 64; ++c) {
         float v = fmaf(__uint_as_float(rv[c]), scale2, brow[c]);
-        if (masked && c < T && lab_s[w * TP + c] != my_lab) v -= 100.f * LOG2E;
+        if (masked && c < T && lab_s[(gi * 2 + w) * TP + c] != my_lab) v -= 100.f * LOG2E;
         sc[c] = v;
         mx = fmaxf(mx, v);
       }
-      if (masked) asm volatile("bar.sync %0, 64;" ::"r"(1 + w) : "memory");      // labels may be overwritten next unit
+      if (masked) asm volatile("bar.sync %0, 64;" ::"r"(1 + gi * 2 + w) : "memory");   // labels may be overwritten next unit
       float sum0 = 0.f, sum1 = 0.f;
       uint32_t pk[32];
 #pragma unroll
@@ -274,28 +279,28 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
       }
       const float inv = 1.f / (sum0 + sum1);
       // previous P V must have completed before P is overwritten
-      ok = ptx::mbar_wait(p_empty, (u & 1) ^ 1, abort_flag, g.status);
+      ok = ptx::mbar_wait(&p_empty[gi], ((u >> 1) & 1) ^ 1, abort_flag, g.status);
       if (!ok) break;
       // P row r: its window's keys are columns w*64 .. w*64+63 = k-block w; chunk c8 at (c8 ^ (r % 8))
 #pragma unroll
       for (int c8 = 0; c8 < 8; ++c8) {
         const uint4 v4 = make_uint4(pk[c8 * 4 + 0], pk[c8 * 4 + 1], pk[c8 * 4 + 2], pk[c8 * 4 + 3]);
-        *reinterpret_cast<uint4*>(sP + w * (128 * 128) + r * 128 + ((c8 ^ (r & 7)) << 4)) = v4;
+        *reinterpret_cast<uint4*>(sP + gi * P_BYTES + w * (128 * 128) + r * 128 + ((c8 ^ (r & 7)) << 4)) = v4;
       }
       ptx::fence_proxy_async();
       ptx::tc_fence_before();
       __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(p_full);
-      // the previous unit's output is drained while this unit's P V runs
-      if (u > 0) epilogue(u - 1, inv_prev, n_prev);
+      if (lane == 0) ptx::mbar_arrive(&p_full[gi]);
+      // this group's previous unit is drained while this unit's P V runs
+      if (done > 0) epilogue(u - 2, inv_prev, n_prev);
       inv_prev = inv;
       n_prev = n;
     }
-    if (ok && u > 0) epilogue(u - 1, inv_prev, n_prev);
+    if (ok && done > 0) epilogue(u - 2, inv_prev, n_prev);
   } else {
     // ---- helper loaders for operands TMA cannot address (e.g. a materialised K^T) ----------------
     if (any_manual) {
-      const int lt = tid - 32 * (2 + kSoftmaxWarps);   // 0 .. 63
+      const int lt = tid - 32 * (2 + kGroups * kSoftmaxWarps);
       bool ok = true;
       uint32_t it = 0;
       for (int p = cidx; p < g.n_pairs && ok; p += cstride, ++it) {
@@ -399,7 +404,8 @@ int launch_window_attention_tc(const WinAttnArgs& a_in, long long n_windows, cud
       g.tma_mask |= 1 << m;
     }
   }
-  const size_t smem = 1024 + NSTAGE * STAGE_BYTES + P_BYTES + TP * 65 * 4 + 3 * TP * 4 + (2 * NSTAGE + 10) * 8 + 16;
+  const size_t smem = 1024 + NSTAGE * STAGE_BYTES + kGroups * P_BYTES + TP * 65 * 4 + (2 * kGroups + 1) * TP * 4 +
+                      (2 * NSTAGE + 12) * 8 + 16;
   static bool configured = false;
   if (!configured) {
     if (cudaFuncSetAttribute(win_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
