@@ -170,7 +170,7 @@ int launch_norm_t(const void* src, void* dst, const void* gamma, const void* bet
     unsigned grid = (unsigned)((rows + rpb - 1) / rpb);                                                   \
     norm_kernel<T, LPR, RMS, RPG, GEN><<<grid, 256, 0, st>>>(s, d, g, b, eps, rows, C, vpl, dm, has);     \
   }
-  if (nvec <= 16) SM_LAUNCH(4, 2, false)
+  if (nvec <= 16) SM_LAUNCH(4, 1, false)
   else if (nvec <= 32) SM_LAUNCH(8, 2, false)
   else if (nvec <= 64) SM_LAUNCH(16, 1, false)
   else if (nvec <= 128) SM_LAUNCH(32, 1, false)
