@@ -22,6 +22,16 @@
 #include "gemm_tc.cuh"
 #include "ptx.cuh"
 
+#ifdef GEMM_EXP_TIMING
+__device__ long long g_gemm_dbg[8192];
+#define GDBG(slot) do { if (blockIdx.x == 0 && (slot) < 8192) g_gemm_dbg[(slot)] = clock64(); } while (0)
+extern "C" __attribute__((visibility("default"))) int smartmem_debug_read_gemm(long long* host, int n) {
+  return (int)cudaMemcpyFromSymbol(host, g_gemm_dbg, sizeof(long long) * n);
+}
+#else
+#define GDBG(slot) do { } while (0)
+#endif
+
 namespace smartmem {
 namespace {
 
@@ -52,19 +62,33 @@ struct GemmArgs {
   DevMap rowmap;
 };
 
-__device__ __forceinline__ void op_coords(const OpCoord& oc, uint32_t tile, uint32_t batch, int tile_rows, int k0,
-                                          int* c) {
+// Tile -> TMA coordinates of an operand: row origin inside the innermost row atom and the digits
+// of the outer row atoms / batch atoms (every tensor map is padded to rank 5, so all five
+// coordinates always exist and stay in registers).
+struct TileCoord {
+  int row0, o0, o1, o2;
+};
+__device__ __forceinline__ TileCoord op_coords(const OpCoord& oc, uint32_t tile, uint32_t batch, int tile_rows) {
   uint32_t q = fd_div(tile, oc.tiles_inner);
-  int row0 = (int)(tile - q * oc.tiles_inner.d) * tile_rows;
-  c[0] = oc.mn_major ? row0 : k0;
-  c[1] = oc.mn_major ? k0 : row0;
-  int n = 2;
-  for (int i = 0; i < oc.n_outer; ++i) {
-    uint32_t& src = (i < oc.n_outer_row) ? q : batch;
-    uint32_t qq = fd_div(src, oc.outer[i]);
-    c[n++] = (int)(src - qq * oc.outer[i].d);
-    src = qq;
+  TileCoord tc;
+  tc.row0 = (int)(tile - q * oc.tiles_inner.d) * tile_rows;
+  int o[3] = {0, 0, 0};
+#pragma unroll
+  for (int i = 0; i < 3; ++i) {
+    if (i < oc.n_outer) {
+      const bool from_rows = i < oc.n_outer_row;
+      const uint32_t src = from_rows ? q : batch;
+      const uint32_t qq = fd_div(src, oc.outer[i]);
+      o[i] = (int)(src - qq * oc.outer[i].d);
+      if (from_rows) q = qq; else batch = qq;
+    }
   }
+  tc.o0 = o[0]; tc.o1 = o[1]; tc.o2 = o[2];
+  return tc;
+}
+__device__ __forceinline__ void tma_load_op(const OpCoord& oc, void* dst, const CUtensorMap* tm, uint64_t* bar, int k0,
+                                            int row0, const TileCoord& tc) {
+  ptx::tma_load_5d(dst, tm, bar, oc.mn_major ? row0 : k0, oc.mn_major ? k0 : row0, tc.o0, tc.o1, tc.o2);
 }
 
 // GELU in the bf16 epilogue: u * Phi(u) with Phi evaluated through the hyperbolic-tangent form
@@ -140,26 +164,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (lane == 0) {
       uint32_t kbg = 0;                                      // k-block counter across tiles
       bool ok = true;
-      for (uint32_t t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+      uint32_t pit = 0;
+      for (uint32_t t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++pit) {
         const uint32_t tile_n = t % g.tiles_n, r = t / g.tiles_n, tile_m = r % g.tiles_m, batch = r / g.tiles_m;
+        GDBG(pit * 16 + 0);
+        const TileCoord ta = op_coords(g.ca, tile_m, batch, BM), tb = op_coords(g.cb, tile_n, batch, BN);
         for (int kb = 0; kb < nkb; ++kb, ++kbg) {
           const int s = kbg % STAGES;
           const uint32_t ph = (kbg / STAGES) & 1;
           ok = ptx::mbar_wait(&empty[s], ph ^ 1, abort_flag, g.status);
+          if (kb == 0) GDBG(pit * 16 + 1);
           if (!ok) break;
           ptx::mbar_expect_tx(&full[s], A_STAGE_BYTES + B_STAGE_BYTES);
-          int c[5];
-          op_coords(g.ca, tile_m, batch, BM, kb * BK, c);
-          if (A_MN) {
-            ptx::tma_load_nd(g.ca.rank, sA + s * A_STAGE_BYTES, &tmA, &full[s], c);
-            c[0] += 64;
-            ptx::tma_load_nd(g.ca.rank, sA + s * A_STAGE_BYTES + A_STAGE_BYTES / 2, &tmA, &full[s], c);
-          } else {
-            ptx::tma_load_nd(g.ca.rank, sA + s * A_STAGE_BYTES, &tmA, &full[s], c);
-          }
-          op_coords(g.cb, tile_n, batch, BN, kb * BK, c);
-          ptx::tma_load_nd(g.cb.rank, sB + s * B_STAGE_BYTES, &tmB, &full[s], c);
+          tma_load_op(g.ca, sA + s * A_STAGE_BYTES, &tmA, &full[s], kb * BK, ta.row0, ta);
+          if (A_MN) tma_load_op(g.ca, sA + s * A_STAGE_BYTES + A_STAGE_BYTES / 2, &tmA, &full[s], kb * BK, ta.row0 + 64, ta);
+          tma_load_op(g.cb, sB + s * B_STAGE_BYTES, &tmB, &full[s], kb * BK, tb.row0, tb);
         }
+        GDBG(pit * 16 + 2);
       }
       if (*abort_flag) {
         // unwinding: give copies already in flight a bounded chance to land before the CTA leaves
@@ -176,8 +197,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       bool ok = true;
       for (uint32_t t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
         const uint32_t buf = it & 1, use = it >> 1;
+        GDBG(it * 16 + 3);
         ok = ptx::mbar_wait(&tmem_empty[buf], (use & 1) ^ 1, abort_flag, g.status);   // epilogue drained it
         if (!ok) break;
+        GDBG(it * 16 + 4);
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * ACC_COLS;
         for (int kb = 0; kb < nkb; ++kb, ++kbg) {
@@ -185,6 +208,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           const uint32_t ph = (kbg / STAGES) & 1;
           ok = ptx::mbar_wait(&full[s], ph, abort_flag, g.status);
           if (!ok) break;
+          if (kb == 0) GDBG(it * 16 + 5);
+          if (kb == 1) GDBG(it * 16 + 6);
           ptx::tc_fence_after();
           const uint32_t a0 = ptx::smem_u32(sA + s * A_STAGE_BYTES), b0 = ptx::smem_u32(sB + s * B_STAGE_BYTES);
           const int ks = (kb == nkb - 1) ? last_ksteps : BK / 16;
@@ -200,6 +225,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           ptx::tc_commit(&empty[s]);
         }
         if (ok) ptx::tc_commit(&tmem_full[buf]);
+        GDBG(it * 16 + 7);
       }
     }
   } else {
@@ -248,8 +274,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       };
       fetch_res(col_of(0));                                  // in flight while this tile's MMAs still run
 
+      if (warp == 2 && lane == 0) GDBG(it * 16 + 8);
       ok = ptx::mbar_wait(&tmem_full[buf], use & 1, abort_flag, g.status);
       if (!ok) break;
+      if (warp == 2 && lane == 0) GDBG(it * 16 + 9);
       ptx::tc_fence_after();
       const uint32_t taddr = tmem_base + buf * ACC_COLS + ((uint32_t)(q * 32) << 16);
 
@@ -345,6 +373,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&tmem_empty[buf]);
+      if (warp == 2 && lane == 0) GDBG(it * 16 + 10);
       if constexpr (QSTAGE) {
         // the four warps of the quadrant have filled a 32 x BN staging tile: store whole rows
         constexpr int VR = BN / 8;                           // 16-byte vectors per row
@@ -360,6 +389,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if (rok && n0 + seg * 8 + 8 <= g.N) *reinterpret_cast<uint4*>(g.out + roff + n0 + seg * 8) = pk;
         }
         asm volatile("bar.sync %0, 128;" ::"r"(1 + q) : "memory");
+        if (warp == 2 && lane == 0) GDBG(it * 16 + 11);
       }
     }
   }
@@ -471,6 +501,13 @@ int build_operand(const TcOperand& op, int tile_rows, CUtensorMap* tm, OpCoord* 
   }
   if (!ok) return SMARTMEM_ERR_UNSUPPORTED;
   if (rank < 2) return SMARTMEM_ERR_UNSUPPORTED;
+  while (rank < 5) {                                   // pad: all kernels issue 5-D loads
+    strides[rank - 1] = strides[rank - 2] * dims[rank - 1];
+    if (strides[rank - 1] >= (1ull << 40)) strides[rank - 1] = strides[rank - 2];
+    dims[rank] = 1;
+    box[rank] = 1;
+    ++rank;
+  }
   oc->rank = rank;
   oc->mn_major = mn ? 1 : 0;
   oc->tiles_inner = make_fastdiv((uint32_t)((in_ext + tile_rows - 1) / tile_rows));
