@@ -106,7 +106,7 @@ __device__ __forceinline__ float gelu_fast(float u) {
 }
 
 constexpr int kEpiWarps = 16;
-constexpr int kThreads = 64 + 32 * kEpiWarps;
+constexpr int kThreads = 64 + 32 * kEpiWarps + 32;      // + a second TMA producer warp (B operand)
 
 // Persistent kernel: one CTA per SM walks over output tiles (tile = blockIdx.x + i * gridDim.x).
 // The shared-memory ring and two TMEM accumulator buffers run across tile boundaries, so the
@@ -135,11 +135,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nkb = (g.K + BK - 1) / BK;
   const int last_ksteps = (g.K - (nkb - 1) * BK + 15) / 16;
+  const bool two_producers = nkb >= 8;
   const uint32_t total_tiles = (uint32_t)g.tiles_n * g.tiles_m * g.batch;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
-      ptx::mbar_init(&full[s], 1);
+      ptx::mbar_init(&full[s], two_producers ? 2 : 1);  // one arrival per producer warp
       ptx::mbar_init(&empty[s], 1);
     }
     for (int b = 0; b < 2; ++b) {
@@ -175,10 +176,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           ok = ptx::mbar_wait(&empty[s], ph ^ 1, abort_flag, g.status);
           if (kb == 0) GDBG(pit * 16 + 1);
           if (!ok) break;
-          ptx::mbar_expect_tx(&full[s], A_STAGE_BYTES + B_STAGE_BYTES);
+          ptx::mbar_expect_tx(&full[s], two_producers ? A_STAGE_BYTES : A_STAGE_BYTES + B_STAGE_BYTES);
           tma_load_op(g.ca, sA + s * A_STAGE_BYTES, &tmA, &full[s], kb * BK, ta.row0, ta);
           if (A_MN) tma_load_op(g.ca, sA + s * A_STAGE_BYTES + A_STAGE_BYTES / 2, &tmA, &full[s], kb * BK, ta.row0 + 64, ta);
-          tma_load_op(g.cb, sB + s * B_STAGE_BYTES, &tmB, &full[s], kb * BK, tb.row0, tb);
+          if (!two_producers) tma_load_op(g.cb, sB + s * B_STAGE_BYTES, &tmB, &full[s], kb * BK, tb.row0, tb);
         }
         GDBG(pit * 16 + 2);
       }
@@ -226,6 +227,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
         if (ok) ptx::tc_commit(&tmem_full[buf]);
         GDBG(it * 16 + 7);
+      }
+    }
+  } else if (warp >= 2 + kEpiWarps) {
+    // second producer: the B operand (long reductions only; a short one is
+    // cheaper to feed from one thread)
+    if (lane == 0 && two_producers) {
+      uint32_t kbg = 0;
+      bool ok = true;
+      for (uint32_t t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+        const uint32_t tile_n = t % g.tiles_n, r = t / g.tiles_n, batch = r / g.tiles_m;
+        const TileCoord tb = op_coords(g.cb, tile_n, batch, BN);
+        for (int kb = 0; kb < nkb; ++kb, ++kbg) {
+          const int s = kbg % STAGES;
+          ok = ptx::mbar_wait(&empty[s], ((kbg / STAGES) & 1) ^ 1, abort_flag, g.status);
+          if (!ok) break;
+          ptx::mbar_expect_tx(&full[s], B_STAGE_BYTES);
+          tma_load_op(g.cb, sB + s * B_STAGE_BYTES, &tmB, &full[s], kb * BK, tb.row0, tb);
+        }
       }
     }
   } else {
