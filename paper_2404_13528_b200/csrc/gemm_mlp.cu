@@ -10,7 +10,9 @@
 // the next chunk is already running (two TMEM buffers for fc1, one accumulator for fc2).
 //
 // Warp roles: warp 0 TMA producer (A tile double-buffered across tiles, weights streamed through a
-// ring: they stay L2-resident), warp 1 MMA issuer + TMEM owner, warps 2-17 epilogue.
+// ring: they stay L2-resident), warp 1 fc1 issuer + TMEM owner, warps 2-17 GELU (TMEM -> shared
+// memory), warps 18-21 output (OUT + b2 + residual -> global, OUT double-buffered in TMEM so they
+// overlap the next tile), warp 22 fc2 issuer.
 #include "gemm_tc.cuh"
 #include "ptx.cuh"
 
@@ -31,11 +33,14 @@ constexpr int BM = 128, BK = 64, HC = 128;         // tile rows, k-block, hidden
 constexpr int KB_BYTES = BM * BK * 2;              // one 128 x 64 bf16 operand block: 16 KB
 constexpr int NST = 3;                             // weight ring stages; one stage = both k-blocks of a chunk's W1 or W2
 constexpr int WST_BYTES = 2 * KB_BYTES;
-constexpr int kEpiWarps = 16, kThreads = 64 + 32 * kEpiWarps;
-constexpr uint32_t TM_S1 = 0, TM_OUT = 256, TMEM_COLS = 512;
+constexpr int kGeluWarps = 16, kOutWarps = 4, kThreads = 32 * (3 + kGeluWarps + kOutWarps);
+constexpr uint32_t TM_S1 = 0, TM_OUT = 256, OUT_STRIDE = 128, TMEM_COLS = 512;
+constexpr int SMEM_TILES = (4 + 4 + 2 * NST) * KB_BYTES;     // A (2 buffers), H (2 buffers), weight ring
+constexpr int N_BARS = 8 + 2 * NST + 8;
 
 struct MlpArgs {
   int M, C, hidden, n_chunks, tiles;
+  uint32_t smem_bytes;
   const __nv_bfloat16 *b1, *b2, *residual;
   __nv_bfloat16* out;
   int* status;
@@ -50,43 +55,62 @@ __device__ __forceinline__ float gelu_tanh(float u) {
   return fmaf(h, t, h);
 }
 
+// n <= 4 k16 steps of one 64-wide k-block; both operands K-major with the 128-byte swizzle, so a
+// k16 step moves the descriptors' start address by 32 bytes (2 in descriptor units).
+__device__ __forceinline__ void issue_kblock(uint32_t d_tmem, uint64_t ad0, uint64_t bd0, uint32_t idesc, int n, bool acc_first) {
+  ptx::tc_mma_bf16(d_tmem, ad0, bd0, idesc, acc_first ? 1u : 0u);
+#pragma unroll
+  for (int k = 1; k < BK / 16; ++k)
+    if (k < n) ptx::tc_mma_bf16(d_tmem, ad0 + 2 * k, bd0 + 2 * k, idesc, 1u);
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW1,
                  const __grid_constant__ CUtensorMap tmW2, const __grid_constant__ MlpArgs g) {
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
-  uint8_t* sA = smem;                              // [2 k-blocks][16 KB]
-  uint8_t* sH = sA + 2 * KB_BYTES;                 // [2 bufs][2 k-blocks][16 KB]
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const uint32_t pad = (1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u;
+  uint8_t* smem = smem_raw + pad;
+  uint8_t* sA = smem;                              // [2 bufs][2 k-blocks][16 KB]
+  uint8_t* sH = sA + 4 * KB_BYTES;                 // [2 bufs][2 k-blocks][16 KB]
   uint8_t* sW = sH + 4 * KB_BYTES;                 // [NST][2 k-blocks][16 KB]
   uint64_t* bars = reinterpret_cast<uint64_t*>(sW + NST * WST_BYTES);
   uint64_t *a_full = bars, *a_empty = bars + 2, *w_full = bars + 4, *w_empty = w_full + NST;
   uint64_t *s1_full = w_empty + NST, *s1_empty = s1_full + 2, *h_full = s1_empty + 2, *h_empty = h_full + 2;
-  uint64_t *out_full = h_empty + 2, *out_empty = out_full + 1;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(out_empty + 1);
+  uint64_t *out_full = h_empty + 2, *out_empty = out_full + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(out_empty + 2);
   int* abort_flag = reinterpret_cast<int*>(tmem_slot + 1);
-  uint8_t* qstage_base = reinterpret_cast<uint8_t*>(tmem_slot + 4);
-  float* b1_s = reinterpret_cast<float*>(qstage_base + 4 * 32 * (g.C == 128 ? 256 : g.C * 2 + 16));   // [hidden]
+  float* b1_s = reinterpret_cast<float*>(tmem_slot + 4);     // [hidden]
+  float* b2_s = b1_s + g.hidden;                             // [C]
+
+  // The tiles fill the 227 KB almost completely, so the launch cannot afford a spare kilobyte of
+  // alignment slack: a base that is not 1024-aligned is reported instead of silently overrun.
+  if (pad + SMEM_TILES + N_BARS * 8 + 16 + (g.hidden + g.C) * 4 > g.smem_bytes) {
+    if (threadIdx.x == 0) atomicExch(g.status, (int)SMARTMEM_ERR_UNSUPPORTED);
+    return;
+  }
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int NC = g.n_chunks;
-  const int k1_last = (g.C - BK + 15) / 16;        // k16 steps of the second k-block of fc1 (C <= 128)
+  const int k1_last = (g.C - BK) / 16;             // k16 steps of the second k-block of fc1 (C <= 128)
   const int nkb1 = g.C > BK ? 2 : 1;
+  const int my_tiles = ((int)g.tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+  const int total = my_tiles * NC;                 // hidden chunks this CTA walks through, over all its tiles
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) {
       ptx::mbar_init(&a_full[i], 1);
       ptx::mbar_init(&a_empty[i], 1);
       ptx::mbar_init(&s1_full[i], 1);
-      ptx::mbar_init(&s1_empty[i], kEpiWarps);
-      ptx::mbar_init(&h_full[i], kEpiWarps);
+      ptx::mbar_init(&s1_empty[i], kGeluWarps);
+      ptx::mbar_init(&h_full[i], kGeluWarps);
       ptx::mbar_init(&h_empty[i], 1);
+      ptx::mbar_init(&out_full[i], 1);
+      ptx::mbar_init(&out_empty[i], kOutWarps);
     }
     for (int i = 0; i < NST; ++i) {
       ptx::mbar_init(&w_full[i], 1);
       ptx::mbar_init(&w_empty[i], 1);
     }
-    ptx::mbar_init(out_full, 1);
-    ptx::mbar_init(out_empty, kEpiWarps);
     *abort_flag = 0;
     ptx::fence_barrier_init();
     ptx::fence_proxy_async();
@@ -97,218 +121,244 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     ptx::prefetch_tensormap(&tmW2);
   }
   for (int i = threadIdx.x; i < g.hidden; i += kThreads) b1_s[i] = __bfloat162float(g.b1[i]);
+  for (int i = threadIdx.x; i < g.C; i += kThreads) b2_s[i] = __bfloat162float(g.b2[i]);
   if (warp == 1) ptx::tmem_alloc(tmem_slot, TMEM_COLS);
   ptx::tc_fence_before();
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
+  // fc1 runs one hidden chunk ahead of fc2 over the CTA's whole chunk sequence, across tile
+  // boundaries; each has its own issuing thread.  The weights of both share one ring, filled in
+  // the order  W1(0), then for j = 0..total-1: W1(j+1), W2(j).
   if (warp == 0) {
     if (lane == 0) {
-      uint32_t wcnt = 0, it = 0;
+      uint32_t ws = 0, wph = 1;
       bool ok = true;
-      auto load_w1 = [&](int c) {                      // [128 hidden rows] x C, as nkb1 k-blocks
-        const int s = wcnt % NST;
-        ok = ok && ptx::mbar_wait(&w_empty[s], ((wcnt / NST) & 1) ^ 1, abort_flag, g.status);
+      auto load_a = [&](int ti) {                      // ti: this CTA's ti-th tile
+        const int b = ti & 1;
+        ok = ok && ptx::mbar_wait(&a_empty[b], ((ti >> 1) & 1) ^ 1, abort_flag, g.status);
         if (!ok) return;
-        ptx::mbar_expect_tx(&w_full[s], nkb1 * KB_BYTES);
-        for (int kb = 0; kb < nkb1; ++kb) ptx::tma_load_2d(sW + s * WST_BYTES + kb * KB_BYTES, &tmW1, &w_full[s], kb * BK, c * HC);
-        ++wcnt;
+        const int t = (int)blockIdx.x + ti * (int)gridDim.x;
+        ptx::mbar_expect_tx(&a_full[b], nkb1 * KB_BYTES);
+        for (int kb = 0; kb < nkb1; ++kb)
+          ptx::tma_load_2d(sA + (b * 2 + kb) * KB_BYTES, &tmA, &a_full[b], kb * BK, t * BM);
+      };
+      auto load_w1 = [&](int c) {                      // [128 hidden rows] x C, as nkb1 k-blocks
+        ok = ok && ptx::mbar_wait(&w_empty[ws], wph, abort_flag, g.status);
+        if (!ok) return;
+        ptx::mbar_expect_tx(&w_full[ws], nkb1 * KB_BYTES);
+        for (int kb = 0; kb < nkb1; ++kb) ptx::tma_load_2d(sW + ws * WST_BYTES + kb * KB_BYTES, &tmW1, &w_full[ws], kb * BK, c * HC);
+        if (++ws == NST) { ws = 0; wph ^= 1; }
       };
       auto load_w2 = [&](int c) {                      // [C rows] x 128 hidden columns, as 2 k-blocks
-        const int s = wcnt % NST;
-        ok = ok && ptx::mbar_wait(&w_empty[s], ((wcnt / NST) & 1) ^ 1, abort_flag, g.status);
+        ok = ok && ptx::mbar_wait(&w_empty[ws], wph, abort_flag, g.status);
         if (!ok) return;
-        ptx::mbar_expect_tx(&w_full[s], 2 * (uint32_t)g.C * BK * 2);
-        for (int kb = 0; kb < 2; ++kb) ptx::tma_load_2d(sW + s * WST_BYTES + kb * KB_BYTES, &tmW2, &w_full[s], c * HC + kb * BK, 0);
-        ++wcnt;
+        ptx::mbar_expect_tx(&w_full[ws], 2 * (uint32_t)g.C * BK * 2);
+        for (int kb = 0; kb < 2; ++kb) ptx::tma_load_2d(sW + ws * WST_BYTES + kb * KB_BYTES, &tmW2, &w_full[ws], c * HC + kb * BK, 0);
+        if (++ws == NST) { ws = 0; wph ^= 1; }
       };
-      for (uint32_t t = blockIdx.x; t < (uint32_t)g.tiles && ok; t += gridDim.x, ++it) {
-        ok = ptx::mbar_wait(&a_empty[0], (it & 1) ^ 1, abort_flag, g.status);
-        if (!ok) break;
-        ptx::mbar_expect_tx(&a_full[0], nkb1 * KB_BYTES);
-        for (int kb = 0; kb < nkb1; ++kb)
-          ptx::tma_load_2d(sA + kb * KB_BYTES, &tmA, &a_full[0], kb * BK, (int)t * BM);
-        // weights in the order the MMA warp consumes them
+      if (total > 0) {
+        load_a(0);
         load_w1(0);
-        for (int c = 0; c < NC && ok; ++c) {
-          if (c + 1 < NC) load_w1(c + 1);
-          load_w2(c);
-        }
+      }
+      int ti = 0, c = 0;
+      for (int j = 0; j < total && ok; ++j) {
+        if (c == 0 && ti + 1 < my_tiles) load_a(ti + 1);     // the next tile's rows, a whole tile ahead
+        const int cn = c + 1 == NC ? 0 : c + 1;
+        if (j + 1 < total) load_w1(cn);
+        load_w2(c);
+        c = cn;
+        if (c == 0) ++ti;
       }
     }
   } else if (warp == 1) {
+    // fc1 issuer: S1[j & 1] = A W1[chunk j]^T, one chunk ahead of fc2.  Weight ring entry of
+    // chunk j's W1: 0 for j = 0, else 2j - 1 (the producer's order above).
     if (lane == 0) {
       const uint32_t idesc1 = ptx::make_idesc_bf16(BM, HC, false, false);
-      const uint32_t idesc2 = ptx::make_idesc_bf16(BM, g.C, false, false);
-      uint32_t wcnt = 0, it = 0, s1cnt = 0, hcnt = 0;
+      const uint32_t a_base = ptx::smem_u32(sA), w_base = ptx::smem_u32(sW);
+      int it1 = 0, c1 = 0;
       bool ok = true;
-      for (uint32_t t = blockIdx.x; t < (uint32_t)g.tiles && ok; t += gridDim.x, ++it) {
-        ok = ptx::mbar_wait(&a_full[0], it & 1, abort_flag, g.status);
+      for (int j = 0; j < total && ok; ++j) {
+        const uint32_t sb = j & 1, ab = it1 & 1;
+        const uint32_t n = j ? 2 * j - 1 : 0, ws = n % NST, wph = (n / NST) & 1;
+        DBG(j * 16 + 0);
+        if (c1 == 0) ok = ptx::mbar_wait(&a_full[ab], (it1 >> 1) & 1, abort_flag, g.status);
+        ok = ok && ptx::mbar_wait(&s1_empty[sb], ((j >> 1) & 1) ^ 1, abort_flag, g.status);
+        DBG(j * 16 + 1);
+        ok = ok && ptx::mbar_wait(&w_full[ws], wph, abort_flag, g.status);
         if (!ok) break;
-        auto fc1 = [&]() {                              // S1[buf] = A W1[chunk]^T
-          const uint32_t sb = s1cnt & 1;
-          ok = ok && ptx::mbar_wait(&s1_empty[sb], ((s1cnt >> 1) & 1) ^ 1, abort_flag, g.status);
-          if (ok) {
-            const int s = wcnt % NST;
-            ok = ptx::mbar_wait(&w_full[s], (wcnt / NST) & 1, abort_flag, g.status);
-            if (ok) {
-              ptx::tc_fence_after();
-              for (int kb = 0; kb < nkb1; ++kb) {
-                const uint32_t a0 = ptx::smem_u32(sA + kb * KB_BYTES), b0 = ptx::smem_u32(sW + s * WST_BYTES + kb * KB_BYTES);
-                const int ks = kb == 0 ? (g.C < BK ? g.C / 16 : BK / 16) : k1_last;
-                for (int k = 0; k < ks; ++k)
-                  ptx::tc_mma_bf16(tmem_base + TM_S1 + sb * HC, ptx::make_smem_desc(a0 + k * 32, 16, 1024),
-                                   ptx::make_smem_desc(b0 + k * 32, 16, 1024), idesc1, (kb | k) ? 1u : 0u);
-              }
-              ptx::tc_commit(&w_empty[s]);
-              ++wcnt;
-            }
-          }
-          if (ok) ptx::tc_commit(&s1_full[sb]);
-          ++s1cnt;
-        };
-        auto fc2 = [&](int c) {                         // OUT += H[chunk] W2[:, chunk]^T
-          const uint32_t hb = hcnt & 1;
-          ok = ok && ptx::mbar_wait(&h_full[hb], (hcnt >> 1) & 1, abort_flag, g.status);
-          if (ok && c == 0) ok = ptx::mbar_wait(out_empty, (it & 1) ^ 1, abort_flag, g.status);
-          if (ok) {
-            const int s = wcnt % NST;
-            ok = ptx::mbar_wait(&w_full[s], (wcnt / NST) & 1, abort_flag, g.status);
-            if (ok) {
-              ptx::tc_fence_after();
-              for (int kb = 0; kb < 2; ++kb) {
-                const uint32_t a0 = ptx::smem_u32(sH + (hb * 2 + kb) * KB_BYTES), b0 = ptx::smem_u32(sW + s * WST_BYTES + kb * KB_BYTES);
-                for (int k = 0; k < BK / 16; ++k)
-                  ptx::tc_mma_bf16(tmem_base + TM_OUT, ptx::make_smem_desc(a0 + k * 32, 16, 1024),
-                                   ptx::make_smem_desc(b0 + k * 32, 16, 1024), idesc2, (c | kb | k) ? 1u : 0u);
-              }
-              ptx::tc_commit(&w_empty[s]);
-              ++wcnt;
-            }
-          }
-          if (ok) ptx::tc_commit(&h_empty[hb]);
-          ++hcnt;
-        };
-        fc1();
-        for (int c = 0; c < NC && ok; ++c) {
-          if (c + 1 < NC) fc1();
-          if (c + 1 == NC && ok) ptx::tc_commit(&a_empty[0]);   // every fc1 MMA of this tile has been issued
-          fc2(c);
+        DBG(j * 16 + 2);
+        ptx::tc_fence_after();
+        const uint32_t d = tmem_base + TM_S1 + sb * HC;
+        const uint64_t ad = ptx::make_smem_desc(a_base + ab * 2 * KB_BYTES, 16, 1024);
+        const uint64_t bd = ptx::make_smem_desc(w_base + ws * WST_BYTES, 16, 1024);
+        issue_kblock(d, ad, bd, idesc1, BK / 16, false);
+        if (nkb1 > 1) issue_kblock(d, ad + (KB_BYTES >> 4), bd + (KB_BYTES >> 4), idesc1, k1_last, true);
+        ptx::tc_commit(&w_empty[ws]);
+        ptx::tc_commit(&s1_full[sb]);
+        DBG(j * 16 + 3);
+        if (++c1 == NC) {
+          ptx::tc_commit(&a_empty[ab]);                 // every fc1 MMA of this tile has been issued
+          c1 = 0;
+          ++it1;
         }
-        if (ok) ptx::tc_commit(out_full);
       }
     }
-  } else {
-    const int e = warp - 2, q = warp & 3, grp = e >> 2;
-    const int QROW = g.C == 128 ? 256 : g.C * 2 + 16;     // C = 128: no room left for the pad
-    uint8_t* qstage = qstage_base + q * (32 * QROW);
-    uint32_t it = 0, s1cnt = 0, hcnt = 0;
-    bool ok = true;
-    for (uint32_t t = blockIdx.x; t < (uint32_t)g.tiles && ok; t += gridDim.x, ++it) {
-      const int r_tile = q * 32 + lane;                  // row inside the tile = TMEM lane
-      const int row = (int)t * BM + r_tile;
-      const bool row_ok = row < g.M;
-      for (int c = 0; c < NC && ok; ++c, ++s1cnt, ++hcnt) {
-        const uint32_t sb = s1cnt & 1, hb = hcnt & 1;
-        float bb[32];                                    // this warp's 32 biases of the chunk, fetched before the wait
-#pragma unroll
-        for (int v = 0; v < 8; ++v) {
-          const float4 b4 = *reinterpret_cast<const float4*>(b1_s + c * HC + grp * 32 + v * 4);
-          bb[v * 4 + 0] = b4.x; bb[v * 4 + 1] = b4.y; bb[v * 4 + 2] = b4.z; bb[v * 4 + 3] = b4.w;
-        }
-        ok = ptx::mbar_wait(&s1_full[sb], (s1cnt >> 1) & 1, abort_flag, g.status);
+  } else if (warp == 2 + kGeluWarps + kOutWarps) {
+    // fc2 issuer: OUT[tile & 1] += H[j & 1] W2[:, chunk j]^T.  Ring entry of chunk j's W2:
+    // 2j + 2, except for the very last chunk, which no W1 load precedes: 2j + 1.
+    if (lane == 0) {
+      const uint32_t idesc2 = ptx::make_idesc_bf16(BM, g.C, false, false);
+      const uint32_t h_base = ptx::smem_u32(sH), w_base = ptx::smem_u32(sW);
+      int it2 = 0, c2 = 0;
+      bool ok = true;
+      for (int j = 0; j < total && ok; ++j) {
+        const uint32_t hb = j & 1, ob = it2 & 1;
+        const uint32_t n = j + 1 < total ? 2 * j + 2 : 2 * j + 1, ws = n % NST, wph = (n / NST) & 1;
+        DBG(j * 16 + 4);
+        ok = ptx::mbar_wait(&h_full[hb], (j >> 1) & 1, abort_flag, g.status);
+        if (c2 == 0) ok = ok && ptx::mbar_wait(&out_empty[ob], ((it2 >> 1) & 1) ^ 1, abort_flag, g.status);
+        DBG(j * 16 + 5);
+        ok = ok && ptx::mbar_wait(&w_full[ws], wph, abort_flag, g.status);
         if (!ok) break;
-        ok = ptx::mbar_wait(&h_empty[hb], ((hcnt >> 1) & 1) ^ 1, abort_flag, g.status);   // fc2 done with this buffer
-        if (!ok) break;
+        DBG(j * 16 + 6);
         ptx::tc_fence_after();
-        uint32_t rv[32];
-        ptx::tmem_ld32(tmem_base + TM_S1 + sb * HC + ((uint32_t)(q * 32) << 16) + grp * 32, rv);
-        ptx::tmem_ld_wait();
-        float acc[32];
-#pragma unroll
-#ifdef MLP_EXP_NOGELU
-        for (int j = 0; j < 32; ++j) acc[j] = __uint_as_float(rv[j]) + bb[j];
-#else
-        for (int j = 0; j < 32; ++j) acc[j] = gelu_tanh(__uint_as_float(rv[j]) + bb[j]);
-#endif
-        // chunk columns grp*32 .. +31 -> k-block (grp >> 1), 16-byte chunks ((grp & 1) * 4 + v) ^ (row & 7)
-        uint8_t* hrow = sH + (hb * 2 + (grp >> 1)) * KB_BYTES + r_tile * 128;
-#pragma unroll
-        for (int v = 0; v < 4; ++v) {
-          uint4 pk;
-          pk.x = float2_to_bf16x2(acc[v * 8 + 0], acc[v * 8 + 1]);
-          pk.y = float2_to_bf16x2(acc[v * 8 + 2], acc[v * 8 + 3]);
-          pk.z = float2_to_bf16x2(acc[v * 8 + 4], acc[v * 8 + 5]);
-          pk.w = float2_to_bf16x2(acc[v * 8 + 6], acc[v * 8 + 7]);
-          *reinterpret_cast<uint4*>(hrow + ((((grp & 1) * 4 + v) ^ (r_tile & 7)) << 4)) = pk;
-        }
-        ptx::fence_proxy_async();                        // make the generic-proxy writes visible to the MMA
-        ptx::tc_fence_before();
-        __syncwarp();
-        if (lane == 0) {
-          ptx::mbar_arrive(&h_full[hb]);
-          ptx::mbar_arrive(&s1_empty[sb]);
+        const uint32_t d = tmem_base + TM_OUT + ob * OUT_STRIDE;
+        const uint64_t ad = ptx::make_smem_desc(h_base + hb * 2 * KB_BYTES, 16, 1024);
+        const uint64_t bd = ptx::make_smem_desc(w_base + ws * WST_BYTES, 16, 1024);
+        issue_kblock(d, ad, bd, idesc2, BK / 16, c2 != 0);
+        issue_kblock(d, ad + (KB_BYTES >> 4), bd + (KB_BYTES >> 4), idesc2, BK / 16, true);
+        ptx::tc_commit(&w_empty[ws]);
+        ptx::tc_commit(&h_empty[hb]);
+        DBG(j * 16 + 7);
+        if (++c2 == NC) {
+          ptx::tc_commit(&out_full[ob]);
+          c2 = 0;
+          ++it2;
         }
       }
+    }
+  } else if (warp < 2 + kGeluWarps) {
+    // GELU warps: S1 chunk (TMEM) -> + b1 -> GELU -> bf16 -> H chunk in shared memory, in the
+    // K-major 128-byte-swizzled layout fc2 reads as its A operand.
+    const int e = warp - 2, q = warp & 3, grp = e >> 2;
+    const int r_tile = q * 32 + lane;                    // row inside the tile = TMEM lane
+    bool ok = true;
+    int c = 0;
+    for (int j = 0; j < total && ok; ++j) {
+      const uint32_t sb = j & 1, hb = j & 1, par = (j >> 1) & 1;
+      float bb[32];                                      // this warp's 32 biases of the chunk, fetched before the wait
+#pragma unroll
+      for (int v = 0; v < 8; ++v) {
+        const float4 b4 = *reinterpret_cast<const float4*>(b1_s + c * HC + grp * 32 + v * 4);
+        bb[v * 4 + 0] = b4.x; bb[v * 4 + 1] = b4.y; bb[v * 4 + 2] = b4.z; bb[v * 4 + 3] = b4.w;
+      }
+      if (e == 0 && lane == 0) DBG(j * 16 + 8);
+      ok = ptx::mbar_wait(&s1_full[sb], par, abort_flag, g.status);
       if (!ok) break;
-      // ---- final epilogue of the tile: OUT + b2 + residual -> out ------------------------------
-      const int CG = g.C / 4;                            // columns per warp: 16, 24 or 32
-      const int c0 = grp * CG;
+      if (e == 0 && lane == 0) DBG(j * 16 + 9);
+      ok = ptx::mbar_wait(&h_empty[hb], par ^ 1, abort_flag, g.status);   // fc2 done with this buffer
+      if (!ok) break;
+      ptx::tc_fence_after();
+      uint32_t rv[32];
+      ptx::tmem_ld32(tmem_base + TM_S1 + sb * HC + ((uint32_t)(q * 32) << 16) + grp * 32, rv);
+      ptx::tmem_ld_wait();
+      if (e == 0 && lane == 0) DBG(j * 16 + 10);
+      if (lane == 0) DBG(1024 + j * 16 + e);
+      float acc[32];
+#pragma unroll
+#ifdef MLP_EXP_NOGELU
+      for (int i = 0; i < 32; ++i) acc[i] = __uint_as_float(rv[i]) + bb[i];
+#else
+      for (int i = 0; i < 32; ++i) acc[i] = gelu_tanh(__uint_as_float(rv[i]) + bb[i]);
+#endif
+      // chunk columns grp*32 .. +31 -> k-block (grp >> 1), 16-byte chunks ((grp & 1) * 4 + v) ^ (row & 7)
+      uint8_t* hrow = sH + (hb * 2 + (grp >> 1)) * KB_BYTES + r_tile * 128;
+#pragma unroll
+      for (int v = 0; v < 4; ++v) {
+        uint4 pk;
+        pk.x = float2_to_bf16x2(acc[v * 8 + 0], acc[v * 8 + 1]);
+        pk.y = float2_to_bf16x2(acc[v * 8 + 2], acc[v * 8 + 3]);
+        pk.z = float2_to_bf16x2(acc[v * 8 + 4], acc[v * 8 + 5]);
+        pk.w = float2_to_bf16x2(acc[v * 8 + 6], acc[v * 8 + 7]);
+        *reinterpret_cast<uint4*>(hrow + ((((grp & 1) * 4 + v) ^ (r_tile & 7)) << 4)) = pk;
+      }
+      if (e == 0 && lane == 0) DBG(j * 16 + 11);
+      if (lane == 0) DBG(2048 + j * 16 + e);
+      ptx::fence_proxy_async();                          // make the generic-proxy writes visible to the MMA
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) {
+        ptx::mbar_arrive(&h_full[hb]);
+        ptx::mbar_arrive(&s1_empty[sb]);
+      }
+      if (++c == NC) c = 0;
+    }
+  } else if (warp < 2 + kGeluWarps + kOutWarps) {
+    // Output warps, one per TMEM lane quadrant: OUT + b2 + residual -> out, a thread per row, in
+    // rounds of 32 columns.  They work on one OUT buffer while fc2 of the next tile fills the other.
+    const int q = warp & 3;
+    const int rounds = g.C / 32;
+    bool ok = true;
+    for (int ti = 0; ti < my_tiles && ok; ++ti) {
+      const uint32_t ob = ti & 1;
+      const int t = (int)blockIdx.x + ti * (int)gridDim.x;
+      const int row = t * BM + q * 32 + lane;
+      const bool row_ok = row < g.M;
       const long long off = (long long)row * g.C;
-      uint4 res[4];
+      uint4 res[4], resn[4];
 #pragma unroll
       for (int v = 0; v < 4; ++v) {
         res[v] = make_uint4(0, 0, 0, 0);
-        if (g.residual && row_ok && v * 8 < CG) res[v] = *reinterpret_cast<const uint4*>(g.residual + off + c0 + v * 8);
+        if (g.residual && row_ok) res[v] = *reinterpret_cast<const uint4*>(g.residual + off + v * 8);
       }
-      ok = ptx::mbar_wait(out_full, it & 1, abort_flag, g.status);
+      if (q == 0 && lane == 0) DBG(ti * NC * 16 + 12);
+      ok = ptx::mbar_wait(&out_full[ob], (ti >> 1) & 1, abort_flag, g.status);
       if (!ok) break;
+      if (q == 0 && lane == 0) DBG(ti * NC * 16 + 13);
       ptx::tc_fence_after();
-      {
-        uint32_t rv[32];
-        const uint32_t ta = tmem_base + TM_OUT + ((uint32_t)(q * 32) << 16) + c0;
-        if (CG == 32) ptx::tmem_ld32(ta, rv);
-        else {
-          ptx::tmem_ld16(ta, rv);
-          if (CG == 24) ptx::tmem_ld8(ta + 16, rv + 16);
-        }
-        ptx::tmem_ld_wait();
 #pragma unroll
-        for (int v = 0; v < 4; ++v) {
-          if (v * 8 < CG) {
-            float a8[8], bb[8];
-            ElemIO<__nv_bfloat16>::load(g.b2 + c0 + v * 8, bb);
+      for (int r = 0; r < 4; ++r) {
+        if (r < rounds) {
+          uint32_t rv[32];
+          ptx::tmem_ld32(tmem_base + TM_OUT + ob * OUT_STRIDE + ((uint32_t)(q * 32) << 16) + r * 32, rv);
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            resn[v] = make_uint4(0, 0, 0, 0);
+            if (g.residual && row_ok && r + 1 < rounds)
+              resn[v] = *reinterpret_cast<const uint4*>(g.residual + off + (r + 1) * 32 + v * 8);
+          }
+          ptx::tmem_ld_wait();
+          if (r + 1 == rounds) {                         // the accumulator is in registers: hand the buffer back
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&out_empty[ob]);
+          }
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
             const uint32_t w[4] = {res[v].x, res[v].y, res[v].z, res[v].w};
+            float a8[8];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const float2 f = bf16x2_to_float2(w[j]);
-              a8[2 * j] = __uint_as_float(rv[v * 8 + 2 * j]) + bb[2 * j] + f.x;
-              a8[2 * j + 1] = __uint_as_float(rv[v * 8 + 2 * j + 1]) + bb[2 * j + 1] + f.y;
+            for (int i = 0; i < 4; ++i) {
+              const float2 f = bf16x2_to_float2(w[i]);
+              const float2 b = *reinterpret_cast<const float2*>(b2_s + r * 32 + v * 8 + 2 * i);
+              a8[2 * i] = __uint_as_float(rv[v * 8 + 2 * i]) + b.x + f.x;
+              a8[2 * i + 1] = __uint_as_float(rv[v * 8 + 2 * i + 1]) + b.y + f.y;
             }
             uint4 pk;
             pk.x = float2_to_bf16x2(a8[0], a8[1]);
             pk.y = float2_to_bf16x2(a8[2], a8[3]);
             pk.z = float2_to_bf16x2(a8[4], a8[5]);
             pk.w = float2_to_bf16x2(a8[6], a8[7]);
-            *reinterpret_cast<uint4*>(qstage + lane * QROW + (c0 + v * 8) * 2) = pk;
+            if (row_ok) *reinterpret_cast<uint4*>(g.out + off + r * 32 + v * 8) = pk;
           }
+#pragma unroll
+          for (int v = 0; v < 4; ++v) res[v] = resn[v];
         }
       }
-      ptx::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(out_empty);
-      // the four warps of the quadrant have filled a 32 x C staging tile: store whole rows
-      asm volatile("bar.sync %0, 128;" ::"r"(1 + q) : "memory");
-      const int VR = g.C / 8, tq = grp * 32 + lane;
-      for (int v = tq; v < 32 * VR; v += 128) {
-        const int rr = v / VR, seg = v - rr * VR;
-        const int grow = (int)t * BM + q * 32 + rr;
-        if (grow < g.M)
-          *reinterpret_cast<uint4*>(g.out + (long long)grow * g.C + seg * 8) =
-              *reinterpret_cast<const uint4*>(qstage + rr * QROW + seg * 16);
-      }
-      asm volatile("bar.sync %0, 128;" ::"r"(1 + q) : "memory");
+      if (q == 0 && lane == 0) DBG(ti * NC * 16 + 14);
     }
   }
   ptx::tc_fence_before();
@@ -322,7 +372,7 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 }  // namespace
 
 bool mlp_fused_supported(long long C, long long hidden) {
-  return (C == 64 || C == 96) && hidden >= HC && hidden % HC == 0 && hidden <= 1024;
+  return (C == 64 || C == 96) && hidden >= HC && hidden % HC == 0 && hidden <= 512;
 }
 
 int launch_mlp_fused(const void* A, const void* W1, const void* b1, const void* W2, const void* b2, const void* residual,
@@ -345,8 +395,10 @@ int launch_mlp_fused(const void* A, const void* W1, const void* b1, const void* 
   g.out = (__nv_bfloat16*)out;
   g.status = device_status_ptr();
   if (!g.status) return SMARTMEM_ERR_CUDA;
-  const size_t smem = 1024 + (2 + 4 + 2 * NST) * KB_BYTES + (8 + 2 * NST + 6) * 8 + 16 + 4 * 32 * (C == 128 ? 256 : C * 2 + 16) +
-                      (size_t)hidden * 4;
+  const size_t need = (size_t)SMEM_TILES + N_BARS * 8 + 16 + (size_t)(hidden + C) * 4;
+  const size_t smem = need + 1024 <= 232448 ? need + 1024 : 232448;     // alignment slack only while it fits
+  if (need > smem) return SMARTMEM_ERR_UNSUPPORTED;
+  g.smem_bytes = (uint32_t)smem;
   static bool configured = false;
   if (!configured) {
     if (cudaFuncSetAttribute(mlp_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448) != cudaSuccess)

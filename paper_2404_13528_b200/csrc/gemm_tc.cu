@@ -163,7 +163,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   if (warp == 0) {
     if (lane == 0) {
-      uint32_t kbg = 0;                                      // k-block counter across tiles
+      uint32_t kbg = 0, s = 0, ph = 0;                       // k-block counter across tiles, ring position
       bool ok = true;
       uint32_t pit = 0;
       for (uint32_t t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++pit) {
@@ -171,8 +171,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         GDBG(pit * 16 + 0);
         const TileCoord ta = op_coords(g.ca, tile_m, batch, BM), tb = op_coords(g.cb, tile_n, batch, BN);
         for (int kb = 0; kb < nkb; ++kb, ++kbg) {
-          const int s = kbg % STAGES;
-          const uint32_t ph = (kbg / STAGES) & 1;
           ok = ptx::mbar_wait(&empty[s], ph ^ 1, abort_flag, g.status);
           if (kb == 0) GDBG(pit * 16 + 1);
           if (!ok) break;
@@ -180,6 +178,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           tma_load_op(g.ca, sA + s * A_STAGE_BYTES, &tmA, &full[s], kb * BK, ta.row0, ta);
           if (A_MN) tma_load_op(g.ca, sA + s * A_STAGE_BYTES + A_STAGE_BYTES / 2, &tmA, &full[s], kb * BK, ta.row0 + 64, ta);
           if (!two_producers) tma_load_op(g.cb, sB + s * B_STAGE_BYTES, &tmB, &full[s], kb * BK, tb.row0, tb);
+          if (++s == STAGES) { s = 0; ph ^= 1; }
         }
         GDBG(pit * 16 + 2);
       }
@@ -194,7 +193,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      uint32_t kbg = 0, it = 0;
+      uint32_t it = 0, s = 0, ph = 0;                 // ring position and its phase carry over tiles
+      const uint32_t a_base = ptx::smem_u32(sA), b_base = ptx::smem_u32(sB);
       bool ok = true;
       for (uint32_t t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
         const uint32_t buf = it & 1, use = it >> 1;
@@ -204,26 +204,30 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         GDBG(it * 16 + 4);
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * ACC_COLS;
-        for (int kb = 0; kb < nkb; ++kb, ++kbg) {
-          const int s = kbg % STAGES;
-          const uint32_t ph = (kbg / STAGES) & 1;
+        for (int kb = 0; kb < nkb; ++kb) {
           ok = ptx::mbar_wait(&full[s], ph, abort_flag, g.status);
           if (!ok) break;
           if (kb == 0) GDBG(it * 16 + 5);
           if (kb == 1) GDBG(it * 16 + 6);
           ptx::tc_fence_after();
-          const uint32_t a0 = ptx::smem_u32(sA + s * A_STAGE_BYTES), b0 = ptx::smem_u32(sB + s * B_STAGE_BYTES);
-          const int ks = (kb == nkb - 1) ? last_ksteps : BK / 16;
-          for (int k = 0; k < ks; ++k) {
-            // K-major, 128-byte swizzle: 8-row groups are 1024 bytes apart; one k16 step is 32 bytes
-            // along the swizzled row.  MN-major: 64-row chunks are 8192 bytes apart (leading offset),
-            // 8-deep k groups 1024 bytes apart, one k16 step is 2048 bytes.
-            const uint64_t ad = A_MN ? ptx::make_smem_desc(a0 + k * 2048, A_STAGE_BYTES / 2, 1024)
-                                     : ptx::make_smem_desc(a0 + k * 32, 16, 1024);
-            const uint64_t bd = ptx::make_smem_desc(b0 + k * 32, 16, 1024);
-            ptx::tc_mma_bf16(d_tmem, ad, bd, IDESC, (kb | k) ? 1u : 0u);
+          // K-major, 128-byte swizzle: 8-row groups are 1024 bytes apart; one k16 step is 32 bytes
+          // along the swizzled row.  MN-major: 64-row chunks are 8192 bytes apart (leading offset),
+          // 8-deep k groups 1024 bytes apart, one k16 step is 2048 bytes.  A k16 step only moves the
+          // start-address field of the descriptor, so the issuing thread adds a constant per MMA.
+          const uint64_t ad0 = A_MN ? ptx::make_smem_desc(a_base + s * A_STAGE_BYTES, A_STAGE_BYTES / 2, 1024)
+                                    : ptx::make_smem_desc(a_base + s * A_STAGE_BYTES, 16, 1024);
+          const uint64_t bd0 = ptx::make_smem_desc(b_base + s * B_STAGE_BYTES, 16, 1024);
+          constexpr uint64_t A_STEP = (A_MN ? 2048 : 32) >> 4, B_STEP = 32 >> 4;
+          if (kb != nkb - 1 || last_ksteps == BK / 16) {
+            ptx::tc_mma_bf16(d_tmem, ad0, bd0, IDESC, kb ? 1u : 0u);
+#pragma unroll
+            for (int k = 1; k < BK / 16; ++k) ptx::tc_mma_bf16(d_tmem, ad0 + k * A_STEP, bd0 + k * B_STEP, IDESC, 1u);
+          } else {
+            for (int k = 0; k < last_ksteps; ++k)
+              ptx::tc_mma_bf16(d_tmem, ad0 + k * A_STEP, bd0 + k * B_STEP, IDESC, (kb | k) ? 1u : 0u);
           }
           ptx::tc_commit(&empty[s]);
+          if (++s == STAGES) { s = 0; ph ^= 1; }
         }
         if (ok) ptx::tc_commit(&tmem_full[buf]);
         GDBG(it * 16 + 7);
@@ -233,17 +237,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // second producer: the B operand (long reductions only; a short one is
     // cheaper to feed from one thread)
     if (lane == 0 && two_producers) {
-      uint32_t kbg = 0;
+      uint32_t s = 0, ph = 1;
       bool ok = true;
       for (uint32_t t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
         const uint32_t tile_n = t % g.tiles_n, r = t / g.tiles_n, batch = r / g.tiles_m;
         const TileCoord tb = op_coords(g.cb, tile_n, batch, BN);
-        for (int kb = 0; kb < nkb; ++kb, ++kbg) {
-          const int s = kbg % STAGES;
-          ok = ptx::mbar_wait(&empty[s], ((kbg / STAGES) & 1) ^ 1, abort_flag, g.status);
+        for (int kb = 0; kb < nkb; ++kb) {
+          ok = ptx::mbar_wait(&empty[s], ph, abort_flag, g.status);
           if (!ok) break;
           ptx::mbar_expect_tx(&full[s], B_STAGE_BYTES);
           tma_load_op(g.cb, sB + s * B_STAGE_BYTES, &tmB, &full[s], kb * BK, tb.row0, tb);
+          if (++s == STAGES) { s = 0; ph ^= 1; }
         }
       }
     }
