@@ -51,7 +51,6 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
       "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
       : "memory");
 }
-__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 __global__ void __launch_bounds__(kThreads, 1)
 causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -238,7 +237,7 @@ causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           for (int c = 0; c < 32; ++c) rv[c] = __float_as_uint(__uint_as_float(rv[c]) * (rescale ? corr : 1.f));
           tmem_st32(to + ch * 32, rv);
         }
-        tmem_st_wait();
+        ptx::tmem_st_wait();
       }
       // P row r: 16 chunks of 8 keys; chunk c8 lives in k-block c8 / 8 at position (c8 % 8) ^ (r % 8)
 #pragma unroll

@@ -31,12 +31,12 @@ namespace {
 
 constexpr int BM = 128, BK = 64, HC = 128;         // tile rows, k-block, hidden chunk
 constexpr int KB_BYTES = BM * BK * 2;              // one 128 x 64 bf16 operand block: 16 KB
-constexpr int NST = 3;                             // weight ring stages; one stage = both k-blocks of a chunk's W1 or W2
+constexpr int NST = 4;                             // weight ring stages; one stage = both k-blocks of a chunk's W1 or W2
 constexpr int WST_BYTES = 2 * KB_BYTES;
 constexpr int kGeluWarps = 16, kOutWarps = 4, kThreads = 32 * (3 + kGeluWarps + kOutWarps);
 constexpr uint32_t TM_S1 = 0, TM_OUT = 256, OUT_STRIDE = 128, TMEM_COLS = 512;
-constexpr int SMEM_TILES = (4 + 4 + 2 * NST) * KB_BYTES;     // A (2 buffers), H (2 buffers), weight ring
-constexpr int N_BARS = 8 + 2 * NST + 8;
+constexpr int SMEM_TILES = (4 + 2 * NST) * KB_BYTES;         // A (2 buffers), weight ring
+constexpr int N_BARS = 4 + 2 * NST + 2 + 2 + 2 + 4;
 
 struct MlpArgs {
   int M, C, hidden, n_chunks, tiles;
@@ -71,12 +71,11 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   const uint32_t pad = (1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u;
   uint8_t* smem = smem_raw + pad;
   uint8_t* sA = smem;                              // [2 bufs][2 k-blocks][16 KB]
-  uint8_t* sH = sA + 4 * KB_BYTES;                 // [2 bufs][2 k-blocks][16 KB]
-  uint8_t* sW = sH + 4 * KB_BYTES;                 // [NST][2 k-blocks][16 KB]
+  uint8_t* sW = sA + 4 * KB_BYTES;                 // [NST][2 k-blocks][16 KB]
   uint64_t* bars = reinterpret_cast<uint64_t*>(sW + NST * WST_BYTES);
   uint64_t *a_full = bars, *a_empty = bars + 2, *w_full = bars + 4, *w_empty = w_full + NST;
-  uint64_t *s1_full = w_empty + NST, *s1_empty = s1_full + 2, *h_full = s1_empty + 2, *h_empty = h_full + 2;
-  uint64_t *out_full = h_empty + 2, *out_empty = out_full + 2;
+  uint64_t *s1_full = w_empty + NST, *s1_empty = s1_full + 2, *h_full = s1_empty + 2;
+  uint64_t *out_full = h_full + 2, *out_empty = out_full + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(out_empty + 2);
   int* abort_flag = reinterpret_cast<int*>(tmem_slot + 1);
   float* b1_s = reinterpret_cast<float*>(tmem_slot + 4);     // [hidden]
@@ -101,9 +100,8 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       ptx::mbar_init(&a_full[i], 1);
       ptx::mbar_init(&a_empty[i], 1);
       ptx::mbar_init(&s1_full[i], 1);
-      ptx::mbar_init(&s1_empty[i], kGeluWarps);
+      ptx::mbar_init(&s1_empty[i], 1);
       ptx::mbar_init(&h_full[i], kGeluWarps);
-      ptx::mbar_init(&h_empty[i], 1);
       ptx::mbar_init(&out_full[i], 1);
       ptx::mbar_init(&out_empty[i], kOutWarps);
     }
@@ -211,7 +209,7 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     // 2j + 2, except for the very last chunk, which no W1 load precedes: 2j + 1.
     if (lane == 0) {
       const uint32_t idesc2 = ptx::make_idesc_bf16(BM, g.C, false, false);
-      const uint32_t h_base = ptx::smem_u32(sH), w_base = ptx::smem_u32(sW);
+      const uint32_t w_base = ptx::smem_u32(sW);
       int it2 = 0, c2 = 0;
       bool ok = true;
       for (int j = 0; j < total && ok; ++j) {
@@ -226,12 +224,14 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         DBG(j * 16 + 6);
         ptx::tc_fence_after();
         const uint32_t d = tmem_base + TM_OUT + ob * OUT_STRIDE;
-        const uint64_t ad = ptx::make_smem_desc(h_base + hb * 2 * KB_BYTES, 16, 1024);
+        const uint32_t a = tmem_base + TM_S1 + hb * HC;     // H chunk: 128 bf16 per lane = 64 columns
         const uint64_t bd = ptx::make_smem_desc(w_base + ws * WST_BYTES, 16, 1024);
-        issue_kblock(d, ad, bd, idesc2, BK / 16, c2 != 0);
-        issue_kblock(d, ad + (KB_BYTES >> 4), bd + (KB_BYTES >> 4), idesc2, BK / 16, true);
+        ptx::tc_mma_bf16_ta(d, a, bd, idesc2, c2 != 0 ? 1u : 0u);
+#pragma unroll
+        for (int k = 1; k < HC / 16; ++k)
+          ptx::tc_mma_bf16_ta(d, a + 8 * k, bd + (k >> 2) * (KB_BYTES >> 4) + 2 * (k & 3), idesc2, 1u);
         ptx::tc_commit(&w_empty[ws]);
-        ptx::tc_commit(&h_empty[hb]);
+        ptx::tc_commit(&s1_empty[hb]);                  // H lived in the S1 buffer: fc1 may overwrite it now
         DBG(j * 16 + 7);
         if (++c2 == NC) {
           ptx::tc_commit(&out_full[ob]);
@@ -241,14 +241,15 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       }
     }
   } else if (warp < 2 + kGeluWarps) {
-    // GELU warps: S1 chunk (TMEM) -> + b1 -> GELU -> bf16 -> H chunk in shared memory, in the
-    // K-major 128-byte-swizzled layout fc2 reads as its A operand.
+    // GELU warps: S1 chunk (TMEM, fp32) -> + b1 -> GELU -> bf16 pairs -> back into the first 64
+    // columns of the same TMEM buffer, where fc2 reads the chunk as its A operand.  The packed H
+    // columns of one warp overlap S1 columns another warp of the quadrant still has to read, so
+    // the quadrant's four warps meet between their loads and their stores.
     const int e = warp - 2, q = warp & 3, grp = e >> 2;
-    const int r_tile = q * 32 + lane;                    // row inside the tile = TMEM lane
     bool ok = true;
     int c = 0;
     for (int j = 0; j < total && ok; ++j) {
-      const uint32_t sb = j & 1, hb = j & 1, par = (j >> 1) & 1;
+      const uint32_t sb = j & 1;
       float bb[32];                                      // this warp's 32 biases of the chunk, fetched before the wait
 #pragma unroll
       for (int v = 0; v < 8; ++v) {
@@ -256,44 +257,43 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         bb[v * 4 + 0] = b4.x; bb[v * 4 + 1] = b4.y; bb[v * 4 + 2] = b4.z; bb[v * 4 + 3] = b4.w;
       }
       if (e == 0 && lane == 0) DBG(j * 16 + 8);
-      ok = ptx::mbar_wait(&s1_full[sb], par, abort_flag, g.status);
-      if (!ok) break;
+      ok = ptx::mbar_wait(&s1_full[sb], (j >> 1) & 1, abort_flag, g.status);
       if (e == 0 && lane == 0) DBG(j * 16 + 9);
-      ok = ptx::mbar_wait(&h_empty[hb], par ^ 1, abort_flag, g.status);   // fc2 done with this buffer
-      if (!ok) break;
-      ptx::tc_fence_after();
+      const uint32_t tq = tmem_base + TM_S1 + sb * HC + ((uint32_t)(q * 32) << 16);
       uint32_t rv[32];
-      ptx::tmem_ld32(tmem_base + TM_S1 + sb * HC + ((uint32_t)(q * 32) << 16) + grp * 32, rv);
-      ptx::tmem_ld_wait();
-      if (e == 0 && lane == 0) DBG(j * 16 + 10);
-      if (lane == 0) DBG(1024 + j * 16 + e);
-      float acc[32];
-#pragma unroll
-#ifdef MLP_EXP_NOGELU
-      for (int i = 0; i < 32; ++i) acc[i] = __uint_as_float(rv[i]) + bb[i];
-#else
-      for (int i = 0; i < 32; ++i) acc[i] = gelu_tanh(__uint_as_float(rv[i]) + bb[i]);
-#endif
-      // chunk columns grp*32 .. +31 -> k-block (grp >> 1), 16-byte chunks ((grp & 1) * 4 + v) ^ (row & 7)
-      uint8_t* hrow = sH + (hb * 2 + (grp >> 1)) * KB_BYTES + r_tile * 128;
-#pragma unroll
-      for (int v = 0; v < 4; ++v) {
-        uint4 pk;
-        pk.x = float2_to_bf16x2(acc[v * 8 + 0], acc[v * 8 + 1]);
-        pk.y = float2_to_bf16x2(acc[v * 8 + 2], acc[v * 8 + 3]);
-        pk.z = float2_to_bf16x2(acc[v * 8 + 4], acc[v * 8 + 5]);
-        pk.w = float2_to_bf16x2(acc[v * 8 + 6], acc[v * 8 + 7]);
-        *reinterpret_cast<uint4*>(hrow + ((((grp & 1) * 4 + v) ^ (r_tile & 7)) << 4)) = pk;
+      if (ok) {
+        ptx::tc_fence_after();
+        ptx::tmem_ld32(tq + grp * 32, rv);
+        ptx::tmem_ld_wait();
       }
+      // always reached by all four warps of the quadrant; they leave together if any gave up waiting
+      uint32_t gave_up;
+      asm volatile(
+          "{\n\t.reg .pred pin, pout;\n\t"
+          "setp.ne.u32 pin, %2, 0;\n\t"
+          "bar.red.or.pred pout, %1, 128, pin;\n\t"
+          "selp.u32 %0, 1, 0, pout;\n\t}"
+          : "=r"(gave_up)
+          : "r"(1 + q), "r"(ok ? 0u : 1u)
+          : "memory");
+      if (gave_up) break;
+      if (e == 0 && lane == 0) DBG(j * 16 + 10);
+      uint32_t pk[16];
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+#ifdef MLP_EXP_NOGELU
+        pk[i] = float2_to_bf16x2(__uint_as_float(rv[2 * i]) + bb[2 * i], __uint_as_float(rv[2 * i + 1]) + bb[2 * i + 1]);
+#else
+        pk[i] = float2_to_bf16x2(gelu_tanh(__uint_as_float(rv[2 * i]) + bb[2 * i]),
+                                 gelu_tanh(__uint_as_float(rv[2 * i + 1]) + bb[2 * i + 1]));
+#endif
+      }
+      ptx::tmem_st16(tq + grp * 16, pk);
+      ptx::tmem_st_wait();
       if (e == 0 && lane == 0) DBG(j * 16 + 11);
-      if (lane == 0) DBG(2048 + j * 16 + e);
-      ptx::fence_proxy_async();                          // make the generic-proxy writes visible to the MMA
       ptx::tc_fence_before();
       __syncwarp();
-      if (lane == 0) {
-        ptx::mbar_arrive(&h_full[hb]);
-        ptx::mbar_arrive(&s1_empty[sb]);
-      }
+      if (lane == 0) ptx::mbar_arrive(&h_full[sb]);
       if (++c == NC) c = 0;
     }
   } else if (warp < 2 + kGeluWarps + kOutWarps) {
