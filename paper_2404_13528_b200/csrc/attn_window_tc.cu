@@ -129,6 +129,8 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();                       // the tables above depend on parameters only: they overlapped the previous kernel's tail
+  pdl_launch_dependents();
   const CUtensorMap* tms[3] = {&tm0, &tm1, &tm2};
   const AttnOperand* ops[3] = {&a.q, &a.k, &a.v};
 
@@ -418,7 +420,7 @@ int launch_window_attention_tc(const WinAttnArgs& a_in, long long n_windows, cud
   if (per_head > g.n_pairs) per_head = g.n_pairs;
   const unsigned grid = (unsigned)(per_head * a.heads);
   profile_tick("window_attention_tc", st);
-  win_attn_tc_kernel<<<grid, kThreads, smem, st>>>(tm[0], tm[1], tm[2], g);
+  launch_pdl(win_attn_tc_kernel, dim3(grid), dim3(kThreads), smem, st, tm[0], tm[1], tm[2], g);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
 }

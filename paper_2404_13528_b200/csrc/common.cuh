@@ -13,6 +13,33 @@ namespace smartmem {
 // ---------------------------------------------------------------------------------------
 int* device_status_ptr();                 // device address of the status word (per process)
 void count_launch(int n = 1);
+
+// Programmatic dependent launch.  A kernel launched through `launch_pdl` may start (be scheduled,
+// set up its barriers and tensor memory, prefetch its descriptors and constants) while the kernel
+// before it in the stream is still draining; it must call `pdl_wait()` before it reads or writes
+// anything that kernel could touch.  The wait returns once the whole preceding grid has finished
+// and its writes are visible.  `pdl_launch_dependents()` lets the NEXT kernel in the stream begin
+// that early start as soon as every CTA of this one has called it.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 // When a profiling session is open (smartmem_profile_begin), records a CUDA event on `st` labelled
 // `name`; every launcher calls it right before its kernel launch.
 void profile_tick(const char* name, cudaStream_t st);

@@ -13,17 +13,20 @@
 // ring: they stay L2-resident), warp 1 fc1 issuer + TMEM owner, warps 2-17 GELU (TMEM -> shared
 // memory), warps 18-21 output (OUT + b2 + residual -> global, OUT double-buffered in TMEM so they
 // overlap the next tile), warp 22 fc2 issuer.
+
 #include "gemm_tc.cuh"
 #include "ptx.cuh"
 
 #ifdef MLP_EXP_TIMING
 __device__ long long g_mlp_dbg[8192];
 #define DBG(slot) do { if (blockIdx.x == 0) g_mlp_dbg[(slot)] = clock64(); } while (0)
+#define DBGT(k) do { if (threadIdx.x == 0) g_mlp_dbg[6000 + blockIdx.x * 4 + (k)] = (long long)smartmem::ptx::globaltimer(); } while (0)
 extern "C" __attribute__((visibility("default"))) int smartmem_debug_read(long long* host, int n) {
   return (int)cudaMemcpyFromSymbol(host, g_mlp_dbg, sizeof(long long) * n);
 }
 #else
 #define DBG(slot) do { } while (0)
+#define DBGT(k) do { } while (0)
 #endif
 
 namespace smartmem {
@@ -46,13 +49,21 @@ struct MlpArgs {
   int* status;
 };
 
-__device__ __forceinline__ float gelu_tanh(float u) {
-  const float u2 = u * u;
-  const float inner = u * fmaf(0.0356774081f, u2, 0.7978845608f);
-  float t;
-  asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(inner));
-  const float h = 0.5f * u;
-  return fmaf(h, t, h);
+// tanh-form GELU of two pre-activations, evaluated on packed bf16 pairs: the result is stored as
+// bf16 anyway, and the packed path costs one conversion, five packed multiply-adds and one
+// tanh.approx per PAIR, where the fp32 form costs seven instructions per element.  These warps are
+// what bounds the kernel, and they are bound by instruction issue and by the special-function unit.
+__device__ __forceinline__ uint32_t gelu_tanh_bf16x2(float a, float b) {
+  const uint32_t u = float2_to_bf16x2(a, b);
+  constexpr uint32_t C0 = 0x3F4C3F4Cu, C1 = 0x3D123D12u, HALF = 0x3F003F00u;   // 0.7979, 0.03568, 0.5
+  uint32_t u2, p, in, t, h, r;
+  asm("mul.rn.bf16x2 %0, %1, %1;" : "=r"(u2) : "r"(u));
+  asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(p) : "r"(C1), "r"(u2), "r"(C0));
+  asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(in) : "r"(u), "r"(p));
+  asm("tanh.approx.bf16x2 %0, %1;" : "=r"(t) : "r"(in));
+  asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(h) : "r"(u), "r"(HALF));
+  asm("fma.rn.bf16x2 %0, %1, %2, %1;" : "=r"(r) : "r"(h), "r"(t));
+  return r;
 }
 
 // n <= 4 k16 steps of one 64-wide k-block; both operands K-major with the 128-byte swizzle, so a
@@ -67,6 +78,7 @@ __device__ __forceinline__ void issue_kblock(uint32_t d_tmem, uint64_t ad0, uint
 __global__ void __launch_bounds__(kThreads, 1)
 mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW1,
                  const __grid_constant__ CUtensorMap tmW2, const __grid_constant__ MlpArgs g) {
+  DBGT(0);
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const uint32_t pad = (1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u;
   uint8_t* smem = smem_raw + pad;
@@ -125,6 +137,9 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();                       // everything above (weights' biases included) overlapped the previous kernel's tail
+  pdl_launch_dependents();
+  DBGT(1);
 
   // fc1 runs one hidden chunk ahead of fc2 over the CTA's whole chunk sequence, across tile
   // boundaries; each has its own issuing thread.  The weights of both share one ring, filled in
@@ -135,7 +150,7 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       bool ok = true;
       auto load_a = [&](int ti) {                      // ti: this CTA's ti-th tile
         const int b = ti & 1;
-        ok = ok && ptx::mbar_wait(&a_empty[b], ((ti >> 1) & 1) ^ 1, abort_flag, g.status);
+        ok = ok && ptx::mbar_wait_relaxed(&a_empty[b], ((ti >> 1) & 1) ^ 1, abort_flag, g.status);
         if (!ok) return;
         const int t = (int)blockIdx.x + ti * (int)gridDim.x;
         ptx::mbar_expect_tx(&a_full[b], nkb1 * KB_BYTES);
@@ -143,14 +158,14 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           ptx::tma_load_2d(sA + (b * 2 + kb) * KB_BYTES, &tmA, &a_full[b], kb * BK, t * BM);
       };
       auto load_w1 = [&](int c) {                      // [128 hidden rows] x C, as nkb1 k-blocks
-        ok = ok && ptx::mbar_wait(&w_empty[ws], wph, abort_flag, g.status);
+        ok = ok && ptx::mbar_wait_relaxed(&w_empty[ws], wph, abort_flag, g.status);
         if (!ok) return;
         ptx::mbar_expect_tx(&w_full[ws], nkb1 * KB_BYTES);
         for (int kb = 0; kb < nkb1; ++kb) ptx::tma_load_2d(sW + ws * WST_BYTES + kb * KB_BYTES, &tmW1, &w_full[ws], kb * BK, c * HC);
         if (++ws == NST) { ws = 0; wph ^= 1; }
       };
       auto load_w2 = [&](int c) {                      // [C rows] x 128 hidden columns, as 2 k-blocks
-        ok = ok && ptx::mbar_wait(&w_empty[ws], wph, abort_flag, g.status);
+        ok = ok && ptx::mbar_wait_relaxed(&w_empty[ws], wph, abort_flag, g.status);
         if (!ok) return;
         ptx::mbar_expect_tx(&w_full[ws], 2 * (uint32_t)g.C * BK * 2);
         for (int kb = 0; kb < 2; ++kb) ptx::tma_load_2d(sW + ws * WST_BYTES + kb * KB_BYTES, &tmW2, &w_full[ws], c * HC + kb * BK, 0);
@@ -284,8 +299,7 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #ifdef MLP_EXP_NOGELU
         pk[i] = float2_to_bf16x2(__uint_as_float(rv[2 * i]) + bb[2 * i], __uint_as_float(rv[2 * i + 1]) + bb[2 * i + 1]);
 #else
-        pk[i] = float2_to_bf16x2(gelu_tanh(__uint_as_float(rv[2 * i]) + bb[2 * i]),
-                                 gelu_tanh(__uint_as_float(rv[2 * i + 1]) + bb[2 * i + 1]));
+        pk[i] = gelu_tanh_bf16x2(__uint_as_float(rv[2 * i]) + bb[2 * i], __uint_as_float(rv[2 * i + 1]) + bb[2 * i + 1]);
 #endif
       }
       ptx::tmem_st16(tq + grp * 16, pk);
@@ -315,7 +329,7 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (g.residual && row_ok) res[v] = *reinterpret_cast<const uint4*>(g.residual + off + v * 8);
       }
       if (q == 0 && lane == 0) DBG(ti * NC * 16 + 12);
-      ok = ptx::mbar_wait(&out_full[ob], (ti >> 1) & 1, abort_flag, g.status);
+      ok = ptx::mbar_wait_relaxed(&out_full[ob], (ti >> 1) & 1, abort_flag, g.status, 256);
       if (!ok) break;
       if (q == 0 && lane == 0) DBG(ti * NC * 16 + 13);
       ptx::tc_fence_after();
@@ -363,6 +377,7 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   }
   ptx::tc_fence_before();
   __syncthreads();
+  DBGT(2);
   if (warp == 1) {
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem_base, TMEM_COLS);
@@ -407,7 +422,7 @@ int launch_mlp_fused(const void* A, const void* W1, const void* b1, const void* 
   }
   profile_tick("mlp_fused", st);
   const unsigned grid = (unsigned)(g.tiles < tc_sm_count() ? g.tiles : tc_sm_count());
-  mlp_fused_kernel<<<grid, kThreads, smem, st>>>(ta, tw1, tw2, g);
+  launch_pdl(mlp_fused_kernel, dim3(grid), dim3(kThreads), smem, st, ta, tw1, tw2, g);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
 }

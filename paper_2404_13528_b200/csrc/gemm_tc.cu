@@ -160,6 +160,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();                       // everything above overlapped the previous kernel's tail
+  pdl_launch_dependents();
 
   if (warp == 0) {
     if (lane == 0) {
@@ -562,7 +564,7 @@ int launch_t(const CUtensorMap& ta, const CUtensorMap& tb, const GemmArgs& g, cu
   profile_tick("gemm_tc", st);
   const long long tiles = (long long)g.tiles_n * g.tiles_m * g.batch;
   const unsigned grid = (unsigned)(tiles < sm_count() ? tiles : sm_count());
-  gemm_tc_kernel<BN, STAGES, A_MN><<<grid, kThreads, smem, st>>>(ta, tb, g);
+  launch_pdl(gemm_tc_kernel<BN, STAGES, A_MN>, dim3(grid), dim3(kThreads), smem, st, ta, tb, g);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
 }

@@ -36,6 +36,8 @@ __global__ void __launch_bounds__(256) norm_kernel(const T* __restrict__ src, T*
   const T* s[RPG];
   bool active[RPG];
   float sum[RPG];
+  pdl_wait();
+  pdl_launch_dependents();
 #pragma unroll
   for (int r = 0; r < RPG; ++r) {
     const long long row = row0 + (long long)r * GPB;
@@ -168,7 +170,7 @@ int launch_norm_t(const void* src, void* dst, const void* gamma, const void* bet
     const int vpl = (nvec + LPR - 1) / LPR;                                                               \
     long long rpb = 8 * (32 / LPR) * RPG;                                                                 \
     unsigned grid = (unsigned)((rows + rpb - 1) / rpb);                                                   \
-    norm_kernel<T, LPR, RMS, RPG, GEN><<<grid, 256, 0, st>>>(s, d, g, b, eps, rows, C, vpl, dm, has);     \
+    launch_pdl(norm_kernel<T, LPR, RMS, RPG, GEN>, dim3(grid), dim3(256), 0, st, s, d, g, b, eps, rows, C, vpl, dm, has);     \
   }
   if (nvec <= 16) SM_LAUNCH(4, 1, false)
   else if (nvec <= 32) SM_LAUNCH(8, 2, false)

@@ -64,6 +64,28 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   }
 }
 
+// Same, for roles that are far off the critical path (a producer with several stages of slack,
+// warps that drain a double-buffered result): sleeping between polls leaves the issue slots of
+// the scheduler they share to the warps that do the arithmetic.
+__device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                                  uint32_t sleep_ns = 128) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = globaltimer();
+  uint32_t polls = 0;
+  while (true) {
+    __nanosleep(sleep_ns);
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((++polls & 15u) == 0) {
+      if (*abort_flag) return false;
+      if (globaltimer() - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        atomicExch(status, (int)SMARTMEM_ERR_TIMEOUT);
+        return false;
+      }
+    }
+  }
+}
+
 // ---- TMA loads (no multicast), completion on an mbarrier --------------------------------
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tm, uint64_t* bar, int c0, int c1) {
   asm volatile(
