@@ -41,6 +41,8 @@ __device__ __forceinline__ void load_tile(__nv_bfloat16* dst, const __nv_bfloat1
 }
 
 __global__ void __launch_bounds__(128) causal_attn_kernel(const __grid_constant__ CausalAttnArgs a) {
+  pdl_wait();
+  pdl_launch_dependents();
   extern __shared__ __align__(16) __nv_bfloat16 sm[];
   __nv_bfloat16* Qs = sm;                       // [64][RS]
   __nv_bfloat16* Ks = sm + TILE_ELEMS;          // [2][64][RS]
@@ -183,6 +185,8 @@ __global__ void __launch_bounds__(128) causal_attn_kernel(const __grid_constant_
 
 // cos/sin table of the rotary embedding: tab[p, i] = (cos, sin)(p * theta^(-2i/D)), i < D/2.
 __global__ void rope_table_kernel(float2* tab, int S, int half, double theta) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= S * half) return;
   const int p = idx / half, i = idx - p * half;
@@ -192,6 +196,8 @@ __global__ void rope_table_kernel(float2* tab, int S, int half, double theta) {
 
 // Stand-alone rotary embedding (explicit variant): rows of [R, D] with position = row % S.
 __global__ void rope_rows_kernel(__nv_bfloat16* x, long long rows, int S, int Dh, const float2* __restrict__ tab) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int half = Dh / 2;
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= rows * half) return;
@@ -228,7 +234,7 @@ int launch_causal_attention(const CausalAttnArgs& a, cudaStream_t st) {
   }
   profile_tick("causal_attention", st);
   dim3 grid((a.S + BMQ - 1) / BMQ, a.heads, a.batch);
-  causal_attn_kernel<<<grid, 128, smem, st>>>(a);
+  launch_pdl(causal_attn_kernel, dim3(grid), dim3(128), smem, st, a);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
 }
@@ -236,7 +242,7 @@ int launch_causal_attention(const CausalAttnArgs& a, cudaStream_t st) {
 int launch_rope_table(float* tab, int S, int head_dim, float theta, cudaStream_t st) {
   const int n = S * (head_dim / 2);
   profile_tick("rope_table", st);
-  rope_table_kernel<<<(n + 255) / 256, 256, 0, st>>>((float2*)tab, S, head_dim / 2, (double)theta);
+  launch_pdl(rope_table_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, st, (float2*)tab, S, head_dim / 2, (double)theta);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
 }
@@ -244,7 +250,7 @@ int launch_rope_table(float* tab, int S, int head_dim, float theta, cudaStream_t
 int launch_rope_rows(void* x, long long rows, int S, int head_dim, const float* tab, cudaStream_t st) {
   const long long n = rows * (head_dim / 2);
   profile_tick("rope_rows", st);
-  rope_rows_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>((__nv_bfloat16*)x, rows, S, head_dim, (const float2*)tab);
+  launch_pdl(rope_rows_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, st, (__nv_bfloat16*)x, rows, S, head_dim, (const float2*)tab);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
 }

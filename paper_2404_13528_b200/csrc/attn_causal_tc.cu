@@ -103,6 +103,8 @@ causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();                       // the set-up above overlapped the previous kernel's tail
+  pdl_launch_dependents();
 
   if (warp == 0) {
     if (lane == 0) {
@@ -336,7 +338,7 @@ int launch_causal_attention_tc(const CausalAttnArgs& a, cudaStream_t st) {
   const long long ctas = (long long)g.n_qt * B * H;
   if (ctas >= (1ll << 31)) return SMARTMEM_ERR_UNSUPPORTED;
   profile_tick("causal_attention_tc", st);
-  causal_attn_tc_kernel<<<(unsigned)ctas, kThreads, smem, st>>>(tq, tk, tv, g);
+  launch_pdl(causal_attn_tc_kernel, dim3((unsigned)ctas), dim3(kThreads), smem, st, tq, tk, tv, g);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
 }

@@ -51,6 +51,8 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 // score element costs one fused multiply-add plus the softmax, and loads overlap the MMAs.
 template <int D>
 __global__ void __launch_bounds__(128) win_attn_bf16_kernel(const __grid_constant__ WinAttnArgs a) {
+  pdl_wait();
+  pdl_launch_dependents();
   constexpr int RS = D + 8;                     // padded row (bf16 elements): conflict-free fragment loads
   constexpr int RW = RS / 2;
   constexpr int TILE = TP * RS;
@@ -274,6 +276,8 @@ __global__ void __launch_bounds__(128) win_attn_bf16_kernel(const __grid_constan
 
 // fp32 variant (plain FMA): one CTA per (window, head); scores live in shared memory.
 __global__ void __launch_bounds__(128) win_attn_f32_kernel(const __grid_constant__ WinAttnArgs a) {
+  pdl_wait();
+  pdl_launch_dependents();
   constexpr int DM = 32;
   __shared__ float Qs[TP * (DM + 1)], Ks[TP * (DM + 1)], Vs[TP * (DM + 1)];
   __shared__ float Ss[TP * (TP + 1)];
@@ -349,7 +353,7 @@ int launch_window_attention(const WinAttnArgs& a, int dtype, long long n_windows
   if (dtype == SMARTMEM_F32) {
     if (a.d > 32) return SMARTMEM_ERR_UNSUPPORTED;
     profile_tick("window_attention_f32", st);
-    win_attn_f32_kernel<<<(unsigned)units, 128, 0, st>>>(a);
+    launch_pdl(win_attn_f32_kernel, dim3((unsigned)units), dim3(128), 0, st, a);
   } else {
     // vector loads need 16-byte aligned rows when the element stride is 1
     const AttnOperand* ops[3] = {&a.q, &a.k, &a.v};
@@ -375,8 +379,8 @@ int launch_window_attention(const WinAttnArgs& a, int dtype, long long n_windows
     if (per_head > n_windows) per_head = n_windows;
     const unsigned grid = (unsigned)(per_head * a.heads);
     profile_tick("window_attention", st);
-    if (a.d == 32) win_attn_bf16_kernel<32><<<grid, 128, 0, st>>>(b);
-    else win_attn_bf16_kernel<16><<<grid, 128, 0, st>>>(b);
+    if (a.d == 32) launch_pdl(win_attn_bf16_kernel<32>, dim3(grid), dim3(128), 0, st, b);
+    else launch_pdl(win_attn_bf16_kernel<16>, dim3(grid), dim3(128), 0, st, b);
   }
   count_launch();
   return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;

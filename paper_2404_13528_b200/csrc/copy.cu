@@ -57,6 +57,8 @@ template <> struct VecT<2> { using type = uint16_t; };
 template <int VB>
 __global__ void __launch_bounds__(256) copy_gather_kernel(const __grid_constant__ DevMap map, const char* __restrict__ src,
                                                           char* __restrict__ dst, uint32_t n_units, int elem_size) {
+  pdl_wait();
+  pdl_launch_dependents();
   using V = typename VecT<VB>::type;
   uint32_t i = blockIdx.x * 256u + threadIdx.x;
   if (i >= n_units) return;
@@ -78,6 +80,8 @@ struct TransposeArgs {
 
 __global__ void __launch_bounds__(256) copy_transpose16_kernel(const __grid_constant__ TransposeArgs a,
                                                                const uint16_t* __restrict__ src, uint16_t* __restrict__ dst) {
+  pdl_wait();
+  pdl_launch_dependents();
   __shared__ uint32_t tile[64][33];          // [j][i-pair]
   uint32_t b = blockIdx.x;
   uint32_t tj = b % a.tiles_j;
@@ -126,6 +130,8 @@ __global__ void __launch_bounds__(256) copy_transpose16_kernel(const __grid_cons
 __global__ void __launch_bounds__(256) copy_block_transpose16_kernel(const __grid_constant__ DevMap outer,
                                                                      const uint16_t* __restrict__ src,
                                                                      uint16_t* __restrict__ dst, int EI, int EJ) {
+  pdl_wait();
+  pdl_launch_dependents();
   extern __shared__ uint16_t blk[];
   const int RS = EJ + 2;
   const int E = EI * EJ;
@@ -160,6 +166,8 @@ __global__ void __launch_bounds__(256) copy_block_transpose16_kernel(const __gri
 template <typename E>
 __global__ void __launch_bounds__(256) copy_seq_kernel(const __grid_constant__ DevSeq q, const E* __restrict__ src,
                                                        E* __restrict__ dst, long long n) {
+  pdl_wait();
+  pdl_launch_dependents();
   const long long i0 = (long long)blockIdx.x * 256 + threadIdx.x;
   if (i0 >= n) return;
   long long idx = i0;
@@ -205,8 +213,8 @@ int launch_copy_seq(const DevSeq& seq, long long n, int elem_size, const void* s
   if (n == 0) return SMARTMEM_OK;
   const long long blocks = (n + 255) / 256;
   if (blocks >= (1ll << 31)) return SMARTMEM_ERR_UNSUPPORTED;
-  if (elem_size == 2) copy_seq_kernel<uint16_t><<<(unsigned)blocks, 256, 0, st>>>(seq, (const uint16_t*)src, (uint16_t*)dst, n);
-  else if (elem_size == 4) copy_seq_kernel<uint32_t><<<(unsigned)blocks, 256, 0, st>>>(seq, (const uint32_t*)src, (uint32_t*)dst, n);
+  if (elem_size == 2) launch_pdl(copy_seq_kernel<uint16_t>, dim3((unsigned)blocks), dim3(256), 0, st, seq, (const uint16_t*)src, (uint16_t*)dst, n);
+  else if (elem_size == 4) launch_pdl(copy_seq_kernel<uint32_t>, dim3((unsigned)blocks), dim3(256), 0, st, seq, (const uint32_t*)src, (uint32_t*)dst, n);
   else return SMARTMEM_ERR_UNSUPPORTED;
   count_launch();
   return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
@@ -227,7 +235,7 @@ int launch_copy_map(const smartmem_index_map_t& map, int elem_size, const void* 
       const int EI = (int)map.extent[n - 1], EJ = (int)map.extent[n - 2];
       const size_t smem = (size_t)EI * (EJ + 2) * 2;
       if (smem <= 40000) {
-      copy_block_transpose16_kernel<<<(unsigned)blocks, 256, smem, st>>>(outer, (const uint16_t*)src, (uint16_t*)dst, EI, EJ);
+      launch_pdl(copy_block_transpose16_kernel, dim3((unsigned)blocks), dim3(256), smem, st, outer, (const uint16_t*)src, (uint16_t*)dst, EI, EJ);
       count_launch();
       return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
       }
@@ -265,7 +273,7 @@ int launch_copy_map(const smartmem_index_map_t& map, int elem_size, const void* 
       t.tiles_j = (int)(map.extent[J] / 64);
       long long blocks = outer * t.tiles_i * t.tiles_j;
       if (ok && blocks < (1ll << 31)) {
-        copy_transpose16_kernel<<<(unsigned)blocks, 256, 0, st>>>(t, (const uint16_t*)src, (uint16_t*)dst);
+        launch_pdl(copy_transpose16_kernel, dim3((unsigned)blocks), dim3(256), 0, st, t, (const uint16_t*)src, (uint16_t*)dst);
         count_launch();
         return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
       }
@@ -279,10 +287,10 @@ int launch_copy_map(const smartmem_index_map_t& map, int elem_size, const void* 
   if (units >= (1ll << 31)) return SMARTMEM_ERR_UNSUPPORTED;
   unsigned grid = (unsigned)((units + 255) / 256);
   switch (vb) {
-    case 16: copy_gather_kernel<16><<<grid, 256, 0, st>>>(d, (const char*)src, (char*)dst, (uint32_t)units, elem_size); break;
-    case 8: copy_gather_kernel<8><<<grid, 256, 0, st>>>(d, (const char*)src, (char*)dst, (uint32_t)units, elem_size); break;
-    case 4: copy_gather_kernel<4><<<grid, 256, 0, st>>>(d, (const char*)src, (char*)dst, (uint32_t)units, elem_size); break;
-    case 2: copy_gather_kernel<2><<<grid, 256, 0, st>>>(d, (const char*)src, (char*)dst, (uint32_t)units, elem_size); break;
+    case 16: launch_pdl(copy_gather_kernel<16>, dim3(grid), dim3(256), 0, st, d, (const char*)src, (char*)dst, (uint32_t)units, elem_size); break;
+    case 8: launch_pdl(copy_gather_kernel<8>, dim3(grid), dim3(256), 0, st, d, (const char*)src, (char*)dst, (uint32_t)units, elem_size); break;
+    case 4: launch_pdl(copy_gather_kernel<4>, dim3(grid), dim3(256), 0, st, d, (const char*)src, (char*)dst, (uint32_t)units, elem_size); break;
+    case 2: launch_pdl(copy_gather_kernel<2>, dim3(grid), dim3(256), 0, st, d, (const char*)src, (char*)dst, (uint32_t)units, elem_size); break;
     default: return SMARTMEM_ERR_UNSUPPORTED;
   }
   count_launch();

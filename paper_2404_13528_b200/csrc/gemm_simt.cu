@@ -8,6 +8,8 @@ namespace smartmem {
 namespace {
 
 __global__ void __launch_bounds__(256) gemm_simt_f32_kernel(const __grid_constant__ SimtGemmArgs g) {
+  pdl_wait();
+  pdl_launch_dependents();
   __shared__ float As[16][17], Ws[16][17];
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
   const int row = blockIdx.y * 16 + ty, col = blockIdx.x * 16 + tx;
@@ -38,7 +40,7 @@ int launch_gemm_simt_f32(const SimtGemmArgs& a, cudaStream_t st) {
   dim3 grid((a.N + 15) / 16, (a.M + 15) / 16);
   if (grid.y > 65535) return SMARTMEM_ERR_UNSUPPORTED;
   profile_tick("gemm_simt_f32", st);
-  gemm_simt_f32_kernel<<<grid, 256, 0, st>>>(a);
+  launch_pdl(gemm_simt_f32_kernel, dim3(grid), dim3(256), 0, st, a);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
 }
