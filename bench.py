@@ -52,6 +52,7 @@ def algorithmic_bytes(w):
         "ln1_gather": 2 * U, "qkv_gemm": U + wq + 3 * U, "window_attention": 3 * U + U,
         "proj_gemm_scatter_residual": U + wp + U + U, "ln2": 2 * U, "fc1_gemm_gelu": U + w1 + r * U,
         "fc2_gemm_residual": r * U + w1 + U + U, "mlp_fused_fc1_gelu_fc2_residual": 3 * U + 2 * w1,
+        "mlp_fused_ln2_fc1_gelu_fc2_residual": 2 * U + 2 * w1,     # x1 in (normalised on chip, also the residual), y out
         # explicit-layout variant: each copy reads and writes its tensor once
         "ln1": 2 * U, "copy_shift": 2 * U, "copy_partition": 2 * U, "copy_head_split": 6 * U, "copy_k_transpose": 2 * U,
         "copy_head_merge": 2 * U, "copy_window_reverse": 2 * U, "copy_unshift": 2 * U, "proj_gemm_residual": 3 * U + wp,

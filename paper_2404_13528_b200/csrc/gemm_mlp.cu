@@ -36,15 +36,17 @@ constexpr int BM = 128, BK = 64, HC = 128;         // tile rows, k-block, hidden
 constexpr int KB_BYTES = BM * BK * 2;              // one 128 x 64 bf16 operand block: 16 KB
 constexpr int NST = 4;                             // weight ring stages; one stage = both k-blocks of a chunk's W1 or W2
 constexpr int WST_BYTES = 2 * KB_BYTES;
-constexpr int kGeluWarps = 16, kOutWarps = 4, kThreads = 32 * (3 + kGeluWarps + kOutWarps);
+constexpr int kGeluWarps = 16, kOutWarps = 4, kNormWarps = 4, kThreads = 32 * (3 + kGeluWarps + kOutWarps + kNormWarps);
 constexpr uint32_t TM_S1 = 0, TM_OUT = 256, OUT_STRIDE = 128, TMEM_COLS = 512;
 constexpr int SMEM_TILES = (4 + 2 * NST) * KB_BYTES;         // A (2 buffers), weight ring
-constexpr int N_BARS = 4 + 2 * NST + 2 + 2 + 2 + 4;
+constexpr int N_BARS = 4 + 2 * NST + 2 + 2 + 2 + 4 + 2;
 
 struct MlpArgs {
   int M, C, hidden, n_chunks, tiles;
   uint32_t smem_bytes;
   const __nv_bfloat16 *b1, *b2, *residual;
+  const __nv_bfloat16 *ln_gamma, *ln_beta;         // LayerNorm applied to the rows of A on their way in (null: A is used as is)
+  float ln_eps;
   __nv_bfloat16* out;
   int* status;
 };
@@ -87,15 +89,17 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   uint64_t* bars = reinterpret_cast<uint64_t*>(sW + NST * WST_BYTES);
   uint64_t *a_full = bars, *a_empty = bars + 2, *w_full = bars + 4, *w_empty = w_full + NST;
   uint64_t *s1_full = w_empty + NST, *s1_empty = s1_full + 2, *h_full = s1_empty + 2;
-  uint64_t *out_full = h_full + 2, *out_empty = out_full + 2;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(out_empty + 2);
+  uint64_t *out_full = h_full + 2, *out_empty = out_full + 2, *a_ready = out_empty + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(a_ready + 2);
   int* abort_flag = reinterpret_cast<int*>(tmem_slot + 1);
   float* b1_s = reinterpret_cast<float*>(tmem_slot + 4);     // [hidden]
   float* b2_s = b1_s + g.hidden;                             // [C]
+  float* ln_s = b2_s + g.C;                                  // [2][C]: gamma, beta
+  const bool fuse_ln = g.ln_gamma != nullptr;
 
   // The tiles fill the 227 KB almost completely, so the launch cannot afford a spare kilobyte of
   // alignment slack: a base that is not 1024-aligned is reported instead of silently overrun.
-  if (pad + SMEM_TILES + N_BARS * 8 + 16 + (g.hidden + g.C) * 4 > g.smem_bytes) {
+  if (pad + SMEM_TILES + N_BARS * 8 + 16 + (g.hidden + 3 * g.C) * 4 > g.smem_bytes) {
     if (threadIdx.x == 0) atomicExch(g.status, (int)SMARTMEM_ERR_UNSUPPORTED);
     return;
   }
@@ -116,6 +120,7 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       ptx::mbar_init(&h_full[i], kGeluWarps);
       ptx::mbar_init(&out_full[i], 1);
       ptx::mbar_init(&out_empty[i], kOutWarps);
+      ptx::mbar_init(&a_ready[i], kNormWarps);
     }
     for (int i = 0; i < NST; ++i) {
       ptx::mbar_init(&w_full[i], 1);
@@ -132,6 +137,11 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   }
   for (int i = threadIdx.x; i < g.hidden; i += kThreads) b1_s[i] = __bfloat162float(g.b1[i]);
   for (int i = threadIdx.x; i < g.C; i += kThreads) b2_s[i] = __bfloat162float(g.b2[i]);
+  if (fuse_ln)
+    for (int i = threadIdx.x; i < g.C; i += kThreads) {
+      ln_s[i] = __bfloat162float(g.ln_gamma[i]);
+      ln_s[g.C + i] = __bfloat162float(g.ln_beta[i]);
+    }
   if (warp == 1) ptx::tmem_alloc(tmem_slot, TMEM_COLS);
   ptx::tc_fence_before();
   __syncthreads();
@@ -197,7 +207,7 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const uint32_t sb = j & 1, ab = it1 & 1;
         const uint32_t n = j ? 2 * j - 1 : 0, ws = n % NST, wph = (n / NST) & 1;
         DBG(j * 16 + 0);
-        if (c1 == 0) ok = ptx::mbar_wait(&a_full[ab], (it1 >> 1) & 1, abort_flag, g.status);
+        if (c1 == 0) ok = ptx::mbar_wait(fuse_ln ? &a_ready[ab] : &a_full[ab], (it1 >> 1) & 1, abort_flag, g.status);
         ok = ok && ptx::mbar_wait(&s1_empty[sb], ((j >> 1) & 1) ^ 1, abort_flag, g.status);
         DBG(j * 16 + 1);
         ok = ok && ptx::mbar_wait(&w_full[ws], wph, abort_flag, g.status);
@@ -265,12 +275,7 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     int c = 0;
     for (int j = 0; j < total && ok; ++j) {
       const uint32_t sb = j & 1;
-      float bb[32];                                      // this warp's 32 biases of the chunk, fetched before the wait
-#pragma unroll
-      for (int v = 0; v < 8; ++v) {
-        const float4 b4 = *reinterpret_cast<const float4*>(b1_s + c * HC + grp * 32 + v * 4);
-        bb[v * 4 + 0] = b4.x; bb[v * 4 + 1] = b4.y; bb[v * 4 + 2] = b4.z; bb[v * 4 + 3] = b4.w;
-      }
+      const float* bb = b1_s + c * HC + grp * 32;        // this warp's 32 biases of the chunk (broadcast reads)
       if (e == 0 && lane == 0) DBG(j * 16 + 8);
       ok = ptx::mbar_wait(&s1_full[sb], (j >> 1) & 1, abort_flag, g.status);
       if (e == 0 && lane == 0) DBG(j * 16 + 9);
@@ -322,12 +327,6 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       const int row = t * BM + q * 32 + lane;
       const bool row_ok = row < g.M;
       const long long off = (long long)row * g.C;
-      uint4 res[4], resn[4];
-#pragma unroll
-      for (int v = 0; v < 4; ++v) {
-        res[v] = make_uint4(0, 0, 0, 0);
-        if (g.residual && row_ok) res[v] = *reinterpret_cast<const uint4*>(g.residual + off + v * 8);
-      }
       if (q == 0 && lane == 0) DBG(ti * NC * 16 + 12);
       ok = ptx::mbar_wait_relaxed(&out_full[ob], (ti >> 1) & 1, abort_flag, g.status, 256);
       if (!ok) break;
@@ -338,11 +337,11 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (r < rounds) {
           uint32_t rv[32];
           ptx::tmem_ld32(tmem_base + TM_OUT + ob * OUT_STRIDE + ((uint32_t)(q * 32) << 16) + r * 32, rv);
+          uint4 res[4];                                  // the residual's latency overlaps the accumulator load
 #pragma unroll
           for (int v = 0; v < 4; ++v) {
-            resn[v] = make_uint4(0, 0, 0, 0);
-            if (g.residual && row_ok && r + 1 < rounds)
-              resn[v] = *reinterpret_cast<const uint4*>(g.residual + off + (r + 1) * 32 + v * 8);
+            res[v] = make_uint4(0, 0, 0, 0);
+            if (g.residual && row_ok) res[v] = *reinterpret_cast<const uint4*>(g.residual + off + r * 32 + v * 8);
           }
           ptx::tmem_ld_wait();
           if (r + 1 == rounds) {                         // the accumulator is in registers: hand the buffer back
@@ -368,11 +367,75 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             pk.w = float2_to_bf16x2(a8[6], a8[7]);
             if (row_ok) *reinterpret_cast<uint4*>(g.out + off + r * 32 + v * 8) = pk;
           }
-#pragma unroll
-          for (int v = 0; v < 4; ++v) res[v] = resn[v];
         }
       }
       if (q == 0 && lane == 0) DBG(ti * NC * 16 + 14);
+    }
+  } else if (warp >= 3 + kGeluWarps + kOutWarps) {
+    // LayerNorm warps: the producer brought the raw rows of the tile into the A buffer (K-major,
+    // 128-byte swizzle); normalise them in place, a thread per row, before fc1 reads them.  Two
+    // passes over the row in registers (mean, then squared deviations), statistics in fp32.
+    if (fuse_ln) {
+      const int nw = warp - (3 + kGeluWarps + kOutWarps);
+      const float invC = 1.0f / (float)g.C;
+      const int nch = g.C / 8;                           // 16-byte chunks per row: 8 or 12
+      bool ok = true;
+      for (int ti = 0; ti < my_tiles && ok; ++ti) {
+        const int b = ti & 1;
+        ok = ptx::mbar_wait_relaxed(&a_full[b], (ti >> 1) & 1, abort_flag, g.status, 64);
+        if (!ok) break;
+        for (int rr = 0; rr < BM / (32 * kNormWarps); ++rr) {
+          const int r = (rr * kNormWarps + nw) * 32 + lane;
+          uint8_t* row0 = sA + (b * 2) * KB_BYTES + r * 128;
+          uint4 x[12];
+#pragma unroll
+          for (int ch = 0; ch < 12; ++ch)
+            if (ch < nch) x[ch] = *reinterpret_cast<const uint4*>(row0 + (ch >> 3) * KB_BYTES + (((ch & 7) ^ (r & 7)) << 4));
+          float s4[4] = {0.f, 0.f, 0.f, 0.f};             // four partial sums: independent dependency chains
+#pragma unroll
+          for (int ch = 0; ch < 12; ++ch)
+            if (ch < nch) {
+              const uint32_t w[4] = {x[ch].x, x[ch].y, x[ch].z, x[ch].w};
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const float2 f = bf16x2_to_float2(w[i]);
+                s4[i] += f.x + f.y;
+              }
+            }
+          const float mean = ((s4[0] + s4[1]) + (s4[2] + s4[3])) * invC;
+          float q4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+          for (int ch = 0; ch < 12; ++ch)
+            if (ch < nch) {
+              const uint32_t w[4] = {x[ch].x, x[ch].y, x[ch].z, x[ch].w};
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const float2 f = bf16x2_to_float2(w[i]);
+                const float dx = f.x - mean, dy = f.y - mean;
+                q4[i] = fmaf(dy, dy, fmaf(dx, dx, q4[i]));
+              }
+            }
+          const float sq = (q4[0] + q4[1]) + (q4[2] + q4[3]);
+          const float rstd = rsqrtf(sq * invC + g.ln_eps);
+#pragma unroll
+          for (int ch = 0; ch < 12; ++ch)
+            if (ch < nch) {
+              const uint32_t w[4] = {x[ch].x, x[ch].y, x[ch].z, x[ch].w};
+              uint32_t o[4];
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const float2 f = bf16x2_to_float2(w[i]);
+                const float2 ga = *reinterpret_cast<const float2*>(ln_s + ch * 8 + 2 * i);
+                const float2 be = *reinterpret_cast<const float2*>(ln_s + g.C + ch * 8 + 2 * i);
+                o[i] = float2_to_bf16x2(fmaf((f.x - mean) * rstd, ga.x, be.x), fmaf((f.y - mean) * rstd, ga.y, be.y));
+              }
+              *reinterpret_cast<uint4*>(row0 + (ch >> 3) * KB_BYTES + (((ch & 7) ^ (r & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+        }
+        ptx::fence_proxy_async();                        // generic-proxy writes -> visible to the MMA's reads
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&a_ready[b]);
+      }
     }
   }
   ptx::tc_fence_before();
@@ -390,10 +453,12 @@ bool mlp_fused_supported(long long C, long long hidden) {
   return (C == 64 || C == 96) && hidden >= HC && hidden % HC == 0 && hidden <= 512;
 }
 
-int launch_mlp_fused(const void* A, const void* W1, const void* b1, const void* W2, const void* b2, const void* residual,
-                     void* out, long long M, long long C, long long hidden, cudaStream_t st) {
+int launch_mlp_fused(const void* A, const void* ln_gamma, const void* ln_beta, float ln_eps, const void* W1, const void* b1,
+                     const void* W2, const void* b2, const void* residual, void* out, long long M, long long C,
+                     long long hidden, cudaStream_t st) {
   if (!mlp_fused_supported(C, hidden) || M < 1 || M >= (1ll << 31) - BM) return SMARTMEM_ERR_UNSUPPORTED;
-  const void* ptrs[] = {A, W1, b1, W2, b2, residual, out};
+  const void* ptrs[] = {A, W1, b1, W2, b2, residual, out, ln_gamma, ln_beta};
+  if ((ln_gamma == nullptr) != (ln_beta == nullptr)) return SMARTMEM_ERR_INVALID_ARG;
   for (const void* p : ptrs)
     if ((uintptr_t)p & 15) return SMARTMEM_ERR_ALIGNMENT;
   if (!b1 || !b2) return SMARTMEM_ERR_INVALID_ARG;
@@ -408,9 +473,10 @@ int launch_mlp_fused(const void* A, const void* W1, const void* b1, const void* 
   g.tiles = (int)((M + BM - 1) / BM);
   g.b1 = (const __nv_bfloat16*)b1; g.b2 = (const __nv_bfloat16*)b2; g.residual = (const __nv_bfloat16*)residual;
   g.out = (__nv_bfloat16*)out;
+  g.ln_gamma = (const __nv_bfloat16*)ln_gamma; g.ln_beta = (const __nv_bfloat16*)ln_beta; g.ln_eps = ln_eps;
   g.status = device_status_ptr();
   if (!g.status) return SMARTMEM_ERR_CUDA;
-  const size_t need = (size_t)SMEM_TILES + N_BARS * 8 + 16 + (size_t)(hidden + C) * 4;
+  const size_t need = (size_t)SMEM_TILES + N_BARS * 8 + 16 + (size_t)(hidden + 3 * C) * 4;
   const size_t smem = need + 1024 <= 232448 ? need + 1024 : 232448;     // alignment slack only while it fits
   if (need > smem) return SMARTMEM_ERR_UNSUPPORTED;
   g.smem_bytes = (uint32_t)smem;

@@ -44,10 +44,13 @@ int tc_encode_2d_sw64(const void* ptr, long long inner, long long outer, long lo
                       int box_outer, CUtensorMap* out);
 int tc_sm_count();
 
-// Fused MLP: out = residual + (GELU(A W1^T + b1)) W2^T + b2 with the hidden activation kept on chip.
-// A [M, C], W1 [hidden, C], W2 [C, hidden], C in {64, 96}, hidden a multiple of 128 (at most 1024).
+// Fused MLP: out = residual + (GELU(LN(A) W1^T + b1)) W2^T + b2 with the hidden activation kept on chip.
+// A [M, C], W1 [hidden, C], W2 [C, hidden], C in {64, 96}, hidden a multiple of 128 (at most 512).
+// ln_gamma/ln_beta [C]: LayerNorm (over C, eps inside the square root) applied to the rows of A as
+// the tile arrives in shared memory; both null: A is used as it is.
 bool mlp_fused_supported(long long C, long long hidden);
-int launch_mlp_fused(const void* A, const void* W1, const void* b1, const void* W2, const void* b2, const void* residual,
-                     void* out, long long M, long long C, long long hidden, cudaStream_t st);
+int launch_mlp_fused(const void* A, const void* ln_gamma, const void* ln_beta, float ln_eps, const void* W1, const void* b1,
+                     const void* W2, const void* b2, const void* residual, void* out, long long M, long long C,
+                     long long hidden, cudaStream_t st);
 
 }  // namespace smartmem

@@ -251,12 +251,13 @@ int run_block(const smartmem_swin_params_t* pp, const void* x, void* y, void* wo
     SM_TRY("proj_gemm_residual", linear(ou, p.w_proj, p.b_proj, y1, C, C, 0, x, nullptr));
   }
   if (p.mlp_ratio > 0) {
-    SM_TRY("ln2", launch_norm(p.dtype, false, y1, at(L.yn), p.ln2_g, p.ln2_b, p.ln_eps, M, (int)C, nullptr, st));
     if (!f32 && mlp_fused_supported(C, hid)) {
-      // narrow blocks: fc1 + GELU + fc2 + residual in one kernel, the hidden activation stays on chip
-      SM_TRY("mlp_fused_fc1_gelu_fc2_residual",
-             launch_mlp_fused(at(L.yn), p.w_fc1, p.b_fc1, p.w_fc2, p.b_fc2, y1, y, M, C, hid, st));
+      // narrow blocks: LN2 + fc1 + GELU + fc2 + residual in one kernel; neither the normalised rows
+      // nor the hidden activation leave the chip
+      SM_TRY("mlp_fused_ln2_fc1_gelu_fc2_residual",
+             launch_mlp_fused(y1, p.ln2_g, p.ln2_b, p.ln_eps, p.w_fc1, p.b_fc1, p.w_fc2, p.b_fc2, y1, y, M, C, hid, st));
     } else {
+      SM_TRY("ln2", launch_norm(p.dtype, false, y1, at(L.yn), p.ln2_g, p.ln2_b, p.ln_eps, M, (int)C, nullptr, st));
       SM_TRY("fc1_gemm_gelu", linear(at(L.yn), p.w_fc1, p.b_fc1, at(L.hid), hid, C, 1, nullptr, nullptr));
       SM_TRY("fc2_gemm_residual", linear(at(L.hid), p.w_fc2, p.b_fc2, y, C, hid, 0, y1, nullptr));
     }
