@@ -21,17 +21,31 @@
 #include "gemm_tc.cuh"
 #include "ptx.cuh"
 
+#ifdef WA_EXP_TIMING
+__device__ long long g_wa_dbg[8192];
+#define WDBG(slot) do { if (blockIdx.x == 0) g_wa_dbg[(slot)] = clock64(); } while (0)
+#define WDBGT(k) do { if (threadIdx.x == 0) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_wa_dbg[6000 + blockIdx.x * 4 + (k)] = (long long)t_; } } while (0)
+extern "C" __attribute__((visibility("default"))) int smartmem_debug_read_wa(long long* host, int n) {
+  return (int)cudaMemcpyFromSymbol(host, g_wa_dbg, sizeof(long long) * n);
+}
+#else
+#define WDBG(slot) do { } while (0)
+#define WDBGT(k) do { } while (0)
+#endif
+
 namespace smartmem {
 namespace {
 
 constexpr int D = 32, TP = 64;
 constexpr int OP_BYTES = 128 * 64;                    // one operand of a pair: 128 rows x 64 bytes
 constexpr int STAGE_BYTES = 3 * OP_BYTES;             // q, k, v
-constexpr int NSTAGE = 3;
+constexpr int NSTAGE = 6;
 constexpr int P_BYTES = 2 * 128 * 128;                // P: 2 k-blocks of [128 rows x 128 bytes] (one per softmax group)
 constexpr uint32_t TM_S = 0, TM_O = 256, TMEM_COLS = 512;
+constexpr int BIAS_ROW = 36;                          // 32-bit words per bias row: 64 bf16 + pad, so that 16-byte row reads of
+                                                      // eight consecutive threads fall into distinct banks
 constexpr int kSoftmaxWarps = 4, kGroups = 2, kLoaderWarps = 4;   // two softmax groups alternate over the units
-constexpr int kThreads = 64 + 32 * (kGroups * kSoftmaxWarps + kLoaderWarps);
+constexpr int kThreads = 32 * (3 + kGroups * kSoftmaxWarps + kLoaderWarps);   // + producer, P V issuer, S issuer
 
 struct WinTcArgs {
   WinAttnArgs a;
@@ -62,12 +76,15 @@ __device__ __forceinline__ float ex2f(float x) {
 __global__ void __launch_bounds__(kThreads, 1)
 win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constant__ CUtensorMap tm1,
                    const __grid_constant__ CUtensorMap tm2, const __grid_constant__ WinTcArgs g) {
+  WDBGT(0);
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
   uint8_t* sIn = smem;                                 // [NSTAGE][q, k, v][128 rows x 64 B]
   uint8_t* sP = sIn + NSTAGE * STAGE_BYTES;            // [kGroups][2 k-blocks][128 x 128 B]
-  float* bias_s = reinterpret_cast<float*>(sP + kGroups * P_BYTES);   // [64][65], log2 domain
-  int* lab_s = reinterpret_cast<int*>(bias_s + TP * 65);         // [kGroups][2][64]
+  uint32_t* bias_s = reinterpret_cast<uint32_t*>(sP + kGroups * P_BYTES);   // [64][36]: bf16 pairs, 144-byte rows
+  int* lab_s = reinterpret_cast<int*>(bias_s + TP * BIAS_ROW);   // scratch: the head's raw table column (<= 256 bf16), then 4 key-mask words
+  uint16_t* raw_s = reinterpret_cast<uint16_t*>(lab_s);
+  uint32_t* kmask_s = reinterpret_cast<uint32_t*>(lab_s) + 128;
   int* tyx_s = lab_s + kGroups * 2 * TP;                         // [64]: ty << 8 | tx
   uint64_t* bars = reinterpret_cast<uint64_t*>(tyx_s + TP);
   uint64_t *in_full = bars, *in_empty = bars + NSTAGE, *s_full = bars + 2 * NSTAGE, *s_empty = s_full + 2;
@@ -102,22 +119,45 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
     ptx::fence_barrier_init();
     ptx::fence_proxy_async();
   }
-  // one-time tables: token coordinates, the head's bias as a [T, T] table, zeroed staging
+  // one-time tables.  First the inputs of the table (one global load per thread, one latency): the
+  // head's column of the relative-position table and the token coordinates; P's off-diagonal blocks
+  // (and, for hand-loaded operands, the padded rows of the input stages) are zeroed meanwhile.
+  const int n_table = (2 * ws - 1) * (2 * ws - 1);
+  for (int i = tid; i < n_table && i < 256; i += kThreads) raw_s[i] = reinterpret_cast<const uint16_t*>(a.table)[i * a.heads + h];
   if (tid < TP) tyx_s[tid] = ((tid / ws) << 8) | (tid % ws);
-  for (int i = tid; i < TP * TP; i += kThreads) {
-    const int r = i / TP, c = i - r * TP;
-    float v = 0.f;
-    if (c >= T) {
-      v = -INFINITY;                                   // padded keys never contribute
-    } else if (r < T) {
-      const int idx = (r / ws - c / ws + ws - 1) * (2 * ws - 1) + (r % ws - c % ws + ws - 1);
-      v = LOG2E * (a.table_f32 ? ((const float*)a.table)[idx * a.heads + h]
-                               : __bfloat162float(((const __nv_bfloat16*)a.table)[idx * a.heads + h]));
-    }
-    bias_s[r * 65 + c] = v;
+  {
+    uint8_t* z0 = any_manual ? smem : sP;
+    const int zbytes = (any_manual ? NSTAGE * STAGE_BYTES : 0) + kGroups * P_BYTES;
+    for (int i = tid; i < zbytes / 16; i += kThreads) reinterpret_cast<uint4*>(z0)[i] = make_uint4(0, 0, 0, 0);
   }
-  for (int i = tid; i < (NSTAGE * STAGE_BYTES + kGroups * P_BYTES) / 16; i += kThreads)
-    reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
+  __syncthreads();
+  // the head's bias as a [T, T] table of bf16 pairs, -inf for padded keys
+  for (int i = tid; i < TP * (TP / 2); i += kThreads) {
+    const int r = i / (TP / 2), c2 = i - r * (TP / 2);
+    const int ry = tyx_s[r] >> 8, rx = tyx_s[r] & 255;
+    uint32_t word = 0;
+    for (int k = 0; k < 2; ++k) {
+      const int c = 2 * c2 + k;
+      uint32_t bits = 0;                               // bf16 bit pattern
+      if (c >= T) {
+        bits = 0xFF80u;                                // -inf: padded keys never contribute
+      } else if (r < T) {
+        const int cy = tyx_s[c] >> 8, cx = tyx_s[c] & 255;
+        bits = raw_s[(ry - cy + ws - 1) * (2 * ws - 1) + (rx - cx + ws - 1)];
+      }
+      word |= bits << (16 * k);
+    }
+    bias_s[r * BIAS_ROW + c2] = word;
+  }
+  // keys below / right of the wrap line of a seam window (bit c = key c)
+  if (warp == 2) {
+    const int c0 = lane, c1 = lane + 32;
+    const bool y0 = c0 < T && (tyx_s[c0] >> 8) >= ws - a.shift, y1 = c1 < T && (tyx_s[c1] >> 8) >= ws - a.shift;
+    const bool x0 = c0 < T && (tyx_s[c0] & 255) >= ws - a.shift, x1 = c1 < T && (tyx_s[c1] & 255) >= ws - a.shift;
+    const uint32_t m0 = __ballot_sync(0xFFFFFFFFu, y0), m1 = __ballot_sync(0xFFFFFFFFu, y1);
+    const uint32_t m2 = __ballot_sync(0xFFFFFFFFu, x0), m3 = __ballot_sync(0xFFFFFFFFu, x1);
+    if (lane == 0) { kmask_s[0] = m0; kmask_s[1] = m1; kmask_s[2] = m2; kmask_s[3] = m3; }
+  }
   if (warp == 0 && lane == 0) {
     ptx::prefetch_tensormap(&tm0);
     ptx::prefetch_tensormap(&tm1);
@@ -129,7 +169,9 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  WDBGT(1);
   pdl_wait();                       // the tables above depend on parameters only: they overlapped the previous kernel's tail
+  WDBGT(2);
   pdl_launch_dependents();
   const CUtensorMap* tms[3] = {&tm0, &tm1, &tm2};
   const AttnOperand* ops[3] = {&a.q, &a.k, &a.v};
@@ -146,6 +188,9 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
         ok = ptx::mbar_wait(&in_empty[s], ((it / NSTAGE) & 1) ^ 1, abort_flag, g.status);
         if (!ok) break;
         const int nwin = (2 * p + 1 < a.n_windows) ? 2 : 1;
+#ifdef WA_EXP_NOLOAD
+        if (it >= NSTAGE) { ptx::mbar_arrive(&in_full[s]); continue; }
+#endif
         ptx::mbar_expect_tx(&in_full[s], (uint32_t)(n_tma * nwin * TP * 64));
         for (int m = 0; m < 3; ++m) {
           if (!((g.tma_mask >> m) & 1)) continue;
@@ -158,42 +203,52 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
       }
     }
   } else if (warp == 1) {
-    // ---- MMA issuer --------------------------------------------------------------------------
+    // ---- P V issuer (and owner of the tensor memory) -----------------------------------------
     if (lane == 0) {
-      const uint32_t idesc_s = ptx::make_idesc_bf16(128, 128, false, false);
       const uint32_t idesc_pv = ptx::make_idesc_bf16(128, D, false, true);     // V: MN-major B operand
       bool ok = true;
       const int my_units = cidx < g.n_pairs ? (g.n_pairs - cidx + cstride - 1) / cstride : 0;
-      auto issue_s = [&](int u) {
-        const int s = u % NSTAGE, sb = u & 1;
-        ok = ok && ptx::mbar_wait(&s_empty[sb], ((u >> 1) & 1) ^ 1, abort_flag, g.status);
-        ok = ok && ptx::mbar_wait(&in_full[s], (u / NSTAGE) & 1, abort_flag, g.status);
-        if (!ok) return;
-        ptx::tc_fence_after();
-        const uint32_t q0 = ptx::smem_u32(sIn + s * STAGE_BYTES), k0 = q0 + OP_BYTES;
-        for (int k = 0; k < D / 16; ++k)
-          ptx::tc_mma_bf16(tmem_base + TM_S + sb * 128, make_desc_sw64(q0 + k * 32, 16, 512),
-                           make_desc_sw64(k0 + k * 32, 16, 512), idesc_s, k ? 1u : 0u);
-        ptx::tc_commit(&s_full[sb]);
-      };
-      auto issue_pv = [&](int u) {
+      for (int u = 0; u < my_units && ok; ++u) {
         const int s = u % NSTAGE, ob = u & 1;
-        ok = ok && ptx::mbar_wait(&p_full[ob], (u >> 1) & 1, abort_flag, g.status);
+        WDBG(u * 16 + 2);
+        ok = ptx::mbar_wait(&p_full[ob], (u >> 1) & 1, abort_flag, g.status);
         ok = ok && ptx::mbar_wait(&o_empty[ob], ((u >> 1) & 1) ^ 1, abort_flag, g.status);
-        if (!ok) return;
+        if (!ok) break;
+        WDBG(u * 16 + 3);
         ptx::tc_fence_after();
         const uint32_t p0 = ptx::smem_u32(sP + ob * P_BYTES), v0 = ptx::smem_u32(sIn + s * STAGE_BYTES + 2 * OP_BYTES);
-        for (int ks = 0; ks < 8; ++ks)                 // 16 keys per step
-          ptx::tc_mma_bf16(tmem_base + TM_O + ob * D, ptx::make_smem_desc(p0 + (ks >> 2) * (128 * 128) + (ks & 3) * 32, 16, 1024),
-                           make_desc_sw64(v0 + ks * 1024, 16, 512), idesc_pv, ks ? 1u : 0u);
+        const uint64_t pd = ptx::make_smem_desc(p0, 16, 1024), vd = make_desc_sw64(v0, 16, 512);
+        const uint32_t od = tmem_base + TM_O + ob * D;
+        ptx::tc_mma_bf16(od, pd, vd, idesc_pv, 0u);
+#pragma unroll
+        for (int ks = 1; ks < 8; ++ks)                 // 16 keys per step: P +32 bytes (next k-block: +16 KB), V +1024 bytes
+          ptx::tc_mma_bf16(od, pd + (ks >> 2) * ((128 * 128) >> 4) + (ks & 3) * 2, vd + ks * (1024 >> 4), idesc_pv, 1u);
         ptx::tc_commit(&in_empty[s]);
         ptx::tc_commit(&p_empty[ob]);
         ptx::tc_commit(&o_full[ob]);
-      };
-      if (my_units > 0) issue_s(0);
+        WDBG(u * 16 + 4);
+      }
+    }
+  } else if (warp == 2 + kGroups * kSoftmaxWarps + kLoaderWarps) {
+    // ---- S issuer: runs ahead of P V as far as the two S buffers and the input ring allow, so a
+    // softmax group finds its next score tile waiting when it has written P ---------------------
+    if (lane == 0) {
+      const uint32_t idesc_s = ptx::make_idesc_bf16(128, 128, false, false);
+      bool ok = true;
+      const int my_units = cidx < g.n_pairs ? (g.n_pairs - cidx + cstride - 1) / cstride : 0;
       for (int u = 0; u < my_units && ok; ++u) {
-        if (u + 1 < my_units) issue_s(u + 1);
-        issue_pv(u);
+        const int s = u % NSTAGE, sb = u & 1;
+        WDBG(u * 16 + 0);
+        ok = ptx::mbar_wait(&s_empty[sb], ((u >> 1) & 1) ^ 1, abort_flag, g.status);
+        ok = ok && ptx::mbar_wait(&in_full[s], (u / NSTAGE) & 1, abort_flag, g.status);
+        if (!ok) break;
+        ptx::tc_fence_after();
+        const uint32_t q0 = ptx::smem_u32(sIn + s * STAGE_BYTES), k0 = q0 + OP_BYTES;
+        const uint64_t qd = make_desc_sw64(q0, 16, 512), kd = make_desc_sw64(k0, 16, 512);
+        ptx::tc_mma_bf16(tmem_base + TM_S + sb * 128, qd, kd, idesc_s, 0u);
+        ptx::tc_mma_bf16(tmem_base + TM_S + sb * 128, qd + 2, kd + 2, idesc_s, 1u);    // next 16 features: +32 bytes
+        ptx::tc_commit(&s_full[sb]);
+        WDBG(u * 16 + 1);
       }
     }
   } else if (warp < 2 + kGroups * kSoftmaxWarps) {
@@ -203,9 +258,11 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
     const int r = q * 32 + lane;                       // row of the pair tile
     const int w = r >> 6, i = r & 63;                  // window of the pair, token
     const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
-    const float scale2 = a.scale * LOG2E;
     const int my_ty = tyx_s[i] >> 8, my_tx = tyx_s[i] & 255;
-    const float* brow = bias_s + i * 65;
+    const uint32_t* brow = bias_s + i * BIAS_ROW;
+    // keys below / right of the wrap line of a seam window (bit c = key c), and this row's own side
+    const uint32_t ky_lo = kmask_s[0], ky_hi = kmask_s[1], kx_lo = kmask_s[2], kx_hi = kmask_s[3];
+    const uint32_t my_fy = my_ty >= ws - a.shift ? 0xFFFFFFFFu : 0u, my_fx = my_tx >= ws - a.shift ? 0xFFFFFFFFu : 0u;
     float inv_prev = 0.f;
     int n_prev = -1;
     bool ok = true;
@@ -213,6 +270,7 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
       const int ob = u & 1;                            // == gi
       ok = ok && ptx::mbar_wait(&o_full[ob], (u >> 1) & 1, abort_flag, g.status);
       if (!ok) return;
+      if (q == 0 && lane == 0) WDBG(u * 16 + 10);
       ptx::tc_fence_after();
       uint32_t rv[32];
       ptx::tmem_ld32(tmem_base + TM_O + ob * D + lane_addr, rv);
@@ -227,59 +285,95 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
           float o8[8];
 #pragma unroll
           for (int e = 0; e < 8; ++e) o8[e] = __uint_as_float(rv[v * 8 + e]) * inv;
+#ifndef WA_EXP_NOSTORE
           ElemIO<__nv_bfloat16>::store(dst + v * 8, o8);
+#else
+          if (o8[0] == 123.456f) ElemIO<__nv_bfloat16>::store(dst + v * 8, o8);
+#endif
         }
       }
+      if (q == 0 && lane == 0) WDBG(u * 16 + 11);
     };
     int u = gi;
     int done = 0;
     for (int p = cidx + gi * cstride; p < g.n_pairs && ok; p += 2 * cstride, u += 2, ++done) {
       const int sb = u & 1;
       const int n = 2 * p + w;
-      // region labels of this window (only windows on the seam of a shifted block are masked)
+      // Shifted blocks: only windows in the last window row or column straddle the seam.  There a key
+      // lies in another region than this row iff the two sit on different sides of the wrap line at
+      // ws - shift, vertically (last window row) or horizontally (last window column): one 64-bit
+      // mask per row, from the two key masks computed once above.
       bool masked = false;
-      int my_lab = 0;
+      uint32_t diff_lo = 0, diff_hi = 0;
       if (a.shift > 0 && n < a.n_windows) {
         const int wl = n - (int)fd_div((uint32_t)n, a.fd_wpi) * a.win_per_img;
         const int wy = (int)fd_div((uint32_t)wl, a.fd_nww), wx = wl - wy * a.nWw;
-        masked = (wy == a.nWh - 1) || (wx == a.nWw - 1);
-        if (masked) my_lab = region_label2(my_ty, my_tx, ws, wy, wx, a.H, a.W, a.shift);
+        const bool last_row = wy == a.nWh - 1, last_col = wx == a.nWw - 1;
+        masked = last_row || last_col;
+        if (last_row) { diff_lo |= ky_lo ^ my_fy; diff_hi |= ky_hi ^ my_fy; }
+        if (last_col) { diff_lo |= kx_lo ^ my_fx; diff_hi |= kx_hi ^ my_fx; }
       }
-      if (masked) {                                    // uniform over the 64 threads of the window
-        lab_s[(gi * 2 + w) * TP + i] = my_lab;
-        asm volatile("bar.sync %0, 64;" ::"r"(1 + gi * 2 + w) : "memory");
-      }
+      if (q == 0 && lane == 0) WDBG(u * 16 + 5);
       ok = ptx::mbar_wait(&s_full[sb], (u >> 1) & 1, abort_flag, g.status);
       if (!ok) break;
+      if (q == 0 && lane == 0) WDBG(u * 16 + 6);
       ptx::tc_fence_after();
       uint32_t rv[64];
       const uint32_t ts = tmem_base + TM_S + sb * 128 + lane_addr + w * 64;    // this window's 64 key columns
       ptx::tmem_ld32(ts, rv);
       ptx::tmem_ld32(ts + 32, rv + 32);
       ptx::tmem_ld_wait();
+      if (q == 0 && lane == 0) WDBG(u * 16 + 7);
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&s_empty[sb]);
       float sc[64];
-      float mx = -INFINITY;
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // independent chains
+#ifdef WA_EXP_TIMING
+      if (q == 0 && lane == 0 && __uint_as_float(rv[63]) != 123.456f) WDBG(u * 16 + 13);
+#endif
+      // scores in natural units: q.k * scale + bias (the row's 64 biases come as eight 16-byte reads
+      // of bf16 pairs); the base-2 conversion is folded into the exponent's multiply-add below
 #pragma unroll
-      for (int c = 0; c < 64; ++c) {
-        float v = fmaf(__uint_as_float(rv[c]), scale2, brow[c]);
-        if (masked && c < T && lab_s[(gi * 2 + w) * TP + c] != my_lab) v -= 100.f * LOG2E;
-        sc[c] = v;
-        mx = fmaxf(mx, v);
+      for (int v8 = 0; v8 < 8; ++v8) {
+        const uint4 b4 = *reinterpret_cast<const uint4*>(brow + v8 * 4);
+        const uint32_t bw[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int c = v8 * 8 + 2 * j;
+          sc[c] = fmaf(__uint_as_float(rv[c]), a.scale, __uint_as_float(bw[j] << 16));
+          sc[c + 1] = fmaf(__uint_as_float(rv[c + 1]), a.scale, __uint_as_float(bw[j] & 0xFFFF0000u));
+        }
       }
-      if (masked) asm volatile("bar.sync %0, 64;" ::"r"(1 + gi * 2 + w) : "memory");   // labels may be overwritten next unit
-      float sum0 = 0.f, sum1 = 0.f;
+      if (masked) {                                    // seam windows only: keys of another region get -100
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+          if ((diff_lo >> c) & 1u) sc[c] -= 100.f;
+          if ((diff_hi >> c) & 1u) sc[c + 32] -= 100.f;
+        }
+      }
+#pragma unroll
+      for (int c = 0; c < 64; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], sc[c]);
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+      const float nmx = -mx * LOG2E;
+#ifdef WA_EXP_TIMING
+      if (q == 0 && lane == 0 && mx > -1e30f) WDBG(u * 16 + 12);
+#endif
+      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
       uint32_t pk[32];
 #pragma unroll
       for (int c = 0; c < 64; c += 2) {
-        const float p0 = ex2f(sc[c] - mx), p1 = ex2f(sc[c + 1] - mx);
-        sum0 += p0;
-        sum1 += p1;
+        const float p0 = ex2f(fmaf(sc[c], LOG2E, nmx)), p1 = ex2f(fmaf(sc[c + 1], LOG2E, nmx));
+        sum4[c & 2] += p0;
+        sum4[(c & 2) + 1] += p1;
         pk[c / 2] = float2_to_bf16x2(p0, p1);
       }
-      const float inv = 1.f / (sum0 + sum1);
+      const float inv = 1.f / ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
+      if (q == 0 && lane == 0) WDBG(u * 16 + 8);
+      // drain this group's previous unit: its P V has finished by now, and the O buffer it frees is
+      // the one this unit's P V accumulates into
+      if (done > 0) epilogue(u - 2, inv_prev, n_prev);
+      if (!ok) break;
       // previous P V must have completed before P is overwritten
       ok = ptx::mbar_wait(&p_empty[gi], ((u >> 1) & 1) ^ 1, abort_flag, g.status);
       if (!ok) break;
@@ -293,13 +387,12 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&p_full[gi]);
-      // this group's previous unit is drained while this unit's P V runs
-      if (done > 0) epilogue(u - 2, inv_prev, n_prev);
+      if (q == 0 && lane == 0) WDBG(u * 16 + 9);
       inv_prev = inv;
       n_prev = n;
     }
     if (ok && done > 0) epilogue(u - 2, inv_prev, n_prev);
-  } else {
+  } else if (warp < 2 + kGroups * kSoftmaxWarps + kLoaderWarps) {
     // ---- helper loaders for operands TMA cannot address (e.g. a materialised K^T) ----------------
     if (any_manual) {
       const int lt = tid - 32 * (2 + kGroups * kSoftmaxWarps);
@@ -363,6 +456,7 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
   }
   ptx::tc_fence_before();
   __syncthreads();
+  WDBGT(3);
   if (warp == 1) {
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem_base, TMEM_COLS);
@@ -374,6 +468,7 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
 // Returns SMARTMEM_ERR_UNSUPPORTED for shapes the kernel does not cover (the caller then uses the
 // warp-MMA kernel).
 int launch_window_attention_tc(const WinAttnArgs& a_in, long long n_windows, cudaStream_t st) {
+  if (a_in.table_f32) return SMARTMEM_ERR_UNSUPPORTED;     // the bias table is kept as bf16 pairs
   if (a_in.d != D || a_in.T > TP || a_in.T < 1 || n_windows < 1 || n_windows >= (1ll << 30)) return SMARTMEM_ERR_UNSUPPORTED;
   if (a_in.o.se != 1 || a_in.o.st % 8 || a_in.o.sn % 8 || a_in.o.sh % 8 || ((uintptr_t)a_in.o.ptr & 15)) return SMARTMEM_ERR_UNSUPPORTED;
   WinTcArgs g;
@@ -406,7 +501,7 @@ int launch_window_attention_tc(const WinAttnArgs& a_in, long long n_windows, cud
       g.tma_mask |= 1 << m;
     }
   }
-  const size_t smem = 1024 + NSTAGE * STAGE_BYTES + kGroups * P_BYTES + TP * 65 * 4 + (2 * kGroups + 1) * TP * 4 +
+  const size_t smem = 1024 + NSTAGE * STAGE_BYTES + kGroups * P_BYTES + TP * BIAS_ROW * 4 + (2 * kGroups + 1) * TP * 4 +
                       (2 * NSTAGE + 12) * 8 + 16;
   static bool configured = false;
   if (!configured) {

@@ -645,7 +645,9 @@ int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep,
   else if (N % 64 == 0) bn = 64;
   if (ep.rope_cols > 0 && (N % 256 || ep.rope_cols % 256 || ep.rope_S < 1)) return SMARTMEM_ERR_UNSUPPORTED;
   const int nkb = (int)((K + BK - 1) / BK);
-  const int stages = (bn == 256 && nkb <= 3) ? 3 : 4;   // short K: wider store rounds instead of a 4th stage
+  // 256 wide, short K: wider store rounds instead of a 4th stage.  Narrow tiles: their stages are
+  // small, and a tile is consumed faster than a load's latency, so the ring runs several tiles ahead.
+  const int stages = bn == 256 ? (nkb <= 3 ? 3 : 4) : (bn <= 96 ? 6 : 4);
   GemmArgs g;
   memset(&g, 0, sizeof(g));
   CUtensorMap ta, tb;
@@ -673,7 +675,7 @@ int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep,
   if ((long long)g.tiles_n * g.tiles_m * g.batch >= (1ll << 31)) return SMARTMEM_ERR_UNSUPPORTED;
 #define SM_CASE(BN_, ST_, MN_)                                                                  \
   if (bn == BN_ && stages == ST_ && a_mn == MN_) return launch_t<BN_, ST_, MN_>(ta, tb, g, st);
-  SM_CASE(256, 3, false) SM_CASE(256, 4, false) SM_CASE(128, 4, false) SM_CASE(96, 4, false) SM_CASE(64, 4, false)
+  SM_CASE(256, 3, false) SM_CASE(256, 4, false) SM_CASE(128, 4, false) SM_CASE(96, 6, false) SM_CASE(64, 6, false)
   SM_CASE(256, 3, true) SM_CASE(256, 4, true) SM_CASE(128, 4, true)
 #undef SM_CASE
   return SMARTMEM_ERR_UNSUPPORTED;
