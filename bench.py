@@ -49,7 +49,7 @@ def algorithmic_bytes(w):
     C, r = w["C"], w["mlp_ratio"]
     wq, wp, w1 = 3 * C * C * 2, C * C * 2, r * C * C * 2
     return {
-        "ln1_gather": 2 * U, "qkv_gemm": U + wq + 3 * U, "window_attention": 3 * U + U,
+        "ln1_gather": 2 * U, "qkv_gemm": U + wq + 3 * U, "ln1_gather_qkv_gemm": U + wq + 3 * U, "ln1_qkv_gemm": U + wq + 3 * U, "window_attention": 3 * U + U,
         "proj_gemm_scatter_residual": U + wp + U + U, "ln2": 2 * U, "fc1_gemm_gelu": U + w1 + r * U,
         "fc2_gemm_residual": r * U + w1 + U + U, "mlp_fused_fc1_gelu_fc2_residual": 3 * U + 2 * w1,
         "mlp_fused_ln2_fc1_gelu_fc2_residual": 2 * U + 2 * w1,     # x1 in (normalised on chip, also the residual), y out

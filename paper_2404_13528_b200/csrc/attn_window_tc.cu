@@ -119,6 +119,7 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
     ptx::fence_barrier_init();
     ptx::fence_proxy_async();
   }
+  if (warp == 1) ptx::tmem_alloc(tmem_slot, TMEM_COLS);   // first: its latency overlaps the table set-up below
   // one-time tables.  First the inputs of the table (one global load per thread, one latency): the
   // head's column of the relative-position table and the token coordinates; P's off-diagonal blocks
   // (and, for hand-loaded operands, the padded rows of the input stages) are zeroed meanwhile.
@@ -163,7 +164,6 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
     ptx::prefetch_tensormap(&tm1);
     ptx::prefetch_tensormap(&tm2);
   }
-  if (warp == 1) ptx::tmem_alloc(tmem_slot, TMEM_COLS);
   ptx::fence_proxy_async();
   ptx::tc_fence_before();
   __syncthreads();

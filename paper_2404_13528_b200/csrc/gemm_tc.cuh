@@ -53,4 +53,11 @@ int launch_mlp_fused(const void* A, const void* ln_gamma, const void* ln_beta, f
                      const void* W2, const void* b2, const void* residual, void* out, long long M, long long C,
                      long long hidden, cudaStream_t st);
 
+// LayerNorm o row-gather o linear for narrow rows: out[m, :] = LN(X[src(m), :]) W^T + bias, with X rows of
+// K in {64, 96} elements, W [N, K], N a multiple of 96 (at most 288).  `rowmap` (null: identity) gives
+// the element offset of consumer row m in X; gamma/beta null: no normalisation (plain gather).
+bool gemm_ln_supported(long long N, long long K);
+int launch_gemm_ln(const void* X, const DevMap* rowmap, const void* gamma, const void* beta, float eps, const void* W,
+                   const void* bias, void* out, long long M, long long N, long long K, cudaStream_t st);
+
 }  // namespace smartmem

@@ -213,10 +213,16 @@ int run_block(const smartmem_swin_params_t* pp, const void* x, void* y, void* wo
   a.nWw = p.W / p.window; a.win_per_img = (p.H / p.window) * (p.W / p.window);
   a.scale = 1.0f / sqrtf((float)d);
 
+  const bool fuse_ln1 = !f32 && gemm_ln_supported(3 * C, C);
 #define SM_TRY(label, expr) do { if (tm) tm->tick(label); rc = (expr); if (rc != SMARTMEM_OK) return rc; } while (0)
   if (elim) {
-    SM_TRY("ln1_gather", launch_norm(p.dtype, false, x, at(L.xn), p.ln1_g, p.ln1_b, p.ln_eps, M, (int)C, &m.e1_rows, st));
-    SM_TRY("qkv_gemm", linear(at(L.xn), p.w_qkv, p.b_qkv, at(L.qkv), 3 * C, C, 0, nullptr, nullptr));
+    if (fuse_ln1) {
+      // narrow blocks: LN1, the shift o partition gather and the QKV projection in one kernel
+      SM_TRY("ln1_gather_qkv_gemm", launch_gemm_ln(x, &m.e1_rows, p.ln1_g, p.ln1_b, p.ln_eps, p.w_qkv, p.b_qkv, at(L.qkv), M, 3 * C, C, st));
+    } else {
+      SM_TRY("ln1_gather", launch_norm(p.dtype, false, x, at(L.xn), p.ln1_g, p.ln1_b, p.ln_eps, M, (int)C, &m.e1_rows, st));
+      SM_TRY("qkv_gemm", linear(at(L.xn), p.w_qkv, p.b_qkv, at(L.qkv), 3 * C, C, 0, nullptr, nullptr));
+    }
     char* qkv = (char*)at(L.qkv);
     a.q = {qkv, T * 3 * C, d, 3 * C, 1};
     a.k = {qkv + C * esz, T * 3 * C, d, 3 * C, 1};
@@ -225,14 +231,24 @@ int run_block(const smartmem_swin_params_t* pp, const void* x, void* y, void* wo
     SM_TRY("window_attention", launch_window_attention(a, p.dtype, nW, st));
     SM_TRY("proj_gemm_scatter_residual", linear(at(L.ao), p.w_proj, p.b_proj, y1, C, C, 0, x, &m.e1_rows));
   } else {
-    SM_TRY("ln1", launch_norm(p.dtype, false, x, at(L.xn), p.ln1_g, p.ln1_b, p.ln_eps, M, (int)C, nullptr, st));
-    void* xs = at(L.xn);
+    // Same kernels as above, but every layout operator is a copy.  Where LN1 is fused into the QKV
+    // kernel the copies move the raw rows and the fused kernel normalises what arrives (LayerNorm is
+    // per token, so it commutes with the two token permutations); otherwise LN1 runs first.
+    const void* xs = x;
+    if (!fuse_ln1) {
+      SM_TRY("ln1", launch_norm(p.dtype, false, x, at(L.xn), p.ln1_g, p.ln1_b, p.ln_eps, M, (int)C, nullptr, st));
+      xs = at(L.xn);
+    }
     if (p.shift > 0) {
-      SM_TRY("copy_shift", launch_copy_map(m.shift, esz, at(L.xn), at(L.xs), st));
+      SM_TRY("copy_shift", launch_copy_map(m.shift, esz, xs, at(L.xs), st));
       xs = at(L.xs);
     }
     SM_TRY("copy_partition", launch_copy_map(m.part, esz, xs, at(L.xw), st));
-    SM_TRY("qkv_gemm", linear(at(L.xw), p.w_qkv, p.b_qkv, at(L.qkv), 3 * C, C, 0, nullptr, nullptr));
+    if (fuse_ln1) {
+      SM_TRY("ln1_qkv_gemm", launch_gemm_ln(at(L.xw), nullptr, p.ln1_g, p.ln1_b, p.ln_eps, p.w_qkv, p.b_qkv, at(L.qkv), M, 3 * C, C, st));
+    } else {
+      SM_TRY("qkv_gemm", linear(at(L.xw), p.w_qkv, p.b_qkv, at(L.qkv), 3 * C, C, 0, nullptr, nullptr));
+    }
     SM_TRY("copy_head_split", launch_copy_map(m.split, esz, at(L.qkv), at(L.split), st));
     char* sp = (char*)at(L.split);
     SM_TRY("copy_k_transpose", launch_copy_map(m.kt, esz, sp + (size_t)M * C * esz, at(L.kt), st));
