@@ -131,6 +131,54 @@ __device__ __forceinline__ long long devmap_eval(const DevMap& m, uint32_t i) {
   return off;
 }
 
+// Same result, with the atom loop fully unrolled: every map constant then is a fixed kernel-parameter
+// operand of the arithmetic instead of an indexed constant load, and the digits of different atoms
+// overlap (only the quotient chain is sequential).  For callers where one thread evaluates the map per
+// row on a critical path; costs code size, so the copy kernels keep the rolled loop.
+__device__ __forceinline__ long long devmap_eval_unrolled(const DevMap& m, uint32_t i) {
+  long long off = m.base;
+  int u0 = 0, u1 = 0, u2 = 0, u3 = 0;
+#pragma unroll
+  for (int a = kMaxDevAtoms - 1; a >= 0; --a) {
+    if (a < m.n_atoms) {
+      const uint32_t q = fd_div(i, m.ext[a]);
+      const int digit = (int)(i - q * m.ext[a].d);
+      i = q;
+      const int r = m.roll_of[a];
+      if (r < 0) {
+        off += (long long)digit * m.stride[a];
+      } else {
+        const int w = digit * m.weight[a];
+        u0 += r == 0 ? w : 0;
+        u1 += r == 1 ? w : 0;
+        u2 += r == 2 ? w : 0;
+        u3 += r == 3 ? w : 0;
+      }
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < SMARTMEM_MAX_ROLLS; ++r) {
+    if (r < m.n_rolls) {
+      int v = (r == 0 ? u0 : r == 1 ? u1 : r == 2 ? u2 : u3) + m.roll_shift[r];
+      if (v >= m.roll_mod[r]) v -= m.roll_mod[r];
+      if (m.roll_n_parts[r] <= 1) {
+        off += (long long)v * m.roll_stride[r];
+      } else {
+        uint32_t vv = (uint32_t)v;
+#pragma unroll
+        for (int k = SMARTMEM_MAX_ROLLS - 1; k >= 0; --k) {
+          if (k < m.roll_n_parts[r]) {
+            const uint32_t q = fd_div(vv, m.roll_part_ext[r][k]);
+            off += (long long)(vv - q * m.roll_part_ext[r][k].d) * m.roll_part_stride[r][k];
+            vv = q;
+          }
+        }
+      }
+    }
+  }
+  return off;
+}
+
 // Host: builds a DevMap over atoms [a0, a1) of a public map, treating `unit` elements of the
 // innermost selected atom as one unit (unit must divide its extent; its stride must be 1 when
 // unit > 1).  `with_base` adds the map's base.  Returns false if it does not fit.

@@ -62,7 +62,7 @@ __global__ void __launch_bounds__(256) copy_gather_kernel(const __grid_constant_
   using V = typename VecT<VB>::type;
   uint32_t i = blockIdx.x * 256u + threadIdx.x;
   if (i >= n_units) return;
-  long long off = devmap_eval(map, i);
+  long long off = devmap_eval_unrolled(map, i);
   V v = *reinterpret_cast<const V*>(src + off * elem_size);
   *reinterpret_cast<V*>(dst + (size_t)i * VB) = v;
 }

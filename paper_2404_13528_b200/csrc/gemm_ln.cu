@@ -238,7 +238,7 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     auto load_row = [&](int ti, uint4* x) {
       const int row = ((int)blockIdx.x + ti * (int)gridDim.x) * BM + r;
       long long off = 0;
-      if (hh == 0 && row < g.M) off = g.has_map ? devmap_eval(g.rowmap, (uint32_t)row) : (long long)row * KDIM;
+      if (hh == 0 && row < g.M) off = g.has_map ? devmap_eval_unrolled(g.rowmap, (uint32_t)row) : (long long)row * KDIM;
       off = __shfl_sync(0xFFFFFFFFu, off, lane & ~1);
       const uint4* src = reinterpret_cast<const uint4*>(g.x + off) + hh * NH;
 #pragma unroll

@@ -281,7 +281,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int row = tile_m * BM + q * 32 + lane;
       const bool row_ok = row < g.M;
       long long off = 0;
-      if (row_ok) off = g.has_rowmap ? devmap_eval(g.rowmap, (uint32_t)row) : (long long)row * g.ldc;
+      if (row_ok) off = g.has_rowmap ? devmap_eval_unrolled(g.rowmap, (uint32_t)row) : (long long)row * g.ldc;
       off += (long long)batch * g.out_batch_stride;
       const __nv_bfloat16* __restrict__ rrow = g.residual ? g.residual + off : nullptr;
       const bool rope_tile = BN == 256 && g.rope_cols > 0 && n0 < g.rope_cols;

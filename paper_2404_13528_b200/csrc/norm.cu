@@ -44,7 +44,7 @@ __global__ void __launch_bounds__(256) norm_kernel(const T* __restrict__ src, T*
     active[r] = row < rows;
     long long soff = 0;
     if (has_map) {
-      if (sub == 0 && active[r]) soff = devmap_eval(rowmap, (uint32_t)row);   // one lane per row, then broadcast
+      if (sub == 0 && active[r]) soff = devmap_eval_unrolled(rowmap, (uint32_t)row);   // one lane per row, then broadcast
       soff = __shfl_sync(0xFFFFFFFFu, soff, lane - sub);
     } else if (active[r]) {
       soff = row * (long long)C;
