@@ -50,6 +50,7 @@ struct OpCoord {
 struct GemmArgs {
   int M, N, K;
   int tiles_n, tiles_m, batch;
+  FastDiv fd_tiles_n, fd_tiles_m;        // tile index -> (tile_n, tile_m, batch) without hardware division
   OpCoord ca, cb;
   __nv_bfloat16* out;
   long long ldc, out_batch_stride;
@@ -89,6 +90,14 @@ __device__ __forceinline__ TileCoord op_coords(const OpCoord& oc, uint32_t tile,
 __device__ __forceinline__ void tma_load_op(const OpCoord& oc, void* dst, const CUtensorMap* tm, uint64_t* bar, int k0,
                                             int row0, const TileCoord& tc) {
   ptx::tma_load_5d(dst, tm, bar, oc.mn_major ? row0 : k0, oc.mn_major ? k0 : row0, tc.o0, tc.o1, tc.o2);
+}
+
+struct TileIdx {
+  uint32_t tile_n, tile_m, batch;
+};
+__device__ __forceinline__ TileIdx split_tile(uint32_t t, const FastDiv& fn, const FastDiv& fm) {
+  const uint32_t r = fd_div(t, fn), b = fd_div(r, fm);
+  return {t - r * fn.d, r - b * fm.d, b};
 }
 
 // GELU in the bf16 epilogue: u * Phi(u) with Phi evaluated through the hyperbolic-tangent form
@@ -169,7 +178,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       bool ok = true;
       uint32_t pit = 0;
       for (uint32_t t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++pit) {
-        const uint32_t tile_n = t % g.tiles_n, r = t / g.tiles_n, tile_m = r % g.tiles_m, batch = r / g.tiles_m;
+        const TileIdx ti_ = split_tile(t, g.fd_tiles_n, g.fd_tiles_m);
+        const uint32_t tile_n = ti_.tile_n, tile_m = ti_.tile_m, batch = ti_.batch;
         GDBG(pit * 16 + 0);
         const TileCoord ta = op_coords(g.ca, tile_m, batch, BM), tb = op_coords(g.cb, tile_n, batch, BN);
         for (int kb = 0; kb < nkb; ++kb, ++kbg) {
@@ -242,7 +252,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       uint32_t s = 0, ph = 1;
       bool ok = true;
       for (uint32_t t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-        const uint32_t tile_n = t % g.tiles_n, r = t / g.tiles_n, batch = r / g.tiles_m;
+        const TileIdx ti_ = split_tile(t, g.fd_tiles_n, g.fd_tiles_m);
+        const uint32_t tile_n = ti_.tile_n, batch = ti_.batch;
         const TileCoord tb = op_coords(g.cb, tile_n, batch, BN);
         for (int kb = 0; kb < nkb; ++kb) {
           ok = ptx::mbar_wait(&empty[s], ph, abort_flag, g.status);
@@ -274,15 +285,28 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     uint8_t* qstage = stage_base + q * (32 * QROW);
     uint32_t it = 0;
     bool ok = true;
+    constexpr bool PREFETCH_NEXT = false;                   // (tried: next-tile offset + residual a tile ahead; the extra live registers spill and it is slower)
+    long long off_next = 0;
+    uint4 res_next[VPR];
     for (uint32_t t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
-      const uint32_t tile_n = t % g.tiles_n, r = t / g.tiles_n, tile_m = r % g.tiles_m, batch = r / g.tiles_m;
+      const TileIdx ti_ = split_tile(t, g.fd_tiles_n, g.fd_tiles_m);
+      const uint32_t tile_n = ti_.tile_n, tile_m = ti_.tile_m, batch = ti_.batch;
       const uint32_t buf = it & 1, use = it >> 1;
       const int n0 = tile_n * BN;
       const int row = tile_m * BM + q * 32 + lane;
       const bool row_ok = row < g.M;
-      long long off = 0;
-      if (row_ok) off = g.has_rowmap ? devmap_eval_unrolled(g.rowmap, (uint32_t)row) : (long long)row * g.ldc;
-      off += (long long)batch * g.out_batch_stride;
+      // Output offset of this thread's row (through the row map when the store is a scatter).  With
+      // one round per tile the offset and the residual of the NEXT tile were requested during the
+      // previous iteration, so neither the map evaluation nor the gather's latency is on the path
+      // between the accumulator becoming ready and its buffer being handed back.
+      long long off;
+      if (PREFETCH_NEXT && it > 0) {
+        off = off_next;
+      } else {
+        off = 0;
+        if (row_ok) off = g.has_rowmap ? devmap_eval_unrolled(g.rowmap, (uint32_t)row) : (long long)row * g.ldc;
+        off += (long long)batch * g.out_batch_stride;
+      }
       const __nv_bfloat16* __restrict__ rrow = g.residual ? g.residual + off : nullptr;
       const bool rope_tile = BN == 256 && g.rope_cols > 0 && n0 < g.rope_cols;
       auto col_of = [&](int rd) {
@@ -297,7 +321,29 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if (rrow && row_ok && n0 + c0 + v * 8 + 8 <= g.N) res[v] = *reinterpret_cast<const uint4*>(rrow + n0 + c0 + v * 8);
         }
       };
-      fetch_res(col_of(0));                                  // in flight while this tile's MMAs still run
+      if (PREFETCH_NEXT && it > 0) {
+#pragma unroll
+        for (int v = 0; v < VPR; ++v) res[v] = res_next[v];
+      } else {
+        fetch_res(col_of(0));                                // in flight while this tile's MMAs still run
+      }
+      if (PREFETCH_NEXT) {                                   // request the next tile's row offset and residual now
+        const uint32_t tn = t + gridDim.x;
+        if (tn < total_tiles) {
+          const TileIdx nx = split_tile(tn, g.fd_tiles_n, g.fd_tiles_m);
+          const int nrow = nx.tile_m * BM + q * 32 + lane;
+          off_next = 0;
+          if (nrow < g.M) off_next = g.has_rowmap ? devmap_eval_unrolled(g.rowmap, (uint32_t)nrow) : (long long)nrow * g.ldc;
+          off_next += (long long)nx.batch * g.out_batch_stride;
+          const int nn0 = nx.tile_n * BN, c0 = col_of(0);
+#pragma unroll
+          for (int v = 0; v < VPR; ++v) {
+            res_next[v] = make_uint4(0, 0, 0, 0);
+            if (g.residual && nrow < g.M && nn0 + c0 + v * 8 + 8 <= g.N)
+              res_next[v] = *reinterpret_cast<const uint4*>(g.residual + off_next + nn0 + c0 + v * 8);
+          }
+        }
+      }
 
       if (warp == 2 && lane == 0) GDBG(it * 16 + 8);
       ok = ptx::mbar_wait(&tmem_full[buf], use & 1, abort_flag, g.status);
@@ -671,6 +717,8 @@ int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep,
   if (!g.status) return SMARTMEM_ERR_CUDA;
   g.tiles_n = (int)((N + bn - 1) / bn);
   g.tiles_m = (int)((M + BM - 1) / BM);
+  g.fd_tiles_n = make_fastdiv((uint32_t)g.tiles_n);
+  g.fd_tiles_m = make_fastdiv((uint32_t)g.tiles_m);
   g.batch = (int)batch;
   if ((long long)g.tiles_n * g.tiles_m * g.batch >= (1ll << 31)) return SMARTMEM_ERR_UNSUPPORTED;
 #define SM_CASE(BN_, ST_, MN_)                                                                  \
