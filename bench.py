@@ -43,6 +43,16 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "source": "fallback (earlier measurement on this pool)"}
 
 
+def algorithmic_flops(w):
+    """Unpadded multiply-add flops of each kernel of the chain (attention: QK^T and PV over T x T per window)."""
+    M = w["B"] * w["H"] * w["W"]
+    C, r, T = w["C"], w["mlp_ratio"], w["window"] ** 2
+    qkv, proj, fc, att = 2 * M * C * 3 * C, 2 * M * C * C, 2 * M * C * r * C, 4 * M * T * C
+    return {"qkv_gemm": qkv, "ln1_gather_qkv_gemm": qkv, "ln1_qkv_gemm": qkv, "window_attention": att,
+            "proj_gemm_scatter_residual": proj, "proj_gemm_residual": proj, "fc1_gemm_gelu": fc, "fc2_gemm_residual": fc,
+            "mlp_fused_fc1_gelu_fc2_residual": 2 * fc, "mlp_fused_ln2_fc1_gelu_fc2_residual": 2 * fc}
+
+
 def algorithmic_bytes(w):
     """Compulsory HBM bytes of each kernel of the ELIMINATE chain: every input once, every output once."""
     U = w["B"] * w["H"] * w["W"] * w["C"] * 2          # one [M, C] bf16 tensor
@@ -460,15 +470,22 @@ def main():
                                                          mode, stream):
                 per[mode].setdefault(name, []).append(ms)
     peaks = measured_peaks()
-    ab = algorithmic_bytes(w)
+    _, tf_peak, _ = _peaks_all()
+    ab, af = algorithmic_bytes(w), algorithmic_flops(w)
     kernels = {}
     for mode, tag in ((sm.ELIMINATE, "eliminate"), (sm.EXPLICIT, "explicit")):
         kernels[tag] = []
         for name, v in per[mode].items():
             ms = statistics.median(v)
             gbs = ab[name] / (ms * 1e-3) / 1e9 if ms > 0 else None
-            kernels[tag].append({"kernel": name, "ms": round(ms, 5), "algorithmic_bytes": ab[name],
-                                 "gbs": gbs and round(gbs, 1), "frac_of_hbm_peak": gbs and round(gbs / peaks["hbm_gbs"], 4)})
+            fl = af.get(name, 0)
+            tfs = fl / (ms * 1e-3) / 1e12 if ms > 0 else None
+            # the roofline that binds the kernel: whichever ideal time is longer, bytes at the HBM peak or flops at the tensor peak
+            tensor_bound = fl / (tf_peak * 1e12) > ab[name] / (peaks["hbm_gbs"] * 1e9)
+            kernels[tag].append({"kernel": name, "ms": round(ms, 5), "algorithmic_bytes": ab[name], "algorithmic_flops": fl,
+                                 "gbs": gbs and round(gbs, 1), "frac_of_hbm_peak": gbs and round(gbs / peaks["hbm_gbs"], 4),
+                                 "tflops": tfs and round(tfs, 1), "frac_of_tensor_peak": tfs and round(tfs / tf_peak, 4),
+                                 "bound": "tensor" if tensor_bound else "hbm"})
     dom = max(kernels["eliminate"], key=lambda k: k["ms"])
 
     # end to end through the C ABI with host buffers: every step copies its input from pinned host
@@ -548,8 +565,11 @@ def main():
                     "h2d_bytes_per_step": x_host.numel() * 2, "d2h_bytes_per_step": y_host.numel() * 2},
             "gpu_launches": launches,
             "clocks": clocks,
-            "roofline": {"bound": "hbm", "kernel": dom["kernel"], "achieved": dom["gbs"], "peak": peaks["hbm_gbs"],
-                         "unit": "GB/s", "frac": dom["frac_of_hbm_peak"], "traffic": traffic, "peak_source": peaks["source"]},
+            "roofline": ({"bound": "tensor", "kernel": dom["kernel"], "achieved": dom["tflops"], "peak": tf_peak,
+                          "unit": "TFLOP/s", "frac": dom["frac_of_tensor_peak"], "traffic": traffic,
+                          "peak_source": peaks["source"] + "; bf16 burst"} if dom["bound"] == "tensor" else
+                         {"bound": "hbm", "kernel": dom["kernel"], "achieved": dom["gbs"], "peak": peaks["hbm_gbs"],
+                          "unit": "GB/s", "frac": dom["frac_of_hbm_peak"], "traffic": traffic, "peak_source": peaks["source"]}),
             "kernels": kernels,
         }
         if cpu is not None:

@@ -253,8 +253,8 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const uint64_t bd = ptx::make_smem_desc(w_base + ws * WST_BYTES, 16, 1024);
         ptx::tc_mma_bf16_ta(d, a, bd, idesc2, c2 != 0 ? 1u : 0u);
 #pragma unroll
-        for (int k = 1; k < HC / 16; ++k)
-          ptx::tc_mma_bf16_ta(d, a + 8 * k, bd + (k >> 2) * (KB_BYTES >> 4) + 2 * (k & 3), idesc2, 1u);
+        for (int k = 1; k < HC / 16; ++k)               // k-step k: GELU warp group k / 2 wrote it at column 32 (k / 2) + 8 (k % 2)
+          ptx::tc_mma_bf16_ta(d, a + 32 * (k >> 1) + 8 * (k & 1), bd + (k >> 2) * (KB_BYTES >> 4) + 2 * (k & 3), idesc2, 1u);
         ptx::tc_commit(&w_empty[ws]);
         ptx::tc_commit(&s1_empty[hb]);                  // H lived in the S1 buffer: fc1 may overwrite it now
         DBG(j * 16 + 7);
@@ -266,10 +266,9 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       }
     }
   } else if (warp < 2 + kGeluWarps) {
-    // GELU warps: S1 chunk (TMEM, fp32) -> + b1 -> GELU -> bf16 pairs -> back into the first 64
-    // columns of the same TMEM buffer, where fc2 reads the chunk as its A operand.  The packed H
-    // columns of one warp overlap S1 columns another warp of the quadrant still has to read, so
-    // the quadrant's four warps meet between their loads and their stores.
+    // GELU warps: S1 chunk (TMEM, fp32) -> + b1 -> GELU -> bf16 pairs -> back into the same TMEM
+    // buffer, where fc2 reads the chunk as its A operand.  Each warp overwrites the first 16 of the
+    // 32 columns it has just read (its own lanes), so no warp waits for another.
     const int e = warp - 2, q = warp & 3, grp = e >> 2;
     bool ok = true;
     int c = 0;
@@ -286,17 +285,7 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         ptx::tmem_ld32(tq + grp * 32, rv);
         ptx::tmem_ld_wait();
       }
-      // always reached by all four warps of the quadrant; they leave together if any gave up waiting
-      uint32_t gave_up;
-      asm volatile(
-          "{\n\t.reg .pred pin, pout;\n\t"
-          "setp.ne.u32 pin, %2, 0;\n\t"
-          "bar.red.or.pred pout, %1, 128, pin;\n\t"
-          "selp.u32 %0, 1, 0, pout;\n\t}"
-          : "=r"(gave_up)
-          : "r"(1 + q), "r"(ok ? 0u : 1u)
-          : "memory");
-      if (gave_up) break;
+      if (!ok) break;
       if (e == 0 && lane == 0) DBG(j * 16 + 10);
       uint32_t pk[16];
 #pragma unroll
@@ -307,7 +296,7 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         pk[i] = gelu_tanh_bf16x2(__uint_as_float(rv[2 * i]) + bb[2 * i], __uint_as_float(rv[2 * i + 1]) + bb[2 * i + 1]);
 #endif
       }
-      ptx::tmem_st16(tq + grp * 16, pk);
+      ptx::tmem_st16(tq + grp * 32, pk);               // over the first half of the columns this warp has just read
       ptx::tmem_st_wait();
       if (e == 0 && lane == 0) DBG(j * 16 + 11);
       ptx::tc_fence_before();
