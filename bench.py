@@ -189,7 +189,7 @@ def run_reference(args):
 # The other configurations (parity-test cases): timed on request with --workload, same protocol.
 # ------------------------------------------------------------------------------------------------
 OTHER_WORKLOADS = ["swin_b_stage3_block_pair", "llama_attention_layer", "chain_2a_qkt", "chain_2b_gemm",
-                   "chain_2a_copy", "chain_2b_copy"]
+                   "chain_2a_copy", "chain_2b_copy", "swin_shift_partition_copy"]
 
 
 def _peaks_all():
@@ -271,9 +271,18 @@ def run_other(args):
         model = [("rmsnorm", 2 * X, 0), ("qkv_gemm_rope", 4 * X + 3 * hidden * hidden * 2, 2 * S * hidden * 3 * hidden),
                  ("causal_attention", 4 * X, 4 * heads * 128 * S * (S + 1) // 2), ("o_proj_gemm", 2 * X + hidden * hidden * 2, 2 * S * hidden * hidden)]
     else:
-        which = "2a" if "2a" in name else "2b"
-        inp = synth.chain_inputs(2, which)
-        if which == "2a":
+        which = "2a" if "2a" in name else "2b" if "2b" in name else "e1"
+        inp = synth.chain_inputs(2, which if which != "e1" else "2a")
+        if which == "e1":
+            # the shift o partition chain of the Swin-T stage-1 block on its own: [32,56,56,96] -> [2048,49,96]
+            B, Hh, Ww, C, wsz, sh = 32, 56, 56, 96, 7, 3
+            x = torch.from_numpy(synth.normal(0x5EED0003, 0, (B, Hh, Ww, C), dtype="bf16").view(np.int16).copy()).cuda().view(torch.bfloat16)
+            ops = [sm.make_op(sm.OP_ROLL, shift=-sh, axis=1), sm.make_op(sm.OP_ROLL, shift=-sh, axis=2),
+                   sm.make_op(sm.OP_WINDOW_PARTITION, window=wsz), sm.make_op(sm.OP_COPY)]
+            srcs, descs, oshape = [x], [sm.make_desc((B, Hh, Ww, C))], (B * (Hh // wsz) * (Ww // wsz), wsz * wsz, C)
+            model = [("copy_map", 2 * B * Hh * Ww * C * 2, 0)]
+            tokens = B * Hh * Ww
+        elif which == "2a":
             B, S, Hh, D = inp["dims"]
             layout = [sm.make_op(sm.OP_RESHAPE, shape=(B, S, Hh, D)), sm.make_op(sm.OP_TRANSPOSE, perm=(0, 2, 1, 3))]
             srcs = [dev(inp["xq"]), dev(inp["xk"])]
@@ -298,7 +307,7 @@ def run_other(args):
                 model = [("gemm_mn_major_operand", B * C * Hh * Ww * 2 + N * C * 2 + B * Hh * Ww * N * 2, 2 * B * Hh * Ww * N * C)]
             tokens = B * Hh * Ww
         sets = 8
-        modes = (sm.ELIMINATE, sm.EXPLICIT) + ((sm.ELIMINATE_NAIVE,) if name.endswith("copy") else ())
+        modes = (sm.ELIMINATE, sm.EXPLICIT) + ((sm.ELIMINATE_NAIVE, sm.ELIMINATE_GATHER, sm.ELIMINATE_SCATTER) if name.endswith("copy") else ())
         plans = {m: sm.smartmem_plan(ops, descs, m) for m in modes}
         wsb = {m: sm.smartmem_plan_workspace_bytes(plans[m]) for m in plans}
         ins = [[t.clone() for t in srcs] for _ in range(sets)]
@@ -327,10 +336,18 @@ def run_other(args):
         step(i, sm.EXPLICIT)
     ms = {m: timed(m, args.steps) for m in (sm.ELIMINATE, sm.EXPLICIT)}
     ms_naive = None
+    placement = None
     if name.endswith("copy"):
         for i in range(args.warmup):
             step(i, sm.ELIMINATE_NAIVE)
         ms_naive = timed(sm.ELIMINATE_NAIVE, args.steps)
+        # the same eliminated map on the consumer side (gather on load) and on the producer side (scatter on store)
+        for m in (sm.ELIMINATE_GATHER, sm.ELIMINATE_SCATTER):
+            for i in range(args.warmup):
+                step(i, m)
+        mg, msc = timed(sm.ELIMINATE_GATHER, args.steps), timed(sm.ELIMINATE_SCATTER, args.steps)
+        placement = {"gather_on_load_ms_per_step": mg / args.steps, "scatter_on_store_ms_per_step": msc / args.steps,
+                     "gather_over_scatter": mg / msc}
     per = {}
     for mode, tag in ((sm.ELIMINATE, "eliminate"), (sm.EXPLICIT, "explicit")):
         acc = None
@@ -363,6 +380,7 @@ def run_other(args):
                              "kernels": [{"launched_as": n, "ms": round(t, 5)} for n, t in per["explicit"]]},
         "naive_index_variant": None if ms_naive is None else {"ms_per_step": ms_naive / args.steps,
                                                                  "speedup_of_strength_reduced_map": ms_naive / ms[sm.ELIMINATE]},
+        "map_placement": placement,
         "clocks": clocks,
         "roofline": {"bound": dom["bound"], "kernel": dom["kernel"], "achieved": dom["achieved"], "unit": dom["unit"],
                      "peak": tf if dom["bound"] == "tensor" else hbm, "frac": dom["frac"], "traffic": None, "peak_source": src},

@@ -58,7 +58,13 @@ typedef enum { SMARTMEM_F32 = 0, SMARTMEM_BF16 = 1 } smartmem_dtype_t;
 /* ELIMINATE_NAIVE (smartmem_plan / smartmem_run_chain only): layout runs are eliminated, but copy
  * consumers evaluate the sequential divide/modulo program instead of the strength-reduced map --
  * the "index computation (no opt.)" form of Fig. 4, kept to measure what strength reduction buys. */
-typedef enum { SMARTMEM_ELIMINATE = 0, SMARTMEM_EXPLICIT = 1, SMARTMEM_ELIMINATE_NAIVE = 2 } smartmem_mode_t;
+/* ELIMINATE_GATHER / ELIMINATE_SCATTER (smartmem_plan / smartmem_run_chain, copy-only chains of invertible
+ * layout operators): the eliminated map is placed on the consumer side (out[i] = in[map(i)]: sub-optimal
+ * read, contiguous write) or on the producer side (out[imap(i)] = in[i], imap = the map of the inverted
+ * chain: contiguous read, sub-optimal write), both with the plain map-driven kernel -- the two
+ * placements Section 3.2.2 compares.  Same result as ELIMINATE, bit for bit. */
+typedef enum { SMARTMEM_ELIMINATE = 0, SMARTMEM_EXPLICIT = 1, SMARTMEM_ELIMINATE_NAIVE = 2,
+               SMARTMEM_ELIMINATE_GATHER = 3, SMARTMEM_ELIMINATE_SCATTER = 4 } smartmem_mode_t;
 
 /* Operator vocabulary of a chain.  Layout operators have a Fixed output layout (Table 3,
  * right column) and are the ones elimination removes; compute operators are kept. */

@@ -153,7 +153,7 @@ EXPORT int smartmem_run_chain(const smartmem_plan_t* plan, const void* const* in
         if (!make_devseq(s.seq[0], &q)) return SMARTMEM_ERR_UNSUPPORTED;
         rc = launch_copy_seq(q, s.map[0].n_elements, esz, buf(s.src[0]), buf(s.dst), st);
       } else {
-        rc = launch_copy_map(s.map[0], esz, buf(s.src[0]), buf(s.dst), st);
+        rc = launch_copy_map(s.map[0], esz, buf(s.src[0]), buf(s.dst), st, s.placement);
       }
     } else if (s.kind == STEP_LINEAR || s.kind == STEP_BMM_NT) {
       if (s.dtype != SMARTMEM_BF16) return SMARTMEM_ERR_UNSUPPORTED;

@@ -246,7 +246,10 @@ struct DevSeq {
 int launch_copy_seq(const DevSeq& seq, long long n_elements, int elem_size, const void* src, void* dst, cudaStream_t st);
 
 // Map-driven copy: out (contiguous) <- src through `map`.
-int launch_copy_map(const smartmem_index_map_t& map, int elem_size, const void* src, void* dst, cudaStream_t st);
+// placement: 0 = best kernel for the map (tiled transposes where they apply); 1 = the plain map-driven
+// gather (out[i] = src[map(i)]); 2 = the plain map-driven scatter (dst[map(i)] = src[i]).
+int launch_copy_map(const smartmem_index_map_t& map, int elem_size, const void* src, void* dst, cudaStream_t st,
+                    int placement = 0);
 
 // LayerNorm / RMSNorm over rows of length C.  Row r of the output (row-major [rows, C]) is
 // read from src at element offset rowmap(r) (rowmap == nullptr: r * C).

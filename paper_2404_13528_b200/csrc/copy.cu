@@ -67,6 +67,22 @@ __global__ void __launch_bounds__(256) copy_gather_kernel(const __grid_constant_
   *reinterpret_cast<V*>(dst + (size_t)i * VB) = v;
 }
 
+// The same map placed on the producer side: one thread per INPUT vector, loaded contiguously
+// (coalesced) and stored through the map (here the map of the inverted chain: where each input
+// vector goes).  The sub-optimal access is the write instead of the read.
+template <int VB>
+__global__ void __launch_bounds__(256) copy_scatter_kernel(const __grid_constant__ DevMap map, const char* __restrict__ src,
+                                                           char* __restrict__ dst, uint32_t n_units, int elem_size) {
+  pdl_wait();
+  pdl_launch_dependents();
+  using V = typename VecT<VB>::type;
+  uint32_t i = blockIdx.x * 256u + threadIdx.x;
+  if (i >= n_units) return;
+  long long off = devmap_eval_unrolled(map, i);
+  V v = *reinterpret_cast<const V*>(src + (size_t)i * VB);
+  *reinterpret_cast<V*>(dst + off * elem_size) = v;
+}
+
 // Affine map whose consumer-innermost atom I is strided in the source while another atom J is
 // source-contiguous: a 64 x 64 tile transpose of 2-byte elements through shared memory.  Loads are
 // 16-byte vectors along J, stores 16-byte vectors along I.
@@ -220,11 +236,12 @@ int launch_copy_seq(const DevSeq& seq, long long n, int elem_size, const void* s
   return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
 }
 
-int launch_copy_map(const smartmem_index_map_t& map, int elem_size, const void* src, void* dst, cudaStream_t st) {
-  profile_tick("copy_map", st);
+int launch_copy_map(const smartmem_index_map_t& map, int elem_size, const void* src, void* dst, cudaStream_t st, int placement) {
+  profile_tick(placement == 2 ? "copy_map_scatter" : placement == 1 ? "copy_map_gather" : "copy_map", st);
   if (map.klass == 3) return SMARTMEM_ERR_UNSUPPORTED;
   if (map.n_elements == 0) return SMARTMEM_OK;
   const int n = map.n_atoms;
+  if (placement == 0) {
   // fast path: batched transpose of small contiguous blocks
   if (map.klass == 1 && elem_size == 2 && n >= 2 && map.src_stride[n - 1] != 1 && map.src_stride[n - 2] == 1 &&
       map.src_stride[n - 1] == map.extent[n - 2] && map.extent[n - 1] * map.extent[n - 2] <= 16384 &&
@@ -279,6 +296,7 @@ int launch_copy_map(const smartmem_index_map_t& map, int elem_size, const void* 
       }
     }
   }
+  }   // placement == 0: the tiled fast paths above; 1 / 2: the plain map-driven kernel on the consumer / producer side
   const int v = map.vec_elems;
   const int vb = v * elem_size;
   DevMap d;
@@ -286,13 +304,18 @@ int launch_copy_map(const smartmem_index_map_t& map, int elem_size, const void* 
   long long units = map.n_elements / v;
   if (units >= (1ll << 31)) return SMARTMEM_ERR_UNSUPPORTED;
   unsigned grid = (unsigned)((units + 255) / 256);
+#define SM_COPY(VB_)                                                                                                     \
+  case VB_:                                                                                                              \
+    if (placement == 2)                                                                                                  \
+      launch_pdl(copy_scatter_kernel<VB_>, dim3(grid), dim3(256), 0, st, d, (const char*)src, (char*)dst, (uint32_t)units, elem_size); \
+    else                                                                                                                 \
+      launch_pdl(copy_gather_kernel<VB_>, dim3(grid), dim3(256), 0, st, d, (const char*)src, (char*)dst, (uint32_t)units, elem_size);  \
+    break;
   switch (vb) {
-    case 16: launch_pdl(copy_gather_kernel<16>, dim3(grid), dim3(256), 0, st, d, (const char*)src, (char*)dst, (uint32_t)units, elem_size); break;
-    case 8: launch_pdl(copy_gather_kernel<8>, dim3(grid), dim3(256), 0, st, d, (const char*)src, (char*)dst, (uint32_t)units, elem_size); break;
-    case 4: launch_pdl(copy_gather_kernel<4>, dim3(grid), dim3(256), 0, st, d, (const char*)src, (char*)dst, (uint32_t)units, elem_size); break;
-    case 2: launch_pdl(copy_gather_kernel<2>, dim3(grid), dim3(256), 0, st, d, (const char*)src, (char*)dst, (uint32_t)units, elem_size); break;
+    SM_COPY(16) SM_COPY(8) SM_COPY(4) SM_COPY(2)
     default: return SMARTMEM_ERR_UNSUPPORTED;
   }
+#undef SM_COPY
   count_launch();
   return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
 }

@@ -554,11 +554,76 @@ int smartmem_pair_decision(int32_t a, int32_t b, int32_t* action, int32_t* resul
   return SMARTMEM_OK;
 }
 
+// Copy-only chains with the eliminated map placed explicitly on one side of the copy
+// (Section 3.2.2: a sub-optimal write is preferred to a sub-optimal read).  GATHER composes the chain
+// as usual and pins the plain map-driven kernel: out[i] = in[map(i)].  SCATTER inverts the chain
+// (operators in reverse order, each replaced by its inverse), composes THAT from the output tensor's
+// point of view, and obtains for every input element the output offset it goes to: out[imap(i)] = in[i].
+static int plan_placement(const smartmem_op_t* ops, int32_t n_ops, const smartmem_tensor_desc_t* inputs, int32_t n_inputs,
+                          int32_t mode, smartmem_plan_t** out_plan) {
+  if (n_ops < 2 || ops[n_ops - 1].kind != SMARTMEM_OP_COPY || n_inputs != 1) return SMARTMEM_ERR_UNSUPPORTED;
+  for (int i = 0; i + 1 < n_ops; ++i)
+    if (!is_layout_kind(ops[i].kind)) return SMARTMEM_ERR_UNSUPPORTED;
+  smartmem_plan_t* fwd = nullptr;
+  int rc = smartmem_plan(ops, n_ops, inputs, n_inputs, SMARTMEM_ELIMINATE, &fwd);
+  if (rc != SMARTMEM_OK) return rc;
+  // both placements run the strength-reduced map; chains that only the sequential program can evaluate are not covered
+  if (fwd->steps.size() != 1 || fwd->steps[0].kind != STEP_COPY || fwd->steps[0].map[0].klass == 3) { delete fwd; return SMARTMEM_ERR_UNSUPPORTED; }
+  if (mode == SMARTMEM_ELIMINATE_GATHER) {
+    fwd->mode = mode;
+    fwd->steps[0].placement = 1;
+    *out_plan = fwd;
+    return SMARTMEM_OK;
+  }
+  if (!state_from_desc(inputs[0]).fresh) { delete fwd; return SMARTMEM_ERR_UNSUPPORTED; }   // the scatter walks the input linearly
+  // invert the stages the forward composition went through (window operators are already expanded)
+  std::vector<smartmem_op_t> inv;
+  const auto& stages = fwd->steps[0].seq[0].stages;
+  for (int k = (int)stages.size() - 1; k >= 0 && rc == SMARTMEM_OK; --k) {
+    const SeqStage& sg = stages[k];
+    smartmem_op_t o;
+    memset(&o, 0, sizeof(o));
+    o.kind = sg.kind;
+    if (sg.kind == SMARTMEM_OP_RESHAPE) {
+      o.ndim = (int)sg.in_shape.size();
+      for (int d = 0; d < o.ndim; ++d) o.shape[d] = sg.in_shape[d];
+    } else if (sg.kind == SMARTMEM_OP_TRANSPOSE) {
+      o.ndim = (int)sg.perm.size();
+      for (int d = 0; d < o.ndim; ++d) o.perm[sg.perm[d]] = d;
+    } else if (sg.kind == SMARTMEM_OP_ROLL) {
+      o.axis = sg.axis;
+      o.shift = -sg.shift;
+    } else {
+      rc = SMARTMEM_ERR_UNSUPPORTED;                 // a Slice drops elements: no inverse
+    }
+    inv.push_back(o);
+  }
+  smartmem_op_t cp;
+  memset(&cp, 0, sizeof(cp));
+  cp.kind = SMARTMEM_OP_COPY;
+  inv.push_back(cp);
+  smartmem_plan_t* bwd = nullptr;
+  const smartmem_tensor_desc_t out_desc = fwd->out_desc;
+  delete fwd;
+  if (rc != SMARTMEM_OK) return rc;
+  rc = smartmem_plan(inv.data(), (int)inv.size(), &out_desc, 1, SMARTMEM_ELIMINATE, &bwd);
+  if (rc != SMARTMEM_OK) return rc;
+  if (bwd->steps.size() != 1 || bwd->steps[0].kind != STEP_COPY || bwd->steps[0].map[0].klass == 3) { delete bwd; return SMARTMEM_ERR_UNSUPPORTED; }
+  bwd->mode = mode;
+  bwd->steps[0].placement = 2;       // map[0]: input linear index -> output offset
+  bwd->out_desc = out_desc;
+  *out_plan = bwd;
+  return SMARTMEM_OK;
+}
+
 int smartmem_plan(const smartmem_op_t* ops, int32_t n_ops, const smartmem_tensor_desc_t* inputs, int32_t n_inputs,
                   int32_t mode, smartmem_plan_t** out_plan) {
   if (!ops || !inputs || !out_plan || n_ops < 1 || n_inputs < 1) return SMARTMEM_ERR_INVALID_ARG;
-  if (mode != SMARTMEM_ELIMINATE && mode != SMARTMEM_EXPLICIT && mode != SMARTMEM_ELIMINATE_NAIVE)
+  if (mode != SMARTMEM_ELIMINATE && mode != SMARTMEM_EXPLICIT && mode != SMARTMEM_ELIMINATE_NAIVE &&
+      mode != SMARTMEM_ELIMINATE_GATHER && mode != SMARTMEM_ELIMINATE_SCATTER)
     return SMARTMEM_ERR_INVALID_ARG;
+  if (mode == SMARTMEM_ELIMINATE_GATHER || mode == SMARTMEM_ELIMINATE_SCATTER)
+    return plan_placement(ops, n_ops, inputs, n_inputs, mode, out_plan);
   for (int i = 0; i < n_inputs; ++i) {
     if (inputs[i].ndim < 1 || inputs[i].ndim > SMARTMEM_MAX_DIMS) return SMARTMEM_ERR_INVALID_ARG;
     if (inputs[i].dtype != SMARTMEM_F32 && inputs[i].dtype != SMARTMEM_BF16) return SMARTMEM_ERR_INVALID_ARG;

@@ -40,6 +40,7 @@ struct Step {
   SeqProgram seq[2];
   int64_t batch = 1, M = 0, N = 0, K = 0;
   bool is_layout_copy = false;
+  int placement = 0;                 // STEP_COPY: 0 best kernel, 1 plain gather through map[0], 2 plain scatter through map[0]
 };
 
 }  // namespace smartmem

@@ -34,7 +34,14 @@ def copy_chain_case(shape, chain, dtype="bf16"):
     ops = _ops_from_chain(chain) + [sm.make_op(sm.OP_COPY)]
     desc = [sm.make_desc(shape, sm.BF16 if dtype == "bf16" else sm.F32)]
     tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
-    for mode in (sm.ELIMINATE, sm.EXPLICIT, sm.ELIMINATE_NAIVE):
+    modes = [sm.ELIMINATE, sm.EXPLICIT, sm.ELIMINATE_NAIVE]
+    if all(o["op"] != "slice" for o in chain):
+        try:                                                # map placed on the consumer / producer side
+            sm.smartmem_plan_destroy(sm.smartmem_plan(ops, desc, sm.ELIMINATE_SCATTER))
+            modes += [sm.ELIMINATE_GATHER, sm.ELIMINATE_SCATTER]
+        except sm.SmartmemError:
+            pass                                            # chains whose inverse does not refine
+    for mode in modes:
         out = run_plan(ops, desc, mode, [xd], ref.shape, tdt)
         assert np.array_equal(to_host_bits(out), ref), f"mode {mode}"
 

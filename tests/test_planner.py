@@ -273,3 +273,46 @@ def test_plan_errors():
         sm.smartmem_plan([sm.make_op(sm.OP_LINEAR, side_input=(1, 0))], [sm.make_desc((4, 6)), sm.make_desc((3, 5))], sm.ELIMINATE)
     assert e.value.code == sm.ERR_SHAPE
     assert sm.smartmem_status_string(sm.ERR_TIMEOUT) == "device-side wait timed out"
+
+
+# ------------------------------------------------------------------ producer-side placement (Section 3.2.2)
+@pytest.mark.parametrize("shape,chain", [
+    ((2, 6, 4 * 3), [{"op": "reshape", "shape": (2, 6, 4, 3)}, {"op": "transpose", "perm": (0, 2, 1, 3)}]),
+    ((2, 5, 3, 4), [{"op": "transpose", "perm": (0, 2, 3, 1)}, {"op": "reshape", "shape": (2, 12, 5)}]),
+    ((2, 8, 8, 3), [{"op": "roll", "shift": -2, "axis": 1}, {"op": "roll", "shift": -2, "axis": 2},
+                    {"op": "window_partition", "window": 4}]),
+    ((2 * 2 * 2, 16, 3), [{"op": "window_reverse", "window": 4, "B": 2, "H": 8, "W": 8},
+                          {"op": "roll", "shift": 2, "axis": 1}, {"op": "roll", "shift": 2, "axis": 2}]),
+    ((5, 5, 5), [{"op": "reshape", "shape": (5, 25)}, {"op": "transpose", "perm": (1, 0)}]),
+])
+def test_scatter_placement_map_is_the_inverse_permutation(shape, chain):
+    """ELIMINATE_SCATTER plans the inverted chain: its map sends input element i to the output position
+    that, in the oracle's materialised result, holds input element i."""
+    src = chains.source_offsets(shape, chain).reshape(-1)          # output position -> input element
+    dest = np.empty_like(src)
+    dest[src] = np.arange(src.size)                                # input element -> output position
+    plan = _plan_copy(shape, chain, mode=sm.ELIMINATE_SCATTER)
+    try:
+        assert sm.smartmem_plan_num_steps(plan) == (1, 0)
+        m = sm.smartmem_plan_get_map(plan, 0)
+        assert m.klass != 3 and m.n_elements == src.size
+        assert [sm.smartmem_map_eval(m, i) for i in range(src.size)] == dest.tolist()
+        d = sm.smartmem_plan_output_desc(plan)
+        assert tuple(d.shape[: d.ndim]) == chains.source_offsets(shape, chain).shape
+    finally:
+        sm.smartmem_plan_destroy(plan)
+    g = _plan_copy(shape, chain, mode=sm.ELIMINATE_GATHER)         # consumer side: the usual map
+    try:
+        mg = sm.smartmem_plan_get_map(g, 0)
+        assert [sm.smartmem_map_eval(mg, i) for i in range(src.size)] == src.tolist()
+    finally:
+        sm.smartmem_plan_destroy(g)
+
+
+def test_placement_modes_reject_what_they_cannot_invert():
+    sl = [{"op": "slice", "start": (1, 0), "extent": (2, 4)}]
+    with pytest.raises(sm.SmartmemError):
+        _plan_copy((4, 4), sl, mode=sm.ELIMINATE_SCATTER)           # a Slice drops elements
+    ops = [sm.make_op(sm.OP_LINEAR, side_input=(1, 0))]
+    with pytest.raises(sm.SmartmemError):
+        sm.smartmem_plan(ops, [sm.make_desc((8, 8)), sm.make_desc((8, 8))], sm.ELIMINATE_SCATTER)   # copy-only chains
