@@ -274,7 +274,7 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     int c = 0;
     for (int j = 0; j < total && ok; ++j) {
       const uint32_t sb = j & 1;
-      const float* bb = b1_s + c * HC + grp * 32;        // this warp's 32 biases of the chunk (broadcast reads)
+      const float4* bb4 = reinterpret_cast<const float4*>(b1_s + c * HC + grp * 32);   // this warp's 32 biases of the chunk: eight 16-byte broadcast reads
       if (e == 0 && lane == 0) DBG(j * 16 + 8);
       ok = ptx::mbar_wait(&s1_full[sb], (j >> 1) & 1, abort_flag, g.status);
       if (e == 0 && lane == 0) DBG(j * 16 + 9);
@@ -289,11 +289,14 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       if (e == 0 && lane == 0) DBG(j * 16 + 10);
       uint32_t pk[16];
 #pragma unroll
-      for (int i = 0; i < 16; ++i) {
+      for (int v = 0; v < 8; ++v) {
+        const float4 b4 = bb4[v];
 #ifdef MLP_EXP_NOGELU
-        pk[i] = float2_to_bf16x2(__uint_as_float(rv[2 * i]) + bb[2 * i], __uint_as_float(rv[2 * i + 1]) + bb[2 * i + 1]);
+        pk[2 * v] = float2_to_bf16x2(__uint_as_float(rv[4 * v]) + b4.x, __uint_as_float(rv[4 * v + 1]) + b4.y);
+        pk[2 * v + 1] = float2_to_bf16x2(__uint_as_float(rv[4 * v + 2]) + b4.z, __uint_as_float(rv[4 * v + 3]) + b4.w);
 #else
-        pk[i] = gelu_tanh_bf16x2(__uint_as_float(rv[2 * i]) + bb[2 * i], __uint_as_float(rv[2 * i + 1]) + bb[2 * i + 1]);
+        pk[2 * v] = gelu_tanh_bf16x2(__uint_as_float(rv[4 * v]) + b4.x, __uint_as_float(rv[4 * v + 1]) + b4.y);
+        pk[2 * v + 1] = gelu_tanh_bf16x2(__uint_as_float(rv[4 * v + 2]) + b4.z, __uint_as_float(rv[4 * v + 3]) + b4.w);
 #endif
       }
       ptx::tmem_st16(tq + grp * 32, pk);               // over the first half of the columns this warp has just read
