@@ -1,13 +1,17 @@
 // Causal attention (prefill, head dimension 128) on the tcgen05 tensor cores.
 //
 // One CTA = 128 query positions of one head.  K and V stream through shared memory in tiles of
-// 128 keys (TMA, double buffered); S = Q K^T and O += P V are tcgen05.mma with the accumulators in
-// TMEM (two S buffers, one O); four softmax warps own one query row per thread (the TMEM lane),
+// 64 keys (TMA, double buffered); S = Q K^T and O += P V are tcgen05.mma with the accumulators in
+// TMEM (two S buffers, one O: 256 columns); four softmax warps own one query row per thread (the TMEM lane),
 // so row maxima and sums need no shuffles.  P goes back to the tensor core through shared memory in
 // the K-major swizzled operand layout; V is consumed as it lies in memory ([key, d] rows) through
 // the MN-major operand mode, so no transpose of V exists anywhere.  The running maximum is only
 // refreshed when it grows by more than 2^8 (then O and the running sum are rescaled), which keeps
 // the TMEM read-modify-write of O off the common path.
+//
+// The 64-key tiles keep a CTA at 112 KB of shared memory and 256 TMEM columns, so TWO CTAs share an
+// SM: while one is in its softmax (which is bound by the exponential unit) the other one's MMAs
+// run, which a single CTA with one softmax group could not overlap.
 //
 // q, k, v are addressed as TMA boxes inside the buffer the QKV GEMM wrote ([B*S, 3*H*D], head split
 // eliminated) or inside materialised [B, H, S, D] tensors (explicit variant); the output tile is
@@ -19,9 +23,10 @@
 namespace smartmem {
 namespace {
 
-constexpr int BQ = 128, BKV = 128, D = 128;
-constexpr int KB = 128 * 64 * 2;                      // one 128 x 64 bf16 block
-constexpr uint32_t TM_S = 0, TM_O = 256, TMEM_COLS = 512;
+constexpr int BQ = 128, BKV = 64, D = 128;
+constexpr int KB = 128 * 64 * 2;                      // one 128 x 64 bf16 block (Q, P)
+constexpr int KBK = BKV * 64 * 2;                     // one 64 x 64 bf16 block (K, V)
+constexpr uint32_t TM_S = 0, TM_O = 128, TMEM_COLS = 256;   // two S buffers of 64 columns, O of 128: two CTAs share an SM's 512
 constexpr int kThreads = 192;
 constexpr float kRescaleThreshold = 8.0f;             // log2 units
 
@@ -32,6 +37,7 @@ struct TcAttnArgs {
   __nv_bfloat16* out;
   long long o_sn, o_sh, o_st;
   float scale_log2;
+  uint32_t smem_bytes;
   int* status;
 };
 
@@ -52,28 +58,33 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
       : "memory");
 }
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 2)
 causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                       const __grid_constant__ CUtensorMap tmV, const __grid_constant__ TcAttnArgs g) {
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const uint32_t pad = (1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u;
+  uint8_t* smem = smem_raw + pad;
   uint8_t* sQ = smem;                                  // [2 k-blocks][16 KB]
-  uint8_t* sK = sQ + 2 * KB;                           // [2 stages][2 k-blocks][16 KB]
-  uint8_t* sV = sK + 4 * KB;                           // [2 stages][2 d-chunks][16 KB]
-  uint8_t* sP = sV + 4 * KB;                           // [2 k-blocks][16 KB]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sP + 2 * KB);
+  uint8_t* sK = sQ + 2 * KB;                           // [2 stages][2 k-blocks][8 KB]
+  uint8_t* sV = sK + 4 * KBK;                          // [2 stages][2 d-chunks][8 KB]
+  uint8_t* sP = sV + 4 * KBK;                          // [16 KB]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sP + KB);
   uint64_t *q_full = bars, *k_full = bars + 1, *k_empty = bars + 3, *v_full = bars + 5, *v_empty = bars + 7;
   uint64_t *s_full = bars + 9, *s_empty = bars + 11, *p_full = bars + 13, *p_empty = bars + 14, *o_done = bars + 15;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
   int* abort_flag = reinterpret_cast<int*>(tmem_slot + 1);
 
+  if (pad + 3 * KB + 8 * KBK + 16 * 8 + 16 > g.smem_bytes) {
+    if (threadIdx.x == 0) atomicExch(g.status, (int)SMARTMEM_ERR_UNSUPPORTED);
+    return;
+  }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // heaviest units (last query tiles) first
   const int bh_count = g.batch * g.heads;
   const int qt = g.n_qt - 1 - (int)(blockIdx.x / bh_count);
   const int bh = (int)(blockIdx.x % bh_count);
   const int b = bh / g.heads, h = bh - b * g.heads;
-  const int n_kv = qt + 1;
+  const int n_kv = min(2 * (qt + 1), (g.S + BKV - 1) / BKV);   // 64-key blocks up to and including the diagonal
   const long long row_base = (long long)b * g.row_per_batch + (long long)h * g.row_per_head;
 
   if (threadIdx.x == 0) {
@@ -118,12 +129,12 @@ causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         const int krow = (int)(row_base + (long long)j * BKV);
         ok = ptx::mbar_wait(&k_empty[s], ph ^ 1, abort_flag, g.status);
         if (!ok) break;
-        ptx::mbar_expect_tx(&k_full[s], 2 * KB);
-        for (int kb = 0; kb < 2; ++kb) ptx::tma_load_2d(sK + (s * 2 + kb) * KB, &tmK, &k_full[s], kc + kb * 64, krow);
+        ptx::mbar_expect_tx(&k_full[s], 2 * KBK);
+        for (int kb = 0; kb < 2; ++kb) ptx::tma_load_2d(sK + (s * 2 + kb) * KBK, &tmK, &k_full[s], kc + kb * 64, krow);
         ok = ptx::mbar_wait(&v_empty[s], ph ^ 1, abort_flag, g.status);
         if (!ok) break;
-        ptx::mbar_expect_tx(&v_full[s], 2 * KB);
-        for (int dc = 0; dc < 2; ++dc) ptx::tma_load_2d(sV + (s * 2 + dc) * KB, &tmV, &v_full[s], vc + dc * 64, krow);
+        ptx::mbar_expect_tx(&v_full[s], 2 * KBK);
+        for (int dc = 0; dc < 2; ++dc) ptx::tma_load_2d(sV + (s * 2 + dc) * KBK, &tmV, &v_full[s], vc + dc * 64, krow);
       }
     }
   } else if (warp == 1) {
@@ -139,7 +150,7 @@ causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         if (!ok) return;
         ptx::tc_fence_after();
         for (int kb = 0; kb < 2; ++kb) {
-          const uint32_t a0 = ptx::smem_u32(sQ + kb * KB), b0 = ptx::smem_u32(sK + (s * 2 + kb) * KB);
+          const uint32_t a0 = ptx::smem_u32(sQ + kb * KB), b0 = ptx::smem_u32(sK + (s * 2 + kb) * KBK);
           for (int k = 0; k < 4; ++k)
             ptx::tc_mma_bf16(tmem_base + TM_S + s * BKV, ptx::make_smem_desc(a0 + k * 32, 16, 1024),
                              ptx::make_smem_desc(b0 + k * 32, 16, 1024), idesc_s, (kb | k) ? 1u : 0u);
@@ -153,10 +164,10 @@ causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         ok = ok && ptx::mbar_wait(&v_full[s], (j >> 1) & 1, abort_flag, g.status);
         if (!ok) return;
         ptx::tc_fence_after();
-        const uint32_t p0 = ptx::smem_u32(sP), v0 = ptx::smem_u32(sV + s * 2 * KB);
-        for (int ks = 0; ks < 8; ++ks)                 // 16 keys per step
-          ptx::tc_mma_bf16(tmem_base + TM_O, ptx::make_smem_desc(p0 + (ks >> 2) * KB + (ks & 3) * 32, 16, 1024),
-                           ptx::make_smem_desc(v0 + ks * 2048, KB, 1024), idesc_pv, (j | ks) ? 1u : 0u);
+        const uint32_t p0 = ptx::smem_u32(sP), v0 = ptx::smem_u32(sV + s * 2 * KBK);
+        for (int ks = 0; ks < BKV / 16; ++ks)          // 16 keys per step: P +32 bytes, V +16 rows of 128 bytes; the two 64-wide d-chunks are KBK apart
+          ptx::tc_mma_bf16(tmem_base + TM_O, ptx::make_smem_desc(p0 + ks * 32, 16, 1024),
+                           ptx::make_smem_desc(v0 + ks * 2048, KBK, 1024), idesc_pv, (j | ks) ? 1u : 0u);
         ptx::tc_commit(&v_empty[s]);
         ptx::tc_commit(p_empty);
       };
@@ -180,21 +191,21 @@ causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       if (!ok) break;
       ptx::tc_fence_after();
       const uint32_t ts = tmem_base + TM_S + sb * BKV + lane_addr;
-      const bool diag = (j == qt);
+      const bool diag = (j >= 2 * qt);                 // the two 64-key blocks that straddle this tile's diagonal
       const int kj0 = j * BKV;
       // the whole score row of this thread: four loads in flight, one wait
-      uint32_t rv[128];
+      uint32_t rv[BKV];
 #pragma unroll
-      for (int ch = 0; ch < 4; ++ch) ptx::tmem_ld32(ts + ch * 32, rv + ch * 32);
+      for (int ch = 0; ch < BKV / 32; ++ch) ptx::tmem_ld32(ts + ch * 32, rv + ch * 32);
       ptx::tmem_ld_wait();
       float mx = -INFINITY;                            // row maximum (log2 domain)
       if (diag) {
 #pragma unroll
-        for (int c = 0; c < 128; ++c)
+        for (int c = 0; c < BKV; ++c)
           if (kj0 + c <= qi) mx = fmaxf(mx, __uint_as_float(rv[c]));
       } else {
 #pragma unroll
-        for (int c = 0; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(rv[c]));
+        for (int c = 0; c < BKV; ++c) mx = fmaxf(mx, __uint_as_float(rv[c]));
       }
       mx *= g.scale_log2;                              // the scale is positive
       float corr = 1.f;
@@ -206,10 +217,10 @@ causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         rescale = j > 0;
       }
       // p = 2^(s - m), packed to bf16 for the second MMA
-      uint32_t pk[64];
+      uint32_t pk[BKV / 2];
       float l0 = 0.f, l1 = 0.f;
 #pragma unroll
-      for (int c = 0; c < 128; c += 2) {
+      for (int c = 0; c < BKV; c += 2) {
         float p0 = ex2(fmaf(__uint_as_float(rv[c]), g.scale_log2, -m_used));
         float p1 = ex2(fmaf(__uint_as_float(rv[c + 1]), g.scale_log2, -m_used));
         if (diag) {
@@ -241,11 +252,11 @@ causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         }
         ptx::tmem_st_wait();
       }
-      // P row r: 16 chunks of 8 keys; chunk c8 lives in k-block c8 / 8 at position (c8 % 8) ^ (r % 8)
+      // P row r: 8 chunks of 8 keys; chunk c8 at position c8 ^ (r % 8) of the 128-byte row
 #pragma unroll
-      for (int c8 = 0; c8 < 16; ++c8) {
+      for (int c8 = 0; c8 < BKV / 8; ++c8) {
         const uint4 v4 = make_uint4(pk[c8 * 4 + 0], pk[c8 * 4 + 1], pk[c8 * 4 + 2], pk[c8 * 4 + 3]);
-        *reinterpret_cast<uint4*>(sP + (c8 >> 3) * KB + r * 128 + (((c8 & 7) ^ (r & 7)) << 4)) = v4;
+        *reinterpret_cast<uint4*>(sP + r * 128 + ((c8 ^ (r & 7)) << 4)) = v4;
       }
       ptx::fence_proxy_async();
       ptx::tc_fence_before();
@@ -306,15 +317,15 @@ int launch_causal_attention_tc(const CausalAttnArgs& a, cudaStream_t st) {
     // one [B*S, row pitch] matrix holds q, k and v side by side; columns are offsets from q
     const long long kcol = ((const char*)a.k.ptr - (const char*)a.q.ptr) / 2, vcol = ((const char*)a.v.ptr - (const char*)a.q.ptr) / 2;
     if (kcol < 0 || vcol < 0 || kcol + H * D > st_ || vcol + H * D > st_) return SMARTMEM_ERR_UNSUPPORTED;
-    if ((rc = tc_encode_2d(a.q.ptr, st_, B * S, st_, 64, 128, &tq)) != SMARTMEM_OK) return rc;
-    tk = tq;
-    tv = tq;
+    if ((rc = tc_encode_2d(a.q.ptr, st_, B * S, st_, 64, BQ, &tq)) != SMARTMEM_OK) return rc;
+    if ((rc = tc_encode_2d(a.q.ptr, st_, B * S, st_, 64, BKV, &tk)) != SMARTMEM_OK) return rc;   // same buffer, 64-row boxes
+    tv = tk;
     g.q_col0 = 0; g.k_col0 = (int)kcol; g.v_col0 = (int)vcol; g.col_per_head = D;
     g.row_per_batch = S; g.row_per_head = 0;
   } else if (head_major) {
     if ((rc = tc_encode_2d(a.q.ptr, D, B * H * S, D, 64, 128, &tq)) != SMARTMEM_OK) return rc;
-    if ((rc = tc_encode_2d(a.k.ptr, D, B * H * S, D, 64, 128, &tk)) != SMARTMEM_OK) return rc;
-    if ((rc = tc_encode_2d(a.v.ptr, D, B * H * S, D, 64, 128, &tv)) != SMARTMEM_OK) return rc;
+    if ((rc = tc_encode_2d(a.k.ptr, D, B * H * S, D, 64, BKV, &tk)) != SMARTMEM_OK) return rc;
+    if ((rc = tc_encode_2d(a.v.ptr, D, B * H * S, D, 64, BKV, &tv)) != SMARTMEM_OK) return rc;
     g.col_per_head = 0;
     g.row_per_batch = H * S; g.row_per_head = S;
   } else {
@@ -328,11 +339,15 @@ int launch_causal_attention_tc(const CausalAttnArgs& a, cudaStream_t st) {
   g.scale_log2 = a.scale * 1.4426950408889634f;
   g.status = device_status_ptr();
   if (!g.status) return SMARTMEM_ERR_CUDA;
-  const size_t smem = 1024 + 12 * KB + 16 * 8 + 16;
+  // 112 KB of tiles: two CTAs per SM only fit without a spare kilobyte of alignment slack (the kernel
+  // reports a misaligned base instead of overrunning)
+  const size_t smem = 3 * KB + 8 * KBK + 16 * 8 + 16;
+  g.smem_bytes = (uint32_t)smem;
   static bool configured = false;
   if (!configured) {
     if (cudaFuncSetAttribute(causal_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return SMARTMEM_ERR_CUDA;
+    cudaFuncSetAttribute(causal_attn_tc_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
     configured = true;
   }
   const long long ctas = (long long)g.n_qt * B * H;
