@@ -20,6 +20,16 @@
 #include "gemm_tc.cuh"
 #include "ptx.cuh"
 
+#ifdef CA_EXP_TIMING
+__device__ long long g_ca_dbg[8192];
+#define CDBG(slot) do { if (blockIdx.x == 0) g_ca_dbg[(slot)] = clock64(); } while (0)
+extern "C" __attribute__((visibility("default"))) int smartmem_debug_read_ca(long long* host, int n) {
+  return (int)cudaMemcpyFromSymbol(host, g_ca_dbg, sizeof(long long) * n);
+}
+#else
+#define CDBG(slot) do { } while (0)
+#endif
+
 namespace smartmem {
 namespace {
 
@@ -127,12 +137,15 @@ causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         const int s = j & 1;
         const uint32_t ph = (j >> 1) & 1;
         const int krow = (int)(row_base + (long long)j * BKV);
+        CDBG(j * 16 + 0);
         ok = ptx::mbar_wait(&k_empty[s], ph ^ 1, abort_flag, g.status);
         if (!ok) break;
+        CDBG(j * 16 + 1);
         ptx::mbar_expect_tx(&k_full[s], 2 * KBK);
         for (int kb = 0; kb < 2; ++kb) ptx::tma_load_2d(sK + (s * 2 + kb) * KBK, &tmK, &k_full[s], kc + kb * 64, krow);
         ok = ptx::mbar_wait(&v_empty[s], ph ^ 1, abort_flag, g.status);
         if (!ok) break;
+        CDBG(j * 16 + 2);
         ptx::mbar_expect_tx(&v_full[s], 2 * KBK);
         for (int dc = 0; dc < 2; ++dc) ptx::tma_load_2d(sV + (s * 2 + dc) * KBK, &tmV, &v_full[s], vc + dc * 64, krow);
       }
@@ -145,31 +158,42 @@ causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       auto issue_s = [&](int j) {
         const int s = j & 1;
         const uint32_t ph = (j >> 1) & 1;
+        CDBG(j * 16 + 3);
         ok = ok && ptx::mbar_wait(&s_empty[s], ph ^ 1, abort_flag, g.status);
+        CDBG(j * 16 + 4);
         ok = ok && ptx::mbar_wait(&k_full[s], ph, abort_flag, g.status);
         if (!ok) return;
+        CDBG(j * 16 + 5);
         ptx::tc_fence_after();
+#pragma unroll
         for (int kb = 0; kb < 2; ++kb) {
-          const uint32_t a0 = ptx::smem_u32(sQ + kb * KB), b0 = ptx::smem_u32(sK + (s * 2 + kb) * KBK);
-          for (int k = 0; k < 4; ++k)
-            ptx::tc_mma_bf16(tmem_base + TM_S + s * BKV, ptx::make_smem_desc(a0 + k * 32, 16, 1024),
-                             ptx::make_smem_desc(b0 + k * 32, 16, 1024), idesc_s, (kb | k) ? 1u : 0u);
+          const uint64_t ad = ptx::make_smem_desc(ptx::smem_u32(sQ + kb * KB), 16, 1024);
+          const uint64_t bd = ptx::make_smem_desc(ptx::smem_u32(sK + (s * 2 + kb) * KBK), 16, 1024);
+#pragma unroll
+          for (int k = 0; k < 4; ++k)                   // a k16 step moves both start addresses by 32 bytes
+            ptx::tc_mma_bf16(tmem_base + TM_S + s * BKV, ad + 2 * k, bd + 2 * k, idesc_s, (kb | k) ? 1u : 0u);
         }
         ptx::tc_commit(&k_empty[s]);
         ptx::tc_commit(&s_full[s]);
+        CDBG(j * 16 + 6);
       };
       auto issue_pv = [&](int j) {
         const int s = j & 1;
+        CDBG(j * 16 + 7);
         ok = ok && ptx::mbar_wait(p_full, j & 1, abort_flag, g.status);
+        CDBG(j * 16 + 8);
         ok = ok && ptx::mbar_wait(&v_full[s], (j >> 1) & 1, abort_flag, g.status);
         if (!ok) return;
+        CDBG(j * 16 + 9);
         ptx::tc_fence_after();
         const uint32_t p0 = ptx::smem_u32(sP), v0 = ptx::smem_u32(sV + s * 2 * KBK);
+        const uint64_t pd = ptx::make_smem_desc(p0, 16, 1024), vd = ptx::make_smem_desc(v0, KBK, 1024);
+#pragma unroll
         for (int ks = 0; ks < BKV / 16; ++ks)          // 16 keys per step: P +32 bytes, V +16 rows of 128 bytes; the two 64-wide d-chunks are KBK apart
-          ptx::tc_mma_bf16(tmem_base + TM_O, ptx::make_smem_desc(p0 + ks * 32, 16, 1024),
-                           ptx::make_smem_desc(v0 + ks * 2048, KBK, 1024), idesc_pv, (j | ks) ? 1u : 0u);
+          ptx::tc_mma_bf16(tmem_base + TM_O, pd + 2 * ks, vd + (2048 >> 4) * ks, idesc_pv, (j | ks) ? 1u : 0u);
         ptx::tc_commit(&v_empty[s]);
         ptx::tc_commit(p_empty);
+        CDBG(j * 16 + 10);
       };
       issue_s(0);
       for (int j = 0; j < n_kv && ok; ++j) {
@@ -187,8 +211,10 @@ causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     bool ok = true;
     for (int j = 0; j < n_kv && ok; ++j) {
       const int sb = j & 1;
+      if (warp == 2 && lane == 0) CDBG(j * 16 + 11);
       ok = ptx::mbar_wait(&s_full[sb], (j >> 1) & 1, abort_flag, g.status);
       if (!ok) break;
+      if (warp == 2 && lane == 0) CDBG(j * 16 + 12);
       ptx::tc_fence_after();
       const uint32_t ts = tmem_base + TM_S + sb * BKV + lane_addr;
       const bool diag = (j >= 2 * qt);                 // the two 64-key blocks that straddle this tile's diagonal
@@ -198,16 +224,16 @@ causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
 #pragma unroll
       for (int ch = 0; ch < BKV / 32; ++ch) ptx::tmem_ld32(ts + ch * 32, rv + ch * 32);
       ptx::tmem_ld_wait();
-      float mx = -INFINITY;                            // row maximum (log2 domain)
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // row maximum (log2 domain), four independent chains
       if (diag) {
 #pragma unroll
         for (int c = 0; c < BKV; ++c)
-          if (kj0 + c <= qi) mx = fmaxf(mx, __uint_as_float(rv[c]));
+          if (kj0 + c <= qi) mx4[c & 3] = fmaxf(mx4[c & 3], __uint_as_float(rv[c]));
       } else {
 #pragma unroll
-        for (int c = 0; c < BKV; ++c) mx = fmaxf(mx, __uint_as_float(rv[c]));
+        for (int c = 0; c < BKV; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], __uint_as_float(rv[c]));
       }
-      mx *= g.scale_log2;                              // the scale is positive
+      float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * g.scale_log2;   // the scale is positive
       float corr = 1.f;
       bool rescale = false;
       if (mx > m_used + kRescaleThreshold) {           // (first tile: m_used = -inf)
@@ -236,8 +262,10 @@ causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&s_empty[sb]);   // this warp has read its part of the S buffer
       // the previous P V must have completed before P is overwritten or O rescaled
+      if (warp == 2 && lane == 0) CDBG(j * 16 + 13);
       ok = ptx::mbar_wait(p_empty, (j & 1) ^ 1, abort_flag, g.status);
       if (!ok) break;
+      if (warp == 2 && lane == 0) CDBG(j * 16 + 14);
       ptx::tc_fence_after();
       if (__any_sync(0xFFFFFFFFu, rescale)) {
         const uint32_t to = tmem_base + TM_O + lane_addr;
@@ -262,6 +290,7 @@ causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(p_full);
+      if (warp == 2 && lane == 0) CDBG(j * 16 + 15);
     }
     if (ok) ok = ptx::mbar_wait(o_done, 0, abort_flag, g.status);
     if (ok) {
