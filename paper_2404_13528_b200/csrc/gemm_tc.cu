@@ -693,7 +693,7 @@ int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep,
   const int nkb = (int)((K + BK - 1) / BK);
   // 256 wide, short K: wider store rounds instead of a 4th stage.  Narrow tiles: their stages are
   // small, and a tile is consumed faster than a load's latency, so the ring runs several tiles ahead.
-  const int stages = bn == 256 ? (nkb <= 3 ? 3 : 4) : (bn <= 96 ? 6 : 4);
+  const int stages = bn == 256 ? (nkb <= 4 ? 3 : 4) : (bn <= 96 ? 6 : 4);
   GemmArgs g;
   memset(&g, 0, sizeof(g));
   CUtensorMap ta, tb;
