@@ -557,9 +557,15 @@ def main():
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        v, secs = oracle_tokens_per_s(w["B"])
-        cpu = {"value": v, "unit": UNIT, "cores": host_threads(), "kind": "oracle",
-               "sample": f"the whole workload once ({w['B']} images, {secs:.1f} s)"}
+        # the oracle on the whole workload, repeated until about 10 s of CPU work have been timed (at most 8 passes)
+        t_cpu, passes, toks = 0.0, 0, 0.0
+        while t_cpu < 10.0 and passes < 8:
+            v, secs = oracle_tokens_per_s(w["B"])
+            t_cpu += secs
+            toks += v * secs
+            passes += 1
+        cpu = {"value": toks / t_cpu, "unit": UNIT, "cores": host_threads(), "kind": "oracle",
+               "sample": f"the whole workload ({w['B']} images) {passes} times, {t_cpu:.1f} s of oracle time"}
 
     if rank == 0:
         tokens = M * world
