@@ -14,9 +14,17 @@
 // lies ([key, d] rows) through the MN-major operand mode.  Results are stored as whole 64-byte rows
 // at column h*32 of [M, C] (head merge eliminated) or into [nW, nH, T, d].
 //
-// Persistent CTAs keep one head (its relative-position bias sits in shared memory as a [T, T]
-// table) and stream window pairs through a 3-stage ring.  Two softmax groups of four warps
-// alternate over the units, each with its own S and O buffers in TMEM and its own P tile.
+// Persistent CTAs keep one head (its relative-position bias is expanded once into a [T, T] table of
+// bf16 pairs in shared memory, read with 16-byte loads) and stream window pairs through a 6-stage
+// ring.  Two softmax groups of four warps alternate over the units, each with its own S and O buffers
+// in TMEM and its own P tile.  S and P V have an issuing thread each: the S issuer runs ahead as far
+// as the S buffers and the ring allow, so a group finds its next score tile waiting when it has
+// written P.  The seam mask of shifted blocks is a 64-bit key mask per row, computed arithmetically
+// (a key is in another region iff it lies on the other side of the wrap line) and only for windows
+// in the last window row or column.
+//
+// What bounds it (clock-stamped build, -DWA_EXP_TIMING): the softmax groups, at about 1700 cycles
+// per window pair; the tensor pipe is busy for about 500 of them.
 #include "attn.cuh"
 #include "gemm_tc.cuh"
 #include "ptx.cuh"

@@ -1,18 +1,23 @@
 // Fused MLP half of a transformer block on tcgen05:
 //
-//   out = residual + GELU(A W1^T + b1) W2^T + b2,        A [M, C], W1 [hidden, C], W2 [C, hidden]
+//   out = residual + GELU(LN(A) W1^T + b1) W2^T + b2,     A [M, C], W1 [hidden, C], W2 [C, hidden]
 //
-// for narrow blocks (C <= 128), where the hidden activation [M, hidden] is four times larger than
-// everything else the block touches.  The hidden tensor never leaves the SM: per 128-row tile the
-// kernel walks over chunks of 128 hidden columns; fc1 of a chunk accumulates in TMEM, the epilogue
-// warps apply bias + GELU and write the chunk as bf16 straight into shared memory in the K-major
-// 128-byte-swizzled operand layout, and fc2 consumes it from there as its A operand while fc1 of
-// the next chunk is already running (two TMEM buffers for fc1, one accumulator for fc2).
+// for narrow blocks (C in {64, 96}), where the hidden activation [M, hidden] is four times larger
+// than everything else the block touches.  Neither the normalised rows nor the hidden tensor leave
+// the SM.  Per 128-row tile: the producer brings the raw rows in by TMA, four warps normalise them
+// in place (LayerNorm, a row per thread); then the kernel walks over chunks of 128 hidden columns:
+// fc1 of a chunk accumulates in TMEM, the GELU warps add the bias, apply GELU on packed bf16 pairs
+// and write the bf16 chunk back into the same TMEM buffer, and fc2 takes it from there as its A
+// operand (tensor memory) while fc1 of the next chunk is already running.  The output accumulator is
+// double-buffered in TMEM, so the output warps (bias, residual, row stores) overlap the next tile.
 //
-// Warp roles: warp 0 TMA producer (A tile double-buffered across tiles, weights streamed through a
-// ring: they stay L2-resident), warp 1 fc1 issuer + TMEM owner, warps 2-17 GELU (TMEM -> shared
-// memory), warps 18-21 output (OUT + b2 + residual -> global, OUT double-buffered in TMEM so they
-// overlap the next tile), warp 22 fc2 issuer.
+// Warp roles: 0 TMA producer (A tile double-buffered across tiles, weights streamed from L2 through
+// a 4-stage ring in the order the two issuers consume them), 1 fc1 issuer + TMEM owner, 2-17 GELU,
+// 18-21 output, 22 fc2 issuer, 23-26 LayerNorm.
+//
+// What bounds it (clock-stamped build, -DMLP_EXP_TIMING): the loop fc1(j) -> GELU(j) -> fc2(j) ->
+// fc1(j+2) over the two S1/H buffers, about 2500 cycles per chunk; the floor under that is the
+// special-function unit (tanh at 16 elements per clock per SM: about 1000 cycles per chunk).
 
 #include "gemm_tc.cuh"
 #include "ptx.cuh"

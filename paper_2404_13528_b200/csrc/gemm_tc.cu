@@ -9,11 +9,12 @@
 // NHWC case) is loaded as it lies and multiplied through the MN-major operand mode of the
 // tensor core, so that transpose disappears as well.
 //
-// Persistent CTAs (one per SM) of 10 warps: warp 0 issues TMA loads into a 4-stage shared-memory
-// ring, warp 1 owns the TMEM allocation and issues tcgen05.mma (one thread) into one of two
-// accumulator buffers, warps 2-9 run the epilogue of the previous tile meanwhile
-// (TMEM -> registers -> bias / GELU / RoPE / residual -> bf16 -> global, optionally scattering
-// rows through an index map: window reverse + reverse cyclic shift folded into the store).
+// Persistent CTAs (one per SM) of 19 warps: warp 0 issues TMA loads into a 3- to 6-stage shared-memory
+// ring (a second producer warp takes the B operand when the reduction is long), warp 1 owns the TMEM
+// allocation and issues tcgen05.mma (one thread) into one of two accumulator buffers, warps 2-17 run
+// the epilogue of the previous tile meanwhile (TMEM -> registers -> bias / GELU / RoPE / residual ->
+// bf16 -> staged whole-row stores, optionally scattering rows through an index map: window reverse +
+// reverse cyclic shift folded into the store).
 #include <mutex>
 #include <unordered_map>
 #include <string>
