@@ -42,7 +42,7 @@ constexpr int KB_BYTES = BM * BK * 2;              // one 128 x 64 bf16 operand 
 constexpr int NST = 4;                             // weight ring stages; one stage = both k-blocks of a chunk's W1 or W2
 constexpr int WST_BYTES = 2 * KB_BYTES;
 constexpr int kGeluWarps = 16, kOutWarps = 4, kNormWarps = 4, kThreads = 32 * (3 + kGeluWarps + kOutWarps + kNormWarps);
-constexpr uint32_t TM_S1 = 0, TM_OUT = 256, OUT_STRIDE = 128, TMEM_COLS = 512;
+constexpr uint32_t TM_S1 = 0, TM_OUT = 256, OUT_STRIDE = 96, TM_H = 448, TMEM_COLS = 512;   // S1 x2 (128), OUT x2 (96), H (64 packed columns)
 constexpr int SMEM_TILES = (4 + 2 * NST) * KB_BYTES;         // A (2 buffers), weight ring
 constexpr int N_BARS = 4 + 2 * NST + 2 + 2 + 2 + 4 + 2;
 
@@ -121,8 +121,8 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       ptx::mbar_init(&a_full[i], 1);
       ptx::mbar_init(&a_empty[i], 1);
       ptx::mbar_init(&s1_full[i], 1);
-      ptx::mbar_init(&s1_empty[i], 1);
-      ptx::mbar_init(&h_full[i], kGeluWarps);
+      ptx::mbar_init(&s1_empty[i], kGeluWarps);
+      ptx::mbar_init(&h_full[i], i == 0 ? kGeluWarps : 1);   // [0]: H written (GELU warps); [1]: H consumed (fc2 commit)
       ptx::mbar_init(&out_full[i], 1);
       ptx::mbar_init(&out_empty[i], kOutWarps);
       ptx::mbar_init(&a_ready[i], kNormWarps);
@@ -243,10 +243,10 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       int it2 = 0, c2 = 0;
       bool ok = true;
       for (int j = 0; j < total && ok; ++j) {
-        const uint32_t hb = j & 1, ob = it2 & 1;
+        const uint32_t ob = it2 & 1;
         const uint32_t n = j + 1 < total ? 2 * j + 2 : 2 * j + 1, ws = n % NST, wph = (n / NST) & 1;
         DBG(j * 16 + 4);
-        ok = ptx::mbar_wait(&h_full[hb], (j >> 1) & 1, abort_flag, g.status);
+        ok = ptx::mbar_wait(&h_full[0], j & 1, abort_flag, g.status);
         if (c2 == 0) ok = ok && ptx::mbar_wait(&out_empty[ob], ((it2 >> 1) & 1) ^ 1, abort_flag, g.status);
         DBG(j * 16 + 5);
         ok = ok && ptx::mbar_wait(&w_full[ws], wph, abort_flag, g.status);
@@ -254,14 +254,14 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         DBG(j * 16 + 6);
         ptx::tc_fence_after();
         const uint32_t d = tmem_base + TM_OUT + ob * OUT_STRIDE;
-        const uint32_t a = tmem_base + TM_S1 + hb * HC;     // H chunk: 128 bf16 per lane = 64 columns
+        const uint32_t a = tmem_base + TM_H;               // H chunk: 128 bf16 per lane = 64 columns
         const uint64_t bd = ptx::make_smem_desc(w_base + ws * WST_BYTES, 16, 1024);
         ptx::tc_mma_bf16_ta(d, a, bd, idesc2, c2 != 0 ? 1u : 0u);
 #pragma unroll
-        for (int k = 1; k < HC / 16; ++k)               // k-step k: GELU warp group k / 2 wrote it at column 32 (k / 2) + 8 (k % 2)
-          ptx::tc_mma_bf16_ta(d, a + 32 * (k >> 1) + 8 * (k & 1), bd + (k >> 2) * (KB_BYTES >> 4) + 2 * (k & 3), idesc2, 1u);
+        for (int k = 1; k < HC / 16; ++k)               // 16 hidden columns = 8 packed TMEM columns per step
+          ptx::tc_mma_bf16_ta(d, a + 8 * k, bd + (k >> 2) * (KB_BYTES >> 4) + 2 * (k & 3), idesc2, 1u);
         ptx::tc_commit(&w_empty[ws]);
-        ptx::tc_commit(&s1_empty[hb]);                  // H lived in the S1 buffer: fc1 may overwrite it now
+        ptx::tc_commit(&h_full[1]);                     // H consumed: the GELU warps may write the next chunk
         DBG(j * 16 + 7);
         if (++c2 == NC) {
           ptx::tc_commit(&out_full[ob]);
@@ -271,9 +271,10 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       }
     }
   } else if (warp < 2 + kGeluWarps) {
-    // GELU warps: S1 chunk (TMEM, fp32) -> + b1 -> GELU -> bf16 pairs -> back into the same TMEM
-    // buffer, where fc2 reads the chunk as its A operand.  Each warp overwrites the first 16 of the
-    // 32 columns it has just read (its own lanes), so no warp waits for another.
+    // GELU warps: S1 chunk (TMEM, fp32) -> + b1 -> GELU -> bf16 pairs -> the H region of TMEM, where
+    // fc2 reads the chunk as its A operand.  The S1 buffer is handed back as soon as it is in
+    // registers, so fc1 of chunk j+2 does not wait for fc2 of chunk j; H is single-buffered, and only
+    // its store waits for fc2 of the previous chunk.
     const int e = warp - 2, q = warp & 3, grp = e >> 2;
     bool ok = true;
     int c = 0;
@@ -289,6 +290,9 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         ptx::tc_fence_after();
         ptx::tmem_ld32(tq + grp * 32, rv);
         ptx::tmem_ld_wait();
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&s1_empty[sb]);
       }
       if (!ok) break;
       if (e == 0 && lane == 0) DBG(j * 16 + 10);
@@ -304,12 +308,15 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         pk[2 * v + 1] = gelu_tanh_bf16x2(__uint_as_float(rv[4 * v + 2]) + b4.z, __uint_as_float(rv[4 * v + 3]) + b4.w);
 #endif
       }
-      ptx::tmem_st16(tq + grp * 32, pk);               // over the first half of the columns this warp has just read
+      ok = ptx::mbar_wait(&h_full[1], (j & 1) ^ 1, abort_flag, g.status);   // fc2 of the previous chunk has read H
+      if (!ok) break;
+      ptx::tc_fence_after();
+      ptx::tmem_st16(tmem_base + TM_H + ((uint32_t)(q * 32) << 16) + grp * 16, pk);
       ptx::tmem_st_wait();
       if (e == 0 && lane == 0) DBG(j * 16 + 11);
       ptx::tc_fence_before();
       __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(&h_full[sb]);
+      if (lane == 0) ptx::mbar_arrive(&h_full[0]);
       if (++c == NC) c = 0;
     }
   } else if (warp < 2 + kGeluWarps + kOutWarps) {
