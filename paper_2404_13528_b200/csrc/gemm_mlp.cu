@@ -41,7 +41,7 @@ constexpr int BM = 128, BK = 64, HC = 128;         // tile rows, k-block, hidden
 constexpr int KB_BYTES = BM * BK * 2;              // one 128 x 64 bf16 operand block: 16 KB
 constexpr int NST = 4;                             // weight ring stages; one stage = both k-blocks of a chunk's W1 or W2
 constexpr int WST_BYTES = 2 * KB_BYTES;
-constexpr int kGeluWarps = 16, kOutWarps = 4, kNormWarps = 4, kThreads = 32 * (3 + kGeluWarps + kOutWarps + kNormWarps);
+constexpr int kGeluWarps = 8, kOutWarps = 4, kNormWarps = 4, kThreads = 32 * (3 + kGeluWarps + kOutWarps + kNormWarps);
 constexpr uint32_t TM_S1 = 0, TM_OUT = 256, OUT_STRIDE = 96, TM_H = 448, TMEM_COLS = 512;   // S1 x2 (128), OUT x2 (96), H (64 packed columns)
 constexpr int SMEM_TILES = (4 + 2 * NST) * KB_BYTES;         // A (2 buffers), weight ring
 constexpr int N_BARS = 4 + 2 * NST + 2 + 2 + 2 + 4 + 2;
@@ -275,30 +275,29 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     // fc2 reads the chunk as its A operand.  The S1 buffer is handed back as soon as it is in
     // registers, so fc1 of chunk j+2 does not wait for fc2 of chunk j; H is single-buffered, and only
     // its store waits for fc2 of the previous chunk.
-    const int e = warp - 2, q = warp & 3, grp = e >> 2;
+    const int e = warp - 2, q = warp & 3, hh = e >> 2;   // quadrant, half of the chunk's 128 columns
     bool ok = true;
     int c = 0;
     for (int j = 0; j < total && ok; ++j) {
       const uint32_t sb = j & 1;
-      const float4* bb4 = reinterpret_cast<const float4*>(b1_s + c * HC + grp * 32);   // this warp's 32 biases of the chunk: eight 16-byte broadcast reads
+      const float4* bb4 = reinterpret_cast<const float4*>(b1_s + c * HC + hh * 64);   // this warp's 64 biases of the chunk: 16-byte broadcast reads
       if (e == 0 && lane == 0) DBG(j * 16 + 8);
       ok = ptx::mbar_wait(&s1_full[sb], (j >> 1) & 1, abort_flag, g.status);
       if (e == 0 && lane == 0) DBG(j * 16 + 9);
-      const uint32_t tq = tmem_base + TM_S1 + sb * HC + ((uint32_t)(q * 32) << 16);
-      uint32_t rv[32];
-      if (ok) {
-        ptx::tc_fence_after();
-        ptx::tmem_ld32(tq + grp * 32, rv);
-        ptx::tmem_ld_wait();
-        ptx::tc_fence_before();
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(&s1_empty[sb]);
-      }
       if (!ok) break;
+      const uint32_t tq = tmem_base + TM_S1 + sb * HC + ((uint32_t)(q * 32) << 16) + hh * 64;
+      uint32_t rv[64];
+      ptx::tc_fence_after();
+      ptx::tmem_ld32(tq, rv);
+      ptx::tmem_ld32(tq + 32, rv + 32);
+      ptx::tmem_ld_wait();
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&s1_empty[sb]);
       if (e == 0 && lane == 0) DBG(j * 16 + 10);
-      uint32_t pk[16];
+      uint32_t pk[32];
 #pragma unroll
-      for (int v = 0; v < 8; ++v) {
+      for (int v = 0; v < 16; ++v) {
         const float4 b4 = bb4[v];
 #ifdef MLP_EXP_NOGELU
         pk[2 * v] = float2_to_bf16x2(__uint_as_float(rv[4 * v]) + b4.x, __uint_as_float(rv[4 * v + 1]) + b4.y);
@@ -311,7 +310,7 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       ok = ptx::mbar_wait(&h_full[1], (j & 1) ^ 1, abort_flag, g.status);   // fc2 of the previous chunk has read H
       if (!ok) break;
       ptx::tc_fence_after();
-      ptx::tmem_st16(tmem_base + TM_H + ((uint32_t)(q * 32) << 16) + grp * 16, pk);
+      ptx::tmem_st32(tmem_base + TM_H + ((uint32_t)(q * 32) << 16) + hh * 32, pk);
       ptx::tmem_st_wait();
       if (e == 0 && lane == 0) DBG(j * 16 + 11);
       ptx::tc_fence_before();
