@@ -17,7 +17,8 @@
 // Persistent CTAs keep one head (its relative-position bias is expanded once into a [T, T] table of
 // bf16 pairs in shared memory, read with 16-byte loads) and stream window pairs through a 6-stage
 // ring.  Two softmax groups of four warps alternate over the units, each with its own S and O buffers
-// in TMEM and its own P tile.  S and P V have an issuing thread each: the S issuer runs ahead as far
+// and its own P region in TMEM (P is written there as bf16 pairs and read by the second MMA as its
+// A operand: it never touches shared memory).  S and P V have an issuing thread each: the S issuer runs ahead as far
 // as the S buffers and the ring allow, so a group finds its next score tile waiting when it has
 // written P.  The seam mask of shifted blocks is a 64-bit key mask per row, computed arithmetically
 // (a key is in another region iff it lies on the other side of the wrap line) and only for windows
@@ -48,8 +49,7 @@ constexpr int D = 32, TP = 64;
 constexpr int OP_BYTES = 128 * 64;                    // one operand of a pair: 128 rows x 64 bytes
 constexpr int STAGE_BYTES = 3 * OP_BYTES;             // q, k, v
 constexpr int NSTAGE = 6;
-constexpr int P_BYTES = 2 * 128 * 128;                // P: 2 k-blocks of [128 rows x 128 bytes] (one per softmax group)
-constexpr uint32_t TM_S = 0, TM_O = 256, TMEM_COLS = 512;
+constexpr uint32_t TM_S = 0, TM_O = 256, TM_P = 320, TMEM_COLS = 512;   // S 2 x 128 columns, O 2 x 32, P 2 x 64 (128 keys as bf16 pairs)
 constexpr int BIAS_ROW = 36;                          // 32-bit words per bias row: 64 bf16 + pad, so that 16-byte row reads of
                                                       // eight consecutive threads fall into distinct banks
 constexpr int kSoftmaxWarps = 4, kGroups = 2, kLoaderWarps = 4;   // two softmax groups alternate over the units
@@ -88,8 +88,7 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
   uint8_t* sIn = smem;                                 // [NSTAGE][q, k, v][128 rows x 64 B]
-  uint8_t* sP = sIn + NSTAGE * STAGE_BYTES;            // [kGroups][2 k-blocks][128 x 128 B]
-  uint32_t* bias_s = reinterpret_cast<uint32_t*>(sP + kGroups * P_BYTES);   // [64][36]: bf16 pairs, 144-byte rows
+  uint32_t* bias_s = reinterpret_cast<uint32_t*>(sIn + NSTAGE * STAGE_BYTES);   // [64][36]: bf16 pairs, 144-byte rows
   int* lab_s = reinterpret_cast<int*>(bias_s + TP * BIAS_ROW);   // scratch: the head's raw table column (<= 256 bf16), then 4 key-mask words
   uint16_t* raw_s = reinterpret_cast<uint16_t*>(lab_s);
   uint32_t* kmask_s = reinterpret_cast<uint32_t*>(lab_s) + 128;
@@ -135,8 +134,8 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
   for (int i = tid; i < n_table && i < 256; i += kThreads) raw_s[i] = reinterpret_cast<const uint16_t*>(a.table)[i * a.heads + h];
   if (tid < TP) tyx_s[tid] = ((tid / ws) << 8) | (tid % ws);
   {
-    uint8_t* z0 = any_manual ? smem : sP;
-    const int zbytes = (any_manual ? NSTAGE * STAGE_BYTES : 0) + kGroups * P_BYTES;
+    uint8_t* z0 = smem;
+    const int zbytes = any_manual ? NSTAGE * STAGE_BYTES : 0;
     for (int i = tid; i < zbytes / 16; i += kThreads) reinterpret_cast<uint4*>(z0)[i] = make_uint4(0, 0, 0, 0);
   }
   __syncthreads();
@@ -224,13 +223,13 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
         if (!ok) break;
         WDBG(u * 16 + 3);
         ptx::tc_fence_after();
-        const uint32_t p0 = ptx::smem_u32(sP + ob * P_BYTES), v0 = ptx::smem_u32(sIn + s * STAGE_BYTES + 2 * OP_BYTES);
-        const uint64_t pd = ptx::make_smem_desc(p0, 16, 1024), vd = make_desc_sw64(v0, 16, 512);
-        const uint32_t od = tmem_base + TM_O + ob * D;
-        ptx::tc_mma_bf16(od, pd, vd, idesc_pv, 0u);
+        const uint32_t v0 = ptx::smem_u32(sIn + s * STAGE_BYTES + 2 * OP_BYTES);
+        const uint64_t vd = make_desc_sw64(v0, 16, 512);
+        const uint32_t od = tmem_base + TM_O + ob * D, pa = tmem_base + TM_P + ob * 64;
+        ptx::tc_mma_bf16_ta(od, pa, vd, idesc_pv, 0u);
 #pragma unroll
-        for (int ks = 1; ks < 8; ++ks)                 // 16 keys per step: P +32 bytes (next k-block: +16 KB), V +1024 bytes
-          ptx::tc_mma_bf16(od, pd + (ks >> 2) * ((128 * 128) >> 4) + (ks & 3) * 2, vd + ks * (1024 >> 4), idesc_pv, 1u);
+        for (int ks = 1; ks < 8; ++ks)                 // 16 keys per step: P +8 packed columns, V +1024 bytes
+          ptx::tc_mma_bf16_ta(od, pa + 8 * ks, vd + ks * (1024 >> 4), idesc_pv, 1u);
         ptx::tc_commit(&in_empty[s]);
         ptx::tc_commit(&p_empty[ob]);
         ptx::tc_commit(&o_full[ob]);
@@ -268,6 +267,13 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
     const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
     const int my_ty = tyx_s[i] >> 8, my_tx = tyx_s[i] & 255;
     const uint32_t* brow = bias_s + i * BIAS_ROW;
+    {                                                  // block-diagonal P: the other window's keys contribute nothing to this row
+      uint32_t zero[32];
+#pragma unroll
+      for (int c = 0; c < 32; ++c) zero[c] = 0u;
+      ptx::tmem_st32(tmem_base + TM_P + gi * 64 + lane_addr + (1 - w) * 32, zero);
+      ptx::tmem_st_wait();
+    }
     // keys below / right of the wrap line of a seam window (bit c = key c), and this row's own side
     const uint32_t ky_lo = kmask_s[0], ky_hi = kmask_s[1], kx_lo = kmask_s[2], kx_hi = kmask_s[3];
     const uint32_t my_fy = my_ty >= ws - a.shift ? 0xFFFFFFFFu : 0u, my_fx = my_tx >= ws - a.shift ? 0xFFFFFFFFu : 0u;
@@ -385,13 +391,11 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
       // previous P V must have completed before P is overwritten
       ok = ptx::mbar_wait(&p_empty[gi], ((u >> 1) & 1) ^ 1, abort_flag, g.status);
       if (!ok) break;
-      // P row r: its window's keys are columns w*64 .. w*64+63 = k-block w; chunk c8 at (c8 ^ (r % 8))
-#pragma unroll
-      for (int c8 = 0; c8 < 8; ++c8) {
-        const uint4 v4 = make_uint4(pk[c8 * 4 + 0], pk[c8 * 4 + 1], pk[c8 * 4 + 2], pk[c8 * 4 + 3]);
-        *reinterpret_cast<uint4*>(sP + gi * P_BYTES + w * (128 * 128) + r * 128 + ((c8 ^ (r & 7)) << 4)) = v4;
-      }
-      ptx::fence_proxy_async();
+      // P row r (bf16 pairs): its window's 64 keys are packed columns w*32 .. w*32+31 of the group's P region;
+      // the other window's half of the row was zeroed once and is never written
+      ptx::tc_fence_after();
+      ptx::tmem_st32(tmem_base + TM_P + gi * 64 + lane_addr + w * 32, pk);
+      ptx::tmem_st_wait();
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&p_full[gi]);
@@ -509,7 +513,7 @@ int launch_window_attention_tc(const WinAttnArgs& a_in, long long n_windows, cud
       g.tma_mask |= 1 << m;
     }
   }
-  const size_t smem = 1024 + NSTAGE * STAGE_BYTES + kGroups * P_BYTES + TP * BIAS_ROW * 4 + (2 * kGroups + 1) * TP * 4 +
+  const size_t smem = 1024 + NSTAGE * STAGE_BYTES + TP * BIAS_ROW * 4 + (2 * kGroups + 1) * TP * 4 +
                       (2 * NSTAGE + 12) * 8 + 16;
   static bool configured = false;
   if (!configured) {
