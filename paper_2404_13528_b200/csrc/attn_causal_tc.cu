@@ -3,13 +3,14 @@
 // One CTA = 128 query positions of one head.  K and V stream through shared memory in tiles of
 // 64 keys (TMA, double buffered); S = Q K^T and O += P V are tcgen05.mma with the accumulators in
 // TMEM (two S buffers, one O: 256 columns); four softmax warps own one query row per thread (the TMEM lane),
-// so row maxima and sums need no shuffles.  P goes back to the tensor core through shared memory in
-// the K-major swizzled operand layout; V is consumed as it lies in memory ([key, d] rows) through
-// the MN-major operand mode, so no transpose of V exists anywhere.  The running maximum is only
+// so row maxima and sums need no shuffles.  P goes back to the tensor core through tensor memory: it is
+// written as bf16 pairs over the S buffer it was computed from and read by the second MMA as its A
+// operand; V is consumed as it lies in memory ([key, d] rows) through the MN-major operand mode, so no
+// transpose of V exists anywhere.  The running maximum is only
 // refreshed when it grows by more than 2^8 (then O and the running sum are rescaled), which keeps
 // the TMEM read-modify-write of O off the common path.
 //
-// The 64-key tiles keep a CTA at 112 KB of shared memory and 256 TMEM columns, so TWO CTAs share an
+// The 64-key tiles keep a CTA at 96 KB of shared memory and 256 TMEM columns, so TWO CTAs share an
 // SM: while one is in its softmax (which is bound by the exponential unit) the other one's MMAs
 // run, which a single CTA with one softmax group could not overlap.
 //
@@ -66,14 +67,13 @@ causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   uint8_t* sQ = smem;                                  // [2 k-blocks][16 KB]
   uint8_t* sK = sQ + 2 * KB;                           // [2 stages][2 k-blocks][8 KB]
   uint8_t* sV = sK + 4 * KBK;                          // [2 stages][2 d-chunks][8 KB]
-  uint8_t* sP = sV + 4 * KBK;                          // [16 KB]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sP + KB);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sV + 4 * KBK);
   uint64_t *q_full = bars, *k_full = bars + 1, *k_empty = bars + 3, *v_full = bars + 5, *v_empty = bars + 7;
   uint64_t *s_full = bars + 9, *s_empty = bars + 11, *p_full = bars + 13, *p_empty = bars + 14, *o_done = bars + 15;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
   int* abort_flag = reinterpret_cast<int*>(tmem_slot + 1);
 
-  if (pad + 3 * KB + 8 * KBK + 16 * 8 + 16 > g.smem_bytes) {
+  if (pad + 2 * KB + 8 * KBK + 16 * 8 + 16 > g.smem_bytes) {
     if (threadIdx.x == 0) atomicExch(g.status, (int)SMARTMEM_ERR_UNSUPPORTED);
     return;
   }
@@ -94,7 +94,7 @@ causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       ptx::mbar_init(&v_full[i], 1);
       ptx::mbar_init(&v_empty[i], 1);
       ptx::mbar_init(&s_full[i], 1);
-      ptx::mbar_init(&s_empty[i], 4);
+      ptx::mbar_init(&s_empty[i], 1);                 // P(j) lives in S buffer j & 1: freed by the commit of P V (j)
     }
     ptx::mbar_init(p_full, 4);
     ptx::mbar_init(p_empty, 1);
@@ -175,12 +175,14 @@ causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         if (!ok) return;
         CDBG(j * 16 + 9);
         ptx::tc_fence_after();
-        const uint32_t p0 = ptx::smem_u32(sP), v0 = ptx::smem_u32(sV + s * 2 * KBK);
-        const uint64_t pd = ptx::make_smem_desc(p0, 16, 1024), vd = ptx::make_smem_desc(v0, KBK, 1024);
+        const uint32_t v0 = ptx::smem_u32(sV + s * 2 * KBK);
+        const uint64_t vd = ptx::make_smem_desc(v0, KBK, 1024);
+        const uint32_t pa = tmem_base + TM_S + s * BKV;  // P(j): bf16 pairs over the first 32 columns of the S buffer it came from
 #pragma unroll
-        for (int ks = 0; ks < BKV / 16; ++ks)          // 16 keys per step: P +32 bytes, V +16 rows of 128 bytes; the two 64-wide d-chunks are KBK apart
-          ptx::tc_mma_bf16(tmem_base + TM_O, pd + 2 * ks, vd + (2048 >> 4) * ks, idesc_pv, (j | ks) ? 1u : 0u);
+        for (int ks = 0; ks < BKV / 16; ++ks)          // 16 keys per step: P +8 packed columns, V +16 rows of 128 bytes; the two 64-wide d-chunks are KBK apart
+          ptx::tc_mma_bf16_ta(tmem_base + TM_O, pa + 8 * ks, vd + (2048 >> 4) * ks, idesc_pv, (j | ks) ? 1u : 0u);
         ptx::tc_commit(&v_empty[s]);
+        ptx::tc_commit(&s_empty[s]);
         ptx::tc_commit(p_empty);
         CDBG(j * 16 + 10);
       };
@@ -247,35 +249,29 @@ causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         pk[c / 2] = float2_to_bf16x2(p0, p1);
       }
       l += l0 + l1;
-      ptx::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(&s_empty[sb]);   // this warp has read its part of the S buffer
-      // the previous P V must have completed before P is overwritten or O rescaled
-      if (warp == 2 && lane == 0) CDBG(j * 16 + 13);
-      ok = ptx::mbar_wait(p_empty, (j & 1) ^ 1, abort_flag, g.status);
-      if (!ok) break;
-      if (warp == 2 && lane == 0) CDBG(j * 16 + 14);
-      ptx::tc_fence_after();
       if (__any_sync(0xFFFFFFFFu, rescale)) {
+        // O is rescaled in place: the previous P V, which accumulates into it, must have completed
+        if (warp == 2 && lane == 0) CDBG(j * 16 + 13);
+        ok = ptx::mbar_wait(p_empty, (j & 1) ^ 1, abort_flag, g.status);
+        if (!ok) break;
+        if (warp == 2 && lane == 0) CDBG(j * 16 + 14);
+        ptx::tc_fence_after();
         const uint32_t to = tmem_base + TM_O + lane_addr;
 #pragma unroll 1
         for (int ch = 0; ch < 4; ++ch) {
-          uint32_t rv[32];
-          ptx::tmem_ld32(to + ch * 32, rv);
+          uint32_t ro[32];
+          ptx::tmem_ld32(to + ch * 32, ro);
           ptx::tmem_ld_wait();
 #pragma unroll
-          for (int c = 0; c < 32; ++c) rv[c] = __float_as_uint(__uint_as_float(rv[c]) * (rescale ? corr : 1.f));
-          ptx::tmem_st32(to + ch * 32, rv);
+          for (int c = 0; c < 32; ++c) ro[c] = __float_as_uint(__uint_as_float(ro[c]) * (rescale ? corr : 1.f));
+          ptx::tmem_st32(to + ch * 32, ro);
         }
         ptx::tmem_st_wait();
       }
-      // P row r: 8 chunks of 8 keys; chunk c8 at position c8 ^ (r % 8) of the 128-byte row
-#pragma unroll
-      for (int c8 = 0; c8 < BKV / 8; ++c8) {
-        const uint4 v4 = make_uint4(pk[c8 * 4 + 0], pk[c8 * 4 + 1], pk[c8 * 4 + 2], pk[c8 * 4 + 3]);
-        *reinterpret_cast<uint4*>(sP + r * 128 + ((c8 ^ (r & 7)) << 4)) = v4;
-      }
-      ptx::fence_proxy_async();
+      // P row r (bf16 pairs) over the first 32 columns of the S buffer this thread has just read: each
+      // warp touches only its own lanes, and the buffer is not reused before P V (j) has completed
+      ptx::tmem_st32(ts, pk);
+      ptx::tmem_st_wait();
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(p_full);
@@ -359,7 +355,7 @@ int launch_causal_attention_tc(const CausalAttnArgs& a, cudaStream_t st) {
   if (!g.status) return SMARTMEM_ERR_CUDA;
   // 112 KB of tiles: two CTAs per SM only fit without a spare kilobyte of alignment slack (the kernel
   // reports a misaligned base instead of overrunning)
-  const size_t smem = 3 * KB + 8 * KBK + 16 * 8 + 16;
+  const size_t smem = 2 * KB + 8 * KBK + 16 * 8 + 16;
   g.smem_bytes = (uint32_t)smem;
   static bool configured = false;
   if (!configured) {
