@@ -88,3 +88,17 @@ def rope(x: np.ndarray, theta: float) -> np.ndarray:
     c, sn = np.cos(phi), np.sin(phi)
     a, b = x[..., :half], x[..., half:]
     return np.concatenate([a * c - b * sn, b * c + a * sn], axis=-1)
+
+
+def rope_at(x: np.ndarray, pos: int, theta: float) -> np.ndarray:
+    """Rotary embedding of vectors [.., D] that all sit at one position `pos` (the decode step of a
+    decoder layer): same pairing and frequencies as `rope`, angle phi_i = pos * theta^(-2i/D)."""
+    D = x.shape[-1]
+    half = D // 2
+    out = np.empty_like(x)
+    for i in range(half):
+        phi = float(pos) * theta ** (-(2.0 * i) / D)
+        c, sn = np.cos(phi), np.sin(phi)
+        out[..., i] = x[..., i] * c - x[..., i + half] * sn
+        out[..., i + half] = x[..., i + half] * c + x[..., i] * sn
+    return out

@@ -269,3 +269,60 @@ def test_attn_layer_against_direct_restatement():
     v = (xn @ p["w_qkv"].T)[:, 2 * hidden:]
     pm = np.cumsum(v, 0) / np.arange(1, S + 1)[:, None]
     assert np.allclose(y0[0], pm @ p["w_o"].T, atol=1e-10)
+
+
+def test_rope_at_pins():
+    """One-position rotary: equals row `pos` of the sequence form, is the identity at position 0,
+    and for D = 2 is the plane rotation by `pos` radians (frequency theta^0 = 1)."""
+    x = rng.standard_normal((3, 5, 16))
+    for pos in (0, 1, 4):
+        assert np.allclose(ops.rope_at(x[:, pos], pos, 10000.0), ops.rope(x, 10000.0)[:, pos], atol=1e-13)
+    assert np.allclose(ops.rope_at(x[:, 2], 0, 10000.0), x[:, 2])
+    r = ops.rope_at(np.array([[1.0, 0.0]]), 3, 10000.0)
+    assert np.allclose(r, [[np.cos(3.0), np.sin(3.0)]], atol=1e-15)
+
+
+def test_decode_step_equals_the_last_row_of_the_prefill():
+    """A decode step on the cache that a prefill of the first S-1 tokens leaves must give row S-1 of the
+    prefill over all S tokens (causal attention: the earlier rows never see the last token), and the
+    appended key / value must be that prefill's row S-1."""
+    S, heads, D, B = 7, 2, 8, 2
+    hidden = heads * D
+    x = rng.standard_normal((B, S, hidden))
+    p = {"rms_g": 1 + 0.1 * rng.standard_normal(hidden), "w_qkv": 0.3 * rng.standard_normal((3 * hidden, hidden)),
+         "w_o": 0.3 * rng.standard_normal((hidden, hidden))}
+    kc, vc, full, keeps = [], [], [], []
+    for b in range(B):
+        keep = {}
+        full.append(llama.attn_layer(x[b:b + 1], p, heads=heads, head_dim=D, add_residual=True, keep=keep)[0])
+        keeps.append(keep)
+        kc.append(np.transpose(keep["k"][:, :S - 1], (1, 0, 2)))     # [S-1,H,D]
+        vc.append(np.transpose(keep["v"][:, :S - 1], (1, 0, 2)))
+    y, kn, vn = llama.decode_step(x[:, S - 1], np.stack(kc), np.stack(vc), p, heads=heads, head_dim=D, add_residual=True)
+    for b in range(B):
+        assert np.allclose(y[b], full[b][S - 1], atol=1e-11)
+        assert np.allclose(kn[b], keeps[b]["k"][:, S - 1], atol=1e-12)
+        assert np.allclose(vn[b], keeps[b]["v"][:, S - 1], atol=1e-12)
+
+
+def test_decode_step_special_cases():
+    """Empty cache: softmax over one position is 1, so y = w_o v_new (+ x).  q-weights zero: uniform
+    attention, so the attended value is the mean of the cached and the new values."""
+    heads, D, B, pos = 2, 4, 3, 5
+    hidden = heads * D
+    x = rng.standard_normal((B, hidden))
+    p = {"rms_g": 1 + 0.1 * rng.standard_normal(hidden), "w_qkv": 0.3 * rng.standard_normal((3 * hidden, hidden)),
+         "w_o": 0.3 * rng.standard_normal((hidden, hidden))}
+    xn = x * p["rms_g"] / np.sqrt((x ** 2).mean(-1, keepdims=True) + 1e-5)
+    v_new = (xn @ p["w_qkv"].T)[:, 2 * hidden:]
+    empty = np.zeros((B, 0, heads, D))
+    y, _, vn = llama.decode_step(x, empty, empty, p, heads=heads, head_dim=D)
+    assert np.allclose(vn.reshape(B, hidden), v_new, atol=1e-12)
+    assert np.allclose(y, v_new @ p["w_o"].T, atol=1e-11)
+    p0 = dict(p)
+    p0["w_qkv"] = p["w_qkv"].copy()
+    p0["w_qkv"][:hidden] = 0
+    kc, vc = rng.standard_normal((B, pos, heads, D)), rng.standard_normal((B, pos, heads, D))
+    y0, _, _ = llama.decode_step(x, kc, vc, p0, heads=heads, head_dim=D, add_residual=True)
+    mean_v = (vc.reshape(B, pos, hidden).sum(1) + v_new) / (pos + 1)
+    assert np.allclose(y0, x + mean_v @ p["w_o"].T, atol=1e-11)
