@@ -250,6 +250,30 @@ int smartmem_attn_layer_workspace_bytes(const smartmem_attn_params_t* p, int32_t
 int smartmem_attn_layer(const smartmem_attn_params_t* p, const void* x, void* y, void* workspace,
                         size_t workspace_bytes, int32_t mode, void* cuda_stream);
 
+/* One decode step of the same layer against a key/value cache (the decode-time form of the chain
+ * of Section 2 / Fig. 1: the Concat that appends the new key and value, the head split and the
+ * head merge are Fixed-output layout operators of Table 3 and are eliminated; Section 3.2.2's
+ * "sub-optimal write" placement puts the append on the producer's store).
+ *
+ * B independent sequences, each holding `pos` cached positions (0 <= pos < S_max); the new token of
+ * each sits at position pos.  x, y: [B,hidden] bf16 (device), x != y.  p->S is S_max, p->causal is
+ * ignored (the last row of a causal mask is all-true), other fields as for smartmem_attn_layer.
+ * k_cache, v_cache (device, bf16, 16-byte aligned, owned by the caller, updated in place: row pos
+ * of every sequence is written, rows [0,pos) are read, nothing else is touched); keys are stored
+ * rotated.  Their layout depends on the mode, because the layout IS the point:
+ *   SMARTMEM_ELIMINATE  [B, S_max, heads, head_dim]  -- the layout the QKV GEMM produces: its
+ *       epilogue rotates q and k at position pos and stores the k and v columns of row b straight
+ *       into cache row (b, pos); attention reads head h as a strided slice and writes its output at
+ *       column h*head_dim of [B,hidden].  No copy kernel runs.
+ *   SMARTMEM_EXPLICIT   [B, heads, S_max, head_dim]  -- the per-head layout of the materialised
+ *       chain: plain QKV GEMM, head-split copy, stand-alone rotary pass, append copy into the cache,
+ *       attention on contiguous per-head tensors.
+ * head_dim must be 128, hidden a multiple of 256, pos + 1 <= 16384; otherwise
+ * SMARTMEM_ERR_UNSUPPORTED.  Errors as for smartmem_attn_layer. */
+int smartmem_attn_decode_workspace_bytes(const smartmem_attn_params_t* p, int32_t mode, size_t* bytes);
+int smartmem_attn_decode(const smartmem_attn_params_t* p, int32_t pos, const void* x, void* k_cache, void* v_cache,
+                         void* y, void* workspace, size_t workspace_bytes, int32_t mode, void* cuda_stream);
+
 /* Synchronises the stream and returns the device status word (SMARTMEM_OK, _TIMEOUT or _BOUNDS)
  * in *status, then clears it. */
 int smartmem_last_device_status(void* cuda_stream, int32_t* status);

@@ -62,7 +62,7 @@ EXPORTED = [
     "smartmem_plan_num_steps", "smartmem_plan_get_map", "smartmem_plan_output_desc",
     "smartmem_plan_workspace_bytes", "smartmem_map_eval", "smartmem_plan_eval_sequential", "smartmem_run_chain",
     "smartmem_swin_block_workspace_bytes", "smartmem_swin_block", "smartmem_attn_layer_workspace_bytes",
-    "smartmem_attn_layer", "smartmem_swin_block_timed", "smartmem_swin_block_static_scratch_bytes",
+    "smartmem_attn_layer", "smartmem_attn_decode_workspace_bytes", "smartmem_attn_decode", "smartmem_swin_block_timed", "smartmem_swin_block_static_scratch_bytes",
     "smartmem_swin_block_noalloc", "smartmem_profile_begin", "smartmem_profile_end", "smartmem_last_device_status", "smartmem_launch_count", "smartmem_status_string",
 ]
 
@@ -100,6 +100,8 @@ def lib() -> C.CDLL:
         "smartmem_swin_block_noalloc": (C.c_int, [P(SwinParams), vp, vp, i32, vp]),
         "smartmem_attn_layer_workspace_bytes": (C.c_int, [P(AttnParams), i32, P(C.c_size_t)]),
         "smartmem_attn_layer": (C.c_int, [P(AttnParams), vp, vp, vp, C.c_size_t, i32, vp]),
+        "smartmem_attn_decode_workspace_bytes": (C.c_int, [P(AttnParams), i32, P(C.c_size_t)]),
+        "smartmem_attn_decode": (C.c_int, [P(AttnParams), i32, vp, vp, vp, vp, vp, C.c_size_t, i32, vp]),
         "smartmem_profile_begin": (C.c_int, []),
         "smartmem_profile_end": (C.c_int, [vp, P(C.c_float), C.c_char_p, i32, i32, P(i32)]),
         "smartmem_last_device_status": (C.c_int, [vp, P(i32)]),
@@ -267,6 +269,18 @@ def smartmem_attn_layer_workspace_bytes(p: AttnParams, mode: int) -> int:
 
 def smartmem_attn_layer(p: AttnParams, x: int, y: int, workspace: int, workspace_bytes: int, mode: int, stream: int):
     _check(lib().smartmem_attn_layer(C.byref(p), x, y, workspace, workspace_bytes, mode, stream), "smartmem_attn_layer")
+
+
+def smartmem_attn_decode_workspace_bytes(p: AttnParams, mode: int) -> int:
+    n = C.c_size_t()
+    _check(lib().smartmem_attn_decode_workspace_bytes(C.byref(p), mode, C.byref(n)), "smartmem_attn_decode_workspace_bytes")
+    return n.value
+
+
+def smartmem_attn_decode(p: AttnParams, pos: int, x: int, k_cache: int, v_cache: int, y: int, workspace: int,
+                         workspace_bytes: int, mode: int, stream: int):
+    _check(lib().smartmem_attn_decode(C.byref(p), pos, x, k_cache, v_cache, y, workspace, workspace_bytes, mode, stream),
+           "smartmem_attn_decode")
 
 
 def smartmem_profile_begin():

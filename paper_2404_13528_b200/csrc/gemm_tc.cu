@@ -58,8 +58,11 @@ struct GemmArgs {
   const __nv_bfloat16* bias;
   const __nv_bfloat16* residual;
   int gelu, has_rowmap;
-  int rope_cols, rope_S;                 // columns [0, rope_cols) are rotated; position = row % rope_S
+  int rope_cols, rope_S, rope_pos0;      // columns [0, rope_cols) are rotated; position = rope_pos0 + row % rope_S
   float rope_c;                          // log2(theta) / 64
+  int seg_cols;                          // > 0: column segment s of a row goes to seg_out[s] + row * seg_ld[s]
+  __nv_bfloat16* seg_out[3];
+  long long seg_ld[3];
   int* status;
   DevMap rowmap;
 };
@@ -300,12 +303,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       // one round per tile the offset and the residual of the NEXT tile were requested during the
       // previous iteration, so neither the map evaluation nor the gather's latency is on the path
       // between the accumulator becoming ready and its buffer being handed back.
+      // column-segmented output: a tile never straddles segments (seg_cols is a multiple of BN), so
+      // the whole tile has one base and one pitch; the base is biased by the segment's first column
+      __nv_bfloat16* out_t = g.out;
+      long long ld_t = g.ldc;
+      if (g.seg_cols > 0) {
+        const int sg = n0 / g.seg_cols;
+        out_t = g.seg_out[sg] - (long long)sg * g.seg_cols;
+        ld_t = g.seg_ld[sg];
+      }
       long long off;
       if (PREFETCH_NEXT && it > 0) {
         off = off_next;
       } else {
         off = 0;
-        if (row_ok) off = g.has_rowmap ? devmap_eval_unrolled(g.rowmap, (uint32_t)row) : (long long)row * g.ldc;
+        if (row_ok) off = g.has_rowmap ? devmap_eval_unrolled(g.rowmap, (uint32_t)row) : (long long)row * ld_t;
         off += (long long)batch * g.out_batch_stride;
       }
       const __nv_bfloat16* __restrict__ rrow = g.residual ? g.residual + off : nullptr;
@@ -369,7 +381,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             // angle = position * theta^(-i/64), reduced mod 2 pi in two steps, then the hardware
             // sine / cosine: no table traffic (a [S, 64] table read 16 bytes per lane per row
             // slowed the whole kernel by a fifth)
-            const float pos = (float)(row_ok ? row % g.rope_S : 0);
+            const float pos = (float)(row_ok ? g.rope_pos0 + row % g.rope_S : 0);
             const int i0 = (grp & 1) * 32 + RC * (rd % RH);
 #pragma unroll
             for (int j = 0; j < RC; ++j) {
@@ -436,7 +448,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const long long roff = __shfl_sync(0xFFFFFFFFu, off, rr);
             const int rok = __shfl_sync(0xFFFFFFFFu, (int)row_ok, rr);
             const uint4 pk = *reinterpret_cast<const uint4*>(stage + rr * STG_ROW + seg * 16);
-            if (rok && n0 + c0 + seg * 8 + 8 <= g.N) *reinterpret_cast<uint4*>(g.out + roff + n0 + c0 + seg * 8) = pk;
+            if (rok && n0 + c0 + seg * 8 + 8 <= g.N) *reinterpret_cast<uint4*>(out_t + roff + n0 + c0 + seg * 8) = pk;
           }
           __syncwarp();
         }
@@ -458,7 +470,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           const long long roff = __shfl_sync(0xFFFFFFFFu, off, rr);
           const int rok = __shfl_sync(0xFFFFFFFFu, (int)row_ok, rr);
           const uint4 pk = *reinterpret_cast<const uint4*>(qstage + rr * QROW + seg * 16);
-          if (rok && n0 + seg * 8 + 8 <= g.N) *reinterpret_cast<uint4*>(g.out + roff + n0 + seg * 8) = pk;
+          if (rok && n0 + seg * 8 + 8 <= g.N) *reinterpret_cast<uint4*>(out_t + roff + n0 + seg * 8) = pk;
         }
         asm volatile("bar.sync %0, 128;" ::"r"(1 + q) : "memory");
         if (warp == 2 && lane == 0) GDBG(it * 16 + 11);
@@ -691,6 +703,11 @@ int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep,
   else if (N % 96 == 0) bn = 96;
   else if (N % 64 == 0) bn = 64;
   if (ep.rope_cols > 0 && (N % 256 || ep.rope_cols % 256 || ep.rope_S < 1)) return SMARTMEM_ERR_UNSUPPORTED;
+  if (ep.seg_cols > 0) {
+    if (ep.seg_cols % 256 || N > 3ll * ep.seg_cols || ep.rowmap || ep.residual || batch != 1) return SMARTMEM_ERR_UNSUPPORTED;
+    for (int i = 0; i * (long long)ep.seg_cols < N; ++i)
+      if (!ep.seg_out[i] || ((uintptr_t)ep.seg_out[i] & 15) || ep.seg_ld[i] % 8) return SMARTMEM_ERR_ALIGNMENT;
+  }
   const int nkb = (int)((K + BK - 1) / BK);
   // 256 wide, short K: wider store rounds instead of a 4th stage.  Narrow tiles: their stages are
   // small, and a tile is consumed faster than a load's latency, so the ring runs several tiles ahead.
@@ -713,6 +730,9 @@ int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep,
   if (ep.rowmap) g.rowmap = *ep.rowmap;
   g.rope_cols = ep.rope_cols;
   g.rope_S = ep.rope_S;
+  g.rope_pos0 = ep.rope_pos0;
+  g.seg_cols = ep.seg_cols;
+  for (int i = 0; i < 3; ++i) { g.seg_out[i] = (__nv_bfloat16*)ep.seg_out[i]; g.seg_ld[i] = ep.seg_ld[i]; }
   g.rope_c = ep.rope_log2_theta / 64.0f;
   g.status = device_status_ptr();
   if (!g.status) return SMARTMEM_ERR_CUDA;

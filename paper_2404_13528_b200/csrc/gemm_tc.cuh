@@ -26,8 +26,15 @@ struct TcEpilogue {
   const void* residual;      // same addressing as out, or null
   int gelu;
   const DevMap* rowmap;      // output row -> element offset, or null
-  int rope_cols, rope_S;     // rotate columns [0, rope_cols) in 128-wide heads; position = row % rope_S
+  int rope_cols, rope_S;     // rotate columns [0, rope_cols) in 128-wide heads; position = rope_pos0 + row % rope_S
   float rope_log2_theta;     // angle of pair i at position p: p * 2^(-i/64 * rope_log2_theta)
+  int rope_pos0;
+  // Column-segmented output (seg_cols > 0, a multiple of 256; no rowmap, residual or batch): columns
+  // [s*seg_cols, (s+1)*seg_cols) of row r go to seg_out[s] + r*seg_ld[s] (elements), s < 3.  `out`
+  // and `ldc` are ignored.  Lets one GEMM store into several destinations of different pitch.
+  int seg_cols;
+  void* seg_out[3];
+  long long seg_ld[3];
 };
 
 int tc_operand_from_map(const smartmem_index_map_t& m, int n_batch_atoms, int n_row_atoms, const void* ptr,

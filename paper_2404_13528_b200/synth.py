@@ -144,6 +144,18 @@ def attn_layer_inputs(config_id: int, S: int, hidden: int, dtype: str = "bf16", 
     }
 
 
+def decode_inputs(config_id: int, B: int, pos: int, hidden: int, heads: int, dtype: str = "bf16") -> dict:
+    """Tensors of one decode step of the decoder attention layer: the layer's weights, one new token per
+    sequence and a key/value cache of `pos` positions, logical shape [B, pos, heads, head_dim] (unit-variance
+    values, like the keys and values a prefill of unit-variance activations leaves)."""
+    seed = SEED_BASE + config_id
+    d = attn_layer_inputs(config_id, 1, hidden, dtype, B)
+    d["x"] = d["x"].reshape(B, hidden)
+    d["k_cache"] = normal(seed, 4, (B, pos, heads, hidden // heads), 1.0, 0.0, dtype)
+    d["v_cache"] = normal(seed, 5, (B, pos, heads, hidden // heads), 1.0, 0.0, dtype)
+    return d
+
+
 def chain_inputs(config_id: int, which: str, dtype: str = "bf16", small: bool = False) -> dict:
     """Inputs of the pure layout chains.
 
