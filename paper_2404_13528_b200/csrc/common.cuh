@@ -1,5 +1,6 @@
 // Shared device/host helpers of the CUDA path.
 #pragma once
+#include <cstdlib>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -33,7 +34,9 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  // SMARTMEM_NO_PDL=1 launches every kernel with ordinary stream ordering (for measuring what the overlap buys)
+  static const int allow = [] { const char* e = getenv("SMARTMEM_NO_PDL"); return (e && e[0] == '1') ? 0 : 1; }();
+  attr[0].val.programmaticStreamSerializationAllowed = allow;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);

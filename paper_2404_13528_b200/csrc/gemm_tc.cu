@@ -702,6 +702,9 @@ int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep,
   else if (N % 128 == 0) bn = 128;
   else if (N % 96 == 0) bn = 96;
   else if (N % 64 == 0) bn = 64;
+  // One row tile only (a decode step: M <= 128) and few wide column tiles: the GEMM streams the weight
+  // once and is bound by how many SMs pull on it, so take the narrowest tile that divides N.
+  if (ep.rope_cols == 0 && batch == 1 && M <= BM && !a_mn && N % 64 == 0 && N / bn < tc_sm_count()) bn = 64;
   if (ep.rope_cols > 0 && (N % 256 || ep.rope_cols % 256 || ep.rope_S < 1)) return SMARTMEM_ERR_UNSUPPORTED;
   if (ep.seg_cols > 0) {
     if (ep.seg_cols % 256 || N > 3ll * ep.seg_cols || ep.rowmap || ep.residual || batch != 1) return SMARTMEM_ERR_UNSUPPORTED;

@@ -150,6 +150,81 @@ __global__ void __launch_bounds__(256) norm_kernel(const T* __restrict__ src, T*
   }
 }
 
+// Wide rows (more than 128 vectors): one CTA per row, every thread keeps up to 4 of the row's 16-byte
+// vectors in registers, so the whole row is requested at once (the generic kernel above walks a
+// row one vector per lane at a time and is bound by that chain of load latencies).
+template <typename T, bool RMS>
+__global__ void __launch_bounds__(256) norm_wide_kernel(const T* __restrict__ src, T* __restrict__ dst,
+                                                        const T* __restrict__ gamma, const T* __restrict__ beta, float eps,
+                                                        int C) {
+  constexpr int KV = ElemIO<T>::kVec;
+  constexpr int NVW = 4;
+  __shared__ float red[8];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int nvec = C / KV;
+  const float invC = 1.0f / (float)C;
+  auto block_sum = [&](float x) {
+#pragma unroll
+    for (int m = 16; m >= 1; m >>= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, m);
+    __syncthreads();                                       // the previous round's reads of red[] are done
+    if (lane == 0) red[warp] = x;
+    __syncthreads();
+    float t = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) t += red[w];
+    return t;
+  };
+  pdl_wait();
+  pdl_launch_dependents();
+  const T* s = src + (long long)blockIdx.x * C;
+  T* d = dst + (long long)blockIdx.x * C;
+  float v[NVW][KV];
+#pragma unroll
+  for (int k = 0; k < NVW; ++k) {
+    const int vi = tid + k * 256;
+    if (vi < nvec) {
+      ElemIO<T>::load(s + vi * KV, v[k]);
+    } else {
+#pragma unroll
+      for (int e = 0; e < KV; ++e) v[k][e] = 0.f;
+    }
+  }
+  float sum = 0.f;
+#pragma unroll
+  for (int k = 0; k < NVW; ++k)
+#pragma unroll
+    for (int e = 0; e < KV; ++e) sum += RMS ? v[k][e] * v[k][e] : v[k][e];
+  sum = block_sum(sum);
+  float mean = 0.f, rstd;
+  if constexpr (RMS) {
+    rstd = rsqrtf(sum * invC + eps);
+  } else {
+    mean = sum * invC;
+    float sq = 0.f;
+#pragma unroll
+    for (int k = 0; k < NVW; ++k)
+      if (tid + k * 256 < nvec) {
+#pragma unroll
+        for (int e = 0; e < KV; ++e) sq += (v[k][e] - mean) * (v[k][e] - mean);
+      }
+    sq = block_sum(sq);
+    rstd = rsqrtf(sq * invC + eps);
+  }
+  const float ms = -mean * rstd;
+#pragma unroll
+  for (int k = 0; k < NVW; ++k) {
+    const int vi = tid + k * 256;
+    if (vi < nvec) {
+      float g[KV], b[KV], y[KV];
+      ElemIO<T>::load(gamma + vi * KV, g);
+      if constexpr (!RMS) ElemIO<T>::load(beta + vi * KV, b);
+#pragma unroll
+      for (int e = 0; e < KV; ++e) y[e] = RMS ? v[k][e] * rstd * g[e] : fmaf(fmaf(v[k][e], rstd, ms), g[e], b[e]);
+      ElemIO<T>::store(d + vi * KV, y);
+    }
+  }
+}
+
 template <typename T, bool RMS>
 int launch_norm_t(const void* src, void* dst, const void* gamma, const void* beta, float eps, long long rows, int C,
                   const DevMap* rowmap, cudaStream_t st) {
@@ -176,6 +251,8 @@ int launch_norm_t(const void* src, void* dst, const void* gamma, const void* bet
   else if (nvec <= 32) SM_LAUNCH(8, 2, false)
   else if (nvec <= 64) SM_LAUNCH(16, 1, false)
   else if (nvec <= 128) SM_LAUNCH(32, 1, false)
+  else if (!rowmap && nvec <= 1024)
+    launch_pdl(norm_wide_kernel<T, RMS>, dim3((unsigned)rows), dim3(256), 0, st, s, d, g, b, eps, C);
   else SM_LAUNCH(32, 1, true)
 #undef SM_LAUNCH
   count_launch();
