@@ -275,7 +275,7 @@ def run_other(args):
         # 2.1 GB per variant, far larger than L2, and is read once per step).  Weights and the new tokens come from
         # the seeded generator; the cache is filled by torch's seeded generator on the device (its values do not
         # affect the timing, and the parity tests use the package's own generator).
-        B, pos, S, hidden, heads = 64, 2047, 2048, 4096, 32
+        B, pos, S, hidden, heads = args.sequences, 2047, 2048, 4096, 32
         inp = synth.attn_layer_inputs(6, 1, hidden, "bf16", B)
         d = {k: dev(v) for k, v in inp.items()}
         p = sm.AttnParams()
@@ -401,11 +401,17 @@ def run_other(args):
         kern.append({"kernel": label, "launched_as": kname, "ms": round(t, 5), "bound": bound, "achieved": round(ach, 1),
                      "unit": "TFLOP/s" if bound == "tensor" else "GB/s", "frac": round(ach / (tf if bound == "tensor" else hbm), 4)})
     dom = max(kern, key=lambda k: k["ms"])
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "traffic.json")
+    if name == "llama_decode_layer" and dom["kernel"] == "decode_attention" and os.path.exists(tpath):
+        with open(tpath) as f:                               # DRAM bytes per sequence from the committed ncu capture, scaled
+            per_seq = json.load(f).get("decode_attention_per_sequence")
+        traffic = None if per_seq is None else int(per_seq) * args.sequences
     print(json.dumps({
         "metric": name + "_tokens_per_s", "value": tokens * args.steps / (ms[sm.ELIMINATE] * 1e-3), "unit": UNIT, "n_gpus": 1,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms[sm.ELIMINATE] / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": name, "mode": "eliminate",
+        "config": {"workload": name, "mode": "eliminate", **({"sequences": args.sequences, "cached_positions": 2047} if name == "llama_decode_layer" else {}),
                    "l2": f"{sets} rotating buffer sets" if sets > 1 else "inputs larger than L2 (the cache read flushes it every step)"},
         "explicit_variant": {"ms_per_step": ms[sm.EXPLICIT] / args.steps, "speedup_of_eliminate": ms[sm.EXPLICIT] / ms[sm.ELIMINATE],
                              "kernels": [{"launched_as": n, "ms": round(t, 5)} for n, t in per["explicit"]]},
@@ -414,7 +420,7 @@ def run_other(args):
         "map_placement": placement,
         "clocks": clocks,
         "roofline": {"bound": dom["bound"], "kernel": dom["kernel"], "achieved": dom["achieved"], "unit": dom["unit"],
-                     "peak": tf if dom["bound"] == "tensor" else hbm, "frac": dom["frac"], "traffic": None, "peak_source": src},
+                     "peak": tf if dom["bound"] == "tensor" else hbm, "frac": dom["frac"], "traffic": traffic, "peak_source": src},
         "kernels": kern,
     }))
 
@@ -426,6 +432,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="smartmem", choices=["smartmem", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sequences", type=int, default=64,
+                    help="llama_decode_layer only: sequences decoded per step (64 is the workload; smaller for profiler captures)")
     ap.add_argument("--workload", default=WORKLOAD["name"],
                     help="swin_t_stage1_block (default, the benchmark line) or one of: " + ", ".join(OTHER_WORKLOADS))
     args = ap.parse_args()

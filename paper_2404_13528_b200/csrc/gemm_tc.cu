@@ -321,7 +321,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         off += (long long)batch * g.out_batch_stride;
       }
       const __nv_bfloat16* __restrict__ rrow = g.residual ? g.residual + off : nullptr;
-      const bool rope_tile = BN == 256 && g.rope_cols > 0 && n0 < g.rope_cols;
+      const bool rope_tile = (BN == 256 || BN == 128) && g.rope_cols > 0 && n0 < g.rope_cols;
       auto col_of = [&](int rd) {
         return BN == 256 ? 128 * (grp >> 1) + 32 * (grp & 1) + RC * (rd % RH) + 64 * (rd / RH) : grp * CG;
       };
@@ -376,13 +376,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             // rotary pairs are (c, c + 64) inside a 128-column head: round 0 holds the first half
             // of the pair, round 1 the second; each round reads both halves from TMEM
             uint32_t rw[RC];
-            ptx::tmem_ld_cols<RC>(taddr + (rd < RH ? c0 + 64 : c0 - 64), rw);
+            // (128-wide tile = one head: column groups 0, 1 hold the first halves, 2, 3 the second)
+            const bool first_half = BN == 256 ? rd < RH : grp < 2;
+            ptx::tmem_ld_cols<RC>(taddr + (first_half ? c0 + 64 : c0 - 64), rw);
             ptx::tmem_ld_wait();
             // angle = position * theta^(-i/64), reduced mod 2 pi in two steps, then the hardware
             // sine / cosine: no table traffic (a [S, 64] table read 16 bytes per lane per row
             // slowed the whole kernel by a fifth)
             const float pos = (float)(row_ok ? g.rope_pos0 + row % g.rope_S : 0);
-            const int i0 = (grp & 1) * 32 + RC * (rd % RH);
+            const int i0 = (grp & 1) * 32 + (BN == 256 ? RC * (rd % RH) : 0);
 #pragma unroll
             for (int j = 0; j < RC; ++j) {
               float f;
@@ -393,7 +395,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               red = fmaf(kk, 1.7484556e-7f, red);
               const float sn = __sinf(red), cs = __cosf(red);
               const float x = __uint_as_float(rv[j]), y = __uint_as_float(rw[j]);
-              acc[j] = rd < RH ? x * cs - y * sn : x * cs + y * sn;
+              acc[j] = first_half ? x * cs - y * sn : x * cs + y * sn;
             }
           } else {
             ptx::tmem_ld_wait();
@@ -697,7 +699,7 @@ int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep,
   if (B.k_stride != 1) return SMARTMEM_ERR_UNSUPPORTED;
   // tile width: the widest of {256, 128, 96, 64} that divides N (fewest wasted columns), else 128
   int bn = 128;
-  if (ep.rope_cols > 0) bn = 256;
+  if (ep.rope_cols > 0) bn = (M <= BM && batch == 1 && N / 256 < tc_sm_count()) ? 128 : 256;   // one head or two per tile
   else if (N % 256 == 0) bn = 256;
   else if (N % 128 == 0) bn = 128;
   else if (N % 96 == 0) bn = 96;
