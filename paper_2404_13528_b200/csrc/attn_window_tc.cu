@@ -81,6 +81,9 @@ __device__ __forceinline__ float ex2f(float x) {
   return y;
 }
 
+// KC: key columns a softmax thread works on (56 when the window has at most 56 tokens -- a 7 x 7 window
+// has 49 -- else 64).  Columns [T, 64) of a score row are padding whose probability is zero.
+template <int KC>
 __global__ void __launch_bounds__(kThreads, 1)
 win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constant__ CUtensorMap tm1,
                    const __grid_constant__ CUtensorMap tm2, const __grid_constant__ WinTcArgs g) {
@@ -332,24 +335,29 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
       if (!ok) break;
       if (q == 0 && lane == 0) WDBG(u * 16 + 6);
       ptx::tc_fence_after();
-      uint32_t rv[64];
+      uint32_t rv[KC];
       const uint32_t ts = tmem_base + TM_S + sb * 128 + lane_addr + w * 64;    // this window's 64 key columns
       ptx::tmem_ld32(ts, rv);
-      ptx::tmem_ld32(ts + 32, rv + 32);
+      if constexpr (KC == 64) {
+        ptx::tmem_ld32(ts + 32, rv + 32);
+      } else {
+        ptx::tmem_ld16(ts + 32, rv + 32);
+        ptx::tmem_ld8(ts + 48, rv + 48);
+      }
       ptx::tmem_ld_wait();
       if (q == 0 && lane == 0) WDBG(u * 16 + 7);
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&s_empty[sb]);
-      float sc[64];
+      float sc[KC];
       float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // independent chains
 #ifdef WA_EXP_TIMING
-      if (q == 0 && lane == 0 && __uint_as_float(rv[63]) != 123.456f) WDBG(u * 16 + 13);
+      if (q == 0 && lane == 0 && __uint_as_float(rv[KC - 1]) != 123.456f) WDBG(u * 16 + 13);
 #endif
       // scores in natural units: q.k * scale + bias (the row's 64 biases come as eight 16-byte reads
       // of bf16 pairs); the base-2 conversion is folded into the exponent's multiply-add below
 #pragma unroll
-      for (int v8 = 0; v8 < 8; ++v8) {
+      for (int v8 = 0; v8 < KC / 8; ++v8) {
         const uint4 b4 = *reinterpret_cast<const uint4*>(brow + v8 * 4);
         const uint32_t bw[4] = {b4.x, b4.y, b4.z, b4.w};
 #pragma unroll
@@ -363,11 +371,11 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
 #pragma unroll
         for (int c = 0; c < 32; ++c) {
           if ((diff_lo >> c) & 1u) sc[c] -= 100.f;
-          if ((diff_hi >> c) & 1u) sc[c + 32] -= 100.f;
+          if (c + 32 < KC && ((diff_hi >> c) & 1u)) sc[c + 32] -= 100.f;
         }
       }
 #pragma unroll
-      for (int c = 0; c < 64; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], sc[c]);
+      for (int c = 0; c < KC; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], sc[c]);
       const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       const float nmx = -mx * LOG2E;
 #ifdef WA_EXP_TIMING
@@ -376,7 +384,9 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
       float sum4[4] = {0.f, 0.f, 0.f, 0.f};
       uint32_t pk[32];
 #pragma unroll
-      for (int c = 0; c < 64; c += 2) {
+      for (int c = KC / 2; c < 32; ++c) pk[c] = 0u;        // padding keys
+#pragma unroll
+      for (int c = 0; c < KC; c += 2) {
         const float p0 = ex2f(fmaf(sc[c], LOG2E, nmx)), p1 = ex2f(fmaf(sc[c + 1], LOG2E, nmx));
         sum4[c & 2] += p0;
         sum4[(c & 2) + 1] += p1;
@@ -517,7 +527,8 @@ int launch_window_attention_tc(const WinAttnArgs& a_in, long long n_windows, cud
                       (2 * NSTAGE + 12) * 8 + 16;
   static bool configured = false;
   if (!configured) {
-    if (cudaFuncSetAttribute(win_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    if (cudaFuncSetAttribute(win_attn_tc_kernel<56>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+        cudaFuncSetAttribute(win_attn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return SMARTMEM_ERR_CUDA;
     configured = true;
   }
@@ -527,7 +538,8 @@ int launch_window_attention_tc(const WinAttnArgs& a_in, long long n_windows, cud
   if (per_head > g.n_pairs) per_head = g.n_pairs;
   const unsigned grid = (unsigned)(per_head * a.heads);
   profile_tick("window_attention_tc", st);
-  launch_pdl(win_attn_tc_kernel, dim3(grid), dim3(kThreads), smem, st, tm[0], tm[1], tm[2], g);
+  if (a.T <= 56) launch_pdl(win_attn_tc_kernel<56>, dim3(grid), dim3(kThreads), smem, st, tm[0], tm[1], tm[2], g);
+  else launch_pdl(win_attn_tc_kernel<64>, dim3(grid), dim3(kThreads), smem, st, tm[0], tm[1], tm[2], g);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
 }
