@@ -75,10 +75,15 @@ typedef enum {
   SMARTMEM_OP_SLICE = 3,            /* start[], shape[] = extent                           */
   SMARTMEM_OP_WINDOW_PARTITION = 4, /* [B,H,W,C] -> [B*H/ws*W/ws, ws*ws, C]; window = ws   */
   SMARTMEM_OP_WINDOW_REVERSE = 5,   /* inverse; shape[0..2] = B,H,W                        */
+  SMARTMEM_OP_DEPTH_TO_SPACE = 6,   /* [N,C*b*b,H,W] -> [N,C,H*b,W*b]: out[n,c,h*b+i,w*b+j] = in[n,(i*b+j)*C+c,h,w]; window = b
+                                       (Table 3's DtoS; depth-column-row order)             */
+  SMARTMEM_OP_SPACE_TO_DEPTH = 7,   /* inverse (Table 3's StoD): [N,C,H,W] -> [N,C*b*b,H/b,W/b]; window = b */
   SMARTMEM_OP_COPY = 16,            /* consumer: writes the current tensor contiguously    */
   SMARTMEM_OP_LINEAR = 17,          /* consumer: out[M,N] = A[M,K] W[N,K]^T, W = side_input[0] */
-  SMARTMEM_OP_BMM_NT = 18           /* consumer: out[..,i,j] = sum_e A[..,i,e] B[..,j,e]; B is the
+  SMARTMEM_OP_BMM_NT = 18,          /* consumer: out[..,i,j] = sum_e A[..,i,e] B[..,j,e]; B is the
                                        result of running the same layout run on side_input[0] */
+  SMARTMEM_OP_LAYERNORM = 19        /* consumer: LayerNorm over the last dimension (an ILD & Variable operator of
+                                       Table 3): gamma = side_input[0], beta = side_input[1], both [C]; eps   */
 } smartmem_op_kind_t;
 
 #define SMARTMEM_MAX_DIMS 8
@@ -93,8 +98,10 @@ typedef struct {
   int64_t start[SMARTMEM_MAX_DIMS];  /* slice                                               */
   int64_t shift;                     /* roll                                                */
   int32_t axis;                      /* roll                                                */
-  int32_t window;                    /* window partition / reverse                          */
+  int32_t window;                    /* window partition / reverse; block size of depth/space */
   int32_t side_input[2];             /* index into the plan's inputs[] (weights, 2nd operand) */
+  float eps;                         /* layernorm                                           */
+  int32_t reserved;                  /* zero                                                */
 } smartmem_op_t;
 
 typedef struct {

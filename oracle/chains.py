@@ -3,7 +3,8 @@ materialised, followed by a consumer.  Test infrastructure only.
 
 An operator is a dict: {"op": "reshape", "shape": [...]}, {"op": "transpose", "perm": [...]},
 {"op": "roll", "shift": s, "axis": a}, {"op": "slice", "start": [...], "extent": [...]},
-{"op": "window_partition", "window": ws}, {"op": "window_reverse", "window": ws, "B":.., "H":.., "W":..}.
+{"op": "window_partition", "window": ws}, {"op": "window_reverse", "window": ws, "B":.., "H":.., "W":..},
+{"op": "depth_to_space", "block": b}, {"op": "space_to_depth", "block": b}.
 """
 from __future__ import annotations
 
@@ -28,6 +29,10 @@ def apply_layout_chain(x: np.ndarray, chain) -> np.ndarray:
             y = layout.window_partition(y, o["window"])
         elif kind == "window_reverse":
             y = layout.window_reverse(y, o["window"], o["B"], o["H"], o["W"])
+        elif kind == "depth_to_space":
+            y = layout.depth_to_space(y, o["block"])
+        elif kind == "space_to_depth":
+            y = layout.space_to_depth(y, o["block"])
         else:
             raise ValueError(f"not a layout operator: {kind}")
     return y

@@ -94,3 +94,38 @@ def head_merge(o: np.ndarray) -> np.ndarray:
     """[nW,nH,T,d] -> transpose (0,2,1,3) -> reshape [nW,T,nH*d]."""
     nW, nH, T, d = o.shape
     return reshape(transpose(o, (0, 2, 1, 3)), (nW, T, nH * d))
+
+
+def depth_to_space(x: np.ndarray, b: int) -> np.ndarray:
+    """[N, C*b*b, H, W] -> [N, C, H*b, W*b], depth-column-row order (the DtoS operator of Table 3, with
+    the ONNX DepthToSpace "DCR" element order): out[n, c, h*b+i, w*b+j] = x[n, (i*b+j)*C + c, h, w].
+    Written as the definition: one strided assignment per (i, j) block offset."""
+    N, Cb, H, W = x.shape
+    assert Cb % (b * b) == 0
+    C = Cb // (b * b)
+    out = np.empty((N, C, H * b, W * b), dtype=x.dtype)
+    for i in range(b):
+        for j in range(b):
+            out[:, :, i::b, j::b] = x[:, (i * b + j) * C:(i * b + j + 1) * C]
+    return out
+
+
+def space_to_depth(x: np.ndarray, b: int) -> np.ndarray:
+    """[N, C, H, W] -> [N, C*b*b, H/b, W/b] (the StoD operator of Table 3, ONNX SpaceToDepth order):
+    out[n, (i*b+j)*C + c, h, w] = x[n, c, h*b+i, w*b+j]."""
+    N, C, H, W = x.shape
+    assert H % b == 0 and W % b == 0
+    out = np.empty((N, C * b * b, H // b, W // b), dtype=x.dtype)
+    for i in range(b):
+        for j in range(b):
+            out[:, (i * b + j) * C:(i * b + j + 1) * C] = x[:, :, i::b, j::b]
+    return out
+
+
+def patch_merge_gather(x: np.ndarray) -> np.ndarray:
+    """Swin patch merging, layout part: [B,H,W,C] -> [B, H/2*W/2, 4C], the channel-wise Concat of the four
+    Slices x[:, 0::2, 0::2], x[:, 1::2, 0::2], x[:, 0::2, 1::2], x[:, 1::2, 1::2] (in that order)."""
+    B, H, W, C = x.shape
+    assert H % 2 == 0 and W % 2 == 0
+    parts = [x[:, 0::2, 0::2], x[:, 1::2, 0::2], x[:, 0::2, 1::2], x[:, 1::2, 1::2]]
+    return np.concatenate(parts, axis=-1).reshape(B, (H // 2) * (W // 2), 4 * C)

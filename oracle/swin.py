@@ -58,3 +58,9 @@ def swin_block(x, p, *, heads, window, shift, mlp_ratio, eps=1e-5, keep=None):
     if keep is not None:
         keep.update(yn=yn, h=h)
     return z
+
+
+def patch_merging(x, gamma, beta, w, eps=1e-5):
+    """Swin patch merging between stages: [B,H,W,C] -> [B, H/2*W/2, 2C]: the 2x2 neighbourhood gathered to 4C
+    channels (Slice x4 + Concat), LayerNorm over 4C, linear 4C -> 2C without bias (w [2C,4C])."""
+    return ops.linear(ops.layernorm(layout.patch_merge_gather(x), gamma, beta, eps), w)

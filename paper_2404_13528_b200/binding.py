@@ -20,13 +20,15 @@ ERR_ALIGNMENT, ERR_CUDA, ERR_TIMEOUT, ERR_BOUNDS = -5, -6, -7, -8
 F32, BF16 = 0, 1
 ELIMINATE, EXPLICIT, ELIMINATE_NAIVE, ELIMINATE_GATHER, ELIMINATE_SCATTER = 0, 1, 2, 3, 4
 OP_RESHAPE, OP_TRANSPOSE, OP_ROLL, OP_SLICE, OP_WINDOW_PARTITION, OP_WINDOW_REVERSE = 0, 1, 2, 3, 4, 5
+OP_DEPTH_TO_SPACE, OP_SPACE_TO_DEPTH = 6, 7
 OP_COPY, OP_LINEAR, OP_BMM_NT = 16, 17, 18
 
 
 class Op(C.Structure):
     _fields_ = [("kind", C.c_int32), ("ndim", C.c_int32), ("shape", C.c_int64 * MAX_DIMS),
                 ("perm", C.c_int32 * MAX_DIMS), ("start", C.c_int64 * MAX_DIMS), ("shift", C.c_int64),
-                ("axis", C.c_int32), ("window", C.c_int32), ("side_input", C.c_int32 * 2)]
+                ("axis", C.c_int32), ("window", C.c_int32), ("side_input", C.c_int32 * 2), ("eps", C.c_float),
+                ("reserved", C.c_int32)]
 
 
 class TensorDesc(C.Structure):
@@ -129,7 +131,7 @@ def _check(rc: int, where: str):
 # ---------------------------------------------------------------------------------------------
 # helpers to build the C structures
 # ---------------------------------------------------------------------------------------------
-def make_op(kind: int, *, shape=(), perm=(), start=(), shift=0, axis=0, window=0, side_input=(0, 0)) -> Op:
+def make_op(kind: int, *, shape=(), perm=(), start=(), shift=0, axis=0, window=0, side_input=(0, 0), eps=0.0) -> Op:
     o = Op()
     o.kind = kind
     o.ndim = max(len(shape), len(perm), len(start))
@@ -141,6 +143,7 @@ def make_op(kind: int, *, shape=(), perm=(), start=(), shift=0, axis=0, window=0
         o.start[i] = int(v)
     o.shift, o.axis, o.window = int(shift), int(axis), int(window)
     o.side_input[0], o.side_input[1] = int(side_input[0]), int(side_input[1])
+    o.eps = float(eps)
     return o
 
 

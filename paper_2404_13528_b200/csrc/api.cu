@@ -172,6 +172,9 @@ EXPORT int smartmem_run_chain(const smartmem_plan_t* plan, const void* const* in
       ep.ldc = s.N;
       ep.out_batch_stride = s.M * s.N;
       rc = launch_gemm_tc(A, B, ep, s.batch, s.M, s.N, s.K, st);
+    } else if (s.kind == STEP_NORM) {
+      rc = launch_layernorm_map(s.dtype, buf(s.src[0]), buf(s.dst), inputs[s.weight], inputs[s.weight2], s.eps, s.map[0],
+                                (int)s.K, st);
     } else {
       rc = SMARTMEM_ERR_UNSUPPORTED;
     }

@@ -256,6 +256,10 @@ int launch_copy_map(const smartmem_index_map_t& map, int elem_size, const void* 
 
 // LayerNorm / RMSNorm over rows of length C.  Row r of the output (row-major [rows, C]) is
 // read from src at element offset rowmap(r) (rowmap == nullptr: r * C).
+// LayerNorm over the last dimension of a [rows, C] tensor whose elements are read through `map` (consumer
+// linear index -> producer element offset, 16-byte vectors intact, C / vector <= 128); writes [rows, C] contiguously.
+int launch_layernorm_map(int dtype, const void* src, void* dst, const void* gamma, const void* beta, float eps,
+                         const smartmem_index_map_t& map, int C, cudaStream_t st);
 int launch_norm(int dtype, bool rms, const void* src, void* dst, const void* gamma, const void* beta, float eps,
                 long long rows, int C, const DevMap* rowmap, cudaStream_t st);
 

@@ -225,6 +225,71 @@ __global__ void __launch_bounds__(256) norm_wide_kernel(const T* __restrict__ sr
   }
 }
 
+// Rows whose elements are fetched through an eliminated layout chain: vector u of the consumer's
+// [rows, C] tensor (16 bytes, never straddling a contiguous run of the producer) lies at element
+// offset map(u).  One warp per row, up to 4 vectors per lane in registers; the result is written
+// contiguously.
+template <typename T, bool RMS>
+__global__ void __launch_bounds__(256) norm_gather_kernel(const T* __restrict__ src, T* __restrict__ dst,
+                                                          const T* __restrict__ gamma, const T* __restrict__ beta, float eps,
+                                                          long long rows, int C, const __grid_constant__ DevMap map) {
+  constexpr int KV = ElemIO<T>::kVec;
+  constexpr int NV = 4;
+  const int lane = threadIdx.x & 31;
+  const long long row = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int nvec = C / KV;
+  const float invC = 1.0f / (float)C;
+  pdl_wait();
+  pdl_launch_dependents();
+  if (row >= rows) return;
+  float v[NV][KV];
+#pragma unroll
+  for (int k = 0; k < NV; ++k) {
+    const int vi = lane + k * 32;
+    if (vi < nvec) {
+      const long long off = devmap_eval_unrolled(map, (uint32_t)(row * nvec + vi));
+      ElemIO<T>::load(src + off, v[k]);
+    } else {
+#pragma unroll
+      for (int e = 0; e < KV; ++e) v[k][e] = 0.f;
+    }
+  }
+  float sum = 0.f;
+#pragma unroll
+  for (int k = 0; k < NV; ++k)
+#pragma unroll
+    for (int e = 0; e < KV; ++e) sum += RMS ? v[k][e] * v[k][e] : v[k][e];
+  sum = group_sum<32>(sum);
+  float mean = 0.f, rstd;
+  if constexpr (RMS) {
+    rstd = rsqrtf(sum * invC + eps);
+  } else {
+    mean = sum * invC;
+    float sq = 0.f;
+#pragma unroll
+    for (int k = 0; k < NV; ++k)
+      if (lane + k * 32 < nvec) {
+#pragma unroll
+        for (int e = 0; e < KV; ++e) sq += (v[k][e] - mean) * (v[k][e] - mean);
+      }
+    sq = group_sum<32>(sq);
+    rstd = rsqrtf(sq * invC + eps);
+  }
+  const float ms = -mean * rstd;
+#pragma unroll
+  for (int k = 0; k < NV; ++k) {
+    const int vi = lane + k * 32;
+    if (vi < nvec) {
+      float g[KV], b[KV], y[KV];
+      ElemIO<T>::load(gamma + vi * KV, g);
+      if constexpr (!RMS) ElemIO<T>::load(beta + vi * KV, b);
+#pragma unroll
+      for (int e = 0; e < KV; ++e) y[e] = RMS ? v[k][e] * rstd * g[e] : fmaf(fmaf(v[k][e], rstd, ms), g[e], b[e]);
+      ElemIO<T>::store(dst + row * (long long)C + vi * KV, y);
+    }
+  }
+}
+
 template <typename T, bool RMS>
 int launch_norm_t(const void* src, void* dst, const void* gamma, const void* beta, float eps, long long rows, int C,
                   const DevMap* rowmap, cudaStream_t st) {
@@ -259,7 +324,29 @@ int launch_norm_t(const void* src, void* dst, const void* gamma, const void* bet
   return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
 }
 
+template <typename T>
+int launch_norm_map_t(const void* src, void* dst, const void* gamma, const void* beta, float eps,
+                      const smartmem_index_map_t& map, int C, cudaStream_t st) {
+  constexpr int KV = ElemIO<T>::kVec;
+  if (C % KV || C / KV > 128 || map.vec_elems != KV || map.klass == 3) return SMARTMEM_ERR_UNSUPPORTED;
+  const long long rows = map.n_elements / C;
+  if (map.n_elements / KV >= (1ll << 31)) return SMARTMEM_ERR_UNSUPPORTED;
+  DevMap dm;
+  if (!make_devmap(map, 0, map.n_atoms, KV, true, &dm)) return SMARTMEM_ERR_UNSUPPORTED;
+  launch_pdl(norm_gather_kernel<T, false>, dim3((unsigned)((rows + 7) / 8)), dim3(256), 0, st, (const T*)src, (T*)dst,
+             (const T*)gamma, (const T*)beta, eps, rows, C, dm);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
+}
+
 }  // namespace
+
+int launch_layernorm_map(int dtype, const void* src, void* dst, const void* gamma, const void* beta, float eps,
+                         const smartmem_index_map_t& map, int C, cudaStream_t st) {
+  profile_tick("layernorm_map", st);
+  if (dtype == SMARTMEM_F32) return launch_norm_map_t<float>(src, dst, gamma, beta, eps, map, C, st);
+  return launch_norm_map_t<__nv_bfloat16>(src, dst, gamma, beta, eps, map, C, st);
+}
 
 int launch_norm(int dtype, bool rms, const void* src, void* dst, const void* gamma, const void* beta, float eps,
                 long long rows, int C, const DevMap* rowmap, cudaStream_t st) {

@@ -289,6 +289,34 @@ int apply_layout_op(const smartmem_op_t& op, TState& s, SeqProgram& seq) {
       push(a); push(b); push(c);
       return SMARTMEM_OK;
     }
+    case SMARTMEM_OP_DEPTH_TO_SPACE: {
+      if (nd != 4 || op.window < 1) return SMARTMEM_ERR_SHAPE;
+      int64_t N = s.shape[0], Cb = s.shape[1], H = s.shape[2], W = s.shape[3], b = op.window;
+      if (Cb % (b * b)) return SMARTMEM_ERR_SHAPE;
+      SeqStage x, y, z;
+      x.kind = SMARTMEM_OP_RESHAPE;
+      x.out_shape = {N, b, b, Cb / (b * b), H, W};
+      y.kind = SMARTMEM_OP_TRANSPOSE;
+      y.perm = {0, 3, 4, 1, 5, 2};
+      z.kind = SMARTMEM_OP_RESHAPE;
+      z.out_shape = {N, Cb / (b * b), H * b, W * b};
+      push(x); push(y); push(z);
+      return SMARTMEM_OK;
+    }
+    case SMARTMEM_OP_SPACE_TO_DEPTH: {
+      if (nd != 4 || op.window < 1) return SMARTMEM_ERR_SHAPE;
+      int64_t N = s.shape[0], C = s.shape[1], H = s.shape[2], W = s.shape[3], b = op.window;
+      if (H % b || W % b) return SMARTMEM_ERR_SHAPE;
+      SeqStage x, y, z;
+      x.kind = SMARTMEM_OP_RESHAPE;
+      x.out_shape = {N, C, H / b, b, W / b, b};
+      y.kind = SMARTMEM_OP_TRANSPOSE;
+      y.perm = {0, 3, 5, 1, 2, 4};
+      z.kind = SMARTMEM_OP_RESHAPE;
+      z.out_shape = {N, C * b * b, H / b, W / b};
+      push(x); push(y); push(z);
+      return SMARTMEM_OK;
+    }
   }
   return SMARTMEM_ERR_INVALID_ARG;
 }
@@ -519,7 +547,7 @@ int process_run(smartmem_plan_t* p, const smartmem_op_t* ops, int i0, int i1, co
   return SMARTMEM_OK;
 }
 
-bool is_layout_kind(int k) { return k >= SMARTMEM_OP_RESHAPE && k <= SMARTMEM_OP_WINDOW_REVERSE; }
+bool is_layout_kind(int k) { return k >= SMARTMEM_OP_RESHAPE && k <= SMARTMEM_OP_SPACE_TO_DEPTH; }
 
 }  // namespace
 
@@ -528,10 +556,11 @@ extern "C" {
 int smartmem_op_quadrant(int32_t kind, int32_t* q) {
   if (!q) return SMARTMEM_ERR_INVALID_ARG;
   switch (kind) {
-    case SMARTMEM_OP_LINEAR: case SMARTMEM_OP_BMM_NT: *q = 0; return SMARTMEM_OK;           // MatMul
+    case SMARTMEM_OP_LINEAR: case SMARTMEM_OP_BMM_NT: case SMARTMEM_OP_LAYERNORM: *q = 0; return SMARTMEM_OK;   // MatMul, LayerNorm
     case SMARTMEM_OP_COPY: *q = 1; return SMARTMEM_OK;                                       // Unary (identity)
     case SMARTMEM_OP_RESHAPE: case SMARTMEM_OP_TRANSPOSE: case SMARTMEM_OP_WINDOW_PARTITION:
-    case SMARTMEM_OP_WINDOW_REVERSE: *q = 2; return SMARTMEM_OK;                             // Reshape / Transpose
+    case SMARTMEM_OP_WINDOW_REVERSE: case SMARTMEM_OP_DEPTH_TO_SPACE: case SMARTMEM_OP_SPACE_TO_DEPTH:
+      *q = 2; return SMARTMEM_OK;                                                             // Reshape / Transpose / DtoS / StoD
     case SMARTMEM_OP_ROLL: case SMARTMEM_OP_SLICE: *q = 3; return SMARTMEM_OK;               // Gather / Slice
   }
   return SMARTMEM_ERR_INVALID_ARG;
@@ -705,6 +734,49 @@ int smartmem_plan(const smartmem_op_t* ops, int32_t n_ops, const smartmem_tensor
       st.n_row_atoms[1] = apg[1];
       oshape.assign(sa.begin(), sa.end() - 1);
       oshape.push_back(st.N);
+    } else if (c.kind == SMARTMEM_OP_LAYERNORM) {
+      st.kind = STEP_NORM;
+      const int gi = c.side_input[0], bi = c.side_input[1];
+      if (gi < 1 || gi >= n_inputs || bi < 1 || bi >= n_inputs) { rc = SMARTMEM_ERR_INVALID_ARG; break; }
+      if (nd < 1 || !(c.eps > 0.f)) { rc = SMARTMEM_ERR_INVALID_ARG; break; }
+      const int64_t C = A.state.shape[nd - 1];
+      for (int wi : {gi, bi}) {
+        const smartmem_tensor_desc_t& w = inputs[wi];
+        if (w.ndim != 1 || w.shape[0] != C || w.dtype != dtype) rc = SMARTMEM_ERR_SHAPE;
+        else if (!state_from_desc(w).fresh) rc = SMARTMEM_ERR_UNSUPPORTED;
+      }
+      if (rc != SMARTMEM_OK) break;
+      st.weight = gi;
+      st.weight2 = bi;
+      st.eps = c.eps;
+      st.K = C;
+      st.M = prod(A.state.shape) / C;
+      rc = finalize_map(A.state, {nd - 1, nd}, esz, &st.map[0], apg);
+      if (rc != SMARTMEM_OK) break;
+      // the kernel fetches a row as 16-byte vectors through the map: they must not straddle a contiguous run, and
+      // a warp holds the row in registers; otherwise the run is materialised first (as EXPLICIT does anyway)
+      const int vec = 16 / esz;
+      const bool foldable = st.map[0].klass != 3 && st.map[0].vec_elems % vec == 0 && C % vec == 0 && C / vec <= 128;
+      if (!foldable && st.map[0].klass != 0) {
+        Step cp;
+        cp.kind = STEP_COPY;
+        cp.dtype = dtype;
+        cp.is_layout_copy = true;
+        cp.src[0] = A.src;
+        int apg1[1];
+        rc = finalize_map(A.state, {nd}, esz, &cp.map[0], apg1);
+        if (rc != SMARTMEM_OK) break;
+        cp.seq[0] = A.seq;
+        cp.dst = new_slot(p, cp.map[0].n_elements, esz);
+        p->steps.push_back(cp);
+        const smartmem_tensor_desc_t ndsc = contiguous_desc(A.state.shape, dtype);
+        TState fresh = state_from_desc(ndsc);
+        st.src[0] = cp.dst;
+        st.seq[0] = seq_from_desc(ndsc);
+        rc = finalize_map(fresh, {nd - 1, nd}, esz, &st.map[0], apg);
+        if (rc != SMARTMEM_OK) break;
+      }
+      oshape = A.state.shape;
     } else {
       rc = SMARTMEM_ERR_INVALID_ARG;
     }

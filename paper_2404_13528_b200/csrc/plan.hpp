@@ -24,7 +24,7 @@ struct SeqProgram {
   int64_t eval(int64_t consumer_linear) const;
 };
 
-enum StepKind { STEP_COPY = 0, STEP_LINEAR = 1, STEP_BMM_NT = 2 };
+enum StepKind { STEP_COPY = 0, STEP_LINEAR = 1, STEP_BMM_NT = 2, STEP_NORM = 3 };
 
 // Buffer reference: >= 0 caller input index; -1 the chain output; <= -2 workspace slot (-2 - slot).
 struct Step {
@@ -32,7 +32,9 @@ struct Step {
   int dtype = SMARTMEM_BF16;
   int src[2] = {0, 0};
   int dst = -1;
-  int weight = -1;                   // LINEAR: caller input index of W[N,K]
+  int weight = -1;                   // LINEAR: caller input index of W[N,K]; NORM: of gamma[C]
+  int weight2 = -1;                  // NORM: caller input index of beta[C]
+  float eps = 0.f;                   // NORM
   smartmem_index_map_t map[2];
   // For GEMM-like consumers the atoms of map[] are grouped: [0, n_batch_atoms) batch,
   // then row atoms, then reduction atoms (never merged across the group boundaries).

@@ -117,3 +117,44 @@ def test_chain_source_offsets_match_closed_forms():
                                                  {"op": "reshape", "shape": (B * Hh * Ww, C)}])
     for b, hw, c in itertools.product(range(B), range(Hh * Ww), range(C)):
         assert off[b * Hh * Ww + hw, c] == b * C * Hh * Ww + c * Hh * Ww + hw
+
+
+@pytest.mark.parametrize("N,C,H,W,b", [(1, 1, 2, 3, 2), (2, 3, 2, 2, 2), (1, 2, 1, 2, 3)])
+def test_depth_to_space_and_space_to_depth_bruteforce(N, C, H, W, b):
+    """Element by element against the index definition, and the two operators invert each other."""
+    x = rng.standard_normal((N, C * b * b, H, W))
+    y = layout.depth_to_space(x, b)
+    assert y.shape == (N, C, H * b, W * b)
+    for n, c, h, w, i, j in itertools.product(range(N), range(C), range(H), range(W), range(b), range(b)):
+        assert y[n, c, h * b + i, w * b + j] == x[n, (i * b + j) * C + c, h, w]
+    assert np.array_equal(layout.space_to_depth(y, b), x)
+    z = rng.standard_normal((N, C, H * b, W * b))
+    s = layout.space_to_depth(z, b)
+    assert s.shape == (N, C * b * b, H, W)
+    for n, c, h, w, i, j in itertools.product(range(N), range(C), range(H), range(W), range(b), range(b)):
+        assert s[n, (i * b + j) * C + c, h, w] == z[n, c, h * b + i, w * b + j]
+    # block size 1 moves nothing
+    assert np.array_equal(layout.depth_to_space(x, 1), x)
+
+
+def test_depth_to_space_equals_its_reshape_transpose_form():
+    """The textbook three-operator form: reshape [N,b,b,C,H,W] -> transpose (0,3,4,1,5,2) -> reshape."""
+    N, C, H, W, b = 2, 3, 4, 5, 2
+    x = rng.standard_normal((N, C * b * b, H, W))
+    ref = x.reshape(N, b, b, C, H, W).transpose(0, 3, 4, 1, 5, 2).reshape(N, C, H * b, W * b)
+    assert np.array_equal(layout.depth_to_space(x, b), ref)
+
+
+def test_patch_merge_gather_bruteforce():
+    """out[b, i*(W/2)+j, q*C + c] = x[b, 2i + q%2, 2j + q//2, c]: the four slices in the order
+    (0,0), (1,0), (0,1), (1,1) of (row, column) offsets."""
+    B, H, W, C = 2, 4, 6, 3
+    x = rng.standard_normal((B, H, W, C))
+    y = layout.patch_merge_gather(x)
+    assert y.shape == (B, (H // 2) * (W // 2), 4 * C)
+    for b, i, j, q, c in itertools.product(range(B), range(H // 2), range(W // 2), range(4), range(C)):
+        assert y[b, i * (W // 2) + j, q * C + c] == x[b, 2 * i + q % 2, 2 * j + q // 2, c]
+    # the same permutation as a reshape -> transpose -> reshape chain (what the planner composes)
+    chain = [{"op": "reshape", "shape": [B, H // 2, 2, W // 2, 2, C]}, {"op": "transpose", "perm": [0, 1, 3, 4, 2, 5]},
+             {"op": "reshape", "shape": [B, (H // 2) * (W // 2), 4 * C]}]
+    assert np.array_equal(chains.apply_layout_chain(x, chain), y)

@@ -326,3 +326,20 @@ def test_decode_step_special_cases():
     y0, _, _ = llama.decode_step(x, kc, vc, p0, heads=heads, head_dim=D, add_residual=True)
     mean_v = (vc.reshape(B, pos, hidden).sum(1) + v_new) / (pos + 1)
     assert np.allclose(y0, x + mean_v @ p["w_o"].T, atol=1e-11)
+
+
+def test_patch_merging_against_direct_restatement():
+    """Token (i, j) of the merged grid = LayerNorm over the 4C channels of its 2x2 neighbourhood, times w^T."""
+    B, H, W, C = 1, 4, 4, 3
+    x = rng.standard_normal((B, H, W, C))
+    g, b = 1 + 0.1 * rng.standard_normal(4 * C), 0.1 * rng.standard_normal(4 * C)
+    w = rng.standard_normal((2 * C, 4 * C))
+    y = swin.patch_merging(x, g, b, w)
+    assert y.shape == (B, 4, 2 * C)
+    for i, j in itertools.product(range(2), range(2)):
+        nb = np.concatenate([x[0, 2 * i, 2 * j], x[0, 2 * i + 1, 2 * j], x[0, 2 * i, 2 * j + 1], x[0, 2 * i + 1, 2 * j + 1]])
+        nn = (nb - nb.mean()) / np.sqrt(nb.var() + 1e-5) * g + b
+        assert np.allclose(y[0, i * 2 + j], w @ nn, atol=1e-12)
+    # constant input: LayerNorm gives beta, so every token maps to w beta
+    yc = swin.patch_merging(np.full((B, H, W, C), 2.5), g, b, w)
+    assert np.allclose(yc, np.broadcast_to(w @ b, yc.shape), atol=1e-9)
