@@ -6,6 +6,7 @@ import pytest
 import torch
 
 from oracle import chains
+from oracle import swin as oswin
 from paper_2404_13528_b200 import binding as sm
 from paper_2404_13528_b200 import synth
 from tests.gpu_util import assert_close_bf16, check_status, stream, to_dev, to_host_bits, to_host_f64
@@ -68,6 +69,10 @@ def swin_e1(s, ws):
                            {"op": "roll", "shift": 3, "axis": 1}, {"op": "roll", "shift": 3, "axis": 2}]),
     ((5, 5, 5), [{"op": "reshape", "shape": (5, 25)}, {"op": "transpose", "perm": (1, 0)}]),
     ((4, 6, 10), [{"op": "slice", "start": (1, 0, 2), "extent": (2, 6, 8)}, {"op": "transpose", "perm": (2, 0, 1)}]),
+    ((2, 64, 12, 20), [{"op": "depth_to_space", "block": 2}]),                     # DtoS / StoD of Table 3
+    ((2, 16, 24, 40), [{"op": "space_to_depth", "block": 2}]),
+    ((3, 36, 5, 7), [{"op": "depth_to_space", "block": 3}, {"op": "transpose", "perm": (0, 2, 3, 1)}]),
+    ((4, 128, 64, 64), [{"op": "depth_to_space", "block": 2}]),                    # a diffusion-decoder-sized upsample
     # split points that do not refine each other: only the sequential program can evaluate it
     ((4, 6), [{"op": "transpose", "perm": (1, 0)}, {"op": "reshape", "shape": (8, 3)}]),
     ((12, 10, 6), [{"op": "transpose", "perm": (2, 0, 1)}, {"op": "reshape", "shape": (8, 9, 10)}, {"op": "roll", "shift": 2, "axis": 1}]),
@@ -136,3 +141,33 @@ def test_run_chain_rejects_bad_arguments():
         sm.smartmem_run_chain(plan, [x.data_ptr()], [out.data_ptr()], 0, 0, stream())
     assert e.value.code == sm.ERR_WORKSPACE
     sm.smartmem_plan_destroy(plan)
+
+
+# ------------------------------------------------------------------ patch merging: gather -> LayerNorm -> linear
+def patch_merging_case(B, H, W, C, dtype="bf16"):
+    from tests.test_planner import _patch_merge_ops
+    x = synth.normal(78, 0, (B, H, W, C), dtype=dtype)
+    g = synth.normal(78, 1, (4 * C,), 0.02, 1.0, dtype)
+    b = synth.normal(78, 2, (4 * C,), 0.02, 0.0, dtype)
+    w = synth.normal(78, 3, (2 * C, 4 * C), 0.02, 0.0, dtype)
+    ref = oswin.patch_merging(synth.to_f64(x), synth.to_f64(g), synth.to_f64(b), synth.to_f64(w))
+    dt = sm.BF16 if dtype == "bf16" else sm.F32
+    descs = [sm.make_desc((B, H, W, C), dt), sm.make_desc((4 * C,), dt), sm.make_desc((4 * C,), dt), sm.make_desc((2 * C, 4 * C), dt)]
+    ins = [to_dev(t) for t in (x, g, b, w)]
+    outs = {}
+    for mode in (sm.ELIMINATE, sm.EXPLICIT):
+        out = run_plan(_patch_merge_ops(B, H, W, C), descs, mode, ins, ref.shape)
+        assert_close_bf16(to_host_f64(out), ref, f"mode {mode}")
+        outs[mode] = out
+    assert torch.equal(outs[sm.ELIMINATE].view(torch.int16), outs[sm.EXPLICIT].view(torch.int16))
+
+
+@pytest.mark.parametrize("B,H,W,C", [(1, 4, 4, 8), (2, 14, 10, 32), (3, 28, 28, 96), (2, 6, 6, 12)])
+def test_patch_merging_chain(B, H, W, C):
+    """(2, 6, 6, 12): 12 channels are not a whole number of 16-byte vectors, so ELIMINATE materialises the gather as well."""
+    patch_merging_case(B, H, W, C)
+
+
+def test_patch_merging_swin_t_stage1_full_size():
+    """[32,56,56,96] -> [32, 784, 192]: the merge between stages 1 and 2 of Swin-T at the benchmark's batch."""
+    patch_merging_case(32, 56, 56, 96)

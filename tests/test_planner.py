@@ -26,6 +26,10 @@ def _ops_from_chain(chain):
             out.append(sm.make_op(sm.OP_WINDOW_PARTITION, window=o["window"]))
         elif k == "window_reverse":
             out.append(sm.make_op(sm.OP_WINDOW_REVERSE, window=o["window"], shape=(o["B"], o["H"], o["W"])))
+        elif k == "depth_to_space":
+            out.append(sm.make_op(sm.OP_DEPTH_TO_SPACE, window=o["block"]))
+        elif k == "space_to_depth":
+            out.append(sm.make_op(sm.OP_SPACE_TO_DEPTH, window=o["block"]))
     return out
 
 
@@ -69,6 +73,9 @@ def test_table3_quadrants():
     assert sm.smartmem_op_quadrant(sm.OP_TRANSPOSE) == ILD_FIX
     assert sm.smartmem_op_quadrant(sm.OP_SLICE) == ILI_FIX
     assert sm.smartmem_op_quadrant(sm.OP_ROLL) == ILI_FIX        # Gather class
+    assert sm.smartmem_op_quadrant(sm.OP_DEPTH_TO_SPACE) == ILD_FIX    # DtoS
+    assert sm.smartmem_op_quadrant(sm.OP_SPACE_TO_DEPTH) == ILD_FIX    # StoD
+    assert sm.smartmem_op_quadrant(sm.OP_LAYERNORM) == ILD_VAR
 
 
 def test_tables_5_and_6_all_cells():
@@ -316,3 +323,83 @@ def test_placement_modes_reject_what_they_cannot_invert():
     ops = [sm.make_op(sm.OP_LINEAR, side_input=(1, 0))]
     with pytest.raises(sm.SmartmemError):
         sm.smartmem_plan(ops, [sm.make_desc((8, 8)), sm.make_desc((8, 8))], sm.ELIMINATE_SCATTER)   # copy-only chains
+
+
+# ------------------------------------------------------------------ DtoS / StoD, LayerNorm consumer
+@pytest.mark.parametrize("shape,chain", [
+    ((2, 12, 3, 4), [{"op": "depth_to_space", "block": 2}]),
+    ((2, 3, 4, 6), [{"op": "space_to_depth", "block": 2}]),
+    ((1, 18, 2, 2), [{"op": "depth_to_space", "block": 3}]),
+    ((2, 3, 4, 6), [{"op": "space_to_depth", "block": 2}, {"op": "depth_to_space", "block": 2}]),       # composes to the identity
+    ((2, 8, 4, 4), [{"op": "depth_to_space", "block": 2}, {"op": "transpose", "perm": (0, 2, 3, 1)}]),  # NCHW -> NHWC after it
+])
+def test_depth_space_maps(shape, chain):
+    m = _check_map_against_oracle(shape, chain)
+    assert m.klass in (0, 1)
+    if len(chain) == 2 and chain[0]["op"] == "space_to_depth" and chain[1]["op"] == "depth_to_space":
+        assert m.klass == 0
+
+
+def test_depth_space_shape_errors():
+    for op, shape in ((sm.OP_DEPTH_TO_SPACE, (1, 6, 2, 2)), (sm.OP_SPACE_TO_DEPTH, (1, 2, 3, 4)), (sm.OP_SPACE_TO_DEPTH, (2, 4, 4))):
+        with pytest.raises(sm.SmartmemError) as e:
+            sm.smartmem_plan([sm.make_op(op, window=2), sm.make_op(sm.OP_COPY)], [sm.make_desc(shape)], sm.ELIMINATE)
+        assert e.value.code == sm.ERR_SHAPE
+
+
+def _patch_merge_ops(B, H, W, C):
+    return [sm.make_op(sm.OP_RESHAPE, shape=(B, H // 2, 2, W // 2, 2, C)), sm.make_op(sm.OP_TRANSPOSE, perm=(0, 1, 3, 4, 2, 5)),
+            sm.make_op(sm.OP_RESHAPE, shape=(B, (H // 2) * (W // 2), 4 * C)),
+            sm.make_op(sm.OP_LAYERNORM, side_input=(1, 2), eps=1e-5), sm.make_op(sm.OP_LINEAR, side_input=(3, 0))]
+
+
+def test_patch_merging_plan_folds_the_gather_into_the_layernorm():
+    B, H, W, C = 2, 4, 6, 8
+    descs = [sm.make_desc((B, H, W, C)), sm.make_desc((4 * C,)), sm.make_desc((4 * C,)), sm.make_desc((2 * C, 4 * C))]
+    ref = chains.source_offsets((B, H, W, C), [{"op": "reshape", "shape": (B, H // 2, 2, W // 2, 2, C)},
+                                               {"op": "transpose", "perm": (0, 1, 3, 4, 2, 5)},
+                                               {"op": "reshape", "shape": (B, (H // 2) * (W // 2), 4 * C)}]).reshape(-1)
+    plan = sm.smartmem_plan(_patch_merge_ops(B, H, W, C), descs, sm.ELIMINATE)
+    try:
+        assert sm.smartmem_plan_num_steps(plan) == (2, 0)                 # LayerNorm (gathering) + GEMM, no copy
+        m = sm.smartmem_plan_get_map(plan, 0)
+        assert m.vec_elems == 8 and m.klass == 1
+        assert [sm.smartmem_map_eval(m, i) for i in range(ref.size)] == ref.tolist()
+        d = sm.smartmem_plan_output_desc(plan)
+        assert tuple(d.shape[: d.ndim]) == (B, (H // 2) * (W // 2), 2 * C)
+    finally:
+        sm.smartmem_plan_destroy(plan)
+    plan = sm.smartmem_plan(_patch_merge_ops(B, H, W, C), descs, sm.EXPLICIT)
+    try:
+        assert sm.smartmem_plan_num_steps(plan) == (3, 1)                 # one materialised transpose
+        assert sm.smartmem_plan_get_map(plan, 1).klass == 0
+    finally:
+        sm.smartmem_plan_destroy(plan)
+    # channels that do not fill a 16-byte vector: ELIMINATE materialises the gather too
+    descs6 = [sm.make_desc((B, H, W, 6)), sm.make_desc((24,)), sm.make_desc((24,)), sm.make_desc((12, 24))]
+    plan = sm.smartmem_plan(_patch_merge_ops(B, H, W, 6), descs6, sm.ELIMINATE)
+    try:
+        assert sm.smartmem_plan_num_steps(plan) == (3, 1)
+    finally:
+        sm.smartmem_plan_destroy(plan)
+
+
+def test_layernorm_consumer_argument_errors():
+    B, H, W, C = 1, 2, 2, 8
+    ops = _patch_merge_ops(B, H, W, C)
+    good = [sm.make_desc((B, H, W, C)), sm.make_desc((4 * C,)), sm.make_desc((4 * C,)), sm.make_desc((2 * C, 4 * C))]
+    bad_gamma = list(good)
+    bad_gamma[1] = sm.make_desc((4 * C + 8,))
+    with pytest.raises(sm.SmartmemError) as e:
+        sm.smartmem_plan(ops, bad_gamma, sm.ELIMINATE)
+    assert e.value.code == sm.ERR_SHAPE
+    ops0 = list(ops)
+    ops0[3] = sm.make_op(sm.OP_LAYERNORM, side_input=(1, 2), eps=0.0)
+    with pytest.raises(sm.SmartmemError) as e:
+        sm.smartmem_plan(ops0, good, sm.ELIMINATE)
+    assert e.value.code == sm.ERR_INVALID_ARG
+    ops1 = list(ops)
+    ops1[3] = sm.make_op(sm.OP_LAYERNORM, side_input=(1, 9), eps=1e-5)
+    with pytest.raises(sm.SmartmemError) as e:
+        sm.smartmem_plan(ops1, good, sm.ELIMINATE)
+    assert e.value.code == sm.ERR_INVALID_ARG
