@@ -189,7 +189,7 @@ def run_reference(args):
 # The other configurations (parity-test cases): timed on request with --workload, same protocol.
 # ------------------------------------------------------------------------------------------------
 OTHER_WORKLOADS = ["swin_b_stage3_block_pair", "llama_attention_layer", "llama_decode_layer", "chain_2a_qkt", "chain_2b_gemm",
-                   "chain_2a_copy", "chain_2b_copy", "swin_shift_partition_copy"]
+                   "chain_2a_copy", "chain_2b_copy", "swin_shift_partition_copy", "depth_to_space_copy", "swin_t_patch_merging"]
 
 
 def _peaks_all():
@@ -301,9 +301,30 @@ def run_other(args):
                  ("decode_attention", 2 * B * (pos + 1) * hidden * 2 + 2 * X, 4 * B * (pos + 1) * hidden),
                  ("o_proj_gemm", 2 * X + hidden * hidden * 2, 2 * B * hidden * hidden)]
     else:
-        which = "2a" if "2a" in name else "2b" if "2b" in name else "e1"
-        inp = synth.chain_inputs(2, which if which != "e1" else "2a")
-        if which == "e1":
+        which = "2a" if "2a" in name else "2b" if "2b" in name else "d2s" if "depth" in name else "pm" if "patch" in name else "e1"
+        inp = synth.chain_inputs(2, which if which in ("2a", "2b") else "2a")
+        if which == "d2s":
+            # DepthToSpace (Table 3's DtoS) of an NCHW activation, block 2: [8,256,64,64] -> [8,64,128,128]
+            B, Cb, Hh, Ww = 8, 256, 64, 64
+            x = torch.from_numpy(synth.normal(0x5EED0007, 0, (B, Cb, Hh, Ww), dtype="bf16").view(np.int16).copy()).cuda().view(torch.bfloat16)
+            ops = [sm.make_op(sm.OP_DEPTH_TO_SPACE, window=2), sm.make_op(sm.OP_COPY)]
+            srcs, descs, oshape = [x], [sm.make_desc((B, Cb, Hh, Ww))], (B, Cb // 4, Hh * 2, Ww * 2)
+            model = [("copy_map", 2 * B * Cb * Hh * Ww * 2, 0)]
+            tokens = B * Hh * Ww
+        elif which == "pm":
+            # patch merging between stages 1 and 2 of Swin-T at the benchmark's batch: [32,56,56,96] -> [32,784,192]
+            B, Hh, Ww, C = 32, 56, 56, 96
+            mk = lambda tid, shape, std, mean: torch.from_numpy(synth.normal(0x5EED0008, tid, shape, std, mean, "bf16").view(np.int16).copy()).cuda().view(torch.bfloat16)
+            srcs = [mk(0, (B, Hh, Ww, C), 1.0, 0.0), mk(1, (4 * C,), 0.02, 1.0), mk(2, (4 * C,), 0.02, 0.0), mk(3, (2 * C, 4 * C), 0.02, 0.0)]
+            descs = [sm.make_desc((B, Hh, Ww, C)), sm.make_desc((4 * C,)), sm.make_desc((4 * C,)), sm.make_desc((2 * C, 4 * C))]
+            ops = [sm.make_op(sm.OP_RESHAPE, shape=(B, Hh // 2, 2, Ww // 2, 2, C)), sm.make_op(sm.OP_TRANSPOSE, perm=(0, 1, 3, 4, 2, 5)),
+                   sm.make_op(sm.OP_RESHAPE, shape=(B, (Hh // 2) * (Ww // 2), 4 * C)),
+                   sm.make_op(sm.OP_LAYERNORM, side_input=(1, 2), eps=1e-5), sm.make_op(sm.OP_LINEAR, side_input=(3, 0))]
+            oshape = (B, (Hh // 2) * (Ww // 2), 2 * C)
+            U = B * Hh * Ww * C * 2
+            model = [("layernorm_gather", 2 * U, 0), ("linear", U + 2 * C * 4 * C * 2 + U // 2, 2 * (B * Hh * Ww // 4) * 4 * C * 2 * C)]
+            tokens = B * Hh * Ww
+        elif which == "e1":
             # the shift o partition chain of the Swin-T stage-1 block on its own: [32,56,56,96] -> [2048,49,96]
             B, Hh, Ww, C, wsz, sh = 32, 56, 56, 96, 7, 3
             x = torch.from_numpy(synth.normal(0x5EED0003, 0, (B, Hh, Ww, C), dtype="bf16").view(np.int16).copy()).cuda().view(torch.bfloat16)
@@ -432,6 +453,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="smartmem", choices=["smartmem", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--images", type=int, default=0,
+                    help="default workload only: images per step instead of the workload's 32 (batch sweep; 0 = the workload)")
     ap.add_argument("--sequences", type=int, default=64,
                     help="llama_decode_layer only: sequences decoded per step (64 is the workload; smaller for profiler captures)")
     ap.add_argument("--workload", default=WORKLOAD["name"],
@@ -460,6 +483,8 @@ def main():
     sm.lib()
 
     w = WORKLOAD
+    if args.images:
+        w["B"] = args.images
     M = w["B"] * w["H"] * w["W"]
     inp = synth.swin_inputs(shard_seed(w["config_id"], rank), w["B"], w["H"], w["W"], w["C"], w["heads"], w["window"],
                             w["mlp_ratio"], w["dtype"])
@@ -470,8 +495,6 @@ def main():
     params = {k: dev(v) for k, v in inp.items() if k != "x"}
     x_host = torch.from_numpy(inp["x"].view("int16").copy()).view(torch.bfloat16).pin_memory()
     y_host = torch.empty_like(x_host).pin_memory()
-    xs = [x_host.cuda() for _ in range(N_SETS)]
-    ys = [torch.empty_like(xs[0]) for _ in range(N_SETS)]
     p = sm.SwinParams()
     p.dtype = sm.BF16
     p.B, p.H, p.W, p.C, p.heads, p.window, p.shift, p.mlp_ratio = (w["B"], w["H"], w["W"], w["C"], w["heads"], w["window"],
@@ -480,6 +503,11 @@ def main():
     for k, t in params.items():
         setattr(p, k, t.data_ptr())
     wsb = {m: sm.smartmem_swin_block_workspace_bytes(p, m) for m in (sm.ELIMINATE, sm.EXPLICIT)}
+    global N_SETS
+    if args.images:          # smaller batches: more rotating sets, so that a set is still evicted from L2 before its reuse
+        N_SETS = int(min(64, max(4, -(-1_100_000_000 // (2 * x_host.numel() * 2 + wsb[sm.EXPLICIT])))))
+    xs = [x_host.cuda() for _ in range(N_SETS)]
+    ys = [torch.empty_like(xs[0]) for _ in range(N_SETS)]
     wss = [torch.empty(wsb[sm.EXPLICIT], dtype=torch.uint8, device="cuda") for _ in range(N_SETS)]
     stream = torch.cuda.current_stream().cuda_stream
 
@@ -614,13 +642,15 @@ def main():
         if os.path.exists(tpath):
             with open(tpath) as f:
                 traffic = json.load(f).get(dom["kernel"])
+            if traffic is not None and w["B"] != 32:         # the capture is of the 32-image workload; traffic grows with the images
+                traffic = int(traffic * w["B"] / 32)
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_elim / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
             "config": {"workload": w["name"], "B_per_gpu": w["B"], "H": w["H"], "W": w["W"], "C": w["C"], "heads": w["heads"],
                        "window": w["window"], "shift": w["shift"], "mlp_ratio": w["mlp_ratio"], "mode": "eliminate",
-                       "l2": f"{N_SETS} rotating buffer sets (> 1 GB touched between reuses of a set)",
+                       "l2": f"{N_SETS} rotating buffer sets ({N_SETS * (2 * x_host.numel() * 2 + wsb[sm.EXPLICIT]) / 1e6:.0f} MB touched between reuses of a set)",
                        "parallelism": f"replicas x{world}" if world > 1 else "single gpu"},
             "explicit_variant": {"value": tokens * args.steps / (ms_expl * 1e-3), "unit": UNIT,
                                  "ms_per_step": ms_expl / args.steps, "speedup_of_eliminate": ms_expl / ms_elim},

@@ -83,6 +83,38 @@ __global__ void __launch_bounds__(256) copy_scatter_kernel(const __grid_constant
   *reinterpret_cast<V*>(dst + off * elem_size) = v;
 }
 
+// Affine map whose innermost consumer atom is SHORT (E <= 8 values, strided in the source) and whose next
+// atom is contiguous in the source -- the interleave of DepthToSpace / pixel shuffle, where neighbouring
+// output elements come from E different planes.  A thread loads one 16-byte vector from each of the E
+// planes (8 consecutive positions of the contiguous atom), interleaves them in registers and stores
+// 8 * E contiguous output elements: both sides move 16-byte vectors, nothing goes through shared memory.
+template <int E>
+__global__ void __launch_bounds__(256) copy_interleave16_kernel(const __grid_constant__ DevMap map, const uint16_t* __restrict__ src,
+                                                                uint16_t* __restrict__ dst, uint32_t n_units, long long stride_e) {
+  pdl_wait();
+  pdl_launch_dependents();
+  const uint32_t i = blockIdx.x * 256u + threadIdx.x;
+  if (i >= n_units) return;
+  const long long off = devmap_eval_unrolled(map, i);
+  uint32_t w[E][4];
+#pragma unroll
+  for (int j = 0; j < E; ++j) {
+    const uint4 v = *reinterpret_cast<const uint4*>(src + off + j * stride_e);
+    w[j][0] = v.x; w[j][1] = v.y; w[j][2] = v.z; w[j][3] = v.w;
+  }
+  uint32_t o[4 * E];
+#pragma unroll
+  for (int m = 0; m < 4 * E; ++m) {
+    // output elements 2m and 2m+1: element t = k * E + j is position k of plane j
+    const int k0 = (2 * m) / E, j0 = (2 * m) % E, k1 = (2 * m + 1) / E, j1 = (2 * m + 1) % E;
+    const uint32_t sel = ((k0 & 1) ? 0x32u : 0x10u) | (((k1 & 1) ? 0x76u : 0x54u) << 8);
+    o[m] = __byte_perm(w[j0][k0 >> 1], w[j1][k1 >> 1], sel);
+  }
+  uint4* d = reinterpret_cast<uint4*>(dst + (size_t)i * (8 * E));
+#pragma unroll
+  for (int j = 0; j < E; ++j) d[j] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+}
+
 // Affine map whose consumer-innermost atom I is strided in the source while another atom J is
 // source-contiguous: a 64 x 64 tile transpose of 2-byte elements through shared memory.  Loads are
 // 16-byte vectors along J, stores 16-byte vectors along I.
@@ -256,6 +288,26 @@ int launch_copy_map(const smartmem_index_map_t& map, int elem_size, const void* 
       count_launch();
       return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
       }
+    }
+  }
+  // fast path: short strided innermost atom over a contiguous one (register interleave)
+  if (map.klass == 1 && elem_size == 2 && n >= 2 && map.src_stride[n - 1] != 1 && map.src_stride[n - 2] == 1 &&
+      map.extent[n - 1] >= 2 && map.extent[n - 1] <= 4 && map.extent[n - 2] % 8 == 0 && map.base % 8 == 0 &&
+      map.src_stride[n - 1] % 8 == 0) {
+    bool ok = true;
+    for (int a = 0; a + 2 < n; ++a) ok = ok && map.src_stride[a] % 8 == 0;
+    const int E = (int)map.extent[n - 1];
+    const long long units = map.n_elements / (8 * E);
+    DevMap d;
+    if (ok && units < (1ll << 31) && make_devmap(map, 0, n - 1, 8, true, &d)) {
+      const unsigned grid = (unsigned)((units + 255) / 256);
+      const uint16_t* s16 = (const uint16_t*)src;
+      uint16_t* d16 = (uint16_t*)dst;
+      if (E == 2) launch_pdl(copy_interleave16_kernel<2>, dim3(grid), dim3(256), 0, st, d, s16, d16, (uint32_t)units, map.src_stride[n - 1]);
+      else if (E == 3) launch_pdl(copy_interleave16_kernel<3>, dim3(grid), dim3(256), 0, st, d, s16, d16, (uint32_t)units, map.src_stride[n - 1]);
+      else launch_pdl(copy_interleave16_kernel<4>, dim3(grid), dim3(256), 0, st, d, s16, d16, (uint32_t)units, map.src_stride[n - 1]);
+      count_launch();
+      return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
     }
   }
   // fast path: tiled transpose
