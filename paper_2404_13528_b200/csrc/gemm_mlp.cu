@@ -12,12 +12,19 @@
 // double-buffered in TMEM, so the output warps (bias, residual, row stores) overlap the next tile.
 //
 // Warp roles: 0 TMA producer (A tile double-buffered across tiles, weights streamed from L2 through
-// a 4-stage ring in the order the two issuers consume them), 1 fc1 issuer + TMEM owner, 2-17 GELU,
-// 18-21 output, 22 fc2 issuer, 23-26 LayerNorm.
+// a 4-stage ring in the order the two issuers consume them), 1 fc1 issuer + TMEM owner, 2-9 GELU
+// (two warps per TMEM lane quadrant, 64 hidden columns each), 10-13 output, 14 fc2 issuer, 15-18
+// LayerNorm.
 //
 // What bounds it (clock-stamped build, -DMLP_EXP_TIMING): the loop fc1(j) -> GELU(j) -> fc2(j) ->
-// fc1(j+2) over the two S1/H buffers, about 2500 cycles per chunk; the floor under that is the
-// special-function unit (tanh at 16 elements per clock per SM: about 1000 cycles per chunk).
+// fc1(j+2) over the two S1/H buffers, about 2500 cycles per chunk.  The arithmetic in it is short
+// (with the GELU arithmetic compiled out the chunk period stays near 2400 cycles and the kernel
+// is only 15 % faster); most of it is the three hand-offs of the loop, each of which waits for the
+// slowest of eight warps or for an issuer thread to be scheduled.  A variant with H in a buffer of
+// its own (so that fc1(j+2) need not wait for fc2(j), but the H store waits for fc2(j-1)) ran at
+// the same speed; a third S1 buffer does not fit the 512 columns next to the double-buffered
+// output.  The floor under all of it is the special-function unit (tanh at 16 elements per clock
+// per SM: about 1000 cycles per chunk).
 
 #include "gemm_tc.cuh"
 #include "ptx.cuh"
@@ -42,7 +49,7 @@ constexpr int KB_BYTES = BM * BK * 2;              // one 128 x 64 bf16 operand 
 constexpr int NST = 4;                             // weight ring stages; one stage = both k-blocks of a chunk's W1 or W2
 constexpr int WST_BYTES = 2 * KB_BYTES;
 constexpr int kGeluWarps = 8, kOutWarps = 4, kNormWarps = 4, kThreads = 32 * (3 + kGeluWarps + kOutWarps + kNormWarps);
-constexpr uint32_t TM_S1 = 0, TM_OUT = 256, OUT_STRIDE = 96, TM_H = 448, TMEM_COLS = 512;   // S1 x2 (128), OUT x2 (96), H (64 packed columns)
+constexpr uint32_t TM_S1 = 0, TM_OUT = 256, OUT_STRIDE = 96, TMEM_COLS = 512;   // S1 x2 (128; H is written over its own S1 buffer), OUT x2 (96)
 constexpr int SMEM_TILES = (4 + 2 * NST) * KB_BYTES;         // A (2 buffers), weight ring
 constexpr int N_BARS = 4 + 2 * NST + 2 + 2 + 2 + 4 + 2;
 
@@ -121,8 +128,8 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       ptx::mbar_init(&a_full[i], 1);
       ptx::mbar_init(&a_empty[i], 1);
       ptx::mbar_init(&s1_full[i], 1);
-      ptx::mbar_init(&s1_empty[i], kGeluWarps);
-      ptx::mbar_init(&h_full[i], i == 0 ? kGeluWarps : 1);   // [0]: H written (GELU warps); [1]: H consumed (fc2 commit)
+      ptx::mbar_init(&s1_empty[i], 1);                       // fc2 of the chunk has consumed the buffer (its H)
+      ptx::mbar_init(&h_full[i], kGeluWarps);                // H of buffer i written (GELU warps)
       ptx::mbar_init(&out_full[i], 1);
       ptx::mbar_init(&out_empty[i], kOutWarps);
       ptx::mbar_init(&a_ready[i], kNormWarps);
@@ -246,7 +253,8 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const uint32_t ob = it2 & 1;
         const uint32_t n = j + 1 < total ? 2 * j + 2 : 2 * j + 1, ws = n % NST, wph = (n / NST) & 1;
         DBG(j * 16 + 4);
-        ok = ptx::mbar_wait(&h_full[0], j & 1, abort_flag, g.status);
+        const uint32_t sb = j & 1;
+        ok = ptx::mbar_wait(&h_full[sb], (j >> 1) & 1, abort_flag, g.status);
         if (c2 == 0) ok = ok && ptx::mbar_wait(&out_empty[ob], ((it2 >> 1) & 1) ^ 1, abort_flag, g.status);
         DBG(j * 16 + 5);
         ok = ok && ptx::mbar_wait(&w_full[ws], wph, abort_flag, g.status);
@@ -254,14 +262,16 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         DBG(j * 16 + 6);
         ptx::tc_fence_after();
         const uint32_t d = tmem_base + TM_OUT + ob * OUT_STRIDE;
-        const uint32_t a = tmem_base + TM_H;               // H chunk: 128 bf16 per lane = 64 columns
+        // H chunk: 128 bf16 per lane, written by the GELU warps over the S1 buffer it was computed from --
+        // hidden columns 0..63 as 32 packed columns at offset 0, columns 64..127 at offset 64
+        const uint32_t a = tmem_base + TM_S1 + sb * HC;
         const uint64_t bd = ptx::make_smem_desc(w_base + ws * WST_BYTES, 16, 1024);
         ptx::tc_mma_bf16_ta(d, a, bd, idesc2, c2 != 0 ? 1u : 0u);
 #pragma unroll
         for (int k = 1; k < HC / 16; ++k)               // 16 hidden columns = 8 packed TMEM columns per step
-          ptx::tc_mma_bf16_ta(d, a + 8 * k, bd + (k >> 2) * (KB_BYTES >> 4) + 2 * (k & 3), idesc2, 1u);
+          ptx::tc_mma_bf16_ta(d, a + 8 * k + (k >= 4 ? 32 : 0), bd + (k >> 2) * (KB_BYTES >> 4) + 2 * (k & 3), idesc2, 1u);
         ptx::tc_commit(&w_empty[ws]);
-        ptx::tc_commit(&h_full[1]);                     // H consumed: the GELU warps may write the next chunk
+        ptx::tc_commit(&s1_empty[sb]);                  // buffer consumed: fc1 of chunk j + 2 may overwrite it
         DBG(j * 16 + 7);
         if (++c2 == NC) {
           ptx::tc_commit(&out_full[ob]);
@@ -272,9 +282,9 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     }
   } else if (warp < 2 + kGeluWarps) {
     // GELU warps: S1 chunk (TMEM, fp32) -> + b1 -> GELU -> bf16 pairs -> the H region of TMEM, where
-    // fc2 reads the chunk as its A operand.  The S1 buffer is handed back as soon as it is in
-    // registers, so fc1 of chunk j+2 does not wait for fc2 of chunk j; H is single-buffered, and only
-    // its store waits for fc2 of the previous chunk.
+    // fc2 reads the chunk as its A operand.  H overwrites (half of) the S1 columns it was computed from,
+    // so each of the two S1 buffers carries its chunk from fc1 through GELU to fc2 and is handed back to
+    // fc1 by fc2's commit; the GELU warps themselves wait for nothing but the next fc1 result.
     const int e = warp - 2, q = warp & 3, hh = e >> 2;   // quadrant, half of the chunk's 128 columns
     bool ok = true;
     int c = 0;
@@ -291,9 +301,6 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       ptx::tmem_ld32(tq, rv);
       ptx::tmem_ld32(tq + 32, rv + 32);
       ptx::tmem_ld_wait();
-      ptx::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(&s1_empty[sb]);
       if (e == 0 && lane == 0) DBG(j * 16 + 10);
       uint32_t pk[32];
 #pragma unroll
@@ -307,15 +314,14 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         pk[2 * v + 1] = gelu_tanh_bf16x2(__uint_as_float(rv[4 * v + 2]) + b4.z, __uint_as_float(rv[4 * v + 3]) + b4.w);
 #endif
       }
-      ok = ptx::mbar_wait(&h_full[1], (j & 1) ^ 1, abort_flag, g.status);   // fc2 of the previous chunk has read H
-      if (!ok) break;
-      ptx::tc_fence_after();
-      ptx::tmem_st32(tmem_base + TM_H + ((uint32_t)(q * 32) << 16) + hh * 32, pk);
+      // the packed result goes over the first 32 of the 64 columns this warp has just read (it is the only
+      // reader and writer of them), so no warp ever waits for fc2 of an earlier chunk
+      ptx::tmem_st32(tq, pk);
       ptx::tmem_st_wait();
       if (e == 0 && lane == 0) DBG(j * 16 + 11);
       ptx::tc_fence_before();
       __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(&h_full[0]);
+      if (lane == 0) ptx::mbar_arrive(&h_full[sb]);
       if (++c == NC) c = 0;
     }
   } else if (warp < 2 + kGeluWarps + kOutWarps) {
