@@ -83,6 +83,34 @@ def test_decode_step_llama_size_sampled_sequences():
     check_case(41, 8, 2047, 2048, 4096, 32, 0, sample=[0, 3, 7])
 
 
+def test_decode_step_benchmark_launch_configuration():
+    """The benchmark's launch: 64 sequences x 2047 cached positions, hidden 4096.  The cache of four seeded
+    sequences is repeated 16 times on the device (every sequence still has its own new token), and the oracle
+    checks sequences that cover all four cache copies and both ends of the batch."""
+    B, B0, pos, s_max, hidden, heads = 64, 4, 2047, 2048, 4096, 32
+    D = hidden // heads
+    inp = synth.decode_inputs(43, B0, pos, hidden, heads)
+    x = synth.normal(synth.SEED_BASE + 43, 6, (B, hidden), 1.0, 0.0, "bf16")
+    dev = {k: to_dev(inp[k]) for k in ("rms_g", "w_qkv", "w_o")}
+    dev["x"] = to_dev(x)
+    kc0, vc0 = to_dev(inp["k_cache"]), to_dev(inp["v_cache"])
+    rows = [0, 1, 22, 43, 63]
+    pf = {k: synth.to_f64(inp[k]) for k in ("rms_g", "w_qkv", "w_o")}
+    y_ref, k_ref, v_ref = ollama.decode_step(synth.to_f64(x)[rows], synth.to_f64(inp["k_cache"])[[r % B0 for r in rows]],
+                                             synth.to_f64(inp["v_cache"])[[r % B0 for r in rows]], pf, heads=heads, head_dim=D)
+    for mode in (sm.ELIMINATE, sm.EXPLICIT):
+        kc = physical_cache(kc0.repeat(B // B0, 1, 1, 1), s_max, mode)
+        vc = physical_cache(vc0.repeat(B // B0, 1, 1, 1), s_max, mode)
+        y = run_decode(dev, kc, vc, B=B, pos=pos, s_max=s_max, hidden=hidden, heads=heads, add_residual=0, mode=mode)
+        assert_close_bf16(to_host_f64(y)[rows], y_ref, f"y, mode {mode}")
+        assert_close_bf16(to_host_f64(logical_view(kc, mode)[:, pos])[rows], k_ref, f"appended k, mode {mode}")
+        assert_close_bf16(to_host_f64(logical_view(vc, mode)[:, pos])[rows], v_ref, f"appended v, mode {mode}")
+        # sequences that share a cache copy and differ only in their new token must differ in y
+        assert not torch.equal(y[0], y[4])
+        del kc, vc
+        torch.cuda.empty_cache()
+
+
 def test_decode_rejects_bad_arguments():
     inp = synth.decode_inputs(42, 2, 3, 256, 2)
     dev = {k: to_dev(v) for k, v in inp.items()}
