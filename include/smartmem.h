@@ -159,6 +159,25 @@ int smartmem_op_quadrant(int32_t op_kind, int32_t* quadrant);
 int smartmem_pair_decision(int32_t first_quadrant, int32_t second_quadrant, int32_t* action,
                            int32_t* result, int32_t* search);
 
+/* Reduction-dimension layout selection for a producer with several consumers (Section 3.2.2, "Global:
+ * layout selections based on reduction dimension"; host only).  The producer's result has `ndim`
+ * dimensions; consumer c aggregates along producer dimension reduction_dim[c] (-1: no requirement) and
+ * counts with weight[c] > 0 (null: all 1; e.g. how often it runs or how many bytes it reads).  `k` is
+ * the number of memory dimensions that can be walked contiguously without index arithmetic (1 for
+ * linear memory, 2 for the paper's 2.5D texture memory).
+ *   Layout 0 serves the k most demanded reduction dimensions (demand = summed weight; ties go to the
+ * dimension that is already innermost-most): they become its k innermost dimensions, the most demanded
+ * one innermost (contiguous); all other dimensions keep their relative order outside.  Consumers whose
+ * reduction dimension is not among them are served by further copies of the tensor ("several copies of
+ * data with different layouts"), layout 1 taking the next k most demanded dimensions, and so on.
+ *   Outputs: *n_layouts; perm[l * SMARTMEM_MAX_DIMS + p] = producer dimension stored at position p of
+ * layout l (position 0 outermost, ndim-1 contiguous); layout_of_consumer[c] = the layout consumer c reads
+ * (0 for consumers without a requirement).  Errors: INVALID_ARG (null, ndim or k out of range, a
+ * reduction dimension >= ndim, weight <= 0), UNSUPPORTED (more than max_layouts layouts needed). */
+int smartmem_select_layouts(int32_t ndim, int32_t n_consumers, const int32_t* reduction_dim, const int64_t* weight,
+                            int32_t k, int32_t max_layouts, int32_t* n_layouts, int32_t* perm,
+                            int32_t* layout_of_consumer);
+
 /* Host only (no CUDA call).  Walks the chain, splits it at compute operators, and for each
  * maximal run of layout operators composes the index map (ELIMINATE) or emits one copy
  * step per data-moving layout operator (EXPLICIT; a Reshape of a contiguous tensor stays

@@ -60,7 +60,7 @@ class AttnParams(C.Structure):
 
 
 EXPORTED = [
-    "smartmem_op_quadrant", "smartmem_pair_decision", "smartmem_plan", "smartmem_plan_destroy",
+    "smartmem_op_quadrant", "smartmem_pair_decision", "smartmem_select_layouts", "smartmem_plan", "smartmem_plan_destroy",
     "smartmem_plan_num_steps", "smartmem_plan_get_map", "smartmem_plan_output_desc",
     "smartmem_plan_workspace_bytes", "smartmem_map_eval", "smartmem_plan_eval_sequential", "smartmem_run_chain",
     "smartmem_swin_block_workspace_bytes", "smartmem_swin_block", "smartmem_attn_layer_workspace_bytes",
@@ -85,6 +85,7 @@ def lib() -> C.CDLL:
     sig = {
         "smartmem_op_quadrant": (C.c_int, [i32, P(i32)]),
         "smartmem_pair_decision": (C.c_int, [i32, i32, P(i32), P(i32), P(i32)]),
+        "smartmem_select_layouts": (C.c_int, [i32, i32, P(i32), P(i64), i32, i32, P(i32), P(i32), P(i32)]),
         "smartmem_plan": (C.c_int, [P(Op), i32, P(TensorDesc), i32, i32, P(vp)]),
         "smartmem_plan_destroy": (C.c_int, [vp]),
         "smartmem_plan_num_steps": (C.c_int, [vp, P(i32), P(i32)]),
@@ -169,6 +170,18 @@ def smartmem_op_quadrant(kind: int) -> int:
     q = C.c_int32()
     _check(lib().smartmem_op_quadrant(kind, C.byref(q)), "smartmem_op_quadrant")
     return q.value
+
+
+def smartmem_select_layouts(ndim: int, reduction_dims, weights=None, k: int = 1, max_layouts: int = MAX_DIMS):
+    """Returns (layouts, layout_of_consumer): layouts[l] = producer dimensions from outermost to contiguous."""
+    n = len(reduction_dims)
+    rd = (C.c_int32 * n)(*[int(v) for v in reduction_dims])
+    w = None if weights is None else (C.c_int64 * n)(*[int(v) for v in weights])
+    nl = C.c_int32()
+    perm = (C.c_int32 * (max_layouts * MAX_DIMS))()
+    loc = (C.c_int32 * n)()
+    _check(lib().smartmem_select_layouts(ndim, n, rd, w, k, max_layouts, C.byref(nl), perm, loc), "smartmem_select_layouts")
+    return [[perm[l * MAX_DIMS + p] for p in range(ndim)] for l in range(nl.value)], list(loc)
 
 
 def smartmem_pair_decision(first: int, second: int):

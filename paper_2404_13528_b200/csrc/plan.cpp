@@ -583,6 +583,44 @@ int smartmem_pair_decision(int32_t a, int32_t b, int32_t* action, int32_t* resul
   return SMARTMEM_OK;
 }
 
+int smartmem_select_layouts(int32_t ndim, int32_t n_consumers, const int32_t* reduction_dim, const int64_t* weight,
+                            int32_t k, int32_t max_layouts, int32_t* n_layouts, int32_t* perm, int32_t* layout_of_consumer) {
+  if (!reduction_dim || !n_layouts || !perm || !layout_of_consumer) return SMARTMEM_ERR_INVALID_ARG;
+  if (ndim < 1 || ndim > SMARTMEM_MAX_DIMS || n_consumers < 1 || k < 1 || k > ndim || max_layouts < 1)
+    return SMARTMEM_ERR_INVALID_ARG;
+  int64_t demand[SMARTMEM_MAX_DIMS] = {0};
+  for (int c = 0; c < n_consumers; ++c) {
+    if (reduction_dim[c] >= ndim || reduction_dim[c] < -1) return SMARTMEM_ERR_INVALID_ARG;
+    const int64_t w = weight ? weight[c] : 1;
+    if (w <= 0) return SMARTMEM_ERR_INVALID_ARG;
+    if (reduction_dim[c] >= 0) demand[reduction_dim[c]] += w;
+  }
+  // demanded dimensions, most demanded first; ties: the one nearer the contiguous end of the natural order
+  std::vector<int> order;
+  for (int d = 0; d < ndim; ++d)
+    if (demand[d] > 0) order.push_back(d);
+  std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return demand[a] != demand[b] ? demand[a] > demand[b] : a > b; });
+  const int need = order.empty() ? 1 : (int)((order.size() + k - 1) / k);
+  if (need > max_layouts) return SMARTMEM_ERR_UNSUPPORTED;
+  int layout_of_dim[SMARTMEM_MAX_DIMS];
+  for (int d = 0; d < ndim; ++d) layout_of_dim[d] = -1;
+  for (int l = 0; l < need; ++l) {
+    std::vector<int> inner;                                   // this layout's served dimensions, most demanded first
+    for (int i = l * k; i < (l + 1) * k && i < (int)order.size(); ++i) {
+      inner.push_back(order[i]);
+      layout_of_dim[order[i]] = l;
+    }
+    int p = 0;
+    for (int d = 0; d < ndim; ++d)
+      if (std::find(inner.begin(), inner.end(), d) == inner.end()) perm[l * SMARTMEM_MAX_DIMS + p++] = d;
+    for (int i = (int)inner.size() - 1; i >= 0; --i) perm[l * SMARTMEM_MAX_DIMS + p++] = inner[i];   // most demanded last = contiguous
+    for (; p < SMARTMEM_MAX_DIMS; ++p) perm[l * SMARTMEM_MAX_DIMS + p] = -1;
+  }
+  for (int c = 0; c < n_consumers; ++c) layout_of_consumer[c] = reduction_dim[c] < 0 ? 0 : layout_of_dim[reduction_dim[c]];
+  *n_layouts = need;
+  return SMARTMEM_OK;
+}
+
 // Copy-only chains with the eliminated map placed explicitly on one side of the copy
 // (Section 3.2.2: a sub-optimal write is preferred to a sub-optimal read).  GATHER composes the chain
 // as usual and pins the plain map-driven kernel: out[i] = in[map(i)].  SCATTER inverts the chain
