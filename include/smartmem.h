@@ -266,11 +266,16 @@ int smartmem_swin_block_noalloc(const smartmem_swin_params_t* p, const void* x, 
                                 void* cuda_stream);
 
 /* One decoder attention layer, prefill.  x, y: [B,S,hidden], bf16.  w_qkv is [3*hidden, hidden]
- * with output columns ordered (q|k|v, head, head_dim); RoPE pairs (i, i + head_dim/2). */
+ * with output columns ordered (q|k|v, head, head_dim); RoPE pairs (i, i + R/2) over the first R =
+ * rotary_dim columns of every head at frequencies theta^(-2i/R), the other columns pass unrotated
+ * (rotary_dim 0 means head_dim: the whole head rotates; 32 and 64 are the partial-rotary layers of
+ * the Pythia / GPT-NeoX family, which the paper's evaluation includes). */
 typedef struct {
   int32_t dtype, B, S, hidden, heads, head_dim, causal, add_residual;
   float rms_eps, rope_theta;
   const void *rms_g, *w_qkv, *w_o;
+  int32_t rotary_dim;                /* 0 (= head_dim), 32, 64 or 128 */
+  int32_t reserved;                  /* zero */
 } smartmem_attn_params_t;
 int smartmem_attn_layer_workspace_bytes(const smartmem_attn_params_t* p, int32_t mode, size_t* bytes);
 int smartmem_attn_layer(const smartmem_attn_params_t* p, const void* x, void* y, void* workspace,

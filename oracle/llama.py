@@ -22,8 +22,8 @@ def causal_attention(q, k, v):
     return out
 
 
-def attn_layer(x, p, *, heads, head_dim, eps=1e-5, theta=10000.0, add_residual=False, keep=None):
-    """x [B,S,hidden] fp64 -> [B,S,hidden]."""
+def attn_layer(x, p, *, heads, head_dim, eps=1e-5, theta=10000.0, add_residual=False, keep=None, rotary_dim=None):
+    """x [B,S,hidden] fp64 -> [B,S,hidden].  rotary_dim: rotate only the first rotary_dim features of each head."""
     B, S, hidden = x.shape
     outs = []
     for b in range(B):
@@ -31,8 +31,12 @@ def attn_layer(x, p, *, heads, head_dim, eps=1e-5, theta=10000.0, add_residual=F
         qkv = ops.linear(xn, p["w_qkv"])                                          # L2 [S,3*hidden]
         t = layout.transpose(layout.reshape(qkv, (S, 3, heads, head_dim)), (1, 2, 0, 3))  # L3
         q, k, v = t[0], t[1], t[2]                                                # [H,S,D] each
-        q = ops.rope(q, theta)                                                    # L4
-        k = ops.rope(k, theta)
+        if rotary_dim is None:
+            q = ops.rope(q, theta)                                                # L4
+            k = ops.rope(k, theta)
+        else:
+            q = ops.rope_partial(q, theta, rotary_dim)
+            k = ops.rope_partial(k, theta, rotary_dim)
         o = causal_attention(q, k, v)                                             # L5
         om = layout.reshape(layout.transpose(o, (1, 0, 2)), (S, hidden))          # L6
         out = ops.linear(om, p["w_o"])                                            # L7
@@ -44,7 +48,7 @@ def attn_layer(x, p, *, heads, head_dim, eps=1e-5, theta=10000.0, add_residual=F
     return np.stack(outs)
 
 
-def decode_step(x, k_cache, v_cache, p, *, heads, head_dim, eps=1e-5, theta=10000.0, add_residual=False):
+def decode_step(x, k_cache, v_cache, p, *, heads, head_dim, eps=1e-5, theta=10000.0, add_residual=False, rotary_dim=None):
     """One decode step of the same layer for B independent sequences that all hold `pos` cached
     positions.  x [B,hidden]; k_cache, v_cache [B,pos,H,D] (keys already rotated, as the prefill left
     them).  Returns (y [B,hidden], k_new [B,H,D], v_new [B,H,D]): the new token sits at position
@@ -57,8 +61,12 @@ def decode_step(x, k_cache, v_cache, p, *, heads, head_dim, eps=1e-5, theta=1000
         xn = ops.rmsnorm(x[b:b + 1], p["rms_g"], eps)                              # [1,hidden]
         qkv = ops.linear(xn, p["w_qkv"])                                           # [1,3*hidden]
         t = layout.transpose(layout.reshape(qkv, (1, 3, heads, head_dim)), (1, 2, 0, 3))   # [3,H,1,D]
-        q = ops.rope_at(t[0], pos, theta)
-        k = ops.rope_at(t[1], pos, theta)
+        if rotary_dim is None:
+            q = ops.rope_at(t[0], pos, theta)
+            k = ops.rope_at(t[1], pos, theta)
+        else:
+            q = ops.rope_partial(t[0], theta, rotary_dim, pos=pos)
+            k = ops.rope_partial(t[1], theta, rotary_dim, pos=pos)
         v = t[2]
         K = np.concatenate([layout.transpose(k_cache[b], (1, 0, 2)), k], axis=1)   # [H,pos+1,D]
         V = np.concatenate([layout.transpose(v_cache[b], (1, 0, 2)), v], axis=1)

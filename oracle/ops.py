@@ -102,3 +102,22 @@ def rope_at(x: np.ndarray, pos: int, theta: float) -> np.ndarray:
         out[..., i] = x[..., i] * c - x[..., i + half] * sn
         out[..., i + half] = x[..., i + half] * c + x[..., i] * sn
     return out
+
+
+def rope_partial(x: np.ndarray, theta: float, rotary_dim: int, pos=None) -> np.ndarray:
+    """Partial rotary embedding (GPT-NeoX / Pythia style): the first `rotary_dim` = R features of a head rotate in
+    pairs (i, i + R/2) at frequencies theta^(-2i/R); features R.. pass through unchanged.  x [.., S, D]
+    with position = index along the second-to-last dim, or, when `pos` is given, x [.., D] all at that position."""
+    R = rotary_dim
+    out = x.copy()
+    for i in range(R // 2):
+        f = theta ** (-(2.0 * i) / R)
+        if pos is None:
+            phi = np.arange(x.shape[-2], dtype=np.float64) * f          # [S], broadcasts over leading dims
+        else:
+            phi = float(pos) * f
+        c, sn = np.cos(phi), np.sin(phi)
+        a, b = x[..., i], x[..., i + R // 2]
+        out[..., i] = a * c - b * sn
+        out[..., i + R // 2] = b * c + a * sn
+    return out

@@ -56,7 +56,8 @@ class SwinParams(C.Structure):
 class AttnParams(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("dtype", "B", "S", "hidden", "heads", "head_dim", "causal", "add_residual")] + \
                [("rms_eps", C.c_float), ("rope_theta", C.c_float)] + \
-               [(n, C.c_void_p) for n in ("rms_g", "w_qkv", "w_o")]
+               [(n, C.c_void_p) for n in ("rms_g", "w_qkv", "w_o")] + \
+               [("rotary_dim", C.c_int32), ("reserved", C.c_int32)]
 
 
 EXPORTED = [

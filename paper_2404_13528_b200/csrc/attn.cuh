@@ -41,9 +41,10 @@ struct CausalAttnArgs {
 };
 int launch_causal_attention(const CausalAttnArgs& a, cudaStream_t st);
 // Rotary embedding: (cos, sin) table [S, head_dim/2] as float2, and the stand-alone in-place
-// rotation of rows [rows, head_dim] (position = row % S) used by the explicit variant.
+// rotation of rows [rows, head_dim] (position = row % S) used by the explicit variant.  With a partial
+// rotary dimension R the table is built for "head_dim" = R and only the first R elements of a row rotate.
 int launch_rope_table(float* tab, int S, int head_dim, float theta, cudaStream_t st);
-int launch_rope_rows(void* x, long long rows, int S, int head_dim, const float* tab, cudaStream_t st);
+int launch_rope_rows(void* x, long long rows, int S, int head_dim, const float* tab, cudaStream_t st, int rotary_dim = 0);
 
 // out[M,N] = A[M,K] W[N,K]^T (+bias)(GELU)(+residual), fp32 with plain FMAs.  Rows of A may be
 // gathered through `amap`, rows of out scattered through `omap` (residual uses the same offsets).

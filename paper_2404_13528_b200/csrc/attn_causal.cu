@@ -195,10 +195,10 @@ __global__ void rope_table_kernel(float2* tab, int S, int half, double theta) {
 }
 
 // Stand-alone rotary embedding (explicit variant): rows of [R, D] with position = row % S.
-__global__ void rope_rows_kernel(__nv_bfloat16* x, long long rows, int S, int Dh, const float2* __restrict__ tab) {
+__global__ void rope_rows_kernel(__nv_bfloat16* x, long long rows, int S, int Dh, int rot, const float2* __restrict__ tab) {
   pdl_wait();
   pdl_launch_dependents();
-  const int half = Dh / 2;
+  const int half = rot / 2;                     // pairs (i, i + rot/2) of the first rot elements of a row of Dh
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= rows * half) return;
   const long long r = idx / half;
@@ -247,10 +247,11 @@ int launch_rope_table(float* tab, int S, int head_dim, float theta, cudaStream_t
   return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
 }
 
-int launch_rope_rows(void* x, long long rows, int S, int head_dim, const float* tab, cudaStream_t st) {
-  const long long n = rows * (head_dim / 2);
+int launch_rope_rows(void* x, long long rows, int S, int head_dim, const float* tab, cudaStream_t st, int rotary_dim) {
+  const int rot = rotary_dim ? rotary_dim : head_dim;
+  const long long n = rows * (rot / 2);
   profile_tick("rope_rows", st);
-  launch_pdl(rope_rows_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, st, (__nv_bfloat16*)x, rows, S, head_dim, (const float2*)tab);
+  launch_pdl(rope_rows_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, st, (__nv_bfloat16*)x, rows, S, head_dim, rot, (const float2*)tab);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
 }

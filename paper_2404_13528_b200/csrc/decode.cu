@@ -202,10 +202,10 @@ int launch_decode_attention(const DecodeAttnArgs& a, int B, cudaStream_t st) {
 }
 
 // Explicit variant: in-place rotary embedding of rows [R, 128] that all sit at position `pos`.
-__global__ void rope_rows_at_kernel(__nv_bfloat16* x, long long rows, int pos, double theta) {
+__global__ void rope_rows_at_kernel(__nv_bfloat16* x, long long rows, int pos, double theta, int rot) {
   pdl_wait();
   pdl_launch_dependents();
-  constexpr int half = DH / 2;
+  const int half = rot / 2;                     // pairs (i, i + rot/2) of the first rot elements of a row
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= rows * half) return;
   const long long r = idx / half;
@@ -231,10 +231,10 @@ __global__ void append_rows_kernel(const __nv_bfloat16* __restrict__ src, __nv_b
   *reinterpret_cast<uint4*>(dst + r * dst_row_stride + v * 8) = *reinterpret_cast<const uint4*>(src + r * DH + v * 8);
 }
 
-int launch_rope_rows_at(void* x, long long rows, int pos, float theta, cudaStream_t st) {
-  const long long n = rows * (DH / 2);
+int launch_rope_rows_at(void* x, long long rows, int pos, float theta, int rot, cudaStream_t st) {
+  const long long n = rows * (rot / 2);
   profile_tick("rope_rows", st);
-  launch_pdl(rope_rows_at_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, st, (__nv_bfloat16*)x, rows, pos, (double)theta);
+  launch_pdl(rope_rows_at_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, st, (__nv_bfloat16*)x, rows, pos, (double)theta, rot);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
 }
@@ -293,6 +293,7 @@ int validate(const smartmem_attn_params_t* p, int mode) {
   if (p->B < 1 || p->S < 1 || p->hidden < 1 || p->heads < 1) return SMARTMEM_ERR_SHAPE;
   if (p->heads * p->head_dim != p->hidden) return SMARTMEM_ERR_SHAPE;
   if (p->head_dim != DH || p->hidden % 256) return SMARTMEM_ERR_UNSUPPORTED;
+  if (p->rotary_dim != 0 && p->rotary_dim != 32 && p->rotary_dim != 64 && p->rotary_dim != 128) return SMARTMEM_ERR_UNSUPPORTED;
   return SMARTMEM_OK;
 }
 
@@ -354,6 +355,7 @@ EXPORT int smartmem_attn_decode(const smartmem_attn_params_t* pp, int32_t pos, c
       ep.rope_S = 1;
       ep.rope_pos0 = pos;
       ep.rope_log2_theta = log2f(p.rope_theta);
+      ep.rope_dim = p.rotary_dim ? p.rotary_dim : DH;
       ep.seg_cols = (int)hid;
       ep.seg_out[0] = at(L.qkv);              ep.seg_ld[0] = hid;
       ep.seg_out[1] = kc + (long long)pos * hid;   ep.seg_ld[1] = Smax * hid;
@@ -371,7 +373,7 @@ EXPORT int smartmem_attn_decode(const smartmem_attn_params_t* pp, int32_t pos, c
     SM_TRY(get_split(p.B, p.heads, DH, &split));
     SM_TRY(launch_copy_map(*split, 2, at(L.qkv), at(L.split), st));
     __nv_bfloat16* sp = (__nv_bfloat16*)at(L.split);
-    SM_TRY(launch_rope_rows_at(sp, 2 * B * H, pos, p.rope_theta, st));
+    SM_TRY(launch_rope_rows_at(sp, 2 * B * H, pos, p.rope_theta, p.rotary_dim ? p.rotary_dim : DH, st));
     SM_TRY(launch_append_rows(sp + B * hid, kc + (long long)pos * DH, B * H, Smax * DH, "append_k", st));
     SM_TRY(launch_append_rows(sp + 2 * B * hid, vc + (long long)pos * DH, B * H, Smax * DH, "append_v", st));
     a.q = sp;

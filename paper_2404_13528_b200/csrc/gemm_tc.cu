@@ -59,7 +59,8 @@ struct GemmArgs {
   const __nv_bfloat16* residual;
   int gelu, has_rowmap;
   int rope_cols, rope_S, rope_pos0;      // columns [0, rope_cols) are rotated; position = rope_pos0 + row % rope_S
-  float rope_c;                          // log2(theta) / 64
+  int rope_half;                         // R / 2: the first R columns of each 128-wide head rotate, pairs (i, i + R/2)
+  float rope_c;                          // log2(theta) / (R / 2)
   int seg_cols;                          // > 0: column segment s of a row goes to seg_out[s] + row * seg_ld[s]
   __nv_bfloat16* seg_out[3];
   long long seg_ld[3];
@@ -372,30 +373,36 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         {
           uint32_t rv[RC];
           ptx::tmem_ld_cols<RC>(taddr + c0, rv);
-          if (rope_tile) {
-            // rotary pairs are (c, c + 64) inside a 128-column head: round 0 holds the first half
-            // of the pair, round 1 the second; each round reads both halves from TMEM
+          // rotary pairs are (i, i + R/2) inside the first R columns of a 128-column head (R = 128: the
+          // whole head).  This round's RC columns start at head-local column hc0; they rotate iff hc0 < R,
+          // and their partners are the RC columns R/2 further up or down (or, when R/2 < RC, the other
+          // half of this very round), read from TMEM a second time.
+          const int hc0 = c0 & 127, half = g.rope_half;
+          if (rope_tile && hc0 < 2 * half) {
+            const bool in_round = half < RC;                 // R = 32 with 32-column rounds: pairs (j, j + 16) of this round
+            const bool first_half = hc0 < half;
             uint32_t rw[RC];
-            // (128-wide tile = one head: column groups 0, 1 hold the first halves, 2, 3 the second)
-            const bool first_half = BN == 256 ? rd < RH : grp < 2;
-            ptx::tmem_ld_cols<RC>(taddr + (first_half ? c0 + 64 : c0 - 64), rw);
+            if (!in_round) ptx::tmem_ld_cols<RC>(taddr + (first_half ? c0 + half : c0 - half), rw);
             ptx::tmem_ld_wait();
-            // angle = position * theta^(-i/64), reduced mod 2 pi in two steps, then the hardware
+            // angle = position * theta^(-i/(R/2)), reduced mod 2 pi in two steps, then the hardware
             // sine / cosine: no table traffic (a [S, 64] table read 16 bytes per lane per row
             // slowed the whole kernel by a fifth)
             const float pos = (float)(row_ok ? g.rope_pos0 + row % g.rope_S : 0);
-            const int i0 = (grp & 1) * 32 + (BN == 256 ? RC * (rd % RH) : 0);
+            const int i0 = in_round ? 0 : hc0 - (first_half ? 0 : half);
 #pragma unroll
             for (int j = 0; j < RC; ++j) {
+              const bool fh = in_round ? j < RC / 2 : first_half;
+              const int i = in_round ? (j & (RC / 2 - 1)) : i0 + j;
               float f;
-              asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(f) : "f"(-(float)(i0 + j) * g.rope_c));
+              asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(f) : "f"(-(float)i * g.rope_c));
               const float ang = pos * f;
               const float kk = rintf(ang * 0.15915494309189535f);
               float red = fmaf(-kk, 6.2831854820251465f, ang);
               red = fmaf(kk, 1.7484556e-7f, red);
               const float sn = __sinf(red), cs = __cosf(red);
-              const float x = __uint_as_float(rv[j]), y = __uint_as_float(rw[j]);
-              acc[j] = first_half ? x * cs - y * sn : x * cs + y * sn;
+              const float x = __uint_as_float(rv[j]);
+              const float y = __uint_as_float(in_round ? rv[j ^ (RC / 2)] : rw[j]);
+              acc[j] = fh ? x * cs - y * sn : x * cs + y * sn;
             }
           } else {
             ptx::tmem_ld_wait();
@@ -708,6 +715,7 @@ int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep,
   // once and is bound by how many SMs pull on it, so take the narrowest tile that divides N.
   if (ep.rope_cols == 0 && batch == 1 && M <= BM && !a_mn && N % 64 == 0 && N / bn < tc_sm_count()) bn = 64;
   if (ep.rope_cols > 0 && (N % 256 || ep.rope_cols % 256 || ep.rope_S < 1)) return SMARTMEM_ERR_UNSUPPORTED;
+  if (ep.rope_cols > 0 && ep.rope_dim != 0 && ep.rope_dim != 32 && ep.rope_dim != 64 && ep.rope_dim != 128) return SMARTMEM_ERR_UNSUPPORTED;
   if (ep.seg_cols > 0) {
     if (ep.seg_cols % 256 || N > 3ll * ep.seg_cols || ep.rowmap || ep.residual || batch != 1) return SMARTMEM_ERR_UNSUPPORTED;
     for (int i = 0; i * (long long)ep.seg_cols < N; ++i)
@@ -738,7 +746,9 @@ int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep,
   g.rope_pos0 = ep.rope_pos0;
   g.seg_cols = ep.seg_cols;
   for (int i = 0; i < 3; ++i) { g.seg_out[i] = (__nv_bfloat16*)ep.seg_out[i]; g.seg_ld[i] = ep.seg_ld[i]; }
-  g.rope_c = ep.rope_log2_theta / 64.0f;
+  const int rope_dim = ep.rope_dim ? ep.rope_dim : 128;
+  g.rope_half = rope_dim / 2;
+  g.rope_c = ep.rope_log2_theta / (float)(rope_dim / 2);
   g.status = device_status_ptr();
   if (!g.status) return SMARTMEM_ERR_CUDA;
   g.tiles_n = (int)((N + bn - 1) / bn);

@@ -29,6 +29,8 @@ struct TcEpilogue {
   int rope_cols, rope_S;     // rotate columns [0, rope_cols) in 128-wide heads; position = rope_pos0 + row % rope_S
   float rope_log2_theta;     // angle of pair i at position p: p * 2^(-i/64 * rope_log2_theta)
   int rope_pos0;
+  int rope_dim;              // rotary dimension R in {32, 64, 128} (0 = 128): only the first R columns of a head rotate,
+                             // in pairs (i, i + R/2), pair i at angle p * 2^(-i/(R/2) * rope_log2_theta)
   // Column-segmented output (seg_cols > 0, a multiple of 256; no rowmap, residual or batch): columns
   // [s*seg_cols, (s+1)*seg_cols) of row r go to seg_out[s] + r*seg_ld[s] (elements), s < 3.  `out`
   // and `ldc` are ignored.  Lets one GEMM store into several destinations of different pitch.

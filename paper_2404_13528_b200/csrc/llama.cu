@@ -75,6 +75,7 @@ int validate(const smartmem_attn_params_t* p, int mode) {
   if (p->heads * p->head_dim != p->hidden) return SMARTMEM_ERR_SHAPE;
   if (p->head_dim != 128 || !p->causal) return SMARTMEM_ERR_UNSUPPORTED;
   if (p->hidden % 256) return SMARTMEM_ERR_UNSUPPORTED;
+  if (p->rotary_dim != 0 && p->rotary_dim != 32 && p->rotary_dim != 64 && p->rotary_dim != 128) return SMARTMEM_ERR_UNSUPPORTED;
   return SMARTMEM_OK;
 }
 
@@ -112,14 +113,15 @@ EXPORT int smartmem_attn_layer(const smartmem_attn_params_t* pp, const void* x, 
   float* tab = (float*)at(L.tab);
 
 #define SM_TRY(expr) do { rc = (expr); if (rc != SMARTMEM_OK) return rc; } while (0)
-  if (!elim) SM_TRY(launch_rope_table(tab, (int)S, (int)D, p.rope_theta, st));   // only the stand-alone RoPE pass reads it
+  const int rot = p.rotary_dim ? p.rotary_dim : (int)D;
+  if (!elim) SM_TRY(launch_rope_table(tab, (int)S, rot, p.rope_theta, st));   // only the stand-alone RoPE pass reads it
   SM_TRY(launch_norm(SMARTMEM_BF16, true, x, at(L.xn), p.rms_g, nullptr, p.rms_eps, M, (int)hid, nullptr, st));
   {
     TcEpilogue ep;
     memset(&ep, 0, sizeof(ep));
     ep.out = at(L.qkv);
     ep.ldc = 3 * hid;
-    if (elim) { ep.rope_cols = (int)(2 * hid); ep.rope_S = (int)S; ep.rope_log2_theta = log2f(p.rope_theta); }
+    if (elim) { ep.rope_cols = (int)(2 * hid); ep.rope_S = (int)S; ep.rope_log2_theta = log2f(p.rope_theta); ep.rope_dim = rot; }
     SM_TRY(launch_gemm_tc(tc_operand_plain(at(L.xn), M, hid, hid), tc_operand_plain(p.w_qkv, 3 * hid, hid, hid), ep, 1, M,
                           3 * hid, hid, st));
   }
@@ -139,7 +141,7 @@ EXPORT int smartmem_attn_layer(const smartmem_attn_params_t* pp, const void* x, 
   } else {
     SM_TRY(launch_copy_map(mp->split, 2, at(L.qkv), at(L.split), st));
     char* sp = (char*)at(L.split);
-    SM_TRY(launch_rope_rows(sp, 2 * M * H, (int)S, (int)D, tab, st));
+    SM_TRY(launch_rope_rows(sp, 2 * M * H, (int)S, (int)D, tab, st, rot));
     const size_t one = (size_t)M * hid * 2;
     a.q = {sp, H * S * D, S * D, D, 1};
     a.k = {sp + one, H * S * D, S * D, D, 1};

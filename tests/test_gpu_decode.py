@@ -28,16 +28,17 @@ def logical_view(cache: torch.Tensor, mode: int) -> torch.Tensor:
     return cache if mode == sm.ELIMINATE else cache.permute(0, 2, 1, 3)
 
 
-def make_params(dev, B, s_max, hidden, heads, add_residual):
+def make_params(dev, B, s_max, hidden, heads, add_residual, rotary_dim=0):
     p = sm.AttnParams()
+    p.rotary_dim = rotary_dim
     p.dtype, p.B, p.S, p.hidden, p.heads, p.head_dim, p.causal, p.add_residual = sm.BF16, B, s_max, hidden, heads, hidden // heads, 1, add_residual
     p.rms_eps, p.rope_theta = 1e-5, 10000.0
     p.rms_g, p.w_qkv, p.w_o = dev["rms_g"].data_ptr(), dev["w_qkv"].data_ptr(), dev["w_o"].data_ptr()
     return p
 
 
-def run_decode(dev, kc, vc, *, B, pos, s_max, hidden, heads, add_residual, mode):
-    p = make_params(dev, B, s_max, hidden, heads, add_residual)
+def run_decode(dev, kc, vc, *, B, pos, s_max, hidden, heads, add_residual, mode, rotary_dim=0):
+    p = make_params(dev, B, s_max, hidden, heads, add_residual, rotary_dim)
     y = torch.full_like(dev["x"], float("nan"))
     n = sm.smartmem_attn_decode_workspace_bytes(p, mode)
     ws = torch.empty(n, dtype=torch.uint8, device="cuda")
@@ -46,7 +47,7 @@ def run_decode(dev, kc, vc, *, B, pos, s_max, hidden, heads, add_residual, mode)
     return y
 
 
-def check_case(config_id, B, pos, s_max, hidden, heads, add_residual, sample=None):
+def check_case(config_id, B, pos, s_max, hidden, heads, add_residual, sample=None, rotary_dim=0):
     D = hidden // heads
     inp = synth.decode_inputs(config_id, B, pos, hidden, heads)
     dev = {k: to_dev(v) for k, v in inp.items()}
@@ -54,11 +55,12 @@ def check_case(config_id, B, pos, s_max, hidden, heads, add_residual, sample=Non
     rows = list(range(B)) if sample is None else sample
     y_ref, k_ref, v_ref = ollama.decode_step(synth.to_f64(inp["x"])[rows], synth.to_f64(inp["k_cache"])[rows],
                                              synth.to_f64(inp["v_cache"])[rows], pf, heads=heads, head_dim=D,
-                                             add_residual=bool(add_residual))
+                                             add_residual=bool(add_residual), rotary_dim=rotary_dim or None)
     for mode in (sm.ELIMINATE, sm.EXPLICIT):
         kc = physical_cache(dev["k_cache"], s_max, mode)
         vc = physical_cache(dev["v_cache"], s_max, mode)
-        y = run_decode(dev, kc, vc, B=B, pos=pos, s_max=s_max, hidden=hidden, heads=heads, add_residual=add_residual, mode=mode)
+        y = run_decode(dev, kc, vc, B=B, pos=pos, s_max=s_max, hidden=hidden, heads=heads, add_residual=add_residual, mode=mode,
+                       rotary_dim=rotary_dim)
         assert_close_bf16(to_host_f64(y)[rows], y_ref, f"y, mode {mode}")
         for name, cache, src, ref in (("k", kc, dev["k_cache"], k_ref), ("v", vc, dev["v_cache"], v_ref)):
             lv = logical_view(cache, mode)
@@ -76,6 +78,11 @@ def check_case(config_id, B, pos, s_max, hidden, heads, add_residual, sample=Non
 ])
 def test_small_decode_steps(B, pos, s_max, hidden, heads, res):
     check_case(40, B, pos, s_max, hidden, heads, res)
+
+
+@pytest.mark.parametrize("rot", [32, 64])
+def test_partial_rotary_decode_steps(rot):
+    check_case(44, 3, 37, 64, 512, 4, 1, rotary_dim=rot)
 
 
 def test_decode_step_llama_size_sampled_sequences():

@@ -11,8 +11,9 @@ from tests.gpu_util import assert_close_bf16, check_status, stream, to_dev, to_h
 pytestmark = pytest.mark.gpu
 
 
-def run_layer(dev, *, B, S, hidden, heads, add_residual, mode):
+def run_layer(dev, *, B, S, hidden, heads, add_residual, mode, rotary_dim=0):
     p = sm.AttnParams()
+    p.rotary_dim = rotary_dim
     p.dtype, p.B, p.S, p.hidden, p.heads, p.head_dim, p.causal, p.add_residual = sm.BF16, B, S, hidden, heads, hidden // heads, 1, add_residual
     p.rms_eps, p.rope_theta = 1e-5, 10000.0
     p.rms_g, p.w_qkv, p.w_o = dev["rms_g"].data_ptr(), dev["w_qkv"].data_ptr(), dev["w_o"].data_ptr()
@@ -24,19 +25,38 @@ def run_layer(dev, *, B, S, hidden, heads, add_residual, mode):
     return y
 
 
-def case(config_id, B, S, hidden, heads, add_residual):
+def case(config_id, B, S, hidden, heads, add_residual, rotary_dim=0):
     inp = synth.attn_layer_inputs(config_id, S, hidden, B=B)
     dev = {k: to_dev(v) for k, v in inp.items()}
     pf = {k: synth.to_f64(v) for k, v in inp.items() if k != "x"}
-    ref = ollama.attn_layer(synth.to_f64(inp["x"]), pf, heads=heads, head_dim=hidden // heads, add_residual=bool(add_residual))
+    ref = ollama.attn_layer(synth.to_f64(inp["x"]), pf, heads=heads, head_dim=hidden // heads, add_residual=bool(add_residual),
+                            rotary_dim=rotary_dim or None)
     for mode in (sm.ELIMINATE, sm.EXPLICIT):
-        y = run_layer(dev, B=B, S=S, hidden=hidden, heads=heads, add_residual=add_residual, mode=mode)
+        y = run_layer(dev, B=B, S=S, hidden=hidden, heads=heads, add_residual=add_residual, mode=mode, rotary_dim=rotary_dim)
         assert_close_bf16(to_host_f64(y), ref, f"mode {mode}")
 
 
 @pytest.mark.parametrize("B,S,hidden,heads,res", [(1, 64, 256, 2, 0), (2, 200, 256, 2, 1), (1, 333, 512, 4, 0)])
 def test_small_attention_layers(B, S, hidden, heads, res):
     case(30, B, S, hidden, heads, res)
+
+
+@pytest.mark.parametrize("B,S,hidden,heads,rot", [
+    (1, 64, 256, 2, 32),        # one row tile, 128-column (one head) tiles, pairs inside a 32-column round
+    (2, 200, 256, 2, 64),       # 256-column tiles, 3-stage variant (32-column rounds)
+    (1, 200, 256, 2, 32),
+    (1, 150, 512, 4, 32),       # 4-stage variant (16-column rounds)
+    (1, 150, 512, 4, 64),
+    (1, 96, 512, 4, 128),       # rotary_dim = head_dim given explicitly
+])
+def test_partial_rotary_layers(B, S, hidden, heads, rot):
+    """Pythia / GPT-NeoX style: only the first rotary_dim features of a head rotate."""
+    case(32, B, S, hidden, heads, 0, rotary_dim=rot)
+
+
+def test_partial_rotary_layer_full_size():
+    """Config 5's shape with rotary_dim 32 (a quarter of the head, as in the Pythia family)."""
+    case(5, 1, 2048, 4096, 32, 0, rotary_dim=32)
 
 
 def test_config5_llama_style_layer_full_size():
@@ -53,3 +73,6 @@ def test_attn_layer_rejects_bad_arguments():
     with pytest.raises(sm.SmartmemError) as e:
         run_layer(dev, B=1, S=64, hidden=256, heads=3, add_residual=0, mode=sm.ELIMINATE)
     assert e.value.code == sm.ERR_SHAPE
+    with pytest.raises(sm.SmartmemError) as e:
+        run_layer(dev, B=1, S=64, hidden=256, heads=2, add_residual=0, mode=sm.ELIMINATE, rotary_dim=48)
+    assert e.value.code == sm.ERR_UNSUPPORTED

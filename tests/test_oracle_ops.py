@@ -343,3 +343,35 @@ def test_patch_merging_against_direct_restatement():
     # constant input: LayerNorm gives beta, so every token maps to w beta
     yc = swin.patch_merging(np.full((B, H, W, C), 2.5), g, b, w)
     assert np.allclose(yc, np.broadcast_to(w @ b, yc.shape), atol=1e-9)
+
+
+def test_rope_partial_pins():
+    """R = D is the full rotary embedding; for R < D the first R features equal the full embedding of a head of
+    dimension R and the rest pass through; the one-position form equals the matching row of the sequence form;
+    rotation preserves the norm of every pair."""
+    x = rng.standard_normal((2, 6, 16))
+    assert np.allclose(ops.rope_partial(x, 10000.0, 16), ops.rope(x, 10000.0), atol=1e-13)
+    for R in (4, 8):
+        y = ops.rope_partial(x, 10000.0, R)
+        assert np.allclose(y[..., :R], ops.rope(x[..., :R], 10000.0), atol=1e-13)
+        assert np.array_equal(y[..., R:], x[..., R:])
+        assert np.allclose(y[..., :R // 2] ** 2 + y[..., R // 2:R] ** 2, x[..., :R // 2] ** 2 + x[..., R // 2:R] ** 2)
+        for pos in (0, 3, 5):
+            assert np.allclose(ops.rope_partial(x[:, pos], 10000.0, R, pos=pos), y[:, pos], atol=1e-13)
+
+
+def test_partial_rotary_layer_and_decode_step_agree():
+    """With a partial rotary dimension the decode step still reproduces the prefill's last row."""
+    S, heads, D, R = 5, 2, 8, 4
+    hidden = heads * D
+    x = rng.standard_normal((1, S, hidden))
+    p = {"rms_g": 1 + 0.1 * rng.standard_normal(hidden), "w_qkv": 0.3 * rng.standard_normal((3 * hidden, hidden)),
+         "w_o": 0.3 * rng.standard_normal((hidden, hidden))}
+    keep = {}
+    full = llama.attn_layer(x, p, heads=heads, head_dim=D, keep=keep, rotary_dim=R)[0]
+    assert not np.allclose(full, llama.attn_layer(x, p, heads=heads, head_dim=D)[0])          # it is a different layer
+    kc = np.transpose(keep["k"][:, :S - 1], (1, 0, 2))[None]
+    vc = np.transpose(keep["v"][:, :S - 1], (1, 0, 2))[None]
+    y, kn, _ = llama.decode_step(x[:, S - 1], kc, vc, p, heads=heads, head_dim=D, rotary_dim=R)
+    assert np.allclose(y[0], full[S - 1], atol=1e-11)
+    assert np.allclose(kn[0], keep["k"][:, S - 1], atol=1e-12)
