@@ -189,7 +189,7 @@ def run_reference(args):
 # The other configurations (parity-test cases): timed on request with --workload, same protocol.
 # ------------------------------------------------------------------------------------------------
 OTHER_WORKLOADS = ["swin_b_stage3_block_pair", "llama_attention_layer", "llama_decode_layer", "chain_2a_qkt", "chain_2b_gemm",
-                   "chain_2a_copy", "chain_2b_copy", "swin_shift_partition_copy", "depth_to_space_copy", "swin_t_patch_merging"]
+                   "chain_2a_copy", "chain_2b_copy", "swin_shift_partition_copy", "depth_to_space_copy", "swin_t_patch_merging", "swin_t_stage1"]
 
 
 def _peaks_all():
@@ -250,6 +250,51 @@ def run_other(args):
                ("proj_gemm_scatter_residual", 3 * U + wp, 2 * M * C * C), ("ln2", 2 * U, 0),
                ("fc1_gemm_gelu", 5 * U + w1, 2 * M * C * 4 * C), ("fc2_gemm_residual", 6 * U + w1, 2 * M * C * 4 * C)]
         model = one + one
+    elif name == "swin_t_stage1":
+        # the whole first stage of Swin-T at the benchmark's batch: block (shift 0), block (shift 3), patch merging
+        B, H, W, C, heads, ws = 32, 56, 56, 96, 3, 7
+        M = B * H * W
+        U = M * C * 2
+        blocks = []
+        for wset, shift in ((0, 0), (1, 3)):
+            inp = synth.swin_inputs(7, B, H, W, C, heads, ws, 4, "bf16", weight_set=wset)
+            d = {k: dev(v) for k, v in inp.items()}
+            p = sm.SwinParams()
+            p.dtype = sm.BF16
+            p.B, p.H, p.W, p.C, p.heads, p.window, p.shift, p.mlp_ratio = B, H, W, C, heads, ws, shift, 4
+            p.ln_eps = 1e-5
+            for k, t in d.items():
+                if k != "x":
+                    setattr(p, k, t.data_ptr())
+            blocks.append((p, d))
+        pmw = [dev(synth.normal(0x5EED0007, tid, shape, 0.02, mean, "bf16")) for tid, shape, mean in
+               ((301, (4 * C,), 1.0), (302, (4 * C,), 0.0), (303, (2 * C, 4 * C), 0.0))]
+        pm_ops = [sm.make_op(sm.OP_RESHAPE, shape=(B, H // 2, 2, W // 2, 2, C)), sm.make_op(sm.OP_TRANSPOSE, perm=(0, 1, 3, 4, 2, 5)),
+                  sm.make_op(sm.OP_RESHAPE, shape=(B, (H // 2) * (W // 2), 4 * C)),
+                  sm.make_op(sm.OP_LAYERNORM, side_input=(1, 2), eps=1e-5), sm.make_op(sm.OP_LINEAR, side_input=(3, 0))]
+        pm_descs = [sm.make_desc((B, H, W, C)), sm.make_desc((4 * C,)), sm.make_desc((4 * C,)), sm.make_desc((2 * C, 4 * C))]
+        pm_plans = {m: sm.smartmem_plan(pm_ops, pm_descs, m) for m in (sm.ELIMINATE, sm.EXPLICIT)}
+        pm_wsb = {m: sm.smartmem_plan_workspace_bytes(pm_plans[m]) for m in pm_plans}
+        sets = 4
+        xs = [blocks[0][1]["x"].clone() for _ in range(sets)]
+        mid = [[torch.empty_like(xs[0]) for _ in range(2)] for _ in range(sets)]
+        ys = [torch.empty((B, (H // 2) * (W // 2), 2 * C), dtype=torch.bfloat16, device="cuda") for _ in range(sets)]
+        wsb = {m: max(sm.smartmem_swin_block_workspace_bytes(blocks[0][0], m), pm_wsb[m]) for m in (sm.ELIMINATE, sm.EXPLICIT)}
+        wss = [torch.empty(wsb[sm.EXPLICIT], dtype=torch.uint8, device="cuda") for _ in range(sets)]
+
+        def step(i, mode):
+            j = i % sets
+            sm.smartmem_swin_block(blocks[0][0], xs[j].data_ptr(), mid[j][0].data_ptr(), wss[j].data_ptr(), wsb[mode], mode, stream)
+            sm.smartmem_swin_block(blocks[1][0], mid[j][0].data_ptr(), mid[j][1].data_ptr(), wss[j].data_ptr(), wsb[mode], mode, stream)
+            sm.smartmem_run_chain(pm_plans[mode], [mid[j][1].data_ptr()] + [t.data_ptr() for t in pmw], [ys[j].data_ptr()],
+                                  wss[j].data_ptr(), wsb[mode], stream)
+        tokens = M
+        wq, wp, w1 = 3 * C * C * 2, C * C * 2, 4 * C * C * 2
+        one = [("ln1_gather_qkv_gemm", 4 * U + wq, 2 * M * C * 3 * C), ("window_attention", 4 * U, 4 * M * 49 * C),
+               ("proj_gemm_scatter_residual", 3 * U + wp, 2 * M * C * C),
+               ("mlp_fused_ln2_fc1_gelu_fc2_residual", 2 * U + 2 * w1, 2 * 2 * M * C * 4 * C)]
+        model = one + one + [("patch_merge_layernorm_gather", 2 * U, 0),
+                             ("patch_merge_linear", U + 2 * C * 4 * C * 2 + U // 2, 2 * (M // 4) * 4 * C * 2 * C)]
     elif name == "llama_attention_layer":
         S, hidden, heads = 2048, 4096, 32
         inp = synth.attn_layer_inputs(5, S, hidden)
