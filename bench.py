@@ -189,7 +189,7 @@ def run_reference(args):
 # The other configurations (parity-test cases): timed on request with --workload, same protocol.
 # ------------------------------------------------------------------------------------------------
 OTHER_WORKLOADS = ["swin_b_stage3_block_pair", "llama_attention_layer", "llama_decode_layer", "chain_2a_qkt", "chain_2b_gemm",
-                   "chain_2a_copy", "chain_2b_copy", "swin_shift_partition_copy", "depth_to_space_copy", "swin_t_patch_merging", "swin_t_stage1"]
+                   "chain_2a_copy", "chain_2b_copy", "swin_shift_partition_copy", "depth_to_space_copy", "swin_t_patch_merging", "swin_t_stage1", "nchw_layernorm_linear"]
 
 
 def _peaks_all():
@@ -346,7 +346,7 @@ def run_other(args):
                  ("decode_attention", 2 * B * (pos + 1) * hidden * 2 + 2 * X, 4 * B * (pos + 1) * hidden),
                  ("o_proj_gemm", 2 * X + hidden * hidden * 2, 2 * B * hidden * hidden)]
     else:
-        which = "2a" if "2a" in name else "2b" if "2b" in name else "d2s" if "depth" in name else "pm" if "patch" in name else "e1"
+        which = "2a" if "2a" in name else "2b" if "2b" in name else "d2s" if "depth" in name else "pm" if "patch" in name else "nln" if "nchw" in name else "e1"
         inp = synth.chain_inputs(2, which if which in ("2a", "2b") else "2a")
         if which == "d2s":
             # DepthToSpace (Table 3's DtoS) of an NCHW activation, block 2: [8,256,64,64] -> [8,64,128,128]
@@ -355,6 +355,18 @@ def run_other(args):
             ops = [sm.make_op(sm.OP_DEPTH_TO_SPACE, window=2), sm.make_op(sm.OP_COPY)]
             srcs, descs, oshape = [x], [sm.make_desc((B, Cb, Hh, Ww))], (B, Cb // 4, Hh * 2, Ww * 2)
             model = [("copy_map", 2 * B * Cb * Hh * Ww * 2, 0)]
+            tokens = B * Hh * Ww
+        elif which == "nln":
+            # channels-first producer -> LayerNorm over C -> linear (the implicit transformation of Fig. 1(b)), at chain 2b's size
+            B, C, Hh, Ww, N = 8, 256, 64, 64, 256
+            mk = lambda tid, shape, std, mean: torch.from_numpy(synth.normal(0x5EED0009, tid, shape, std, mean, "bf16").view(np.int16).copy()).cuda().view(torch.bfloat16)
+            srcs = [mk(0, (B, C, Hh, Ww), 1.0, 0.0), mk(1, (C,), 0.02, 1.0), mk(2, (C,), 0.02, 0.0), mk(3, (N, C), 0.02, 0.0)]
+            descs = [sm.make_desc((B, C, Hh, Ww)), sm.make_desc((C,)), sm.make_desc((C,)), sm.make_desc((N, C))]
+            ops = [sm.make_op(sm.OP_TRANSPOSE, perm=(0, 2, 3, 1)), sm.make_op(sm.OP_RESHAPE, shape=(B, Hh * Ww, C)),
+                   sm.make_op(sm.OP_LAYERNORM, side_input=(1, 2), eps=1e-5), sm.make_op(sm.OP_LINEAR, side_input=(3, 0))]
+            oshape = (B, Hh * Ww, N)
+            U = B * C * Hh * Ww * 2
+            model = [("layernorm_channels_first", 2 * U, 0), ("linear", U + N * C * 2 + B * Hh * Ww * N * 2, 2 * B * Hh * Ww * N * C)]
             tokens = B * Hh * Ww
         elif which == "pm":
             # patch merging between stages 1 and 2 of Swin-T at the benchmark's batch: [32,56,56,96] -> [32,784,192]

@@ -258,6 +258,9 @@ int launch_copy_map(const smartmem_index_map_t& map, int elem_size, const void* 
 // read from src at element offset rowmap(r) (rowmap == nullptr: r * C).
 // LayerNorm over the last dimension of a [rows, C] tensor whose elements are read through `map` (consumer
 // linear index -> producer element offset, 16-byte vectors intact, C / vector <= 128); writes [rows, C] contiguously.
+// True when `map` is the strided-channel form (tokens contiguous in the producer, the normalised dimension strided:
+// a channels-first producer) that launch_layernorm_map handles with its slab kernel.  Host only.
+bool layernorm_map_strided_supported(const smartmem_index_map_t& map, int elem_size, long long C);
 int launch_layernorm_map(int dtype, const void* src, void* dst, const void* gamma, const void* beta, float eps,
                          const smartmem_index_map_t& map, int C, cudaStream_t st);
 int launch_norm(int dtype, bool rms, const void* src, void* dst, const void* gamma, const void* beta, float eps,

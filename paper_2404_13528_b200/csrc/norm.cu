@@ -3,7 +3,10 @@
 // folded into the loads), so the normalised rows come out in the consumer's order with no
 // layout copy in between.  Statistics are fp32 and two-pass (mean, then centred variance);
 // reductions use warp shuffles.
+#include <mutex>
+
 #include "common.cuh"
+#include "gemm_tc.cuh"
 
 namespace smartmem {
 namespace {
@@ -334,6 +337,190 @@ int launch_norm_t(const void* src, void* dst, const void* gamma, const void* bet
   return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
 }
 
+// LayerNorm over a dimension that is STRIDED in the producer's buffer while the token dimension is the
+// contiguous one -- a channels-first (NCHW) producer normalised over C, the implicit layout
+// transformation of Fig. 1(b).  A CTA takes 64 consecutive tokens of one image.  Eight lanes cover a
+// channel's 64 tokens with one 16-byte load each (128 contiguous bytes per channel), 32 channels per
+// pass; a thread keeps its 8 tokens x NK channels in registers, so both statistics passes run on
+// registers and only per-token partial sums cross threads (two shuffles, then shared memory across the
+// eight warps).  The normalised values are written to shared memory transposed ([token][C], odd word
+// pitch), from where whole channels-last rows leave with coalesced stores.  No transposed copy of the
+// input is ever stored.
+constexpr int NS_TOK = 64;
+// 8 bf16 from global memory: one 16-byte load when the producer's strides keep it aligned, else four 4-byte loads
+__device__ __forceinline__ uint4 ld_vec16(const __nv_bfloat16* p, bool aligned16) {
+  if (aligned16) return *reinterpret_cast<const uint4*>(p);
+  const uint32_t* q = reinterpret_cast<const uint32_t*>(p);
+  return make_uint4(q[0], q[1], q[2], q[3]);
+}
+__device__ __forceinline__ void unpack8_bf16(const uint4& u, float (&f)[8]) {
+  const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    f[2 * q] = __uint_as_float(w[q] << 16);
+    f[2 * q + 1] = __uint_as_float(w[q] & 0xFFFF0000u);
+  }
+}
+
+// Channel of slot k of a thread with channel row cr: slots come in adjacent pairs (2 cr, 2 cr + 1) + 64 (k / 2), so the
+// two normalised channels of a token leave as one 32-bit shared-memory store; a pass (fixed k) still covers 32 distinct
+// channel rows with eight lanes each.
+__device__ __forceinline__ int ns_channel(int k, int cr) { return (k >> 1) * 64 + 2 * cr + (k & 1); }
+
+template <int NK>                                        // channel slots per thread (even): C <= 32 * NK
+__global__ void __launch_bounds__(256, NK == 8 ? 2 : 1) norm_strided_kernel(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ dst,
+                                                           const __nv_bfloat16* __restrict__ gamma,
+                                                           const __nv_bfloat16* __restrict__ beta, float eps, int C,
+                                                           long long c_stride, long long img_stride, int tiles_per_img,
+                                                           long long base, bool vec_ok, int n_tiles) {
+  extern __shared__ __align__(16) unsigned char ns_smem[];
+  const int P = C + 2;                                                      // bf16 per transposed row: (C + 2) / 2 words, odd
+  __nv_bfloat16* slab = reinterpret_cast<__nv_bfloat16*>(ns_smem);          // [64][P]
+  float* part = reinterpret_cast<float*>(slab + (size_t)NS_TOK * P);       // [2][8 warps][64 tokens]
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tg = tid & 7, cr = tid >> 3;                                    // token group (8 tokens), channel row of a pass
+  pdl_wait();
+  pdl_launch_dependents();
+  // persistent over the slabs: the next slab's loads are requested before this one is worked on, so every thread
+  // always has NK 16-byte loads in flight
+  auto request = [&](int t, uint4 (&v)[NK]) {
+    const int img = t / tiles_per_img, tile = t - img * tiles_per_img;
+    const __nv_bfloat16* s = src + base + (long long)img * img_stride + (long long)tile * NS_TOK + 8 * tg;
+#pragma unroll
+    for (int k = 0; k < NK; ++k) {
+      const int c = ns_channel(k, cr);
+      v[k] = make_uint4(0, 0, 0, 0);
+      if (t < n_tiles && c < C) v[k] = ld_vec16(s + c * c_stride, vec_ok);
+    }
+  };
+  uint4 r[NK], rn[NK];
+  request((int)blockIdx.x, rn);
+  for (int tcur = (int)blockIdx.x; tcur < n_tiles; tcur += (int)gridDim.x) {
+#pragma unroll
+  for (int k = 0; k < NK; ++k) r[k] = rn[k];
+  request(tcur + (int)gridDim.x, rn);
+  // sums of this thread's channels for its 8 tokens, then over the four channel rows of the warp, then over the warps
+  auto reduce_tokens = [&](float (&v)[8], float* buf) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      v[j] += __shfl_xor_sync(0xFFFFFFFFu, v[j], 8);
+      v[j] += __shfl_xor_sync(0xFFFFFFFFu, v[j], 16);
+    }
+    if (lane < 8) {
+      float4* o = reinterpret_cast<float4*>(buf + warp * NS_TOK + 8 * tg);
+      o[0] = make_float4(v[0], v[1], v[2], v[3]);
+      o[1] = make_float4(v[4], v[5], v[6], v[7]);
+    }
+    __syncthreads();
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v[j] = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) {
+      const float4* i4 = reinterpret_cast<const float4*>(buf + w * NS_TOK + 8 * tg);
+      const float4 a = i4[0], b = i4[1];
+      v[0] += a.x; v[1] += a.y; v[2] += a.z; v[3] += a.w;
+      v[4] += b.x; v[5] += b.y; v[6] += b.z; v[7] += b.w;
+    }
+  };
+  const float invC = 1.0f / (float)C;
+  float mean[8], rstd[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) mean[j] = 0.f;
+#pragma unroll
+  for (int k = 0; k < NK; ++k) {
+    float f[8];
+    unpack8_bf16(r[k], f);                                                  // absent channel slots hold zeros
+#pragma unroll
+    for (int j = 0; j < 8; ++j) mean[j] += f[j];
+  }
+  reduce_tokens(mean, part);
+#pragma unroll
+  for (int j = 0; j < 8; ++j) { mean[j] *= invC; rstd[j] = 0.f; }
+#pragma unroll
+  for (int k = 0; k < NK; ++k) {
+    if (ns_channel(k, cr) < C) {
+      float f[8];
+      unpack8_bf16(r[k], f);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) rstd[j] = fmaf(f[j] - mean[j], f[j] - mean[j], rstd[j]);
+    }
+  }
+  reduce_tokens(rstd, part + 8 * NS_TOK);
+#pragma unroll
+  for (int j = 0; j < 8; ++j) rstd[j] = rsqrtf(rstd[j] * invC + eps);
+  // normalise and store transposed: the channel pair (c, c + 1) of a token is one 32-bit word of its row (C is even)
+  float ms[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) ms[j] = -mean[j] * rstd[j];
+  uint32_t* slab32 = reinterpret_cast<uint32_t*>(slab);
+#pragma unroll
+  for (int k = 0; k < NK; k += 2) {
+    const int c = ns_channel(k, cr);
+    if (c < C) {
+      float f0[8], f1[8];
+      unpack8_bf16(r[k], f0);
+      unpack8_bf16(r[k + 1], f1);
+      const float2 g = bf16x2_to_float2(*reinterpret_cast<const uint32_t*>(gamma + c));
+      const float2 b = bf16x2_to_float2(*reinterpret_cast<const uint32_t*>(beta + c));
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        slab32[(8 * tg + j) * (P / 2) + (c >> 1)] =
+            float2_to_bf16x2(fmaf(fmaf(f0[j], rstd[j], ms[j]), g.x, b.x), fmaf(fmaf(f1[j], rstd[j], ms[j]), g.y, b.y));
+    }
+  }
+  __syncthreads();
+  // channels-last rows: a warp per token, a bf16 pair per lane and step
+  uint32_t* d = reinterpret_cast<uint32_t*>(dst + ((long long)tcur * NS_TOK) * C);
+  const uint32_t* sl = reinterpret_cast<const uint32_t*>(slab);
+  for (int t = warp; t < NS_TOK; t += 8)
+    for (int c2 = lane; c2 < C / 2; c2 += 32) d[(long long)t * (C / 2) + c2] = sl[t * (P / 2) + c2];
+  __syncthreads();                                   // the slab is rewritten by the next round
+  }
+}
+
+// The strided-channel form of a map: [images] x [tokens, contiguous] x [C, strided]; tokens a multiple of 64.
+bool norm_strided_supported(const smartmem_index_map_t& m, int elem_size, long long C) {
+  const int n = m.n_atoms;
+  if (m.klass != 1 || elem_size != 2 || n < 2 || n > 3 || C % 2 || C > 512) return false;
+  if (m.extent[n - 1] != C || m.src_stride[n - 1] == 1 || m.src_stride[n - 2] != 1 || m.extent[n - 2] % NS_TOK) return false;
+  if (m.base % 2 || m.src_stride[n - 1] % 2 || (n == 3 && m.src_stride[0] % 2)) return false;
+  if (m.n_elements / C / NS_TOK >= (1ll << 31)) return false;
+  return true;
+}
+
+int launch_norm_strided(const void* src, void* dst, const void* gamma, const void* beta, float eps,
+                        const smartmem_index_map_t& m, int C, cudaStream_t st) {
+  const int n = m.n_atoms;
+  const long long tokens = m.extent[n - 2], images = n == 3 ? m.extent[0] : 1;
+  const size_t smem = (size_t)NS_TOK * (C + 2) * 2 + 2 * 8 * NS_TOK * sizeof(float);
+  static std::mutex mu;
+  static size_t configured = 48 * 1024;
+  {
+    std::lock_guard<std::mutex> lk(mu);
+    if (smem > configured) {
+      if (cudaFuncSetAttribute(norm_strided_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+          cudaFuncSetAttribute(norm_strided_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return SMARTMEM_ERR_CUDA;
+      configured = smem;
+    }
+  }
+  const bool vec_ok = ((uintptr_t)src & 15) == 0 && m.base % 8 == 0 && m.src_stride[n - 1] % 8 == 0 && (n < 3 || m.src_stride[0] % 8 == 0);
+  const long long n_tiles = images * (tokens / NS_TOK);
+  const long long slots = (long long)tc_sm_count() * (C <= 256 ? 2 : 1);
+  const dim3 grid((unsigned)(n_tiles < slots ? n_tiles : slots));
+  const long long img_stride = n == 3 ? (long long)m.src_stride[0] : 0ll;
+  if (C <= 256)
+    launch_pdl(norm_strided_kernel<8>, grid, dim3(256), smem, st, (const __nv_bfloat16*)src, (__nv_bfloat16*)dst,
+               (const __nv_bfloat16*)gamma, (const __nv_bfloat16*)beta, eps, C, (long long)m.src_stride[n - 1], img_stride,
+               (int)(tokens / NS_TOK), (long long)m.base, vec_ok, (int)n_tiles);
+  else
+    launch_pdl(norm_strided_kernel<16>, grid, dim3(256), smem, st, (const __nv_bfloat16*)src, (__nv_bfloat16*)dst,
+               (const __nv_bfloat16*)gamma, (const __nv_bfloat16*)beta, eps, C, (long long)m.src_stride[n - 1], img_stride,
+               (int)(tokens / NS_TOK), (long long)m.base, vec_ok, (int)n_tiles);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
+}
+
 template <typename T>
 int launch_norm_map_t(const void* src, void* dst, const void* gamma, const void* beta, float eps,
                       const smartmem_index_map_t& map, int C, cudaStream_t st) {
@@ -358,9 +545,14 @@ int launch_norm_map_t(const void* src, void* dst, const void* gamma, const void*
 
 }  // namespace
 
+bool layernorm_map_strided_supported(const smartmem_index_map_t& map, int elem_size, long long C) {
+  return norm_strided_supported(map, elem_size, C);
+}
+
 int launch_layernorm_map(int dtype, const void* src, void* dst, const void* gamma, const void* beta, float eps,
                          const smartmem_index_map_t& map, int C, cudaStream_t st) {
   profile_tick("layernorm_map", st);
+  if (dtype == SMARTMEM_BF16 && norm_strided_supported(map, 2, C)) return launch_norm_strided(src, dst, gamma, beta, eps, map, C, st);
   if (dtype == SMARTMEM_F32) return launch_norm_map_t<float>(src, dst, gamma, beta, eps, map, C, st);
   return launch_norm_map_t<__nv_bfloat16>(src, dst, gamma, beta, eps, map, C, st);
 }

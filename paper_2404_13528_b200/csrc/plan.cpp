@@ -547,6 +547,16 @@ int process_run(smartmem_plan_t* p, const smartmem_op_t* ops, int i0, int i1, co
   return SMARTMEM_OK;
 }
 
+// The map of a LayerNorm over a dimension that is strided in the producer while the tokens are contiguous
+// ([images] x [tokens] x [C]: a channels-first producer).  Must agree with the kernel-side check in norm.cu.
+bool layernorm_strided_form(const smartmem_index_map_t& m, int elem_size, int64_t C) {
+  const int n = m.n_atoms;
+  if (m.klass != 1 || elem_size != 2 || n < 2 || n > 3 || C % 2 || C > 512) return false;
+  if (m.extent[n - 1] != C || m.src_stride[n - 1] == 1 || m.src_stride[n - 2] != 1 || m.extent[n - 2] % 64) return false;
+  if (m.base % 2 || m.src_stride[n - 1] % 2 || (n == 3 && m.src_stride[0] % 2)) return false;
+  return m.n_elements / C / 64 < (1ll << 31);
+}
+
 bool is_layout_kind(int k) { return k >= SMARTMEM_OP_RESHAPE && k <= SMARTMEM_OP_SPACE_TO_DEPTH; }
 
 }  // namespace
@@ -794,7 +804,8 @@ int smartmem_plan(const smartmem_op_t* ops, int32_t n_ops, const smartmem_tensor
       // the kernel fetches a row as 16-byte vectors through the map: they must not straddle a contiguous run, and
       // a warp holds the row in registers; otherwise the run is materialised first (as EXPLICIT does anyway)
       const int vec = 16 / esz;
-      const bool foldable = st.map[0].klass != 3 && st.map[0].vec_elems % vec == 0 && C % vec == 0 && C / vec <= 128;
+      const bool foldable = (st.map[0].klass != 3 && st.map[0].vec_elems % vec == 0 && C % vec == 0 && C / vec <= 128) ||
+                            layernorm_strided_form(st.map[0], esz, C);       // or: channels-first producer, tokens contiguous
       if (!foldable && st.map[0].klass != 0) {
         Step cp;
         cp.kind = STEP_COPY;

@@ -403,3 +403,20 @@ def test_layernorm_consumer_argument_errors():
     with pytest.raises(sm.SmartmemError) as e:
         sm.smartmem_plan(ops1, good, sm.ELIMINATE)
     assert e.value.code == sm.ERR_INVALID_ARG
+
+
+def test_layernorm_over_the_strided_dimension_of_a_channels_first_producer_is_folded():
+    """NCHW -> (NHWC view) -> LayerNorm over C: tokens are contiguous in the producer, channels strided.  The planner keeps
+    the map on the LayerNorm's load side when the tokens of an image are a multiple of 64, else materialises."""
+    def steps(B, C, H, W):
+        ops = [sm.make_op(sm.OP_TRANSPOSE, perm=(0, 2, 3, 1)), sm.make_op(sm.OP_RESHAPE, shape=(B, H * W, C)),
+               sm.make_op(sm.OP_LAYERNORM, side_input=(1, 2), eps=1e-5), sm.make_op(sm.OP_COPY)]
+        plan = sm.smartmem_plan(ops, [sm.make_desc((B, C, H, W)), sm.make_desc((C,)), sm.make_desc((C,))], sm.ELIMINATE)
+        try:
+            return sm.smartmem_plan_num_steps(plan)
+        finally:
+            sm.smartmem_plan_destroy(plan)
+    assert steps(2, 64, 8, 16)[1] == 0
+    assert steps(1, 32, 8, 8)[1] == 0
+    assert steps(2, 64, 6, 6)[1] == 1          # 36 tokens per image
+    assert steps(2, 63, 8, 8)[1] == 1          # odd channel count
