@@ -86,7 +86,7 @@ __device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, uint32_t parity
   }
 }
 
-// ---- TMA loads (no multicast), completion on an mbarrier --------------------------------
+// ---- TMA loads (each CTA fetches its own tile), completion on an mbarrier ----------------------
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tm, uint64_t* bar, int c0, int c1) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(
