@@ -151,8 +151,8 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   for (int i = threadIdx.x; i < g.C; i += kThreads) b2_s[i] = __bfloat162float(g.b2[i]);
   if (fuse_ln)
     for (int i = threadIdx.x; i < g.C; i += kThreads) {
-      ln_s[i] = __bfloat162float(g.ln_gamma[i]);
-      ln_s[g.C + i] = __bfloat162float(g.ln_beta[i]);
+      reinterpret_cast<__nv_bfloat16*>(ln_s)[i] = g.ln_gamma[i];              // packed bf16: [C] gamma at word 0, [C] beta at word C
+      reinterpret_cast<__nv_bfloat16*>(ln_s + g.C)[i] = g.ln_beta[i];
     }
   if (warp == 1) ptx::tmem_alloc(tmem_slot, TMEM_COLS);
   ptx::tc_fence_before();
@@ -426,17 +426,21 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             }
           const float sq = (q4[0] + q4[1]) + (q4[2] + q4[3]);
           const float rstd = rsqrtf(sq * invC + g.ln_eps);
+          const float nmr = -mean * rstd;
 #pragma unroll
           for (int ch = 0; ch < 12; ++ch)
             if (ch < nch) {
               const uint32_t w[4] = {x[ch].x, x[ch].y, x[ch].z, x[ch].w};
+              // (x - mean) rstd in fp32, rounded to bf16 pairs; the affine part as one packed multiply-add per pair
+              const uint4 ga = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(ln_s) + ch * 8);
+              const uint4 be = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(ln_s + g.C) + ch * 8);
+              const uint32_t gw[4] = {ga.x, ga.y, ga.z, ga.w}, bw[4] = {be.x, be.y, be.z, be.w};
               uint32_t o[4];
 #pragma unroll
               for (int i = 0; i < 4; ++i) {
                 const float2 f = bf16x2_to_float2(w[i]);
-                const float2 ga = *reinterpret_cast<const float2*>(ln_s + ch * 8 + 2 * i);
-                const float2 be = *reinterpret_cast<const float2*>(ln_s + g.C + ch * 8 + 2 * i);
-                o[i] = float2_to_bf16x2(fmaf((f.x - mean) * rstd, ga.x, be.x), fmaf((f.y - mean) * rstd, ga.y, be.y));
+                const uint32_t t = float2_to_bf16x2(fmaf(f.x, rstd, nmr), fmaf(f.y, rstd, nmr));
+                asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(o[i]) : "r"(t), "r"(gw[i]), "r"(bw[i]));
               }
               *reinterpret_cast<uint4*>(row0 + (ch >> 3) * KB_BYTES + (((ch & 7) ^ (r & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
             }
