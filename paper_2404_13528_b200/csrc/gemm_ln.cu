@@ -116,8 +116,8 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   for (int i = threadIdx.x; i < g.N; i += kThreads) bias_s[i] = g.bias ? __bfloat162float(g.bias[i]) : 0.f;
   if (g.has_ln)
     for (int i = threadIdx.x; i < KDIM; i += kThreads) {
-      ln_s[i] = __bfloat162float(g.gamma[i]);
-      ln_s[KDIM + i] = __bfloat162float(g.beta[i]);
+      reinterpret_cast<__nv_bfloat16*>(ln_s)[i] = g.gamma[i];                 // packed bf16: gamma at word 0, beta at word KDIM
+      reinterpret_cast<__nv_bfloat16*>(ln_s + KDIM)[i] = g.beta[i];
     }
   ptx::tc_fence_before();
   __syncthreads();
@@ -280,17 +280,21 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         float sq = (q4[0] + q4[1]) + (q4[2] + q4[3]);
         sq += __shfl_xor_sync(0xFFFFFFFFu, sq, 1);
         const float rstd = rsqrtf(sq * invK + g.eps);
+        const float nmr = -mean * rstd;
+        // (x - mean) rstd in fp32, rounded to bf16 pairs; the affine part as one packed multiply-add per pair
 #pragma unroll
         for (int c = 0; c < NH; ++c) {
           const uint32_t w[4] = {cur[c].x, cur[c].y, cur[c].z, cur[c].w};
           uint32_t o[4];
           const int col = (hh * NH + c) * 8;
+          const uint4 ga = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(ln_s) + col);
+          const uint4 be = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(ln_s + KDIM) + col);
+          const uint32_t gw[4] = {ga.x, ga.y, ga.z, ga.w}, bw[4] = {be.x, be.y, be.z, be.w};
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             const float2 f = bf16x2_to_float2(w[i]);
-            const float2 ga = *reinterpret_cast<const float2*>(ln_s + col + 2 * i);
-            const float2 be = *reinterpret_cast<const float2*>(ln_s + KDIM + col + 2 * i);
-            o[i] = float2_to_bf16x2(fmaf((f.x - mean) * rstd, ga.x, be.x), fmaf((f.y - mean) * rstd, ga.y, be.y));
+            const uint32_t t = float2_to_bf16x2(fmaf(f.x, rstd, nmr), fmaf(f.y, rstd, nmr));
+            asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(o[i]) : "r"(t), "r"(gw[i]), "r"(bw[i]));
           }
           cur[c] = make_uint4(o[0], o[1], o[2], o[3]);
         }
