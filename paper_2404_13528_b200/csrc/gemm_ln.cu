@@ -253,32 +253,28 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       if (ti + 1 < my_tiles) load_row(ti + 1, nxt);    // in flight while this tile is normalised
       if (pw == 0 && lane == 0) LDBG(ti * 32 + 21);
       if (g.has_ln) {
-        float s4[4] = {0.f, 0.f, 0.f, 0.f};
+        // one pass for both moments on data shifted by the row's first element p (d = x - p): mean = p + sum(d) / K,
+        // variance = (sum(d^2) - sum(d)^2 / K) / K; p lies within the row's own spread, so the subtraction of the
+        // two sums loses a few bits at most.  The two threads of a row share p and add their partial sums.
+        const float p = __shfl_sync(0xFFFFFFFFu, __uint_as_float(cur[0].x << 16), lane & ~1);
+        float s4[4] = {0.f, 0.f, 0.f, 0.f}, q4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int c = 0; c < NH; ++c) {
           const uint32_t w[4] = {cur[c].x, cur[c].y, cur[c].z, cur[c].w};
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             const float2 f = bf16x2_to_float2(w[i]);
-            s4[i] += f.x + f.y;
-          }
-        }
-        float sum = (s4[0] + s4[1]) + (s4[2] + s4[3]);
-        sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 1);
-        const float mean = sum * invK;
-        float q4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-        for (int c = 0; c < NH; ++c) {
-          const uint32_t w[4] = {cur[c].x, cur[c].y, cur[c].z, cur[c].w};
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const float2 f = bf16x2_to_float2(w[i]);
-            const float dx = f.x - mean, dy = f.y - mean;
+            const float dx = f.x - p, dy = f.y - p;
+            s4[i] += dx + dy;
             q4[i] = fmaf(dy, dy, fmaf(dx, dx, q4[i]));
           }
         }
+        float sd = (s4[0] + s4[1]) + (s4[2] + s4[3]);
         float sq = (q4[0] + q4[1]) + (q4[2] + q4[3]);
+        sd += __shfl_xor_sync(0xFFFFFFFFu, sd, 1);
         sq += __shfl_xor_sync(0xFFFFFFFFu, sq, 1);
+        const float mean = fmaf(sd, invK, p);
+        sq = fmaxf(sq - sd * sd * invK, 0.f);
         const float rstd = rsqrtf(sq * invK + g.eps);
         const float nmr = -mean * rstd;
         // (x - mean) rstd in fp32, rounded to bf16 pairs; the affine part as one packed multiply-add per pair

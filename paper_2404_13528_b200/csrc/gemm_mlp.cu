@@ -400,7 +400,11 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
           for (int ch = 0; ch < 12; ++ch)
             if (ch < nch) x[ch] = *reinterpret_cast<const uint4*>(row0 + (ch >> 3) * KB_BYTES + (((ch & 7) ^ (r & 7)) << 4));
-          float s4[4] = {0.f, 0.f, 0.f, 0.f};             // four partial sums: independent dependency chains
+          // one pass over the row for both moments, on data shifted by the row's first element p (d = x - p):
+          // mean = p + sum(d) / C, variance = (sum(d^2) - sum(d)^2 / C) / C.  p lies within the row's own spread,
+          // so the subtraction of the two sums loses a few bits at most.  Four independent partial sums each.
+          const float p = __uint_as_float(x[0].x << 16);
+          float s4[4] = {0.f, 0.f, 0.f, 0.f}, q4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
           for (int ch = 0; ch < 12; ++ch)
             if (ch < nch) {
@@ -408,23 +412,14 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
               for (int i = 0; i < 4; ++i) {
                 const float2 f = bf16x2_to_float2(w[i]);
-                s4[i] += f.x + f.y;
-              }
-            }
-          const float mean = ((s4[0] + s4[1]) + (s4[2] + s4[3])) * invC;
-          float q4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-          for (int ch = 0; ch < 12; ++ch)
-            if (ch < nch) {
-              const uint32_t w[4] = {x[ch].x, x[ch].y, x[ch].z, x[ch].w};
-#pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                const float2 f = bf16x2_to_float2(w[i]);
-                const float dx = f.x - mean, dy = f.y - mean;
+                const float dx = f.x - p, dy = f.y - p;
+                s4[i] += dx + dy;
                 q4[i] = fmaf(dy, dy, fmaf(dx, dx, q4[i]));
               }
             }
-          const float sq = (q4[0] + q4[1]) + (q4[2] + q4[3]);
+          const float sd = (s4[0] + s4[1]) + (s4[2] + s4[3]);
+          const float mean = fmaf(sd, invC, p);
+          const float sq = fmaxf(((q4[0] + q4[1]) + (q4[2] + q4[3])) - sd * sd * invC, 0.f);
           const float rstd = rsqrtf(sq * invC + g.ln_eps);
           const float nmr = -mean * rstd;
 #pragma unroll
