@@ -76,6 +76,21 @@ def test_small_bf16_blocks(cfg):
     case(20, dtype="bf16", **cfg)
 
 
+@pytest.mark.parametrize("offset,spread", [(40.0, 1.0), (-12.0, 0.25), (0.0, 30.0)])
+def test_layernorm_statistics_on_rows_with_a_large_common_offset(offset, spread):
+    """Rows whose mean dwarfs their spread (and rows with a huge spread): the fused kernels take both LayerNorm
+    moments in one pass over data shifted by the row's first element, which must stay as accurate as two passes."""
+    B, H, W, C, heads, ws = 2, 14, 14, 96, 3, 7
+    inp = synth.swin_inputs(21, B, H, W, C, heads, ws, 4, "bf16")
+    x = synth.to_f64(inp["x"]) * spread + offset
+    inp["x"] = synth.f64_to_bf16_bits(x).reshape(x.shape)
+    dev = {k: to_dev(v) for k, v in inp.items()}
+    ref = oracle_block(inp, [0, 1], heads=heads, window=ws, shift=3, mlp_ratio=4)
+    for mode in (sm.ELIMINATE, sm.EXPLICIT):
+        y = run_block(inp, dev, B=B, H=H, W=W, C=C, heads=heads, window=ws, shift=3, mlp_ratio=4, dtype="bf16", mode=mode)
+        assert_close_bf16(to_host_f64(y), ref, f"mode {mode}")
+
+
 def test_config3_swin_t_stage1_full_size():
     """B=32, 56x56, C=96, 3 heads, window 7, shift 3, MLP x4 at full size; the oracle checks two images."""
     case(3, B=32, H=56, W=56, C=96, heads=3, window=7, shift=3, mlp_ratio=4, dtype="bf16", images=[0, 31])
