@@ -28,19 +28,28 @@ def stream() -> int:
     return torch.cuda.current_stream().cuda_stream
 
 
-def assert_close_bf16(got: np.ndarray, ref: np.ndarray, what: str = ""):
-    """bf16 rule, against the fp64 oracle: |got - ref| <= 2e-2 * max(1, scale) elementwise, where scale
-    is the largest |ref| of the element's output row (last dimension).  The forward error of a
-    mixed-precision contraction grows with the magnitude of the row it belongs to, not with the
-    magnitude of the individual result (an element near zero in a large row still carries the
-    row's rounding noise), so the relative part of the bound is taken per row."""
+def assert_close_bf16(got: np.ndarray, ref: np.ndarray, what: str = "", max_strict_violations: int = 0,
+                      allowed_rows=None):
+    """bf16 rule, against the fp64 oracle: |got - ref| <= 2e-2 * max(1, |ref|) for every element.
+
+    `max_strict_violations` is a named, counted exception for one known case (the first rows of a causal
+    layer, whose softmax runs over one to three keys, so that the bf16 rounding of q and k is not averaged
+    out): at most that many elements may exceed the per-element bound, each of them must lie in a row (index
+    along the second-to-last axis) listed in `allowed_rows`, and each must still satisfy the bound scaled by
+    the largest |ref| of its own output row."""
     err = np.abs(got - ref)
-    scale = np.maximum(1.0, np.abs(ref).max(axis=-1, keepdims=True))
-    bad = err > 2e-2 * scale
-    strict = (err > 2e-2 * np.maximum(1.0, np.abs(ref))).sum()
-    assert not bad.any(), (f"{what}: {bad.sum()} of {bad.size} elements out of tolerance; max err {err.max():.4g} "
-                           f"at {np.unravel_index(err.argmax(), err.shape)} (ref {ref.flat[err.argmax()]:.4g}); "
-                           f"{strict} beyond the per-element bound; max err / max |ref| = {err.max() / np.abs(ref).max():.3g}")
+    bad = err > 2e-2 * np.maximum(1.0, np.abs(ref))
+    n_bad = int(bad.sum())
+    if n_bad == 0:
+        return
+    where = np.argwhere(bad)
+    msg = (f"{what}: {n_bad} of {bad.size} elements beyond 2e-2 * max(1, |ref|); max err {err.max():.4g} at "
+           f"{np.unravel_index(err.argmax(), err.shape)} (ref {ref.flat[err.argmax()]:.4g}); first at {where[:4].tolist()}")
+    assert n_bad <= max_strict_violations, msg
+    rows = set(int(w[-2]) for w in where)
+    assert allowed_rows is not None and rows <= set(allowed_rows), msg + f"; rows {sorted(rows)} not in the allowed set"
+    row_scale = np.maximum(1.0, np.abs(ref).max(axis=-1, keepdims=True))
+    assert not (err > 2e-2 * row_scale).any(), msg + "; also beyond the row-scaled bound"
 
 
 def assert_close_f32(got: np.ndarray, ref: np.ndarray, what: str = ""):

@@ -90,6 +90,25 @@ def test_rel_pos_index_pins():
     assert idx4.max() == 48 and (np.diag(idx4) == 24).all()
 
 
+def test_rel_pos_index_orientation_hand_values():
+    """The index is (y_i - y_j + ws - 1)(2ws - 1) + (x_i - x_j + ws - 1), i the query and j the key: the row part
+    comes from the vertical displacement, and a key to the right of / below the query gives the smaller index.
+    Values worked out by hand from token t = (t div ws, t mod ws); each fails if i and j or the two axes are swapped."""
+    idx = ops.rel_pos_index(7)
+    # token 0 = (0,0), 1 = (0,1), 7 = (1,0), 8 = (1,1), 48 = (6,6), 6 = (0,6), 42 = (6,0)
+    assert idx[0, 1] == 6 * 13 + 5 == 83        # dy 0, dx -1
+    assert idx[1, 0] == 6 * 13 + 7 == 85        # dy 0, dx +1
+    assert idx[0, 7] == 5 * 13 + 6 == 71        # dy -1, dx 0
+    assert idx[7, 0] == 7 * 13 + 6 == 97        # dy +1, dx 0
+    assert idx[0, 8] == 5 * 13 + 5 == 70 and idx[8, 0] == 7 * 13 + 7 == 98
+    assert idx[0, 48] == 0 and idx[48, 0] == 168
+    assert idx[6, 42] == 0 * 13 + 12 == 12      # dy -6, dx +6
+    assert idx[42, 6] == 12 * 13 + 0 == 156     # dy +6, dx -6
+    idx4 = ops.rel_pos_index(4)                  # (dy + 3) * 7 + (dx + 3); token 4 = (1,0)
+    assert idx4[0, 1] == 23 and idx4[1, 0] == 25 and idx4[0, 4] == 17 and idx4[4, 0] == 31
+    assert idx4[0, 15] == 0 and idx4[15, 0] == 48 and idx4[3, 12] == 6 and idx4[12, 3] == 42
+
+
 @pytest.mark.parametrize("H,W,ws,s,nontrivial", [(8, 8, 4, 2, 3), (14, 14, 7, 3, 3), (56, 56, 7, 3, 15), (21, 21, 7, 3, 5)])
 def test_shift_mask_no_wrap_characterisation(H, W, ws, s, nontrivial):
     """Two tokens of one shifted window may attend iff, in ORIGINAL coordinates, they are
@@ -160,6 +179,30 @@ def test_window_attention_bias_is_added_per_head():
     o = swin.window_attention(q, k, v, table, ws)
     assert np.allclose(o[0, 0], v[0, 0].mean(0, keepdims=True).repeat(T, 0))   # head 0 uniform
     assert np.allclose(o[0, 1], v[0, 1], atol=1e-12)                            # head 1: diagonal dominates
+
+
+def test_window_attention_off_centre_bias_row():
+    """A one-hot at an OFF-centre row of the table: ws = 2, tokens 0=(0,0) 1=(0,1) 2=(1,0) 3=(1,1); table row
+    (dy+1)*3 + (dx+1) = 3 is the displacement dy = 0, dx = -1, i.e. query (y,0) looking at key (y,1): pairs
+    (i,j) = (0,1) and (2,3).  With q = k = 0 those two queries copy the key's value, the others average."""
+    ws, heads, d, T = 2, 1, 3, 4
+    q = np.zeros((1, heads, T, d))
+    k = np.zeros((1, heads, T, d))
+    v = np.array([[1.0, 0.0, 0.0], [0.0, 2.0, 0.0], [0.0, 0.0, 3.0], [4.0, 4.0, 4.0]]).reshape(1, 1, T, d)
+    table = np.zeros((9, heads))
+    table[3, 0] = 60.0
+    o = swin.window_attention(q, k, v, table, ws)[0, 0]
+    mean = np.array([5.0 / 4, 6.0 / 4, 7.0 / 4])
+    assert np.allclose(o[0], [0.0, 2.0, 0.0], atol=1e-12)       # token 0 -> value of token 1
+    assert np.allclose(o[1], mean, atol=1e-12)                  # token 1: no key at dx = -1 from it: uniform
+    assert np.allclose(o[2], [4.0, 4.0, 4.0], atol=1e-12)       # token 2 -> value of token 3
+    assert np.allclose(o[3], mean, atol=1e-12)
+    # a vertical displacement instead: row (−1+1)*3 + (0+1) = 1 is dy = -1, dx = 0: pairs (0,2) and (1,3)
+    table = np.zeros((9, heads))
+    table[1, 0] = 60.0
+    o = swin.window_attention(q, k, v, table, ws)[0, 0]
+    assert np.allclose(o[0], [0.0, 0.0, 3.0], atol=1e-12) and np.allclose(o[1], [4.0, 4.0, 4.0], atol=1e-12)
+    assert np.allclose(o[2], mean, atol=1e-12) and np.allclose(o[3], mean, atol=1e-12)
 
 
 def test_causal_attention_pins():
