@@ -50,7 +50,8 @@ def algorithmic_flops(w):
     qkv, proj, fc, att = 2 * M * C * 3 * C, 2 * M * C * C, 2 * M * C * r * C, 4 * M * T * C
     return {"qkv_gemm": qkv, "ln1_gather_qkv_gemm": qkv, "ln1_qkv_gemm": qkv, "window_attention": att,
             "proj_gemm_scatter_residual": proj, "proj_gemm_residual": proj, "fc1_gemm_gelu": fc, "fc2_gemm_residual": fc,
-            "mlp_fused_fc1_gelu_fc2_residual": 2 * fc, "mlp_fused_ln2_fc1_gelu_fc2_residual": 2 * fc}
+            "mlp_fused_fc1_gelu_fc2_residual": 2 * fc, "mlp_fused_ln2_fc1_gelu_fc2_residual": 2 * fc,
+            "attn_half_fused": qkv + att + proj}
 
 
 def algorithmic_bytes(w):
@@ -59,6 +60,7 @@ def algorithmic_bytes(w):
     C, r = w["C"], w["mlp_ratio"]
     wq, wp, w1 = 3 * C * C * 2, C * C * 2, r * C * C * 2
     return {
+        "attn_half_fused": 2 * U + wq + wp,                 # x in (also the residual), y1 out; q, k, v and the attention output stay on chip
         "ln1_gather": 2 * U, "qkv_gemm": U + wq + 3 * U, "ln1_gather_qkv_gemm": U + wq + 3 * U, "ln1_qkv_gemm": U + wq + 3 * U, "window_attention": 3 * U + U,
         "proj_gemm_scatter_residual": U + wp + U + U, "ln2": 2 * U, "fc1_gemm_gelu": U + w1 + r * U,
         "fc2_gemm_residual": r * U + w1 + U + U, "mlp_fused_fc1_gelu_fc2_residual": 3 * U + 2 * w1,

@@ -63,8 +63,13 @@ typedef enum { SMARTMEM_F32 = 0, SMARTMEM_BF16 = 1 } smartmem_dtype_t;
  * read, contiguous write) or on the producer side (out[imap(i)] = in[i], imap = the map of the inverted
  * chain: contiguous read, sub-optimal write), both with the plain map-driven kernel -- the two
  * placements Section 3.2.2 compares.  Same result as ELIMINATE, bit for bit. */
+/* ELIMINATE_UNFUSED (smartmem_swin_block only): the eliminated chain run kernel by kernel -- LayerNorm + gather +
+ * QKV, window attention, projection + scatter + residual, MLP -- each reading its producer's buffer through the
+ * composed map.  ELIMINATE additionally fuses the attention half of a narrow block into one kernel (Section 3.2.1:
+ * elimination is what makes the fusion possible; Table 5's "try fuse").  Kept so that the two gains are measured apart,
+ * and because it runs exactly the arithmetic of EXPLICIT (bit-identical results).  Wide blocks: same as ELIMINATE. */
 typedef enum { SMARTMEM_ELIMINATE = 0, SMARTMEM_EXPLICIT = 1, SMARTMEM_ELIMINATE_NAIVE = 2,
-               SMARTMEM_ELIMINATE_GATHER = 3, SMARTMEM_ELIMINATE_SCATTER = 4 } smartmem_mode_t;
+               SMARTMEM_ELIMINATE_GATHER = 3, SMARTMEM_ELIMINATE_SCATTER = 4, SMARTMEM_ELIMINATE_UNFUSED = 5 } smartmem_mode_t;
 
 /* Operator vocabulary of a chain.  Layout operators have a Fixed output layout (Table 3,
  * right column) and are the ones elimination removes; compute operators are kept. */

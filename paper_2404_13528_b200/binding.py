@@ -18,7 +18,7 @@ OK = 0
 ERR_INVALID_ARG, ERR_SHAPE, ERR_UNSUPPORTED, ERR_WORKSPACE = -1, -2, -3, -4
 ERR_ALIGNMENT, ERR_CUDA, ERR_TIMEOUT, ERR_BOUNDS = -5, -6, -7, -8
 F32, BF16 = 0, 1
-ELIMINATE, EXPLICIT, ELIMINATE_NAIVE, ELIMINATE_GATHER, ELIMINATE_SCATTER = 0, 1, 2, 3, 4
+ELIMINATE, EXPLICIT, ELIMINATE_NAIVE, ELIMINATE_GATHER, ELIMINATE_SCATTER, ELIMINATE_UNFUSED = 0, 1, 2, 3, 4, 5
 OP_RESHAPE, OP_TRANSPOSE, OP_ROLL, OP_SLICE, OP_WINDOW_PARTITION, OP_WINDOW_REVERSE = 0, 1, 2, 3, 4, 5
 OP_DEPTH_TO_SPACE, OP_SPACE_TO_DEPTH = 6, 7
 OP_COPY, OP_LINEAR, OP_BMM_NT, OP_LAYERNORM = 16, 17, 18, 19

@@ -1,6 +1,8 @@
 // C-ABI entry points (see include/smartmem.h).
 #include <atomic>
 #include <mutex>
+#include <set>
+#include <utility>
 #include <vector>
 
 #include "common.cuh"
@@ -30,17 +32,37 @@ void profile_tick(const char* name, cudaStream_t st) {
 
 __device__ int g_status_word;
 
+// Both caches below are per device: the address of a __device__ symbol and a kernel's attributes belong to the
+// context of the device that was current when they were looked up or set.
+static constexpr int kMaxDevices = 64;
+static std::mutex g_dev_mu;
+static int* g_status_ptr[kMaxDevices] = {nullptr};
+
 int* device_status_ptr() {
-  static int* p = nullptr;
-  static std::once_flag once;
-  std::call_once(once, [] {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  std::lock_guard<std::mutex> lk(g_dev_mu);
+  if (!g_status_ptr[dev]) {
     void* q = nullptr;
-    if (cudaGetSymbolAddress(&q, g_status_word) == cudaSuccess) {
-      p = (int*)q;
-      cudaMemset(p, 0, sizeof(int));
-    }
-  });
-  return p;
+    if (cudaGetSymbolAddress(&q, g_status_word) != cudaSuccess || !q) return nullptr;
+    if (cudaMemset(q, 0, sizeof(int)) != cudaSuccess) return nullptr;
+    g_status_ptr[dev] = (int*)q;
+  }
+  return g_status_ptr[dev];
+}
+
+static std::set<std::pair<int, const void*>> g_smem_configured;
+
+int ensure_max_dynamic_smem(const void* kernel, int bytes, int carveout) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) return SMARTMEM_ERR_CUDA;
+  std::lock_guard<std::mutex> lk(g_dev_mu);
+  const auto key = std::make_pair(dev, kernel);
+  if (g_smem_configured.count(key)) return SMARTMEM_OK;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return SMARTMEM_ERR_CUDA;
+  if (carveout >= 0) cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, carveout);
+  g_smem_configured.insert(key);
+  return SMARTMEM_OK;
 }
 
 }  // namespace smartmem

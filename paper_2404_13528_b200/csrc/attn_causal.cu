@@ -226,12 +226,7 @@ int launch_causal_attention(const CausalAttnArgs& a, cudaStream_t st) {
   for (auto* o : ops)
     if (o->se != 1 || o->st % 8 || o->sn % 8 || o->sh % 8 || ((uintptr_t)o->ptr & 15)) return SMARTMEM_ERR_ALIGNMENT;
   const size_t smem = 5 * (size_t)TILE_ELEMS * 2;
-  static bool configured = false;
-  if (!configured) {
-    if (cudaFuncSetAttribute(causal_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return SMARTMEM_ERR_CUDA;
-    configured = true;
-  }
+  if (ensure_max_dynamic_smem((const void*)causal_attn_kernel, (int)smem) != SMARTMEM_OK) return SMARTMEM_ERR_CUDA;
   profile_tick("causal_attention", st);
   dim3 grid((a.S + BMQ - 1) / BMQ, a.heads, a.batch);
   launch_pdl(causal_attn_kernel, dim3(grid), dim3(128), smem, st, a);

@@ -357,13 +357,7 @@ int launch_causal_attention_tc(const CausalAttnArgs& a, cudaStream_t st) {
   // reports a misaligned base instead of overrunning)
   const size_t smem = 2 * KB + 8 * KBK + 16 * 8 + 16;
   g.smem_bytes = (uint32_t)smem;
-  static bool configured = false;
-  if (!configured) {
-    if (cudaFuncSetAttribute(causal_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return SMARTMEM_ERR_CUDA;
-    cudaFuncSetAttribute(causal_attn_tc_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
-    configured = true;
-  }
+  if (ensure_max_dynamic_smem((const void*)causal_attn_tc_kernel, (int)smem, 100) != SMARTMEM_OK) return SMARTMEM_ERR_CUDA;
   const long long ctas = (long long)g.n_qt * B * H;
   if (ctas >= (1ll << 31)) return SMARTMEM_ERR_UNSUPPORTED;
   profile_tick("causal_attention_tc", st);

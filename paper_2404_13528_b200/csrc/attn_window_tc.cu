@@ -525,13 +525,9 @@ int launch_window_attention_tc(const WinAttnArgs& a_in, long long n_windows, cud
   }
   const size_t smem = 1024 + NSTAGE * STAGE_BYTES + TP * BIAS_ROW * 4 + (2 * kGroups + 1) * TP * 4 +
                       (2 * NSTAGE + 12) * 8 + 16;
-  static bool configured = false;
-  if (!configured) {
-    if (cudaFuncSetAttribute(win_attn_tc_kernel<56>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
-        cudaFuncSetAttribute(win_attn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return SMARTMEM_ERR_CUDA;
-    configured = true;
-  }
+  if (ensure_max_dynamic_smem((const void*)win_attn_tc_kernel<56>, (int)smem) != SMARTMEM_OK ||
+      ensure_max_dynamic_smem((const void*)win_attn_tc_kernel<64>, (int)smem) != SMARTMEM_OK)
+    return SMARTMEM_ERR_CUDA;
   const int sms = tc_sm_count();
   long long per_head = (long long)sms / a.heads;
   if (per_head < 1) per_head = 1;

@@ -12,8 +12,11 @@ namespace smartmem {
 // ---------------------------------------------------------------------------------------
 // Device status word (bounded waits / debug bounds) and launch accounting.
 // ---------------------------------------------------------------------------------------
-int* device_status_ptr();                 // device address of the status word (per process)
+int* device_status_ptr();                 // device address of the status word on the CURRENT device (looked up once per device)
 void count_launch(int n = 1);
+// Raises a kernel's dynamic shared-memory limit, once per (device, kernel); returns a smartmem_status_t.
+// `carveout` >= 0 also sets the preferred shared-memory carve-out (percent).
+int ensure_max_dynamic_smem(const void* kernel, int bytes, int carveout = -1);
 
 // Programmatic dependent launch.  A kernel launched through `launch_pdl` may start (be scheduled,
 // set up its barriers and tensor memory, prefetch its descriptors and constants) while the kernel
@@ -181,6 +184,57 @@ __device__ __forceinline__ long long devmap_eval_unrolled(const DevMap& m, uint3
   }
   return off;
 }
+
+// Partial evaluation.  The digit decomposition is linear up to the final wrap of the rolled coordinates, so a consumer
+// index i = n * P + t (P = the product of the extents of the trailing atoms [split, n_atoms)) can be evaluated as the sum
+// of the contributions of n over the leading atoms and of t over the trailing ones, wrapped once: a kernel that walks
+// over tiles (n) of P rows keeps a table of the trailing contributions and evaluates the leading atoms once per tile.
+struct DevMapPart {
+  long long off;
+  int u0, u1, u2, u3;
+};
+// contribution of the digits of `i` over atoms [a0, a1) (i below the product of their extents); the base is not included
+__device__ __forceinline__ DevMapPart devmap_part(const DevMap& m, int a0, int a1, uint32_t i) {
+  DevMapPart p{0, 0, 0, 0, 0};
+#pragma unroll
+  for (int a = kMaxDevAtoms - 1; a >= 0; --a) {
+    if (a >= a0 && a < a1) {
+      const uint32_t q = fd_div(i, m.ext[a]);
+      const int digit = (int)(i - q * m.ext[a].d);
+      i = q;
+      const int r = m.roll_of[a];
+      if (r < 0) {
+        p.off += (long long)digit * m.stride[a];
+      } else {
+        const int w = digit * m.weight[a];
+        p.u0 += r == 0 ? w : 0;
+        p.u1 += r == 1 ? w : 0;
+        p.u2 += r == 2 ? w : 0;
+        p.u3 += r == 3 ? w : 0;
+      }
+    }
+  }
+  return p;
+}
+// sum of two contributions -> source offset (base added, rolled coordinates wrapped); maps with at most two rolls whose
+// wrapped coordinate is an affine coordinate of the producer (roll_n_parts <= 1)
+__device__ __forceinline__ long long devmap_finish2(const DevMap& m, long long off, int u0, int u1) {
+  off += m.base;
+  if (m.n_rolls > 0) {
+    int v = u0 + m.roll_shift[0];
+    if (v >= m.roll_mod[0]) v -= m.roll_mod[0];
+    off += (long long)v * m.roll_stride[0];
+  }
+  if (m.n_rolls > 1) {
+    int v = u1 + m.roll_shift[1];
+    if (v >= m.roll_mod[1]) v -= m.roll_mod[1];
+    off += (long long)v * m.roll_stride[1];
+  }
+  return off;
+}
+// Host: first trailing atom such that the atoms [split, n_atoms) have extents whose product is P and devmap_finish2
+// applies; -1 if the map does not split there (callers then evaluate every index in full).
+int devmap_split(const DevMap& m, long long P);
 
 // Host: builds a DevMap over atoms [a0, a1) of a public map, treating `unit` elements of the
 // innermost selected atom as one unit (unit must divide its extent; its stride must be 1 when

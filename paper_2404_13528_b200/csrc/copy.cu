@@ -44,6 +44,16 @@ bool make_devmap(const smartmem_index_map_t& m, int a0, int a1, int unit, bool w
   return true;
 }
 
+int devmap_split(const DevMap& m, long long P) {
+  if (m.n_rolls > 2) return -1;
+  for (int r = 0; r < m.n_rolls; ++r)
+    if (m.roll_n_parts[r] > 1) return -1;
+  long long prod = 1;
+  int a = m.n_atoms;
+  while (a > 0 && prod < P) prod *= m.ext[--a].d;
+  return prod == P ? a : -1;
+}
+
 namespace {
 
 template <int VB> struct VecT;

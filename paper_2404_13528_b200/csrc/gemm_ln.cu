@@ -325,12 +325,7 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
 
 template <int KDIM>
 int launch_t(const CUtensorMap& tw, const CUtensorMap& toa, const CUtensorMap& tob, LnGemmArgs& g, size_t smem, cudaStream_t st) {
-  static bool configured = false;
-  if (!configured) {
-    if (cudaFuncSetAttribute(gemm_ln_kernel<KDIM>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448) != cudaSuccess)
-      return SMARTMEM_ERR_CUDA;
-    configured = true;
-  }
+  if (ensure_max_dynamic_smem((const void*)gemm_ln_kernel<KDIM>, 232448) != SMARTMEM_OK) return SMARTMEM_ERR_CUDA;
   const unsigned grid = (unsigned)(g.tiles < tc_sm_count() ? g.tiles : tc_sm_count());
   if (launch_pdl(gemm_ln_kernel<KDIM>, dim3(grid), dim3(kThreads), smem, st, tw, toa, tob, g) != cudaSuccess) return SMARTMEM_ERR_CUDA;
   count_launch();

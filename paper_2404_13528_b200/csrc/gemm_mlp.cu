@@ -489,12 +489,7 @@ int launch_mlp_fused(const void* A, const void* ln_gamma, const void* ln_beta, f
   const size_t smem = need + 1024 <= 232448 ? need + 1024 : 232448;     // alignment slack only while it fits
   if (need > smem) return SMARTMEM_ERR_UNSUPPORTED;
   g.smem_bytes = (uint32_t)smem;
-  static bool configured = false;
-  if (!configured) {
-    if (cudaFuncSetAttribute(mlp_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448) != cudaSuccess)
-      return SMARTMEM_ERR_CUDA;
-    configured = true;
-  }
+  if (ensure_max_dynamic_smem((const void*)mlp_fused_kernel, 232448) != SMARTMEM_OK) return SMARTMEM_ERR_CUDA;
   profile_tick("mlp_fused", st);
   const unsigned grid = (unsigned)(g.tiles < tc_sm_count() ? g.tiles : tc_sm_count());
   launch_pdl(mlp_fused_kernel, dim3(grid), dim3(kThreads), smem, st, ta, tw1, tw2, g);

@@ -622,13 +622,7 @@ int launch_t(const CUtensorMap& ta, const CUtensorMap& tb, const GemmArgs& g, cu
   constexpr int RCc = (BN == 256 && STAGES == 4) ? 16 : ((BN / 4) > 32 ? 32 : (BN / 4));
   constexpr size_t smem = 1024 + STAGES * (A_STAGE_BYTES + BN * BK * 2) + (2 * STAGES + 4) * 8 + 16 +
                           ((BN == 256 && STAGES == 4) ? kEpiWarps * 32 * (RCc * 2 + 16) : 4 * 32 * (BN * 2 + 16));
-  static bool configured = false;
-  if (!configured) {
-    if (cudaFuncSetAttribute(gemm_tc_kernel<BN, STAGES, A_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-        cudaSuccess)
-      return SMARTMEM_ERR_CUDA;
-    configured = true;
-  }
+  if (ensure_max_dynamic_smem((const void*)gemm_tc_kernel<BN, STAGES, A_MN>, (int)smem) != SMARTMEM_OK) return SMARTMEM_ERR_CUDA;
   profile_tick("gemm_tc", st);
   const long long tiles = (long long)g.tiles_n * g.tiles_m * g.batch;
   const unsigned grid = (unsigned)(tiles < sm_count() ? tiles : sm_count());
@@ -655,6 +649,22 @@ int tc_encode_2d_sw64(const void* ptr, long long inner, long long outer, long lo
   const uint64_t strides[1] = {(uint64_t)pitch_elems * 2};
   const uint32_t box[2] = {(uint32_t)box_inner, (uint32_t)box_outer};
   return encode_cached(ptr, 2, dims, strides, box, out, 64);
+}
+
+int tc_encode_nd_sw64(const void* ptr, int rank, const long long* dims, const long long* strides_elems, const int* box,
+                      CUtensorMap* out) {
+  if (rank < 2 || rank > 5 || ((uintptr_t)ptr & 15) || box[0] * 2 != 64) return SMARTMEM_ERR_ALIGNMENT;
+  uint64_t d[5], sb[4];
+  uint32_t b[5];
+  for (int i = 0; i < rank; ++i) {
+    d[i] = (uint64_t)dims[i];
+    b[i] = (uint32_t)box[i];
+    if (i > 0) {
+      sb[i - 1] = (uint64_t)strides_elems[i - 1] * 2;
+      if (sb[i - 1] % 16) return SMARTMEM_ERR_ALIGNMENT;
+    }
+  }
+  return encode_cached(ptr, rank, d, sb, b, out, 64);
 }
 
 int tc_sm_count() { return sm_count(); }

@@ -51,6 +51,10 @@ int tc_encode_2d(const void* ptr, long long inner, long long outer, long long pi
 // Same with 64-byte swizzle: boxes of 32 bf16 columns (64-byte rows).
 int tc_encode_2d_sw64(const void* ptr, long long inner, long long outer, long long pitch_elems, int box_inner,
                       int box_outer, CUtensorMap* out);
+// bf16 tensor of `rank` dimensions (innermost first; strides in elements for dimensions 1..rank-1) with 64-byte swizzle and a box
+// of 32 innermost elements.
+int tc_encode_nd_sw64(const void* ptr, int rank, const long long* dims, const long long* strides_elems, const int* box,
+                      CUtensorMap* out);
 int tc_sm_count();
 
 // Fused MLP: out = residual + (GELU(LN(A) W1^T + b1)) W2^T + b2 with the hidden activation kept on chip.
@@ -68,5 +72,11 @@ int launch_mlp_fused(const void* A, const void* ln_gamma, const void* ln_beta, f
 bool gemm_ln_supported(long long N, long long K);
 int launch_gemm_ln(const void* X, const DevMap* rowmap, const void* gamma, const void* beta, float eps, const void* W,
                    const void* bias, void* out, long long M, long long N, long long K, cudaStream_t st);
+
+// Attention half of a narrow Swin block (bf16, head dimension 32, 2 or 3 heads, window^2 <= 64) in one kernel:
+// y = x + unshift(unpartition(proj(window_attention(qkv(LN1(partition(shift(x)))))))), every layout operator folded into the
+// row gather / row scatter through `rowmap` (windowed row -> element offset of the token in x and y).  x and y must not alias.
+bool swin_attn_fused_supported(int dtype, int C, int heads, int window);
+int launch_swin_attn_fused(const smartmem_swin_params_t& p, const DevMap& rowmap, const void* x, void* y, cudaStream_t st);
 
 }  // namespace smartmem

@@ -86,20 +86,39 @@ struct Layout {
 
 size_t al(size_t b) { return (b + 255) & ~(size_t)255; }
 
+// Which fused kernels a block takes (they decide which intermediates exist at all).
+struct Path {
+  bool fuse_attn, fuse_ln1, fuse_mlp;
+};
+Path choose_path(const smartmem_swin_params_t& p, int mode) {
+  const bool bf16 = p.dtype == SMARTMEM_BF16;
+  Path t;
+  t.fuse_attn = mode == SMARTMEM_ELIMINATE && swin_attn_fused_supported(p.dtype, p.C, p.heads, p.window);
+  t.fuse_ln1 = bf16 && gemm_ln_supported(3 * (long long)p.C, p.C);
+  t.fuse_mlp = bf16 && p.mlp_ratio > 0 && mlp_fused_supported(p.C, (long long)p.C * p.mlp_ratio);
+  return t;
+}
+
+// Only the intermediates the chosen path writes are reserved.
 Layout ws_layout(const smartmem_swin_params_t& p, int mode) {
   const size_t esz = p.dtype == SMARTMEM_F32 ? 4 : 2;
   const size_t MC = al((size_t)p.B * p.H * p.W * p.C * esz);
+  const Path t = choose_path(p, mode);
   Layout L;
   memset(&L, 0, sizeof(L));
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += bytes; return o; };
-  L.xn = take(MC);
-  L.qkv = take(3 * MC);
-  L.ao = take(MC);
+  if (!t.fuse_attn) {
+    if (!t.fuse_ln1) L.xn = take(MC);
+    L.qkv = take(3 * MC);
+    L.ao = take(MC);
+  }
   if (p.mlp_ratio > 0) {
     L.y1 = take(MC);
-    L.yn = take(MC);
-    L.hid = take((size_t)p.mlp_ratio * MC);
+    if (!t.fuse_mlp) {
+      L.yn = take(MC);
+      L.hid = take((size_t)p.mlp_ratio * MC);
+    }
   }
   if (mode == SMARTMEM_EXPLICIT) {
     L.xs = take(MC);
@@ -111,13 +130,13 @@ Layout ws_layout(const smartmem_swin_params_t& p, int mode) {
     L.orev = take(MC);
     L.ouns = take(MC);
   }
-  L.total = off;
+  L.total = off > 256 ? off : 256;                 // never zero: callers pass a non-null workspace
   return L;
 }
 
 int validate(const smartmem_swin_params_t* p, int mode) {
   if (!p) return SMARTMEM_ERR_INVALID_ARG;
-  if (mode != SMARTMEM_ELIMINATE && mode != SMARTMEM_EXPLICIT) return SMARTMEM_ERR_INVALID_ARG;
+  if (mode != SMARTMEM_ELIMINATE && mode != SMARTMEM_EXPLICIT && mode != SMARTMEM_ELIMINATE_UNFUSED) return SMARTMEM_ERR_INVALID_ARG;
   if (p->dtype != SMARTMEM_F32 && p->dtype != SMARTMEM_BF16) return SMARTMEM_ERR_UNSUPPORTED;
   if (p->B < 1 || p->H < 1 || p->W < 1 || p->C < 1 || p->heads < 1 || p->window < 1 || p->mlp_ratio < 0)
     return SMARTMEM_ERR_SHAPE;
@@ -182,7 +201,8 @@ int run_block(const smartmem_swin_params_t* pp, const void* x, void* y, void* wo
   cudaStream_t st = (cudaStream_t)cuda_stream;
   const bool f32 = p.dtype == SMARTMEM_F32;
   const int esz = f32 ? 4 : 2;
-  const bool elim = mode == SMARTMEM_ELIMINATE;
+  const bool elim = mode != SMARTMEM_EXPLICIT;
+  const Path path = choose_path(p, mode);
   const long long C = p.C, nH = p.heads, d = C / nH, ws = p.window, T = ws * ws;
   const long long M = (long long)p.B * p.H * p.W, nW = M / T, hid = C * p.mlp_ratio;
   char* w = (char*)workspace;
@@ -213,9 +233,12 @@ int run_block(const smartmem_swin_params_t* pp, const void* x, void* y, void* wo
   a.nWw = p.W / p.window; a.win_per_img = (p.H / p.window) * (p.W / p.window);
   a.scale = 1.0f / sqrtf((float)d);
 
-  const bool fuse_ln1 = !f32 && gemm_ln_supported(3 * C, C);
+  const bool fuse_ln1 = path.fuse_ln1;
 #define SM_TRY(label, expr) do { if (tm) tm->tick(label); rc = (expr); if (rc != SMARTMEM_OK) return rc; } while (0)
-  if (elim) {
+  if (path.fuse_attn) {
+    // narrow blocks: the whole attention half in one kernel (rows gathered and scattered through the composed map)
+    SM_TRY("attn_half_fused", launch_swin_attn_fused(p, m.e1_rows, x, y1, st));
+  } else if (elim) {
     if (fuse_ln1) {
       // narrow blocks: LN1, the shift o partition gather and the QKV projection in one kernel
       SM_TRY("ln1_gather_qkv_gemm", launch_gemm_ln(x, &m.e1_rows, p.ln1_g, p.ln1_b, p.ln_eps, p.w_qkv, p.b_qkv, at(L.qkv), M, 3 * C, C, st));
@@ -267,7 +290,7 @@ int run_block(const smartmem_swin_params_t* pp, const void* x, void* y, void* wo
     SM_TRY("proj_gemm_residual", linear(ou, p.w_proj, p.b_proj, y1, C, C, 0, x, nullptr));
   }
   if (p.mlp_ratio > 0) {
-    if (!f32 && mlp_fused_supported(C, hid)) {
+    if (path.fuse_mlp) {
       // narrow blocks: LN2 + fc1 + GELU + fc2 + residual in one kernel; neither the normalised rows
       // nor the hidden activation leave the chip
       SM_TRY("mlp_fused_ln2_fc1_gelu_fc2_residual",

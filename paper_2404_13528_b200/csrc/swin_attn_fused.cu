@@ -1,0 +1,911 @@
+// Attention half of a narrow Swin block (head dimension 32, 2 or 3 heads, C = 32 * heads) in ONE kernel:
+//
+//   y = x + unshift(unpartition( proj( window_attention( qkv( LN1( partition(shift(x)) ) ) ) ) ))
+//
+// The cyclic shift, the window partition, the head split, the K transpose, the head merge, the window
+// reverse and the reverse shift are all index arithmetic here: rows of x are gathered through the
+// composed shift o partition map straight into the MMA operand layout, q / k / v and the attention
+// output never leave the SM, and the result rows are scattered through the same map.  Per token the
+// kernel reads C and writes C elements of global memory; the three-kernel form of the same chain
+// moves 11 C.
+//
+// Unit of work: a pair of windows = one 128-row MMA tile (window w of the pair in rows 64 w .. 64 w + T - 1,
+// the rows between T and 64 stay zero), taken round-robin by persistent CTAs that keep every weight resident.
+// An "item" is (unit, head).  Per item, all in one 128-column buffer of tensor memory (one buffer per head):
+//
+//   acc  = [X | e] [Wq_h; Wk_h; Wv_h | f]^T    128 x 96 x (C + 16)  tcgen05; X = the RAW rows (bf16) in shared memory
+//   q,k,v = rstd acc                           LayerNorm applied algebraically (below); q goes back to tensor memory as
+//                                              bf16 pairs, k and v to shared memory in operand layout
+//   S    = q k^T                               128 x 128 x 32, q read from tensor memory (the two diagonal 64 x 64 blocks are used)
+//   P    = softmax(scale S + bias + mask)      one query row per thread (= its TMEM lane); P stored as bf16 pairs
+//                                              over the S columns it came from
+//   O    = P [v0; v1]                          128 x 32 x 128, P read from tensor memory, block diagonal
+//   Ob   = bf16(O / rowsum)                    back into tensor memory as packed pairs
+//   Y   += Ob Wp[:, 32 h : 32 h + 32]^T        128 x C x 32: the head merge is the accumulation over heads
+//
+// and per unit  y_row = Y + b_proj + x_row, written in place over the raw row in shared memory (the A tile doubles as the
+// residual) and stored with 16-byte vectors, a row's C elements by consecutive lanes.
+//
+// LayerNorm without a normalised tile:  LN(x) W^T + b = rstd (x W'^T - mean c + sigma b'),  W' = bf16(gamma . W) (column
+// scaling), c_n = sum_k W'_nk, b'_n = b_n + sum_k beta_k W_nk, sigma = 1 / rstd.  c is summed from the ROUNDED W', so the
+// mean term cancels exactly what the raw rows contribute through W' -- rows with a large common offset lose nothing.  The two
+// rank-one terms ride on the tensor core as one extra k-step: row r of the operand carries (-mean_r, sigma_r), column n of the
+// weights (c_n, b'_n), each fp32 value split into three bf16 pieces (the six largest cross products of the pieces are kept:
+// exact to 2^-24), so the epilogue of the QKV product is one multiply per element.  Every CTA folds gamma into its resident
+// copy of the weights once (prologue, overlapped with the previous kernel's tail); the row statistics (two passes over the
+// row in registers, fp32) are taken by the warps that gather the rows.
+//
+// Warp roles (16 warps): 0-3 gather the rows of the units ahead (16-byte asynchronous copies through the index map), 4-7 and
+// 8-11 two row groups that alternate over the items (q/k/v epilogue, softmax, O epilogue) -- each group issues its own MMAs
+// from one elected thread right after the group's barrier, so a hand-off costs a barrier and not a trip through another
+// warp --, 12-15 row statistics of the units ahead, Y epilogue and row scatter.  Every wait is bounded.
+#include "attn.cuh"
+#include "gemm_tc.cuh"
+#include "ptx.cuh"
+
+#ifdef FUSED_TIMING
+__device__ long long g_fused_dbg[8192];
+#define FDBG(slot) do { if ((slot) >= 8000) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_fused_dbg[7000 + blockIdx.x * 4 + ((slot) - 8000)] = (long long)t_; } \
+                         if (blockIdx.x == 0) g_fused_dbg[(slot) >= 8000 ? (slot) - 8000 + 6990 : (slot)] = clock64(); } while (0)
+extern "C" __attribute__((visibility("default"))) int smartmem_debug_read_fused(long long* host, int n) {
+  return (int)cudaMemcpyFromSymbol(host, g_fused_dbg, sizeof(long long) * n);
+}
+#else
+#define FDBG(slot) do { } while (0)
+#endif
+
+namespace smartmem {
+namespace {
+
+using ptx::f32x2;
+
+constexpr int D = 32, TP = 64, BM = 128;
+constexpr int KBT = BM * 64;                        // a 128-row x 32-column bf16 tile: 64-byte rows, 64-byte swizzle
+constexpr int AX_BYTES = BM * 32;                   // the extra k-step of a unit: 128 rows x 16 bf16, no swizzle
+constexpr int WROWS = 96;                           // rows of a per-head QKV weight tile: q_h, k_h, v_h
+constexpr int WQ_TILE = WROWS * 64;
+constexpr int WX_TILE = WROWS * 32;                 // the extra k-step of a head's weights
+constexpr int KV_SLOT = 2 * KBT;                    // k, v tiles of one item
+constexpr int NSLOT = 2;
+constexpr int kLoaderThreads = 128, kThreads = 512;
+constexpr uint32_t TMEM_COLS = 512;
+constexpr uint32_t TM_Y = 384, TM_Q = 480;          // after three 128-column item buffers: Y (C columns), two q slots of 16
+constexpr uint32_t ROW_INVALID = 0xFFFFFFFFu, ROW_BOX = 0xFFFFFFFEu;   // no such row / a row of a window moved as a TMA box
+constexpr int WIN_MISSING = 0, WIN_GATHER = 1, WIN_BOX = 2;
+constexpr int N_BARS = 24;
+
+struct FusedArgs {
+  int n_windows, n_pairs, T, ws, shift;
+  int nWw, nWh, win_per_img;
+  FastDiv fd_wpi, fd_nww;
+  int na;                                           // depth of the row ring (2 or 3)
+  uint32_t smem_bytes;
+  float eps, scale;
+  const __nv_bfloat16 *x, *ln_g, *ln_b, *b_qkv, *b_proj, *table;
+  __nv_bfloat16* y;
+  int* status;
+  int use_box;                                      // windows off the seam move as TMA boxes (tensor maps over x and y are valid)
+  int split;                                        // first atom of rowmap that indexes the token inside its window (-1: evaluate every row in full)
+  DevMap rowmap;                                    // row n T + i of the windowed view -> element offset of the token in x (and y)
+};
+
+__device__ __forceinline__ uint64_t desc_sw64(uint32_t smem_addr) {   // 64-byte rows, 8-row groups 512 bytes apart
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)(16 >> 4) << 16;
+  d |= (uint64_t)(512 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)4 << 61;
+  return d;
+}
+// K-major tile without swizzle: 8 x 16-byte core matrices; the two of a k16 step 128 bytes apart, 8-row groups 256 bytes apart
+__device__ __forceinline__ uint64_t desc_plain(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)(128 >> 4) << 16;
+  d |= (uint64_t)(256 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  return d;
+}
+__device__ __forceinline__ uint32_t plain_off(int row, int kc) { return (uint32_t)((row >> 3) * 256 + kc * 128 + (row & 7) * 16); }
+__device__ __forceinline__ float ex2f(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// byte offset of 16-byte chunk `ch` (0..3) of row `row` inside a 64-byte-row tile with the 64-byte swizzle
+__device__ __forceinline__ uint32_t sw64_off(int row, int ch) { return (uint32_t)(row * 64 + ((ch ^ ((row >> 1) & 3)) << 4)); }
+
+// v = hi + mid + lo with three bf16 pieces (24 significant bits)
+__device__ __forceinline__ void split3(float v, uint32_t& hi, uint32_t& mid, uint32_t& lo) {
+  const __nv_bfloat16 a = __float2bfloat16_rn(v);
+  const float r1 = v - __bfloat162float(a);
+  const __nv_bfloat16 b = __float2bfloat16_rn(r1);
+  const __nv_bfloat16 c = __float2bfloat16_rn(r1 - __bfloat162float(b));
+  hi = __bfloat16_as_ushort(a); mid = __bfloat16_as_ushort(b); lo = __bfloat16_as_ushort(c);
+}
+// The extra k-step.  Operand side (per row): pieces of u = -mean and s = sigma; weight side (per column): pieces of c and b'.
+// Position by position the products are  u_h c_h, u_h c_m, u_m c_h, u_h c_l, u_l c_h, u_m c_m  and the same for (s, b').
+__device__ __forceinline__ void extra_row(float u, float s, uint4& k0, uint4& k1) {
+  uint32_t uh, um, ul, sh, sm_, sl;
+  split3(u, uh, um, ul);
+  split3(s, sh, sm_, sl);
+  k0 = make_uint4(uh | (uh << 16), um | (uh << 16), ul | (um << 16), sh | (sh << 16));
+  k1 = make_uint4(sm_ | (sh << 16), sl | (sm_ << 16), 0u, 0u);
+}
+__device__ __forceinline__ void extra_col(float c, float b, uint4& k0, uint4& k1) {
+  uint32_t ch, cm, cl, bh, bm, bl;
+  split3(c, ch, cm, cl);
+  split3(b, bh, bm, bl);
+  k0 = make_uint4(ch | (cm << 16), ch | (cl << 16), ch | (cm << 16), bh | (bm << 16));
+  k1 = make_uint4(bh | (bl << 16), bh | (bm << 16), 0u, 0u);
+}
+
+template <int NH, int KC>
+__global__ void __launch_bounds__(kThreads, 1)
+swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_constant__ CUtensorMap tmWp,
+                       const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY,
+                       const __grid_constant__ FusedArgs g) {
+  constexpr int C = NH * D, NCH = C / 8;             // channels, 16-byte chunks per row
+  constexpr int A_BYTES = NH * KBT;                  // a unit's raw rows: NH k-blocks of 32 columns
+  constexpr int WP_TILE = C * 64;                    // Wp[:, 32 h : 32 h + 32]: C rows x 64 bytes
+  constexpr int BR = KC == 56 ? 28 : 36;             // 32-bit words per bias row (16-byte reads of 8 consecutive rows hit distinct banks)
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t pad = (1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u;
+  uint8_t* smem = smem_raw + pad;
+  const int T = g.T, ws = g.ws, na = g.na;
+  uint8_t* sA = smem;                                              // [na][NH k-blocks][8 KB]
+  uint8_t* sKV = sA + na * A_BYTES;                                // [2 slots][k, v][8 KB]
+  uint8_t* sWq = sKV + NSLOT * KV_SLOT;                            // [NH heads][NH k-blocks][96 rows x 64 B]
+  uint8_t* sWp = sWq + NH * NH * WQ_TILE;                          // [NH heads][C rows x 64 B]
+  uint8_t* sAx = sWp + NH * WP_TILE;                               // [na][128 rows x 32 B]
+  uint8_t* sWx = sAx + na * AX_BYTES;                              // [NH heads][96 rows x 32 B]
+  uint32_t* bias_s = reinterpret_cast<uint32_t*>(sWx + NH * WX_TILE);   // [NH][T][BR]: bf16 pairs
+  float* bp_s = reinterpret_cast<float*>(bias_s + NH * T * BR);    // [C]
+  float* rstd_s = bp_s + C;                                        // [na][128]
+  uint32_t* rowoff_s = reinterpret_cast<uint32_t*>(rstd_s + na * BM);   // [na][128]: row offset in 16-byte units
+  float* ln_s = reinterpret_cast<float*>(rowoff_s + na * BM);      // [2][C]: gamma, beta
+  int* tyx_s = reinterpret_cast<int*>(ln_s + 2 * C);               // [64]: ty << 8 | tx
+  uint32_t* kmask_s = reinterpret_cast<uint32_t*>(tyx_s + TP);     // [4]
+  int4* tok_s = reinterpret_cast<int4*>(kmask_s + 4);              // [64]: the map's contribution of token t: (offset, u0, u1, -)
+  int4* win_s = tok_s + TP;                                        // [2 units][2 windows]: the contribution of window n: (offset lo, hi, u0, u1)
+  int4* wbox_s = win_s + 4;                                        // [na][2 windows]: (kind, first column, first row, image) of the window
+  uint64_t* bars = reinterpret_cast<uint64_t*>(wbox_s + 6);
+  uint64_t* w_full = bars;
+  uint64_t *a_full = bars + 1, *a_free = a_full + 3, *landed = a_free + 3;     // [3] each
+  uint64_t *acc_full = landed + 3, *s_full = acc_full + 3, *o_full = s_full + 3;
+  uint64_t *y_full = o_full + 3, *y_empty = y_full + 1, *pj_done = y_empty + 1, *ysync = pj_done + 1;   // ysync [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ysync + 2);
+  int* abort_flag = reinterpret_cast<int*>(tmem_slot + 1);
+  uint16_t* raw_s = reinterpret_cast<uint16_t*>(sKV);              // prologue scratch: the raw table columns, [NH][256]
+
+  if (pad + (uint32_t)(reinterpret_cast<uint8_t*>(tmem_slot + 4) - smem) > g.smem_bytes) {
+    if (threadIdx.x == 0) atomicExch(g.status, (int)SMARTMEM_ERR_UNSUPPORTED);
+    return;
+  }
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
+  if (tid == 0) FDBG(8000);
+  const int cidx = blockIdx.x, cstride = gridDim.x;
+  const int U = cidx < g.n_pairs ? (g.n_pairs - cidx + cstride - 1) / cstride : 0;   // units of this CTA
+  const int total = U * NH;                                                         // items
+  const float LOG2E = 1.4426950408889634f;
+
+  if (tid == 0) {
+    ptx::mbar_init(w_full, 1);
+    for (int i = 0; i < 3; ++i) {
+      ptx::mbar_init(&a_full[i], 4);
+      ptx::mbar_init(&a_free[i], 4);
+      ptx::mbar_init(&landed[i], 4);
+      ptx::mbar_init(&acc_full[i], 1);
+      ptx::mbar_init(&s_full[i], 1);
+      ptx::mbar_init(&o_full[i], 1);
+    }
+    ptx::mbar_init(y_full, 1);
+    ptx::mbar_init(y_empty, 4);
+    ptx::mbar_init(pj_done, 1);
+    ptx::mbar_init(&ysync[0], 2);
+    ptx::mbar_init(&ysync[1], 2);
+    *abort_flag = 0;
+    ptx::fence_barrier_init();
+    ptx::fence_proxy_async();
+    // the weights do not depend on the kernel before this one: fetch them right away
+    ptx::prefetch_tensormap(&tmWq);
+    ptx::prefetch_tensormap(&tmWp);
+    ptx::prefetch_tensormap(&tmX);
+    ptx::prefetch_tensormap(&tmY);
+    ptx::mbar_expect_tx(w_full, (uint32_t)(NH * NH * WQ_TILE + NH * WP_TILE));
+    for (int h = 0; h < NH; ++h) {
+      for (int kb = 0; kb < NH; ++kb)
+        for (int which = 0; which < 3; ++which)
+          ptx::tma_load_2d(sWq + (h * NH + kb) * WQ_TILE + which * (D * 64), &tmWq, w_full, kb * D, which * C + h * D);
+      ptx::tma_load_2d(sWp + h * WP_TILE, &tmWp, w_full, h * D, 0);
+    }
+  }
+  if (warp == 0) ptx::tmem_alloc(tmem_slot, TMEM_COLS);
+  // parameter-only tables
+  const int n_table = (2 * ws - 1) * (2 * ws - 1);
+  for (int i = tid; i < NH * 256; i += kThreads) {
+    const int h = i >> 8, e = i & 255;
+    raw_s[i] = e < n_table ? reinterpret_cast<const uint16_t*>(g.table)[e * NH + h] : (uint16_t)0;
+  }
+  if (tid < TP) {
+    tyx_s[tid] = ((tid / ws) << 8) | (tid % ws);
+    int4 tk = make_int4(0, 0, 0, 0);
+    if (g.split >= 0 && tid < T) {
+      const DevMapPart pt = devmap_part(g.rowmap, g.split, g.rowmap.n_atoms, (uint32_t)tid);
+      tk = make_int4((int)pt.off, pt.u0, pt.u1, 0);
+    }
+    tok_s[tid] = tk;
+  }
+  for (int i = tid; i < C; i += kThreads) {
+    ln_s[i] = __bfloat162float(g.ln_g[i]);
+    ln_s[C + i] = __bfloat162float(g.ln_b[i]);
+    bp_s[i] = __bfloat162float(g.b_proj[i]);
+  }
+  for (int i = tid; i < na * A_BYTES / 16; i += kThreads) reinterpret_cast<uint4*>(sA)[i] = make_uint4(0, 0, 0, 0);
+  for (int i = tid; i < na * AX_BYTES / 16; i += kThreads) reinterpret_cast<uint4*>(sAx)[i] = make_uint4(0, 0, 0, 0);
+  for (int i = tid; i < na * BM; i += kThreads) {
+    rstd_s[i] = 0.f;
+    rowoff_s[i] = ROW_INVALID;
+  }
+  __syncthreads();
+  // each head's bias as a [T, T] table of bf16 pairs, -inf for the padded keys
+  for (int i = tid; i < NH * T * (KC / 2); i += kThreads) {
+    const int hr = i / (KC / 2), c2 = i - hr * (KC / 2);            // (head, row), pair of keys
+    const int h = hr / T, r = hr - h * T;
+    const int ry = tyx_s[r] >> 8, rx = tyx_s[r] & 255;
+    uint32_t word = 0;
+    for (int k = 0; k < 2; ++k) {
+      const int c = 2 * c2 + k;
+      uint32_t bits = 0xFF80u;                         // -inf: padded keys never contribute
+      if (c < T) {
+        const int cy = tyx_s[c] >> 8, cx = tyx_s[c] & 255;
+        bits = raw_s[h * 256 + (ry - cy + ws - 1) * (2 * ws - 1) + (rx - cx + ws - 1)];
+      }
+      word |= bits << (16 * k);
+    }
+    bias_s[hr * BR + c2] = word;
+  }
+  // keys below / right of the wrap line of a seam window (bit c = key c)
+  if (warp == 2) {
+    const int c0 = lane, c1 = lane + 32;
+    const bool y0 = c0 < T && (tyx_s[c0] >> 8) >= ws - g.shift, y1 = c1 < T && (tyx_s[c1] >> 8) >= ws - g.shift;
+    const bool x0 = c0 < T && (tyx_s[c0] & 255) >= ws - g.shift, x1 = c1 < T && (tyx_s[c1] & 255) >= ws - g.shift;
+    const uint32_t m0 = __ballot_sync(0xFFFFFFFFu, y0), m1 = __ballot_sync(0xFFFFFFFFu, y1);
+    const uint32_t m2 = __ballot_sync(0xFFFFFFFFu, x0), m3 = __ballot_sync(0xFFFFFFFFu, x1);
+    if (lane == 0) { kmask_s[0] = m0; kmask_s[1] = m1; kmask_s[2] = m2; kmask_s[3] = m3; }
+  }
+  // fold gamma into the resident QKV weights; the column terms c_n and b'_n go into the extra k-step (thread = one weight row)
+  const bool w_ok = ptx::mbar_wait(w_full, 0, abort_flag, g.status);
+  if (w_ok && tid < NH * WROWS) {
+    const int h = tid / WROWS, rr = tid - h * WROWS;
+    const int which = rr >> 5, j = rr & 31;
+    float csum = 0.f, bsum = __bfloat162float(g.b_qkv[which * C + h * D + j]);
+#pragma unroll
+    for (int kb = 0; kb < NH; ++kb) {
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint4* p = reinterpret_cast<uint4*>(sWq + (h * NH + kb) * WQ_TILE + sw64_off(rr, c));
+        const uint4 wv = *p;
+        const uint32_t w4[4] = {wv.x, wv.y, wv.z, wv.w};
+        uint32_t o4[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int k = kb * D + c * 8 + 2 * e;
+          const float2 f = bf16x2_to_float2(w4[e]);
+          bsum = fmaf(ln_s[C + k], f.x, bsum);
+          bsum = fmaf(ln_s[C + k + 1], f.y, bsum);
+          o4[e] = float2_to_bf16x2(ln_s[k] * f.x, ln_s[k + 1] * f.y);
+          const float2 r2 = bf16x2_to_float2(o4[e]);
+          csum += r2.x + r2.y;
+        }
+        *p = make_uint4(o4[0], o4[1], o4[2], o4[3]);
+      }
+    }
+    uint4 k0, k1;
+    extra_col(csum, bsum, k0, k1);
+    *reinterpret_cast<uint4*>(sWx + h * WX_TILE + plain_off(rr, 0)) = k0;
+    *reinterpret_cast<uint4*>(sWx + h * WX_TILE + plain_off(rr, 1)) = k1;
+  }
+  ptx::fence_proxy_async();                           // the rewritten weights -> visible to the MMAs
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  if (tid == 0) FDBG(8001);
+  pdl_wait();                                         // everything above depends on parameters only
+  pdl_launch_dependents();
+  if (tid == 0) FDBG(8002);
+
+  if (warp < 4) {
+    // ---- gather: rows of the units ahead through the index map, as 16-byte asynchronous copies into the operand layout ----
+    const int lt = tid;                                // 0 .. 127
+    constexpr int RPI = kLoaderThreads / NCH;          // rows per round of the copy loop: a row by NCH consecutive threads
+    const int my_ch = lt % NCH, my_slot = lt / NCH;
+    bool ok = true;
+    auto vote = [&](bool pred, bool all) {             // OR (all = false) or AND (all = true) over the loader threads; also a barrier
+      uint32_t res;
+      if (all)
+        asm volatile("{\n\t.reg .pred pin, pout;\n\tsetp.ne.u32 pin, %1, 0;\n\tbar.red.and.pred pout, 1, 128, pin;\n\tselp.u32 %0, 1, 0, pout;\n\t}"
+                     : "=r"(res) : "r"(pred ? 1u : 0u) : "memory");
+      else
+        asm volatile("{\n\t.reg .pred pin, pout;\n\tsetp.ne.u32 pin, %1, 0;\n\tbar.red.or.pred pout, 1, 128, pin;\n\tselp.u32 %0, 1, 0, pout;\n\t}"
+                     : "=r"(res) : "r"(pred ? 1u : 0u) : "memory");
+      return res != 0;
+    };
+    auto window_part = [&](int ul) {                   // threads 0, 1: the leading atoms' contribution of the unit's two windows
+      if (lt < 2 && ul < U && g.split >= 0) {
+        const int n = 2 * (cidx + ul * cstride) + lt;
+        int4 wp = make_int4(0, 0, 0, 0);
+        if (n < g.n_windows) {
+          const DevMapPart pw = devmap_part(g.rowmap, 0, g.split, (uint32_t)n);
+          wp = make_int4((int)(uint32_t)(pw.off & 0xFFFFFFFFll), (int)(pw.off >> 32), pw.u0, pw.u1);
+        }
+        win_s[(ul & 1) * 2 + lt] = wp;
+      }
+    };
+    // A window that does not straddle the seam of the shifted image is an affine box [32 channels, ws, ws] of x per k-block: one
+    // TMA copy lands it in the operand layout.  A seam window is gathered row by row through the map.
+    auto issue_loads = [&](int ul) {
+      const int ab = ul % na;
+      const int p = cidx + ul * cstride;
+      {                                                 // a thread per row of the pair tile: the window's kind, the row's offset
+        const int w = lt >> 6, i = lt & 63, n = 2 * p + w;
+        int kind = WIN_MISSING, wy = 0, wx = 0, b = 0;
+        if (n < g.n_windows) {
+          b = (int)fd_div((uint32_t)n, g.fd_wpi);
+          const int wl = n - b * g.win_per_img;
+          wy = (int)fd_div((uint32_t)wl, g.fd_nww);
+          wx = wl - wy * g.nWw;
+          const bool seam = g.shift > 0 && (wy == g.nWh - 1 || wx == g.nWw - 1);
+          kind = (seam || !g.use_box) ? WIN_GATHER : WIN_BOX;
+        }
+        uint32_t off16 = ROW_INVALID;
+        if (i < T && kind == WIN_BOX) off16 = ROW_BOX;
+        if (i < T && kind == WIN_GATHER) {
+          long long off;
+          if (g.split >= 0) {
+            const int4 wp = win_s[(ul & 1) * 2 + w], tk = tok_s[i];
+            const long long woff = (long long)(((unsigned long long)(uint32_t)wp.y << 32) | (uint32_t)wp.x);
+            off = devmap_finish2(g.rowmap, woff + tk.x, wp.z + tk.y, wp.w + tk.z);
+          } else {
+            off = devmap_eval_unrolled(g.rowmap, (uint32_t)(n * T + i));
+          }
+          off16 = (uint32_t)(off >> 3);
+        }
+        rowoff_s[ab * BM + lt] = off16;
+        if (i == 0) {
+          wbox_s[ab * 2 + w] = make_int4(kind, wx * ws + g.shift, wy * ws + g.shift, b);
+          if (kind == WIN_BOX) {                        // this thread moves the window
+            ptx::mbar_add_tx(&landed[ab], (uint32_t)(T * C * 2));     // (no arrival: the loader warps arrive when their copies have landed)
+#pragma unroll
+            for (int kb = 0; kb < NH; ++kb)
+              ptx::tma_load_4d(sA + ab * A_BYTES + kb * KBT + w * (64 * 64), &tmX, &landed[ab], kb * D, wx * ws + g.shift,
+                               wy * ws + g.shift, b);
+          }
+        }
+      }
+      asm volatile("bar.sync 2, 128;" ::: "memory");
+      uint8_t* tile = sA + ab * A_BYTES + (my_ch >> 2) * KBT;
+      for (int v = my_slot; v < 2 * T && my_slot < RPI; v += RPI) {
+        const int w = v >= T ? 1 : 0, row = w * 64 + (v - w * T);
+        const uint32_t o = rowoff_s[ab * BM + row];
+        uint8_t* dst = tile + sw64_off(row, my_ch & 3);
+        if (o == ROW_INVALID) *reinterpret_cast<uint4*>(dst) = make_uint4(0, 0, 0, 0);    // a missing window: no stale rows
+        else if (o != ROW_BOX) ptx::cp_async16(dst, g.x + ((size_t)o << 3) + my_ch * 8);
+      }
+      ptx::cp_async_commit();
+      window_part(ul + 1);                             // read after the next barrier of the loader threads
+    };
+    // A unit's gather is issued as soon as its ring slot is free (the epilogue of unit ul - na has scattered its rows); when no
+    // slot is free the oldest gather in flight is waited for and handed on.
+    window_part(0);
+    asm volatile("bar.sync 2, 128;" ::: "memory");
+    int issued = 0, done = 0;
+    while (done < U) {
+      if (issued < U && issued - done < na) {
+        uint64_t* bar = &a_free[issued % na];
+        const uint32_t par = (uint32_t)(((issued / na) & 1) ^ 1);
+        bool ready;
+        if (issued == done) {
+          ok = ptx::mbar_wait_relaxed(bar, par, abort_flag, g.status, 64);
+          if (vote(!ok, false)) break;
+          ready = true;
+        } else {
+          ready = vote(ptx::mbar_test(bar, par), true);
+        }
+        if (ready) {
+          if (lt == 0) FDBG(4096 + issued * 8 + 0);
+          issue_loads(issued);
+          if (lt == 0) FDBG(4096 + issued * 8 + 1);
+          ++issued;
+          continue;
+        }
+      }
+      const int pending = issued - done;               // cp.async groups in flight; the oldest belongs to unit `done`
+      if (pending >= 3) ptx::cp_async_wait<2>();
+      else if (pending == 2) ptx::cp_async_wait<1>();
+      else ptx::cp_async_wait<0>();
+      ptx::fence_proxy_async();                        // the gathered rows -> visible to the MMAs
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&landed[done % na]);
+      if (lt == 0) FDBG(4096 + done * 8 + 2);
+      ++done;
+    }
+  } else if (warp < 12) {
+    // ---- row groups: group gi takes the items it = gi (mod 2); one row of the pair tile per thread.  The group's elected thread
+    // issues the item's S, P V and projection products, and the QKV product of the SAME head of the next unit (whose accumulator
+    // takes over the tensor-memory buffer this item leaves), each right after the group barrier that completes its inputs. ------
+    const int gi = (warp - 4) >> 2;
+    const int q = warp & 3;                            // TMEM lane quadrant
+    const int r = q * 32 + lane;
+    const int w = r >> 6, i = r & 63;                  // window of the pair, token
+    const bool elected = q == 0 && lane == 0;
+    const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
+    const int my_ty = tyx_s[i] >> 8, my_tx = tyx_s[i] & 255;
+    const uint32_t ky_lo = kmask_s[0], ky_hi = kmask_s[1], kx_lo = kmask_s[2], kx_hi = kmask_s[3];
+    const uint32_t my_fy = my_ty >= ws - g.shift ? 0xFFFFFFFFu : 0u, my_fx = my_tx >= ws - g.shift ? 0xFFFFFFFFu : 0u;
+    uint8_t* slot_base = sKV + gi * KV_SLOT;
+    const f32x2 scale2 = ptx::pack2(g.scale, g.scale), log2e2 = ptx::pack2(LOG2E, LOG2E);
+    bool ok = true;
+    auto group_sync = [&]() {                          // barrier of the group's 128 threads; true if one of them gave up waiting
+      uint32_t gave_up;
+      asm volatile(
+          "{\n\t.reg .pred pin, pout;\n\t"
+          "setp.ne.u32 pin, %2, 0;\n\t"
+          "bar.red.or.pred pout, %1, 128, pin;\n\t"
+          "selp.u32 %0, 1, 0, pout;\n\t}"
+          : "=r"(gave_up)
+          : "r"(3 + gi), "r"(ok ? 0u : 1u)
+          : "memory");
+      return gave_up != 0;
+    };
+    // acc[h] = [X | e] [Wq_h; Wk_h; Wv_h | f]^T of item `it` (elected thread)
+    auto issue_qkv = [&](int it) {
+      const int ul = it / NH, h = it - ul * NH, ab = ul % na;
+      ok = ok && ptx::mbar_wait(&a_full[ab], (ul / na) & 1, abort_flag, g.status);
+      if (!ok) return;
+      ptx::tc_fence_after();
+      const uint32_t idesc = ptx::make_idesc_bf16(BM, WROWS, false, false);
+      const uint32_t d = tmem_base + h * 128;
+      const uint32_t a_base = ptx::smem_u32(sA) + ab * A_BYTES, w_base = ptx::smem_u32(sWq) + h * NH * WQ_TILE;
+#pragma unroll
+      for (int kb = 0; kb < NH; ++kb) {
+        const uint64_t ad = desc_sw64(a_base + kb * KBT), bd = desc_sw64(w_base + kb * WQ_TILE);
+        ptx::tc_mma_bf16(d, ad, bd, idesc, kb ? 1u : 0u);
+        ptx::tc_mma_bf16(d, ad + 2, bd + 2, idesc, 1u);          // next 16 channels: +32 bytes
+      }
+      ptx::tc_mma_bf16(d, desc_plain(ptx::smem_u32(sAx) + ab * AX_BYTES), desc_plain(ptx::smem_u32(sWx) + h * WX_TILE), idesc, 1u);
+      ptx::tc_commit(&acc_full[h]);
+    };
+    if (elected)                                       // the first unit's items of this group; later ones follow their predecessor's epilogue
+      for (int it0 = gi; it0 < NH && it0 < total; it0 += 2) issue_qkv(it0);
+    for (int it = gi; it < total; it += 2) {
+      const int ul = it / NH, h = it - ul * NH;
+      const int ab = ul % na;
+      const uint32_t tb = tmem_base + h * 128 + lane_addr;
+      // -- q, k, v of this row: rstd times the accumulator (the mean and bias terms rode on the extra k-step) --
+      if (elected) FDBG(it * 16 + 0);
+      ok = ok && ptx::mbar_wait(&a_full[ab], (ul / na) & 1, abort_flag, g.status) &&     // (long complete: orders the read of rstd)
+           ptx::mbar_wait(&acc_full[h], ul & 1, abort_flag, g.status);
+      if (elected) FDBG(it * 16 + 1);
+      if (ok) {
+        ptx::tc_fence_after();
+        const float rstd = rstd_s[ab * BM + r];
+        const f32x2 r2 = ptx::pack2(rstd, rstd);
+        uint32_t rv[96];
+        ptx::tmem_ld32(tb, rv);
+        ptx::tmem_ld32(tb + 32, rv + 32);
+        ptx::tmem_ld32(tb + 64, rv + 64);
+        ptx::tmem_ld_wait();
+        uint32_t pk[48];
+#pragma unroll
+        for (int c = 0; c < 48; ++c) {
+          float v0, v1;
+          ptx::unpack2(ptx::mul2(ptx::pack2(__uint_as_float(rv[2 * c]), __uint_as_float(rv[2 * c + 1])), r2), v0, v1);
+          pk[c] = float2_to_bf16x2(v0, v1);
+        }
+        ptx::tmem_st16(tmem_base + TM_Q + gi * 16 + lane_addr, pk);           // q: the S product's A operand
+#pragma unroll
+        for (int kv = 0; kv < 2; ++kv)
+#pragma unroll
+          for (int c = 0; c < 4; ++c)
+            *reinterpret_cast<uint4*>(slot_base + kv * KBT + sw64_off(r, c)) =
+                make_uint4(pk[16 + kv * 16 + c * 4], pk[17 + kv * 16 + c * 4], pk[18 + kv * 16 + c * 4], pk[19 + kv * 16 + c * 4]);
+        ptx::tmem_st_wait();
+        ptx::fence_proxy_async();                      // generic-proxy writes -> visible to the MMAs
+        ptx::tc_fence_before();
+      }
+      if (group_sync()) break;
+      if (elected) {
+        // S = q k^T into the buffer the accumulator has just left; q from its tensor-memory slot
+        ptx::tc_fence_after();
+        const uint32_t idesc = ptx::make_idesc_bf16(BM, 128, false, false);
+        const uint32_t qa = tmem_base + TM_Q + gi * 16;
+        const uint64_t kd = desc_sw64(ptx::smem_u32(slot_base));
+        ptx::tc_mma_bf16_ta(tmem_base + h * 128, qa, kd, idesc, 0u);
+        ptx::tc_mma_bf16_ta(tmem_base + h * 128, qa + 8, kd + 2, idesc, 1u);
+        ptx::tc_commit(&s_full[h]);
+        FDBG(it * 16 + 2);
+      }
+      // -- seam mask of this row's window (shifted blocks: windows in the last window row or column) --
+      const int n = 2 * (cidx + ul * cstride) + w;
+      bool masked = false;
+      uint32_t diff_lo = 0, diff_hi = 0;
+      if (g.shift > 0 && n < g.n_windows) {
+        const int wl = n - (int)fd_div((uint32_t)n, g.fd_wpi) * g.win_per_img;
+        const int wy = (int)fd_div((uint32_t)wl, g.fd_nww), wx = wl - wy * g.nWw;
+        const bool last_row = wy == g.nWh - 1, last_col = wx == g.nWw - 1;
+        masked = last_row || last_col;
+        if (last_row) { diff_lo |= ky_lo ^ my_fy; diff_hi |= ky_hi ^ my_fy; }
+        if (last_col) { diff_lo |= kx_lo ^ my_fx; diff_hi |= kx_hi ^ my_fx; }
+      }
+      const uint32_t* brow = bias_s + (h * T + (i < T ? i : 0)) * BR;
+      // -- softmax of this row over its window's keys --
+      ok = ptx::mbar_wait(&s_full[h], ul & 1, abort_flag, g.status);
+      if (elected) FDBG(it * 16 + 3);
+      float inv = 0.f;
+      if (ok) {
+        ptx::tc_fence_after();
+        uint32_t rv[KC];
+        const uint32_t ts = tb + w * 64;               // this window's 64 key columns
+        ptx::tmem_ld32(ts, rv);
+        if constexpr (KC == 64) {
+          ptx::tmem_ld32(ts + 32, rv + 32);
+        } else {
+          ptx::tmem_ld16(ts + 32, rv + 32);
+          ptx::tmem_ld8(ts + 48, rv + 48);
+        }
+        ptx::tmem_ld_wait();
+        float sc[KC];
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+        for (int v8 = 0; v8 < KC / 8; ++v8) {
+          const uint4 b4 = *reinterpret_cast<const uint4*>(brow + v8 * 4);
+          const uint32_t bw[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int c = v8 * 8 + 2 * j;
+            ptx::unpack2(ptx::fma2(ptx::pack2(__uint_as_float(rv[c]), __uint_as_float(rv[c + 1])), scale2,
+                                   ptx::pack2(__uint_as_float(bw[j] << 16), __uint_as_float(bw[j] & 0xFFFF0000u))),
+                         sc[c], sc[c + 1]);
+          }
+        }
+        if (masked) {                                  // keys of another region get -100
+#pragma unroll
+          for (int c = 0; c < 32; ++c) {
+            if ((diff_lo >> c) & 1u) sc[c] -= 100.f;
+            if (c + 32 < KC && ((diff_hi >> c) & 1u)) sc[c + 32] -= 100.f;
+          }
+        }
+#pragma unroll
+        for (int c = 0; c < KC; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], sc[c]);
+        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+        const float nmx = -mx * LOG2E;
+        const f32x2 nmx2 = ptx::pack2(nmx, nmx);
+        f32x2 sum2[2] = {0ull, 0ull};
+        uint32_t pk[32];
+#pragma unroll
+        for (int c = KC / 2; c < 32; ++c) pk[c] = 0u;        // padding keys
+#pragma unroll
+        for (int c = 0; c < KC; c += 2) {
+          float e0, e1;
+          ptx::unpack2(ptx::fma2(ptx::pack2(sc[c], sc[c + 1]), log2e2, nmx2), e0, e1);
+          const float p0 = ex2f(e0), p1 = ex2f(e1);
+          sum2[(c >> 1) & 1] = ptx::add2(sum2[(c >> 1) & 1], ptx::pack2(p0, p1));
+          pk[c / 2] = float2_to_bf16x2(p0, p1);
+        }
+        float s0, s1, s2, s3;
+        ptx::unpack2(sum2[0], s0, s1);
+        ptx::unpack2(sum2[1], s2, s3);
+        inv = 1.f / ((s0 + s1) + (s2 + s3));
+        // P row (bf16 pairs) over the first 64 columns of the buffer: this window's keys at packed columns
+        // 32 w .. 32 w + 31, zeros for the other window's keys (block-diagonal P)
+        ptx::tmem_st32(tb + w * 32, pk);
+#pragma unroll
+        for (int c = 0; c < 32; ++c) pk[c] = 0u;
+        ptx::tmem_st32(tb + (1 - w) * 32, pk);
+        ptx::tmem_st_wait();
+        ptx::tc_fence_before();
+      }
+      if (group_sync()) break;
+      if (elected) {
+        // O = P [v0; v1]: P from tensor memory (bf16 pairs), V as it lies (MN-major B operand); 16 keys per step:
+        // P +8 packed columns, V +16 rows = 1024 bytes
+        ptx::tc_fence_after();
+        const uint32_t idesc = ptx::make_idesc_bf16(BM, D, false, true);
+        const uint64_t vd = desc_sw64(ptx::smem_u32(slot_base) + KBT);
+        const uint32_t od = tmem_base + h * 128 + 64, pa = tmem_base + h * 128;
+        ptx::tc_mma_bf16_ta(od, pa, vd, idesc, 0u);
+#pragma unroll
+        for (int ks = 1; ks < 8; ++ks) ptx::tc_mma_bf16_ta(od, pa + 8 * ks, vd + ks * (1024 >> 4), idesc, 1u);
+        ptx::tc_commit(&o_full[h]);
+        FDBG(it * 16 + 4);
+      }
+      // -- O row: normalise, bf16 pairs, back into tensor memory as the projection's A operand --
+      ok = ptx::mbar_wait(&o_full[h], ul & 1, abort_flag, g.status);
+      if (elected) FDBG(it * 16 + 5);
+      if (ok) {
+        ptx::tc_fence_after();
+        uint32_t rv[32], ob[16];
+        const f32x2 inv2 = ptx::pack2(inv, inv);
+        ptx::tmem_ld32(tb + 64, rv);
+        ptx::tmem_ld_wait();
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+          float v0, v1;
+          ptx::unpack2(ptx::mul2(ptx::pack2(__uint_as_float(rv[2 * e]), __uint_as_float(rv[2 * e + 1])), inv2), v0, v1);
+          ob[e] = float2_to_bf16x2(v0, v1);
+        }
+        ptx::tmem_st16(tb + 96, ob);
+        ptx::tmem_st_wait();
+        ptx::tc_fence_before();
+      }
+      if (group_sync()) break;
+      if (elected) {
+        // Y (+)= Ob_h Wp[:, 32 h : 32 h + 32]^T; the last head of a unit hands Y to the epilogue.  The heads of a unit are
+        // issued by the threads of both groups, so each waits for its predecessor's product (accumulation order); the first
+        // head overwrites Y: the epilogue of the previous unit must have read it.
+        if (it > 0) ok = ptx::mbar_wait(pj_done, (it - 1) & 1, abort_flag, g.status);
+        if (h == 0) ok = ok && ptx::mbar_wait(y_empty, (ul & 1) ^ 1, abort_flag, g.status);
+        if (ok) {
+          ptx::tc_fence_after();
+          const uint32_t idesc = ptx::make_idesc_bf16(BM, C, false, false);
+          const uint32_t a = tmem_base + h * 128 + 96;
+          const uint64_t bd = desc_sw64(ptx::smem_u32(sWp) + h * WP_TILE);
+          ptx::tc_mma_bf16_ta(tmem_base + TM_Y, a, bd, idesc, h ? 1u : 0u);
+          ptx::tc_mma_bf16_ta(tmem_base + TM_Y, a + 8, bd + 2, idesc, 1u);
+          ptx::tc_commit(pj_done);
+          if (h == NH - 1) ptx::tc_commit(y_full);
+          FDBG(it * 16 + 6);
+          // the same head of the next unit: its accumulator replaces P and O (read by now); Ob, which the product above is
+          // still reading, lies beside it
+          if (it + NH < total) issue_qkv(it + NH);
+        }
+      }
+    }
+  } else {
+    // ---- row statistics of the units ahead, and the Y epilogue: y_row = Y + b_proj + x_row in place over the raw row, then the
+    // rows go out the way they came in (one TMA box per k-block for a window off the seam, a scatter through the map for a seam
+    // window).  One row per thread; whichever of the two jobs has its input ready is taken next. -----------------------------
+    const int q = warp & 3;
+    const int r = q * 32 + lane;
+    const int w = r >> 6, i = r & 63;
+    const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
+    bool ok = true;
+    auto row_ptr = [&](int ab, int row, int ch) { return sA + ab * A_BYTES + (ch >> 2) * KBT + sw64_off(row, ch & 3); };
+    int n_box = 0;                                     // box epilogues of this warp's window so far (phase of ysync[w])
+    auto statistics = [&](int ul) {
+      const int ab = ul % na;
+      if (q == 0 && lane == 0) FDBG(4096 + ul * 8 + 3);
+      if (i < T) {
+        float rstd = 0.f;
+        uint4 k0 = make_uint4(0, 0, 0, 0), k1 = k0;
+        if (rowoff_s[ab * BM + r] != ROW_INVALID) {
+          uint4 xr[NCH];
+#pragma unroll
+          for (int ch = 0; ch < NCH; ++ch) xr[ch] = *reinterpret_cast<const uint4*>(row_ptr(ab, r, ch));
+          f32x2 s2[2] = {0ull, 0ull};
+#pragma unroll
+          for (int ch = 0; ch < NCH; ++ch) {
+            const uint32_t x4[4] = {xr[ch].x, xr[ch].y, xr[ch].z, xr[ch].w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+              s2[e & 1] = ptx::add2(s2[e & 1], ptx::pack2(__uint_as_float(x4[e] << 16), __uint_as_float(x4[e] & 0xFFFF0000u)));
+          }
+          float a0, a1, a2, a3;
+          ptx::unpack2(s2[0], a0, a1);
+          ptx::unpack2(s2[1], a2, a3);
+          const float mean = ((a0 + a1) + (a2 + a3)) * (1.0f / (float)C);
+          const f32x2 nm2 = ptx::pack2(-mean, -mean);
+          f32x2 q2[2] = {0ull, 0ull};
+#pragma unroll
+          for (int ch = 0; ch < NCH; ++ch) {
+            const uint32_t x4[4] = {xr[ch].x, xr[ch].y, xr[ch].z, xr[ch].w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const f32x2 d2 = ptx::add2(ptx::pack2(__uint_as_float(x4[e] << 16), __uint_as_float(x4[e] & 0xFFFF0000u)), nm2);
+              q2[e & 1] = ptx::fma2(d2, d2, q2[e & 1]);
+            }
+          }
+          ptx::unpack2(q2[0], a0, a1);
+          ptx::unpack2(q2[1], a2, a3);
+          const float var = ((a0 + a1) + (a2 + a3)) * (1.0f / (float)C) + g.eps;
+          rstd = rsqrtf(var);
+          extra_row(-mean, var * rstd, k0, k1);          // sigma = var / sqrt(var)
+        }
+        rstd_s[ab * BM + r] = rstd;
+        *reinterpret_cast<uint4*>(sAx + ab * AX_BYTES + plain_off(r, 0)) = k0;
+        *reinterpret_cast<uint4*>(sAx + ab * AX_BYTES + plain_off(r, 1)) = k1;
+      }
+      ptx::fence_proxy_async();                        // the extra k-step -> visible to the MMAs
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&a_full[ab]);
+      if (q == 0 && lane == 0) FDBG(4096 + ul * 8 + 4);
+    };
+    auto y_epilogue = [&](int ul) {
+      const int ab = ul % na;
+      if (q == 0 && lane == 0) FDBG(4096 + ul * 8 + 5);
+      ptx::tc_fence_after();
+      const uint32_t my_off = rowoff_s[ab * BM + r];
+      const bool valid = i < T && my_off != ROW_INVALID;
+#pragma unroll
+      for (int k = 0; k < NH; ++k) {                   // 32 columns = 4 chunks of the row at a time
+        uint32_t rv[32];
+        ptx::tmem_ld32(tmem_base + TM_Y + lane_addr + k * 32, rv);
+        uint4 xv[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) xv[c] = valid ? *reinterpret_cast<const uint4*>(row_ptr(ab, r, k * 4 + c)) : make_uint4(0, 0, 0, 0);
+        ptx::tmem_ld_wait();
+        if (k == NH - 1) {                             // Y is in registers: the next unit's projection may overwrite it
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(y_empty);
+        }
+        if (valid) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const uint32_t x4[4] = {xv[c].x, xv[c].y, xv[c].z, xv[c].w};
+            const float4 b0 = *reinterpret_cast<const float4*>(bp_s + k * 32 + c * 8);
+            const float4 b1 = *reinterpret_cast<const float4*>(bp_s + k * 32 + c * 8 + 4);
+            const f32x2 bb[4] = {ptx::pack2(b0.x, b0.y), ptx::pack2(b0.z, b0.w), ptx::pack2(b1.x, b1.y), ptx::pack2(b1.z, b1.w)};
+            uint32_t o4[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const int col = c * 8 + 2 * e;
+              float v0, v1;
+              ptx::unpack2(ptx::add2(ptx::add2(ptx::pack2(__uint_as_float(rv[col]), __uint_as_float(rv[col + 1])), bb[e]),
+                                     ptx::pack2(__uint_as_float(x4[e] << 16), __uint_as_float(x4[e] & 0xFFFF0000u))), v0, v1);
+              o4[e] = float2_to_bf16x2(v0, v1);
+            }
+            *reinterpret_cast<uint4*>(row_ptr(ab, r, k * 4 + c)) = make_uint4(o4[0], o4[1], o4[2], o4[3]);
+          }
+        }
+      }
+      const int4 wb = wbox_s[ab * 2 + w];
+      if (wb.x == WIN_BOX) {
+        // the window's rows belong to two warps: both hand them over, the first one's lane 0 stores the window
+        ptx::fence_proxy_async();                      // the rows written above -> visible to the TMA stores
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&ysync[w]);
+        if ((q & 1) == 0 && lane == 0 && ptx::mbar_wait(&ysync[w], n_box & 1, abort_flag, g.status)) {
+#pragma unroll
+          for (int kb = 0; kb < NH; ++kb)
+            ptx::tma_store_4d(&tmY, sA + ab * A_BYTES + kb * KBT + w * (64 * 64), kb * D, wb.y, wb.z, wb.w);
+          ptx::bulk_commit_group();
+          ptx::bulk_wait_group_read<0>();              // the stores have read the slot: it may be refilled
+        }
+        ++n_box;
+      } else {
+        __syncwarp();
+        if (wb.x == WIN_GATHER) {
+          uint4 yv[NCH];
+          uint32_t ro[NCH];
+#pragma unroll
+          for (int k = 0; k < NCH; ++k) {               // the warp's 32 rows x NCH chunks: a row by consecutive lanes
+            const int idx = k * 32 + lane;
+            const int rr = idx / NCH, ch = idx - rr * NCH, row = q * 32 + rr;
+            ro[k] = (row & 63) < T ? rowoff_s[ab * BM + row] : ROW_INVALID;
+            yv[k] = *reinterpret_cast<const uint4*>(row_ptr(ab, row, ch));
+          }
+#pragma unroll
+          for (int k = 0; k < NCH; ++k) {
+            const int idx = k * 32 + lane;
+            const int ch = idx - (idx / NCH) * NCH;
+            if (ro[k] != ROW_INVALID) *reinterpret_cast<uint4*>(g.y + ((size_t)ro[k] << 3) + ch * 8) = yv[k];
+          }
+        }
+      }
+      __syncwarp();                                     // the warp's rows are read: the ring slot may be refilled
+      if (lane == 0) ptx::mbar_arrive(&a_free[ab]);
+      if (q == 0 && lane == 0) FDBG(4096 + ul * 8 + 6);
+    };
+    int sdone = 0, edone = 0;                          // units whose statistics / whose epilogue this warp has done
+    uint32_t idle = 0;
+    unsigned long long t_idle = 0;
+    while (edone < U) {
+      int job = 0;                                     // lane 0 looks, the warp follows
+      if (lane == 0) {
+        if (sdone < U && sdone - edone < na && ptx::mbar_test(&landed[sdone % na], (sdone / na) & 1)) job = 1;
+        else if (edone < sdone && ptx::mbar_test(y_full, edone & 1)) job = 2;
+        else if ((++idle & 63u) == 0) {
+          const unsigned long long now = ptx::globaltimer();
+          if (idle == 64u) t_idle = now;
+          else if (*(volatile int*)abort_flag || now - t_idle > ptx::kWaitLimitNs) {
+            *abort_flag = 1;
+            atomicExch(g.status, (int)SMARTMEM_ERR_TIMEOUT);
+            job = 3;
+          }
+        }
+      }
+      job = __shfl_sync(0xFFFFFFFFu, job, 0);
+      if (job == 1) { statistics(sdone); ++sdone; idle = 0; }
+      else if (job == 2) { y_epilogue(edone); ++edone; idle = 0; }
+      else if (job == 3) break;
+      else __nanosleep(32);
+    }
+    ptx::bulk_wait_group<0>();                         // this thread's TMA stores are complete
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (tid == 0) FDBG(8003);
+  if (warp == 0) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+}  // namespace
+
+bool swin_attn_fused_supported(int dtype, int C, int heads, int window) {
+  return dtype == SMARTMEM_BF16 && (heads == 2 || heads == 3) && C == heads * D && window * window <= TP && window >= 1;
+}
+
+int launch_swin_attn_fused(const smartmem_swin_params_t& p, const DevMap& rowmap, const void* x, void* y, cudaStream_t st) {
+  if (!swin_attn_fused_supported(p.dtype, p.C, p.heads, p.window)) return SMARTMEM_ERR_UNSUPPORTED;
+  const int NH = p.heads, C = p.C, T = p.window * p.window;
+  const long long n_windows = (long long)p.B * (p.H / p.window) * (p.W / p.window);
+  if (n_windows < 1 || n_windows * T >= (1ll << 31) || (long long)p.B * p.H * p.W * C >= (1ll << 34)) return SMARTMEM_ERR_UNSUPPORTED;
+  const void* ptrs[] = {x, y, p.ln1_g, p.ln1_b, p.w_qkv, p.b_qkv, p.w_proj, p.b_proj};
+  for (const void* q : ptrs)
+    if (!q || ((uintptr_t)q & 15)) return SMARTMEM_ERR_ALIGNMENT;
+  if (!p.rel_bias_table) return SMARTMEM_ERR_INVALID_ARG;
+  CUtensorMap twq, twp;
+  int rc;
+  if ((rc = tc_encode_2d_sw64(p.w_qkv, C, 3 * C, C, D, D, &twq)) != SMARTMEM_OK) return rc;
+  if ((rc = tc_encode_2d_sw64(p.w_proj, C, C, C, D, C, &twp)) != SMARTMEM_OK) return rc;
+  CUtensorMap tx, ty;
+  memset(&tx, 0, sizeof(tx));
+  memset(&ty, 0, sizeof(ty));
+  const long long dims[4] = {C, p.W, p.H, p.B}, strides[3] = {C, (long long)p.W * C, (long long)p.H * p.W * C};
+  const int box[4] = {D, p.window, p.window, 1};
+  const bool use_box = tc_encode_nd_sw64(x, 4, dims, strides, box, &tx) == SMARTMEM_OK &&
+                       tc_encode_nd_sw64(y, 4, dims, strides, box, &ty) == SMARTMEM_OK;
+  FusedArgs g;
+  memset(&g, 0, sizeof(g));
+  g.use_box = use_box ? 1 : 0;
+  g.n_windows = (int)n_windows;
+  g.n_pairs = (int)((n_windows + 1) / 2);
+  g.T = T; g.ws = p.window; g.shift = p.shift;
+  g.nWw = p.W / p.window; g.nWh = p.H / p.window; g.win_per_img = g.nWw * g.nWh;
+  g.fd_wpi = make_fastdiv((uint32_t)g.win_per_img);
+  g.fd_nww = make_fastdiv((uint32_t)g.nWw);
+  g.eps = p.ln_eps;
+  g.scale = 1.0f / sqrtf((float)D);
+  g.x = (const __nv_bfloat16*)x; g.y = (__nv_bfloat16*)y;
+  g.ln_g = (const __nv_bfloat16*)p.ln1_g; g.ln_b = (const __nv_bfloat16*)p.ln1_b;
+  g.b_qkv = (const __nv_bfloat16*)p.b_qkv; g.b_proj = (const __nv_bfloat16*)p.b_proj;
+  g.table = (const __nv_bfloat16*)p.rel_bias_table;
+  g.rowmap = rowmap;
+  g.split = devmap_split(rowmap, T);
+  g.status = device_status_ptr();
+  if (!g.status) return SMARTMEM_ERR_CUDA;
+  const bool kc56 = T <= 56;
+  const int br = kc56 ? 28 : 36;
+  auto need = [&](int na) {
+    return (size_t)na * NH * KBT + (size_t)NSLOT * KV_SLOT + (size_t)NH * NH * WQ_TILE + (size_t)NH * C * 64 +
+           (size_t)na * AX_BYTES + (size_t)NH * WX_TILE + (size_t)NH * T * br * 4 + (size_t)C * 4 + (size_t)na * BM * 8 +
+           (size_t)2 * C * 4 + TP * 4 + 16 + TP * 16 + 4 * 16 + 6 * 16 + N_BARS * 8 + 16;
+  };
+  const size_t kMaxSmem = 232448;
+  g.na = need(3) <= kMaxSmem ? 3 : 2;
+  if (need(g.na) > kMaxSmem) return SMARTMEM_ERR_UNSUPPORTED;
+  const size_t smem = need(g.na) + 1024 <= kMaxSmem ? need(g.na) + 1024 : kMaxSmem;   // alignment slack only while it fits
+  g.smem_bytes = (uint32_t)smem;
+  const void* fn = NH == 3 ? (kc56 ? (const void*)swin_attn_fused_kernel<3, 56> : (const void*)swin_attn_fused_kernel<3, 64>)
+                           : (kc56 ? (const void*)swin_attn_fused_kernel<2, 56> : (const void*)swin_attn_fused_kernel<2, 64>);
+  if ((rc = ensure_max_dynamic_smem(fn, (int)kMaxSmem)) != SMARTMEM_OK) return rc;
+  const int sms = tc_sm_count();
+  const unsigned grid = (unsigned)(g.n_pairs < sms ? g.n_pairs : sms);
+  profile_tick("attn_half_fused", st);
+  cudaError_t e;
+  if (NH == 3) e = kc56 ? launch_pdl(swin_attn_fused_kernel<3, 56>, dim3(grid), dim3(kThreads), smem, st, twq, twp, tx, ty, g)
+                        : launch_pdl(swin_attn_fused_kernel<3, 64>, dim3(grid), dim3(kThreads), smem, st, twq, twp, tx, ty, g);
+  else e = kc56 ? launch_pdl(swin_attn_fused_kernel<2, 56>, dim3(grid), dim3(kThreads), smem, st, twq, twp, tx, ty, g)
+                : launch_pdl(swin_attn_fused_kernel<2, 64>, dim3(grid), dim3(kThreads), smem, st, twq, twp, tx, ty, g);
+  count_launch();
+  return e == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
+}
+
+}  // namespace smartmem

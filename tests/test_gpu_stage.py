@@ -28,13 +28,13 @@ def stage_case(config_id, B, H, W, C, heads, window, images):
     descs = [sm.make_desc((B, H, W, C)), sm.make_desc((4 * C,)), sm.make_desc((4 * C,)), sm.make_desc((2 * C, 4 * C))]
     pmd = [to_dev(pm[k]) for k in ("g", "b", "w")]
     outs = {}
-    for mode in (sm.ELIMINATE, sm.EXPLICIT):
+    for mode in (sm.ELIMINATE, sm.ELIMINATE_UNFUSED, sm.EXPLICIT):
         t = to_dev(blocks[0]["x"])
         for inp, shift in zip(blocks, (0, window // 2)):
             dev = {k: to_dev(v) for k, v in inp.items() if k != "x"}
             t = run_block(inp, dev, B=B, H=H, W=W, C=C, heads=heads, window=window, shift=shift, mlp_ratio=4, dtype="bf16",
                           mode=mode, x_dev=t)
-        plan = sm.smartmem_plan(_patch_merge_ops(B, H, W, C), descs, mode)
+        plan = sm.smartmem_plan(_patch_merge_ops(B, H, W, C), descs, sm.EXPLICIT if mode == sm.EXPLICIT else sm.ELIMINATE)
         try:
             wsb = sm.smartmem_plan_workspace_bytes(plan)
             ws = torch.empty(max(wsb, 16), dtype=torch.uint8, device="cuda")
@@ -45,7 +45,8 @@ def stage_case(config_id, B, H, W, C, heads, window, images):
             sm.smartmem_plan_destroy(plan)
         assert_close_bf16(to_host_f64(out)[images], ref, f"stage, mode {mode}")
         outs[mode] = out
-    assert torch.equal(outs[sm.ELIMINATE].view(torch.int16), outs[sm.EXPLICIT].view(torch.int16))
+    # kernel by kernel, the eliminated and the explicit chain are bit-identical (ELIMINATE fuses the attention halves)
+    assert torch.equal(outs[sm.ELIMINATE_UNFUSED].view(torch.int16), outs[sm.EXPLICIT].view(torch.int16))
 
 
 def test_small_stage():

@@ -38,24 +38,28 @@ def test_noalloc_matches_workspace_entry_point_twice(dtype, cfg):
                                 cfg["mlp_ratio"], dtype)
         dev = {k: to_dev(v) for k, v in inp.items()}
         p = _params(cfg, dev, dtype)
-        for mode in (sm.ELIMINATE, sm.EXPLICIT):
+        for mode in (sm.ELIMINATE, sm.ELIMINATE_UNFUSED, sm.EXPLICIT):
             n = sm.smartmem_swin_block_workspace_bytes(p, mode)
             assert n <= sm.smartmem_swin_block_static_scratch_bytes()
             ws = torch.empty(n, dtype=torch.uint8, device="cuda")
             ref = torch.full_like(dev["x"], float("nan"))
             sm.smartmem_swin_block(p, dev["x"].data_ptr(), ref.data_ptr(), ws.data_ptr(), n, mode, stream())
             got = torch.full_like(dev["x"], float("nan"))
+            torch.cuda.synchronize()
+            free_before = torch.cuda.mem_get_info()[0]
             sm.smartmem_swin_block_noalloc(p, dev["x"].data_ptr(), got.data_ptr(), mode, stream())
             check_status()
+            if call == 1:                      # past the first call's one-time set-up: the device's free memory does not move
+                assert torch.cuda.mem_get_info()[0] == free_before
             # same kernels on the same inputs: identical bits (well inside the bf16 / fp32 tolerances)
             assert torch.isfinite(got.float()).all()
             assert torch.equal(got, ref), f"call {call} mode {mode}"
             outs.append(got)
-    assert not torch.equal(outs[0], outs[2])   # the two calls really had different inputs
+    assert not torch.equal(outs[0], outs[3])   # the two calls really had different inputs
 
 
 def test_noalloc_rejects_blocks_beyond_the_fixed_array():
-    cfg = dict(B=32, H=56, W=56, C=96, heads=3, window=7, shift=3, mlp_ratio=4)
+    cfg = dict(B=64, H=56, W=56, C=96, heads=3, window=7, shift=3, mlp_ratio=4)
     p = sm.SwinParams()
     p.dtype = sm.BF16
     for k, v in cfg.items():
