@@ -6,25 +6,26 @@
 // reverse and the reverse shift are all index arithmetic here: rows of x are gathered through the
 // composed shift o partition map straight into the MMA operand layout, q / k / v and the attention
 // output never leave the SM, and the result rows are scattered through the same map.  Per token the
-// kernel reads C and writes C elements of global memory; the three-kernel form of the same chain
-// moves 11 C.
+// kernel reads C (twice: once for the operand tile, once more -- from L2 -- for the residual) and writes C
+// elements of global memory; the three-kernel form of the same chain moves 11 C through HBM.
 //
 // Unit of work: a pair of windows = one 128-row MMA tile (window w of the pair in rows 64 w .. 64 w + T - 1,
 // the rows between T and 64 stay zero), taken round-robin by persistent CTAs that keep every weight resident.
-// An "item" is (unit, head).  Per item, all in one 128-column buffer of tensor memory (one buffer per head):
+// An "item" is (unit, head); head h is the work of row group h.  Per item, all in one 96-column buffer of tensor
+// memory (four buffers in rotation):
 //
 //   acc  = [X | e] [Wq_h; Wk_h; Wv_h | f]^T    128 x 96 x (C + 16)  tcgen05; X = the RAW rows (bf16) in shared memory
 //   q,k,v = rstd acc                           LayerNorm applied algebraically (below); q goes back to tensor memory as
 //                                              bf16 pairs, k and v to shared memory in operand layout
-//   S    = q k^T                               128 x 128 x 32, q read from tensor memory (the two diagonal 64 x 64 blocks are used)
+//   S    = [q0 0; 0 q1] [k0 | k1]^T            128 x 64 x 64: the two windows' keys are stacked along the reduction
+//                                              dimension and each query row carries zeros in the other window's half,
+//                                              so a row's 64 scores are its own window's; q is read from tensor memory
 //   P    = softmax(scale S + bias + mask)      one query row per thread (= its TMEM lane); P stored as bf16 pairs
-//                                              over the S columns it came from
-//   O    = P [v0; v1]                          128 x 32 x 128, P read from tensor memory, block diagonal
+//   O    = [P0 0; 0 P1] [v0; v1]               128 x 32 x 128, P read from tensor memory, V as it lies (MN-major)
 //   Ob   = bf16(O / rowsum)                    back into tensor memory as packed pairs
 //   Y   += Ob Wp[:, 32 h : 32 h + 32]^T        128 x C x 32: the head merge is the accumulation over heads
 //
-// and per unit  y_row = Y + b_proj + x_row, written in place over the raw row in shared memory (the A tile doubles as the
-// residual) and stored with 16-byte vectors, a row's C elements by consecutive lanes.
+// and per unit  y_row = Y + b_proj + x_row, stored with 16-byte vectors at the row's offset under the map.
 //
 // LayerNorm without a normalised tile:  LN(x) W^T + b = rstd (x W'^T - mean c + sigma b'),  W' = bf16(gamma . W) (column
 // scaling), c_n = sum_k W'_nk, b'_n = b_n + sum_k beta_k W_nk, sigma = 1 / rstd.  c is summed from the ROUNDED W', so the
@@ -32,13 +33,14 @@
 // rank-one terms ride on the tensor core as one extra k-step: row r of the operand carries (-mean_r, sigma_r), column n of the
 // weights (c_n, b'_n), each fp32 value split into three bf16 pieces (the six largest cross products of the pieces are kept:
 // exact to 2^-24), so the epilogue of the QKV product is one multiply per element.  Every CTA folds gamma into its resident
-// copy of the weights once (prologue, overlapped with the previous kernel's tail); the row statistics (two passes over the
-// row in registers, fp32) are taken by the warps that gather the rows.
+// copy of the weights once (prologue); the row statistics are two passes over the row in registers, fp32.
 //
-// Warp roles (16 warps): 0-3 gather the rows of the units ahead (16-byte asynchronous copies through the index map), 4-7 and
-// 8-11 two row groups that alternate over the items (q/k/v epilogue, softmax, O epilogue) -- each group issues its own MMAs
-// from one elected thread right after the group's barrier, so a hand-off costs a barrier and not a trip through another
-// warp --, 12-15 row statistics of the units ahead, Y epilogue and row scatter.  Every wait is bounded.
+// Warp roles (8 + 4 heads warps): 0-3 bring in the rows of the units ahead -- a window that does not straddle the seam of the
+// shifted image is an affine box [32 channels, ws, ws] of x per k-block, one TMA copy each; a seam window is gathered row by
+// row with 16-byte asynchronous copies through the index map --; then one group of four warps per head (q/k/v epilogue,
+// softmax, O epilogue: one row of the pair tile per thread; each group issues its own MMAs from one elected thread right
+// after the group's barrier, so a hand-off costs a barrier and not a trip through another warp); the last four warps take
+// the row statistics of the units ahead and run the Y epilogue.  Every wait is bounded.
 #include "attn.cuh"
 #include "gemm_tc.cuh"
 #include "ptx.cuh"
@@ -66,16 +68,17 @@ constexpr int WROWS = 96;                           // rows of a per-head QKV we
 constexpr int WQ_TILE = WROWS * 64;
 constexpr int WX_TILE = WROWS * 32;                 // the extra k-step of a head's weights
 constexpr int KV_SLOT = 2 * KBT;                    // k, v tiles of one item
-constexpr int NSLOT = 2;
-constexpr int kLoaderThreads = 128, kThreads = 512;
+constexpr int NBUF = 4, BUF_COLS = 96;              // item buffers of tensor memory
+constexpr int NRING = 8;                            // units whose row offsets are kept (a unit's epilogue runs long after its gather)
+constexpr int kLoaderThreads = 128;
 constexpr uint32_t TMEM_COLS = 512;
-constexpr uint32_t TM_Y = 384, TM_Q = 480;          // after three 128-column item buffers: Y (C columns), two q slots of 16
-constexpr uint32_t ROW_INVALID = 0xFFFFFFFFu, ROW_BOX = 0xFFFFFFFEu;   // no such row / a row of a window moved as a TMA box
+constexpr uint32_t TM_Y = NBUF * BUF_COLS;          // the projection's accumulator (C columns) after the item buffers
+constexpr uint32_t ROW_INVALID = 0xFFFFFFFFu;       // no such row (a padding row of the tile, or a window past the end)
 constexpr int WIN_MISSING = 0, WIN_GATHER = 1, WIN_BOX = 2;
-constexpr int N_BARS = 24;
+constexpr int N_BARS = 26;
 
 struct FusedArgs {
-  int n_windows, n_pairs, T, ws, shift;
+  int n_windows, n_pairs, T, ws, shift, H, W;
   int nWw, nWh, win_per_img;
   FastDiv fd_wpi, fd_nww;
   int na;                                           // depth of the row ring (2 or 3)
@@ -84,7 +87,7 @@ struct FusedArgs {
   const __nv_bfloat16 *x, *ln_g, *ln_b, *b_qkv, *b_proj, *table;
   __nv_bfloat16* y;
   int* status;
-  int use_box;                                      // windows off the seam move as TMA boxes (tensor maps over x and y are valid)
+  int use_box;                                      // windows off the seam move as TMA boxes (the tensor map over x is valid)
   int split;                                        // first atom of rowmap that indexes the token inside its window (-1: evaluate every row in full)
   DevMap rowmap;                                    // row n T + i of the windowed view -> element offset of the token in x (and y)
 };
@@ -142,11 +145,11 @@ __device__ __forceinline__ void extra_col(float c, float b, uint4& k0, uint4& k1
 }
 
 template <int NH, int KC>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(32 * (9 + 4 * NH), 1)
 swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_constant__ CUtensorMap tmWp,
-                       const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmY,
-                       const __grid_constant__ FusedArgs g) {
+                       const __grid_constant__ CUtensorMap tmX, const __grid_constant__ FusedArgs g) {
   constexpr int C = NH * D, NCH = C / 8;             // channels, 16-byte chunks per row
+  constexpr int kThreads = 32 * (9 + 4 * NH);
   constexpr int A_BYTES = NH * KBT;                  // a unit's raw rows: NH k-blocks of 32 columns
   constexpr int WP_TILE = C * 64;                    // Wp[:, 32 h : 32 h + 32]: C rows x 64 bytes
   constexpr int BR = KC == 56 ? 28 : 36;             // 32-bit words per bias row (16-byte reads of 8 consecutive rows hit distinct banks)
@@ -155,27 +158,28 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
   uint8_t* smem = smem_raw + pad;
   const int T = g.T, ws = g.ws, na = g.na;
   uint8_t* sA = smem;                                              // [na][NH k-blocks][8 KB]
-  uint8_t* sKV = sA + na * A_BYTES;                                // [2 slots][k, v][8 KB]
-  uint8_t* sWq = sKV + NSLOT * KV_SLOT;                            // [NH heads][NH k-blocks][96 rows x 64 B]
+  uint8_t* sKV = sA + na * A_BYTES;                                // [NH groups][k, v][8 KB]
+  uint8_t* sWq = sKV + NH * KV_SLOT;                               // [NH heads][NH k-blocks][96 rows x 64 B]
   uint8_t* sWp = sWq + NH * NH * WQ_TILE;                          // [NH heads][C rows x 64 B]
   uint8_t* sAx = sWp + NH * WP_TILE;                               // [na][128 rows x 32 B]
   uint8_t* sWx = sAx + na * AX_BYTES;                              // [NH heads][96 rows x 32 B]
   uint32_t* bias_s = reinterpret_cast<uint32_t*>(sWx + NH * WX_TILE);   // [NH][T][BR]: bf16 pairs
   float* bp_s = reinterpret_cast<float*>(bias_s + NH * T * BR);    // [C]
   float* rstd_s = bp_s + C;                                        // [na][128]
-  uint32_t* rowoff_s = reinterpret_cast<uint32_t*>(rstd_s + na * BM);   // [na][128]: row offset in 16-byte units
-  float* ln_s = reinterpret_cast<float*>(rowoff_s + na * BM);      // [2][C]: gamma, beta
+  uint32_t* rowoff_s = reinterpret_cast<uint32_t*>(rstd_s + na * BM);   // [NRING][128]: row offset in 16-byte units
+  float* ln_s = reinterpret_cast<float*>(rowoff_s + NRING * BM);   // [2][C]: gamma, beta
   int* tyx_s = reinterpret_cast<int*>(ln_s + 2 * C);               // [64]: ty << 8 | tx
   uint32_t* kmask_s = reinterpret_cast<uint32_t*>(tyx_s + TP);     // [4]
   int4* tok_s = reinterpret_cast<int4*>(kmask_s + 4);              // [64]: the map's contribution of token t: (offset, u0, u1, -)
   int4* win_s = tok_s + TP;                                        // [2 units][2 windows]: the contribution of window n: (offset lo, hi, u0, u1)
-  int4* wbox_s = win_s + 4;                                        // [na][2 windows]: (kind, first column, first row, image) of the window
-  uint64_t* bars = reinterpret_cast<uint64_t*>(wbox_s + 6);
+  int* wkind_s = reinterpret_cast<int*>(win_s + 4);                // [na][2 windows] (+ pad): how the window's rows come in
+  uint64_t* bars = reinterpret_cast<uint64_t*>(wkind_s + 8);
   uint64_t* w_full = bars;
-  uint64_t *a_full = bars + 1, *a_free = a_full + 3, *landed = a_free + 3;     // [3] each
-  uint64_t *acc_full = landed + 3, *s_full = acc_full + 3, *o_full = s_full + 3;
-  uint64_t *y_full = o_full + 3, *y_empty = y_full + 1, *pj_done = y_empty + 1, *ysync = pj_done + 1;   // ysync [2]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ysync + 2);
+  uint64_t *a_full = bars + 1, *a_free = a_full + 3, *landed = a_free + 3;     // [3] each: per slot of the row ring
+  uint64_t *s_full = landed + 3, *o_full = s_full + 3;             // [3] each: per group (the group issues these products itself)
+  uint64_t *acc_full = o_full + 3, *ob_full = acc_full + NBUF;     // [NBUF] each: per item buffer (items 4 apart share one)
+  uint64_t *y_full = ob_full + NBUF, *y_empty = y_full + 1;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(y_empty + 1);
   int* abort_flag = reinterpret_cast<int*>(tmem_slot + 1);
   uint16_t* raw_s = reinterpret_cast<uint16_t*>(sKV);              // prologue scratch: the raw table columns, [NH][256]
 
@@ -195,17 +199,17 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
     ptx::mbar_init(w_full, 1);
     for (int i = 0; i < 3; ++i) {
       ptx::mbar_init(&a_full[i], 4);
-      ptx::mbar_init(&a_free[i], 4);
+      ptx::mbar_init(&a_free[i], NH);
       ptx::mbar_init(&landed[i], 4);
-      ptx::mbar_init(&acc_full[i], 1);
       ptx::mbar_init(&s_full[i], 1);
       ptx::mbar_init(&o_full[i], 1);
     }
+    for (int i = 0; i < NBUF; ++i) {
+      ptx::mbar_init(&acc_full[i], 1);
+      ptx::mbar_init(&ob_full[i], 4);
+    }
     ptx::mbar_init(y_full, 1);
     ptx::mbar_init(y_empty, 4);
-    ptx::mbar_init(pj_done, 1);
-    ptx::mbar_init(&ysync[0], 2);
-    ptx::mbar_init(&ysync[1], 2);
     *abort_flag = 0;
     ptx::fence_barrier_init();
     ptx::fence_proxy_async();
@@ -213,7 +217,6 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
     ptx::prefetch_tensormap(&tmWq);
     ptx::prefetch_tensormap(&tmWp);
     ptx::prefetch_tensormap(&tmX);
-    ptx::prefetch_tensormap(&tmY);
     ptx::mbar_expect_tx(w_full, (uint32_t)(NH * NH * WQ_TILE + NH * WP_TILE));
     for (int h = 0; h < NH; ++h) {
       for (int kb = 0; kb < NH; ++kb)
@@ -245,10 +248,8 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
   }
   for (int i = tid; i < na * A_BYTES / 16; i += kThreads) reinterpret_cast<uint4*>(sA)[i] = make_uint4(0, 0, 0, 0);
   for (int i = tid; i < na * AX_BYTES / 16; i += kThreads) reinterpret_cast<uint4*>(sAx)[i] = make_uint4(0, 0, 0, 0);
-  for (int i = tid; i < na * BM; i += kThreads) {
-    rstd_s[i] = 0.f;
-    rowoff_s[i] = ROW_INVALID;
-  }
+  for (int i = tid; i < na * BM; i += kThreads) rstd_s[i] = 0.f;
+  for (int i = tid; i < NRING * BM; i += kThreads) rowoff_s[i] = ROW_INVALID;
   __syncthreads();
   // each head's bias as a [T, T] table of bf16 pairs, -inf for the padded keys
   for (int i = tid; i < NH * T * (KC / 2); i += kThreads) {
@@ -319,9 +320,9 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
   if (tid == 0) FDBG(8002);
 
   if (warp < 4) {
-    // ---- gather: rows of the units ahead through the index map, as 16-byte asynchronous copies into the operand layout ----
+    // ---- rows of the units ahead -> the operand layout in shared memory ------------------------------------------------------
     const int lt = tid;                                // 0 .. 127
-    constexpr int RPI = kLoaderThreads / NCH;          // rows per round of the copy loop: a row by NCH consecutive threads
+    constexpr int RPI = kLoaderThreads / NCH;          // rows per round of the gather loop: a row by NCH consecutive threads
     const int my_ch = lt % NCH, my_slot = lt / NCH;
     bool ok = true;
     auto vote = [&](bool pred, bool all) {             // OR (all = false) or AND (all = true) over the loader threads; also a barrier
@@ -345,8 +346,6 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
         win_s[(ul & 1) * 2 + lt] = wp;
       }
     };
-    // A window that does not straddle the seam of the shifted image is an affine box [32 channels, ws, ws] of x per k-block: one
-    // TMA copy lands it in the operand layout.  A seam window is gathered row by row through the map.
     auto issue_loads = [&](int ul) {
       const int ab = ul % na;
       const int p = cidx + ul * cstride;
@@ -362,8 +361,7 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
           kind = (seam || !g.use_box) ? WIN_GATHER : WIN_BOX;
         }
         uint32_t off16 = ROW_INVALID;
-        if (i < T && kind == WIN_BOX) off16 = ROW_BOX;
-        if (i < T && kind == WIN_GATHER) {
+        if (i < T && kind != WIN_MISSING) {            // the offset under the map: the gather of a seam window, the residual and the scatter use it
           long long off;
           if (g.split >= 0) {
             const int4 wp = win_s[(ul & 1) * 2 + w], tk = tok_s[i];
@@ -374,11 +372,11 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
           }
           off16 = (uint32_t)(off >> 3);
         }
-        rowoff_s[ab * BM + lt] = off16;
+        rowoff_s[(ul % NRING) * BM + lt] = off16;
         if (i == 0) {
-          wbox_s[ab * 2 + w] = make_int4(kind, wx * ws + g.shift, wy * ws + g.shift, b);
-          if (kind == WIN_BOX) {                        // this thread moves the window
-            ptx::mbar_add_tx(&landed[ab], (uint32_t)(T * C * 2));     // (no arrival: the loader warps arrive when their copies have landed)
+          wkind_s[ab * 2 + w] = kind;
+          if (kind == WIN_BOX) {                        // this thread moves the window (no arrival: the loader warps arrive below)
+            ptx::mbar_add_tx(&landed[ab], (uint32_t)(T * C * 2));
 #pragma unroll
             for (int kb = 0; kb < NH; ++kb)
               ptx::tma_load_4d(sA + ab * A_BYTES + kb * KBT + w * (64 * 64), &tmX, &landed[ab], kb * D, wx * ws + g.shift,
@@ -387,19 +385,23 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
         }
       }
       asm volatile("bar.sync 2, 128;" ::: "memory");
-      uint8_t* tile = sA + ab * A_BYTES + (my_ch >> 2) * KBT;
-      for (int v = my_slot; v < 2 * T && my_slot < RPI; v += RPI) {
-        const int w = v >= T ? 1 : 0, row = w * 64 + (v - w * T);
-        const uint32_t o = rowoff_s[ab * BM + row];
-        uint8_t* dst = tile + sw64_off(row, my_ch & 3);
-        if (o == ROW_INVALID) *reinterpret_cast<uint4*>(dst) = make_uint4(0, 0, 0, 0);    // a missing window: no stale rows
-        else if (o != ROW_BOX) ptx::cp_async16(dst, g.x + ((size_t)o << 3) + my_ch * 8);
+      const int kind0 = wkind_s[ab * 2], kind1 = wkind_s[ab * 2 + 1];
+      if (kind0 != WIN_BOX || kind1 != WIN_BOX) {
+        uint8_t* tile = sA + ab * A_BYTES + (my_ch >> 2) * KBT;
+        for (int v = my_slot; v < 2 * T && my_slot < RPI; v += RPI) {
+          const int w = v >= T ? 1 : 0, row = w * 64 + (v - w * T);
+          const int kind = w ? kind1 : kind0;
+          uint8_t* dst = tile + sw64_off(row, my_ch & 3);
+          if (kind == WIN_MISSING) *reinterpret_cast<uint4*>(dst) = make_uint4(0, 0, 0, 0);    // no stale rows
+          else if (kind == WIN_GATHER)
+            ptx::cp_async16(dst, g.x + ((size_t)rowoff_s[(ul % NRING) * BM + row] << 3) + my_ch * 8);
+        }
       }
       ptx::cp_async_commit();
       window_part(ul + 1);                             // read after the next barrier of the loader threads
     };
-    // A unit's gather is issued as soon as its ring slot is free (the epilogue of unit ul - na has scattered its rows); when no
-    // slot is free the oldest gather in flight is waited for and handed on.
+    // A unit's rows are requested as soon as its ring slot is free (the QKV products of the unit that held it are done); when
+    // no slot is free the oldest request in flight is waited for and handed to the statistics warps.
     window_part(0);
     asm volatile("bar.sync 2, 128;" ::: "memory");
     int issued = 0, done = 0;
@@ -433,11 +435,11 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
       if (lt == 0) FDBG(4096 + done * 8 + 2);
       ++done;
     }
-  } else if (warp < 12) {
-    // ---- row groups: group gi takes the items it = gi (mod 2); one row of the pair tile per thread.  The group's elected thread
-    // issues the item's S, P V and projection products, and the QKV product of the SAME head of the next unit (whose accumulator
-    // takes over the tensor-memory buffer this item leaves), each right after the group barrier that completes its inputs. ------
-    const int gi = (warp - 4) >> 2;
+  } else if (warp < 4 + 4 * NH) {
+    // ---- row groups: group h takes head h of every unit; one row of the pair tile per thread.  The group's elected thread issues
+    // the item's S, P V and projection products, and the QKV product of its NEXT item as soon as the tensor-memory buffer that
+    // item rotates into is free (the projection of the item before this one has completed). ------------------------------------
+    const int gi = (warp - 4) >> 2;                    // group = head
     const int q = warp & 3;                            // TMEM lane quadrant
     const int r = q * 32 + lane;
     const int w = r >> 6, i = r & 63;                  // window of the pair, token
@@ -447,6 +449,7 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
     const uint32_t ky_lo = kmask_s[0], ky_hi = kmask_s[1], kx_lo = kmask_s[2], kx_hi = kmask_s[3];
     const uint32_t my_fy = my_ty >= ws - g.shift ? 0xFFFFFFFFu : 0u, my_fx = my_tx >= ws - g.shift ? 0xFFFFFFFFu : 0u;
     uint8_t* slot_base = sKV + gi * KV_SLOT;
+    const uint32_t* brow = bias_s + (gi * T + (i < T ? i : 0)) * BR;
     const f32x2 scale2 = ptx::pack2(g.scale, g.scale), log2e2 = ptx::pack2(LOG2E, LOG2E);
     bool ok = true;
     auto group_sync = [&]() {                          // barrier of the group's 128 threads; true if one of them gave up waiting
@@ -461,72 +464,71 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
           : "memory");
       return gave_up != 0;
     };
-    // acc[h] = [X | e] [Wq_h; Wk_h; Wv_h | f]^T of item `it` (elected thread)
-    auto issue_qkv = [&](int it) {
-      const int ul = it / NH, h = it - ul * NH, ab = ul % na;
-      ok = ok && ptx::mbar_wait(&a_full[ab], (ul / na) & 1, abort_flag, g.status);
-      if (!ok) return;
-      ptx::tc_fence_after();
-      const uint32_t idesc = ptx::make_idesc_bf16(BM, WROWS, false, false);
-      const uint32_t d = tmem_base + h * 128;
-      const uint32_t a_base = ptx::smem_u32(sA) + ab * A_BYTES, w_base = ptx::smem_u32(sWq) + h * NH * WQ_TILE;
-#pragma unroll
-      for (int kb = 0; kb < NH; ++kb) {
-        const uint64_t ad = desc_sw64(a_base + kb * KBT), bd = desc_sw64(w_base + kb * WQ_TILE);
-        ptx::tc_mma_bf16(d, ad, bd, idesc, kb ? 1u : 0u);
-        ptx::tc_mma_bf16(d, ad + 2, bd + 2, idesc, 1u);          // next 16 channels: +32 bytes
-      }
-      ptx::tc_mma_bf16(d, desc_plain(ptx::smem_u32(sAx) + ab * AX_BYTES), desc_plain(ptx::smem_u32(sWx) + h * WX_TILE), idesc, 1u);
-      ptx::tc_commit(&acc_full[h]);
-    };
-    if (elected)                                       // the first unit's items of this group; later ones follow their predecessor's epilogue
-      for (int it0 = gi; it0 < NH && it0 < total; it0 += 2) issue_qkv(it0);
-    for (int it = gi; it < total; it += 2) {
-      const int ul = it / NH, h = it - ul * NH;
+    for (int ul = 0; ul < U; ++ul) {
+      const int it = ul * NH + gi;
       const int ab = ul % na;
-      const uint32_t tb = tmem_base + h * 128 + lane_addr;
+      const uint32_t tb = tmem_base + (it & (NBUF - 1)) * BUF_COLS + lane_addr;
       // -- q, k, v of this row: rstd times the accumulator (the mean and bias terms rode on the extra k-step) --
       if (elected) FDBG(it * 16 + 0);
       ok = ok && ptx::mbar_wait(&a_full[ab], (ul / na) & 1, abort_flag, g.status) &&     // (long complete: orders the read of rstd)
-           ptx::mbar_wait(&acc_full[h], ul & 1, abort_flag, g.status);
+           ptx::mbar_wait(&acc_full[it & (NBUF - 1)], (it >> 2) & 1, abort_flag, g.status);
       if (elected) FDBG(it * 16 + 1);
       if (ok) {
+        if (elected) ptx::mbar_arrive(&a_free[ab]);      // this head's product has read the unit's rows
         ptx::tc_fence_after();
         const float rstd = rstd_s[ab * BM + r];
         const f32x2 r2 = ptx::pack2(rstd, rstd);
-        uint32_t rv[96];
-        ptx::tmem_ld32(tb, rv);
-        ptx::tmem_ld32(tb + 32, rv + 32);
-        ptx::tmem_ld32(tb + 64, rv + 64);
+        uint32_t rv[32], q16[16];
+        auto scaled_pairs = [&](uint32_t* out) {         // 32 accumulator columns in rv -> 16 bf16 pairs of rstd * acc
+#pragma unroll
+          for (int c = 0; c < 16; ++c) {
+            float v0, v1;
+            ptx::unpack2(ptx::mul2(ptx::pack2(__uint_as_float(rv[2 * c]), __uint_as_float(rv[2 * c + 1])), r2), v0, v1);
+            out[c] = float2_to_bf16x2(v0, v1);
+          }
+        };
+        ptx::tmem_ld32(tb, rv);                          // q
         ptx::tmem_ld_wait();
-        uint32_t pk[48];
+        if (elected) FDBG(it * 16 + 7);
+        scaled_pairs(q16);
 #pragma unroll
-        for (int c = 0; c < 48; ++c) {
-          float v0, v1;
-          ptx::unpack2(ptx::mul2(ptx::pack2(__uint_as_float(rv[2 * c]), __uint_as_float(rv[2 * c + 1])), r2), v0, v1);
-          pk[c] = float2_to_bf16x2(v0, v1);
-        }
-        ptx::tmem_st16(tmem_base + TM_Q + gi * 16 + lane_addr, pk);           // q: the S product's A operand
-#pragma unroll
-        for (int kv = 0; kv < 2; ++kv)
+        for (int kv = 0; kv < 2; ++kv) {                 // k, v -> this group's operand tiles
+          uint32_t o16[16];
+          ptx::tmem_ld32(tb + 32 + kv * 32, rv);
+          ptx::tmem_ld_wait();
+          scaled_pairs(o16);
 #pragma unroll
           for (int c = 0; c < 4; ++c)
             *reinterpret_cast<uint4*>(slot_base + kv * KBT + sw64_off(r, c)) =
-                make_uint4(pk[16 + kv * 16 + c * 4], pk[17 + kv * 16 + c * 4], pk[18 + kv * 16 + c * 4], pk[19 + kv * 16 + c * 4]);
+                make_uint4(o16[c * 4], o16[c * 4 + 1], o16[c * 4 + 2], o16[c * 4 + 3]);
+        }
+        // q as the S product's A operand: 64 bf16 = 32 packed columns over the accumulator's last 32 (v has been read): this
+        // window's half carries q, the other half zeros (the two windows' keys are stacked along the reduction dimension)
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+          rv[c] = w ? 0u : q16[c];
+          rv[16 + c] = w ? q16[c] : 0u;
+        }
+        if (elected) FDBG(it * 16 + 8);
+        ptx::tmem_st32(tb + 64, rv);
         ptx::tmem_st_wait();
+        if (elected) FDBG(it * 16 + 9);
         ptx::fence_proxy_async();                      // generic-proxy writes -> visible to the MMAs
         ptx::tc_fence_before();
+        if (elected) FDBG(it * 16 + 10);
       }
       if (group_sync()) break;
       if (elected) {
-        // S = q k^T into the buffer the accumulator has just left; q from its tensor-memory slot
+        // S = [q0 0; 0 q1] [k0 | k1]^T: four k16 steps, the first two over window 0's keys, the last two over window 1's
         ptx::tc_fence_after();
-        const uint32_t idesc = ptx::make_idesc_bf16(BM, 128, false, false);
-        const uint32_t qa = tmem_base + TM_Q + gi * 16;
-        const uint64_t kd = desc_sw64(ptx::smem_u32(slot_base));
-        ptx::tc_mma_bf16_ta(tmem_base + h * 128, qa, kd, idesc, 0u);
-        ptx::tc_mma_bf16_ta(tmem_base + h * 128, qa + 8, kd + 2, idesc, 1u);
-        ptx::tc_commit(&s_full[h]);
+        const uint32_t idesc = ptx::make_idesc_bf16(BM, 64, false, false);
+        const uint32_t d = tb - lane_addr, qa = d + 64;
+        const uint64_t kd0 = desc_sw64(ptx::smem_u32(slot_base)), kd1 = desc_sw64(ptx::smem_u32(slot_base) + 64 * 64);
+        ptx::tc_mma_bf16_ta(d, qa, kd0, idesc, 0u);
+        ptx::tc_mma_bf16_ta(d, qa + 8, kd0 + 2, idesc, 1u);
+        ptx::tc_mma_bf16_ta(d, qa + 16, kd1, idesc, 1u);
+        ptx::tc_mma_bf16_ta(d, qa + 24, kd1 + 2, idesc, 1u);
+        ptx::tc_commit(&s_full[gi]);
         FDBG(it * 16 + 2);
       }
       // -- seam mask of this row's window (shifted blocks: windows in the last window row or column) --
@@ -541,23 +543,22 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
         if (last_row) { diff_lo |= ky_lo ^ my_fy; diff_hi |= ky_hi ^ my_fy; }
         if (last_col) { diff_lo |= kx_lo ^ my_fx; diff_hi |= kx_hi ^ my_fx; }
       }
-      const uint32_t* brow = bias_s + (h * T + (i < T ? i : 0)) * BR;
       // -- softmax of this row over its window's keys --
-      ok = ptx::mbar_wait(&s_full[h], ul & 1, abort_flag, g.status);
+      ok = ptx::mbar_wait(&s_full[gi], ul & 1, abort_flag, g.status);
       if (elected) FDBG(it * 16 + 3);
       float inv = 0.f;
       if (ok) {
         ptx::tc_fence_after();
         uint32_t rv[KC];
-        const uint32_t ts = tb + w * 64;               // this window's 64 key columns
-        ptx::tmem_ld32(ts, rv);
+        ptx::tmem_ld32(tb, rv);
         if constexpr (KC == 64) {
-          ptx::tmem_ld32(ts + 32, rv + 32);
+          ptx::tmem_ld32(tb + 32, rv + 32);
         } else {
-          ptx::tmem_ld16(ts + 32, rv + 32);
-          ptx::tmem_ld8(ts + 48, rv + 48);
+          ptx::tmem_ld16(tb + 32, rv + 32);
+          ptx::tmem_ld8(tb + 48, rv + 48);
         }
         ptx::tmem_ld_wait();
+        if (elected) FDBG(it * 16 + 11);
         float sc[KC];
         float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
@@ -600,31 +601,33 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
         ptx::unpack2(sum2[0], s0, s1);
         ptx::unpack2(sum2[1], s2, s3);
         inv = 1.f / ((s0 + s1) + (s2 + s3));
-        // P row (bf16 pairs) over the first 64 columns of the buffer: this window's keys at packed columns
-        // 32 w .. 32 w + 31, zeros for the other window's keys (block-diagonal P)
+        if (elected && inv > 0.f) FDBG(it * 16 + 12);
+        // P row (bf16 pairs) over the score columns: this window's keys at packed columns 32 w .. 32 w + 31, zeros for the
+        // other window's keys (block-diagonal P against the stacked values)
         ptx::tmem_st32(tb + w * 32, pk);
 #pragma unroll
         for (int c = 0; c < 32; ++c) pk[c] = 0u;
         ptx::tmem_st32(tb + (1 - w) * 32, pk);
         ptx::tmem_st_wait();
         ptx::tc_fence_before();
+        if (elected) FDBG(it * 16 + 13);
       }
       if (group_sync()) break;
       if (elected) {
-        // O = P [v0; v1]: P from tensor memory (bf16 pairs), V as it lies (MN-major B operand); 16 keys per step:
-        // P +8 packed columns, V +16 rows = 1024 bytes
+        // O = P [v0; v1] over the columns q has left: P from tensor memory, V as it lies (MN-major B operand); 16 keys per
+        // step: P +8 packed columns, V +16 rows = 1024 bytes
         ptx::tc_fence_after();
         const uint32_t idesc = ptx::make_idesc_bf16(BM, D, false, true);
         const uint64_t vd = desc_sw64(ptx::smem_u32(slot_base) + KBT);
-        const uint32_t od = tmem_base + h * 128 + 64, pa = tmem_base + h * 128;
+        const uint32_t pa = tb - lane_addr, od = pa + 64;
         ptx::tc_mma_bf16_ta(od, pa, vd, idesc, 0u);
 #pragma unroll
         for (int ks = 1; ks < 8; ++ks) ptx::tc_mma_bf16_ta(od, pa + 8 * ks, vd + ks * (1024 >> 4), idesc, 1u);
-        ptx::tc_commit(&o_full[h]);
+        ptx::tc_commit(&o_full[gi]);
         FDBG(it * 16 + 4);
       }
       // -- O row: normalise, bf16 pairs, back into tensor memory as the projection's A operand --
-      ok = ptx::mbar_wait(&o_full[h], ul & 1, abort_flag, g.status);
+      ok = ptx::mbar_wait(&o_full[gi], ul & 1, abort_flag, g.status);
       if (elected) FDBG(it * 16 + 5);
       if (ok) {
         ptx::tc_fence_after();
@@ -638,51 +641,93 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
           ptx::unpack2(ptx::mul2(ptx::pack2(__uint_as_float(rv[2 * e]), __uint_as_float(rv[2 * e + 1])), inv2), v0, v1);
           ob[e] = float2_to_bf16x2(v0, v1);
         }
-        ptx::tmem_st16(tb + 96, ob);
+        ptx::tmem_st16(tb + 64, ob);
         ptx::tmem_st_wait();
         ptx::tc_fence_before();
       }
-      if (group_sync()) break;
-      if (elected) {
-        // Y (+)= Ob_h Wp[:, 32 h : 32 h + 32]^T; the last head of a unit hands Y to the epilogue.  The heads of a unit are
-        // issued by the threads of both groups, so each waits for its predecessor's product (accumulation order); the first
-        // head overwrites Y: the epilogue of the previous unit must have read it.
-        if (it > 0) ok = ptx::mbar_wait(pj_done, (it - 1) & 1, abort_flag, g.status);
-        if (h == 0) ok = ok && ptx::mbar_wait(y_empty, (ul & 1) ^ 1, abort_flag, g.status);
-        if (ok) {
+      __syncwarp();
+      if (!ok) break;
+      if (lane == 0) ptx::mbar_arrive(&ob_full[it & (NBUF - 1)]);       // the projection of this item may be issued
+      if (elected) FDBG(it * 16 + 6);
+    }
+  } else if (warp == 8 + 4 * NH) {
+    // ---- the products that have slack -- QKV of the items ahead, the projections -- are issued by a thread of their own, in item
+    // order, so that no group thread ever waits on their inputs.  Issue order is accumulation order (the heads of a unit add
+    // up in Y) and also orders a buffer's next accumulator behind the projection that reads the buffer last. -----------------
+    if (lane == 0 && w_ok) {
+      const uint32_t idesc_qkv = ptx::make_idesc_bf16(BM, WROWS, false, false);
+      const uint32_t idesc_pj = ptx::make_idesc_bf16(BM, C, false, false);
+      const uint32_t a_base = ptx::smem_u32(sA), ax_base = ptx::smem_u32(sAx), wq_base = ptx::smem_u32(sWq);
+      const uint32_t wx_base = ptx::smem_u32(sWx), wp_base = ptx::smem_u32(sWp);
+      int qi = 0, qh = 0, qu = 0, qab = 0, qaph = 0;   // QKV queue: item, head, unit, row-ring slot and its phase
+      int ji = 0, jh = 0, ju = 0;                      // projection queue
+      uint32_t idle = 0;
+      unsigned long long t_idle = 0;
+      while (ji < total) {
+        bool progress = false;
+        if (ptx::mbar_test(&ob_full[ji & (NBUF - 1)], (ji >> 2) & 1) && (jh != 0 || ptx::mbar_test(y_empty, (ju & 1) ^ 1))) {
+          // Y (+)= Ob_h Wp[:, 32 h : 32 h + 32]^T; the first head overwrites Y (the epilogue of the unit before has read it), the
+          // last one hands Y to the epilogue
           ptx::tc_fence_after();
-          const uint32_t idesc = ptx::make_idesc_bf16(BM, C, false, false);
-          const uint32_t a = tmem_base + h * 128 + 96;
-          const uint64_t bd = desc_sw64(ptx::smem_u32(sWp) + h * WP_TILE);
-          ptx::tc_mma_bf16_ta(tmem_base + TM_Y, a, bd, idesc, h ? 1u : 0u);
-          ptx::tc_mma_bf16_ta(tmem_base + TM_Y, a + 8, bd + 2, idesc, 1u);
-          ptx::tc_commit(pj_done);
-          if (h == NH - 1) ptx::tc_commit(y_full);
-          FDBG(it * 16 + 6);
-          // the same head of the next unit: its accumulator replaces P and O (read by now); Ob, which the product above is
-          // still reading, lies beside it
-          if (it + NH < total) issue_qkv(it + NH);
+          const uint32_t a = tmem_base + (ji & (NBUF - 1)) * BUF_COLS + 64;
+          const uint64_t bd = desc_sw64(wp_base + jh * WP_TILE);
+          ptx::tc_mma_bf16_ta(tmem_base + TM_Y, a, bd, idesc_pj, jh ? 1u : 0u);
+          ptx::tc_mma_bf16_ta(tmem_base + TM_Y, a + 8, bd + 2, idesc_pj, 1u);
+          if (jh == NH - 1) ptx::tc_commit(y_full);
+          ++ji;
+          if (++jh == NH) { jh = 0; ++ju; }
+          progress = true;
+        }
+        if (qi < total && qi < ji + NBUF && ptx::mbar_test(&a_full[qab], qaph)) {
+          // acc = [X | e] [Wq_h; Wk_h; Wv_h | f]^T into the buffer item qi - NBUF has left (its projection was issued above)
+          ptx::tc_fence_after();
+          const uint32_t d = tmem_base + (qi & (NBUF - 1)) * BUF_COLS;
+#pragma unroll
+          for (int kb = 0; kb < NH; ++kb) {
+            const uint64_t ad = desc_sw64(a_base + qab * A_BYTES + kb * KBT);
+            const uint64_t bd = desc_sw64(wq_base + (qh * NH + kb) * WQ_TILE);
+            ptx::tc_mma_bf16(d, ad, bd, idesc_qkv, kb ? 1u : 0u);
+            ptx::tc_mma_bf16(d, ad + 2, bd + 2, idesc_qkv, 1u);      // next 16 channels: +32 bytes
+          }
+          ptx::tc_mma_bf16(d, desc_plain(ax_base + qab * AX_BYTES), desc_plain(wx_base + qh * WX_TILE), idesc_qkv, 1u);
+          ptx::tc_commit(&acc_full[qi & (NBUF - 1)]);
+          ++qi;
+          if (++qh == NH) {
+            qh = 0; ++qu;
+            if (++qab == na) { qab = 0; qaph ^= 1; }
+          }
+          progress = true;
+        }
+        if (progress) {
+          idle = 0;
+        } else if ((++idle & 255u) == 0) {
+          if (*(volatile int*)abort_flag) break;
+          const unsigned long long now = ptx::globaltimer();
+          if (idle == 256u) t_idle = now;
+          else if (now - t_idle > ptx::kWaitLimitNs) {
+            *abort_flag = 1;
+            atomicExch(g.status, (int)SMARTMEM_ERR_TIMEOUT);
+            break;
+          }
         }
       }
     }
   } else {
-    // ---- row statistics of the units ahead, and the Y epilogue: y_row = Y + b_proj + x_row in place over the raw row, then the
-    // rows go out the way they came in (one TMA box per k-block for a window off the seam, a scatter through the map for a seam
-    // window).  One row per thread; whichever of the two jobs has its input ready is taken next. -----------------------------
+    // ---- row statistics of the units ahead, and the Y epilogue: y_row = Y + b_proj + x_row, stored at the row's offset under the
+    // map (the residual row comes from L2: the same kernel read it moments ago).  One row per thread; whichever of the two
+    // jobs has its input ready is taken next. ------------------------------------------------------------------------------------
     const int q = warp & 3;
     const int r = q * 32 + lane;
-    const int w = r >> 6, i = r & 63;
+    const int i = r & 63;
     const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
-    bool ok = true;
     auto row_ptr = [&](int ab, int row, int ch) { return sA + ab * A_BYTES + (ch >> 2) * KBT + sw64_off(row, ch & 3); };
-    int n_box = 0;                                     // box epilogues of this warp's window so far (phase of ysync[w])
     auto statistics = [&](int ul) {
       const int ab = ul % na;
       if (q == 0 && lane == 0) FDBG(4096 + ul * 8 + 3);
       if (i < T) {
         float rstd = 0.f;
         uint4 k0 = make_uint4(0, 0, 0, 0), k1 = k0;
-        if (rowoff_s[ab * BM + r] != ROW_INVALID) {
+        if (rowoff_s[(ul % NRING) * BM + r] != ROW_INVALID) {
           uint4 xr[NCH];
 #pragma unroll
           for (int ch = 0; ch < NCH; ++ch) xr[ch] = *reinterpret_cast<const uint4*>(row_ptr(ab, r, ch));
@@ -725,18 +770,19 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
       if (q == 0 && lane == 0) FDBG(4096 + ul * 8 + 4);
     };
     auto y_epilogue = [&](int ul) {
-      const int ab = ul % na;
       if (q == 0 && lane == 0) FDBG(4096 + ul * 8 + 5);
       ptx::tc_fence_after();
-      const uint32_t my_off = rowoff_s[ab * BM + r];
+      const uint32_t my_off = rowoff_s[(ul % NRING) * BM + r];
       const bool valid = i < T && my_off != ROW_INVALID;
+      const uint4* xg = reinterpret_cast<const uint4*>(g.x + ((size_t)(valid ? my_off : 0u) << 3));
+      uint4* yg = reinterpret_cast<uint4*>(g.y + ((size_t)(valid ? my_off : 0u) << 3));
+      uint4 xv[NCH];
+#pragma unroll
+      for (int ch = 0; ch < NCH; ++ch) xv[ch] = valid ? __ldg(xg + ch) : make_uint4(0, 0, 0, 0);   // the residual row (L2)
 #pragma unroll
       for (int k = 0; k < NH; ++k) {                   // 32 columns = 4 chunks of the row at a time
         uint32_t rv[32];
         ptx::tmem_ld32(tmem_base + TM_Y + lane_addr + k * 32, rv);
-        uint4 xv[4];
-#pragma unroll
-        for (int c = 0; c < 4; ++c) xv[c] = valid ? *reinterpret_cast<const uint4*>(row_ptr(ab, r, k * 4 + c)) : make_uint4(0, 0, 0, 0);
         ptx::tmem_ld_wait();
         if (k == NH - 1) {                             // Y is in registers: the next unit's projection may overwrite it
           ptx::tc_fence_before();
@@ -746,7 +792,7 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
         if (valid) {
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
-            const uint32_t x4[4] = {xv[c].x, xv[c].y, xv[c].z, xv[c].w};
+            const uint32_t x4[4] = {xv[k * 4 + c].x, xv[k * 4 + c].y, xv[k * 4 + c].z, xv[k * 4 + c].w};
             const float4 b0 = *reinterpret_cast<const float4*>(bp_s + k * 32 + c * 8);
             const float4 b1 = *reinterpret_cast<const float4*>(bp_s + k * 32 + c * 8 + 4);
             const f32x2 bb[4] = {ptx::pack2(b0.x, b0.y), ptx::pack2(b0.z, b0.w), ptx::pack2(b1.x, b1.y), ptx::pack2(b1.z, b1.w)};
@@ -759,46 +805,10 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
                                      ptx::pack2(__uint_as_float(x4[e] << 16), __uint_as_float(x4[e] & 0xFFFF0000u))), v0, v1);
               o4[e] = float2_to_bf16x2(v0, v1);
             }
-            *reinterpret_cast<uint4*>(row_ptr(ab, r, k * 4 + c)) = make_uint4(o4[0], o4[1], o4[2], o4[3]);
+            yg[k * 4 + c] = make_uint4(o4[0], o4[1], o4[2], o4[3]);
           }
         }
       }
-      const int4 wb = wbox_s[ab * 2 + w];
-      if (wb.x == WIN_BOX) {
-        // the window's rows belong to two warps: both hand them over, the first one's lane 0 stores the window
-        ptx::fence_proxy_async();                      // the rows written above -> visible to the TMA stores
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(&ysync[w]);
-        if ((q & 1) == 0 && lane == 0 && ptx::mbar_wait(&ysync[w], n_box & 1, abort_flag, g.status)) {
-#pragma unroll
-          for (int kb = 0; kb < NH; ++kb)
-            ptx::tma_store_4d(&tmY, sA + ab * A_BYTES + kb * KBT + w * (64 * 64), kb * D, wb.y, wb.z, wb.w);
-          ptx::bulk_commit_group();
-          ptx::bulk_wait_group_read<0>();              // the stores have read the slot: it may be refilled
-        }
-        ++n_box;
-      } else {
-        __syncwarp();
-        if (wb.x == WIN_GATHER) {
-          uint4 yv[NCH];
-          uint32_t ro[NCH];
-#pragma unroll
-          for (int k = 0; k < NCH; ++k) {               // the warp's 32 rows x NCH chunks: a row by consecutive lanes
-            const int idx = k * 32 + lane;
-            const int rr = idx / NCH, ch = idx - rr * NCH, row = q * 32 + rr;
-            ro[k] = (row & 63) < T ? rowoff_s[ab * BM + row] : ROW_INVALID;
-            yv[k] = *reinterpret_cast<const uint4*>(row_ptr(ab, row, ch));
-          }
-#pragma unroll
-          for (int k = 0; k < NCH; ++k) {
-            const int idx = k * 32 + lane;
-            const int ch = idx - (idx / NCH) * NCH;
-            if (ro[k] != ROW_INVALID) *reinterpret_cast<uint4*>(g.y + ((size_t)ro[k] << 3) + ch * 8) = yv[k];
-          }
-        }
-      }
-      __syncwarp();                                     // the warp's rows are read: the ring slot may be refilled
-      if (lane == 0) ptx::mbar_arrive(&a_free[ab]);
       if (q == 0 && lane == 0) FDBG(4096 + ul * 8 + 6);
     };
     int sdone = 0, edone = 0;                          // units whose statistics / whose epilogue this warp has done
@@ -807,8 +817,8 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
     while (edone < U) {
       int job = 0;                                     // lane 0 looks, the warp follows
       if (lane == 0) {
-        if (sdone < U && sdone - edone < na && ptx::mbar_test(&landed[sdone % na], (sdone / na) & 1)) job = 1;
-        else if (edone < sdone && ptx::mbar_test(y_full, edone & 1)) job = 2;
+        if (edone < sdone && ptx::mbar_test(y_full, edone & 1)) job = 2;
+        else if (sdone < U && ptx::mbar_test(&landed[sdone % na], (sdone / na) & 1)) job = 1;
         else if ((++idle & 63u) == 0) {
           const unsigned long long now = ptx::globaltimer();
           if (idle == 64u) t_idle = now;
@@ -825,7 +835,6 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
       else if (job == 3) break;
       else __nanosleep(32);
     }
-    ptx::bulk_wait_group<0>();                         // this thread's TMA stores are complete
   }
   ptx::tc_fence_before();
   __syncthreads();
@@ -851,23 +860,20 @@ int launch_swin_attn_fused(const smartmem_swin_params_t& p, const DevMap& rowmap
   for (const void* q : ptrs)
     if (!q || ((uintptr_t)q & 15)) return SMARTMEM_ERR_ALIGNMENT;
   if (!p.rel_bias_table) return SMARTMEM_ERR_INVALID_ARG;
-  CUtensorMap twq, twp;
+  CUtensorMap twq, twp, tx;
   int rc;
   if ((rc = tc_encode_2d_sw64(p.w_qkv, C, 3 * C, C, D, D, &twq)) != SMARTMEM_OK) return rc;
   if ((rc = tc_encode_2d_sw64(p.w_proj, C, C, C, D, C, &twp)) != SMARTMEM_OK) return rc;
-  CUtensorMap tx, ty;
   memset(&tx, 0, sizeof(tx));
-  memset(&ty, 0, sizeof(ty));
   const long long dims[4] = {C, p.W, p.H, p.B}, strides[3] = {C, (long long)p.W * C, (long long)p.H * p.W * C};
   const int box[4] = {D, p.window, p.window, 1};
-  const bool use_box = tc_encode_nd_sw64(x, 4, dims, strides, box, &tx) == SMARTMEM_OK &&
-                       tc_encode_nd_sw64(y, 4, dims, strides, box, &ty) == SMARTMEM_OK;
+  const bool use_box = tc_encode_nd_sw64(x, 4, dims, strides, box, &tx) == SMARTMEM_OK;
   FusedArgs g;
   memset(&g, 0, sizeof(g));
   g.use_box = use_box ? 1 : 0;
   g.n_windows = (int)n_windows;
   g.n_pairs = (int)((n_windows + 1) / 2);
-  g.T = T; g.ws = p.window; g.shift = p.shift;
+  g.T = T; g.ws = p.window; g.shift = p.shift; g.H = p.H; g.W = p.W;
   g.nWw = p.W / p.window; g.nWh = p.H / p.window; g.win_per_img = g.nWw * g.nWh;
   g.fd_wpi = make_fastdiv((uint32_t)g.win_per_img);
   g.fd_nww = make_fastdiv((uint32_t)g.nWw);
@@ -884,9 +890,9 @@ int launch_swin_attn_fused(const smartmem_swin_params_t& p, const DevMap& rowmap
   const bool kc56 = T <= 56;
   const int br = kc56 ? 28 : 36;
   auto need = [&](int na) {
-    return (size_t)na * NH * KBT + (size_t)NSLOT * KV_SLOT + (size_t)NH * NH * WQ_TILE + (size_t)NH * C * 64 +
-           (size_t)na * AX_BYTES + (size_t)NH * WX_TILE + (size_t)NH * T * br * 4 + (size_t)C * 4 + (size_t)na * BM * 8 +
-           (size_t)2 * C * 4 + TP * 4 + 16 + TP * 16 + 4 * 16 + 6 * 16 + N_BARS * 8 + 16;
+    return (size_t)na * NH * KBT + (size_t)NH * KV_SLOT + (size_t)NH * NH * WQ_TILE + (size_t)NH * C * 64 +
+           (size_t)na * AX_BYTES + (size_t)NH * WX_TILE + (size_t)NH * T * br * 4 + (size_t)C * 4 + (size_t)na * BM * 4 +
+           (size_t)NRING * BM * 4 + (size_t)2 * C * 4 + TP * 4 + 16 + TP * 16 + 4 * 16 + 32 + N_BARS * 8 + 16;
   };
   const size_t kMaxSmem = 232448;
   g.na = need(3) <= kMaxSmem ? 3 : 2;
@@ -898,12 +904,13 @@ int launch_swin_attn_fused(const smartmem_swin_params_t& p, const DevMap& rowmap
   if ((rc = ensure_max_dynamic_smem(fn, (int)kMaxSmem)) != SMARTMEM_OK) return rc;
   const int sms = tc_sm_count();
   const unsigned grid = (unsigned)(g.n_pairs < sms ? g.n_pairs : sms);
+  const unsigned threads = 32u * (9 + 4 * NH);
   profile_tick("attn_half_fused", st);
   cudaError_t e;
-  if (NH == 3) e = kc56 ? launch_pdl(swin_attn_fused_kernel<3, 56>, dim3(grid), dim3(kThreads), smem, st, twq, twp, tx, ty, g)
-                        : launch_pdl(swin_attn_fused_kernel<3, 64>, dim3(grid), dim3(kThreads), smem, st, twq, twp, tx, ty, g);
-  else e = kc56 ? launch_pdl(swin_attn_fused_kernel<2, 56>, dim3(grid), dim3(kThreads), smem, st, twq, twp, tx, ty, g)
-                : launch_pdl(swin_attn_fused_kernel<2, 64>, dim3(grid), dim3(kThreads), smem, st, twq, twp, tx, ty, g);
+  if (NH == 3) e = kc56 ? launch_pdl(swin_attn_fused_kernel<3, 56>, dim3(grid), dim3(threads), smem, st, twq, twp, tx, g)
+                        : launch_pdl(swin_attn_fused_kernel<3, 64>, dim3(grid), dim3(threads), smem, st, twq, twp, tx, g);
+  else e = kc56 ? launch_pdl(swin_attn_fused_kernel<2, 56>, dim3(grid), dim3(threads), smem, st, twq, twp, tx, g)
+                : launch_pdl(swin_attn_fused_kernel<2, 64>, dim3(grid), dim3(threads), smem, st, twq, twp, tx, g);
   count_launch();
   return e == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
 }
