@@ -216,6 +216,28 @@ __device__ __forceinline__ DevMapPart devmap_part(const DevMap& m, int a0, int a
   }
   return p;
 }
+// Same with a rolled loop over the atoms (indexed loads of the map constants): a fraction of the code, for callers that run
+// once in a long while, where the fetch of the instructions costs more than their execution.
+__device__ __forceinline__ DevMapPart devmap_part_rolled(const DevMap& m, int a0, int a1, uint32_t i) {
+  DevMapPart p{0, 0, 0, 0, 0};
+#pragma unroll 1
+  for (int a = a1 - 1; a >= a0; --a) {
+    const uint32_t q = fd_div(i, m.ext[a]);
+    const int digit = (int)(i - q * m.ext[a].d);
+    i = q;
+    const int r = m.roll_of[a];
+    if (r < 0) {
+      p.off += (long long)digit * m.stride[a];
+    } else {
+      const int w = digit * m.weight[a];
+      p.u0 += r == 0 ? w : 0;
+      p.u1 += r == 1 ? w : 0;
+      p.u2 += r == 2 ? w : 0;
+      p.u3 += r == 3 ? w : 0;
+    }
+  }
+  return p;
+}
 // sum of two contributions -> source offset (base added, rolled coordinates wrapped); maps with at most two rolls whose
 // wrapped coordinate is an affine coordinate of the producer (roll_n_parts <= 1)
 __device__ __forceinline__ long long devmap_finish2(const DevMap& m, long long off, int u0, int u1) {

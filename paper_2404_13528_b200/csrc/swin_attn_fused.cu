@@ -61,6 +61,8 @@ namespace {
 
 using ptx::f32x2;
 
+#define GWAIT(bar, par) ptx::mbar_wait(bar, par, abort_flag, g.status)
+
 constexpr int D = 32, TP = 64, BM = 128;
 constexpr int KBT = BM * 64;                        // a 128-row x 32-column bf16 tile: 64-byte rows, 64-byte swizzle
 constexpr int AX_BYTES = BM * 32;                   // the extra k-step of a unit: 128 rows x 16 bf16, no swizzle
@@ -69,7 +71,7 @@ constexpr int WQ_TILE = WROWS * 64;
 constexpr int WX_TILE = WROWS * 32;                 // the extra k-step of a head's weights
 constexpr int KV_SLOT = 2 * KBT;                    // k, v tiles of one item
 constexpr int NBUF = 4, BUF_COLS = 96;              // item buffers of tensor memory
-constexpr int NRING = 8;                            // units whose row offsets are kept (a unit's epilogue runs long after its gather)
+constexpr int NRING = 4;                            // units whose row offsets are kept (a unit's epilogue runs long after its gather)
 constexpr int kLoaderThreads = 128;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t TM_Y = NBUF * BUF_COLS;          // the projection's accumulator (C columns) after the item buffers
@@ -163,7 +165,8 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
   uint8_t* sWp = sWq + NH * NH * WQ_TILE;                          // [NH heads][C rows x 64 B]
   uint8_t* sAx = sWp + NH * WP_TILE;                               // [na][128 rows x 32 B]
   uint8_t* sWx = sAx + na * AX_BYTES;                              // [NH heads][96 rows x 32 B]
-  uint32_t* bias_s = reinterpret_cast<uint32_t*>(sWx + NH * WX_TILE);   // [NH][T][BR]: bf16 pairs
+  uint8_t* sId = sWx + NH * WX_TILE;                               // [NH k-blocks][C rows x 64 B]: the identity (the residual rides on the tensor core)
+  uint32_t* bias_s = reinterpret_cast<uint32_t*>(sId + NH * WP_TILE);   // [NH][T][BR]: bf16 pairs
   float* bp_s = reinterpret_cast<float*>(bias_s + NH * T * BR);    // [C]
   float* rstd_s = bp_s + C;                                        // [na][128]
   uint32_t* rowoff_s = reinterpret_cast<uint32_t*>(rstd_s + na * BM);   // [NRING][128]: row offset in 16-byte units
@@ -197,13 +200,15 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
 
   if (tid == 0) {
     ptx::mbar_init(w_full, 1);
+#pragma unroll 1
     for (int i = 0; i < 3; ++i) {
       ptx::mbar_init(&a_full[i], 4);
-      ptx::mbar_init(&a_free[i], NH);
+      ptx::mbar_init(&a_free[i], NH + 1);
       ptx::mbar_init(&landed[i], 4);
       ptx::mbar_init(&s_full[i], 1);
       ptx::mbar_init(&o_full[i], 1);
     }
+#pragma unroll 1
     for (int i = 0; i < NBUF; ++i) {
       ptx::mbar_init(&acc_full[i], 1);
       ptx::mbar_init(&ob_full[i], 4);
@@ -218,14 +223,18 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
     ptx::prefetch_tensormap(&tmWp);
     ptx::prefetch_tensormap(&tmX);
     ptx::mbar_expect_tx(w_full, (uint32_t)(NH * NH * WQ_TILE + NH * WP_TILE));
-    for (int h = 0; h < NH; ++h) {
+#pragma unroll 1
+    for (int h = 0; h < NH; ++h)                       // (head, k-block, q / k / v): a box of 32 weight rows x 32 columns
+#pragma unroll 1
       for (int kb = 0; kb < NH; ++kb)
+#pragma unroll
         for (int which = 0; which < 3; ++which)
           ptx::tma_load_2d(sWq + (h * NH + kb) * WQ_TILE + which * (D * 64), &tmWq, w_full, kb * D, which * C + h * D);
-      ptx::tma_load_2d(sWp + h * WP_TILE, &tmWp, w_full, h * D, 0);
-    }
+#pragma unroll 1
+    for (int h = 0; h < NH; ++h) ptx::tma_load_2d(sWp + h * WP_TILE, &tmWp, w_full, h * D, 0);
   }
   if (warp == 0) ptx::tmem_alloc(tmem_slot, TMEM_COLS);
+  if (tid == 0) FDBG(6900);
   // parameter-only tables
   const int n_table = (2 * ws - 1) * (2 * ws - 1);
   for (int i = tid; i < NH * 256; i += kThreads) {
@@ -236,7 +245,7 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
     tyx_s[tid] = ((tid / ws) << 8) | (tid % ws);
     int4 tk = make_int4(0, 0, 0, 0);
     if (g.split >= 0 && tid < T) {
-      const DevMapPart pt = devmap_part(g.rowmap, g.split, g.rowmap.n_atoms, (uint32_t)tid);
+      const DevMapPart pt = devmap_part_rolled(g.rowmap, g.split, g.rowmap.n_atoms, (uint32_t)tid);
       tk = make_int4((int)pt.off, pt.u0, pt.u1, 0);
     }
     tok_s[tid] = tk;
@@ -248,25 +257,35 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
   }
   for (int i = tid; i < na * A_BYTES / 16; i += kThreads) reinterpret_cast<uint4*>(sA)[i] = make_uint4(0, 0, 0, 0);
   for (int i = tid; i < na * AX_BYTES / 16; i += kThreads) reinterpret_cast<uint4*>(sAx)[i] = make_uint4(0, 0, 0, 0);
+  for (int i = tid; i < NH * WP_TILE / 16; i += kThreads) reinterpret_cast<uint4*>(sId)[i] = make_uint4(0, 0, 0, 0);
   for (int i = tid; i < na * BM; i += kThreads) rstd_s[i] = 0.f;
   for (int i = tid; i < NRING * BM; i += kThreads) rowoff_s[i] = ROW_INVALID;
+  if (tid == 0) FDBG(6901);
   __syncthreads();
-  // each head's bias as a [T, T] table of bf16 pairs, -inf for the padded keys
-  for (int i = tid; i < NH * T * (KC / 2); i += kThreads) {
-    const int hr = i / (KC / 2), c2 = i - hr * (KC / 2);            // (head, row), pair of keys
+  if (tid == 0) FDBG(6902);
+  if (tid < C)                                        // identity: row n of k-block n / 32 has a one in column n
+    *reinterpret_cast<uint16_t*>(sId + (tid >> 5) * WP_TILE + sw64_off(tid, (tid & 31) >> 3) + (tid & 7) * 2) = 0x3F80u;
+  // each head's bias as a [T, T] table of bf16 pairs, -inf for the padded keys; a task = a quarter of a row
+  for (int task = tid; task < NH * T * 4; task += kThreads) {
+    const int hr = task >> 2, qtr = task & 3;                       // (head, row), quarter of the row's key pairs
     const int h = hr / T, r = hr - h * T;
     const int ry = tyx_s[r] >> 8, rx = tyx_s[r] & 255;
-    uint32_t word = 0;
-    for (int k = 0; k < 2; ++k) {
-      const int c = 2 * c2 + k;
-      uint32_t bits = 0xFF80u;                         // -inf: padded keys never contribute
-      if (c < T) {
-        const int cy = tyx_s[c] >> 8, cx = tyx_s[c] & 255;
-        bits = raw_s[h * 256 + (ry - cy + ws - 1) * (2 * ws - 1) + (rx - cx + ws - 1)];
+    const uint16_t* tab = raw_s + h * 256 + (ry + ws - 1) * (2 * ws - 1) + (rx + ws - 1);
+#pragma unroll 1
+    for (int c2 = qtr * (KC / 8); c2 < (qtr + 1) * (KC / 8); ++c2) {
+      uint32_t word = 0;
+#pragma unroll
+      for (int k = 0; k < 2; ++k) {
+        const int c = 2 * c2 + k;
+        uint32_t bits = 0xFF80u;                       // -inf: padded keys never contribute
+        if (c < T) {
+          const int cyx = tyx_s[c];
+          bits = tab[-(cyx >> 8) * (2 * ws - 1) - (cyx & 255)];
+        }
+        word |= bits << (16 * k);
       }
-      word |= bits << (16 * k);
+      bias_s[hr * BR + c2] = word;
     }
-    bias_s[hr * BR + c2] = word;
   }
   // keys below / right of the wrap line of a seam window (bit c = key c)
   if (warp == 2) {
@@ -278,36 +297,49 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
     if (lane == 0) { kmask_s[0] = m0; kmask_s[1] = m1; kmask_s[2] = m2; kmask_s[3] = m3; }
   }
   // fold gamma into the resident QKV weights; the column terms c_n and b'_n go into the extra k-step (thread = one weight row)
+  if (tid == 0) FDBG(6903);
   const bool w_ok = ptx::mbar_wait(w_full, 0, abort_flag, g.status);
-  if (w_ok && tid < NH * WROWS) {
-    const int h = tid / WROWS, rr = tid - h * WROWS;
+  if (tid == 0) FDBG(6904);
+  if (w_ok && tid < 2 * NH * WROWS) {                  // (whole warps: 2 * NH * 96 is a multiple of 32)
+    const int row = tid >> 1, half = tid & 1;          // two threads per weight row: the first and second half of its chunks
+    const int h = row / WROWS, rr = row - h * WROWS;
     const int which = rr >> 5, j = rr & 31;
-    float csum = 0.f, bsum = __bfloat162float(g.b_qkv[which * C + h * D + j]);
+    float csum = 0.f, bsum = half ? 0.f : __bfloat162float(g.b_qkv[which * C + h * D + j]);
+#pragma unroll 2
+    for (int ci = half * (NCH / 2); ci < (half + 1) * (NCH / 2); ++ci) {     // chunk ci of the row: k-block ci / 4, chunk ci % 4
+      uint4* p = reinterpret_cast<uint4*>(sWq + (h * NH + (ci >> 2)) * WQ_TILE + sw64_off(rr, ci & 3));
+      const uint4 wv = *p;
+      const uint32_t w4[4] = {wv.x, wv.y, wv.z, wv.w};
+      uint32_t o4[4];
 #pragma unroll
-    for (int kb = 0; kb < NH; ++kb) {
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint4* p = reinterpret_cast<uint4*>(sWq + (h * NH + kb) * WQ_TILE + sw64_off(rr, c));
-        const uint4 wv = *p;
-        const uint32_t w4[4] = {wv.x, wv.y, wv.z, wv.w};
-        uint32_t o4[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int k = kb * D + c * 8 + 2 * e;
-          const float2 f = bf16x2_to_float2(w4[e]);
-          bsum = fmaf(ln_s[C + k], f.x, bsum);
-          bsum = fmaf(ln_s[C + k + 1], f.y, bsum);
-          o4[e] = float2_to_bf16x2(ln_s[k] * f.x, ln_s[k + 1] * f.y);
-          const float2 r2 = bf16x2_to_float2(o4[e]);
-          csum += r2.x + r2.y;
-        }
-        *p = make_uint4(o4[0], o4[1], o4[2], o4[3]);
+      for (int e = 0; e < 4; ++e) {
+        const int k = ci * 8 + 2 * e;
+        const float2 f = bf16x2_to_float2(w4[e]);
+        bsum = fmaf(ln_s[C + k], f.x, bsum);
+        bsum = fmaf(ln_s[C + k + 1], f.y, bsum);
+        o4[e] = float2_to_bf16x2(ln_s[k] * f.x, ln_s[k + 1] * f.y);
+        const float2 r2 = bf16x2_to_float2(o4[e]);
+        csum += r2.x + r2.y;
       }
+      *p = make_uint4(o4[0], o4[1], o4[2], o4[3]);
     }
-    uint4 k0, k1;
-    extra_col(csum, bsum, k0, k1);
-    *reinterpret_cast<uint4*>(sWx + h * WX_TILE + plain_off(rr, 0)) = k0;
-    *reinterpret_cast<uint4*>(sWx + h * WX_TILE + plain_off(rr, 1)) = k1;
+    csum += __shfl_xor_sync(0xFFFFFFFFu, csum, 1);
+    bsum += __shfl_xor_sync(0xFFFFFFFFu, bsum, 1);
+    if (half == 0) {
+      uint4 k0, k1;
+      extra_col(csum, bsum, k0, k1);
+      *reinterpret_cast<uint4*>(sWx + h * WX_TILE + plain_off(rr, 0)) = k0;
+      *reinterpret_cast<uint4*>(sWx + h * WX_TILE + plain_off(rr, 1)) = k1;
+    }
+  }
+  if (tid < 2 && U > 0 && g.split >= 0) {              // the first unit's windows under the map (parameters only)
+    const int n = 2 * cidx + tid;
+    int4 wp = make_int4(0, 0, 0, 0);
+    if (n < g.n_windows) {
+      const DevMapPart pw = devmap_part_rolled(g.rowmap, 0, g.split, (uint32_t)n);
+      wp = make_int4((int)(uint32_t)(pw.off & 0xFFFFFFFFll), (int)(pw.off >> 32), pw.u0, pw.u1);
+    }
+    win_s[tid] = wp;
   }
   ptx::fence_proxy_async();                           // the rewritten weights -> visible to the MMAs
   ptx::tc_fence_before();
@@ -340,7 +372,7 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
         const int n = 2 * (cidx + ul * cstride) + lt;
         int4 wp = make_int4(0, 0, 0, 0);
         if (n < g.n_windows) {
-          const DevMapPart pw = devmap_part(g.rowmap, 0, g.split, (uint32_t)n);
+          const DevMapPart pw = devmap_part_rolled(g.rowmap, 0, g.split, (uint32_t)n);
           wp = make_int4((int)(uint32_t)(pw.off & 0xFFFFFFFFll), (int)(pw.off >> 32), pw.u0, pw.u1);
         }
         win_s[(ul & 1) * 2 + lt] = wp;
@@ -400,10 +432,58 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
       ptx::cp_async_commit();
       window_part(ul + 1);                             // read after the next barrier of the loader threads
     };
+    auto statistics = [&](int ul) {
+      const int ab = ul % na;
+      if (lt == 0) FDBG(4096 + ul * 8 + 3);
+      const int r = lt, i = lt & 63;
+      if (i < T) {
+        float rstd = 0.f;
+        uint4 k0 = make_uint4(0, 0, 0, 0), k1 = k0;
+        if (rowoff_s[(ul % NRING) * BM + r] != ROW_INVALID) {
+          // two passes over the row in shared memory (mean, then squared deviations); the loops are only partly unrolled: this code
+          // runs once per unit, and fetching its instructions costs as much as executing them
+          f32x2 s2[2] = {0ull, 0ull};
+#pragma unroll 4
+          for (int ch = 0; ch < NCH; ++ch) {
+            const uint4 xv = *reinterpret_cast<const uint4*>(sA + ab * A_BYTES + (ch >> 2) * KBT + sw64_off(r, ch & 3));
+            const uint32_t x4[4] = {xv.x, xv.y, xv.z, xv.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+              s2[e & 1] = ptx::add2(s2[e & 1], ptx::pack2(__uint_as_float(x4[e] << 16), __uint_as_float(x4[e] & 0xFFFF0000u)));
+          }
+          float a0, a1, a2, a3;
+          ptx::unpack2(s2[0], a0, a1);
+          ptx::unpack2(s2[1], a2, a3);
+          const float mean = ((a0 + a1) + (a2 + a3)) * (1.0f / (float)C);
+          const f32x2 nm2 = ptx::pack2(-mean, -mean);
+          f32x2 q2[2] = {0ull, 0ull};
+#pragma unroll 4
+          for (int ch = 0; ch < NCH; ++ch) {
+            const uint4 xv = *reinterpret_cast<const uint4*>(sA + ab * A_BYTES + (ch >> 2) * KBT + sw64_off(r, ch & 3));
+            const uint32_t x4[4] = {xv.x, xv.y, xv.z, xv.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const f32x2 d2 = ptx::add2(ptx::pack2(__uint_as_float(x4[e] << 16), __uint_as_float(x4[e] & 0xFFFF0000u)), nm2);
+              q2[e & 1] = ptx::fma2(d2, d2, q2[e & 1]);
+            }
+          }
+          ptx::unpack2(q2[0], a0, a1);
+          ptx::unpack2(q2[1], a2, a3);
+          const float var = ((a0 + a1) + (a2 + a3)) * (1.0f / (float)C) + g.eps;
+          rstd = rsqrtf(var);
+          extra_row(-mean, var * rstd, k0, k1);          // sigma = var / sqrt(var)
+        }
+        rstd_s[ab * BM + r] = rstd;
+        *reinterpret_cast<uint4*>(sAx + ab * AX_BYTES + plain_off(r, 0)) = k0;
+        *reinterpret_cast<uint4*>(sAx + ab * AX_BYTES + plain_off(r, 1)) = k1;
+      }
+      ptx::fence_proxy_async();                        // the extra k-step -> visible to the MMAs
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&a_full[ab]);
+      if (lt == 0) FDBG(4096 + ul * 8 + 4);
+    };
     // A unit's rows are requested as soon as its ring slot is free (the QKV products of the unit that held it are done); when
     // no slot is free the oldest request in flight is waited for and handed to the statistics warps.
-    window_part(0);
-    asm volatile("bar.sync 2, 128;" ::: "memory");
     int issued = 0, done = 0;
     while (done < U) {
       if (issued < U && issued - done < na) {
@@ -432,7 +512,11 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
       ptx::fence_proxy_async();                        // the gathered rows -> visible to the MMAs
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&landed[done % na]);
+      // every row of the unit is in (the loader warps' copies and the TMA boxes): its statistics, a thread per row
+      ok = ptx::mbar_wait_relaxed(&landed[done % na], (done / na) & 1, abort_flag, g.status, 32);
+      if (vote(!ok, false)) break;
       if (lt == 0) FDBG(4096 + done * 8 + 2);
+      statistics(done);
       ++done;
     }
   } else if (warp < 4 + 4 * NH) {
@@ -470,8 +554,8 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
       const uint32_t tb = tmem_base + (it & (NBUF - 1)) * BUF_COLS + lane_addr;
       // -- q, k, v of this row: rstd times the accumulator (the mean and bias terms rode on the extra k-step) --
       if (elected) FDBG(it * 16 + 0);
-      ok = ok && ptx::mbar_wait(&a_full[ab], (ul / na) & 1, abort_flag, g.status) &&     // (long complete: orders the read of rstd)
-           ptx::mbar_wait(&acc_full[it & (NBUF - 1)], (it >> 2) & 1, abort_flag, g.status);
+      ok = ok && GWAIT(&a_full[ab], (ul / na) & 1) &&     // (long complete: orders the read of rstd)
+           GWAIT(&acc_full[it & (NBUF - 1)], (it >> 2) & 1);
       if (elected) FDBG(it * 16 + 1);
       if (ok) {
         if (elected) ptx::mbar_arrive(&a_free[ab]);      // this head's product has read the unit's rows
@@ -544,7 +628,7 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
         if (last_col) { diff_lo |= kx_lo ^ my_fx; diff_hi |= kx_hi ^ my_fx; }
       }
       // -- softmax of this row over its window's keys --
-      ok = ptx::mbar_wait(&s_full[gi], ul & 1, abort_flag, g.status);
+      ok = GWAIT(&s_full[gi], ul & 1);
       if (elected) FDBG(it * 16 + 3);
       float inv = 0.f;
       if (ok) {
@@ -627,7 +711,7 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
         FDBG(it * 16 + 4);
       }
       // -- O row: normalise, bf16 pairs, back into tensor memory as the projection's A operand --
-      ok = ptx::mbar_wait(&o_full[gi], ul & 1, abort_flag, g.status);
+      ok = GWAIT(&o_full[gi], ul & 1);
       if (elected) FDBG(it * 16 + 5);
       if (ok) {
         ptx::tc_fence_after();
@@ -661,17 +745,33 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
       const uint32_t wx_base = ptx::smem_u32(sWx), wp_base = ptx::smem_u32(sWp);
       int qi = 0, qh = 0, qu = 0, qab = 0, qaph = 0;   // QKV queue: item, head, unit, row-ring slot and its phase
       int ji = 0, jh = 0, ju = 0;                      // projection queue
+      int xu = 0, xab = 0, xaph = 0;                   // residual queue: unit, its row-ring slot and phase
+      const uint32_t id_base = ptx::smem_u32(sId);
       uint32_t idle = 0;
       unsigned long long t_idle = 0;
       while (ji < total) {
         bool progress = false;
-        if (ptx::mbar_test(&ob_full[ji & (NBUF - 1)], (ji >> 2) & 1) && (jh != 0 || ptx::mbar_test(y_empty, (ju & 1) ^ 1))) {
-          // Y (+)= Ob_h Wp[:, 32 h : 32 h + 32]^T; the first head overwrites Y (the epilogue of the unit before has read it), the
-          // last one hands Y to the epilogue
+        if (xu < U && xu <= ju && ptx::mbar_test(y_empty, (xu & 1) ^ 1) && ptx::mbar_test(&a_full[xab], xaph)) {
+          // Y = X I: the unit's raw rows open the accumulation (the epilogue of the unit before has read Y); exact, since every
+          // product is a bf16 value times one.  The product is the last reader of the unit's rows: its completion frees the slot.
+          ptx::tc_fence_after();
+#pragma unroll
+          for (int kb = 0; kb < NH; ++kb) {
+            const uint64_t ad = desc_sw64(a_base + xab * A_BYTES + kb * KBT), bd = desc_sw64(id_base + kb * WP_TILE);
+            ptx::tc_mma_bf16(tmem_base + TM_Y, ad, bd, idesc_pj, kb ? 1u : 0u);
+            ptx::tc_mma_bf16(tmem_base + TM_Y, ad + 2, bd + 2, idesc_pj, 1u);
+          }
+          ptx::tc_commit(&a_free[xab]);
+          ++xu;
+          if (++xab == na) { xab = 0; xaph ^= 1; }
+          progress = true;
+        }
+        if (xu > ju && ptx::mbar_test(&ob_full[ji & (NBUF - 1)], (ji >> 2) & 1)) {
+          // Y += Ob_h Wp[:, 32 h : 32 h + 32]^T; the last head hands Y to the epilogue
           ptx::tc_fence_after();
           const uint32_t a = tmem_base + (ji & (NBUF - 1)) * BUF_COLS + 64;
           const uint64_t bd = desc_sw64(wp_base + jh * WP_TILE);
-          ptx::tc_mma_bf16_ta(tmem_base + TM_Y, a, bd, idesc_pj, jh ? 1u : 0u);
+          ptx::tc_mma_bf16_ta(tmem_base + TM_Y, a, bd, idesc_pj, 1u);
           ptx::tc_mma_bf16_ta(tmem_base + TM_Y, a + 8, bd + 2, idesc_pj, 1u);
           if (jh == NH - 1) ptx::tc_commit(y_full);
           ++ji;
@@ -713,78 +813,27 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
       }
     }
   } else {
-    // ---- row statistics of the units ahead, and the Y epilogue: y_row = Y + b_proj + x_row, stored at the row's offset under the
-    // map (the residual row comes from L2: the same kernel read it moments ago).  One row per thread; whichever of the two
-    // jobs has its input ready is taken next. ------------------------------------------------------------------------------------
+    // ---- Y epilogue: Y already holds x_row + sum_h Ob_h Wp_h^T (the residual rode on the tensor core as a product with the
+    // identity); add the bias, round once, store the row at its offset under the map.  One row per thread. ------------------
     const int q = warp & 3;
     const int r = q * 32 + lane;
     const int i = r & 63;
     const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
-    auto row_ptr = [&](int ab, int row, int ch) { return sA + ab * A_BYTES + (ch >> 2) * KBT + sw64_off(row, ch & 3); };
-    auto statistics = [&](int ul) {
-      const int ab = ul % na;
-      if (q == 0 && lane == 0) FDBG(4096 + ul * 8 + 3);
-      if (i < T) {
-        float rstd = 0.f;
-        uint4 k0 = make_uint4(0, 0, 0, 0), k1 = k0;
-        if (rowoff_s[(ul % NRING) * BM + r] != ROW_INVALID) {
-          uint4 xr[NCH];
-#pragma unroll
-          for (int ch = 0; ch < NCH; ++ch) xr[ch] = *reinterpret_cast<const uint4*>(row_ptr(ab, r, ch));
-          f32x2 s2[2] = {0ull, 0ull};
-#pragma unroll
-          for (int ch = 0; ch < NCH; ++ch) {
-            const uint32_t x4[4] = {xr[ch].x, xr[ch].y, xr[ch].z, xr[ch].w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e)
-              s2[e & 1] = ptx::add2(s2[e & 1], ptx::pack2(__uint_as_float(x4[e] << 16), __uint_as_float(x4[e] & 0xFFFF0000u)));
-          }
-          float a0, a1, a2, a3;
-          ptx::unpack2(s2[0], a0, a1);
-          ptx::unpack2(s2[1], a2, a3);
-          const float mean = ((a0 + a1) + (a2 + a3)) * (1.0f / (float)C);
-          const f32x2 nm2 = ptx::pack2(-mean, -mean);
-          f32x2 q2[2] = {0ull, 0ull};
-#pragma unroll
-          for (int ch = 0; ch < NCH; ++ch) {
-            const uint32_t x4[4] = {xr[ch].x, xr[ch].y, xr[ch].z, xr[ch].w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const f32x2 d2 = ptx::add2(ptx::pack2(__uint_as_float(x4[e] << 16), __uint_as_float(x4[e] & 0xFFFF0000u)), nm2);
-              q2[e & 1] = ptx::fma2(d2, d2, q2[e & 1]);
-            }
-          }
-          ptx::unpack2(q2[0], a0, a1);
-          ptx::unpack2(q2[1], a2, a3);
-          const float var = ((a0 + a1) + (a2 + a3)) * (1.0f / (float)C) + g.eps;
-          rstd = rsqrtf(var);
-          extra_row(-mean, var * rstd, k0, k1);          // sigma = var / sqrt(var)
-        }
-        rstd_s[ab * BM + r] = rstd;
-        *reinterpret_cast<uint4*>(sAx + ab * AX_BYTES + plain_off(r, 0)) = k0;
-        *reinterpret_cast<uint4*>(sAx + ab * AX_BYTES + plain_off(r, 1)) = k1;
-      }
-      ptx::fence_proxy_async();                        // the extra k-step -> visible to the MMAs
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(&a_full[ab]);
-      if (q == 0 && lane == 0) FDBG(4096 + ul * 8 + 4);
-    };
-    auto y_epilogue = [&](int ul) {
+    bool ok = true;
+    for (int ul = 0; ul < U && ok; ++ul) {
+      ok = ptx::mbar_wait_relaxed(y_full, ul & 1, abort_flag, g.status, 32);
+      if (!ok) break;
       if (q == 0 && lane == 0) FDBG(4096 + ul * 8 + 5);
       ptx::tc_fence_after();
       const uint32_t my_off = rowoff_s[(ul % NRING) * BM + r];
       const bool valid = i < T && my_off != ROW_INVALID;
-      const uint4* xg = reinterpret_cast<const uint4*>(g.x + ((size_t)(valid ? my_off : 0u) << 3));
       uint4* yg = reinterpret_cast<uint4*>(g.y + ((size_t)(valid ? my_off : 0u) << 3));
-      uint4 xv[NCH];
-#pragma unroll
-      for (int ch = 0; ch < NCH; ++ch) xv[ch] = valid ? __ldg(xg + ch) : make_uint4(0, 0, 0, 0);   // the residual row (L2)
-#pragma unroll
+#pragma unroll 1
       for (int k = 0; k < NH; ++k) {                   // 32 columns = 4 chunks of the row at a time
         uint32_t rv[32];
         ptx::tmem_ld32(tmem_base + TM_Y + lane_addr + k * 32, rv);
         ptx::tmem_ld_wait();
-        if (k == NH - 1) {                             // Y is in registers: the next unit's projection may overwrite it
+        if (k == NH - 1) {                             // Y is in registers: the next unit's products may overwrite it
           ptx::tc_fence_before();
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive(y_empty);
@@ -792,7 +841,6 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
         if (valid) {
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
-            const uint32_t x4[4] = {xv[k * 4 + c].x, xv[k * 4 + c].y, xv[k * 4 + c].z, xv[k * 4 + c].w};
             const float4 b0 = *reinterpret_cast<const float4*>(bp_s + k * 32 + c * 8);
             const float4 b1 = *reinterpret_cast<const float4*>(bp_s + k * 32 + c * 8 + 4);
             const f32x2 bb[4] = {ptx::pack2(b0.x, b0.y), ptx::pack2(b0.z, b0.w), ptx::pack2(b1.x, b1.y), ptx::pack2(b1.z, b1.w)};
@@ -801,8 +849,7 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
             for (int e = 0; e < 4; ++e) {
               const int col = c * 8 + 2 * e;
               float v0, v1;
-              ptx::unpack2(ptx::add2(ptx::add2(ptx::pack2(__uint_as_float(rv[col]), __uint_as_float(rv[col + 1])), bb[e]),
-                                     ptx::pack2(__uint_as_float(x4[e] << 16), __uint_as_float(x4[e] & 0xFFFF0000u))), v0, v1);
+              ptx::unpack2(ptx::add2(ptx::pack2(__uint_as_float(rv[col]), __uint_as_float(rv[col + 1])), bb[e]), v0, v1);
               o4[e] = float2_to_bf16x2(v0, v1);
             }
             yg[k * 4 + c] = make_uint4(o4[0], o4[1], o4[2], o4[3]);
@@ -810,30 +857,6 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
         }
       }
       if (q == 0 && lane == 0) FDBG(4096 + ul * 8 + 6);
-    };
-    int sdone = 0, edone = 0;                          // units whose statistics / whose epilogue this warp has done
-    uint32_t idle = 0;
-    unsigned long long t_idle = 0;
-    while (edone < U) {
-      int job = 0;                                     // lane 0 looks, the warp follows
-      if (lane == 0) {
-        if (edone < sdone && ptx::mbar_test(y_full, edone & 1)) job = 2;
-        else if (sdone < U && ptx::mbar_test(&landed[sdone % na], (sdone / na) & 1)) job = 1;
-        else if ((++idle & 63u) == 0) {
-          const unsigned long long now = ptx::globaltimer();
-          if (idle == 64u) t_idle = now;
-          else if (*(volatile int*)abort_flag || now - t_idle > ptx::kWaitLimitNs) {
-            *abort_flag = 1;
-            atomicExch(g.status, (int)SMARTMEM_ERR_TIMEOUT);
-            job = 3;
-          }
-        }
-      }
-      job = __shfl_sync(0xFFFFFFFFu, job, 0);
-      if (job == 1) { statistics(sdone); ++sdone; idle = 0; }
-      else if (job == 2) { y_epilogue(edone); ++edone; idle = 0; }
-      else if (job == 3) break;
-      else __nanosleep(32);
     }
   }
   ptx::tc_fence_before();
@@ -847,8 +870,18 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
 
 }  // namespace
 
+// shared memory of a CTA with a row ring of `na` slots
+static size_t fused_smem_need(int NH, int T, int na) {
+  const int C = NH * D, br = T <= 56 ? 28 : 36;
+  return (size_t)na * NH * KBT + (size_t)NH * KV_SLOT + (size_t)NH * NH * WQ_TILE + (size_t)NH * C * 64 +
+         (size_t)na * AX_BYTES + (size_t)NH * WX_TILE + (size_t)NH * C * 64 + (size_t)NH * T * br * 4 + (size_t)C * 4 +
+         (size_t)na * BM * 4 + (size_t)NRING * BM * 4 + (size_t)2 * C * 4 + TP * 4 + 16 + TP * 16 + 4 * 16 + 32 + N_BARS * 8 + 16;
+}
+static constexpr size_t kMaxSmem = 232448;
+
 bool swin_attn_fused_supported(int dtype, int C, int heads, int window) {
-  return dtype == SMARTMEM_BF16 && (heads == 2 || heads == 3) && C == heads * D && window * window <= TP && window >= 1;
+  return dtype == SMARTMEM_BF16 && (heads == 2 || heads == 3) && C == heads * D && window * window <= TP && window >= 1 &&
+         fused_smem_need(heads, window * window, 2) <= kMaxSmem;
 }
 
 int launch_swin_attn_fused(const smartmem_swin_params_t& p, const DevMap& rowmap, const void* x, void* y, cudaStream_t st) {
@@ -888,13 +921,7 @@ int launch_swin_attn_fused(const smartmem_swin_params_t& p, const DevMap& rowmap
   g.status = device_status_ptr();
   if (!g.status) return SMARTMEM_ERR_CUDA;
   const bool kc56 = T <= 56;
-  const int br = kc56 ? 28 : 36;
-  auto need = [&](int na) {
-    return (size_t)na * NH * KBT + (size_t)NH * KV_SLOT + (size_t)NH * NH * WQ_TILE + (size_t)NH * C * 64 +
-           (size_t)na * AX_BYTES + (size_t)NH * WX_TILE + (size_t)NH * T * br * 4 + (size_t)C * 4 + (size_t)na * BM * 4 +
-           (size_t)NRING * BM * 4 + (size_t)2 * C * 4 + TP * 4 + 16 + TP * 16 + 4 * 16 + 32 + N_BARS * 8 + 16;
-  };
-  const size_t kMaxSmem = 232448;
+  auto need = [&](int na) { return fused_smem_need(NH, T, na); };
   g.na = need(3) <= kMaxSmem ? 3 : 2;
   if (need(g.na) > kMaxSmem) return SMARTMEM_ERR_UNSUPPORTED;
   const size_t smem = need(g.na) + 1024 <= kMaxSmem ? need(g.na) + 1024 : kMaxSmem;   // alignment slack only while it fits
