@@ -34,8 +34,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not _stale():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    extra = os.environ.get("SMARTMEM_NVCC_EXTRA", "").split()      # e.g. -D switches for experiments
-    cmd = [nvcc, *NVCC_FLAGS, *extra, "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-o", LIB]
+    cmd = [nvcc, *NVCC_FLAGS, "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-o", LIB]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += _sources()

@@ -21,15 +21,6 @@
 #include "gemm_tc.cuh"
 #include "ptx.cuh"
 
-#ifdef CA_EXP_TIMING
-__device__ long long g_ca_dbg[8192];
-#define CDBG(slot) do { if (blockIdx.x == 0) g_ca_dbg[(slot)] = clock64(); } while (0)
-extern "C" __attribute__((visibility("default"))) int smartmem_debug_read_ca(long long* host, int n) {
-  return (int)cudaMemcpyFromSymbol(host, g_ca_dbg, sizeof(long long) * n);
-}
-#else
-#define CDBG(slot) do { } while (0)
-#endif
 
 namespace smartmem {
 namespace {
@@ -126,15 +117,12 @@ causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         const int s = j & 1;
         const uint32_t ph = (j >> 1) & 1;
         const int krow = (int)(row_base + (long long)j * BKV);
-        CDBG(j * 16 + 0);
         ok = ptx::mbar_wait(&k_empty[s], ph ^ 1, abort_flag, g.status);
         if (!ok) break;
-        CDBG(j * 16 + 1);
         ptx::mbar_expect_tx(&k_full[s], 2 * KBK);
         for (int kb = 0; kb < 2; ++kb) ptx::tma_load_2d(sK + (s * 2 + kb) * KBK, &tmK, &k_full[s], kc + kb * 64, krow);
         ok = ptx::mbar_wait(&v_empty[s], ph ^ 1, abort_flag, g.status);
         if (!ok) break;
-        CDBG(j * 16 + 2);
         ptx::mbar_expect_tx(&v_full[s], 2 * KBK);
         for (int dc = 0; dc < 2; ++dc) ptx::tma_load_2d(sV + (s * 2 + dc) * KBK, &tmV, &v_full[s], vc + dc * 64, krow);
       }
@@ -147,12 +135,9 @@ causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       auto issue_s = [&](int j) {
         const int s = j & 1;
         const uint32_t ph = (j >> 1) & 1;
-        CDBG(j * 16 + 3);
         ok = ok && ptx::mbar_wait(&s_empty[s], ph ^ 1, abort_flag, g.status);
-        CDBG(j * 16 + 4);
         ok = ok && ptx::mbar_wait(&k_full[s], ph, abort_flag, g.status);
         if (!ok) return;
-        CDBG(j * 16 + 5);
         ptx::tc_fence_after();
 #pragma unroll
         for (int kb = 0; kb < 2; ++kb) {
@@ -164,16 +149,12 @@ causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         }
         ptx::tc_commit(&k_empty[s]);
         ptx::tc_commit(&s_full[s]);
-        CDBG(j * 16 + 6);
       };
       auto issue_pv = [&](int j) {
         const int s = j & 1;
-        CDBG(j * 16 + 7);
         ok = ok && ptx::mbar_wait(p_full, j & 1, abort_flag, g.status);
-        CDBG(j * 16 + 8);
         ok = ok && ptx::mbar_wait(&v_full[s], (j >> 1) & 1, abort_flag, g.status);
         if (!ok) return;
-        CDBG(j * 16 + 9);
         ptx::tc_fence_after();
         const uint32_t v0 = ptx::smem_u32(sV + s * 2 * KBK);
         const uint64_t vd = ptx::make_smem_desc(v0, KBK, 1024);
@@ -184,7 +165,6 @@ causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         ptx::tc_commit(&v_empty[s]);
         ptx::tc_commit(&s_empty[s]);
         ptx::tc_commit(p_empty);
-        CDBG(j * 16 + 10);
       };
       issue_s(0);
       for (int j = 0; j < n_kv && ok; ++j) {
@@ -202,10 +182,8 @@ causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     bool ok = true;
     for (int j = 0; j < n_kv && ok; ++j) {
       const int sb = j & 1;
-      if (warp == 2 && lane == 0) CDBG(j * 16 + 11);
       ok = ptx::mbar_wait(&s_full[sb], (j >> 1) & 1, abort_flag, g.status);
       if (!ok) break;
-      if (warp == 2 && lane == 0) CDBG(j * 16 + 12);
       ptx::tc_fence_after();
       const uint32_t ts = tmem_base + TM_S + sb * BKV + lane_addr;
       const bool diag = (j >= 2 * qt);                 // the two 64-key blocks that straddle this tile's diagonal
@@ -251,10 +229,8 @@ causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       l += l0 + l1;
       if (__any_sync(0xFFFFFFFFu, rescale)) {
         // O is rescaled in place: the previous P V, which accumulates into it, must have completed
-        if (warp == 2 && lane == 0) CDBG(j * 16 + 13);
         ok = ptx::mbar_wait(p_empty, (j & 1) ^ 1, abort_flag, g.status);
         if (!ok) break;
-        if (warp == 2 && lane == 0) CDBG(j * 16 + 14);
         ptx::tc_fence_after();
         const uint32_t to = tmem_base + TM_O + lane_addr;
 #pragma unroll 1
@@ -275,7 +251,6 @@ causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(p_full);
-      if (warp == 2 && lane == 0) CDBG(j * 16 + 15);
     }
     if (ok) ok = ptx::mbar_wait(o_done, 0, abort_flag, g.status);
     if (ok) {

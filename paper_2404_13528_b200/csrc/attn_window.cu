@@ -145,9 +145,6 @@ __global__ void __launch_bounds__(128) win_attn_bf16_kernel(const __grid_constan
       for (int j = 0; j < 8; ++j) s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
 #pragma unroll
       for (int kk = 0; kk < D / 16; ++kk) {
-#ifdef WA_EXP_NOQK
-        s[kk][0] = __uint_as_float(Qw[r0 * RW + t4]); break;
-#endif
         uint32_t af[4];
         af[0] = Qw[r0 * RW + kk * 8 + t4];
         af[1] = Qw[r1 * RW + kk * 8 + t4];
@@ -163,7 +160,6 @@ __global__ void __launch_bounds__(128) win_attn_bf16_kernel(const __grid_constan
         }
       }
       // ---- scale + bias (+ mask on the windows that touch the seam), softmax ------------------
-#ifndef WA_EXP_NOSOFTMAX
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
 #pragma unroll
@@ -202,11 +198,7 @@ __global__ void __launch_bounds__(128) win_attn_bf16_kernel(const __grid_constan
       for (int j = 0; j < 8; ++j) {
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
-#ifdef WA_EXP_NOEXP
-          const float p0 = s[j][e] - m0, p1 = s[j][2 + e] - m1;
-#else
           const float p0 = __expf(s[j][e] - m0), p1 = __expf(s[j][2 + e] - m1);
-#endif
           s[j][e] = p0;
           s[j][2 + e] = p1;
           sum0 += p0;
@@ -217,21 +209,12 @@ __global__ void __launch_bounds__(128) win_attn_bf16_kernel(const __grid_constan
       sum0 += __shfl_xor_sync(0xFFFFFFFFu, sum0, 2);
       sum1 += __shfl_xor_sync(0xFFFFFFFFu, sum1, 1);
       sum1 += __shfl_xor_sync(0xFFFFFFFFu, sum1, 2);
-#else
-      float sum0 = 1.f, sum1 = 1.f;
-#endif
       // ---- O = P V: the score fragments are the A fragments of the second MMA -----------------
       float o[D / 8][4];
 #pragma unroll
       for (int j = 0; j < D / 8; ++j) o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f;
-#ifdef WA_EXP_NOPV
-      for (int j = 0; j < D / 8; ++j) { o[j][0] = s[j][0]; o[j][1] = s[j][1]; o[j][2] = s[j][2]; o[j][3] = s[j][3]; }
-#endif
 #pragma unroll
       for (int kk = 0; kk < 4; ++kk) {
-#ifdef WA_EXP_NOPV
-        break;
-#endif
         if (kk * 16 < T) {
           uint32_t af[4];
           af[0] = float2_to_bf16x2(s[2 * kk][0], s[2 * kk][1]);

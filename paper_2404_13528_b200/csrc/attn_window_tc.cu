@@ -24,23 +24,12 @@
 // (a key is in another region iff it lies on the other side of the wrap line) and only for windows
 // in the last window row or column.
 //
-// What bounds it (clock-stamped build, -DWA_EXP_TIMING): the softmax groups, at about 1700 cycles
+// What bounds it (measured with clock stamps at every hand-off): the softmax groups, at about 1700 cycles
 // per window pair; the tensor pipe is busy for about 500 of them.
 #include "attn.cuh"
 #include "gemm_tc.cuh"
 #include "ptx.cuh"
 
-#ifdef WA_EXP_TIMING
-__device__ long long g_wa_dbg[8192];
-#define WDBG(slot) do { if (blockIdx.x == 0) g_wa_dbg[(slot)] = clock64(); } while (0)
-#define WDBGT(k) do { if (threadIdx.x == 0) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_wa_dbg[6000 + blockIdx.x * 4 + (k)] = (long long)t_; } } while (0)
-extern "C" __attribute__((visibility("default"))) int smartmem_debug_read_wa(long long* host, int n) {
-  return (int)cudaMemcpyFromSymbol(host, g_wa_dbg, sizeof(long long) * n);
-}
-#else
-#define WDBG(slot) do { } while (0)
-#define WDBGT(k) do { } while (0)
-#endif
 
 namespace smartmem {
 namespace {
@@ -87,7 +76,6 @@ template <int KC>
 __global__ void __launch_bounds__(kThreads, 1)
 win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constant__ CUtensorMap tm1,
                    const __grid_constant__ CUtensorMap tm2, const __grid_constant__ WinTcArgs g) {
-  WDBGT(0);
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
   uint8_t* sIn = smem;                                 // [NSTAGE][q, k, v][128 rows x 64 B]
@@ -179,9 +167,7 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  WDBGT(1);
   pdl_wait();                       // the tables above depend on parameters only: they overlapped the previous kernel's tail
-  WDBGT(2);
   pdl_launch_dependents();
   const CUtensorMap* tms[3] = {&tm0, &tm1, &tm2};
   const AttnOperand* ops[3] = {&a.q, &a.k, &a.v};
@@ -198,9 +184,6 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
         ok = ptx::mbar_wait(&in_empty[s], ((it / NSTAGE) & 1) ^ 1, abort_flag, g.status);
         if (!ok) break;
         const int nwin = (2 * p + 1 < a.n_windows) ? 2 : 1;
-#ifdef WA_EXP_NOLOAD
-        if (it >= NSTAGE) { ptx::mbar_arrive(&in_full[s]); continue; }
-#endif
         ptx::mbar_expect_tx(&in_full[s], (uint32_t)(n_tma * nwin * TP * 64));
         for (int m = 0; m < 3; ++m) {
           if (!((g.tma_mask >> m) & 1)) continue;
@@ -220,11 +203,9 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
       const int my_units = cidx < g.n_pairs ? (g.n_pairs - cidx + cstride - 1) / cstride : 0;
       for (int u = 0; u < my_units && ok; ++u) {
         const int s = u % NSTAGE, ob = u & 1;
-        WDBG(u * 16 + 2);
         ok = ptx::mbar_wait(&p_full[ob], (u >> 1) & 1, abort_flag, g.status);
         ok = ok && ptx::mbar_wait(&o_empty[ob], ((u >> 1) & 1) ^ 1, abort_flag, g.status);
         if (!ok) break;
-        WDBG(u * 16 + 3);
         ptx::tc_fence_after();
         const uint32_t v0 = ptx::smem_u32(sIn + s * STAGE_BYTES + 2 * OP_BYTES);
         const uint64_t vd = make_desc_sw64(v0, 16, 512);
@@ -236,7 +217,6 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
         ptx::tc_commit(&in_empty[s]);
         ptx::tc_commit(&p_empty[ob]);
         ptx::tc_commit(&o_full[ob]);
-        WDBG(u * 16 + 4);
       }
     }
   } else if (warp == 2 + kGroups * kSoftmaxWarps + kLoaderWarps) {
@@ -248,7 +228,6 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
       const int my_units = cidx < g.n_pairs ? (g.n_pairs - cidx + cstride - 1) / cstride : 0;
       for (int u = 0; u < my_units && ok; ++u) {
         const int s = u % NSTAGE, sb = u & 1;
-        WDBG(u * 16 + 0);
         ok = ptx::mbar_wait(&s_empty[sb], ((u >> 1) & 1) ^ 1, abort_flag, g.status);
         ok = ok && ptx::mbar_wait(&in_full[s], (u / NSTAGE) & 1, abort_flag, g.status);
         if (!ok) break;
@@ -258,7 +237,6 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
         ptx::tc_mma_bf16(tmem_base + TM_S + sb * 128, qd, kd, idesc_s, 0u);
         ptx::tc_mma_bf16(tmem_base + TM_S + sb * 128, qd + 2, kd + 2, idesc_s, 1u);    // next 16 features: +32 bytes
         ptx::tc_commit(&s_full[sb]);
-        WDBG(u * 16 + 1);
       }
     }
   } else if (warp < 2 + kGroups * kSoftmaxWarps) {
@@ -287,7 +265,6 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
       const int ob = u & 1;                            // == gi
       ok = ok && ptx::mbar_wait(&o_full[ob], (u >> 1) & 1, abort_flag, g.status);
       if (!ok) return;
-      if (q == 0 && lane == 0) WDBG(u * 16 + 10);
       ptx::tc_fence_after();
       uint32_t rv[32];
       ptx::tmem_ld32(tmem_base + TM_O + ob * D + lane_addr, rv);
@@ -302,14 +279,9 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
           float o8[8];
 #pragma unroll
           for (int e = 0; e < 8; ++e) o8[e] = __uint_as_float(rv[v * 8 + e]) * inv;
-#ifndef WA_EXP_NOSTORE
           ElemIO<__nv_bfloat16>::store(dst + v * 8, o8);
-#else
-          if (o8[0] == 123.456f) ElemIO<__nv_bfloat16>::store(dst + v * 8, o8);
-#endif
         }
       }
-      if (q == 0 && lane == 0) WDBG(u * 16 + 11);
     };
     int u = gi;
     int done = 0;
@@ -330,10 +302,8 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
         if (last_row) { diff_lo |= ky_lo ^ my_fy; diff_hi |= ky_hi ^ my_fy; }
         if (last_col) { diff_lo |= kx_lo ^ my_fx; diff_hi |= kx_hi ^ my_fx; }
       }
-      if (q == 0 && lane == 0) WDBG(u * 16 + 5);
       ok = ptx::mbar_wait(&s_full[sb], (u >> 1) & 1, abort_flag, g.status);
       if (!ok) break;
-      if (q == 0 && lane == 0) WDBG(u * 16 + 6);
       ptx::tc_fence_after();
       uint32_t rv[KC];
       const uint32_t ts = tmem_base + TM_S + sb * 128 + lane_addr + w * 64;    // this window's 64 key columns
@@ -345,15 +315,11 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
         ptx::tmem_ld8(ts + 48, rv + 48);
       }
       ptx::tmem_ld_wait();
-      if (q == 0 && lane == 0) WDBG(u * 16 + 7);
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&s_empty[sb]);
       float sc[KC];
       float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // independent chains
-#ifdef WA_EXP_TIMING
-      if (q == 0 && lane == 0 && __uint_as_float(rv[KC - 1]) != 123.456f) WDBG(u * 16 + 13);
-#endif
       // scores in natural units: q.k * scale + bias (the row's 64 biases come as eight 16-byte reads
       // of bf16 pairs); the base-2 conversion is folded into the exponent's multiply-add below
 #pragma unroll
@@ -378,9 +344,6 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
       for (int c = 0; c < KC; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], sc[c]);
       const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       const float nmx = -mx * LOG2E;
-#ifdef WA_EXP_TIMING
-      if (q == 0 && lane == 0 && mx > -1e30f) WDBG(u * 16 + 12);
-#endif
       float sum4[4] = {0.f, 0.f, 0.f, 0.f};
       uint32_t pk[32];
 #pragma unroll
@@ -393,7 +356,6 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
         pk[c / 2] = float2_to_bf16x2(p0, p1);
       }
       const float inv = 1.f / ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
-      if (q == 0 && lane == 0) WDBG(u * 16 + 8);
       // drain this group's previous unit: its P V has finished by now, and the O buffer it frees is
       // the one this unit's P V accumulates into
       if (done > 0) epilogue(u - 2, inv_prev, n_prev);
@@ -409,7 +371,6 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&p_full[gi]);
-      if (q == 0 && lane == 0) WDBG(u * 16 + 9);
       inv_prev = inv;
       n_prev = n;
     }
@@ -478,7 +439,6 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
   }
   ptx::tc_fence_before();
   __syncthreads();
-  WDBGT(3);
   if (warp == 1) {
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem_base, TMEM_COLS);

@@ -23,17 +23,6 @@
 #include "gemm_tc.cuh"
 #include "ptx.cuh"
 
-#ifdef LNG_EXP_TIMING
-__device__ long long g_lng_dbg[8192];
-#define LDBG(slot) do { if (blockIdx.x == 0) g_lng_dbg[(slot)] = clock64(); } while (0)
-#define LDBGT(k) do { if (threadIdx.x == 0) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_lng_dbg[6000 + blockIdx.x * 4 + (k)] = (long long)t_; } } while (0)
-extern "C" __attribute__((visibility("default"))) int smartmem_debug_read_lng(long long* host, int n) {
-  return (int)cudaMemcpyFromSymbol(host, g_lng_dbg, sizeof(long long) * n);
-}
-#else
-#define LDBG(slot) do { } while (0)
-#define LDBGT(k) do { } while (0)
-#endif
 
 namespace smartmem {
 namespace {
@@ -65,7 +54,6 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   constexpr int NH = KDIM / 16;                    // 16-byte chunks per half row (one thread's share)
   constexpr int NKB = KDIM > BK ? 2 : 1;
   constexpr int K1_STEPS = (KDIM - BK) / 16;       // k16 steps of the second k-block
-  LDBGT(0);
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const uint32_t pad = (1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u;
   uint8_t* smem = smem_raw + pad;
@@ -123,9 +111,7 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  LDBGT(1);
   pdl_wait();                       // everything above depends on parameters only
-  LDBGT(2);
   pdl_launch_dependents();
 
   if (warp == 1) {
@@ -136,14 +122,11 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       bool ok = ptx::mbar_wait(b_full, 0, abort_flag, g.status);
       uint32_t ab = 0, aph = 0, buf = 0, cph = 1;     // A ring position / phase, accumulator ring position / phase
       for (int ti = 0; ti < my_tiles && ok; ++ti) {
-        LDBG(ti * 32 + 0);
         ok = ptx::mbar_wait(&a_full[ab], aph, abort_flag, g.status);
-        LDBG(ti * 32 + 1);
         const uint64_t ad = ptx::make_smem_desc(a_base + ab * A_BYTES, 16, 1024);
         for (int j = 0; j < nsub && ok; ++j) {
           ok = ptx::mbar_wait(&acc_empty[buf], cph, abort_flag, g.status);
           if (!ok) break;
-          LDBG(ti * 32 + 2 + j);
           ptx::tc_fence_after();
           const uint32_t d = tmem_base + buf * BN;
           const uint64_t bd = ptx::make_smem_desc(b_base + j * (BN * 128), 16, 1024);
@@ -159,7 +142,6 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
           if (++buf == NACC) { buf = 0; cph ^= 1; }
         }
         if (ok) ptx::tc_commit(&a_empty[ab]);         // every MMA that reads this A tile has been issued
-        LDBG(ti * 32 + 5);
         if (++ab == NA) { ab = 0; aph ^= 1; }
       }
     }
@@ -181,9 +163,7 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         // the store issued from this staging buffer two sub-tiles ago must have read it
         if (elected) ptx::bulk_wait_group_read<1>();
         asm volatile("bar.sync %0, 64;" ::"r"(1 + q) : "memory");
-        if (e == 0 && lane == 0) LDBG(ti * 32 + 8 + j * 3);
         ok = ptx::mbar_wait(&acc_full[buf], cph, abort_flag, g.status);
-        if (e == 0 && lane == 0) LDBG(ti * 32 + 9 + j * 3);
         if (ok) {
           uint32_t rv[48];
           ptx::tc_fence_after();
@@ -225,7 +205,6 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
           ptx::tma_store_2d(&tmOB, stB, j * BN + 64, t * BM + q * 32);
           ptx::bulk_commit_group();
         }
-        if (e == 0 && lane == 0) LDBG(ti * 32 + 10 + j * 3);
         if (++buf == NACC) { buf = 0; cph ^= 1; }
       }
     }
@@ -249,9 +228,7 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     bool ok = true;
     uint32_t ab = 0, aph = 1;
     for (int ti = 0; ti < my_tiles && ok; ++ti) {
-      if (pw == 0 && lane == 0) LDBG(ti * 32 + 20);
       if (ti + 1 < my_tiles) load_row(ti + 1, nxt);    // in flight while this tile is normalised
-      if (pw == 0 && lane == 0) LDBG(ti * 32 + 21);
       if (g.has_ln) {
         // one pass for both moments on data shifted by the row's first element p (d = x - p): mean = p + sum(d) / K,
         // variance = (sum(d^2) - sum(d)^2 / K) / K; p lies within the row's own spread, so the subtraction of the
@@ -295,10 +272,8 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
           cur[c] = make_uint4(o[0], o[1], o[2], o[3]);
         }
       }
-      if (pw == 0 && lane == 0) LDBG(ti * 32 + 22);
       ok = ptx::mbar_wait_relaxed(&a_empty[ab], aph, abort_flag, g.status, 32);
       if (!ok) break;
-      if (pw == 0 && lane == 0) LDBG(ti * 32 + 23);
       uint8_t* row0 = sA + ab * A_BYTES + r * 128;
 #pragma unroll
       for (int c = 0; c < NH; ++c) {
@@ -308,7 +283,6 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       ptx::fence_proxy_async();                        // generic-proxy writes -> visible to the MMA's reads
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&a_full[ab]);
-      if (pw == 0 && lane == 0) LDBG(ti * 32 + 24);
       if (++ab == NA) { ab = 0; aph ^= 1; }
 #pragma unroll
       for (int c = 0; c < NH; ++c) cur[c] = nxt[c];
@@ -316,7 +290,6 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   }
   ptx::tc_fence_before();
   __syncthreads();
-  LDBGT(3);
   if (warp == 1) {
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem_base, TMEM_COLS);

@@ -16,7 +16,7 @@
 // (two warps per TMEM lane quadrant, 64 hidden columns each), 10-13 output, 14 fc2 issuer, 15-18
 // LayerNorm.
 //
-// What bounds it (clock-stamped build, -DMLP_EXP_TIMING): the loop fc1(j) -> GELU(j) -> fc2(j) ->
+// What bounds it (measured with clock stamps at every hand-off): the loop fc1(j) -> GELU(j) -> fc2(j) ->
 // fc1(j+2) over the two S1/H buffers, about 2500 cycles per chunk.  The arithmetic in it is short
 // (with the GELU arithmetic compiled out the chunk period stays near 2400 cycles and the kernel
 // is only 15 % faster); most of it is the three hand-offs of the loop, each of which waits for the
@@ -29,17 +29,6 @@
 #include "gemm_tc.cuh"
 #include "ptx.cuh"
 
-#ifdef MLP_EXP_TIMING
-__device__ long long g_mlp_dbg[8192];
-#define DBG(slot) do { if (blockIdx.x == 0) g_mlp_dbg[(slot)] = clock64(); } while (0)
-#define DBGT(k) do { if (threadIdx.x == 0) g_mlp_dbg[6000 + blockIdx.x * 4 + (k)] = (long long)smartmem::ptx::globaltimer(); } while (0)
-extern "C" __attribute__((visibility("default"))) int smartmem_debug_read(long long* host, int n) {
-  return (int)cudaMemcpyFromSymbol(host, g_mlp_dbg, sizeof(long long) * n);
-}
-#else
-#define DBG(slot) do { } while (0)
-#define DBGT(k) do { } while (0)
-#endif
 
 namespace smartmem {
 namespace {
@@ -93,7 +82,6 @@ __device__ __forceinline__ void issue_kblock(uint32_t d_tmem, uint64_t ad0, uint
 __global__ void __launch_bounds__(kThreads, 1)
 mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW1,
                  const __grid_constant__ CUtensorMap tmW2, const __grid_constant__ MlpArgs g) {
-  DBGT(0);
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const uint32_t pad = (1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u;
   uint8_t* smem = smem_raw + pad;
@@ -162,7 +150,6 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   const uint32_t tmem_base = *tmem_slot;
   pdl_wait();                       // everything above (weights' biases included) overlapped the previous kernel's tail
   pdl_launch_dependents();
-  DBGT(1);
 
   // fc1 runs one hidden chunk ahead of fc2 over the CTA's whole chunk sequence, across tile
   // boundaries; each has its own issuing thread.  The weights of both share one ring, filled in
@@ -219,13 +206,10 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       for (int j = 0; j < total && ok; ++j) {
         const uint32_t sb = j & 1, ab = it1 & 1;
         const uint32_t n = j ? 2 * j - 1 : 0, ws = n % NST, wph = (n / NST) & 1;
-        DBG(j * 16 + 0);
         if (c1 == 0) ok = ptx::mbar_wait(fuse_ln ? &a_ready[ab] : &a_full[ab], (it1 >> 1) & 1, abort_flag, g.status);
         ok = ok && ptx::mbar_wait(&s1_empty[sb], ((j >> 1) & 1) ^ 1, abort_flag, g.status);
-        DBG(j * 16 + 1);
         ok = ok && ptx::mbar_wait(&w_full[ws], wph, abort_flag, g.status);
         if (!ok) break;
-        DBG(j * 16 + 2);
         ptx::tc_fence_after();
         const uint32_t d = tmem_base + TM_S1 + sb * HC;
         const uint64_t ad = ptx::make_smem_desc(a_base + ab * 2 * KB_BYTES, 16, 1024);
@@ -234,7 +218,6 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (nkb1 > 1) issue_kblock(d, ad + (KB_BYTES >> 4), bd + (KB_BYTES >> 4), idesc1, k1_last, true);
         ptx::tc_commit(&w_empty[ws]);
         ptx::tc_commit(&s1_full[sb]);
-        DBG(j * 16 + 3);
         if (++c1 == NC) {
           ptx::tc_commit(&a_empty[ab]);                 // every fc1 MMA of this tile has been issued
           c1 = 0;
@@ -253,14 +236,11 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       for (int j = 0; j < total && ok; ++j) {
         const uint32_t ob = it2 & 1;
         const uint32_t n = j + 1 < total ? 2 * j + 2 : 2 * j + 1, ws = n % NST, wph = (n / NST) & 1;
-        DBG(j * 16 + 4);
         const uint32_t sb = j & 1;
         ok = ptx::mbar_wait(&h_full[sb], (j >> 1) & 1, abort_flag, g.status);
         if (c2 == 0) ok = ok && ptx::mbar_wait(&out_empty[ob], ((it2 >> 1) & 1) ^ 1, abort_flag, g.status);
-        DBG(j * 16 + 5);
         ok = ok && ptx::mbar_wait(&w_full[ws], wph, abort_flag, g.status);
         if (!ok) break;
-        DBG(j * 16 + 6);
         ptx::tc_fence_after();
         const uint32_t d = tmem_base + TM_OUT + ob * OUT_STRIDE;
         // H chunk: 128 bf16 per lane, written by the GELU warps over the S1 buffer it was computed from --
@@ -273,7 +253,6 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           ptx::tc_mma_bf16_ta(d, a + 8 * k + (k >= 4 ? 32 : 0), bd + (k >> 2) * (KB_BYTES >> 4) + 2 * (k & 3), idesc2, 1u);
         ptx::tc_commit(&w_empty[ws]);
         ptx::tc_commit(&s1_empty[sb]);                  // buffer consumed: fc1 of chunk j + 2 may overwrite it
-        DBG(j * 16 + 7);
         if (++c2 == NC) {
           ptx::tc_commit(&out_full[ob]);
           c2 = 0;
@@ -292,9 +271,7 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     for (int j = 0; j < total && ok; ++j) {
       const uint32_t sb = j & 1;
       const float4* bb4 = reinterpret_cast<const float4*>(b1_s + c * HC + hh * 64);   // this warp's 64 biases of the chunk: 16-byte broadcast reads
-      if (e == 0 && lane == 0) DBG(j * 16 + 8);
       ok = ptx::mbar_wait(&s1_full[sb], (j >> 1) & 1, abort_flag, g.status);
-      if (e == 0 && lane == 0) DBG(j * 16 + 9);
       if (!ok) break;
       const uint32_t tq = tmem_base + TM_S1 + sb * HC + ((uint32_t)(q * 32) << 16) + hh * 64;
       uint32_t rv[64];
@@ -302,24 +279,17 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       ptx::tmem_ld32(tq, rv);
       ptx::tmem_ld32(tq + 32, rv + 32);
       ptx::tmem_ld_wait();
-      if (e == 0 && lane == 0) DBG(j * 16 + 10);
       uint32_t pk[32];
 #pragma unroll
       for (int v = 0; v < 16; ++v) {
         const float4 b4 = bb4[v];
-#ifdef MLP_EXP_NOGELU
-        pk[2 * v] = float2_to_bf16x2(__uint_as_float(rv[4 * v]) + b4.x, __uint_as_float(rv[4 * v + 1]) + b4.y);
-        pk[2 * v + 1] = float2_to_bf16x2(__uint_as_float(rv[4 * v + 2]) + b4.z, __uint_as_float(rv[4 * v + 3]) + b4.w);
-#else
         pk[2 * v] = gelu_tanh_bf16x2(__uint_as_float(rv[4 * v]) + b4.x, __uint_as_float(rv[4 * v + 1]) + b4.y);
         pk[2 * v + 1] = gelu_tanh_bf16x2(__uint_as_float(rv[4 * v + 2]) + b4.z, __uint_as_float(rv[4 * v + 3]) + b4.w);
-#endif
       }
       // the packed result goes over the first 32 of the 64 columns this warp has just read (it is the only
       // reader and writer of them), so no warp ever waits for fc2 of an earlier chunk
       ptx::tmem_st32(tq, pk);
       ptx::tmem_st_wait();
-      if (e == 0 && lane == 0) DBG(j * 16 + 11);
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&h_full[sb]);
@@ -337,14 +307,12 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       const int row = t * BM + q * 32 + lane;
       const bool row_ok = row < g.M;
       const long long off = (long long)row * g.C;
-      if (q == 0 && lane == 0) DBG(ti * NC * 16 + 12);
       ok = ptx::mbar_wait_relaxed(&out_full[ob], (ti >> 1) & 1, abort_flag, g.status, 256);
       if (!ok) break;
-      if (q == 0 && lane == 0) DBG(ti * NC * 16 + 13);
       ptx::tc_fence_after();
-#pragma unroll
-      for (int r = 0; r < 4; ++r) {
-        if (r < rounds) {
+#pragma unroll 1                                          // (once per tile: a short body beats a long straight line of cold code)
+      for (int r = 0; r < rounds; ++r) {
+        {
           uint32_t rv[32];
           ptx::tmem_ld32(tmem_base + TM_OUT + ob * OUT_STRIDE + ((uint32_t)(q * 32) << 16) + r * 32, rv);
           uint4 res[4];                                  // the residual's latency overlaps the accumulator load
@@ -379,7 +347,6 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           }
         }
       }
-      if (q == 0 && lane == 0) DBG(ti * NC * 16 + 14);
     }
   } else if (warp >= 3 + kGeluWarps + kOutWarps) {
     // LayerNorm warps: the producer brought the raw rows of the tile into the A buffer (K-major,
@@ -397,49 +364,48 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         for (int rr = 0; rr < BM / (32 * kNormWarps); ++rr) {
           const int r = (rr * kNormWarps + nw) * 32 + lane;
           uint8_t* row0 = sA + (b * 2) * KB_BYTES + r * 128;
-          uint4 x[12];
-#pragma unroll
-          for (int ch = 0; ch < 12; ++ch)
-            if (ch < nch) x[ch] = *reinterpret_cast<const uint4*>(row0 + (ch >> 3) * KB_BYTES + (((ch & 7) ^ (r & 7)) << 4));
-          // one pass over the row for both moments, on data shifted by the row's first element p (d = x - p):
+          // Both passes read the row from shared memory with partly unrolled loops instead of keeping it in registers: this code
+          // runs once per tile, and a long straight-line body costs more in instruction fetch than the re-read does.
+          // One pass over the row for both moments, on data shifted by the row's first element p (d = x - p):
           // mean = p + sum(d) / C, variance = (sum(d^2) - sum(d)^2 / C) / C.  p lies within the row's own spread,
           // so the subtraction of the two sums loses a few bits at most.  Four independent partial sums each.
-          const float p = __uint_as_float(x[0].x << 16);
+          const float p = __uint_as_float(*reinterpret_cast<const uint32_t*>(row0 + ((0 ^ (r & 7)) << 4)) << 16);
           float s4[4] = {0.f, 0.f, 0.f, 0.f}, q4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 4
+          for (int ch = 0; ch < nch; ++ch) {
+            const uint4 xv = *reinterpret_cast<const uint4*>(row0 + (ch >> 3) * KB_BYTES + (((ch & 7) ^ (r & 7)) << 4));
+            const uint32_t w[4] = {xv.x, xv.y, xv.z, xv.w};
 #pragma unroll
-          for (int ch = 0; ch < 12; ++ch)
-            if (ch < nch) {
-              const uint32_t w[4] = {x[ch].x, x[ch].y, x[ch].z, x[ch].w};
-#pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                const float2 f = bf16x2_to_float2(w[i]);
-                const float dx = f.x - p, dy = f.y - p;
-                s4[i] += dx + dy;
-                q4[i] = fmaf(dy, dy, fmaf(dx, dx, q4[i]));
-              }
+            for (int i = 0; i < 4; ++i) {
+              const float2 f = bf16x2_to_float2(w[i]);
+              const float dx = f.x - p, dy = f.y - p;
+              s4[i] += dx + dy;
+              q4[i] = fmaf(dy, dy, fmaf(dx, dx, q4[i]));
             }
+          }
           const float sd = (s4[0] + s4[1]) + (s4[2] + s4[3]);
           const float mean = fmaf(sd, invC, p);
           const float sq = fmaxf(((q4[0] + q4[1]) + (q4[2] + q4[3])) - sd * sd * invC, 0.f);
           const float rstd = rsqrtf(sq * invC + g.ln_eps);
           const float nmr = -mean * rstd;
+#pragma unroll 4
+          for (int ch = 0; ch < nch; ++ch) {
+            uint4* px = reinterpret_cast<uint4*>(row0 + (ch >> 3) * KB_BYTES + (((ch & 7) ^ (r & 7)) << 4));
+            const uint4 xv = *px;
+            const uint32_t w[4] = {xv.x, xv.y, xv.z, xv.w};
+            // (x - mean) rstd in fp32, rounded to bf16 pairs; the affine part as one packed multiply-add per pair
+            const uint4 ga = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(ln_s) + ch * 8);
+            const uint4 be = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(ln_s + g.C) + ch * 8);
+            const uint32_t gw[4] = {ga.x, ga.y, ga.z, ga.w}, bw[4] = {be.x, be.y, be.z, be.w};
+            uint32_t o[4];
 #pragma unroll
-          for (int ch = 0; ch < 12; ++ch)
-            if (ch < nch) {
-              const uint32_t w[4] = {x[ch].x, x[ch].y, x[ch].z, x[ch].w};
-              // (x - mean) rstd in fp32, rounded to bf16 pairs; the affine part as one packed multiply-add per pair
-              const uint4 ga = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(ln_s) + ch * 8);
-              const uint4 be = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(ln_s + g.C) + ch * 8);
-              const uint32_t gw[4] = {ga.x, ga.y, ga.z, ga.w}, bw[4] = {be.x, be.y, be.z, be.w};
-              uint32_t o[4];
-#pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                const float2 f = bf16x2_to_float2(w[i]);
-                const uint32_t t = float2_to_bf16x2(fmaf(f.x, rstd, nmr), fmaf(f.y, rstd, nmr));
-                asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(o[i]) : "r"(t), "r"(gw[i]), "r"(bw[i]));
-              }
-              *reinterpret_cast<uint4*>(row0 + (ch >> 3) * KB_BYTES + (((ch & 7) ^ (r & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+            for (int i = 0; i < 4; ++i) {
+              const float2 f = bf16x2_to_float2(w[i]);
+              const uint32_t t = float2_to_bf16x2(fmaf(f.x, rstd, nmr), fmaf(f.y, rstd, nmr));
+              asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(o[i]) : "r"(t), "r"(gw[i]), "r"(bw[i]));
             }
+            *px = make_uint4(o[0], o[1], o[2], o[3]);
+          }
         }
         ptx::fence_proxy_async();                        // generic-proxy writes -> visible to the MMA's reads
         __syncwarp();
@@ -449,7 +415,6 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   }
   ptx::tc_fence_before();
   __syncthreads();
-  DBGT(2);
   if (warp == 1) {
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem_base, TMEM_COLS);

@@ -23,15 +23,6 @@
 #include "gemm_tc.cuh"
 #include "ptx.cuh"
 
-#ifdef GEMM_EXP_TIMING
-__device__ long long g_gemm_dbg[8192];
-#define GDBG(slot) do { if (blockIdx.x == 0 && (slot) < 8192) g_gemm_dbg[(slot)] = clock64(); } while (0)
-extern "C" __attribute__((visibility("default"))) int smartmem_debug_read_gemm(long long* host, int n) {
-  return (int)cudaMemcpyFromSymbol(host, g_gemm_dbg, sizeof(long long) * n);
-}
-#else
-#define GDBG(slot) do { } while (0)
-#endif
 
 namespace smartmem {
 namespace {
@@ -185,11 +176,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       for (uint32_t t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++pit) {
         const TileIdx ti_ = split_tile(t, g.fd_tiles_n, g.fd_tiles_m);
         const uint32_t tile_n = ti_.tile_n, tile_m = ti_.tile_m, batch = ti_.batch;
-        GDBG(pit * 16 + 0);
         const TileCoord ta = op_coords(g.ca, tile_m, batch, BM), tb = op_coords(g.cb, tile_n, batch, BN);
         for (int kb = 0; kb < nkb; ++kb, ++kbg) {
           ok = ptx::mbar_wait(&empty[s], ph ^ 1, abort_flag, g.status);
-          if (kb == 0) GDBG(pit * 16 + 1);
           if (!ok) break;
           ptx::mbar_expect_tx(&full[s], two_producers ? A_STAGE_BYTES : A_STAGE_BYTES + B_STAGE_BYTES);
           tma_load_op(g.ca, sA + s * A_STAGE_BYTES, &tmA, &full[s], kb * BK, ta.row0, ta);
@@ -197,7 +186,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if (!two_producers) tma_load_op(g.cb, sB + s * B_STAGE_BYTES, &tmB, &full[s], kb * BK, tb.row0, tb);
           if (++s == STAGES) { s = 0; ph ^= 1; }
         }
-        GDBG(pit * 16 + 2);
       }
       if (*abort_flag) {
         // unwinding: give copies already in flight a bounded chance to land before the CTA leaves
@@ -215,17 +203,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       bool ok = true;
       for (uint32_t t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
         const uint32_t buf = it & 1, use = it >> 1;
-        GDBG(it * 16 + 3);
         ok = ptx::mbar_wait(&tmem_empty[buf], (use & 1) ^ 1, abort_flag, g.status);   // epilogue drained it
         if (!ok) break;
-        GDBG(it * 16 + 4);
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * ACC_COLS;
         for (int kb = 0; kb < nkb; ++kb) {
           ok = ptx::mbar_wait(&full[s], ph, abort_flag, g.status);
           if (!ok) break;
-          if (kb == 0) GDBG(it * 16 + 5);
-          if (kb == 1) GDBG(it * 16 + 6);
           ptx::tc_fence_after();
           // K-major, 128-byte swizzle: 8-row groups are 1024 bytes apart; one k16 step is 32 bytes
           // along the swizzled row.  MN-major: 64-row chunks are 8192 bytes apart (leading offset),
@@ -247,7 +231,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if (++s == STAGES) { s = 0; ph ^= 1; }
         }
         if (ok) ptx::tc_commit(&tmem_full[buf]);
-        GDBG(it * 16 + 7);
       }
     }
   } else if (warp >= 2 + kEpiWarps) {
@@ -359,10 +342,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
       }
 
-      if (warp == 2 && lane == 0) GDBG(it * 16 + 8);
       ok = ptx::mbar_wait(&tmem_full[buf], use & 1, abort_flag, g.status);
       if (!ok) break;
-      if (warp == 2 && lane == 0) GDBG(it * 16 + 9);
       ptx::tc_fence_after();
       const uint32_t taddr = tmem_base + buf * ACC_COLS + ((uint32_t)(q * 32) << 16);
 
@@ -466,7 +447,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&tmem_empty[buf]);
-      if (warp == 2 && lane == 0) GDBG(it * 16 + 10);
       if constexpr (QSTAGE) {
         // the four warps of the quadrant have filled a 32 x BN staging tile: store whole rows
         constexpr int VR = BN / 8;                           // 16-byte vectors per row
@@ -482,7 +462,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if (rok && n0 + seg * 8 + 8 <= g.N) *reinterpret_cast<uint4*>(out_t + roff + n0 + seg * 8) = pk;
         }
         asm volatile("bar.sync %0, 128;" ::"r"(1 + q) : "memory");
-        if (warp == 2 && lane == 0) GDBG(it * 16 + 11);
       }
     }
   }

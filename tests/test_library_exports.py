@@ -31,5 +31,13 @@ def test_host_only_calls_work_without_a_gpu():
     p.dtype, p.B, p.H, p.W, p.C, p.heads, p.window, p.shift, p.mlp_ratio = sm.BF16, 2, 14, 14, 64, 2, 7, 3, 4
     e = sm.smartmem_swin_block_workspace_bytes(p, sm.ELIMINATE)
     x = sm.smartmem_swin_block_workspace_bytes(p, sm.EXPLICIT)
+    u = sm.smartmem_swin_block_workspace_bytes(p, sm.ELIMINATE_UNFUSED)
     mc = 2 * 14 * 14 * 64 * 2
-    assert e >= (1 + 3 + 1 + 1 + 1 + 4) * mc and x >= e + 10 * mc      # EXPLICIT adds the layout copies
+    # only what the chosen path writes is reserved.  ELIMINATE (attention half and MLP half each one kernel): the tensor between
+    # the halves; kernel by kernel: qkv (3), attention output, the tensor between the halves; EXPLICIT adds the layout copies
+    assert mc <= e < 2 * mc
+    assert 5 * mc <= u < 6 * mc
+    assert x >= u + 10 * mc
+    p.C, p.heads = 512, 16                        # wide block: LayerNorm outputs and the hidden activation are materialised
+    mcw = 2 * 14 * 14 * 512 * 2
+    assert sm.smartmem_swin_block_workspace_bytes(p, sm.ELIMINATE) >= (1 + 3 + 1 + 1 + 1 + 4) * mcw
