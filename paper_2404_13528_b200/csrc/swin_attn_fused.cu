@@ -6,8 +6,8 @@
 // reverse and the reverse shift are all index arithmetic here: rows of x are gathered through the
 // composed shift o partition map straight into the MMA operand layout, q / k / v and the attention
 // output never leave the SM, and the result rows are scattered through the same map.  Per token the
-// kernel reads C (twice: once for the operand tile, once more -- from L2 -- for the residual) and writes C
-// elements of global memory; the three-kernel form of the same chain moves 11 C through HBM.
+// kernel reads C and writes C elements of global memory; the three-kernel form of the same chain
+// moves 11 C through HBM.
 //
 // Unit of work: a pair of windows = one 128-row MMA tile (window w of the pair in rows 64 w .. 64 w + T - 1,
 // the rows between T and 64 stay zero), taken round-robin by persistent CTAs that keep every weight resident.
@@ -25,7 +25,9 @@
 //   Ob   = bf16(O / rowsum)                    back into tensor memory as packed pairs
 //   Y   += Ob Wp[:, 32 h : 32 h + 32]^T        128 x C x 32: the head merge is the accumulation over heads
 //
-// and per unit  y_row = Y + b_proj + x_row, stored with 16-byte vectors at the row's offset under the map.
+// and per unit  Y starts as X I (the unit's raw rows times the identity: the residual rides on the tensor core, exactly, since
+// every product is a bf16 value times one), the heads' projections accumulate on top, and the epilogue stores
+// y_row = Y + b_proj with 16-byte vectors at the row's offset under the map.
 //
 // LayerNorm without a normalised tile:  LN(x) W^T + b = rstd (x W'^T - mean c + sigma b'),  W' = bf16(gamma . W) (column
 // scaling), c_n = sum_k W'_nk, b'_n = b_n + sum_k beta_k W_nk, sigma = 1 / rstd.  c is summed from the ROUNDED W', so the
@@ -33,28 +35,28 @@
 // rank-one terms ride on the tensor core as one extra k-step: row r of the operand carries (-mean_r, sigma_r), column n of the
 // weights (c_n, b'_n), each fp32 value split into three bf16 pieces (the six largest cross products of the pieces are kept:
 // exact to 2^-24), so the epilogue of the QKV product is one multiply per element.  Every CTA folds gamma into its resident
-// copy of the weights once (prologue); the row statistics are two passes over the row in registers, fp32.
+// copy of the weights once (prologue); the row statistics are two passes over the row, fp32.
 //
-// Warp roles (8 + 4 heads warps): 0-3 bring in the rows of the units ahead -- a window that does not straddle the seam of the
-// shifted image is an affine box [32 channels, ws, ws] of x per k-block, one TMA copy each; a seam window is gathered row by
-// row with 16-byte asynchronous copies through the index map --; then one group of four warps per head (q/k/v epilogue,
-// softmax, O epilogue: one row of the pair tile per thread; each group issues its own MMAs from one elected thread right
-// after the group's barrier, so a hand-off costs a barrier and not a trip through another warp); the last four warps take
-// the row statistics of the units ahead and run the Y epilogue.  Every wait is bounded.
+// Warp roles (9 + 4 heads warps):
+//   0-3   bring in the rows of the units ahead -- a window that does not straddle the seam of the shifted image is an affine
+//         box [32 channels, ws, ws] of x per k-block, one TMA copy each; a seam window is gathered row by row with 16-byte
+//         asynchronous copies through the index map -- and take their statistics, a thread per row;
+//   then  one group of four warps per head (q/k/v epilogue, softmax, O epilogue: one row of the pair tile per thread).  A
+//         group issues its own S and P V products from an elected thread right after the group's barrier: those hand-offs
+//         are on the item's critical path, and a barrier is cheaper than a trip through another warp;
+//   then  four warps for the Y epilogue (one row per thread);
+//   last  one thread that issues, in item order, the products that have slack: QKV of the items ahead (into the buffer the
+//         item four before has left), the residual product that opens a unit's Y, and the heads' projections.  Issue order is
+//         accumulation order, and orders a buffer's next accumulator behind the projection that reads the buffer last.
+// What bounds it (clock stamps at every hand-off, and builds with the arithmetic of one role removed): not arithmetic -- with
+// the whole softmax compiled out the kernel is 5 % faster -- but the chain of hand-offs of an item (tensor-memory round trips,
+// three barriers, two waits for small products behind other groups' products in the tensor pipe), about 9000 cycles per item
+// with three items in flight; and instruction fetch: code that runs once per unit (statistics, epilogue, the prologue) is
+// kept in rolled loops because its straight-line form ran at the speed of the instruction cache misses.  Every wait is bounded.
 #include "attn.cuh"
 #include "gemm_tc.cuh"
 #include "ptx.cuh"
 
-#ifdef FUSED_TIMING
-__device__ long long g_fused_dbg[8192];
-#define FDBG(slot) do { if ((slot) >= 8000) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_fused_dbg[7000 + blockIdx.x * 4 + ((slot) - 8000)] = (long long)t_; } \
-                         if (blockIdx.x == 0) g_fused_dbg[(slot) >= 8000 ? (slot) - 8000 + 6990 : (slot)] = clock64(); } while (0)
-extern "C" __attribute__((visibility("default"))) int smartmem_debug_read_fused(long long* host, int n) {
-  return (int)cudaMemcpyFromSymbol(host, g_fused_dbg, sizeof(long long) * n);
-}
-#else
-#define FDBG(slot) do { } while (0)
-#endif
 
 namespace smartmem {
 namespace {
@@ -71,6 +73,7 @@ constexpr int WQ_TILE = WROWS * 64;
 constexpr int WX_TILE = WROWS * 32;                 // the extra k-step of a head's weights
 constexpr int KV_SLOT = 2 * KBT;                    // k, v tiles of one item
 constexpr int NBUF = 4, BUF_COLS = 96;              // item buffers of tensor memory
+constexpr int ID_BYTES = 32 * 64;                   // the identity tile
 constexpr int NRING = 4;                            // units whose row offsets are kept (a unit's epilogue runs long after its gather)
 constexpr int kLoaderThreads = 128;
 constexpr uint32_t TMEM_COLS = 512;
@@ -165,8 +168,8 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
   uint8_t* sWp = sWq + NH * NH * WQ_TILE;                          // [NH heads][C rows x 64 B]
   uint8_t* sAx = sWp + NH * WP_TILE;                               // [na][128 rows x 32 B]
   uint8_t* sWx = sAx + na * AX_BYTES;                              // [NH heads][96 rows x 32 B]
-  uint8_t* sId = sWx + NH * WX_TILE;                               // [NH k-blocks][C rows x 64 B]: the identity (the residual rides on the tensor core)
-  uint32_t* bias_s = reinterpret_cast<uint32_t*>(sId + NH * WP_TILE);   // [NH][T][BR]: bf16 pairs
+  uint8_t* sId = sWx + NH * WX_TILE;                               // [32 rows x 64 B]: the 32 x 32 identity (the residual rides on the tensor core)
+  uint32_t* bias_s = reinterpret_cast<uint32_t*>(sId + ID_BYTES);  // [NH][T][BR]: bf16 pairs
   float* bp_s = reinterpret_cast<float*>(bias_s + NH * T * BR);    // [C]
   float* rstd_s = bp_s + C;                                        // [na][128]
   uint32_t* rowoff_s = reinterpret_cast<uint32_t*>(rstd_s + na * BM);   // [NRING][128]: row offset in 16-byte units
@@ -192,7 +195,6 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
   }
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
-  if (tid == 0) FDBG(8000);
   const int cidx = blockIdx.x, cstride = gridDim.x;
   const int U = cidx < g.n_pairs ? (g.n_pairs - cidx + cstride - 1) / cstride : 0;   // units of this CTA
   const int total = U * NH;                                                         // items
@@ -234,7 +236,6 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
     for (int h = 0; h < NH; ++h) ptx::tma_load_2d(sWp + h * WP_TILE, &tmWp, w_full, h * D, 0);
   }
   if (warp == 0) ptx::tmem_alloc(tmem_slot, TMEM_COLS);
-  if (tid == 0) FDBG(6900);
   // parameter-only tables
   const int n_table = (2 * ws - 1) * (2 * ws - 1);
   for (int i = tid; i < NH * 256; i += kThreads) {
@@ -257,14 +258,12 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
   }
   for (int i = tid; i < na * A_BYTES / 16; i += kThreads) reinterpret_cast<uint4*>(sA)[i] = make_uint4(0, 0, 0, 0);
   for (int i = tid; i < na * AX_BYTES / 16; i += kThreads) reinterpret_cast<uint4*>(sAx)[i] = make_uint4(0, 0, 0, 0);
-  for (int i = tid; i < NH * WP_TILE / 16; i += kThreads) reinterpret_cast<uint4*>(sId)[i] = make_uint4(0, 0, 0, 0);
+  for (int i = tid; i < ID_BYTES / 16; i += kThreads) reinterpret_cast<uint4*>(sId)[i] = make_uint4(0, 0, 0, 0);
   for (int i = tid; i < na * BM; i += kThreads) rstd_s[i] = 0.f;
   for (int i = tid; i < NRING * BM; i += kThreads) rowoff_s[i] = ROW_INVALID;
-  if (tid == 0) FDBG(6901);
   __syncthreads();
-  if (tid == 0) FDBG(6902);
-  if (tid < C)                                        // identity: row n of k-block n / 32 has a one in column n
-    *reinterpret_cast<uint16_t*>(sId + (tid >> 5) * WP_TILE + sw64_off(tid, (tid & 31) >> 3) + (tid & 7) * 2) = 0x3F80u;
+  if (tid < 32)                                       // identity: row n has a one in column n
+    *reinterpret_cast<uint16_t*>(sId + sw64_off(tid, tid >> 3) + (tid & 7) * 2) = 0x3F80u;
   // each head's bias as a [T, T] table of bf16 pairs, -inf for the padded keys; a task = a quarter of a row
   for (int task = tid; task < NH * T * 4; task += kThreads) {
     const int hr = task >> 2, qtr = task & 3;                       // (head, row), quarter of the row's key pairs
@@ -297,9 +296,7 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
     if (lane == 0) { kmask_s[0] = m0; kmask_s[1] = m1; kmask_s[2] = m2; kmask_s[3] = m3; }
   }
   // fold gamma into the resident QKV weights; the column terms c_n and b'_n go into the extra k-step (thread = one weight row)
-  if (tid == 0) FDBG(6903);
   const bool w_ok = ptx::mbar_wait(w_full, 0, abort_flag, g.status);
-  if (tid == 0) FDBG(6904);
   if (w_ok && tid < 2 * NH * WROWS) {                  // (whole warps: 2 * NH * 96 is a multiple of 32)
     const int row = tid >> 1, half = tid & 1;          // two threads per weight row: the first and second half of its chunks
     const int h = row / WROWS, rr = row - h * WROWS;
@@ -346,10 +343,8 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  if (tid == 0) FDBG(8001);
   pdl_wait();                                         // everything above depends on parameters only
   pdl_launch_dependents();
-  if (tid == 0) FDBG(8002);
 
   if (warp < 4) {
     // ---- rows of the units ahead -> the operand layout in shared memory ------------------------------------------------------
@@ -434,7 +429,6 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
     };
     auto statistics = [&](int ul) {
       const int ab = ul % na;
-      if (lt == 0) FDBG(4096 + ul * 8 + 3);
       const int r = lt, i = lt & 63;
       if (i < T) {
         float rstd = 0.f;
@@ -480,7 +474,6 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
       ptx::fence_proxy_async();                        // the extra k-step -> visible to the MMAs
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&a_full[ab]);
-      if (lt == 0) FDBG(4096 + ul * 8 + 4);
     };
     // A unit's rows are requested as soon as its ring slot is free (the QKV products of the unit that held it are done); when
     // no slot is free the oldest request in flight is waited for and handed to the statistics warps.
@@ -498,9 +491,7 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
           ready = vote(ptx::mbar_test(bar, par), true);
         }
         if (ready) {
-          if (lt == 0) FDBG(4096 + issued * 8 + 0);
           issue_loads(issued);
-          if (lt == 0) FDBG(4096 + issued * 8 + 1);
           ++issued;
           continue;
         }
@@ -515,7 +506,6 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
       // every row of the unit is in (the loader warps' copies and the TMA boxes): its statistics, a thread per row
       ok = ptx::mbar_wait_relaxed(&landed[done % na], (done / na) & 1, abort_flag, g.status, 32);
       if (vote(!ok, false)) break;
-      if (lt == 0) FDBG(4096 + done * 8 + 2);
       statistics(done);
       ++done;
     }
@@ -553,10 +543,8 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
       const int ab = ul % na;
       const uint32_t tb = tmem_base + (it & (NBUF - 1)) * BUF_COLS + lane_addr;
       // -- q, k, v of this row: rstd times the accumulator (the mean and bias terms rode on the extra k-step) --
-      if (elected) FDBG(it * 16 + 0);
       ok = ok && GWAIT(&a_full[ab], (ul / na) & 1) &&     // (long complete: orders the read of rstd)
            GWAIT(&acc_full[it & (NBUF - 1)], (it >> 2) & 1);
-      if (elected) FDBG(it * 16 + 1);
       if (ok) {
         if (elected) ptx::mbar_arrive(&a_free[ab]);      // this head's product has read the unit's rows
         ptx::tc_fence_after();
@@ -573,7 +561,6 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
         };
         ptx::tmem_ld32(tb, rv);                          // q
         ptx::tmem_ld_wait();
-        if (elected) FDBG(it * 16 + 7);
         scaled_pairs(q16);
 #pragma unroll
         for (int kv = 0; kv < 2; ++kv) {                 // k, v -> this group's operand tiles
@@ -593,13 +580,10 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
           rv[c] = w ? 0u : q16[c];
           rv[16 + c] = w ? q16[c] : 0u;
         }
-        if (elected) FDBG(it * 16 + 8);
         ptx::tmem_st32(tb + 64, rv);
         ptx::tmem_st_wait();
-        if (elected) FDBG(it * 16 + 9);
         ptx::fence_proxy_async();                      // generic-proxy writes -> visible to the MMAs
         ptx::tc_fence_before();
-        if (elected) FDBG(it * 16 + 10);
       }
       if (group_sync()) break;
       if (elected) {
@@ -613,7 +597,6 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
         ptx::tc_mma_bf16_ta(d, qa + 16, kd1, idesc, 1u);
         ptx::tc_mma_bf16_ta(d, qa + 24, kd1 + 2, idesc, 1u);
         ptx::tc_commit(&s_full[gi]);
-        FDBG(it * 16 + 2);
       }
       // -- seam mask of this row's window (shifted blocks: windows in the last window row or column) --
       const int n = 2 * (cidx + ul * cstride) + w;
@@ -629,7 +612,6 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
       }
       // -- softmax of this row over its window's keys --
       ok = GWAIT(&s_full[gi], ul & 1);
-      if (elected) FDBG(it * 16 + 3);
       float inv = 0.f;
       if (ok) {
         ptx::tc_fence_after();
@@ -642,7 +624,6 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
           ptx::tmem_ld8(tb + 48, rv + 48);
         }
         ptx::tmem_ld_wait();
-        if (elected) FDBG(it * 16 + 11);
         float sc[KC];
         float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
@@ -685,7 +666,6 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
         ptx::unpack2(sum2[0], s0, s1);
         ptx::unpack2(sum2[1], s2, s3);
         inv = 1.f / ((s0 + s1) + (s2 + s3));
-        if (elected && inv > 0.f) FDBG(it * 16 + 12);
         // P row (bf16 pairs) over the score columns: this window's keys at packed columns 32 w .. 32 w + 31, zeros for the
         // other window's keys (block-diagonal P against the stacked values)
         ptx::tmem_st32(tb + w * 32, pk);
@@ -694,7 +674,6 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
         ptx::tmem_st32(tb + (1 - w) * 32, pk);
         ptx::tmem_st_wait();
         ptx::tc_fence_before();
-        if (elected) FDBG(it * 16 + 13);
       }
       if (group_sync()) break;
       if (elected) {
@@ -708,11 +687,9 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
 #pragma unroll
         for (int ks = 1; ks < 8; ++ks) ptx::tc_mma_bf16_ta(od, pa + 8 * ks, vd + ks * (1024 >> 4), idesc, 1u);
         ptx::tc_commit(&o_full[gi]);
-        FDBG(it * 16 + 4);
       }
       // -- O row: normalise, bf16 pairs, back into tensor memory as the projection's A operand --
       ok = GWAIT(&o_full[gi], ul & 1);
-      if (elected) FDBG(it * 16 + 5);
       if (ok) {
         ptx::tc_fence_after();
         uint32_t rv[32], ob[16];
@@ -732,7 +709,6 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
       __syncwarp();
       if (!ok) break;
       if (lane == 0) ptx::mbar_arrive(&ob_full[it & (NBUF - 1)]);       // the projection of this item may be issued
-      if (elected) FDBG(it * 16 + 6);
     }
   } else if (warp == 8 + 4 * NH) {
     // ---- the products that have slack -- QKV of the items ahead, the projections -- are issued by a thread of their own, in item
@@ -741,6 +717,7 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
     if (lane == 0 && w_ok) {
       const uint32_t idesc_qkv = ptx::make_idesc_bf16(BM, WROWS, false, false);
       const uint32_t idesc_pj = ptx::make_idesc_bf16(BM, C, false, false);
+      const uint32_t idesc_id = ptx::make_idesc_bf16(BM, D, false, false);
       const uint32_t a_base = ptx::smem_u32(sA), ax_base = ptx::smem_u32(sAx), wq_base = ptx::smem_u32(sWq);
       const uint32_t wx_base = ptx::smem_u32(sWx), wp_base = ptx::smem_u32(sWp);
       int qi = 0, qh = 0, qu = 0, qab = 0, qaph = 0;   // QKV queue: item, head, unit, row-ring slot and its phase
@@ -755,11 +732,12 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
           // Y = X I: the unit's raw rows open the accumulation (the epilogue of the unit before has read Y); exact, since every
           // product is a bf16 value times one.  The product is the last reader of the unit's rows: its completion frees the slot.
           ptx::tc_fence_after();
+          const uint64_t bd = desc_sw64(id_base);
 #pragma unroll
-          for (int kb = 0; kb < NH; ++kb) {
-            const uint64_t ad = desc_sw64(a_base + xab * A_BYTES + kb * KBT), bd = desc_sw64(id_base + kb * WP_TILE);
-            ptx::tc_mma_bf16(tmem_base + TM_Y, ad, bd, idesc_pj, kb ? 1u : 0u);
-            ptx::tc_mma_bf16(tmem_base + TM_Y, ad + 2, bd + 2, idesc_pj, 1u);
+          for (int kb = 0; kb < NH; ++kb) {            // 32 channels at a time: Y[:, 32 kb : 32 kb + 32] = X[:, 32 kb : 32 kb + 32] I_32
+            const uint64_t ad = desc_sw64(a_base + xab * A_BYTES + kb * KBT);
+            ptx::tc_mma_bf16(tmem_base + TM_Y + kb * D, ad, bd, idesc_id, 0u);
+            ptx::tc_mma_bf16(tmem_base + TM_Y + kb * D, ad + 2, bd + 2, idesc_id, 1u);
           }
           ptx::tc_commit(&a_free[xab]);
           ++xu;
@@ -823,7 +801,6 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
     for (int ul = 0; ul < U && ok; ++ul) {
       ok = ptx::mbar_wait_relaxed(y_full, ul & 1, abort_flag, g.status, 32);
       if (!ok) break;
-      if (q == 0 && lane == 0) FDBG(4096 + ul * 8 + 5);
       ptx::tc_fence_after();
       const uint32_t my_off = rowoff_s[(ul % NRING) * BM + r];
       const bool valid = i < T && my_off != ROW_INVALID;
@@ -856,12 +833,10 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
           }
         }
       }
-      if (q == 0 && lane == 0) FDBG(4096 + ul * 8 + 6);
     }
   }
   ptx::tc_fence_before();
   __syncthreads();
-  if (tid == 0) FDBG(8003);
   if (warp == 0) {
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem_base, TMEM_COLS);
@@ -874,7 +849,7 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
 static size_t fused_smem_need(int NH, int T, int na) {
   const int C = NH * D, br = T <= 56 ? 28 : 36;
   return (size_t)na * NH * KBT + (size_t)NH * KV_SLOT + (size_t)NH * NH * WQ_TILE + (size_t)NH * C * 64 +
-         (size_t)na * AX_BYTES + (size_t)NH * WX_TILE + (size_t)NH * C * 64 + (size_t)NH * T * br * 4 + (size_t)C * 4 +
+         (size_t)na * AX_BYTES + (size_t)NH * WX_TILE + (size_t)ID_BYTES + (size_t)NH * T * br * 4 + (size_t)C * 4 +
          (size_t)na * BM * 4 + (size_t)NRING * BM * 4 + (size_t)2 * C * 4 + TP * 4 + 16 + TP * 16 + 4 * 16 + 32 + N_BARS * 8 + 16;
 }
 static constexpr size_t kMaxSmem = 232448;
