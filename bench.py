@@ -203,9 +203,9 @@ def _peaks_all():
     return 6650.0, 1590.0, "fallback (earlier measurement on this pool)"
 
 
-def run_other(args):
-    """Times one of the other configurations: K steps per variant, per-kernel CUDA-event durations through
-    smartmem_profile_begin/_end, and the roofline position of every kernel of the ELIMINATE variant."""
+def run_other(args, name, n_steps):
+    """Times one of the other configurations: n_steps steps per variant, per-kernel CUDA-event durations through
+    smartmem_profile_begin/_end, and the roofline position of every kernel of the ELIMINATE variant.  Returns the JSON line."""
     import numpy as np
     import torch
     from paper_2404_13528_b200 import binding as sm
@@ -213,7 +213,13 @@ def run_other(args):
 
     torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
     stream = torch.cuda.current_stream().cuda_stream
-    name = args.workload
+
+    class _A:                                           # (the body below reads its step count from `args`)
+        pass
+    a2 = _A()
+    a2.__dict__.update(vars(args))
+    a2.steps = n_steps
+    args = a2
 
     def dev(a):
         return torch.from_numpy(a.view("int16").copy()).cuda().view(torch.bfloat16)
@@ -292,8 +298,7 @@ def run_other(args):
                                   wss[j].data_ptr(), wsb[mode], stream)
         tokens = M
         wq, wp, w1 = 3 * C * C * 2, C * C * 2, 4 * C * C * 2
-        one = [("ln1_gather_qkv_gemm", 4 * U + wq, 2 * M * C * 3 * C), ("window_attention", 4 * U, 4 * M * 49 * C),
-               ("proj_gemm_scatter_residual", 3 * U + wp, 2 * M * C * C),
+        one = [("attn_half_fused", 2 * U + wq + wp, 2 * M * C * 3 * C + 4 * M * 49 * C + 2 * M * C * C),
                ("mlp_fused_ln2_fc1_gelu_fc2_residual", 2 * U + 2 * w1, 2 * 2 * M * C * 4 * C)]
         model = one + one + [("patch_merge_layernorm_gather", 2 * U, 0),
                              ("patch_merge_linear", U + 2 * C * 4 * C * 2 + U // 2, 2 * (M // 4) * 4 * C * 2 * C)]
@@ -487,7 +492,7 @@ def run_other(args):
         with open(tpath) as f:                               # DRAM bytes per sequence from the committed ncu capture, scaled
             per_seq = json.load(f).get("decode_attention_per_sequence")
         traffic = None if per_seq is None else int(per_seq) * args.sequences
-    print(json.dumps({
+    return ({
         "metric": name + "_tokens_per_s", "value": tokens * args.steps / (ms[sm.ELIMINATE] * 1e-3), "unit": UNIT, "n_gpus": 1,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms[sm.ELIMINATE] / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
@@ -502,7 +507,7 @@ def run_other(args):
         "roofline": {"bound": dom["bound"], "kernel": dom["kernel"], "achieved": dom["achieved"], "unit": dom["unit"],
                      "peak": tf if dom["bound"] == "tensor" else hbm, "frac": dom["frac"], "traffic": traffic, "peak_source": src},
         "kernels": kern,
-    }))
+    })
 
 
 def main():
@@ -510,8 +515,12 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=500)
     ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--repeats", type=int, default=25,
+                    help="the steps-long timed loop is repeated this many times and the median per-step time is reported")
     ap.add_argument("--impl", default="smartmem", choices=["smartmem", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-other-workloads", action="store_true",
+                    help="skip the short runs of the other configurations that the default line carries")
     ap.add_argument("--images", type=int, default=0,
                     help="default workload only: images per step instead of the workload's 32 (batch sweep; 0 = the workload)")
     ap.add_argument("--sequences", type=int, default=64,
@@ -519,18 +528,23 @@ def main():
     ap.add_argument("--workload", default=WORKLOAD["name"],
                     help="swin_t_stage1_block (default, the benchmark line) or one of: " + ", ".join(OTHER_WORKLOADS))
     args = ap.parse_args()
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.gpus != world:
+        raise SystemExit(f"bench.py --gpus {args.gpus} needs {args.gpus} ranks, found WORLD_SIZE={world}: launch it as "
+                         f"`python -m torch.distributed.run --nnodes=1 --nproc-per-node {args.gpus} --master-addr 127.0.0.1 "
+                         f"--master-port <port> bench.py --gpus {args.gpus} ...` (one replica per GPU; the path has no collective)")
     if args.impl == "reference":
         return run_reference(args)
     args.warmup = max(args.warmup, 3)
     if args.workload != WORKLOAD["name"]:
-        return run_other(args)
+        print(json.dumps(run_other(args, args.workload, args.steps)))
+        return
 
     import torch
     from paper_2404_13528_b200 import binding as sm
     from paper_2404_13528_b200 import synth
 
     rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
@@ -553,7 +567,6 @@ def main():
 
     params = {k: dev(v) for k, v in inp.items() if k != "x"}
     x_host = torch.from_numpy(inp["x"].view("int16").copy()).view(torch.bfloat16).pin_memory()
-    y_host = torch.empty_like(x_host).pin_memory()
     p = sm.SwinParams()
     p.dtype = sm.BF16
     p.B, p.H, p.W, p.C, p.heads, p.window, p.shift, p.mlp_ratio = (w["B"], w["H"], w["W"], w["C"], w["heads"], w["window"],
@@ -561,13 +574,16 @@ def main():
     p.ln_eps = 1e-5
     for k, t in params.items():
         setattr(p, k, t.data_ptr())
-    wsb = {m: sm.smartmem_swin_block_workspace_bytes(p, m) for m in (sm.ELIMINATE, sm.EXPLICIT)}
+    MODES = {"eliminate": sm.ELIMINATE, "eliminate_unfused": sm.ELIMINATE_UNFUSED, "explicit": sm.EXPLICIT}
+    wsb = {m: sm.smartmem_swin_block_workspace_bytes(p, m) for m in MODES.values()}
+    U_bytes = x_host.numel() * 2
     global N_SETS
-    if args.images:          # smaller batches: more rotating sets, so that a set is still evicted from L2 before its reuse
-        N_SETS = int(min(64, max(4, -(-1_100_000_000 // (2 * x_host.numel() * 2 + wsb[sm.EXPLICIT])))))
+    # enough rotating sets that the timed variant touches more than 512 MB between reuses of a set (L2 is 126 MB)
+    touched = {m: 2 * U_bytes + wsb[m] for m in MODES.values()}
+    N_SETS = int(min(64, max(4, -(-600_000_000 // touched[sm.ELIMINATE]))))
     xs = [x_host.cuda() for _ in range(N_SETS)]
     ys = [torch.empty_like(xs[0]) for _ in range(N_SETS)]
-    wss = [torch.empty(wsb[sm.EXPLICIT], dtype=torch.uint8, device="cuda") for _ in range(N_SETS)]
+    wss = [torch.empty(max(wsb.values()), dtype=torch.uint8, device="cuda") for _ in range(N_SETS)]
     stream = torch.cuda.current_stream().cuda_stream
 
     def step(i, mode):
@@ -579,33 +595,43 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    def timed(mode, steps):
+    def timed(fn, steps):
+        """EXACTLY `steps` calls between two events, barrier + synchronize on both sides; max over ranks."""
         barrier()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         n0 = sm.smartmem_launch_count()
         e0.record()
         for i in range(steps):
-            step(i, mode)
+            fn(i)
         e1.record()
         barrier()
-        ms = max_over_ranks(dist, e0.elapsed_time(e1), "cuda")
-        launches = sm.smartmem_launch_count() - n0
-        return ms, launches
+        return max_over_ranks(dist, e0.elapsed_time(e1), "cuda"), sm.smartmem_launch_count() - n0
+
+    def timed_median(fn, steps, repeats):
+        runs = [timed(fn, steps) for _ in range(repeats)]
+        ms = sorted(r[0] for r in runs)
+        return statistics.median(ms), ms[0], ms[-1], runs[0][1]
 
     sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ else
                            os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local])
     sampler.start()
     for i in range(args.warmup):
-        step(i, sm.ELIMINATE)
-        step(i, sm.EXPLICIT)
-    ms_elim, launches = timed(sm.ELIMINATE, args.steps)
-    ms_expl, _ = timed(sm.EXPLICIT, args.steps)
+        for m in MODES.values():
+            step(i, m)
+    # the steps-long loop, repeated: the GPU is under load for a few hundred milliseconds and the median is reported
+    tot = {}
+    for tag, m in MODES.items():
+        reps = args.repeats if tag == "eliminate" else max(3, args.repeats // 5)
+        tot[tag] = timed_median(lambda i, m=m: step(i, m), args.steps, reps)
+    ms_elim, ms_elim_min, ms_elim_max, launches = tot["eliminate"]
     st = sm.smartmem_last_device_status(stream)
     if st != sm.OK:
         raise SystemExit(f"device status {st}: {sm.smartmem_status_string(st)}")
 
-    # per-kernel durations (CUDA events recorded on the launching stream around every launch)
-    per = {sm.ELIMINATE: {}, sm.EXPLICIT: {}}
+    # per-kernel durations, two ways.  (1) event-separated: a CUDA event before every launch (the 1 us event tick and the
+    # serialisation of the programmatic early launch are in these); (2) back to back: each half of the eliminated block is
+    # one kernel, launched 16 times between one event pair over the rotating sets, so the tick is amortised
+    per = {m: {} for m in MODES.values()}
     reps = min(args.steps, 30)
     for mode in per:
         for i in range(reps):
@@ -613,47 +639,72 @@ def main():
             for name, ms in sm.smartmem_swin_block_timed(p, xs[j].data_ptr(), ys[j].data_ptr(), wss[j].data_ptr(), wsb[mode],
                                                          mode, stream):
                 per[mode].setdefault(name, []).append(ms)
+    b2b = {}
+    if p.mlp_ratio > 0:
+        for half, label in ((0, "attn_half_fused"), (1, "mlp_fused_ln2_fc1_gelu_fc2_residual")):
+            def half_call(i, half=half):
+                j = i % N_SETS
+                sm.smartmem_swin_block_half(p, xs[j].data_ptr(), ys[j].data_ptr(), wss[j].data_ptr(), wsb[sm.ELIMINATE],
+                                            sm.ELIMINATE, half, stream)
+            for i in range(4):
+                half_call(i)
+            med, lo, hi, _ = timed_median(half_call, 16, 15)
+            b2b[label] = {"ms": med / 16, "ms_min": lo / 16, "ms_max": hi / 16}
     peaks = measured_peaks()
     _, tf_peak, _ = _peaks_all()
     ab, af = algorithmic_bytes(w), algorithmic_flops(w)
     kernels = {}
-    for mode, tag in ((sm.ELIMINATE, "eliminate"), (sm.EXPLICIT, "explicit")):
+    for tag, mode in MODES.items():
         kernels[tag] = []
         for name, v in per[mode].items():
             ms = statistics.median(v)
-            gbs = ab[name] / (ms * 1e-3) / 1e9 if ms > 0 else None
+            ms_roof = b2b[name]["ms"] if (tag == "eliminate" and name in b2b) else ms
+            gbs = ab[name] / (ms_roof * 1e-3) / 1e9 if ms_roof > 0 else None
             fl = af.get(name, 0)
-            tfs = fl / (ms * 1e-3) / 1e12 if ms > 0 else None
+            tfs = fl / (ms_roof * 1e-3) / 1e12 if ms_roof > 0 else None
             # the roofline that binds the kernel: whichever ideal time is longer, bytes at the HBM peak or flops at the tensor peak
             tensor_bound = fl / (tf_peak * 1e12) > ab[name] / (peaks["hbm_gbs"] * 1e9)
-            kernels[tag].append({"kernel": name, "ms": round(ms, 5), "algorithmic_bytes": ab[name], "algorithmic_flops": fl,
-                                 "gbs": gbs and round(gbs, 1), "frac_of_hbm_peak": gbs and round(gbs / peaks["hbm_gbs"], 4),
-                                 "tflops": tfs and round(tfs, 1), "frac_of_tensor_peak": tfs and round(tfs / tf_peak, 4),
-                                 "bound": "tensor" if tensor_bound else "hbm"})
+            k = {"kernel": name, "ms_event_separated": round(ms, 5), "algorithmic_bytes": ab[name], "algorithmic_flops": fl,
+                 "gbs": gbs and round(gbs, 1), "frac_of_hbm_peak": gbs and round(gbs / peaks["hbm_gbs"], 4),
+                 "tflops": tfs and round(tfs, 1), "frac_of_tensor_peak": tfs and round(tfs / tf_peak, 4),
+                 "bound": "tensor" if tensor_bound else "hbm"}
+            if tag == "eliminate" and name in b2b:
+                k["ms_back_to_back"] = round(b2b[name]["ms"], 5)
+                k["fractions_from"] = "ms_back_to_back"
+            k["ms"] = round(ms_roof, 5)
+            kernels[tag].append(k)
     dom = max(kernels["eliminate"], key=lambda k: k["ms"])
+    # what the explicit variant's extra time is made of (event-separated medians)
+    ex = {k["kernel"]: k["ms_event_separated"] for k in kernels["explicit"]}
+    un = {k["kernel"]: k["ms_event_separated"] for k in kernels["eliminate_unfused"]}
+    copies_ms = sum(v for k, v in ex.items() if k.startswith("copy_"))
+    compute_ms = sum(v for k, v in ex.items() if not k.startswith("copy_"))
+    kt_penalty = max(0.0, ex.get("window_attention", 0.0) - un.get("window_attention", 0.0))
+    ms_expl, ms_unf = tot["explicit"][0], tot["eliminate_unfused"][0]
 
     # end to end through the C ABI with host buffers: every step copies its input from pinned host
     # memory and its result back.  Copies and compute run on three streams over the rotating buffer
     # sets, so the PCIe transfers of neighbouring steps overlap the kernels (each step still has
     # its own H2D copy, its own block call and its own D2H copy).
     e2e_steps = min(max(args.steps, 8), 64)
-    y_hosts = [torch.empty_like(x_host).pin_memory() for _ in range(N_SETS)]
+    y_hosts = [torch.empty_like(x_host).pin_memory() for _ in range(min(N_SETS, 8))]
+    NE = len(y_hosts)
     s_in, s_comp, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
-    ev_in = [torch.cuda.Event() for _ in range(N_SETS)]
-    ev_comp = [torch.cuda.Event() for _ in range(N_SETS)]
-    ev_out = [torch.cuda.Event() for _ in range(N_SETS)]
+    ev_in = [torch.cuda.Event() for _ in range(NE)]
+    ev_comp = [torch.cuda.Event() for _ in range(NE)]
+    ev_out = [torch.cuda.Event() for _ in range(NE)]
 
     def e2e_loop(n):
         for i in range(n):
-            j = i % N_SETS
+            j = i % NE
             with torch.cuda.stream(s_in):
-                if i >= N_SETS:
+                if i >= NE:
                     s_in.wait_event(ev_comp[j])             # the block that last read xs[j] is done
                 xs[j].copy_(x_host, non_blocking=True)
                 ev_in[j].record(s_in)
             with torch.cuda.stream(s_comp):
                 s_comp.wait_event(ev_in[j])
-                if i >= N_SETS:
+                if i >= NE:
                     s_comp.wait_event(ev_out[j])            # ys[j] has been read back
                 sm.smartmem_swin_block(p, xs[j].data_ptr(), ys[j].data_ptr(), wss[j].data_ptr(), wsb[sm.ELIMINATE],
                                        sm.ELIMINATE, s_comp.cuda_stream)
@@ -663,7 +714,7 @@ def main():
                 y_hosts[j].copy_(ys[j], non_blocking=True)
                 ev_out[j].record(s_out)
 
-    e2e_loop(N_SETS)
+    e2e_loop(NE)
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     cur = torch.cuda.current_stream()
@@ -678,8 +729,24 @@ def main():
     e1.record(cur)
     barrier()
     ms_e2e = max_over_ranks(dist, e0.elapsed_time(e1), "cuda")
-    y_host = y_hosts[0]
     clocks = sampler.stop()
+    l2_note = (f"{N_SETS} rotating buffer sets; the timed (eliminated) variant touches "
+               f"{N_SETS * touched[sm.ELIMINATE] / 1e6:.0f} MB between reuses of a set, the explicit variant "
+               f"{N_SETS * touched[sm.EXPLICIT] / 1e6:.0f} MB (L2: 126 MB)")
+
+    others = None
+    if rank == 0 and world == 1 and not args.no_other_workloads and not args.images:
+        # the other full-size configurations, a few steps each, so that the one line carries them
+        del xs, ys, wss, y_hosts
+        torch.cuda.empty_cache()
+        others = []
+        for name, k in (("swin_b_stage3_block_pair", 30), ("llama_attention_layer", 20)):
+            r = run_other(args, name, k)
+            others.append({"workload": name, "ms_per_step": r["ms_per_step"], "tokens_per_s": r["value"],
+                           "explicit_ms_per_step": r["explicit_variant"]["ms_per_step"],
+                           "explicit_speedup": r["explicit_variant"]["speedup_of_eliminate"], "steps": k,
+                           "roofline": {kk: r["roofline"][kk] for kk in ("kernel", "bound", "frac", "achieved", "unit")},
+                           "kernels": [{"kernel": q["kernel"], "ms": q["ms"], "bound": q["bound"], "frac": q["frac"]} for q in r["kernels"]]})
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -696,34 +763,50 @@ def main():
     if rank == 0:
         tokens = M * world
         value = whole_job_tokens_per_s(M, world, args.steps, ms_elim)
-        traffic = None
+        traffic, traffic_source = None, None
         tpath = os.path.join(ROOT, "profiles", "traffic.json")      # per-launch DRAM bytes from an ncu capture
         if os.path.exists(tpath):
             with open(tpath) as f:
                 traffic = json.load(f).get(dom["kernel"])
-            if traffic is not None and w["B"] != 32:         # the capture is of the 32-image workload; traffic grows with the images
-                traffic = int(traffic * w["B"] / 32)
+            if traffic is not None:
+                traffic_source = "profiles/traffic.json (ncu dram__bytes_read + dram__bytes_write of one launch of this kernel on this workload)"
+                if w["B"] != 32:                              # the capture is of the 32-image workload; traffic grows with the images
+                    traffic = int(traffic * w["B"] / 32)
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_elim / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
+            "timing": {"timed_loops": args.repeats, "steps_per_loop": args.steps, "statistic": "median over the loops of (loop time / steps)",
+                       "ms_per_step_min": ms_elim_min / args.steps, "ms_per_step_max": ms_elim_max / args.steps},
             "config": {"workload": w["name"], "B_per_gpu": w["B"], "H": w["H"], "W": w["W"], "C": w["C"], "heads": w["heads"],
-                       "window": w["window"], "shift": w["shift"], "mlp_ratio": w["mlp_ratio"], "mode": "eliminate",
-                       "l2": f"{N_SETS} rotating buffer sets ({N_SETS * (2 * x_host.numel() * 2 + wsb[sm.EXPLICIT]) / 1e6:.0f} MB touched between reuses of a set)",
+                       "window": w["window"], "shift": w["shift"], "mlp_ratio": w["mlp_ratio"], "mode": "eliminate", "l2": l2_note,
                        "parallelism": f"replicas x{world}" if world > 1 else "single gpu"},
             "explicit_variant": {"value": tokens * args.steps / (ms_expl * 1e-3), "unit": UNIT,
-                                 "ms_per_step": ms_expl / args.steps, "speedup_of_eliminate": ms_expl / ms_elim},
+                                 "ms_per_step": ms_expl / args.steps, "speedup_of_eliminate": ms_expl / ms_elim,
+                                 # event-separated medians of the explicit chain: its layout copies, its compute kernels, and how much
+                                 # slower its window attention is than the eliminated chain's (its materialised K^T has 98-byte rows,
+                                 # which TMA cannot address, so the operand comes in through the hand loader)
+                                 "copies_ms": round(copies_ms, 5), "compute_ms": round(compute_ms, 5),
+                                 "kt_hand_loader_penalty_ms": round(kt_penalty, 5),
+                                 "speedup_of_eliminate_without_that_penalty": (ms_expl / args.steps - kt_penalty) / (ms_elim / args.steps)},
+            # the eliminated chain kernel by kernel (no fusion of the attention half): elimination alone against the explicit chain
+            "eliminate_unfused_variant": {"ms_per_step": ms_unf / args.steps, "speedup_over_explicit": ms_expl / ms_unf,
+                                          "speedup_over_explicit_without_kt_penalty": (ms_expl / args.steps - kt_penalty) / (ms_unf / args.steps),
+                                          "fused_over_unfused": ms_unf / ms_elim},
             "e2e": {"value": tokens * e2e_steps / (ms_e2e * 1e-3), "unit": UNIT,
-                    "h2d_bytes_per_step": x_host.numel() * 2, "d2h_bytes_per_step": y_host.numel() * 2},
+                    "h2d_bytes_per_step": x_host.numel() * 2, "d2h_bytes_per_step": x_host.numel() * 2},
             "gpu_launches": launches,
             "clocks": clocks,
             "roofline": ({"bound": "tensor", "kernel": dom["kernel"], "achieved": dom["tflops"], "peak": tf_peak,
-                          "unit": "TFLOP/s", "frac": dom["frac_of_tensor_peak"], "traffic": traffic,
-                          "peak_source": peaks["source"] + "; bf16 burst"} if dom["bound"] == "tensor" else
+                          "unit": "TFLOP/s", "frac": dom["frac_of_tensor_peak"], "traffic": traffic, "traffic_source": traffic_source,
+                          "peak_source": peaks["source"] + "; bf16 burst", "duration_ms": dom["ms"]} if dom["bound"] == "tensor" else
                          {"bound": "hbm", "kernel": dom["kernel"], "achieved": dom["gbs"], "peak": peaks["hbm_gbs"],
-                          "unit": "GB/s", "frac": dom["frac_of_hbm_peak"], "traffic": traffic, "peak_source": peaks["source"]}),
+                          "unit": "GB/s", "frac": dom["frac_of_hbm_peak"], "traffic": traffic, "traffic_source": traffic_source,
+                          "peak_source": peaks["source"], "duration_ms": dom["ms"]}),
             "kernels": kernels,
         }
+        if others is not None:
+            out["other_workloads"] = others
         if cpu is not None:
             out["cpu_baseline"] = cpu
         print(json.dumps(out))

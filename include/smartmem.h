@@ -227,6 +227,15 @@ int smartmem_swin_block_workspace_bytes(const smartmem_swin_params_t* p, int32_t
 int smartmem_swin_block(const smartmem_swin_params_t* p, const void* x, void* y, void* workspace,
                         size_t workspace_bytes, int32_t mode, void* cuda_stream);
 
+/* One half of the block on its own (Section 3.2.1's chain splits at the residual between the two halves):
+ * half = 0: y = x + proj(attention(LN1(x)))  (the attention half; what mlp_ratio = 0 computes),
+ * half = 1: y = x + fc2(GELU(fc1(LN2(x))))   (the MLP half; x is an attention half's result; needs mlp_ratio > 0).
+ * Same requirements, modes and workspace size as smartmem_swin_block; running half 0 into a buffer and half 1 from it
+ * gives the block's result bit for bit.  Lets a caller place its own work between the halves, and a benchmark time
+ * each half back to back. */
+int smartmem_swin_block_half(const smartmem_swin_params_t* p, const void* x, void* y, void* workspace,
+                             size_t workspace_bytes, int32_t mode, int32_t half, void* cuda_stream);
+
 /* Measurement aid (no counterpart in the paper): the same block, with a CUDA event recorded on
  * `cuda_stream` before every kernel launch.  Synchronises the stream, then writes the duration of
  * each kernel in milliseconds to kernel_ms[i] (host) and its label, NUL-terminated, to

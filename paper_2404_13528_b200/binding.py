@@ -64,7 +64,7 @@ EXPORTED = [
     "smartmem_op_quadrant", "smartmem_pair_decision", "smartmem_select_layouts", "smartmem_plan", "smartmem_plan_destroy",
     "smartmem_plan_num_steps", "smartmem_plan_get_map", "smartmem_plan_output_desc",
     "smartmem_plan_workspace_bytes", "smartmem_map_eval", "smartmem_plan_eval_sequential", "smartmem_run_chain",
-    "smartmem_swin_block_workspace_bytes", "smartmem_swin_block", "smartmem_attn_layer_workspace_bytes",
+    "smartmem_swin_block_workspace_bytes", "smartmem_swin_block", "smartmem_swin_block_half", "smartmem_attn_layer_workspace_bytes",
     "smartmem_attn_layer", "smartmem_attn_decode_workspace_bytes", "smartmem_attn_decode", "smartmem_swin_block_timed", "smartmem_swin_block_static_scratch_bytes",
     "smartmem_swin_block_noalloc", "smartmem_profile_begin", "smartmem_profile_end", "smartmem_last_device_status", "smartmem_launch_count", "smartmem_status_string",
 ]
@@ -98,6 +98,7 @@ def lib() -> C.CDLL:
         "smartmem_run_chain": (C.c_int, [vp, P(vp), P(vp), vp, C.c_size_t, vp]),
         "smartmem_swin_block_workspace_bytes": (C.c_int, [P(SwinParams), i32, P(C.c_size_t)]),
         "smartmem_swin_block": (C.c_int, [P(SwinParams), vp, vp, vp, C.c_size_t, i32, vp]),
+        "smartmem_swin_block_half": (C.c_int, [P(SwinParams), vp, vp, vp, C.c_size_t, i32, i32, vp]),
         "smartmem_swin_block_timed": (C.c_int, [P(SwinParams), vp, vp, vp, C.c_size_t, i32, vp, P(C.c_float), C.c_char_p,
                                       i32, i32, P(i32)]),
         "smartmem_swin_block_static_scratch_bytes": (C.c_int, [P(C.c_size_t)]),
@@ -251,6 +252,10 @@ def smartmem_swin_block_workspace_bytes(p: SwinParams, mode: int) -> int:
 
 def smartmem_swin_block(p: SwinParams, x: int, y: int, workspace: int, workspace_bytes: int, mode: int, stream: int):
     _check(lib().smartmem_swin_block(C.byref(p), x, y, workspace, workspace_bytes, mode, stream), "smartmem_swin_block")
+
+
+def smartmem_swin_block_half(p: SwinParams, x: int, y: int, workspace: int, workspace_bytes: int, mode: int, half: int, stream: int):
+    _check(lib().smartmem_swin_block_half(C.byref(p), x, y, workspace, workspace_bytes, mode, half, stream), "smartmem_swin_block_half")
 
 
 def smartmem_swin_block_timed(p: SwinParams, x: int, y: int, workspace: int, workspace_bytes: int, mode: int, stream: int):

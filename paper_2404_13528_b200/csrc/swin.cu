@@ -173,10 +173,12 @@ struct KernelTimer {
   }
 };
 
+// half: -1 the whole block, 0 the attention half only, 1 the MLP half only (x is then the attention half's result)
 int run_block(const smartmem_swin_params_t* pp, const void* x, void* y, void* workspace, size_t workspace_bytes,
-              int32_t mode, void* cuda_stream, KernelTimer* tm) {
+              int32_t mode, void* cuda_stream, KernelTimer* tm, int half = -1) {
   int rc = validate(pp, mode);
   if (rc != SMARTMEM_OK) return rc;
+  if (half < -1 || half > 1 || (half == 1 && pp->mlp_ratio == 0)) return SMARTMEM_ERR_INVALID_ARG;
   const smartmem_swin_params_t& p = *pp;
   if (!x || !y || !workspace || x == y) return SMARTMEM_ERR_INVALID_ARG;
   const void* need[] = {p.ln1_g, p.ln1_b, p.w_qkv, p.b_qkv, p.rel_bias_table, p.w_proj, p.b_proj};
@@ -225,7 +227,8 @@ int run_block(const smartmem_swin_params_t* pp, const void* x, void* y, void* wo
     return launch_gemm_tc(tc_operand_plain(A, M, K, K), tc_operand_plain(Wt, N, K, K), ep, 1, M, N, K, st);
   };
 
-  void* y1 = p.mlp_ratio > 0 ? at(L.y1) : y;      // result of the attention half
+  void* y1 = (p.mlp_ratio > 0 && half != 0) ? at(L.y1) : y;      // result of the attention half
+  if (half == 1) y1 = const_cast<void*>(x);
   WinAttnArgs a;
   memset(&a, 0, sizeof(a));
   a.table = p.rel_bias_table; a.table_f32 = f32 ? 1 : 0;
@@ -235,7 +238,9 @@ int run_block(const smartmem_swin_params_t* pp, const void* x, void* y, void* wo
 
   const bool fuse_ln1 = path.fuse_ln1;
 #define SM_TRY(label, expr) do { if (tm) tm->tick(label); rc = (expr); if (rc != SMARTMEM_OK) return rc; } while (0)
-  if (path.fuse_attn) {
+  if (half == 1) {
+    // MLP half only
+  } else if (path.fuse_attn) {
     // narrow blocks: the whole attention half in one kernel (rows gathered and scattered through the composed map)
     SM_TRY("attn_half_fused", launch_swin_attn_fused(p, m.e1_rows, x, y1, st));
   } else if (elim) {
@@ -289,7 +294,7 @@ int run_block(const smartmem_swin_params_t* pp, const void* x, void* y, void* wo
     }
     SM_TRY("proj_gemm_residual", linear(ou, p.w_proj, p.b_proj, y1, C, C, 0, x, nullptr));
   }
-  if (p.mlp_ratio > 0) {
+  if (p.mlp_ratio > 0 && half != 0) {
     if (path.fuse_mlp) {
       // narrow blocks: LN2 + fc1 + GELU + fc2 + residual in one kernel; neither the normalised rows
       // nor the hidden activation leave the chip
@@ -310,6 +315,12 @@ int run_block(const smartmem_swin_params_t* pp, const void* x, void* y, void* wo
 EXPORT int smartmem_swin_block(const smartmem_swin_params_t* p, const void* x, void* y, void* workspace,
                                size_t workspace_bytes, int32_t mode, void* cuda_stream) {
   return run_block(p, x, y, workspace, workspace_bytes, mode, cuda_stream, nullptr);
+}
+
+EXPORT int smartmem_swin_block_half(const smartmem_swin_params_t* p, const void* x, void* y, void* workspace,
+                                    size_t workspace_bytes, int32_t mode, int32_t half, void* cuda_stream) {
+  if (half != 0 && half != 1) return SMARTMEM_ERR_INVALID_ARG;
+  return run_block(p, x, y, workspace, workspace_bytes, mode, cuda_stream, nullptr, half);
 }
 
 EXPORT int smartmem_swin_block_timed(const smartmem_swin_params_t* p, const void* x, void* y, void* workspace,

@@ -45,3 +45,12 @@ def test_two_gloo_ranks_report_the_slowest_time_and_distinct_shards():
     import bench
     assert bench.whole_job_tokens_per_s(100352, 2, 10, 15.0) == 2 * 100352 * 10 / 0.015
     assert bench.max_over_ranks(None, 3.0, "cpu") == 3.0
+
+
+def test_gpus_flag_must_match_the_launched_ranks():
+    """`bench.py --gpus N` started without N ranks refuses (it never silently runs one rank and calls it N)."""
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "8"], capture_output=True, text=True, env=env, timeout=120)
+    assert r.returncode != 0
+    assert "needs 8 ranks" in r.stderr and "torch.distributed.run" in r.stderr

@@ -136,3 +136,34 @@ def test_swin_block_rejects_bad_arguments():
         with pytest.raises(sm.SmartmemError) as e:
             run_block(inp, dev, **{**base, **bad})
         assert e.value.code == code, bad
+
+
+@pytest.mark.parametrize("cfg", [
+    dict(B=2, H=14, W=14, C=96, heads=3, window=7, shift=3, mlp_ratio=4),      # fused halves
+    dict(B=1, H=14, W=14, C=128, heads=4, window=7, shift=3, mlp_ratio=2),     # kernel by kernel
+])
+def test_block_halves_compose_to_the_block(cfg):
+    """smartmem_swin_block_half: the attention half into a buffer, the MLP half from it = the block, bit for bit."""
+    inp = synth.swin_inputs(22, cfg["B"], cfg["H"], cfg["W"], cfg["C"], cfg["heads"], cfg["window"], cfg["mlp_ratio"], "bf16")
+    dev = {k: to_dev(v) for k, v in inp.items()}
+    p = sm.SwinParams()
+    p.dtype = sm.BF16
+    for k, v in cfg.items():
+        setattr(p, k, v)
+    p.ln_eps = 1e-5
+    for n in PARAM_NAMES:
+        setattr(p, n, dev[n].data_ptr())
+    for mode in (sm.ELIMINATE, sm.ELIMINATE_UNFUSED, sm.EXPLICIT):
+        n = sm.smartmem_swin_block_workspace_bytes(p, mode)
+        ws = torch.empty(n, dtype=torch.uint8, device="cuda")
+        whole = torch.full_like(dev["x"], float("nan"))
+        sm.smartmem_swin_block(p, dev["x"].data_ptr(), whole.data_ptr(), ws.data_ptr(), n, mode, stream())
+        mid, out = torch.full_like(whole, float("nan")), torch.full_like(whole, float("nan"))
+        sm.smartmem_swin_block_half(p, dev["x"].data_ptr(), mid.data_ptr(), ws.data_ptr(), n, mode, 0, stream())
+        sm.smartmem_swin_block_half(p, mid.data_ptr(), out.data_ptr(), ws.data_ptr(), n, mode, 1, stream())
+        check_status()
+        assert torch.equal(out, whole), f"mode {mode}"
+        assert not torch.equal(mid, whole)
+    with pytest.raises(sm.SmartmemError) as e:
+        sm.smartmem_swin_block_half(p, dev["x"].data_ptr(), out.data_ptr(), ws.data_ptr(), n, sm.ELIMINATE, 2, stream())
+    assert e.value.code == sm.ERR_INVALID_ARG
