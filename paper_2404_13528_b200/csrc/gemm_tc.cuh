@@ -57,14 +57,14 @@ int tc_encode_nd_sw64(const void* ptr, int rank, const long long* dims, const lo
                       CUtensorMap* out);
 int tc_sm_count();
 
-// Fused MLP: out = residual + (GELU(LN(A) W1^T + b1)) W2^T + b2 with the hidden activation kept on chip.
-// A [M, C], W1 [hidden, C], W2 [C, hidden], C in {64, 96}, hidden a multiple of 128 (at most 512).
-// ln_gamma/ln_beta [C]: LayerNorm (over C, eps inside the square root) applied to the rows of A as
-// the tile arrives in shared memory; both null: A is used as it is.
+// Fused MLP half of a block: out = A + GELU(LN(A) W1^T + b1) W2^T + b2 with the hidden activation and the
+// normalised rows kept on chip.  A [M, C], W1 [hidden, C], W2 [C, hidden], C in {64, 96}, hidden a multiple
+// of 128 with both weight matrices fitting shared memory; ln_gamma/ln_beta [C]: LayerNorm over C, eps inside
+// the square root.  out may not alias A.
 bool mlp_fused_supported(long long C, long long hidden);
 int launch_mlp_fused(const void* A, const void* ln_gamma, const void* ln_beta, float ln_eps, const void* W1, const void* b1,
-                     const void* W2, const void* b2, const void* residual, void* out, long long M, long long C,
-                     long long hidden, cudaStream_t st);
+                     const void* W2, const void* b2, void* out, long long M, long long C, long long hidden,
+                     cudaStream_t st);
 
 // LayerNorm o row-gather o linear for narrow rows: out[m, :] = LN(X[src(m), :]) W^T + bias, with X rows of
 // K in {64, 96} elements, W [N, K], N a multiple of 96 (at most 288).  `rowmap` (null: identity) gives

@@ -299,7 +299,7 @@ int run_block(const smartmem_swin_params_t* pp, const void* x, void* y, void* wo
       // narrow blocks: LN2 + fc1 + GELU + fc2 + residual in one kernel; neither the normalised rows
       // nor the hidden activation leave the chip
       SM_TRY("mlp_fused_ln2_fc1_gelu_fc2_residual",
-             launch_mlp_fused(y1, p.ln2_g, p.ln2_b, p.ln_eps, p.w_fc1, p.b_fc1, p.w_fc2, p.b_fc2, y1, y, M, C, hid, st));
+             launch_mlp_fused(y1, p.ln2_g, p.ln2_b, p.ln_eps, p.w_fc1, p.b_fc1, p.w_fc2, p.b_fc2, y, M, C, hid, st));
     } else {
       SM_TRY("ln2", launch_norm(p.dtype, false, y1, at(L.yn), p.ln2_g, p.ln2_b, p.ln_eps, M, (int)C, nullptr, st));
       SM_TRY("fc1_gemm_gelu", linear(at(L.yn), p.w_fc1, p.b_fc1, at(L.hid), hid, C, 1, nullptr, nullptr));
