@@ -16,20 +16,29 @@
 //
 // Per 128-row tile: the producer brings the raw rows in by TMA (double-buffered across tiles), four
 // warps take the row statistics (a thread per row); then the kernel walks over chunks of 128 hidden
-// columns: fc1 of a chunk accumulates in TMEM, the GELU warps apply rstd and GELU on packed bf16
-// pairs and write the bf16 chunk back into the same TMEM buffer, and fc2 takes it from there as its
-// A operand (tensor memory) while fc1 of the next chunk is already running.  The output accumulator
-// is double-buffered in TMEM, so the output warps (b2, row stores) overlap the next tile.
+// columns: fc1 of a chunk accumulates in one of two S1 buffers in TMEM, a set of GELU warps applies rstd
+// and GELU on packed bf16 pairs and writes the bf16 chunk into one of two H buffers in TMEM, and fc2
+// takes it from there as its A operand (tensor memory).  The S1 buffer goes back to fc1 as soon as the
+// GELU warps have read it, the H buffer comes back with fc2's commit, so fc1, GELU and fc2 of
+// neighbouring chunks overlap.  There is one output accumulator; the output warps copy it to registers
+// and hand it back before they convert and store.
 //
-// Warp roles: 0 TMA producer, 1 fc1 issuer (+ the residual product) and TMEM owner, 2-9 GELU (two
-// warps per TMEM lane quadrant, 64 hidden columns each), 10-13 output, 14 fc2 issuer, 15-18 row
-// statistics.
+// Warp roles: 0 TMA producer, 1 fc1 issuer and TMEM owner, 2-17 GELU (two sets of eight for the even
+// and the odd chunks; in a set two warps per TMEM lane quadrant, 64 hidden columns each), 18-21
+// output, 22 fc2 issuer (+ the residual / bias product), 23-26 row statistics.  The issuer warps walk
+// their loops with all lanes and elect one lane for the tensor-core instructions: with warp-uniform
+// control flow the descriptors stay in uniform registers, which roughly halves the cost of issuing a
+// product compared with a branch on lane 0.
 //
-// What bounds it: the GELU warps -- tanh on the special-function unit (16 elements per clock per SM:
-// about 1000 cycles per chunk) and their instruction issue -- and the loop fc1(j) -> GELU(j) ->
-// fc2(j) -> fc1(j+2) over the two S1/H buffers.  An earlier version streamed the weights from L2
-// through a ring for every tile (113 MB of L2 reads per launch at 100 352 rows, against 21 MB now)
-// and normalised the rows in place; with all of its arithmetic compiled out it still took 18 us.
+// What bounds it (clock stamps of every hand-off): the fc2 issuer's chain -- per chunk its eight
+// products queue behind the seven of fc1 on the one tensor pipe (about 800 cycles), per tile the
+// residual / bias products and the wait for the output warps to hand the accumulator back -- and the
+// GELU warps (tanh on the special-function unit, 16 elements per clock per SM).  Isolated, the kernel
+// runs 17 us at 100 352 rows, 4 us of which are the prologue (144 KB of weights per SM from L2 and the
+// fold); back to back with other kernels that prologue overlaps the previous kernel's tail.  An earlier
+// version streamed the weights from L2 through a ring for every tile (113 MB of L2 reads per launch,
+// against 21 MB now) and normalised the rows in place; with all of its arithmetic compiled out it still
+// took 18 us.
 
 #include "gemm_tc.cuh"
 #include "ptx.cuh"
@@ -45,9 +54,8 @@ constexpr int KBT = BM * KB * 2;                   // one 128 x 32 bf16 block: 8
 constexpr int AX_BYTES = BM * 32;                  // the extra k-step of a tile: 128 rows x 16 bf16
 constexpr int ID_BYTES = 32 * 64;                  // identity tile
 constexpr int kGeluWarps = 16, kOutWarps = 4, kStatWarps = 4, kThreads = 32 * (3 + kGeluWarps + kOutWarps + kStatWarps);
-constexpr int NS1 = 3;                             // S1 / H buffers: chunks in flight between fc1 and fc2
-constexpr uint32_t TM_S1 = 0, TM_OUT = NS1 * HC, TMEM_COLS = 512;   // S1 x3 (128 columns; H is written over its own S1 buffer), OUT (C columns)
-constexpr int N_BARS = 19;
+constexpr uint32_t TM_S1 = 0, TM_H = 2 * HC, TM_OUT = 3 * HC, TMEM_COLS = 512;   // S1 x2 (128 columns), H x2 (64 columns of bf16 pairs), OUT (C columns)
+constexpr int N_BARS = 18;
 constexpr int RSTD_RING = 4;                       // tiles whose rstd may be live at once (statistics run up to two tiles ahead of GELU)
 
 struct MlpArgs {
@@ -60,10 +68,10 @@ struct MlpArgs {
 };
 
 __host__ __device__ inline size_t mlp_smem_tiles(int C, int hidden) {
-  return (size_t)2 * (C / KB) * KBT + (size_t)2 * hidden * C * 2 + 2 * AX_BYTES + (size_t)hidden * 32 + ID_BYTES;
+  return (size_t)2 * (C / KB) * KBT + (size_t)2 * hidden * C * 2 + 2 * AX_BYTES + (size_t)hidden * 32 + ID_BYTES + (size_t)C * 32;
 }
 __host__ __device__ inline size_t mlp_smem_need(int C, int hidden) {
-  return mlp_smem_tiles(C, hidden) + N_BARS * 8 + 16 + (size_t)(3 * C + RSTD_RING * BM) * 4;
+  return mlp_smem_tiles(C, hidden) + N_BARS * 8 + 16 + (size_t)(2 * C + RSTD_RING * BM) * 4;
 }
 
 // tanh-form GELU (times two, see below) of two pre-activations, evaluated on packed bf16 pairs: the result is stored as
@@ -102,13 +110,15 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   uint8_t* sAx = sW2 + (g.hidden / KB) * W2_KB;    // [2][128 rows x 32 B]
   uint8_t* sW1x = sAx + 2 * AX_BYTES;              // [hidden rows x 32 B]
   uint8_t* sId = sW1x + g.hidden * 32;             // [32 rows x 64 B]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sId + ID_BYTES);
-  uint64_t *a_full = bars, *a_empty = bars + 2, *a_ready = bars + 4, *s1_full = bars + 6, *s1_empty = bars + 9;
-  uint64_t *h_full = bars + 12, *out_full = bars + 15, *out_empty = bars + 16, *w1_full = bars + 17, *w2_full = bars + 18;
+  uint8_t* sB2x = sId + ID_BYTES;                  // [C rows x 32 B]: 2 b2 on the positions where the extra k-step's rows hold ones
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sB2x + C * 32);
+  uint64_t *a_full = bars, *a_empty = bars + 2, *a_ready = bars + 4, *s1_full = bars + 6, *s1_free = bars + 8;
+  uint64_t *h_full = bars + 10, *h_empty = bars + 12, *out_full = bars + 14, *out_empty = bars + 15;
+  uint64_t *w1_full = bars + 16, *w2_full = bars + 17;
+
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + N_BARS);
   int* abort_flag = reinterpret_cast<int*>(tmem_slot + 1);
-  float* b2_s = reinterpret_cast<float*>(tmem_slot + 4);     // [C]
-  float* ln_s = b2_s + C;                                    // [2][C]: gamma, beta
+  float* ln_s = reinterpret_cast<float*>(tmem_slot + 4);     // [2][C]: gamma, beta
   float* rstd_s = ln_s + 2 * C;                              // [RSTD_RING][128]
 
   // The tiles fill the 227 KB almost completely, so the launch cannot afford a spare kilobyte of
@@ -118,7 +128,7 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     return;
   }
 
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tid = threadIdx.x, warp = __shfl_sync(0xFFFFFFFFu, tid >> 5, 0), lane = tid & 31;   // (warp: provably uniform)
   const int my_tiles = ((int)g.tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
   const int total = my_tiles * NC;                 // hidden chunks this CTA walks through, over all its tiles
 
@@ -128,10 +138,11 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       ptx::mbar_init(&a_empty[i], 2);                        // the last fc1 product and the residual product of the tile
       ptx::mbar_init(&a_ready[i], kStatWarps);
     }
-    for (int i = 0; i < NS1; ++i) {
+    for (int i = 0; i < 2; ++i) {
       ptx::mbar_init(&s1_full[i], 1);
-      ptx::mbar_init(&s1_empty[i], 1);                       // fc2 of the chunk has consumed the buffer (its H)
-      ptx::mbar_init(&h_full[i], kGeluWarps);                // H of buffer i written
+      ptx::mbar_init(&s1_free[i], kGeluWarps / 2);           // the chunk's GELU warps have read S1 buffer i
+      ptx::mbar_init(&h_full[i], kGeluWarps / 2);            // H buffer i written (by the set of GELU warps that has the chunk)
+      ptx::mbar_init(&h_empty[i], 1);                        // fc2 of the chunk has consumed H buffer i
     }
     ptx::mbar_init(out_full, 1);
     ptx::mbar_init(out_empty, kOutWarps);
@@ -155,9 +166,12 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   }
 #pragma unroll 1
   for (int i = tid; i < C; i += kThreads) {
-    b2_s[i] = __bfloat162float(g.b2[i]);
     ln_s[i] = __bfloat162float(g.ln_gamma[i]);
     ln_s[C + i] = __bfloat162float(g.ln_beta[i]);
+    uint4 k0, k1;
+    bias_col(2.0f * __bfloat162float(g.b2[i]), k0, k1);     // (the output accumulator holds twice the result)
+    *reinterpret_cast<uint4*>(sB2x + plain_off(i, 0)) = k0;
+    *reinterpret_cast<uint4*>(sB2x + plain_off(i, 1)) = k1;
   }
 #pragma unroll 1
   for (int i = tid; i < (2 * AX_BYTES + ID_BYTES) / 16; i += kThreads) {
@@ -234,122 +248,154 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       }
     }
   } else if (warp == 1) {
-    // fc1 issuer: S1[j % 3] = A W1'[chunk j]^T + the extra k-step, up to three chunks ahead of fc2
-    if (lane == 0 && w_ok) {
+    // fc1 issuer: S1[j & 1] = A W1'[chunk j]^T + the extra k-step, as soon as the GELU warps have read the buffer
+    if (w_ok) {                                         // (the whole warp walks the loop; one elected lane issues)
       const uint32_t idesc1 = ptx::make_idesc_bf16(BM, HC, false, false);
       const uint32_t a_base = ptx::smem_u32(sA), w_base = ptx::smem_u32(sW1), ax_base = ptx::smem_u32(sAx);
       const uint32_t wx_base = ptx::smem_u32(sW1x);
       int it1 = 0, c1 = 0;
-      uint32_t sb = 0, ph = 0;
       bool ok = true;
 #pragma unroll 1
       for (int j = 0; j < total && ok; ++j) {
-        const uint32_t ab = it1 & 1;
+        const uint32_t ab = it1 & 1, sb = j & 1, ph = (j >> 1) & 1;
         if (c1 == 0) ok = ptx::mbar_wait(&a_ready[ab], (it1 >> 1) & 1, abort_flag, g.status);
-        ok = ok && ptx::mbar_wait(&s1_empty[sb], ph ^ 1, abort_flag, g.status);
+        ok = ok && ptx::mbar_wait(&s1_free[sb], ph ^ 1, abort_flag, g.status);
+        ok = __all_sync(0xFFFFFFFFu, ok ? 1 : 0) != 0;
         if (!ok) break;
         ptx::tc_fence_after();
         const uint32_t d = tmem_base + TM_S1 + sb * HC;
         const uint64_t ad = desc_sw64(a_base + ab * A_BYTES);
         const uint64_t bd = desc_sw64(w_base + c1 * KBT);
+        const bool last = c1 + 1 == NC;
+        if (ptx::elect_one()) {
 #pragma unroll
-        for (int kb = 0; kb < NKB; ++kb) {
-          ptx::tc_mma_bf16(d, ad + kb * (KBT >> 4), bd + kb * (W1_KB >> 4), idesc1, kb ? 1u : 0u);
-          ptx::tc_mma_bf16(d, ad + kb * (KBT >> 4) + 2, bd + kb * (W1_KB >> 4) + 2, idesc1, 1u);
+          for (int kb = 0; kb < NKB; ++kb) {
+            ptx::tc_mma_bf16(d, ad + kb * (KBT >> 4), bd + kb * (W1_KB >> 4), idesc1, kb ? 1u : 0u);
+            ptx::tc_mma_bf16(d, ad + kb * (KBT >> 4) + 2, bd + kb * (W1_KB >> 4) + 2, idesc1, 1u);
+          }
+          ptx::tc_mma_bf16(d, desc_plain(ax_base + ab * AX_BYTES), desc_plain(wx_base + c1 * (HC * 32)), idesc1, 1u);
+          ptx::tc_commit(&s1_full[sb]);
+          if (last) ptx::tc_commit(&a_empty[ab]);       // every fc1 product of this tile has been issued
         }
-        ptx::tc_mma_bf16(d, desc_plain(ax_base + ab * AX_BYTES), desc_plain(wx_base + c1 * (HC * 32)), idesc1, 1u);
-        ptx::tc_commit(&s1_full[sb]);
-        if (++c1 == NC) {
-          ptx::tc_commit(&a_empty[ab]);                 // every fc1 product of this tile has been issued
+        __syncwarp();
+        if (last) {
           c1 = 0;
           ++it1;
+        } else {
+          ++c1;
         }
-        if (++sb == NS1) { sb = 0; ph ^= 1; }
       }
     }
   } else if (warp == 2 + kGeluWarps + kOutWarps) {
-    // fc2 issuer: at the first chunk of a tile OUT = A (2 I), the residual; then OUT += H[j % 3] W2[:, chunk j]^T
-    if (lane == 0 && w_ok) {
+    // fc2 issuer: at the first chunk of a tile OUT = A (2 I) + 2 b2; then OUT += H[j & 1] W2[:, chunk j]^T
+    if (w_ok) {
       const uint32_t idesc2 = ptx::make_idesc_bf16(BM, C, false, false);
       const uint32_t idesc_id = ptx::make_idesc_bf16(BM, 32, false, false);
       const uint32_t w_base = ptx::smem_u32(sW2), a_base = ptx::smem_u32(sA);
-      const uint64_t idd = desc_sw64(ptx::smem_u32(sId));
+      const uint64_t idd = desc_sw64(ptx::smem_u32(sId)), b2d = desc_plain(ptx::smem_u32(sB2x));
+      const uint32_t ax_base = ptx::smem_u32(sAx);
       const uint32_t d = tmem_base + TM_OUT;
       int it2 = 0, c2 = 0;
-      uint32_t sb = 0, ph = 0;
-      bool ok = ptx::mbar_wait(w2_full, 0, abort_flag, g.status);
+      bool ok = __all_sync(0xFFFFFFFFu, ptx::mbar_wait(w2_full, 0, abort_flag, g.status) ? 1 : 0) != 0;
 #pragma unroll 1
       for (int j = 0; j < total && ok; ++j) {
+        const uint32_t sb = j & 1, ph = (j >> 1) & 1;
         ok = ptx::mbar_wait(&h_full[sb], ph, abort_flag, g.status);
         if (c2 == 0) ok = ok && ptx::mbar_wait(out_empty, (it2 & 1) ^ 1, abort_flag, g.status);
+        ok = __all_sync(0xFFFFFFFFu, ok ? 1 : 0) != 0;
         if (!ok) break;
         ptx::tc_fence_after();
-        if (c2 == 0) {
-          const uint64_t ad = desc_sw64(a_base + (it2 & 1) * A_BYTES);
-#pragma unroll
-          for (int kb = 0; kb < NKB; ++kb) {
-            ptx::tc_mma_bf16(d + kb * KB, ad + kb * (KBT >> 4), idd, idesc_id, 0u);
-            ptx::tc_mma_bf16(d + kb * KB, ad + kb * (KBT >> 4) + 2, idd + 2, idesc_id, 1u);
-          }
-          ptx::tc_commit(&a_empty[it2 & 1]);            // the raw rows have had their last reader
-        }
-        // H chunk: written by the GELU warps over the S1 buffer it was computed from -- the 32 hidden columns of part p
-        // as 16 packed columns at offset 32 p
-        const uint32_t a = tmem_base + TM_S1 + sb * HC;
+        // H chunk: 128 hidden columns as 64 columns of bf16 pairs
+        const uint32_t a = tmem_base + TM_H + sb * (HC / 2);
         const uint64_t bd = desc_sw64(w_base + c2 * 4 * W2_KB);
+        const uint64_t ad = desc_sw64(a_base + (it2 & 1) * A_BYTES);
+        const bool first = c2 == 0, last = c2 + 1 == NC;
+        if (ptx::elect_one()) {
+          if (first) {
 #pragma unroll
-        for (int k = 0; k < HC / 16; ++k)               // 16 hidden columns = 8 packed TMEM columns per step
-          ptx::tc_mma_bf16_ta(d, a + 32 * (k >> 1) + 8 * (k & 1), bd + (k >> 1) * (W2_KB >> 4) + 2 * (k & 1), idesc2, 1u);
-        ptx::tc_commit(&s1_empty[sb]);                  // buffer consumed: fc1 of chunk j + 3 may overwrite it
-        if (++c2 == NC) {
-          ptx::tc_commit(out_full);
+            for (int kb = 0; kb < NKB; ++kb) {
+              ptx::tc_mma_bf16(d + kb * KB, ad + kb * (KBT >> 4), idd, idesc_id, 0u);
+              ptx::tc_mma_bf16(d + kb * KB, ad + kb * (KBT >> 4) + 2, idd + 2, idesc_id, 1u);
+            }
+            ptx::tc_mma_bf16(d, desc_plain(ax_base + (it2 & 1) * AX_BYTES), b2d, idesc2, 1u);   // + 2 b2
+            ptx::tc_commit(&a_empty[it2 & 1]);          // the raw rows have had their last reader
+          }
+#pragma unroll
+          for (int k = 0; k < HC / 16; ++k)             // 16 hidden columns = 8 packed TMEM columns per step
+            ptx::tc_mma_bf16_ta(d, a + 8 * k, bd + (k >> 1) * (W2_KB >> 4) + 2 * (k & 1), idesc2, 1u);
+          ptx::tc_commit(&h_empty[sb]);                 // H buffer consumed: GELU of chunk j + 2 may overwrite it
+          if (last) ptx::tc_commit(out_full);
+        }
+        __syncwarp();
+        if (last) {
           c2 = 0;
           ++it2;
+        } else {
+          ++c2;
         }
-        if (++sb == NS1) { sb = 0; ph ^= 1; }
       }
     }
   } else if (warp < 2 + kGeluWarps) {
-    // GELU warps: S1 chunk (TMEM, fp32) -> x rstd -> GELU -> bf16 pairs -> the H region of TMEM, where
-    // fc2 reads the chunk as its A operand.  Four warps per TMEM lane quadrant, 32 hidden columns each; the 16
-    // packed columns go over the first half of the columns the warp has just read (it is their only reader and
-    // writer), so each S1 buffer carries its chunk from fc1 through GELU to fc2 and is handed back to fc1 by
-    // fc2's commit; the GELU warps themselves wait for nothing but the next fc1 result.
-    const int e = warp - 2, q = warp & 3, part = e >> 2;
+    // GELU warps: S1 chunk (TMEM, fp32) -> x rstd -> GELU -> bf16 pairs -> an H buffer in TMEM, where fc2 reads
+    // the chunk as its A operand.  Two sets of eight warps take the even and the odd chunks (S1 and H buffer
+    // = set), so that one set's tensor-memory loads and stores overlap the other's arithmetic (tanh on the
+    // special-function unit is what bounds them); in a set, two warps per TMEM lane quadrant with 64 hidden
+    // columns each, in two rounds of 32.  The S1 buffer goes back to fc1 as soon as the set has read it; the H
+    // buffer comes back from fc2's commit.
+    const int e = warp - 2, set = e >> 3, q = warp & 3, hh = (e & 7) >> 2;
     bool ok = w_ok;
-    int c = 0, ti = 0;
-    uint32_t sb = 0, ph = 0;
+    int c = set, ti = 0;
+    while (c >= NC) { c -= NC; ++ti; }
+    uint32_t ph = 0;
+    const uint32_t lane_q = (uint32_t)(q * 32) << 16;
+    const uint32_t ts = tmem_base + TM_S1 + set * HC + lane_q + hh * 64;
+    const uint32_t th = tmem_base + TM_H + set * (HC / 2) + lane_q + hh * 32;
 #pragma unroll 1
-    for (int j = 0; j < total && ok; ++j) {
-      ok = ptx::mbar_wait(&s1_full[sb], ph, abort_flag, g.status);
+    for (int j = set; j < total && ok; j += 2) {
+      ok = ptx::mbar_wait(&s1_full[set], ph, abort_flag, g.status);
       if (!ok) break;
       const float rstd = rstd_s[(ti & (RSTD_RING - 1)) * BM + q * 32 + lane];
       const f32x2 r2 = ptx::pack2(rstd, rstd);
-      const uint32_t tq = tmem_base + TM_S1 + sb * HC + ((uint32_t)(q * 32) << 16) + part * 32;
       ptx::tc_fence_after();
-      uint32_t rv[32];
-      ptx::tmem_ld32(tq, rv);
-      ptx::tmem_ld_wait();
-      uint32_t pk[16];
 #pragma unroll
-      for (int v = 0; v < 16; ++v) {
-        float xa, xb;
-        ptx::unpack2(ptx::mul2(ptx::pack2(__uint_as_float(rv[2 * v]), __uint_as_float(rv[2 * v + 1])), r2), xa, xb);
-        pk[v] = gelu_tanh_bf16x2(xa, xb);
+      for (int h2 = 0; h2 < 2; ++h2) {
+        uint32_t rv[32];
+        ptx::tmem_ld32(ts + h2 * 32, rv);
+        ptx::tmem_ld_wait();
+        if (h2 == 1) {                                   // S1 is in registers: fc1 of chunk j + 2 may overwrite the buffer
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(&s1_free[set]);
+        }
+        uint32_t pk[16];
+#pragma unroll
+        for (int v = 0; v < 16; ++v) {
+          float xa, xb;
+          ptx::unpack2(ptx::mul2(ptx::pack2(__uint_as_float(rv[2 * v]), __uint_as_float(rv[2 * v + 1])), r2), xa, xb);
+          pk[v] = gelu_tanh_bf16x2(xa, xb);
+        }
+        if (h2 == 0) {                                   // fc2 of chunk j - 2 has read the H buffer
+          ok = ptx::mbar_wait(&h_empty[set], ph ^ 1, abort_flag, g.status);
+          if (!ok) break;
+          ptx::tc_fence_after();
+        }
+        ptx::tmem_st16(th + h2 * 16, pk);
       }
-      ptx::tmem_st16(tq, pk);
+      if (!ok) break;
       ptx::tmem_st_wait();
       ptx::tc_fence_before();
       __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(&h_full[sb]);
-      if (++c == NC) { c = 0; ++ti; }
-      if (++sb == NS1) { sb = 0; ph ^= 1; }
+      if (lane == 0) ptx::mbar_arrive(&h_full[set]);
+      c += 2;
+      while (c >= NC) { c -= NC; ++ti; }
+      ph ^= 1;
     }
   } else if (warp < 2 + kGeluWarps + kOutWarps) {
     // Output warps, one per TMEM lane quadrant: OUT / 2 + b2 -> out, a thread per row, in rounds of 32
     // columns.  They work on one OUT buffer while the products of the next tile fill the other.
     const int q = warp & 3;
     const int rounds = C / 32;
+    const f32x2 half2 = ptx::pack2(0.5f, 0.5f);
     bool ok = w_ok;
 #pragma unroll 1
     for (int ti = 0; ti < my_tiles && ok; ++ti) {
@@ -374,10 +420,10 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         for (int v = 0; v < 4; ++v) {
           uint32_t o[4];
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const float2 b = *reinterpret_cast<const float2*>(b2_s + r * 32 + v * 8 + 2 * i);
-            o[i] = float2_to_bf16x2(fmaf(__uint_as_float(rv[v * 8 + 2 * i]), 0.5f, b.x),       // the accumulator holds 2 (A + H W2^T)
-                                    fmaf(__uint_as_float(rv[v * 8 + 2 * i + 1]), 0.5f, b.y));
+          for (int i = 0; i < 4; ++i) {                // the accumulator holds 2 (A + H W2^T + b2)
+            float xa, xb;
+            ptx::unpack2(ptx::mul2(ptx::pack2(__uint_as_float(rv[v * 8 + 2 * i]), __uint_as_float(rv[v * 8 + 2 * i + 1])), half2), xa, xb);
+            o[i] = float2_to_bf16x2(xa, xb);
           }
           if (row_ok) *reinterpret_cast<uint4*>(g.out + off + r * 32 + v * 8) = make_uint4(o[0], o[1], o[2], o[3]);
         }

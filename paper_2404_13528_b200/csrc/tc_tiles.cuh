@@ -50,7 +50,15 @@ __device__ __forceinline__ void extra_row(float u, float s, uint4& k0, uint4& k1
   split3(u, uh, um, ul);
   split3(s, sh, sm_, sl);
   k0 = make_uint4(uh | (uh << 16), um | (uh << 16), ul | (um << 16), sh | (sh << 16));
-  k1 = make_uint4(sm_ | (sh << 16), sl | (sm_ << 16), 0u, 0u);
+  k1 = make_uint4(sm_ | (sh << 16), sl | (sm_ << 16), 0x3F803F80u, 0x00003F80u);   // positions 12..14: ones (see bias_col)
+}
+// Weight side of a bias that rides on the same operand rows: positions 12..14 of a row hold ones, so a column whose
+// positions 12..14 hold the three pieces of v (and zeros elsewhere) adds v to every row of the product.
+__device__ __forceinline__ void bias_col(float v, uint4& k0, uint4& k1) {
+  uint32_t h, m, l;
+  split3(v, h, m, l);
+  k0 = make_uint4(0u, 0u, 0u, 0u);
+  k1 = make_uint4(0u, 0u, h | (m << 16), l);
 }
 __device__ __forceinline__ void extra_col(float c, float b, uint4& k0, uint4& k1) {
   uint32_t ch, cm, cl, bh, bm, bl;
