@@ -149,7 +149,8 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
     return;
   }
 
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int warp = __shfl_sync(0xFFFFFFFFu, tid >> 5, 0);   // (provably warp-uniform: the issuing code below keeps its operands in uniform registers)
   const int cidx = blockIdx.x, cstride = gridDim.x;
   const int U = cidx < g.n_pairs ? (g.n_pairs - cidx + cstride - 1) / cstride : 0;   // units of this CTA
   const int total = U * NH;                                                         // items
@@ -472,7 +473,7 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
     const int q = warp & 3;                            // TMEM lane quadrant
     const int r = q * 32 + lane;
     const int w = r >> 6, i = r & 63;                  // window of the pair, token
-    const bool elected = q == 0 && lane == 0;
+    const bool elected = q == 0 && lane == 0;          // (arrivals on behalf of the group)
     const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
     const int my_ty = tyx_s[i] >> 8, my_tx = tyx_s[i] & 255;
     const uint32_t ky_lo = kmask_s[0], ky_hi = kmask_s[1], kx_lo = kmask_s[2], kx_hi = kmask_s[3];
@@ -540,8 +541,8 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
         ptx::fence_proxy_async();                      // generic-proxy writes -> visible to the MMAs
         ptx::tc_fence_before();
       }
-      if (group_sync()) break;
-      if (elected) {
+      if (__any_sync(0xFFFFFFFFu, group_sync())) break;
+      if (q == 0 && ptx::elect_one()) {
         // S = [q0 0; 0 q1] [k0 | k1]^T: four k16 steps, the first two over window 0's keys, the last two over window 1's
         ptx::tc_fence_after();
         const uint32_t idesc = ptx::make_idesc_bf16(BM, 64, false, false);
@@ -630,8 +631,8 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
         ptx::tmem_st_wait();
         ptx::tc_fence_before();
       }
-      if (group_sync()) break;
-      if (elected) {
+      if (__any_sync(0xFFFFFFFFu, group_sync())) break;
+      if (q == 0 && ptx::elect_one()) {
         // O = P [v0; v1] over the columns q has left: P from tensor memory, V as it lies (MN-major B operand); 16 keys per
         // step: P +8 packed columns, V +16 rows = 1024 bytes
         ptx::tc_fence_after();
@@ -669,7 +670,7 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
     // ---- the products that have slack -- QKV of the items ahead, the projections -- are issued by a thread of their own, in item
     // order, so that no group thread ever waits on their inputs.  Issue order is accumulation order (the heads of a unit add
     // up in Y) and also orders a buffer's next accumulator behind the projection that reads the buffer last. -----------------
-    if (lane == 0 && w_ok) {
+    if (__all_sync(0xFFFFFFFFu, w_ok ? 1 : 0)) {          // the whole warp walks the queues; an elected lane issues
       const uint32_t idesc_qkv = ptx::make_idesc_bf16(BM, WROWS, false, false);
       const uint32_t idesc_pj = ptx::make_idesc_bf16(BM, C, false, false);
       const uint32_t idesc_id = ptx::make_idesc_bf16(BM, D, false, false);
@@ -683,47 +684,58 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
       unsigned long long t_idle = 0;
       while (ji < total) {
         bool progress = false;
-        if (xu < U && xu <= ju && ptx::mbar_test(y_empty, (xu & 1) ^ 1) && ptx::mbar_test(&a_full[xab], xaph)) {
+        if (xu < U && xu <= ju && __all_sync(0xFFFFFFFFu, ptx::mbar_test(y_empty, (xu & 1) ^ 1) && ptx::mbar_test(&a_full[xab], xaph))) {
           // Y = X I: the unit's raw rows open the accumulation (the epilogue of the unit before has read Y); exact, since every
           // product is a bf16 value times one.  The product is the last reader of the unit's rows: its completion frees the slot.
           ptx::tc_fence_after();
           const uint64_t bd = desc_sw64(id_base);
+          const uint64_t ad0 = desc_sw64(a_base + xab * A_BYTES);
+          if (ptx::elect_one()) {
 #pragma unroll
-          for (int kb = 0; kb < NH; ++kb) {            // 32 channels at a time: Y[:, 32 kb : 32 kb + 32] = X[:, 32 kb : 32 kb + 32] I_32
-            const uint64_t ad = desc_sw64(a_base + xab * A_BYTES + kb * KBT);
-            ptx::tc_mma_bf16(tmem_base + TM_Y + kb * D, ad, bd, idesc_id, 0u);
-            ptx::tc_mma_bf16(tmem_base + TM_Y + kb * D, ad + 2, bd + 2, idesc_id, 1u);
+            for (int kb = 0; kb < NH; ++kb) {          // 32 channels at a time: Y[:, 32 kb : 32 kb + 32] = X[:, 32 kb : 32 kb + 32] I_32
+              const uint64_t ad = ad0 + kb * (KBT >> 4);
+              ptx::tc_mma_bf16(tmem_base + TM_Y + kb * D, ad, bd, idesc_id, 0u);
+              ptx::tc_mma_bf16(tmem_base + TM_Y + kb * D, ad + 2, bd + 2, idesc_id, 1u);
+            }
+            ptx::tc_commit(&a_free[xab]);
           }
-          ptx::tc_commit(&a_free[xab]);
+          __syncwarp();
           ++xu;
           if (++xab == na) { xab = 0; xaph ^= 1; }
           progress = true;
         }
-        if (xu > ju && ptx::mbar_test(&ob_full[ji & (NBUF - 1)], (ji >> 2) & 1)) {
+        if (xu > ju && __all_sync(0xFFFFFFFFu, ptx::mbar_test(&ob_full[ji & (NBUF - 1)], (ji >> 2) & 1))) {
           // Y += Ob_h Wp[:, 32 h : 32 h + 32]^T; the last head hands Y to the epilogue
           ptx::tc_fence_after();
           const uint32_t a = tmem_base + (ji & (NBUF - 1)) * BUF_COLS + 64;
           const uint64_t bd = desc_sw64(wp_base + jh * WP_TILE);
-          ptx::tc_mma_bf16_ta(tmem_base + TM_Y, a, bd, idesc_pj, 1u);
-          ptx::tc_mma_bf16_ta(tmem_base + TM_Y, a + 8, bd + 2, idesc_pj, 1u);
-          if (jh == NH - 1) ptx::tc_commit(y_full);
+          if (ptx::elect_one()) {
+            ptx::tc_mma_bf16_ta(tmem_base + TM_Y, a, bd, idesc_pj, 1u);
+            ptx::tc_mma_bf16_ta(tmem_base + TM_Y, a + 8, bd + 2, idesc_pj, 1u);
+            if (jh == NH - 1) ptx::tc_commit(y_full);
+          }
+          __syncwarp();
           ++ji;
           if (++jh == NH) { jh = 0; ++ju; }
           progress = true;
         }
-        if (qi < total && qi < ji + NBUF && ptx::mbar_test(&a_full[qab], qaph)) {
+        if (qi < total && qi < ji + NBUF && __all_sync(0xFFFFFFFFu, ptx::mbar_test(&a_full[qab], qaph))) {
           // acc = [X | e] [Wq_h; Wk_h; Wv_h | f]^T into the buffer item qi - NBUF has left (its projection was issued above)
           ptx::tc_fence_after();
           const uint32_t d = tmem_base + (qi & (NBUF - 1)) * BUF_COLS;
+          const uint64_t ad0 = desc_sw64(a_base + qab * A_BYTES), bd0 = desc_sw64(wq_base + qh * NH * WQ_TILE);
+          const uint64_t axd = desc_plain(ax_base + qab * AX_BYTES), wxd = desc_plain(wx_base + qh * WX_TILE);
+          if (ptx::elect_one()) {
 #pragma unroll
-          for (int kb = 0; kb < NH; ++kb) {
-            const uint64_t ad = desc_sw64(a_base + qab * A_BYTES + kb * KBT);
-            const uint64_t bd = desc_sw64(wq_base + (qh * NH + kb) * WQ_TILE);
-            ptx::tc_mma_bf16(d, ad, bd, idesc_qkv, kb ? 1u : 0u);
-            ptx::tc_mma_bf16(d, ad + 2, bd + 2, idesc_qkv, 1u);      // next 16 channels: +32 bytes
+            for (int kb = 0; kb < NH; ++kb) {
+              const uint64_t ad = ad0 + kb * (KBT >> 4), bd = bd0 + kb * (WQ_TILE >> 4);
+              ptx::tc_mma_bf16(d, ad, bd, idesc_qkv, kb ? 1u : 0u);
+              ptx::tc_mma_bf16(d, ad + 2, bd + 2, idesc_qkv, 1u);    // next 16 channels: +32 bytes
+            }
+            ptx::tc_mma_bf16(d, axd, wxd, idesc_qkv, 1u);
+            ptx::tc_commit(&acc_full[qi & (NBUF - 1)]);
           }
-          ptx::tc_mma_bf16(d, desc_plain(ax_base + qab * AX_BYTES), desc_plain(wx_base + qh * WX_TILE), idesc_qkv, 1u);
-          ptx::tc_commit(&acc_full[qi & (NBUF - 1)]);
+          __syncwarp();
           ++qi;
           if (++qh == NH) {
             qh = 0; ++qu;
@@ -734,12 +746,14 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
         if (progress) {
           idle = 0;
         } else if ((++idle & 255u) == 0) {
-          if (*(volatile int*)abort_flag) break;
-          const unsigned long long now = ptx::globaltimer();
+          if (__any_sync(0xFFFFFFFFu, *(volatile int*)abort_flag)) break;
+          const unsigned long long now = __shfl_sync(0xFFFFFFFFu, ptx::globaltimer(), 0);
           if (idle == 256u) t_idle = now;
           else if (now - t_idle > ptx::kWaitLimitNs) {
-            *abort_flag = 1;
-            atomicExch(g.status, (int)SMARTMEM_ERR_TIMEOUT);
+            if (lane == 0) {
+              *abort_flag = 1;
+              atomicExch(g.status, (int)SMARTMEM_ERR_TIMEOUT);
+            }
             break;
           }
         }
