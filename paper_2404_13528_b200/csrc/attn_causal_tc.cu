@@ -68,7 +68,7 @@ causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     if (threadIdx.x == 0) atomicExch(g.status, (int)SMARTMEM_ERR_UNSUPPORTED);
     return;
   }
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int warp = __shfl_sync(0xFFFFFFFFu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;   // (warp: provably uniform)
   // heaviest units (last query tiles) first
   const int bh_count = g.batch * g.heads;
   const int qt = g.n_qt - 1 - (int)(blockIdx.x / bh_count);
@@ -128,50 +128,60 @@ causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
+    // the whole warp walks the issue loop and an elected lane issues: warp-uniform control flow keeps the
+    // descriptors in uniform registers
+    {
       const uint32_t idesc_s = ptx::make_idesc_bf16(BQ, BKV, false, false);
       const uint32_t idesc_pv = ptx::make_idesc_bf16(BQ, D, false, true);      // V: MN-major B operand
-      bool ok = ptx::mbar_wait(q_full, 0, abort_flag, g.status);
+      bool ok = __all_sync(0xFFFFFFFFu, ptx::mbar_wait(q_full, 0, abort_flag, g.status) ? 1 : 0) != 0;
       auto issue_s = [&](int j) {
         const int s = j & 1;
         const uint32_t ph = (j >> 1) & 1;
         ok = ok && ptx::mbar_wait(&s_empty[s], ph ^ 1, abort_flag, g.status);
         ok = ok && ptx::mbar_wait(&k_full[s], ph, abort_flag, g.status);
+        ok = __all_sync(0xFFFFFFFFu, ok ? 1 : 0) != 0;
         if (!ok) return;
         ptx::tc_fence_after();
+        if (ptx::elect_one()) {
 #pragma unroll
-        for (int kb = 0; kb < 2; ++kb) {
-          const uint64_t ad = ptx::make_smem_desc(ptx::smem_u32(sQ + kb * KB), 16, 1024);
-          const uint64_t bd = ptx::make_smem_desc(ptx::smem_u32(sK + (s * 2 + kb) * KBK), 16, 1024);
+          for (int kb = 0; kb < 2; ++kb) {
+            const uint64_t ad = ptx::make_smem_desc(ptx::smem_u32(sQ + kb * KB), 16, 1024);
+            const uint64_t bd = ptx::make_smem_desc(ptx::smem_u32(sK + (s * 2 + kb) * KBK), 16, 1024);
 #pragma unroll
-          for (int k = 0; k < 4; ++k)                   // a k16 step moves both start addresses by 32 bytes
-            ptx::tc_mma_bf16(tmem_base + TM_S + s * BKV, ad + 2 * k, bd + 2 * k, idesc_s, (kb | k) ? 1u : 0u);
+            for (int k = 0; k < 4; ++k)                 // a k16 step moves both start addresses by 32 bytes
+              ptx::tc_mma_bf16(tmem_base + TM_S + s * BKV, ad + 2 * k, bd + 2 * k, idesc_s, (kb | k) ? 1u : 0u);
+          }
+          ptx::tc_commit(&k_empty[s]);
+          ptx::tc_commit(&s_full[s]);
         }
-        ptx::tc_commit(&k_empty[s]);
-        ptx::tc_commit(&s_full[s]);
+        __syncwarp();
       };
       auto issue_pv = [&](int j) {
         const int s = j & 1;
         ok = ok && ptx::mbar_wait(p_full, j & 1, abort_flag, g.status);
         ok = ok && ptx::mbar_wait(&v_full[s], (j >> 1) & 1, abort_flag, g.status);
+        ok = __all_sync(0xFFFFFFFFu, ok ? 1 : 0) != 0;
         if (!ok) return;
         ptx::tc_fence_after();
         const uint32_t v0 = ptx::smem_u32(sV + s * 2 * KBK);
         const uint64_t vd = ptx::make_smem_desc(v0, KBK, 1024);
         const uint32_t pa = tmem_base + TM_S + s * BKV;  // P(j): bf16 pairs over the first 32 columns of the S buffer it came from
+        if (ptx::elect_one()) {
 #pragma unroll
-        for (int ks = 0; ks < BKV / 16; ++ks)          // 16 keys per step: P +8 packed columns, V +16 rows of 128 bytes; the two 64-wide d-chunks are KBK apart
-          ptx::tc_mma_bf16_ta(tmem_base + TM_O, pa + 8 * ks, vd + (2048 >> 4) * ks, idesc_pv, (j | ks) ? 1u : 0u);
-        ptx::tc_commit(&v_empty[s]);
-        ptx::tc_commit(&s_empty[s]);
-        ptx::tc_commit(p_empty);
+          for (int ks = 0; ks < BKV / 16; ++ks)        // 16 keys per step: P +8 packed columns, V +16 rows of 128 bytes; the two 64-wide d-chunks are KBK apart
+            ptx::tc_mma_bf16_ta(tmem_base + TM_O, pa + 8 * ks, vd + (2048 >> 4) * ks, idesc_pv, (j | ks) ? 1u : 0u);
+          ptx::tc_commit(&v_empty[s]);
+          ptx::tc_commit(&s_empty[s]);
+          ptx::tc_commit(p_empty);
+        }
+        __syncwarp();
       };
       issue_s(0);
       for (int j = 0; j < n_kv && ok; ++j) {
         if (j + 1 < n_kv) issue_s(j + 1);
         issue_pv(j);
       }
-      if (ok) ptx::tc_commit(o_done);
+      if (ok && ptx::elect_one()) ptx::tc_commit(o_done);
     }
   } else {
     const int q = warp & 3;                            // TMEM lane quadrant

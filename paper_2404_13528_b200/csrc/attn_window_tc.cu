@@ -91,7 +91,8 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
   int* abort_flag = reinterpret_cast<int*>(tmem_slot + 1);
 
   const WinAttnArgs& a = g.a;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int warp = __shfl_sync(0xFFFFFFFFu, tid >> 5, 0);   // (provably warp-uniform: the issuer warps keep their operands in uniform registers)
   const int T = a.T, ws = a.ws;
   const int h = blockIdx.x % a.heads;
   const int cidx = blockIdx.x / a.heads, cstride = gridDim.x / a.heads;
@@ -196,8 +197,8 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
       }
     }
   } else if (warp == 1) {
-    // ---- P V issuer (and owner of the tensor memory) -----------------------------------------
-    if (lane == 0) {
+    // ---- P V issuer (and owner of the tensor memory): the whole warp walks the loop, an elected lane issues ----
+    {
       const uint32_t idesc_pv = ptx::make_idesc_bf16(128, D, false, true);     // V: MN-major B operand
       bool ok = true;
       const int my_units = cidx < g.n_pairs ? (g.n_pairs - cidx + cstride - 1) / cstride : 0;
@@ -205,24 +206,28 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
         const int s = u % NSTAGE, ob = u & 1;
         ok = ptx::mbar_wait(&p_full[ob], (u >> 1) & 1, abort_flag, g.status);
         ok = ok && ptx::mbar_wait(&o_empty[ob], ((u >> 1) & 1) ^ 1, abort_flag, g.status);
+        ok = __all_sync(0xFFFFFFFFu, ok ? 1 : 0) != 0;
         if (!ok) break;
         ptx::tc_fence_after();
         const uint32_t v0 = ptx::smem_u32(sIn + s * STAGE_BYTES + 2 * OP_BYTES);
         const uint64_t vd = make_desc_sw64(v0, 16, 512);
         const uint32_t od = tmem_base + TM_O + ob * D, pa = tmem_base + TM_P + ob * 64;
-        ptx::tc_mma_bf16_ta(od, pa, vd, idesc_pv, 0u);
+        if (ptx::elect_one()) {
+          ptx::tc_mma_bf16_ta(od, pa, vd, idesc_pv, 0u);
 #pragma unroll
-        for (int ks = 1; ks < 8; ++ks)                 // 16 keys per step: P +8 packed columns, V +1024 bytes
-          ptx::tc_mma_bf16_ta(od, pa + 8 * ks, vd + ks * (1024 >> 4), idesc_pv, 1u);
-        ptx::tc_commit(&in_empty[s]);
-        ptx::tc_commit(&p_empty[ob]);
-        ptx::tc_commit(&o_full[ob]);
+          for (int ks = 1; ks < 8; ++ks)               // 16 keys per step: P +8 packed columns, V +1024 bytes
+            ptx::tc_mma_bf16_ta(od, pa + 8 * ks, vd + ks * (1024 >> 4), idesc_pv, 1u);
+          ptx::tc_commit(&in_empty[s]);
+          ptx::tc_commit(&p_empty[ob]);
+          ptx::tc_commit(&o_full[ob]);
+        }
+        __syncwarp();
       }
     }
   } else if (warp == 2 + kGroups * kSoftmaxWarps + kLoaderWarps) {
     // ---- S issuer: runs ahead of P V as far as the two S buffers and the input ring allow, so a
     // softmax group finds its next score tile waiting when it has written P ---------------------
-    if (lane == 0) {
+    {
       const uint32_t idesc_s = ptx::make_idesc_bf16(128, 128, false, false);
       bool ok = true;
       const int my_units = cidx < g.n_pairs ? (g.n_pairs - cidx + cstride - 1) / cstride : 0;
@@ -230,13 +235,17 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
         const int s = u % NSTAGE, sb = u & 1;
         ok = ptx::mbar_wait(&s_empty[sb], ((u >> 1) & 1) ^ 1, abort_flag, g.status);
         ok = ok && ptx::mbar_wait(&in_full[s], (u / NSTAGE) & 1, abort_flag, g.status);
+        ok = __all_sync(0xFFFFFFFFu, ok ? 1 : 0) != 0;
         if (!ok) break;
         ptx::tc_fence_after();
         const uint32_t q0 = ptx::smem_u32(sIn + s * STAGE_BYTES), k0 = q0 + OP_BYTES;
         const uint64_t qd = make_desc_sw64(q0, 16, 512), kd = make_desc_sw64(k0, 16, 512);
-        ptx::tc_mma_bf16(tmem_base + TM_S + sb * 128, qd, kd, idesc_s, 0u);
-        ptx::tc_mma_bf16(tmem_base + TM_S + sb * 128, qd + 2, kd + 2, idesc_s, 1u);    // next 16 features: +32 bytes
-        ptx::tc_commit(&s_full[sb]);
+        if (ptx::elect_one()) {
+          ptx::tc_mma_bf16(tmem_base + TM_S + sb * 128, qd, kd, idesc_s, 0u);
+          ptx::tc_mma_bf16(tmem_base + TM_S + sb * 128, qd + 2, kd + 2, idesc_s, 1u);  // next 16 features: +32 bytes
+          ptx::tc_commit(&s_full[sb]);
+        }
+        __syncwarp();
       }
     }
   } else if (warp < 2 + kGroups * kSoftmaxWarps) {

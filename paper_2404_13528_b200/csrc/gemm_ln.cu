@@ -74,7 +74,7 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     return;
   }
 
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int warp = __shfl_sync(0xFFFFFFFFu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;   // (warp: provably uniform)
   const int nsub = g.nsub;
   const int my_tiles = ((int)g.tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
 
@@ -115,33 +115,38 @@ gemm_ln_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   pdl_launch_dependents();
 
   if (warp == 1) {
-    // ---- MMA issuer ----------------------------------------------------------------------------
-    if (lane == 0) {
+    // ---- MMA issuer: the whole warp walks the loop, one elected lane issues (warp-uniform control flow keeps the
+    // descriptors in uniform registers) -----------------------------------------------------------
+    {
       const uint32_t idesc = ptx::make_idesc_bf16(BM, BN, false, false);
       const uint32_t a_base = ptx::smem_u32(sA), b_base = ptx::smem_u32(sB);
-      bool ok = ptx::mbar_wait(b_full, 0, abort_flag, g.status);
+      bool ok = __all_sync(0xFFFFFFFFu, ptx::mbar_wait(b_full, 0, abort_flag, g.status) ? 1 : 0) != 0;
       uint32_t ab = 0, aph = 0, buf = 0, cph = 1;     // A ring position / phase, accumulator ring position / phase
       for (int ti = 0; ti < my_tiles && ok; ++ti) {
-        ok = ptx::mbar_wait(&a_full[ab], aph, abort_flag, g.status);
+        ok = __all_sync(0xFFFFFFFFu, ptx::mbar_wait(&a_full[ab], aph, abort_flag, g.status) ? 1 : 0) != 0;
         const uint64_t ad = ptx::make_smem_desc(a_base + ab * A_BYTES, 16, 1024);
         for (int j = 0; j < nsub && ok; ++j) {
-          ok = ptx::mbar_wait(&acc_empty[buf], cph, abort_flag, g.status);
+          ok = __all_sync(0xFFFFFFFFu, ptx::mbar_wait(&acc_empty[buf], cph, abort_flag, g.status) ? 1 : 0) != 0;
           if (!ok) break;
           ptx::tc_fence_after();
           const uint32_t d = tmem_base + buf * BN;
           const uint64_t bd = ptx::make_smem_desc(b_base + j * (BN * 128), 16, 1024);
-          ptx::tc_mma_bf16(d, ad, bd, idesc, 0u);
+          const bool last = j + 1 == nsub;
+          if (ptx::elect_one()) {
+            ptx::tc_mma_bf16(d, ad, bd, idesc, 0u);
 #pragma unroll
-          for (int k = 1; k < BK / 16; ++k) ptx::tc_mma_bf16(d, ad + 2 * k, bd + 2 * k, idesc, 1u);
-          if (NKB > 1) {
-            const uint64_t ad1 = ad + (KB_BYTES >> 4), bd1 = bd + (uint64_t)(b_kb_bytes >> 4);
+            for (int k = 1; k < BK / 16; ++k) ptx::tc_mma_bf16(d, ad + 2 * k, bd + 2 * k, idesc, 1u);
+            if (NKB > 1) {
+              const uint64_t ad1 = ad + (KB_BYTES >> 4), bd1 = bd + (uint64_t)(b_kb_bytes >> 4);
 #pragma unroll
-            for (int k = 0; k < K1_STEPS; ++k) ptx::tc_mma_bf16(d, ad1 + 2 * k, bd1 + 2 * k, idesc, 1u);
+              for (int k = 0; k < K1_STEPS; ++k) ptx::tc_mma_bf16(d, ad1 + 2 * k, bd1 + 2 * k, idesc, 1u);
+            }
+            ptx::tc_commit(&acc_full[buf]);
+            if (last) ptx::tc_commit(&a_empty[ab]);   // every MMA that reads this A tile has been issued
           }
-          ptx::tc_commit(&acc_full[buf]);
+          __syncwarp();
           if (++buf == NACC) { buf = 0; cph ^= 1; }
         }
-        if (ok) ptx::tc_commit(&a_empty[ab]);         // every MMA that reads this A tile has been issued
         if (++ab == NA) { ab = 0; aph ^= 1; }
       }
     }

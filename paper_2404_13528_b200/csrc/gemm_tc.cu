@@ -137,7 +137,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   int* abort_flag = reinterpret_cast<int*>(tmem_slot + 1);
   uint8_t* stage_base = reinterpret_cast<uint8_t*>(tmem_slot + 4);                      // 16-byte aligned
 
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int warp = __shfl_sync(0xFFFFFFFFu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;   // (warp: provably uniform)
   const int nkb = (g.K + BK - 1) / BK;
   const int last_ksteps = (g.K - (nkb - 1) * BK + 15) / 16;
   const bool two_producers = nkb >= 8;
@@ -197,18 +197,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
+    // The whole warp walks the loop and one elected lane issues: with warp-uniform control flow the descriptors
+    // stay in uniform registers (under a branch on lane 0 each operand is moved there in front of every product).
+    {
       uint32_t it = 0, s = 0, ph = 0;                 // ring position and its phase carry over tiles
       const uint32_t a_base = ptx::smem_u32(sA), b_base = ptx::smem_u32(sB);
       bool ok = true;
       for (uint32_t t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
         const uint32_t buf = it & 1, use = it >> 1;
-        ok = ptx::mbar_wait(&tmem_empty[buf], (use & 1) ^ 1, abort_flag, g.status);   // epilogue drained it
+        ok = __all_sync(0xFFFFFFFFu, ptx::mbar_wait(&tmem_empty[buf], (use & 1) ^ 1, abort_flag, g.status) ? 1 : 0) != 0;   // epilogue drained it
         if (!ok) break;
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * ACC_COLS;
         for (int kb = 0; kb < nkb; ++kb) {
-          ok = ptx::mbar_wait(&full[s], ph, abort_flag, g.status);
+          ok = __all_sync(0xFFFFFFFFu, ptx::mbar_wait(&full[s], ph, abort_flag, g.status) ? 1 : 0) != 0;
           if (!ok) break;
           ptx::tc_fence_after();
           // K-major, 128-byte swizzle: 8-row groups are 1024 bytes apart; one k16 step is 32 bytes
@@ -219,18 +221,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                                     : ptx::make_smem_desc(a_base + s * A_STAGE_BYTES, 16, 1024);
           const uint64_t bd0 = ptx::make_smem_desc(b_base + s * B_STAGE_BYTES, 16, 1024);
           constexpr uint64_t A_STEP = (A_MN ? 2048 : 32) >> 4, B_STEP = 32 >> 4;
-          if (kb != nkb - 1 || last_ksteps == BK / 16) {
-            ptx::tc_mma_bf16(d_tmem, ad0, bd0, IDESC, kb ? 1u : 0u);
+          const bool last_kb = kb == nkb - 1;
+          if (ptx::elect_one()) {
+            if (!last_kb || last_ksteps == BK / 16) {
+              ptx::tc_mma_bf16(d_tmem, ad0, bd0, IDESC, kb ? 1u : 0u);
 #pragma unroll
-            for (int k = 1; k < BK / 16; ++k) ptx::tc_mma_bf16(d_tmem, ad0 + k * A_STEP, bd0 + k * B_STEP, IDESC, 1u);
-          } else {
-            for (int k = 0; k < last_ksteps; ++k)
-              ptx::tc_mma_bf16(d_tmem, ad0 + k * A_STEP, bd0 + k * B_STEP, IDESC, (kb | k) ? 1u : 0u);
+              for (int k = 1; k < BK / 16; ++k) ptx::tc_mma_bf16(d_tmem, ad0 + k * A_STEP, bd0 + k * B_STEP, IDESC, 1u);
+            } else {
+              for (int k = 0; k < last_ksteps; ++k)
+                ptx::tc_mma_bf16(d_tmem, ad0 + k * A_STEP, bd0 + k * B_STEP, IDESC, (kb | k) ? 1u : 0u);
+            }
+            ptx::tc_commit(&empty[s]);
+            if (last_kb) ptx::tc_commit(&tmem_full[buf]);
           }
-          ptx::tc_commit(&empty[s]);
+          __syncwarp();
           if (++s == STAGES) { s = 0; ph ^= 1; }
         }
-        if (ok) ptx::tc_commit(&tmem_full[buf]);
       }
     }
   } else if (warp >= 2 + kEpiWarps) {
