@@ -50,8 +50,7 @@ typedef enum {
   SMARTMEM_ERR_WORKSPACE = -4,   /* workspace too small                                  */
   SMARTMEM_ERR_ALIGNMENT = -5,   /* a base pointer is not 16-byte aligned                */
   SMARTMEM_ERR_CUDA = -6,        /* a CUDA runtime/driver call failed (or no device)     */
-  SMARTMEM_ERR_TIMEOUT = -7,     /* a bounded device-side wait ran out                   */
-  SMARTMEM_ERR_BOUNDS = -8       /* debug bounds check tripped                           */
+  SMARTMEM_ERR_TIMEOUT = -7      /* a bounded device-side wait ran out                   */
 } smartmem_status_t;
 
 typedef enum { SMARTMEM_F32 = 0, SMARTMEM_BF16 = 1 } smartmem_dtype_t;
@@ -319,9 +318,17 @@ int smartmem_attn_decode_workspace_bytes(const smartmem_attn_params_t* p, int32_
 int smartmem_attn_decode(const smartmem_attn_params_t* p, int32_t pos, const void* x, void* k_cache, void* v_cache,
                          void* y, void* workspace, size_t workspace_bytes, int32_t mode, void* cuda_stream);
 
-/* Synchronises the stream and returns the device status word (SMARTMEM_OK, _TIMEOUT or _BOUNDS)
+/* Synchronises the stream and returns the device status word (SMARTMEM_OK, _TIMEOUT or _UNSUPPORTED)
  * in *status, then clears it. */
 int smartmem_last_device_status(void* cuda_stream, int32_t* status);
+/* Limit, in nanoseconds, of every bounded device-side wait of the current device (default 1e9, at most 6e10).
+ * A wait that runs out makes its kernel unwind and return normally with SMARTMEM_ERR_TIMEOUT in the device
+ * status word.  Synchronises the device.  SMARTMEM_ERR_INVALID_ARG for 0 or more than 60 s. */
+int smartmem_set_wait_limit_ns(uint64_t limit_ns);
+/* Self-test of that unwind: launches one warp that waits, through the kernels' own bounded wait, on a barrier
+ * nothing arrives at.  After the wait limit the kernel returns; smartmem_last_device_status() then reports
+ * SMARTMEM_ERR_TIMEOUT and the context stays usable.  No memory is touched besides the status word. */
+int smartmem_selftest_bounded_wait(void* cuda_stream);
 /* Number of kernels this library has launched since it was loaded (for benchmark accounting). */
 int64_t smartmem_launch_count(void);
 const char* smartmem_status_string(int32_t status);

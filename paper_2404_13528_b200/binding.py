@@ -16,7 +16,7 @@ LIB_PATH = os.path.join(_HERE, "libsmartmem.so")
 MAX_DIMS, MAX_ATOMS, MAX_ROLLS = 8, 16, 4
 OK = 0
 ERR_INVALID_ARG, ERR_SHAPE, ERR_UNSUPPORTED, ERR_WORKSPACE = -1, -2, -3, -4
-ERR_ALIGNMENT, ERR_CUDA, ERR_TIMEOUT, ERR_BOUNDS = -5, -6, -7, -8
+ERR_ALIGNMENT, ERR_CUDA, ERR_TIMEOUT = -5, -6, -7
 F32, BF16 = 0, 1
 ELIMINATE, EXPLICIT, ELIMINATE_NAIVE, ELIMINATE_GATHER, ELIMINATE_SCATTER, ELIMINATE_UNFUSED = 0, 1, 2, 3, 4, 5
 OP_RESHAPE, OP_TRANSPOSE, OP_ROLL, OP_SLICE, OP_WINDOW_PARTITION, OP_WINDOW_REVERSE = 0, 1, 2, 3, 4, 5
@@ -66,7 +66,7 @@ EXPORTED = [
     "smartmem_plan_workspace_bytes", "smartmem_map_eval", "smartmem_plan_eval_sequential", "smartmem_run_chain",
     "smartmem_swin_block_workspace_bytes", "smartmem_swin_block", "smartmem_swin_block_half", "smartmem_attn_layer_workspace_bytes",
     "smartmem_attn_layer", "smartmem_attn_decode_workspace_bytes", "smartmem_attn_decode", "smartmem_swin_block_timed", "smartmem_swin_block_static_scratch_bytes",
-    "smartmem_swin_block_noalloc", "smartmem_profile_begin", "smartmem_profile_end", "smartmem_last_device_status", "smartmem_launch_count", "smartmem_status_string",
+    "smartmem_swin_block_noalloc", "smartmem_profile_begin", "smartmem_profile_end", "smartmem_last_device_status", "smartmem_set_wait_limit_ns", "smartmem_selftest_bounded_wait", "smartmem_launch_count", "smartmem_status_string",
 ]
 
 _lib = None
@@ -110,6 +110,8 @@ def lib() -> C.CDLL:
         "smartmem_profile_begin": (C.c_int, []),
         "smartmem_profile_end": (C.c_int, [vp, P(C.c_float), C.c_char_p, i32, i32, P(i32)]),
         "smartmem_last_device_status": (C.c_int, [vp, P(i32)]),
+        "smartmem_set_wait_limit_ns": (C.c_int, [C.c_uint64]),
+        "smartmem_selftest_bounded_wait": (C.c_int, [vp]),
         "smartmem_launch_count": (i64, []),
         "smartmem_status_string": (C.c_char_p, [i32]),
     }
@@ -324,6 +326,14 @@ def smartmem_last_device_status(stream: int) -> int:
     s = C.c_int32()
     _check(lib().smartmem_last_device_status(stream, C.byref(s)), "smartmem_last_device_status")
     return s.value
+
+
+def smartmem_set_wait_limit_ns(limit_ns: int) -> None:
+    _check(lib().smartmem_set_wait_limit_ns(int(limit_ns)), "smartmem_set_wait_limit_ns")
+
+
+def smartmem_selftest_bounded_wait(stream: int) -> None:
+    _check(lib().smartmem_selftest_bounded_wait(stream), "smartmem_selftest_bounded_wait")
 
 
 def smartmem_launch_count() -> int:

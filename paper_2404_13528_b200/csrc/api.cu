@@ -8,6 +8,7 @@
 #include "common.cuh"
 #include "gemm_tc.cuh"
 #include "plan.hpp"
+#include "ptx.cuh"
 
 #define EXPORT extern "C" __attribute__((visibility("default")))
 
@@ -30,7 +31,8 @@ void profile_tick(const char* name, cudaStream_t st) {
   g_prof_names.push_back(name);
 }
 
-__device__ int g_status_word;
+// Status block of the device: word 0 the status, words 2-3 the limit (ns) of every bounded device-side wait.
+__device__ __align__(16) int g_status_word[4];
 
 // Both caches below are per device: the address of a __device__ symbol and a kernel's attributes belong to the
 // context of the device that was current when they were looked up or set.
@@ -45,7 +47,9 @@ int* device_status_ptr() {
   if (!g_status_ptr[dev]) {
     void* q = nullptr;
     if (cudaGetSymbolAddress(&q, g_status_word) != cudaSuccess || !q) return nullptr;
-    if (cudaMemset(q, 0, sizeof(int)) != cudaSuccess) return nullptr;
+    const unsigned long long limit = smartmem::ptx::kWaitLimitNs;
+    if (cudaMemset(q, 0, 4 * sizeof(int)) != cudaSuccess) return nullptr;
+    if (cudaMemcpy((int*)q + 2, &limit, sizeof(limit), cudaMemcpyHostToDevice) != cudaSuccess) return nullptr;
     g_status_ptr[dev] = (int*)q;
   }
   return g_status_ptr[dev];
@@ -116,6 +120,40 @@ EXPORT int smartmem_last_device_status(void* cuda_stream, int32_t* status) {
   if (v != 0) cudaMemsetAsync(p, 0, sizeof(int), st);
   *status = v;
   return SMARTMEM_OK;
+}
+
+namespace {
+// A wait that nothing will ever satisfy, through the same bounded wait the kernels use: one warp waits on
+// a barrier that expects an arrival which never comes.  The wait gives up after the device's wait limit,
+// raises SMARTMEM_ERR_TIMEOUT in the status word and the kernel returns normally.
+__global__ void selftest_wait_kernel(int* status) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(&bar, 1);
+    abort_flag = 0;
+    ptx::fence_barrier_init();
+  }
+  __syncthreads();
+  ptx::mbar_wait(&bar, 0, &abort_flag, status);
+}
+}  // namespace
+
+extern "C" int smartmem_set_wait_limit_ns(uint64_t limit_ns) {
+  int* p = device_status_ptr();
+  if (!p) return SMARTMEM_ERR_CUDA;
+  if (limit_ns == 0 || limit_ns > 60000000000ull) return SMARTMEM_ERR_INVALID_ARG;
+  const unsigned long long v = limit_ns;
+  if (cudaDeviceSynchronize() != cudaSuccess) return SMARTMEM_ERR_CUDA;       // no kernel reads the limit while it changes
+  return cudaMemcpy(p + 2, &v, sizeof(v), cudaMemcpyHostToDevice) == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
+}
+
+extern "C" int smartmem_selftest_bounded_wait(void* cuda_stream) {
+  int* p = device_status_ptr();
+  if (!p) return SMARTMEM_ERR_CUDA;
+  selftest_wait_kernel<<<1, 32, 0, (cudaStream_t)cuda_stream>>>(p);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
 }
 
 namespace {

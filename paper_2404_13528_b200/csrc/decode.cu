@@ -254,17 +254,17 @@ typedef std::tuple<int, int, int> DKey;
 std::mutex g_mu;
 std::map<DKey, smartmem_index_map_t> g_split;
 
-int get_split(int B, int H, int D, const smartmem_index_map_t** out) {
+int get_split(int B, int H, int D, smartmem_index_map_t* out) {   // (a copy: clearing the cache cannot invalidate it)
   DKey key(B, H, D);
   std::lock_guard<std::mutex> lk(g_mu);
   auto it = g_split.find(key);
-  if (it != g_split.end()) { *out = &it->second; return SMARTMEM_OK; }
+  if (it != g_split.end()) { *out = it->second; return SMARTMEM_OK; }
   smartmem_index_map_t m;
   const int64_t b = B, h = H, d = D;
   int rc = chain_map({b, 1, 3 * h * d}, {op_reshape({b, 1, 3, h, d}), op_transpose({2, 0, 3, 1, 4})}, SMARTMEM_BF16, &m);
   if (rc != SMARTMEM_OK) return rc;
   if (g_split.size() > 64) g_split.clear();
-  *out = &g_split.emplace(key, m).first->second;
+  *out = g_split.emplace(key, m).first->second;
   return SMARTMEM_OK;
 }
 
@@ -369,9 +369,9 @@ EXPORT int smartmem_attn_decode(const smartmem_attn_params_t* pp, int32_t pos, c
     a.q_sb = hid; a.q_sh = DH;
     a.kv_sb = Smax * hid; a.kv_sh = DH; a.kv_ss = hid;
   } else {
-    const smartmem_index_map_t* split = nullptr;
+    smartmem_index_map_t split;
     SM_TRY(get_split(p.B, p.heads, DH, &split));
-    SM_TRY(launch_copy_map(*split, 2, at(L.qkv), at(L.split), st));
+    SM_TRY(launch_copy_map(split, 2, at(L.qkv), at(L.split), st));
     __nv_bfloat16* sp = (__nv_bfloat16*)at(L.split);
     SM_TRY(launch_rope_rows_at(sp, 2 * B * H, pos, p.rope_theta, p.rotary_dim ? p.rotary_dim : DH, st));
     SM_TRY(launch_append_rows(sp + B * hid, kc + (long long)pos * DH, B * H, Smax * DH, "append_k", st));

@@ -7,6 +7,7 @@
 // EXPLICIT: the same kernels with a plain QKV epilogue, a head-split copy to [3, B, H, S, D], a
 // separate rotary pass over q and k, attention on the materialised tensors, a head-merge copy.
 #include <map>
+#include <memory>
 #include <mutex>
 #include <tuple>
 
@@ -26,13 +27,13 @@ struct LlamaMaps {
 };
 typedef std::tuple<int, int, int, int> LKey;
 std::mutex g_mu;
-std::map<LKey, LlamaMaps> g_maps;
+std::map<LKey, std::shared_ptr<const LlamaMaps>> g_maps;   // entries are handed out by shared pointer: clearing the cache never invalidates a caller's copy
 
-int get_maps(const smartmem_attn_params_t& p, const LlamaMaps** out) {
+int get_maps(const smartmem_attn_params_t& p, std::shared_ptr<const LlamaMaps>* out) {
   LKey key(p.B, p.S, p.heads, p.head_dim);
   std::lock_guard<std::mutex> lk(g_mu);
   auto it = g_maps.find(key);
-  if (it != g_maps.end()) { *out = &it->second; return SMARTMEM_OK; }
+  if (it != g_maps.end()) { *out = it->second; return SMARTMEM_OK; }
   LlamaMaps m;
   const int64_t B = p.B, S = p.S, H = p.heads, D = p.head_dim;
   int rc;
@@ -41,7 +42,7 @@ int get_maps(const smartmem_attn_params_t& p, const LlamaMaps** out) {
   if ((rc = chain_map({B, H, S, D}, {op_transpose({0, 2, 1, 3}), op_reshape({B, S, H * D})}, SMARTMEM_BF16, &m.merge)))
     return rc;
   if (g_maps.size() > 64) g_maps.clear();
-  *out = &g_maps.emplace(key, m).first->second;
+  *out = g_maps.emplace(key, std::make_shared<const LlamaMaps>(m)).first->second;
   return SMARTMEM_OK;
 }
 
@@ -102,7 +103,7 @@ EXPORT int smartmem_attn_layer(const smartmem_attn_params_t* pp, const void* x, 
   if (workspace_bytes < L.total) return SMARTMEM_ERR_WORKSPACE;
   int ndev = 0;
   if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) return SMARTMEM_ERR_CUDA;
-  const LlamaMaps* mp = nullptr;
+  std::shared_ptr<const LlamaMaps> mp;
   if ((rc = get_maps(p, &mp)) != SMARTMEM_OK) return rc;
 
   cudaStream_t st = (cudaStream_t)cuda_stream;

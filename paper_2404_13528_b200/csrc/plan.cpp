@@ -921,7 +921,6 @@ const char* smartmem_status_string(int32_t s) {
     case SMARTMEM_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
     case SMARTMEM_ERR_CUDA: return "CUDA error or no device";
     case SMARTMEM_ERR_TIMEOUT: return "device-side wait timed out";
-    case SMARTMEM_ERR_BOUNDS: return "device-side bounds check failed";
   }
   return "unknown status";
 }

@@ -12,7 +12,8 @@
 namespace smartmem {
 namespace ptx {
 
-constexpr unsigned long long kWaitLimitNs = 1000000000ull;   // 1 s
+constexpr unsigned long long kWaitLimitNs = 1000000000ull;   // 1 s: the default; the limit in force sits behind the status word
+// (words 2-3 of the device's status block), where the host can change it
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -62,6 +63,9 @@ __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+__device__ __forceinline__ unsigned long long wait_limit_ns(const int* status) {
+  return *reinterpret_cast<const volatile unsigned long long*>(status + 2);
+}
 // Bounded wait.  Returns false if it gave up (or another role already did).
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
   if (mbar_try_wait(bar, parity)) return true;
@@ -71,7 +75,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     if (mbar_try_wait(bar, parity)) return true;
     if ((++polls & 63u) == 0) {
       if (*abort_flag) return false;
-      if (globaltimer() - t0 > kWaitLimitNs) {
+      if (globaltimer() - t0 > wait_limit_ns(status)) {
         *abort_flag = 1;
         atomicExch(status, (int)SMARTMEM_ERR_TIMEOUT);
         return false;
@@ -93,7 +97,7 @@ __device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, uint32_t parity
     if (mbar_try_wait(bar, parity)) return true;
     if ((++polls & 15u) == 0) {
       if (*abort_flag) return false;
-      if (globaltimer() - t0 > kWaitLimitNs) {
+      if (globaltimer() - t0 > wait_limit_ns(status)) {
         *abort_flag = 1;
         atomicExch(status, (int)SMARTMEM_ERR_TIMEOUT);
         return false;

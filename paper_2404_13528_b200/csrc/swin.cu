@@ -8,6 +8,7 @@
 // EXPLICIT: the same compute kernels with identity maps, and one copy kernel per layout
 // operator (shift, partition, head split, K transpose, head merge, window reverse, unshift).
 #include <map>
+#include <memory>
 #include <mutex>
 #include <tuple>
 #include <vector>
@@ -30,14 +31,14 @@ struct SwinMaps {
 
 typedef std::tuple<int, int, int, int, int, int, int, int> SwinKey;
 std::mutex g_mu;
-std::map<SwinKey, SwinMaps> g_maps;
+std::map<SwinKey, std::shared_ptr<const SwinMaps>> g_maps;   // entries are handed out by shared pointer: clearing the cache never invalidates a caller's copy
 
-int get_maps(const smartmem_swin_params_t& p, const SwinMaps** out) {
+int get_maps(const smartmem_swin_params_t& p, std::shared_ptr<const SwinMaps>* out) {
   SwinKey key(p.dtype, p.B, p.H, p.W, p.C, p.heads, p.window, p.shift);
   std::lock_guard<std::mutex> lk(g_mu);
   auto it = g_maps.find(key);
   if (it != g_maps.end()) {
-    *out = &it->second;
+    *out = it->second;
     return SMARTMEM_OK;
   }
   SwinMaps m;
@@ -75,8 +76,7 @@ int get_maps(const smartmem_swin_params_t& p, const SwinMaps** out) {
   if (n < 2 || m.e1.extent[n - 1] != C || m.e1.src_stride[n - 1] != 1 || m.e1.klass == 3) return SMARTMEM_ERR_UNSUPPORTED;
   if (!make_devmap(m.e1, 0, n - 1, 1, true, &m.e1_rows)) return SMARTMEM_ERR_UNSUPPORTED;
   if (g_maps.size() > 64) g_maps.clear();
-  auto ins = g_maps.emplace(key, m);
-  *out = &ins.first->second;
+  *out = g_maps.emplace(key, std::make_shared<const SwinMaps>(m)).first->second;
   return SMARTMEM_OK;
 }
 
@@ -196,7 +196,7 @@ int run_block(const smartmem_swin_params_t* pp, const void* x, void* y, void* wo
   if (workspace_bytes < L.total) return SMARTMEM_ERR_WORKSPACE;
   int ndev = 0;
   if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) return SMARTMEM_ERR_CUDA;
-  const SwinMaps* mp = nullptr;
+  std::shared_ptr<const SwinMaps> mp;
   if ((rc = get_maps(p, &mp)) != SMARTMEM_OK) return rc;
   const SwinMaps& m = *mp;
 

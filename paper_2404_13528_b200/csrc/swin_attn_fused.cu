@@ -749,7 +749,7 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
           if (__any_sync(0xFFFFFFFFu, *(volatile int*)abort_flag)) break;
           const unsigned long long now = __shfl_sync(0xFFFFFFFFu, ptx::globaltimer(), 0);
           if (idle == 256u) t_idle = now;
-          else if (now - t_idle > ptx::kWaitLimitNs) {
+          else if (now - t_idle > ptx::wait_limit_ns(g.status)) {
             if (lane == 0) {
               *abort_flag = 1;
               atomicExch(g.status, (int)SMARTMEM_ERR_TIMEOUT);
