@@ -702,8 +702,14 @@ int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep,
   // tile width: the widest of {256, 128, 96, 64} that divides N (fewest wasted columns), else 128
   int bn = 128;
   if (ep.rope_cols > 0) bn = (M <= BM && batch == 1 && N / 256 < tc_sm_count()) ? 128 : 256;   // one head or two per tile
-  else if (N % 256 == 0) bn = 256;
-  else if (N % 128 == 0) bn = 128;
+  else if (N % 256 == 0) {
+    // 256 or 128 wide: whichever leaves fewer idle SMs in the last wave (time of a wave ~ tile width plus a fixed part).
+    // Only for short reductions: a 128-wide tile reads as many operand bytes per product as shared memory delivers,
+    // so over a long K the wider tile wins even with a ragged last wave (measured at K = 2048).
+    const long long tm = (M + BM - 1) / BM * batch, sms = tc_sm_count();
+    const long long w256 = (tm * (N / 256) + sms - 1) / sms, w128 = (tm * (N / 128) + sms - 1) / sms;
+    bn = (K <= 1024 && w128 * (128 + 48) < w256 * (256 + 48)) ? 128 : 256;
+  } else if (N % 128 == 0) bn = 128;
   else if (N % 96 == 0) bn = 96;
   else if (N % 64 == 0) bn = 64;
   // One row tile only (a decode step: M <= 128) and few wide column tiles: the GEMM streams the weight
