@@ -191,7 +191,62 @@ def run_reference(args):
 # The other configurations (parity-test cases): timed on request with --workload, same protocol.
 # ------------------------------------------------------------------------------------------------
 OTHER_WORKLOADS = ["swin_b_stage3_block_pair", "llama_attention_layer", "llama_decode_layer", "chain_2a_qkt", "chain_2b_gemm",
-                   "chain_2a_copy", "chain_2b_copy", "swin_shift_partition_copy", "depth_to_space_copy", "swin_t_patch_merging", "swin_t_stage1", "nchw_layernorm_linear"]
+                   "chain_2a_copy", "chain_2b_copy", "swin_shift_partition_copy", "depth_to_space_copy", "swin_t_patch_merging", "swin_t_stage1", "nchw_layernorm_linear", "fanout_two_consumers"]
+
+
+def run_fanout(args, n_steps):
+    """A producer with two consumers of different reduction dimensions (Section 3.2.2, "Global"): one copy of the
+    producer's result read two ways, two copies written by the producer's epilogue, and the explicit variant (default
+    layout + a transposing copy kernel).  Reports the time of each and the bytes of the result written / copied."""
+    import torch
+    from paper_2404_13528_b200 import binding as sm
+    from paper_2404_13528_b200 import synth
+
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    stream = torch.cuda.current_stream().cuda_stream
+    B, S, K, N, Na, Nb = 32, 512, 512, 1024, 512, 256
+
+    def dev(a):
+        return torch.from_numpy(a.view("int16").copy()).cuda().view(torch.bfloat16)
+
+    x = dev(synth.normal(91, 0, (B * S, K), dtype="bf16"))
+    w = [dev(synth.normal(91, 1 + i, shp, std=shp[1] ** -0.5, dtype="bf16")) for i, shp in enumerate(((N, K), (Na, N), (Nb, S)))]
+    sets = 4                                             # rotating buffers: x, P (x2), YA, YB of a set are 100 MB; four sets exceed L2
+    xs = [x.clone() for _ in range(sets)]
+    yas = [torch.empty(B * S, Na, dtype=torch.bfloat16, device="cuda") for _ in range(sets)]
+    ybs = [torch.empty(B, N, Nb, dtype=torch.bfloat16, device="cuda") for _ in range(sets)]
+    variants = (("one_copy", sm.ELIMINATE, 2), ("two_copies_by_the_producer", sm.ELIMINATE, 1), ("explicit", sm.EXPLICIT, 1))
+    out = {"workload": "fanout_two_consumers", "shape": {"B": B, "S": S, "K": K, "N": N, "Na": Na, "Nb": Nb}, "steps": n_steps,
+           "l2": f"{sets} rotating buffer sets", "variants": {}}
+    for name, mode, k in variants:
+        p = sm.FanoutParams()
+        p.B, p.S, p.K, p.N, p.Na, p.Nb, p.k_contig = B, S, K, N, Na, Nb, k
+        p.w_p, p.w_a, p.w_b = (t.data_ptr() for t in w)
+        info = sm.smartmem_fanout_plan(p, mode)
+        wss = [torch.empty(info["workspace_bytes"], dtype=torch.uint8, device="cuda") for _ in range(sets)]
+
+        def step(i):
+            j = i % sets
+            sm.smartmem_fanout(p, xs[j].data_ptr(), yas[j].data_ptr(), ybs[j].data_ptr(), wss[j].data_ptr(), info["workspace_bytes"], mode, stream)
+
+        for i in range(max(args.warmup, 3)):
+            step(i)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(n_steps):
+            step(i)
+        e1.record()
+        torch.cuda.synchronize()
+        if sm.smartmem_last_device_status(stream) != sm.OK:
+            raise SystemExit("device status not OK")
+        out["variants"][name] = {"ms_per_step": e0.elapsed_time(e1) / n_steps, "copies_of_the_result_written": info["copies_written"],
+                                 "producer_bytes_written": info["producer_bytes_written"], "copy_kernel_bytes": info["copy_kernel_bytes"]}
+        del wss
+    v = out["variants"]
+    out["explicit_over_one_copy"] = v["explicit"]["ms_per_step"] / v["one_copy"]["ms_per_step"]
+    out["explicit_over_two_copies"] = v["explicit"]["ms_per_step"] / v["two_copies_by_the_producer"]["ms_per_step"]
+    return out
 
 
 def _peaks_all():
@@ -536,6 +591,9 @@ def main():
     if args.impl == "reference":
         return run_reference(args)
     args.warmup = max(args.warmup, 3)
+    if args.workload == "fanout_two_consumers":
+        print(json.dumps(run_fanout(args, args.steps)))
+        return
     if args.workload != WORKLOAD["name"]:
         print(json.dumps(run_other(args, args.workload, args.steps)))
         return
@@ -747,6 +805,7 @@ def main():
                            "explicit_speedup": r["explicit_variant"]["speedup_of_eliminate"], "steps": k,
                            "roofline": {kk: r["roofline"][kk] for kk in ("kernel", "bound", "frac", "achieved", "unit")},
                            "kernels": [{"kernel": q["kernel"], "ms": q["ms"], "bound": q["bound"], "frac": q["frac"]} for q in r["kernels"]]})
+        others.append(run_fanout(args, 30))
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

@@ -321,6 +321,33 @@ int smartmem_attn_decode(const smartmem_attn_params_t* p, int32_t pos, const voi
 /* Synchronises the stream and returns the device status word (SMARTMEM_OK, _TIMEOUT or _UNSUPPORTED)
  * in *status, then clears it. */
 int smartmem_last_device_status(void* cuda_stream, int32_t* status);
+/* ---- A producer with two consumers of different reduction dimensions (Section 3.2.2, "Global: layout
+ * selections based on reduction dimension", and the redundant-copy remark in the discussion of the evaluation).
+ *   P  = X Wp^T           X [B*S, K], Wp [N, K]; P is the tensor [B, S, N]
+ *   YA = P Wa^T           Wa [Na, N]: aggregates along N (dimension 2 of P);          YA [B*S, Na]
+ *   YB[b] = P[b]^T Wb^T   Wb [Nb, S]: aggregates along S (dimension 1 of P);          YB [B, N, Nb]
+ * bf16, device pointers, every extent a multiple of 8.  k_contig is the k of smartmem_select_layouts: with
+ * k_contig = 2 the planner keeps ONE copy of P in [B, S, N] and consumer B reads it with S as its reduction
+ * dimension through a tiled (TMA) operand; with k_contig = 1 it asks for two copies and the producer's epilogue
+ * writes [B, S, N] and [B, N, S].  SMARTMEM_EXPLICIT writes [B, S, N] and transposes it with a copy kernel.
+ * The three variants give identical YA; YB is identical between k_contig = 1 and EXPLICIT. */
+typedef struct {
+  int32_t B, S, K, N, Na, Nb;
+  int32_t k_contig;                 /* 1 or 2 (ignored by SMARTMEM_EXPLICIT) */
+  const void *w_p, *w_a, *w_b;      /* device, bf16 */
+} smartmem_fanout_params_t;
+/* What the planner decided (host only; any output pointer may be null): copies of P written in total, the layout
+ * consumer B reads (0: [B,S,N], 1: [B,N,S]), bytes of P the producer's epilogue writes, bytes the transposing copy
+ * kernel moves (EXPLICIT only, read + write), and the workspace the call needs. */
+int smartmem_fanout_plan(const smartmem_fanout_params_t* p, int32_t mode, int32_t* n_copies_written,
+                         int32_t* layout_of_consumer_b, int64_t* producer_bytes_written, int64_t* copy_kernel_bytes,
+                         size_t* workspace_bytes);
+/* Runs producer and consumers on the stream.  x, ya, yb and the workspace are device memory owned by the caller
+ * (16-byte aligned); nothing is allocated.  Errors: INVALID_ARG (null pointer, extent < 1, mode other than
+ * ELIMINATE / EXPLICIT, k_contig outside 1..2), UNSUPPORTED (an extent that is not a multiple of 8), WORKSPACE. */
+int smartmem_fanout(const smartmem_fanout_params_t* p, const void* x, void* ya, void* yb, void* workspace,
+                    size_t workspace_bytes, int32_t mode, void* cuda_stream);
+
 /* Limit, in nanoseconds, of every bounded device-side wait of the current device (default 1e9, at most 6e10).
  * A wait that runs out makes its kernel unwind and return normally with SMARTMEM_ERR_TIMEOUT in the device
  * status word.  Synchronises the device.  SMARTMEM_ERR_INVALID_ARG for 0 or more than 60 s. */

@@ -10,7 +10,7 @@ from __future__ import annotations
 
 import numpy as np
 
-from . import layout
+from . import layout, ops
 
 
 def apply_layout_chain(x: np.ndarray, chain) -> np.ndarray:
@@ -62,3 +62,14 @@ def chain_2b_gemm(x: np.ndarray, w: np.ndarray) -> np.ndarray:
     B, C, H, W = x.shape
     a = apply_layout_chain(x, [{"op": "transpose", "perm": (0, 2, 3, 1)}, {"op": "reshape", "shape": (B * H * W, C)}])
     return a @ w.T
+
+
+def fanout(x: np.ndarray, w_p: np.ndarray, w_a: np.ndarray, w_b: np.ndarray, B: int, S: int):
+    """A producer with two consumers of different reduction dimensions (Section 3.2.2, "Global"):
+    P = x w_p^T as [B, S, N];  YA = P w_a^T aggregates along N;  YB[b] = P[b]^T w_b^T aggregates along S.
+    The layout of P is the implementation's business: the results do not depend on it.  Returns (YA [B*S, Na], YB [B, N, Nb])."""
+    P = ops.linear(x, w_p)                               # [B*S, N]
+    ya = ops.linear(P, w_a)
+    P3 = layout.reshape(P, (B, S, P.shape[1]))
+    yb = np.stack([layout.transpose(P3[b], (1, 0)) @ w_b.T for b in range(B)])
+    return ya, yb

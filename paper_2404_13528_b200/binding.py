@@ -53,6 +53,11 @@ class SwinParams(C.Structure):
                                           "ln2_g", "ln2_b", "w_fc1", "b_fc1", "w_fc2", "b_fc2")]
 
 
+class FanoutParams(C.Structure):
+    _fields_ = [("B", C.c_int32), ("S", C.c_int32), ("K", C.c_int32), ("N", C.c_int32), ("Na", C.c_int32), ("Nb", C.c_int32),
+                ("k_contig", C.c_int32), ("w_p", C.c_void_p), ("w_a", C.c_void_p), ("w_b", C.c_void_p)]
+
+
 class AttnParams(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("dtype", "B", "S", "hidden", "heads", "head_dim", "causal", "add_residual")] + \
                [("rms_eps", C.c_float), ("rope_theta", C.c_float)] + \
@@ -66,7 +71,7 @@ EXPORTED = [
     "smartmem_plan_workspace_bytes", "smartmem_map_eval", "smartmem_plan_eval_sequential", "smartmem_run_chain",
     "smartmem_swin_block_workspace_bytes", "smartmem_swin_block", "smartmem_swin_block_half", "smartmem_attn_layer_workspace_bytes",
     "smartmem_attn_layer", "smartmem_attn_decode_workspace_bytes", "smartmem_attn_decode", "smartmem_swin_block_timed", "smartmem_swin_block_static_scratch_bytes",
-    "smartmem_swin_block_noalloc", "smartmem_profile_begin", "smartmem_profile_end", "smartmem_last_device_status", "smartmem_set_wait_limit_ns", "smartmem_selftest_bounded_wait", "smartmem_launch_count", "smartmem_status_string",
+    "smartmem_swin_block_noalloc", "smartmem_profile_begin", "smartmem_profile_end", "smartmem_last_device_status", "smartmem_set_wait_limit_ns", "smartmem_selftest_bounded_wait", "smartmem_fanout_plan", "smartmem_fanout", "smartmem_launch_count", "smartmem_status_string",
 ]
 
 _lib = None
@@ -112,6 +117,8 @@ def lib() -> C.CDLL:
         "smartmem_last_device_status": (C.c_int, [vp, P(i32)]),
         "smartmem_set_wait_limit_ns": (C.c_int, [C.c_uint64]),
         "smartmem_selftest_bounded_wait": (C.c_int, [vp]),
+        "smartmem_fanout_plan": (C.c_int, [P(FanoutParams), i32, P(i32), P(i32), P(C.c_int64), P(C.c_int64), P(C.c_size_t)]),
+        "smartmem_fanout": (C.c_int, [P(FanoutParams), vp, vp, vp, vp, C.c_size_t, i32, vp]),
         "smartmem_launch_count": (i64, []),
         "smartmem_status_string": (C.c_char_p, [i32]),
     }
@@ -334,6 +341,18 @@ def smartmem_set_wait_limit_ns(limit_ns: int) -> None:
 
 def smartmem_selftest_bounded_wait(stream: int) -> None:
     _check(lib().smartmem_selftest_bounded_wait(stream), "smartmem_selftest_bounded_wait")
+
+
+def smartmem_fanout_plan(p: FanoutParams, mode: int) -> dict:
+    n, lb, pb, cb, ws = C.c_int32(), C.c_int32(), C.c_int64(), C.c_int64(), C.c_size_t()
+    _check(lib().smartmem_fanout_plan(C.byref(p), mode, C.byref(n), C.byref(lb), C.byref(pb), C.byref(cb), C.byref(ws)),
+           "smartmem_fanout_plan")
+    return {"copies_written": n.value, "layout_of_consumer_b": lb.value, "producer_bytes_written": pb.value,
+            "copy_kernel_bytes": cb.value, "workspace_bytes": ws.value}
+
+
+def smartmem_fanout(p: FanoutParams, x: int, ya: int, yb: int, workspace: int, workspace_bytes: int, mode: int, stream: int):
+    _check(lib().smartmem_fanout(C.byref(p), x, ya, yb, workspace, workspace_bytes, mode, stream), "smartmem_fanout")
 
 
 def smartmem_launch_count() -> int:

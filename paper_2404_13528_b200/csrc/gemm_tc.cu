@@ -55,6 +55,8 @@ struct GemmArgs {
   int seg_cols;                          // > 0: column segment s of a row goes to seg_out[s] + row * seg_ld[s]
   __nv_bfloat16* seg_out[3];
   long long seg_ld[3];
+  __nv_bfloat16* out2;                   // second copy of the result, transposed inside groups of out2_S rows (null: none)
+  FastDiv fd_out2_S;
   int* status;
   DevMap rowmap;
 };
@@ -289,6 +291,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int n0 = tile_n * BN;
       const int row = tile_m * BM + q * 32 + lane;
       const bool row_ok = row < g.M;
+      long long o2_base = 0;                                 // second copy: row = b * S + s goes to out2[b][col][s]
+      if (g.out2) {
+        const uint32_t b2 = fd_div((uint32_t)row, g.fd_out2_S);
+        o2_base = (long long)b2 * g.N * g.fd_out2_S.d + ((uint32_t)row - b2 * g.fd_out2_S.d);
+      }
       // Output offset of this thread's row (through the row map when the store is a scatter).  With
       // one round per tile the offset and the residual of the NEXT tile were requested during the
       // previous iteration, so neither the map evaluation nor the gather's latency is on the path
@@ -424,6 +431,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
           }
           if (rd + 1 < ROUNDS) fetch_res(col_of(rd + 1));
+        }
+        if (g.out2 && row_ok) {
+          // The redundant copy of a producer with consumers of different reduction dimensions: the same values with the
+          // row's position inside its group as the contiguous dimension.  A warp's 32 rows write 64 contiguous bytes per column.
+#pragma unroll
+          for (int j = 0; j < RC; ++j)
+            if (n0 + c0 + j < g.N) g.out2[o2_base + (long long)(n0 + c0 + j) * g.fd_out2_S.d] = __float2bfloat16_rn(acc[j]);
         }
 #pragma unroll
         for (int v = 0; v < VPR; ++v) {
@@ -715,6 +729,7 @@ int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep,
   // One row tile only (a decode step: M <= 128) and few wide column tiles: the GEMM streams the weight
   // once and is bound by how many SMs pull on it, so take the narrowest tile that divides N.
   if (ep.rope_cols == 0 && batch == 1 && M <= BM && !a_mn && N % 64 == 0 && N / bn < tc_sm_count()) bn = 64;
+  if (a_mn && bn < 128) bn = 128;                         // MN-major A operands come with 128- and 256-wide tiles only
   if (ep.rope_cols > 0 && (N % 256 || ep.rope_cols % 256 || ep.rope_S < 1)) return SMARTMEM_ERR_UNSUPPORTED;
   if (ep.rope_cols > 0 && ep.rope_dim != 0 && ep.rope_dim != 32 && ep.rope_dim != 64 && ep.rope_dim != 128) return SMARTMEM_ERR_UNSUPPORTED;
   if (ep.seg_cols > 0) {
@@ -750,6 +765,11 @@ int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep,
   const int rope_dim = ep.rope_dim ? ep.rope_dim : 128;
   g.rope_half = rope_dim / 2;
   g.rope_c = ep.rope_log2_theta / (float)(rope_dim / 2);
+  if (ep.out2) {
+    if (ep.out2_S < 1 || M % ep.out2_S || batch != 1 || ((uintptr_t)ep.out2 & 1)) return SMARTMEM_ERR_UNSUPPORTED;
+    g.out2 = (__nv_bfloat16*)ep.out2;
+    g.fd_out2_S = make_fastdiv((uint32_t)ep.out2_S);
+  }
   g.status = device_status_ptr();
   if (!g.status) return SMARTMEM_ERR_CUDA;
   g.tiles_n = (int)((N + bn - 1) / bn);

@@ -37,6 +37,11 @@ struct TcEpilogue {
   int seg_cols;
   void* seg_out[3];
   long long seg_ld[3];
+  // Second copy of the result (null: none) for a consumer whose reduction dimension is the row index inside groups of
+  // out2_S rows: element (row, col) also goes to out2[(row / out2_S) * N * out2_S + col * out2_S + row % out2_S].
+  // batch == 1, M a multiple of out2_S.
+  void* out2;
+  long long out2_S;
 };
 
 int tc_operand_from_map(const smartmem_index_map_t& m, int n_batch_atoms, int n_row_atoms, const void* ptr,
