@@ -151,8 +151,12 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
 
   const int tid = threadIdx.x, lane = tid & 31;
   const int warp = __shfl_sync(0xFFFFFFFFu, tid >> 5, 0);   // (provably warp-uniform: the issuing code below keeps its operands in uniform registers)
-  const int cidx = blockIdx.x, cstride = gridDim.x;
-  const int U = cidx < g.n_pairs ? (g.n_pairs - cidx + cstride - 1) / cstride : 0;   // units of this CTA
+  // A CTA takes a contiguous run of window pairs.  (Dealing the pairs out round-robin looks equivalent but is not: with 32 pairs
+  // per image and a stride of 148 a CTA sees the same pairs of every image, so a quarter of the CTAs got nothing but seam
+  // windows -- the slow path: gathered rows and masked scores -- and finished microseconds after the rest.)
+  const int uq = g.n_pairs / (int)gridDim.x, urem = g.n_pairs - uq * (int)gridDim.x;
+  const int U = uq + ((int)blockIdx.x < urem ? 1 : 0);                              // units of this CTA
+  const int ubase = (int)blockIdx.x * uq + ((int)blockIdx.x < urem ? (int)blockIdx.x : urem);   // its first pair
   const int total = U * NH;                                                         // items
   const float LOG2E = 1.4426950408889634f;
 
@@ -220,28 +224,6 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
   __syncthreads();
   if (tid < 32)                                       // identity: row n has a one in column n
     *reinterpret_cast<uint16_t*>(sId + sw64_off(tid, tid >> 3) + (tid & 7) * 2) = 0x3F80u;
-  // each head's bias as a [T, T] table of bf16 pairs, -inf for the padded keys; a task = a quarter of a row
-  for (int task = tid; task < NH * T * 4; task += kThreads) {
-    const int hr = task >> 2, qtr = task & 3;                       // (head, row), quarter of the row's key pairs
-    const int h = hr / T, r = hr - h * T;
-    const int ry = tyx_s[r] >> 8, rx = tyx_s[r] & 255;
-    const uint16_t* tab = raw_s + h * 256 + (ry + ws - 1) * (2 * ws - 1) + (rx + ws - 1);
-#pragma unroll 1
-    for (int c2 = qtr * (KC / 8); c2 < (qtr + 1) * (KC / 8); ++c2) {
-      uint32_t word = 0;
-#pragma unroll
-      for (int k = 0; k < 2; ++k) {
-        const int c = 2 * c2 + k;
-        uint32_t bits = 0xFF80u;                       // -inf: padded keys never contribute
-        if (c < T) {
-          const int cyx = tyx_s[c];
-          bits = tab[-(cyx >> 8) * (2 * ws - 1) - (cyx & 255)];
-        }
-        word |= bits << (16 * k);
-      }
-      bias_s[hr * BR + c2] = word;
-    }
-  }
   // keys below / right of the wrap line of a seam window (bit c = key c)
   if (warp == 2) {
     const int c0 = lane, c1 = lane + 32;
@@ -286,7 +268,7 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
     }
   }
   if (tid < 2 && U > 0 && g.split >= 0) {              // the first unit's windows under the map (parameters only)
-    const int n = 2 * cidx + tid;
+    const int n = 2 * ubase + tid;
     int4 wp = make_int4(0, 0, 0, 0);
     if (n < g.n_windows) {
       const DevMapPart pw = devmap_part_rolled(g.rowmap, 0, g.split, (uint32_t)n);
@@ -320,7 +302,7 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
     };
     auto window_part = [&](int ul) {                   // threads 0, 1: the leading atoms' contribution of the unit's two windows
       if (lt < 2 && ul < U && g.split >= 0) {
-        const int n = 2 * (cidx + ul * cstride) + lt;
+        const int n = 2 * (ubase + ul) + lt;
         int4 wp = make_int4(0, 0, 0, 0);
         if (n < g.n_windows) {
           const DevMapPart pw = devmap_part_rolled(g.rowmap, 0, g.split, (uint32_t)n);
@@ -331,7 +313,7 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
     };
     auto issue_loads = [&](int ul) {
       const int ab = ul % na;
-      const int p = cidx + ul * cstride;
+      const int p = ubase + ul;
       {                                                 // a thread per row of the pair tile: the window's kind, the row's offset
         const int w = lt >> 6, i = lt & 63, n = 2 * p + w;
         int kind = WIN_MISSING, wy = 0, wx = 0, b = 0;
@@ -481,6 +463,28 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
     uint8_t* slot_base = sKV + gi * KV_SLOT;
     const uint32_t* brow = bias_s + (gi * T + (i < T ? i : 0)) * BR;
     const f32x2 scale2 = ptx::pack2(g.scale, g.scale), log2e2 = ptx::pack2(LOG2E, LOG2E);
+    // This head's bias as a [T, T] table of bf16 pairs, -inf for the padded keys, built by the group itself while the first unit's
+    // rows are on their way (a task = a quarter of a row).  The first group barrier below orders it before the first softmax.
+    for (int task = (warp - 4 - 4 * gi) * 32 + lane; task < T * 4; task += 128) {
+      const int r = task >> 2, qtr = task & 3;                        // row, quarter of the row's key pairs
+      const int ry = tyx_s[r] >> 8, rx = tyx_s[r] & 255;
+      const uint16_t* tab = raw_s + gi * 256 + (ry + ws - 1) * (2 * ws - 1) + (rx + ws - 1);
+#pragma unroll 1
+      for (int c2 = qtr * (KC / 8); c2 < (qtr + 1) * (KC / 8); ++c2) {
+        uint32_t word = 0;
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+          const int c = 2 * c2 + k;
+          uint32_t bits = 0xFF80u;                       // -inf: padded keys never contribute
+          if (c < T) {
+            const int cyx = tyx_s[c];
+            bits = tab[-(cyx >> 8) * (2 * ws - 1) - (cyx & 255)];
+          }
+          word |= bits << (16 * k);
+        }
+        bias_s[(gi * T + r) * BR + c2] = word;
+      }
+    }
     bool ok = true;
     auto group_sync = [&]() {                          // barrier of the group's 128 threads; true if one of them gave up waiting
       uint32_t gave_up;
@@ -555,7 +559,7 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
         ptx::tc_commit(&s_full[gi]);
       }
       // -- seam mask of this row's window (shifted blocks: windows in the last window row or column) --
-      const int n = 2 * (cidx + ul * cstride) + w;
+      const int n = 2 * (ubase + ul) + w;
       bool masked = false;
       uint32_t diff_lo = 0, diff_hi = 0;
       if (g.shift > 0 && n < g.n_windows) {
