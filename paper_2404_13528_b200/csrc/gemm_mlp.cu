@@ -198,24 +198,29 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       for (int t2 = tid - 32; t2 < 2 * g.hidden; t2 += kThreads - 32) {
         const int row = t2 >> 1, half = t2 & 1;
         float csum = 0.f, bsum = half ? 0.f : __bfloat162float(g.b1[row]);
+        float bsum2 = 0.f;
 #pragma unroll 2
         for (int ci = half * (nch / 2); ci < (half + 1) * (nch / 2); ++ci) {     // chunk ci of the row: k-block ci / 4, chunk ci % 4
           uint4* p = reinterpret_cast<uint4*>(sW1 + (ci >> 2) * W1_KB + sw64_off(row, ci & 3));
           const uint4 wv = *p;
           const uint32_t w4[4] = {wv.x, wv.y, wv.z, wv.w};
+          const float4 ga0 = *reinterpret_cast<const float4*>(ln_s + ci * 8), ga1 = *reinterpret_cast<const float4*>(ln_s + ci * 8 + 4);
+          const float4 be0 = *reinterpret_cast<const float4*>(ln_s + C + ci * 8), be1 = *reinterpret_cast<const float4*>(ln_s + C + ci * 8 + 4);
+          const float ga[8] = {ga0.x, ga0.y, ga0.z, ga0.w, ga1.x, ga1.y, ga1.z, ga1.w};
+          const float be[8] = {be0.x, be0.y, be0.z, be0.w, be1.x, be1.y, be1.z, be1.w};
           uint32_t o4[4];
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            const int k = ci * 8 + 2 * e;
             const float2 f = bf16x2_to_float2(w4[e]);
-            bsum = fmaf(ln_s[C + k], f.x, bsum);
-            bsum = fmaf(ln_s[C + k + 1], f.y, bsum);
-            o4[e] = float2_to_bf16x2(ln_s[k] * f.x, ln_s[k + 1] * f.y);
+            bsum = fmaf(be[2 * e], f.x, bsum);
+            bsum2 = fmaf(be[2 * e + 1], f.y, bsum2);
+            o4[e] = float2_to_bf16x2(ga[2 * e] * f.x, ga[2 * e + 1] * f.y);
             const float2 r2 = bf16x2_to_float2(o4[e]);
             csum += r2.x + r2.y;
           }
           *p = make_uint4(o4[0], o4[1], o4[2], o4[3]);
         }
+        bsum += bsum2;
         csum += __shfl_xor_sync(0xFFFFFFFFu, csum, 1);
         bsum += __shfl_xor_sync(0xFFFFFFFFu, bsum, 1);
         if (half == 0) {
