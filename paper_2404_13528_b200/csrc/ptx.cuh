@@ -17,9 +17,11 @@ constexpr unsigned long long kWaitLimitNs = 1000000000ull;   // 1 s: the default
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
+// (the "memory" clobber keeps the read where it is written: without it the compiler may move it across a __syncthreads(),
+// and a time stamp "after the barrier" silently becomes the time the thread reached it)
 __device__ __forceinline__ unsigned long long globaltimer() {
   unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t) : : "memory");
   return t;
 }
 
