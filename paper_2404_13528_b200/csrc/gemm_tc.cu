@@ -89,6 +89,11 @@ __device__ __forceinline__ void tma_load_op(const OpCoord& oc, void* dst, const 
                                             int row0, const TileCoord& tc) {
   ptx::tma_load_5d(dst, tm, bar, oc.mn_major ? row0 : k0, oc.mn_major ? k0 : row0, tc.o0, tc.o1, tc.o2);
 }
+// CTA pair: the bytes are counted on the even CTA's barrier (a shared::cluster address)
+__device__ __forceinline__ void tma_load_op_pair(const OpCoord& oc, void* dst, const CUtensorMap* tm, uint32_t bar_cluster, int k0,
+                                                 int row0, const TileCoord& tc) {
+  ptx::tma_load_5d_pair(dst, tm, bar_cluster, k0, row0, tc.o0, tc.o1, tc.o2);
+}
 
 struct TileIdx {
   uint32_t tile_n, tile_m, batch;
@@ -118,14 +123,22 @@ constexpr int kThreads = 64 + 32 * kEpiWarps + 32;      // + a second TMA produc
 // Persistent kernel: one CTA per SM walks over output tiles (tile = blockIdx.x + i * gridDim.x).
 // The shared-memory ring and two TMEM accumulator buffers run across tile boundaries, so the
 // loads and MMAs of tile i+1 overlap the epilogue of tile i.
-template <int BN, int STAGES, bool A_MN>
+//
+// PAIR: the two CTAs of a cluster share one 256 x BN tile (cta_group::2).  Each loads its own 128 rows of A and its own
+// half of the B tile's rows -- two thirds of the operand bytes a lone CTA pulls in per product, which is what bounds a
+// 128 x 256 tile (48 KB per k-block against the ~64 bytes per clock an SM takes in) -- and keeps its own 128 rows of the
+// accumulator, which it drains itself.  The even CTA counts both CTAs' bytes on its `full` barriers, issues the products
+// and signals `empty` / `tmem_full` in both CTAs; both CTAs' epilogue warps arrive on its `tmem_empty`.
+template <int BN, int STAGES, bool A_MN, bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ GemmArgs g) {
-  constexpr int B_STAGE_BYTES = BN * BK * 2;
+  static_assert(!PAIR || (BN == 256 && !A_MN), "CTA pairs: 256-wide tiles, K-major A");
+  constexpr int BN_CTA = PAIR ? BN / 2 : BN;               // rows of B this CTA loads
+  constexpr int B_STAGE_BYTES = BN_CTA * BK * 2;
   constexpr uint32_t ACC_COLS = BN <= 32 ? 32 : BN <= 64 ? 64 : BN <= 128 ? 128 : 256;   // one accumulator buffer
   constexpr uint32_t TMEM_COLS = 2 * ACC_COLS;
-  constexpr uint32_t IDESC = ptx::make_idesc_bf16(BM, BN, A_MN, false);
+  constexpr uint32_t IDESC = ptx::make_idesc_bf16(PAIR ? 2 * BM : BM, BN, A_MN, false);
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -143,7 +156,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int nkb = (g.K + BK - 1) / BK;
   const int last_ksteps = (g.K - (nkb - 1) * BK + 15) / 16;
   const bool two_producers = nkb >= 8;
-  const uint32_t total_tiles = (uint32_t)g.tiles_n * g.tiles_m * g.batch;
+  const uint32_t total_tiles = (uint32_t)g.tiles_n * g.tiles_m * g.batch;   // PAIR: tiles_m counts 256-row tiles
+  const uint32_t rank = PAIR ? ptx::cluster_ctarank() : 0u;                  // which half of the pair's tile
+  const bool leader = rank == 0;
+  const uint32_t cta_first = PAIR ? blockIdx.x >> 1 : blockIdx.x, cta_step = PAIR ? gridDim.x >> 1 : gridDim.x;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
@@ -152,7 +168,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     for (int b = 0; b < 2; ++b) {
       ptx::mbar_init(&tmem_full[b], 1);
-      ptx::mbar_init(&tmem_empty[b], kEpiWarps);
+      ptx::mbar_init(&tmem_empty[b], PAIR ? 2 * kEpiWarps : kEpiWarps);
     }
     *abort_flag = 0;
     ptx::fence_barrier_init();
@@ -162,9 +178,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     ptx::prefetch_tensormap(&tmA);
     ptx::prefetch_tensormap(&tmB);
   }
-  if (warp == 1) ptx::tmem_alloc(tmem_slot, TMEM_COLS);
+  if (warp == 1) {
+    if constexpr (PAIR) ptx::tmem_alloc_pair(tmem_slot, TMEM_COLS);
+    else ptx::tmem_alloc(tmem_slot, TMEM_COLS);
+  }
   ptx::tc_fence_before();
-  __syncthreads();
+  if constexpr (PAIR) {
+    __syncwarp();
+    ptx::cluster_sync();            // the peer's barriers are initialised before anything of this CTA signals them
+  } else {
+    __syncthreads();
+  }
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   pdl_wait();                       // everything above overlapped the previous kernel's tail
@@ -175,21 +199,35 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       uint32_t kbg = 0, s = 0, ph = 0;                       // k-block counter across tiles, ring position
       bool ok = true;
       uint32_t pit = 0;
-      for (uint32_t t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++pit) {
+      const uint32_t full0 = PAIR ? ptx::mapa(ptx::smem_u32(full), 0) : 0u;     // the even CTA's `full` barriers
+      for (uint32_t t = cta_first; t < total_tiles && ok; t += cta_step, ++pit) {
         const TileIdx ti_ = split_tile(t, g.fd_tiles_n, g.fd_tiles_m);
-        const uint32_t tile_n = ti_.tile_n, tile_m = ti_.tile_m, batch = ti_.batch;
+        const uint32_t tile_n = ti_.tile_n, tile_m = PAIR ? 2 * ti_.tile_m + rank : ti_.tile_m, batch = ti_.batch;
         const TileCoord ta = op_coords(g.ca, tile_m, batch, BM), tb = op_coords(g.cb, tile_n, batch, BN);
+        const int brow0 = tb.row0 + (int)rank * BN_CTA;
         for (int kb = 0; kb < nkb; ++kb, ++kbg) {
           ok = ptx::mbar_wait(&empty[s], ph ^ 1, abort_flag, g.status);
           if (!ok) break;
-          ptx::mbar_expect_tx(&full[s], two_producers ? A_STAGE_BYTES : A_STAGE_BYTES + B_STAGE_BYTES);
-          tma_load_op(g.ca, sA + s * A_STAGE_BYTES, &tmA, &full[s], kb * BK, ta.row0, ta);
-          if (A_MN) tma_load_op(g.ca, sA + s * A_STAGE_BYTES + A_STAGE_BYTES / 2, &tmA, &full[s], kb * BK, ta.row0 + 64, ta);
-          if (!two_producers) tma_load_op(g.cb, sB + s * B_STAGE_BYTES, &tmB, &full[s], kb * BK, tb.row0, tb);
+          if constexpr (PAIR) {
+            if (leader) ptx::mbar_expect_tx(&full[s], 2 * (two_producers ? A_STAGE_BYTES : A_STAGE_BYTES + B_STAGE_BYTES));
+            tma_load_op_pair(g.ca, sA + s * A_STAGE_BYTES, &tmA, full0 + s * 8, kb * BK, ta.row0, ta);
+            if (!two_producers) tma_load_op_pair(g.cb, sB + s * B_STAGE_BYTES, &tmB, full0 + s * 8, kb * BK, brow0, tb);
+          } else {
+            ptx::mbar_expect_tx(&full[s], two_producers ? A_STAGE_BYTES : A_STAGE_BYTES + B_STAGE_BYTES);
+            tma_load_op(g.ca, sA + s * A_STAGE_BYTES, &tmA, &full[s], kb * BK, ta.row0, ta);
+            if (A_MN) tma_load_op(g.ca, sA + s * A_STAGE_BYTES + A_STAGE_BYTES / 2, &tmA, &full[s], kb * BK, ta.row0 + 64, ta);
+            if (!two_producers) tma_load_op(g.cb, sB + s * B_STAGE_BYTES, &tmB, &full[s], kb * BK, tb.row0, tb);
+          }
           if (++s == STAGES) { s = 0; ph ^= 1; }
         }
       }
-      if (*abort_flag) {
+      if (*abort_flag && PAIR) {
+        // unwinding a pair: the copies of the odd CTA are counted on the even CTA's barriers, so each side just gives
+        // whatever is in flight a fixed time to land
+        const unsigned long long t0 = ptx::globaltimer();
+        while (ptx::globaltimer() - t0 < 100000ull) {
+        }
+      } else if (*abort_flag) {
         // unwinding: give copies already in flight a bounded chance to land before the CTA leaves
         for (uint32_t k = (kbg > (uint32_t)STAGES ? kbg - STAGES : 0); k < kbg; ++k) {
           const unsigned long long t0 = ptx::globaltimer();
@@ -201,11 +239,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   } else if (warp == 1) {
     // The whole warp walks the loop and one elected lane issues: with warp-uniform control flow the descriptors
     // stay in uniform registers (under a branch on lane 0 each operand is moved there in front of every product).
-    {
+    if (leader) {                                     // (the odd CTA's warp 1 only owns its tensor-memory allocation)
       uint32_t it = 0, s = 0, ph = 0;                 // ring position and its phase carry over tiles
       const uint32_t a_base = ptx::smem_u32(sA), b_base = ptx::smem_u32(sB);
       bool ok = true;
-      for (uint32_t t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
+      for (uint32_t t = cta_first; t < total_tiles && ok; t += cta_step, ++it) {
         const uint32_t buf = it & 1, use = it >> 1;
         ok = __all_sync(0xFFFFFFFFu, ptx::mbar_wait(&tmem_empty[buf], (use & 1) ^ 1, abort_flag, g.status) ? 1 : 0) != 0;   // epilogue drained it
         if (!ok) break;
@@ -224,17 +262,25 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           const uint64_t bd0 = ptx::make_smem_desc(b_base + s * B_STAGE_BYTES, 16, 1024);
           constexpr uint64_t A_STEP = (A_MN ? 2048 : 32) >> 4, B_STEP = 32 >> 4;
           const bool last_kb = kb == nkb - 1;
+          auto mma = [&](uint64_t ad, uint64_t bd, uint32_t acc) {
+            if constexpr (PAIR) ptx::tc_mma_bf16_pair(d_tmem, ad, bd, IDESC, acc);
+            else ptx::tc_mma_bf16(d_tmem, ad, bd, IDESC, acc);
+          };
           if (ptx::elect_one()) {
             if (!last_kb || last_ksteps == BK / 16) {
-              ptx::tc_mma_bf16(d_tmem, ad0, bd0, IDESC, kb ? 1u : 0u);
+              mma(ad0, bd0, kb ? 1u : 0u);
 #pragma unroll
-              for (int k = 1; k < BK / 16; ++k) ptx::tc_mma_bf16(d_tmem, ad0 + k * A_STEP, bd0 + k * B_STEP, IDESC, 1u);
+              for (int k = 1; k < BK / 16; ++k) mma(ad0 + k * A_STEP, bd0 + k * B_STEP, 1u);
             } else {
-              for (int k = 0; k < last_ksteps; ++k)
-                ptx::tc_mma_bf16(d_tmem, ad0 + k * A_STEP, bd0 + k * B_STEP, IDESC, (kb | k) ? 1u : 0u);
+              for (int k = 0; k < last_ksteps; ++k) mma(ad0 + k * A_STEP, bd0 + k * B_STEP, (kb | k) ? 1u : 0u);
             }
-            ptx::tc_commit(&empty[s]);
-            if (last_kb) ptx::tc_commit(&tmem_full[buf]);
+            if constexpr (PAIR) {
+              ptx::tc_commit_pair(&empty[s], 3);
+              if (last_kb) ptx::tc_commit_pair(&tmem_full[buf], 3);
+            } else {
+              ptx::tc_commit(&empty[s]);
+              if (last_kb) ptx::tc_commit(&tmem_full[buf]);
+            }
           }
           __syncwarp();
           if (++s == STAGES) { s = 0; ph ^= 1; }
@@ -247,15 +293,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (lane == 0 && two_producers) {
       uint32_t s = 0, ph = 1;
       bool ok = true;
-      for (uint32_t t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+      const uint32_t full0 = PAIR ? ptx::mapa(ptx::smem_u32(full), 0) : 0u;
+      for (uint32_t t = cta_first; t < total_tiles && ok; t += cta_step) {
         const TileIdx ti_ = split_tile(t, g.fd_tiles_n, g.fd_tiles_m);
         const uint32_t tile_n = ti_.tile_n, batch = ti_.batch;
         const TileCoord tb = op_coords(g.cb, tile_n, batch, BN);
+        const int brow0 = tb.row0 + (int)rank * BN_CTA;
         for (int kb = 0; kb < nkb; ++kb) {
           ok = ptx::mbar_wait(&empty[s], ph, abort_flag, g.status);
           if (!ok) break;
-          ptx::mbar_expect_tx(&full[s], B_STAGE_BYTES);
-          tma_load_op(g.cb, sB + s * B_STAGE_BYTES, &tmB, &full[s], kb * BK, tb.row0, tb);
+          if constexpr (PAIR) {
+            if (leader) ptx::mbar_expect_tx(&full[s], 2 * B_STAGE_BYTES);
+            tma_load_op_pair(g.cb, sB + s * B_STAGE_BYTES, &tmB, full0 + s * 8, kb * BK, brow0, tb);
+          } else {
+            ptx::mbar_expect_tx(&full[s], B_STAGE_BYTES);
+            tma_load_op(g.cb, sB + s * B_STAGE_BYTES, &tmB, &full[s], kb * BK, tb.row0, tb);
+          }
           if (++s == STAGES) { s = 0; ph ^= 1; }
         }
       }
@@ -267,7 +320,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     //   phase 2 (threads spread along the row): 16-byte stores, RC*2 contiguous bytes per row,
     // so a store instruction writes whole 32-byte sectors and several sectors of one line at once.
     constexpr int CG = BN / 4;
-    constexpr int RC = (BN == 256 && STAGES == 4) ? 16 : (CG > 32 ? 32 : CG);   // 4 stages leave less staging room
+    constexpr int RC = (BN == 256 && STAGES == 4 && !PAIR) ? 16 : (CG > 32 ? 32 : CG);   // 4 stages leave less staging room
     constexpr int ROUNDS = CG / RC;
     constexpr int RH = ROUNDS > 1 ? ROUNDS / 2 : 1;          // BN == 256: rounds [0, RH) hold the first halves of rotary pairs
     constexpr int VPR = RC / 8;                              // 16-byte vectors per row per round
@@ -275,7 +328,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int e = warp - 2;
     const int q = warp & 3;                                  // TMEM lane quadrant this warp may read
     const int grp = e >> 2;
-    constexpr bool QSTAGE = !(BN == 256 && STAGES == 4);     // per-quadrant staging of whole rows
+    constexpr bool QSTAGE = PAIR || !(BN == 256 && STAGES == 4);     // per-quadrant staging of whole rows
     constexpr int QROW = BN * 2 + 16;                        // bytes; the pad keeps phase 1 conflict-free
     uint8_t* stage = stage_base + e * (32 * STG_ROW);
     uint8_t* qstage = stage_base + q * (32 * QROW);
@@ -284,9 +337,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     constexpr bool PREFETCH_NEXT = false;                   // (tried: next-tile offset + residual a tile ahead; the extra live registers spill and it is slower)
     long long off_next = 0;
     uint4 res_next[VPR];
-    for (uint32_t t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
+    const uint32_t tmem_empty0 = PAIR ? ptx::mapa(ptx::smem_u32(tmem_empty), 0) : 0u;   // the even CTA's barriers
+    for (uint32_t t = cta_first; t < total_tiles && ok; t += cta_step, ++it) {
       const TileIdx ti_ = split_tile(t, g.fd_tiles_n, g.fd_tiles_m);
-      const uint32_t tile_n = ti_.tile_n, tile_m = ti_.tile_m, batch = ti_.batch;
+      const uint32_t tile_n = ti_.tile_n, tile_m = PAIR ? 2 * ti_.tile_m + rank : ti_.tile_m, batch = ti_.batch;
       const uint32_t buf = it & 1, use = it >> 1;
       const int n0 = tile_n * BN;
       const int row = tile_m * BM + q * 32 + lane;
@@ -338,7 +392,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         fetch_res(col_of(0));                                // in flight while this tile's MMAs still run
       }
       if (PREFETCH_NEXT) {                                   // request the next tile's row offset and residual now
-        const uint32_t tn = t + gridDim.x;
+        const uint32_t tn = t + cta_step;
         if (tn < total_tiles) {
           const TileIdx nx = split_tile(tn, g.fd_tiles_n, g.fd_tiles_m);
           const int nrow = nx.tile_m * BM + q * 32 + lane;
@@ -466,7 +520,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       // all of this warp's TMEM reads of the buffer have completed (wait::ld above)
       ptx::tc_fence_before();
       __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(&tmem_empty[buf]);
+      if (lane == 0) {
+        if constexpr (PAIR) ptx::mbar_arrive_cluster(tmem_empty0 + buf * 8);
+        else ptx::mbar_arrive(&tmem_empty[buf]);
+      }
       if constexpr (QSTAGE) {
         // the four warps of the quadrant have filled a 32 x BN staging tile: store whole rows
         constexpr int VR = BN / 8;                           // 16-byte vectors per row
@@ -486,10 +543,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
   }
   ptx::tc_fence_before();
-  __syncthreads();
+  if constexpr (PAIR) {
+    __syncwarp();
+    ptx::cluster_sync();            // neither CTA leaves (or frees tensor memory) while the other may still read or signal it
+  } else {
+    __syncthreads();
+  }
   if (warp == 1) {
     ptx::tc_fence_after();
-    ptx::tmem_dealloc(tmem_base, TMEM_COLS);
+    if constexpr (PAIR) ptx::tmem_dealloc_pair(tmem_base, TMEM_COLS);
+    else ptx::tmem_dealloc(tmem_base, TMEM_COLS);
   }
 }
 
@@ -554,7 +617,8 @@ int encode_cached(const void* ptr, int rank, const uint64_t* dims, const uint64_
 }
 
 // Turns an operand description into a tensor map + the coordinate rule of the kernel.
-int build_operand(const TcOperand& op, int tile_rows, CUtensorMap* tm, OpCoord* oc) {
+// `box_rows` rows per copy (a CTA pair fetches a tile of `tile_rows` rows as two boxes, one per CTA).
+int build_operand(const TcOperand& op, int tile_rows, int box_rows, CUtensorMap* tm, OpCoord* oc) {
   if (op.n_row_atoms < 1 || op.n_row_atoms + op.n_batch_atoms > 4) return SMARTMEM_ERR_UNSUPPORTED;
   if (((uintptr_t)op.ptr & 15) != 0) return SMARTMEM_ERR_ALIGNMENT;
   const int nr = op.n_row_atoms, nb = op.n_batch_atoms;
@@ -577,7 +641,7 @@ int build_operand(const TcOperand& op, int tile_rows, CUtensorMap* tm, OpCoord* 
   };
   bool ok = true;
   if (!mn) {
-    ok = ok && push(op.K, 1, BK) && push(in_ext, in_str, (uint32_t)tile_rows);
+    ok = ok && push(op.K, 1, BK) && push(in_ext, in_str, (uint32_t)box_rows);
   } else {
     ok = ok && push(in_ext, 1, 64) && push(op.K, op.k_stride, BK);
   }
@@ -616,16 +680,24 @@ int sm_count() {
   return n;
 }
 
-template <int BN, int STAGES, bool A_MN>
+template <int BN, int STAGES, bool A_MN, bool PAIR = false>
 int launch_t(const CUtensorMap& ta, const CUtensorMap& tb, const GemmArgs& g, cudaStream_t st) {
-  constexpr int RCc = (BN == 256 && STAGES == 4) ? 16 : ((BN / 4) > 32 ? 32 : (BN / 4));
-  constexpr size_t smem = 1024 + STAGES * (A_STAGE_BYTES + BN * BK * 2) + (2 * STAGES + 4) * 8 + 16 +
-                          ((BN == 256 && STAGES == 4) ? kEpiWarps * 32 * (RCc * 2 + 16) : 4 * 32 * (BN * 2 + 16));
-  if (ensure_max_dynamic_smem((const void*)gemm_tc_kernel<BN, STAGES, A_MN>, (int)smem) != SMARTMEM_OK) return SMARTMEM_ERR_CUDA;
+  constexpr bool QST = PAIR || !(BN == 256 && STAGES == 4);
+  constexpr int RCc = !QST ? 16 : ((BN / 4) > 32 ? 32 : (BN / 4));
+  constexpr size_t smem = 1024 + STAGES * (A_STAGE_BYTES + (PAIR ? BN / 2 : BN) * BK * 2) + (2 * STAGES + 4) * 8 + 16 +
+                          (!QST ? kEpiWarps * 32 * (RCc * 2 + 16) : 4 * 32 * (BN * 2 + 16));
+  if (ensure_max_dynamic_smem((const void*)gemm_tc_kernel<BN, STAGES, A_MN, PAIR>, (int)smem) != SMARTMEM_OK) return SMARTMEM_ERR_CUDA;
   profile_tick("gemm_tc", st);
   const long long tiles = (long long)g.tiles_n * g.tiles_m * g.batch;
-  const unsigned grid = (unsigned)(tiles < sm_count() ? tiles : sm_count());
-  launch_pdl(gemm_tc_kernel<BN, STAGES, A_MN>, dim3(grid), dim3(kThreads), smem, st, ta, tb, g);
+  if constexpr (PAIR) {
+    // one cluster of two CTAs per tile of 256 rows; the two CTAs of a cluster are neighbours in blockIdx.x
+    const long long pairs = sm_count() / 2;
+    const unsigned grid = (unsigned)(2 * (tiles < pairs ? tiles : pairs));
+    launch_pdl_cluster(gemm_tc_kernel<BN, STAGES, A_MN, PAIR>, dim3(grid), dim3(kThreads), smem, st, 2u, ta, tb, g);
+  } else {
+    const unsigned grid = (unsigned)(tiles < sm_count() ? tiles : sm_count());
+    launch_pdl(gemm_tc_kernel<BN, STAGES, A_MN, PAIR>, dim3(grid), dim3(kThreads), smem, st, ta, tb, g);
+  }
   count_launch();
   return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
 }
@@ -741,12 +813,19 @@ int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep,
   // 256 wide, short K: wider store rounds instead of a 4th stage.  Narrow tiles: their stages are
   // small, and a tile is consumed faster than a load's latency, so the ring runs several tiles ahead.
   const int stages = bn == 256 ? (nkb <= 4 ? 3 : 4) : (bn <= 96 ? 6 : 4);
+  // CTA pairs (two SMs on one 256 x 256 tile) where the row tiles pair up and there is more than one wave of work for
+  // the single-CTA kernel: below that the operand feed is not what bounds the GEMM.
+  // SMARTMEM_GEMM_PAIR=0 keeps every GEMM on single CTAs (for measuring what pairing buys).
+  static const int allow_pair = [] { const char* e = getenv("SMARTMEM_GEMM_PAIR"); return (e && e[0] == '0') ? 0 : 1; }();
+  const long long tiles_m1 = (M + BM - 1) / BM;
+  const bool pair = allow_pair && bn == 256 && !a_mn && tiles_m1 % 2 == 0 && nkb > 4 &&
+                    tiles_m1 * ((N + bn - 1) / bn) * batch > tc_sm_count();
   GemmArgs g;
   memset(&g, 0, sizeof(g));
   CUtensorMap ta, tb;
-  int rc = build_operand(A, BM, &ta, &g.ca);
+  int rc = build_operand(A, BM, BM, &ta, &g.ca);
   if (rc != SMARTMEM_OK) return rc;
-  rc = build_operand(B, bn, &tb, &g.cb);
+  rc = build_operand(B, bn, pair ? bn / 2 : bn, &tb, &g.cb);
   if (rc != SMARTMEM_OK) return rc;
   g.M = (int)M; g.N = (int)N; g.K = (int)K;
   g.out = (__nv_bfloat16*)ep.out;
@@ -773,11 +852,12 @@ int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep,
   g.status = device_status_ptr();
   if (!g.status) return SMARTMEM_ERR_CUDA;
   g.tiles_n = (int)((N + bn - 1) / bn);
-  g.tiles_m = (int)((M + BM - 1) / BM);
+  g.tiles_m = (int)(pair ? tiles_m1 / 2 : tiles_m1);       // pairs walk over tiles of 256 rows
   g.fd_tiles_n = make_fastdiv((uint32_t)g.tiles_n);
   g.fd_tiles_m = make_fastdiv((uint32_t)g.tiles_m);
   g.batch = (int)batch;
   if ((long long)g.tiles_n * g.tiles_m * g.batch >= (1ll << 31)) return SMARTMEM_ERR_UNSUPPORTED;
+  if (pair) return launch_t<256, 4, false, true>(ta, tb, g, st);
 #define SM_CASE(BN_, ST_, MN_)                                                                  \
   if (bn == BN_ && stages == ST_ && a_mn == MN_) return launch_t<BN_, ST_, MN_>(ta, tb, g, st);
   SM_CASE(256, 3, false) SM_CASE(256, 4, false) SM_CASE(128, 4, false) SM_CASE(96, 6, false) SM_CASE(64, 6, false)
