@@ -320,6 +320,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     //   phase 2 (threads spread along the row): 16-byte stores, RC*2 contiguous bytes per row,
     // so a store instruction writes whole 32-byte sectors and several sectors of one line at once.
     constexpr int CG = BN / 4;
+    constexpr bool DIRECT = PAIR;                            // rows leave the registers as 32-byte stores: no staging at all
     constexpr int RC = (BN == 256 && STAGES == 4 && !PAIR) ? 16 : (CG > 32 ? 32 : CG);   // 4 stages leave less staging room
     constexpr int ROUNDS = CG / RC;
     constexpr int RH = ROUNDS > 1 ? ROUNDS / 2 : 1;          // BN == 256: rounds [0, RH) hold the first halves of rotary pairs
@@ -328,7 +329,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int e = warp - 2;
     const int q = warp & 3;                                  // TMEM lane quadrant this warp may read
     const int grp = e >> 2;
-    constexpr bool QSTAGE = PAIR || !(BN == 256 && STAGES == 4);     // per-quadrant staging of whole rows
+    constexpr bool QSTAGE = !DIRECT && !(BN == 256 && STAGES == 4);  // per-quadrant staging of whole rows
     constexpr int QROW = BN * 2 + 16;                        // bytes; the pad keeps phase 1 conflict-free
     uint8_t* stage = stage_base + e * (32 * STG_ROW);
     uint8_t* qstage = stage_base + q * (32 * QROW);
@@ -413,11 +414,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       if (!ok) break;
       ptx::tc_fence_after();
       const uint32_t taddr = tmem_base + buf * ACC_COLS + ((uint32_t)(q * 32) << 16);
+      if constexpr (QSTAGE) {
+        // the previous tile's row copies have read the staging rows before anyone overwrites them
+        if (lane < 8) ptx::bulk_wait_group_read<0>();
+        asm volatile("bar.sync %0, 128;" ::"r"(1 + q) : "memory");
+      }
 
 #pragma unroll
       for (int rd = 0; rd < ROUNDS; ++rd) {
         const int c0 = col_of(rd);
         float acc[RC];
+        uint4 bv[VPR];                                       // this round's bias columns: requested before the wait on tensor memory
+        if (g.bias) {
+#pragma unroll
+          for (int v = 0; v < VPR; ++v) {
+            bv[v] = make_uint4(0, 0, 0, 0);
+            if (n0 + c0 + v * 8 + 8 <= g.N) bv[v] = *reinterpret_cast<const uint4*>(g.bias + n0 + c0 + v * 8);
+          }
+        }
         {
           uint32_t rv[RC];
           ptx::tmem_ld_cols<RC>(taddr + c0, rv);
@@ -461,11 +475,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (g.bias) {
 #pragma unroll
           for (int v = 0; v < VPR; ++v) {
-            if (n0 + c0 + v * 8 + 8 <= g.N) {
-              float bb[8];
-              ElemIO<__nv_bfloat16>::load(g.bias + n0 + c0 + v * 8, bb);
+            const uint32_t w[4] = {bv[v].x, bv[v].y, bv[v].z, bv[v].w};
 #pragma unroll
-              for (int j = 0; j < 8; ++j) acc[v * 8 + j] += bb[j];
+            for (int j = 0; j < 4; ++j) {
+              const float2 f = bf16x2_to_float2(w[j]);
+              acc[v * 8 + 2 * j] += f.x;
+              acc[v * 8 + 2 * j + 1] += f.y;
             }
           }
         }
@@ -493,6 +508,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           for (int j = 0; j < RC; ++j)
             if (n0 + c0 + j < g.N) g.out2[o2_base + (long long)(n0 + c0 + j) * g.fd_out2_S.d] = __float2bfloat16_rn(acc[j]);
         }
+        uint4 pk_prev = make_uint4(0, 0, 0, 0);
 #pragma unroll
         for (int v = 0; v < VPR; ++v) {
           uint4 pk;
@@ -500,10 +516,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           pk.y = float2_to_bf16x2(acc[v * 8 + 2], acc[v * 8 + 3]);
           pk.z = float2_to_bf16x2(acc[v * 8 + 4], acc[v * 8 + 5]);
           pk.w = float2_to_bf16x2(acc[v * 8 + 6], acc[v * 8 + 7]);
-          if constexpr (QSTAGE) *reinterpret_cast<uint4*>(qstage + lane * QROW + (c0 + v * 8) * 2) = pk;
+          if constexpr (DIRECT) {
+            // 64 contiguous bytes of the thread's own row per round, as two 32-byte stores: whole sectors, and the
+            // shared memory (whose bandwidth the operands need) is left to the ring, which gets six stages
+            if (v & 1) {
+              if (row_ok) ptx::st_global_v8(out_t + off + n0 + c0 + (v - 1) * 8, pk_prev, pk);
+            } else {
+              pk_prev = pk;
+            }
+          } else if constexpr (QSTAGE) *reinterpret_cast<uint4*>(qstage + lane * QROW + (c0 + v * 8) * 2) = pk;
           else *reinterpret_cast<uint4*>(stage + lane * STG_ROW + v * 16) = pk;
         }
-        if constexpr (!QSTAGE) {
+        if constexpr (!QSTAGE && !DIRECT) {
           __syncwarp();
 #pragma unroll
           for (int i = 0; i < VPR; ++i) {
@@ -525,23 +549,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         else ptx::mbar_arrive(&tmem_empty[buf]);
       }
       if constexpr (QSTAGE) {
-        // the four warps of the quadrant have filled a 32 x BN staging tile: store whole rows
-        constexpr int VR = BN / 8;                           // 16-byte vectors per row
+        // the four warps of the quadrant have filled a 32 x BN staging tile: every row leaves as one bulk copy
+        // (shared memory -> global, BN * 2 contiguous bytes), eight rows per warp, so no thread spends
+        // instructions on moving the tile
+        ptx::fence_proxy_async();
         asm volatile("bar.sync %0, 128;" ::"r"(1 + q) : "memory");
-        const int tq = grp * 32 + lane;
-#pragma unroll
-        for (int i = 0; i < VR / 4; ++i) {
-          const int v = tq + 128 * i;
-          const int rr = v / VR, seg = v - rr * VR;
-          const long long roff = __shfl_sync(0xFFFFFFFFu, off, rr);
-          const int rok = __shfl_sync(0xFFFFFFFFu, (int)row_ok, rr);
-          const uint4 pk = *reinterpret_cast<const uint4*>(qstage + rr * QROW + seg * 16);
-          if (rok && n0 + seg * 8 + 8 <= g.N) *reinterpret_cast<uint4*>(out_t + roff + n0 + seg * 8) = pk;
+        const int rr = grp * 8 + (lane & 7);
+        const long long roff = __shfl_sync(0xFFFFFFFFu, off, rr);
+        const int rok = __shfl_sync(0xFFFFFFFFu, (int)row_ok, rr);
+        const int ncols = g.N - n0 < BN ? g.N - n0 : BN;
+        if (lane < 8) {
+          if (rok) ptx::bulk_store(out_t + roff + n0, qstage + rr * QROW, (uint32_t)ncols * 2u);
+          ptx::bulk_commit_group();
         }
-        asm volatile("bar.sync %0, 128;" ::"r"(1 + q) : "memory");
       }
     }
   }
+  ptx::bulk_wait_group_read<0>();   // row copies of the last tile have read their staging rows
   ptx::tc_fence_before();
   if constexpr (PAIR) {
     __syncwarp();
@@ -682,10 +706,10 @@ int sm_count() {
 
 template <int BN, int STAGES, bool A_MN, bool PAIR = false>
 int launch_t(const CUtensorMap& ta, const CUtensorMap& tb, const GemmArgs& g, cudaStream_t st) {
-  constexpr bool QST = PAIR || !(BN == 256 && STAGES == 4);
+  constexpr bool QST = !PAIR && !(BN == 256 && STAGES == 4);
   constexpr int RCc = !QST ? 16 : ((BN / 4) > 32 ? 32 : (BN / 4));
   constexpr size_t smem = 1024 + STAGES * (A_STAGE_BYTES + (PAIR ? BN / 2 : BN) * BK * 2) + (2 * STAGES + 4) * 8 + 16 +
-                          (!QST ? kEpiWarps * 32 * (RCc * 2 + 16) : 4 * 32 * (BN * 2 + 16));
+                          (PAIR ? 0 : !QST ? kEpiWarps * 32 * (RCc * 2 + 16) : 4 * 32 * (BN * 2 + 16));   // pairs store from registers
   if (ensure_max_dynamic_smem((const void*)gemm_tc_kernel<BN, STAGES, A_MN, PAIR>, (int)smem) != SMARTMEM_OK) return SMARTMEM_ERR_CUDA;
   profile_tick("gemm_tc", st);
   const long long tiles = (long long)g.tiles_n * g.tiles_m * g.batch;
@@ -818,8 +842,10 @@ int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep,
   // SMARTMEM_GEMM_PAIR=0 keeps every GEMM on single CTAs (for measuring what pairing buys).
   static const int allow_pair = [] { const char* e = getenv("SMARTMEM_GEMM_PAIR"); return (e && e[0] == '0') ? 0 : 1; }();
   const long long tiles_m1 = (M + BM - 1) / BM;
-  const bool pair = allow_pair && bn == 256 && !a_mn && tiles_m1 % 2 == 0 && nkb > 4 &&
-                    tiles_m1 * ((N + bn - 1) / bn) * batch > tc_sm_count();
+  const bool pair = allow_pair && bn == 256 && !a_mn && tiles_m1 % 2 == 0 && nkb > 4 && N % 256 == 0 &&
+                    tiles_m1 * ((N + bn - 1) / bn) * batch > tc_sm_count() &&
+                    !ep.rowmap && ep.seg_cols == 0 && !ep.out2 && ep.ldc % 16 == 0 && ep.out_batch_stride % 16 == 0 &&
+                    ((uintptr_t)ep.out & 31) == 0;                     // (its epilogue writes 32-byte vectors)
   GemmArgs g;
   memset(&g, 0, sizeof(g));
   CUtensorMap ta, tb;
@@ -857,7 +883,7 @@ int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep,
   g.fd_tiles_m = make_fastdiv((uint32_t)g.tiles_m);
   g.batch = (int)batch;
   if ((long long)g.tiles_n * g.tiles_m * g.batch >= (1ll << 31)) return SMARTMEM_ERR_UNSUPPORTED;
-  if (pair) return launch_t<256, 4, false, true>(ta, tb, g, st);
+  if (pair) return launch_t<256, 6, false, true>(ta, tb, g, st);
 #define SM_CASE(BN_, ST_, MN_)                                                                  \
   if (bn == BN_ && stages == ST_ && a_mn == MN_) return launch_t<BN_, ST_, MN_>(ta, tb, g, st);
   SM_CASE(256, 3, false) SM_CASE(256, 4, false) SM_CASE(128, 4, false) SM_CASE(96, 6, false) SM_CASE(64, 6, false)
