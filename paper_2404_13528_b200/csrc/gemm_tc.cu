@@ -129,11 +129,15 @@ constexpr int kThreads = 64 + 32 * kEpiWarps + 32;      // + a second TMA produc
 // 128 x 256 tile (48 KB per k-block against the ~64 bytes per clock an SM takes in) -- and keeps its own 128 rows of the
 // accumulator, which it drains itself.  The even CTA counts both CTAs' bytes on its `full` barriers, issues the products
 // and signals `empty` / `tmem_full` in both CTAs; both CTAs' epilogue warps arrive on its `tmem_empty`.
-template <int BN, int STAGES, bool A_MN, bool PAIR>
+// LEAN (pairs only): the epilogue knows bias and GELU only (no rotary embedding, residual or second copy), which leaves it
+// the registers to pull its whole accumulator slice out of tensor memory at once and hand the buffer back before any
+// arithmetic -- for short reductions, where a tile's products take no longer than its epilogue.
+template <int BN, int STAGES, bool A_MN, bool PAIR, bool LEAN>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ GemmArgs g) {
   static_assert(!PAIR || (BN == 256 && !A_MN), "CTA pairs: 256-wide tiles, K-major A");
+  static_assert(!LEAN || PAIR, "the lean epilogue comes with CTA pairs");
   constexpr int BN_CTA = PAIR ? BN / 2 : BN;               // rows of B this CTA loads
   constexpr int B_STAGE_BYTES = BN_CTA * BK * 2;
   constexpr uint32_t ACC_COLS = BN <= 32 ? 32 : BN <= 64 ? 64 : BN <= 128 ? 128 : 256;   // one accumulator buffer
@@ -321,6 +325,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // so a store instruction writes whole 32-byte sectors and several sectors of one line at once.
     constexpr int CG = BN / 4;
     constexpr bool DIRECT = PAIR;                            // rows leave the registers as 32-byte stores: no staging at all
+    constexpr bool EARLY = DIRECT && LEAN;                   // accumulator slice to registers first, buffer released at once
     constexpr int RC = (BN == 256 && STAGES == 4 && !PAIR) ? 16 : (CG > 32 ? 32 : CG);   // 4 stages leave less staging room
     constexpr int ROUNDS = CG / RC;
     constexpr int RH = ROUNDS > 1 ? ROUNDS / 2 : 1;          // BN == 256: rounds [0, RH) hold the first halves of rotary pairs
@@ -347,7 +352,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int row = tile_m * BM + q * 32 + lane;
       const bool row_ok = row < g.M;
       long long o2_base = 0;                                 // second copy: row = b * S + s goes to out2[b][col][s]
-      if (g.out2) {
+      if (!LEAN && g.out2) {
         const uint32_t b2 = fd_div((uint32_t)row, g.fd_out2_S);
         o2_base = (long long)b2 * g.N * g.fd_out2_S.d + ((uint32_t)row - b2 * g.fd_out2_S.d);
       }
@@ -372,8 +377,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (row_ok) off = g.has_rowmap ? devmap_eval_unrolled(g.rowmap, (uint32_t)row) : (long long)row * ld_t;
         off += (long long)batch * g.out_batch_stride;
       }
-      const __nv_bfloat16* __restrict__ rrow = g.residual ? g.residual + off : nullptr;
-      const bool rope_tile = (BN == 256 || BN == 128) && g.rope_cols > 0 && n0 < g.rope_cols;
+      const __nv_bfloat16* __restrict__ rrow = (!LEAN && g.residual) ? g.residual + off : nullptr;
+      const bool rope_tile = !LEAN && (BN == 256 || BN == 128) && g.rope_cols > 0 && n0 < g.rope_cols;
       auto col_of = [&](int rd) {
         return BN == 256 ? 128 * (grp >> 1) + 32 * (grp & 1) + RC * (rd % RH) + 64 * (rd / RH) : grp * CG;
       };
@@ -420,6 +425,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         asm volatile("bar.sync %0, 128;" ::"r"(1 + q) : "memory");
       }
 
+      // EARLY: the whole accumulator slice of the thread (ROUNDS x RC values) moves to registers first and the buffer goes
+      // back to the issuing warp before any arithmetic or store, so the next tile but one starts as early as it can
+      uint32_t rall[EARLY ? ROUNDS : 1][RC];
+      if constexpr (EARLY) {
+#pragma unroll
+        for (int rd = 0; rd < ROUNDS; ++rd) ptx::tmem_ld_cols<RC>(taddr + col_of(rd), rall[rd]);
+        ptx::tmem_ld_wait();
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive_cluster(tmem_empty0 + buf * 8);
+      }
 #pragma unroll
       for (int rd = 0; rd < ROUNDS; ++rd) {
         const int c0 = col_of(rd);
@@ -433,8 +449,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           }
         }
         {
-          uint32_t rv[RC];
-          ptx::tmem_ld_cols<RC>(taddr + c0, rv);
+          uint32_t rv_local[EARLY ? 1 : RC], rw[EARLY ? 1 : RC];
+          uint32_t* rv = EARLY ? rall[EARLY ? rd : 0] : rv_local;
+          if constexpr (!EARLY) ptx::tmem_ld_cols<RC>(taddr + c0, rv);
           // rotary pairs are (i, i + R/2) inside the first R columns of a 128-column head (R = 128: the
           // whole head).  This round's RC columns start at head-local column hc0; they rotate iff hc0 < R,
           // and their partners are the RC columns R/2 further up or down (or, when R/2 < RC, the other
@@ -443,9 +460,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if (rope_tile && hc0 < 2 * half) {
             const bool in_round = half < RC;                 // R = 32 with 32-column rounds: pairs (j, j + 16) of this round
             const bool first_half = hc0 < half;
-            uint32_t rw[RC];
-            if (!in_round) ptx::tmem_ld_cols<RC>(taddr + (first_half ? c0 + half : c0 - half), rw);
-            ptx::tmem_ld_wait();
+            if constexpr (!EARLY) {
+              if (!in_round) ptx::tmem_ld_cols<RC>(taddr + (first_half ? c0 + half : c0 - half), rw);
+              ptx::tmem_ld_wait();
+            }
             // angle = position * theta^(-i/(R/2)), reduced mod 2 pi in two steps, then the hardware
             // sine / cosine: no table traffic (a [S, 64] table read 16 bytes per lane per row
             // slowed the whole kernel by a fifth)
@@ -467,7 +485,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               acc[j] = fh ? x * cs - y * sn : x * cs + y * sn;
             }
           } else {
-            ptx::tmem_ld_wait();
+            if constexpr (!EARLY) ptx::tmem_ld_wait();
 #pragma unroll
             for (int j = 0; j < RC; ++j) acc[j] = __uint_as_float(rv[j]);
           }
@@ -501,7 +519,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           }
           if (rd + 1 < ROUNDS) fetch_res(col_of(rd + 1));
         }
-        if (g.out2 && row_ok) {
+        if (!LEAN && g.out2 && row_ok) {
           // The redundant copy of a producer with consumers of different reduction dimensions: the same values with the
           // row's position inside its group as the contiguous dimension.  A warp's 32 rows write 64 contiguous bytes per column.
 #pragma unroll
@@ -542,11 +560,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
       }
       // all of this warp's TMEM reads of the buffer have completed (wait::ld above)
-      ptx::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) {
-        if constexpr (PAIR) ptx::mbar_arrive_cluster(tmem_empty0 + buf * 8);
-        else ptx::mbar_arrive(&tmem_empty[buf]);
+      if constexpr (!EARLY) {
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+          if constexpr (PAIR) ptx::mbar_arrive_cluster(tmem_empty0 + buf * 8);
+          else ptx::mbar_arrive(&tmem_empty[buf]);
+        }
       }
       if constexpr (QSTAGE) {
         // the four warps of the quadrant have filled a 32 x BN staging tile: every row leaves as one bulk copy
@@ -704,23 +724,23 @@ int sm_count() {
   return n;
 }
 
-template <int BN, int STAGES, bool A_MN, bool PAIR = false>
+template <int BN, int STAGES, bool A_MN, bool PAIR = false, bool LEAN = false>
 int launch_t(const CUtensorMap& ta, const CUtensorMap& tb, const GemmArgs& g, cudaStream_t st) {
   constexpr bool QST = !PAIR && !(BN == 256 && STAGES == 4);
   constexpr int RCc = !QST ? 16 : ((BN / 4) > 32 ? 32 : (BN / 4));
   constexpr size_t smem = 1024 + STAGES * (A_STAGE_BYTES + (PAIR ? BN / 2 : BN) * BK * 2) + (2 * STAGES + 4) * 8 + 16 +
                           (PAIR ? 0 : !QST ? kEpiWarps * 32 * (RCc * 2 + 16) : 4 * 32 * (BN * 2 + 16));   // pairs store from registers
-  if (ensure_max_dynamic_smem((const void*)gemm_tc_kernel<BN, STAGES, A_MN, PAIR>, (int)smem) != SMARTMEM_OK) return SMARTMEM_ERR_CUDA;
+  if (ensure_max_dynamic_smem((const void*)gemm_tc_kernel<BN, STAGES, A_MN, PAIR, LEAN>, (int)smem) != SMARTMEM_OK) return SMARTMEM_ERR_CUDA;
   profile_tick("gemm_tc", st);
   const long long tiles = (long long)g.tiles_n * g.tiles_m * g.batch;
   if constexpr (PAIR) {
     // one cluster of two CTAs per tile of 256 rows; the two CTAs of a cluster are neighbours in blockIdx.x
     const long long pairs = sm_count() / 2;
     const unsigned grid = (unsigned)(2 * (tiles < pairs ? tiles : pairs));
-    launch_pdl_cluster(gemm_tc_kernel<BN, STAGES, A_MN, PAIR>, dim3(grid), dim3(kThreads), smem, st, 2u, ta, tb, g);
+    launch_pdl_cluster(gemm_tc_kernel<BN, STAGES, A_MN, PAIR, LEAN>, dim3(grid), dim3(kThreads), smem, st, 2u, ta, tb, g);
   } else {
     const unsigned grid = (unsigned)(tiles < sm_count() ? tiles : sm_count());
-    launch_pdl(gemm_tc_kernel<BN, STAGES, A_MN, PAIR>, dim3(grid), dim3(kThreads), smem, st, ta, tb, g);
+    launch_pdl(gemm_tc_kernel<BN, STAGES, A_MN, PAIR, LEAN>, dim3(grid), dim3(kThreads), smem, st, ta, tb, g);
   }
   count_launch();
   return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
@@ -883,6 +903,7 @@ int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep,
   g.fd_tiles_m = make_fastdiv((uint32_t)g.tiles_m);
   g.batch = (int)batch;
   if ((long long)g.tiles_n * g.tiles_m * g.batch >= (1ll << 31)) return SMARTMEM_ERR_UNSUPPORTED;
+  if (pair && nkb <= 16 && ep.rope_cols == 0 && !ep.residual) return launch_t<256, 6, false, true, true>(ta, tb, g, st);
   if (pair) return launch_t<256, 6, false, true>(ta, tb, g, st);
 #define SM_CASE(BN_, ST_, MN_)                                                                  \
   if (bn == BN_ && stages == ST_ && a_mn == MN_) return launch_t<BN_, ST_, MN_>(ta, tb, g, st);
