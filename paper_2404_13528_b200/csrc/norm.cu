@@ -18,12 +18,23 @@ __device__ __forceinline__ float group_sum(float v) {
   return v;
 }
 
+__device__ __forceinline__ void unpack8_bf16(const uint4& u, float (&f)[8]) {
+  const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    f[2 * q] = __uint_as_float(w[q] << 16);
+    f[2 * q + 1] = __uint_as_float(w[q] & 0xFFFF0000u);
+  }
+}
+
 // LPR lanes cooperate on one row and keep up to 4 16-byte vectors each in registers (vector k of
 // lane l is vector l + k * LPR of the row, so a warp-wide load covers 32 / LPR rows with runs of
 // LPR * 16 contiguous bytes).  RPG rows per lane group are in flight together.  GENERIC: any row
 // length; the row is re-read from L1/L2 for each pass instead of being kept.
+// 16-bit elements stay packed in registers (16 instead of 32 per row slice) and are unpacked for each pass: with six CTAs
+// per SM the 12 544 rows of a 14 x 14 x 64 activation are all in flight in a single wave (four CTAs made it 1.3 waves).
 template <typename T, int LPR, bool RMS, int RPG, bool GENERIC>
-__global__ void __launch_bounds__(256) norm_kernel(const T* __restrict__ src, T* __restrict__ dst,
+__global__ void __launch_bounds__(256, (!GENERIC && sizeof(T) == 2 && RPG == 1) ? 6 : 1) norm_kernel(const T* __restrict__ src, T* __restrict__ dst,
                                                    const T* __restrict__ gamma, const T* __restrict__ beta, float eps,
                                                    long long rows, int C, int vpl, const __grid_constant__ DevMap rowmap,
                                                    int has_map) {
@@ -35,7 +46,17 @@ __global__ void __launch_bounds__(256) norm_kernel(const T* __restrict__ src, T*
   const long long row0 = (long long)blockIdx.x * (GPB * RPG) + grp;
   const int nvec = C / KV;
   const float invC = 1.0f / (float)C;
-  float v[RPG][NV][KV];
+  constexpr bool PACKED = !GENERIC && sizeof(T) == 2;       // (KV == 8: one 16-byte vector)
+  float v[PACKED ? 1 : RPG][PACKED ? 1 : NV][KV];
+  uint4 pv[PACKED ? RPG : 1][PACKED ? NV : 1];
+  auto slice = [&](int r, int k, float (&f)[KV]) {           // values of (row r, vector k) as fp32
+    if constexpr (PACKED) {
+      unpack8_bf16(pv[r][k], reinterpret_cast<float(&)[8]>(f));
+    } else {
+#pragma unroll
+      for (int e = 0; e < KV; ++e) f[e] = v[r][k][e];
+    }
+  };
   const T* s[RPG];
   bool active[RPG];
   float sum[RPG];
@@ -61,7 +82,10 @@ __global__ void __launch_bounds__(256) norm_kernel(const T* __restrict__ src, T*
 #pragma unroll
       for (int k = 0; k < NV; ++k) {
         const int vi = sub + k * LPR;
-        if (k < vpl && active[r] && vi < nvec) {
+        if constexpr (PACKED) {
+          pv[r][k] = make_uint4(0, 0, 0, 0);
+          if (k < vpl && active[r] && vi < nvec) pv[r][k] = *reinterpret_cast<const uint4*>(s[r] + vi * KV);
+        } else if (k < vpl && active[r] && vi < nvec) {
           ElemIO<T>::load(s[r] + vi * KV, v[r][k]);
         } else {
 #pragma unroll
@@ -76,8 +100,10 @@ __global__ void __launch_bounds__(256) norm_kernel(const T* __restrict__ src, T*
 #pragma unroll
       for (int k = 0; k < NV; ++k)
         if (k < vpl) {
+          float f[KV];
+          slice(r, k, f);
 #pragma unroll
-          for (int e = 0; e < KV; ++e) sum[r] += RMS ? v[r][k][e] * v[r][k][e] : v[r][k][e];
+          for (int e = 0; e < KV; ++e) sum[r] += RMS ? f[e] * f[e] : f[e];
         }
     } else {
       for (int vi = sub; vi < nvec && active[r]; vi += LPR) {
@@ -102,8 +128,10 @@ __global__ void __launch_bounds__(256) norm_kernel(const T* __restrict__ src, T*
         for (int k = 0; k < NV; ++k) {
           const int vi = sub + k * LPR;
           if (k < vpl && active[r] && vi < nvec) {
+            float f[KV];
+            slice(r, k, f);
 #pragma unroll
-            for (int e = 0; e < KV; ++e) sq += (v[r][k][e] - mean[r]) * (v[r][k][e] - mean[r]);
+            for (int e = 0; e < KV; ++e) sq += (f[e] - mean[r]) * (f[e] - mean[r]);
           }
         }
       } else {
@@ -135,7 +163,11 @@ __global__ void __launch_bounds__(256) norm_kernel(const T* __restrict__ src, T*
         if constexpr (!RMS) ElemIO<T>::load(beta + vi * KV, b);
 #pragma unroll
         for (int r = 0; r < RPG; ++r)
-          if (active[r]) emit(r, vi, v[r][k], g, b);
+          if (active[r]) {
+            float f[KV];
+            slice(r, k, f);
+            emit(r, vi, f, g, b);
+          }
       }
     }
   } else {
@@ -352,14 +384,6 @@ __device__ __forceinline__ uint4 ld_vec16(const __nv_bfloat16* p, bool aligned16
   if (aligned16) return *reinterpret_cast<const uint4*>(p);
   const uint32_t* q = reinterpret_cast<const uint32_t*>(p);
   return make_uint4(q[0], q[1], q[2], q[3]);
-}
-__device__ __forceinline__ void unpack8_bf16(const uint4& u, float (&f)[8]) {
-  const uint32_t w[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    f[2 * q] = __uint_as_float(w[q] << 16);
-    f[2 * q + 1] = __uint_as_float(w[q] & 0xFFFF0000u);
-  }
 }
 
 // Channel of slot k of a thread with channel row cr: slots come in adjacent pairs (2 cr, 2 cr + 1) + 64 (k / 2), so the
