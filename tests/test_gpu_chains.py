@@ -129,6 +129,18 @@ def test_plain_linear_shapes():
         assert_close_bf16(to_host_f64(out), synth.to_f64(a) @ synth.to_f64(w).T, f"linear {M}x{N}x{K}")
 
 
+def test_linear_shapes_that_run_on_cta_pairs():
+    """Enough 256-wide tiles for more than one wave, an even number of row tiles: two SMs share a 256 x 256 tile.  The
+    short reduction takes the epilogue that releases its accumulator early, the long one the general epilogue; the ragged M
+    leaves the last pair tile with out-of-range rows in its second half."""
+    for M, N, K in [(2304, 2304, 576), (2264, 2304, 576), (2560, 2048, 1280)]:
+        a = synth.normal(6, M + N, (M, K), dtype="bf16")
+        w = synth.normal(6, K + N + 1, (N, K), std=K ** -0.5, dtype="bf16")
+        out = run_plan([sm.make_op(sm.OP_LINEAR, side_input=(1, 0))], [sm.make_desc((M, K)), sm.make_desc((N, K))],
+                       sm.ELIMINATE, [to_dev(a), to_dev(w)], (M, N))
+        assert_close_bf16(to_host_f64(out), synth.to_f64(a) @ synth.to_f64(w).T, f"linear {M}x{N}x{K}")
+
+
 def test_run_chain_rejects_bad_arguments():
     plan = sm.smartmem_plan([sm.make_op(sm.OP_TRANSPOSE, perm=(1, 0)), sm.make_op(sm.OP_COPY)],
                             [sm.make_desc((64, 64))], sm.EXPLICIT)
