@@ -136,7 +136,7 @@ template <int BN, int STAGES, bool A_MN, bool PAIR, bool LEAN>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ GemmArgs g) {
-  static_assert(!PAIR || (BN == 256 && !A_MN), "CTA pairs: 256-wide tiles, K-major A");
+  static_assert(!PAIR || ((BN == 256 || BN == 128) && !A_MN), "CTA pairs: 256- or 128-wide tiles, K-major A");
   static_assert(!LEAN || PAIR, "the lean epilogue comes with CTA pairs");
   constexpr int BN_CTA = PAIR ? BN / 2 : BN;               // rows of B this CTA loads
   constexpr int B_STAGE_BYTES = BN_CTA * BK * 2;
@@ -714,6 +714,19 @@ int build_operand(const TcOperand& op, int tile_rows, int box_rows, CUtensorMap*
   return encode_cached(op.ptr, rank, dims, strides, box, tm);
 }
 
+// every offset the map can produce is a multiple of `q` elements
+bool devmap_offsets_multiple_of(const DevMap& m, long long q) {
+  if (m.base % q) return false;
+  for (int a = 0; a < m.n_atoms; ++a)
+    if (m.roll_of[a] < 0 && m.stride[a] % q) return false;
+  for (int r = 0; r < m.n_rolls; ++r) {
+    if (m.roll_stride[r] % q) return false;
+    for (int i = 0; i < m.roll_n_parts[r] && m.roll_n_parts[r] > 1; ++i)
+      if (m.roll_part_stride[r][i] % q) return false;
+  }
+  return true;
+}
+
 int sm_count() {
   static int n = 0;
   if (n == 0) {
@@ -862,10 +875,18 @@ int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep,
   // SMARTMEM_GEMM_PAIR=0 keeps every GEMM on single CTAs (for measuring what pairing buys).
   static const int allow_pair = [] { const char* e = getenv("SMARTMEM_GEMM_PAIR"); return (e && e[0] == '0') ? 0 : 1; }();
   const long long tiles_m1 = (M + BM - 1) / BM;
-  const bool pair = allow_pair && bn == 256 && !a_mn && tiles_m1 % 2 == 0 && nkb > 4 && N % 256 == 0 &&
-                    tiles_m1 * ((N + bn - 1) / bn) * batch > tc_sm_count() &&
-                    !ep.rowmap && ep.seg_cols == 0 && !ep.out2 && ep.ldc % 16 == 0 && ep.out_batch_stride % 16 == 0 &&
-                    ((uintptr_t)ep.out & 31) == 0;                     // (its epilogue writes 32-byte vectors)
+  const bool pair = allow_pair && (bn == 256 || bn == 128) && !a_mn && tiles_m1 % 2 == 0 && nkb > 4 && N % 256 == 0 &&
+              tiles_m1 * (N / 256) * batch > tc_sm_count() &&
+              (!ep.rowmap || devmap_offsets_multiple_of(*ep.rowmap, 16)) && ep.seg_cols == 0 && !ep.out2 && ep.ldc % 16 == 0 &&
+              ep.out_batch_stride % 16 == 0 && ((uintptr_t)ep.out & 31) == 0;   // (its epilogue writes 32-byte vectors)
+  if (pair) {
+    // width of a pair's tile: 256 unless the last wave of 256-wide tiles is so ragged that the waves of half the width
+    // are shorter.  Microseconds per tile, fitted to measurements: per k-block a 256-wide tile costs its products and a
+    // 128-wide one its operand feed (about 2/3 of that), plus a fixed part for the epilogue the ring cannot hide.
+    const long long pairs = tc_sm_count() / 2, t256 = tiles_m1 / 2 * (N / 256) * batch;
+    const long long w256 = (t256 + pairs - 1) / pairs, w128 = (2 * t256 + pairs - 1) / pairs;
+    bn = (ep.rope_cols == 0 && w128 * (nkb * 0.21 + 1.2) < w256 * (nkb * 0.33 + 2.2)) ? 128 : 256;
+  }
   GemmArgs g;
   memset(&g, 0, sizeof(g));
   CUtensorMap ta, tb;
@@ -903,8 +924,9 @@ int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep,
   g.fd_tiles_m = make_fastdiv((uint32_t)g.tiles_m);
   g.batch = (int)batch;
   if ((long long)g.tiles_n * g.tiles_m * g.batch >= (1ll << 31)) return SMARTMEM_ERR_UNSUPPORTED;
-  if (pair && nkb <= 16 && ep.rope_cols == 0 && !ep.residual) return launch_t<256, 6, false, true, true>(ta, tb, g, st);
-  if (pair) return launch_t<256, 6, false, true>(ta, tb, g, st);
+  if (pair && bn == 256 && nkb <= 16 && ep.rope_cols == 0 && !ep.residual) return launch_t<256, 6, false, true, true>(ta, tb, g, st);
+  if (pair && bn == 256) return launch_t<256, 6, false, true>(ta, tb, g, st);
+  if (pair) return launch_t<128, 8, false, true>(ta, tb, g, st);
 #define SM_CASE(BN_, ST_, MN_)                                                                  \
   if (bn == BN_ && stages == ST_ && a_mn == MN_) return launch_t<BN_, ST_, MN_>(ta, tb, g, st);
   SM_CASE(256, 3, false) SM_CASE(256, 4, false) SM_CASE(128, 4, false) SM_CASE(96, 6, false) SM_CASE(64, 6, false)
