@@ -58,6 +58,7 @@ struct GemmArgs {
   __nv_bfloat16* out2;                   // second copy of the result, transposed inside groups of out2_S rows (null: none)
   FastDiv fd_out2_S;
   int* status;
+  int tma_out;                           // lean epilogue: the output leaves as TMA boxes (tensor map tmC) instead of per-thread stores
   DevMap rowmap;
 };
 
@@ -135,7 +136,7 @@ constexpr int kThreads = 64 + 32 * kEpiWarps + 32;      // + a second TMA produc
 template <int BN, int STAGES, bool A_MN, bool PAIR, bool LEAN>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-               const __grid_constant__ GemmArgs g) {
+               const __grid_constant__ CUtensorMap tmC, const __grid_constant__ GemmArgs g) {
   static_assert(!PAIR || ((BN == 256 || BN == 128) && !A_MN), "CTA pairs: 256- or 128-wide tiles, K-major A");
   static_assert(!LEAN || PAIR, "the lean epilogue comes with CTA pairs");
   constexpr int BN_CTA = PAIR ? BN / 2 : BN;               // rows of B this CTA loads
@@ -148,7 +149,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   uint8_t* smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
   uint8_t* sA = smem;
   uint8_t* sB = smem + STAGES * A_STAGE_BYTES;
-  uint64_t* full = reinterpret_cast<uint64_t*>(sB + STAGES * B_STAGE_BYTES);
+  // lean epilogue: a 32 x 32 output box per epilogue warp (64-byte rows, 64-byte swizzle), right behind the ring
+  constexpr int CBOX_BYTES = 32 * 64;
+  uint8_t* cstage = sB + STAGES * B_STAGE_BYTES;
+  uint64_t* full = reinterpret_cast<uint64_t*>(cstage + (LEAN ? kEpiWarps * CBOX_BYTES : 0));
   uint64_t* empty = full + STAGES;
   uint64_t* tmem_full = empty + STAGES;                      // [2]
   uint64_t* tmem_empty = tmem_full + 2;                      // [2]
@@ -181,6 +185,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   if (warp == 0 && lane == 0) {
     ptx::prefetch_tensormap(&tmA);
     ptx::prefetch_tensormap(&tmB);
+    if (LEAN && g.tma_out) ptx::prefetch_tensormap(&tmC);
   }
   if (warp == 1) {
     if constexpr (PAIR) ptx::tmem_alloc_pair(tmem_slot, TMEM_COLS);
@@ -537,7 +542,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if constexpr (DIRECT) {
             // 64 contiguous bytes of the thread's own row per round, as two 32-byte stores: whole sectors, and the
             // shared memory (whose bandwidth the operands need) is left to the ring, which gets six stages
-            if (v & 1) {
+            if (LEAN && g.tma_out) {
+              // lean epilogue: the warp's 32 x 32 box goes through its own 2 KB of shared memory and leaves as one TMA
+              // store -- a row-per-thread store touches 32 lines per instruction, and those stores and the next tile's
+              // operand loads were in each other's way
+              if (v == 0) {
+                if (lane == 0) ptx::bulk_wait_group_read<0>();     // the previous round's box has been read
+                __syncwarp();
+              }
+              *reinterpret_cast<uint4*>(cstage + e * CBOX_BYTES + lane * 64 + ((v ^ ((lane >> 1) & 3)) << 4)) = pk;
+              if (v == VPR - 1) {
+                ptx::fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) {
+                  ptx::tma_store_2d(&tmC, cstage + e * CBOX_BYTES, n0 + c0, (int)tile_m * BM + q * 32);
+                  ptx::bulk_commit_group();
+                }
+              }
+            } else if (v & 1) {
               if (row_ok) ptx::st_global_v8(out_t + off + n0 + c0 + (v - 1) * 8, pk_prev, pk);
             } else {
               pk_prev = pk;
@@ -738,11 +760,11 @@ int sm_count() {
 }
 
 template <int BN, int STAGES, bool A_MN, bool PAIR = false, bool LEAN = false>
-int launch_t(const CUtensorMap& ta, const CUtensorMap& tb, const GemmArgs& g, cudaStream_t st) {
+int launch_t(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, const GemmArgs& g, cudaStream_t st) {
   constexpr bool QST = !PAIR && !(BN == 256 && STAGES == 4);
   constexpr int RCc = !QST ? 16 : ((BN / 4) > 32 ? 32 : (BN / 4));
   constexpr size_t smem = 1024 + STAGES * (A_STAGE_BYTES + (PAIR ? BN / 2 : BN) * BK * 2) + (2 * STAGES + 4) * 8 + 16 +
-                          (PAIR ? 0 : !QST ? kEpiWarps * 32 * (RCc * 2 + 16) : 4 * 32 * (BN * 2 + 16));   // pairs store from registers
+                          (LEAN ? kEpiWarps * 32 * 64 : PAIR ? 0 : !QST ? kEpiWarps * 32 * (RCc * 2 + 16) : 4 * 32 * (BN * 2 + 16));   // pairs store from registers
   if (ensure_max_dynamic_smem((const void*)gemm_tc_kernel<BN, STAGES, A_MN, PAIR, LEAN>, (int)smem) != SMARTMEM_OK) return SMARTMEM_ERR_CUDA;
   profile_tick("gemm_tc", st);
   const long long tiles = (long long)g.tiles_n * g.tiles_m * g.batch;
@@ -750,10 +772,10 @@ int launch_t(const CUtensorMap& ta, const CUtensorMap& tb, const GemmArgs& g, cu
     // one cluster of two CTAs per tile of 256 rows; the two CTAs of a cluster are neighbours in blockIdx.x
     const long long pairs = sm_count() / 2;
     const unsigned grid = (unsigned)(2 * (tiles < pairs ? tiles : pairs));
-    launch_pdl_cluster(gemm_tc_kernel<BN, STAGES, A_MN, PAIR, LEAN>, dim3(grid), dim3(kThreads), smem, st, 2u, ta, tb, g);
+    launch_pdl_cluster(gemm_tc_kernel<BN, STAGES, A_MN, PAIR, LEAN>, dim3(grid), dim3(kThreads), smem, st, 2u, ta, tb, tc, g);
   } else {
     const unsigned grid = (unsigned)(tiles < sm_count() ? tiles : sm_count());
-    launch_pdl(gemm_tc_kernel<BN, STAGES, A_MN, PAIR, LEAN>, dim3(grid), dim3(kThreads), smem, st, ta, tb, g);
+    launch_pdl(gemm_tc_kernel<BN, STAGES, A_MN, PAIR, LEAN>, dim3(grid), dim3(kThreads), smem, st, ta, tb, tc, g);
   }
   count_launch();
   return cudaGetLastError() == cudaSuccess ? SMARTMEM_OK : SMARTMEM_ERR_CUDA;
@@ -924,11 +946,20 @@ int launch_gemm_tc(const TcOperand& A, const TcOperand& B, const TcEpilogue& ep,
   g.fd_tiles_m = make_fastdiv((uint32_t)g.tiles_m);
   g.batch = (int)batch;
   if ((long long)g.tiles_n * g.tiles_m * g.batch >= (1ll << 31)) return SMARTMEM_ERR_UNSUPPORTED;
-  if (pair && bn == 256 && nkb <= 16 && ep.rope_cols == 0 && !ep.residual) return launch_t<256, 6, false, true, true>(ta, tb, g, st);
-  if (pair && bn == 256) return launch_t<256, 6, false, true>(ta, tb, g, st);
-  if (pair) return launch_t<128, 8, false, true>(ta, tb, g, st);
+  CUtensorMap tc = ta;                                     // (a valid map for the kernels that store without TMA)
+  if (pair && bn == 256 && nkb <= 16 && ep.rope_cols == 0 && !ep.residual) {
+    if (batch == 1 && !ep.rowmap) {                        // output as 32 x 32 boxes of [M, N] with pitch ldc
+      const uint64_t dims[2] = {(uint64_t)N, (uint64_t)M}, strides[1] = {(uint64_t)ep.ldc * 2};
+      const uint32_t box[2] = {32, 32};
+      if (encode_cached(ep.out, 2, dims, strides, box, &tc, 64) == SMARTMEM_OK) g.tma_out = 1;
+      else tc = ta;
+    }
+    return launch_t<256, 6, false, true, true>(ta, tb, tc, g, st);
+  }
+  if (pair && bn == 256) return launch_t<256, 6, false, true>(ta, tb, tc, g, st);
+  if (pair) return launch_t<128, 8, false, true>(ta, tb, tc, g, st);
 #define SM_CASE(BN_, ST_, MN_)                                                                  \
-  if (bn == BN_ && stages == ST_ && a_mn == MN_) return launch_t<BN_, ST_, MN_>(ta, tb, g, st);
+  if (bn == BN_ && stages == ST_ && a_mn == MN_) return launch_t<BN_, ST_, MN_>(ta, tb, tc, g, st);
   SM_CASE(256, 3, false) SM_CASE(256, 4, false) SM_CASE(128, 4, false) SM_CASE(96, 6, false) SM_CASE(64, 6, false)
   SM_CASE(256, 3, true) SM_CASE(256, 4, true) SM_CASE(128, 4, true)
 #undef SM_CASE
