@@ -401,6 +401,7 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int q = warp & 3;
     const int rounds = C / 32;
     const f32x2 half2 = ptx::pack2(0.5f, 0.5f);
+    const bool wide_store = (reinterpret_cast<uintptr_t>(g.out) & 31) == 0;
     bool ok = w_ok;
 #pragma unroll 1
     for (int ti = 0; ti < my_tiles && ok; ++ti) {
@@ -421,6 +422,7 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive(out_empty);
         }
+        uint4 o_prev = make_uint4(0, 0, 0, 0);
 #pragma unroll
         for (int v = 0; v < 4; ++v) {
           uint32_t o[4];
@@ -430,7 +432,14 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             ptx::unpack2(ptx::mul2(ptx::pack2(__uint_as_float(rv[v * 8 + 2 * i]), __uint_as_float(rv[v * 8 + 2 * i + 1])), half2), xa, xb);
             o[i] = float2_to_bf16x2(xa, xb);
           }
-          if (row_ok) *reinterpret_cast<uint4*>(g.out + off + r * 32 + v * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+          // whole 32-byte sectors per store when the output is aligned for it (rows are 128 or 192 bytes apart)
+          if (wide_store) {
+            if (v & 1) {
+              if (row_ok) ptx::st_global_v8(g.out + off + r * 32 + (v - 1) * 8, o_prev, make_uint4(o[0], o[1], o[2], o[3]));
+            } else {
+              o_prev = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+          } else if (row_ok) *reinterpret_cast<uint4*>(g.out + off + r * 32 + v * 8) = make_uint4(o[0], o[1], o[2], o[3]);
         }
       }
     }

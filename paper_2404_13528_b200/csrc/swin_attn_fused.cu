@@ -775,6 +775,7 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
     const int r = q * 32 + lane;
     const int i = r & 63;
     const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
+    const bool wide_store = (reinterpret_cast<uintptr_t>(g.y) & 31) == 0;
     bool ok = true;
     for (int ul = 0; ul < U && ok; ++ul) {
       ok = ptx::mbar_wait_relaxed(y_full, ul & 1, abort_flag, g.status, 32);
@@ -794,6 +795,7 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
           if (lane == 0) ptx::mbar_arrive(y_empty);
         }
         if (valid) {
+          uint4 o_prev = make_uint4(0, 0, 0, 0);
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
             const float4 b0 = *reinterpret_cast<const float4*>(bp_s + k * 32 + c * 8);
@@ -807,7 +809,13 @@ swin_attn_fused_kernel(const __grid_constant__ CUtensorMap tmWq, const __grid_co
               ptx::unpack2(ptx::add2(ptx::pack2(__uint_as_float(rv[col]), __uint_as_float(rv[col + 1])), bb[e]), v0, v1);
               o4[e] = float2_to_bf16x2(v0, v1);
             }
-            yg[k * 4 + c] = make_uint4(o4[0], o4[1], o4[2], o4[3]);
+            // whole 32-byte sectors per store when y is aligned for it (rows are 128 or 192 bytes apart)
+            if (wide_store) {
+              if (c & 1) ptx::st_global_v8(yg + k * 4 + c - 1, o_prev, make_uint4(o4[0], o4[1], o4[2], o4[3]));
+              else o_prev = make_uint4(o4[0], o4[1], o4[2], o4[3]);
+            } else {
+              yg[k * 4 + c] = make_uint4(o4[0], o4[1], o4[2], o4[3]);
+            }
           }
         }
       }
