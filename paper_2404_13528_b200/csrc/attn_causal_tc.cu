@@ -266,6 +266,7 @@ causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     if (ok) {
       ptx::tc_fence_after();
       const float inv = 1.f / l;
+      const bool wide_store = (reinterpret_cast<uintptr_t>(g.out) & 31) == 0 && g.o_sn % 16 == 0 && g.o_sh % 16 == 0 && g.o_st % 16 == 0;
       __nv_bfloat16* orow = g.out + (long long)b * g.o_sn + (long long)h * g.o_sh + (long long)qi * g.o_st;
       const uint32_t to = tmem_base + TM_O + lane_addr;
 #pragma unroll 1
@@ -273,7 +274,16 @@ causal_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         uint32_t rv[32];
         ptx::tmem_ld32(to + ch * 32, rv);
         ptx::tmem_ld_wait();
-        if (qi < g.S) {
+        if (qi < g.S && wide_store) {                    // whole 32-byte sectors per store
+#pragma unroll
+          for (int v = 0; v < 2; ++v) {
+            uint32_t w[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+              w[e] = float2_to_bf16x2(__uint_as_float(rv[v * 16 + 2 * e]) * inv, __uint_as_float(rv[v * 16 + 2 * e + 1]) * inv);
+            ptx::st_global_v8(orow + ch * 32 + v * 16, make_uint4(w[0], w[1], w[2], w[3]), make_uint4(w[4], w[5], w[6], w[7]));
+          }
+        } else if (qi < g.S) {
 #pragma unroll
           for (int v = 0; v < 4; ++v) {
             float o8[8];

@@ -270,6 +270,7 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
     float inv_prev = 0.f;
     int n_prev = -1;
     bool ok = true;
+    const bool wide_store = (reinterpret_cast<uintptr_t>(a.o.ptr) & 31) == 0 && a.o.sn % 16 == 0 && a.o.sh % 16 == 0 && a.o.st % 16 == 0;
     auto epilogue = [&](int u, float inv, int n) {     // O(u) -> global
       const int ob = u & 1;                            // == gi
       ok = ok && ptx::mbar_wait(&o_full[ob], (u >> 1) & 1, abort_flag, g.status);
@@ -283,12 +284,23 @@ win_attn_tc_kernel(const __grid_constant__ CUtensorMap tm0, const __grid_constan
       if (lane == 0) ptx::mbar_arrive(&o_empty[ob]);
       if (i < T && n < a.n_windows) {
         __nv_bfloat16* dst = (__nv_bfloat16*)a.o.ptr + (long long)n * a.o.sn + (long long)h * a.o.sh + (long long)i * a.o.st;
+        if (wide_store) {                              // whole 32-byte sectors per store
 #pragma unroll
-        for (int v = 0; v < 4; ++v) {
-          float o8[8];
+          for (int v = 0; v < 2; ++v) {
+            uint32_t w[8];
 #pragma unroll
-          for (int e = 0; e < 8; ++e) o8[e] = __uint_as_float(rv[v * 8 + e]) * inv;
-          ElemIO<__nv_bfloat16>::store(dst + v * 8, o8);
+            for (int e = 0; e < 8; ++e)
+              w[e] = float2_to_bf16x2(__uint_as_float(rv[v * 16 + 2 * e]) * inv, __uint_as_float(rv[v * 16 + 2 * e + 1]) * inv);
+            ptx::st_global_v8(dst + v * 16, make_uint4(w[0], w[1], w[2], w[3]), make_uint4(w[4], w[5], w[6], w[7]));
+          }
+        } else {
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            float o8[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) o8[e] = __uint_as_float(rv[v * 8 + e]) * inv;
+            ElemIO<__nv_bfloat16>::store(dst + v * 8, o8);
+          }
         }
       }
     };
