@@ -345,6 +345,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     uint8_t* qstage = stage_base + q * (32 * QROW);
     uint32_t it = 0;
     bool ok = true;
+    const bool res_wide = (reinterpret_cast<uintptr_t>(g.residual) & 31) == 0;   // (row offsets of a pair's output are multiples of 16 elements)
     constexpr bool PREFETCH_NEXT = false;                   // (tried: next-tile offset + residual a tile ahead; the extra live registers spill and it is slower)
     long long off_next = 0;
     uint4 res_next[VPR];
@@ -390,6 +391,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
       uint4 res[VPR];
       auto fetch_res = [&](int c0) {
+        if constexpr (DIRECT) {                              // (pairs: full tiles, 32-byte aligned rows) whole sectors per load
+          if (rrow && row_ok && res_wide) {
+#pragma unroll
+            for (int v = 0; v < VPR; v += 2) ptx::ld_global_v8(rrow + n0 + c0 + v * 8, res[v], res[v + 1]);
+            return;
+          }
+        }
 #pragma unroll
         for (int v = 0; v < VPR; ++v) {
           res[v] = make_uint4(0, 0, 0, 0);
