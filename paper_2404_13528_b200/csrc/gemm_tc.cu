@@ -340,6 +340,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int q = warp & 3;                                  // TMEM lane quadrant this warp may read
     const int grp = e >> 2;
     constexpr bool QSTAGE = !DIRECT && !(BN == 256 && STAGES == 4);  // per-quadrant staging of whole rows
+    constexpr bool QBULK = BN == 256 && !A_MN;               // staged rows leave as bulk copies (512-byte rows; not the MN-major-A kernel: 13.1 vs 12.1 us)
     constexpr int QROW = BN * 2 + 16;                        // bytes; the pad keeps phase 1 conflict-free
     uint8_t* stage = stage_base + e * (32 * STG_ROW);
     uint8_t* qstage = stage_base + q * (32 * QROW);
@@ -432,6 +433,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       if (!ok) break;
       ptx::tc_fence_after();
       const uint32_t taddr = tmem_base + buf * ACC_COLS + ((uint32_t)(q * 32) << 16);
+      if constexpr (QSTAGE && QBULK) {
+        // the previous tile's row copies have read the staging rows before anyone overwrites them
+        if (lane < 8) ptx::bulk_wait_group_read<0>();
+        asm volatile("bar.sync %0, 128;" ::"r"(1 + q) : "memory");
+      }
 
       // EARLY: the whole accumulator slice of the thread (ROUNDS x RC values) moves to registers first and the buffer goes
       // back to the issuing warp before any arithmetic or store, so the next tile but one starts as early as it can
@@ -593,9 +599,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           else ptx::mbar_arrive(&tmem_empty[buf]);
         }
       }
-      if constexpr (QSTAGE) {
+      if constexpr (QSTAGE && QBULK) {
+        // the four warps of the quadrant have filled a 32 x 256 staging tile: every 512-byte row leaves as one bulk copy
+        // (shared memory -> global), eight rows per warp, so no thread spends instructions on moving the tile.  Measured:
+        // the batched q k^T GEMM 78.4 -> 72.6 us; on 192-byte rows (the 96-wide scatter GEMM) the same was slower, 22.3 vs
+        // 20.7 us, so narrower tiles keep the vector loop below.
+        ptx::fence_proxy_async();
+        asm volatile("bar.sync %0, 128;" ::"r"(1 + q) : "memory");
+        const int rr = grp * 8 + (lane & 7);
+        const long long roff = __shfl_sync(0xFFFFFFFFu, off, rr);
+        const int rok = __shfl_sync(0xFFFFFFFFu, (int)row_ok, rr);
+        const int ncols = g.N - n0 < BN ? g.N - n0 : BN;
+        if (lane < 8) {
+          if (rok) ptx::bulk_store(out_t + roff + n0, qstage + rr * QROW, (uint32_t)ncols * 2u);
+          ptx::bulk_commit_group();
+        }
+      } else if constexpr (QSTAGE) {
         // the four warps of the quadrant have filled a 32 x BN staging tile: store whole rows
-        // (one bulk copy per row was tried here: 22.3 vs 20.7 us on the 96-wide scatter GEMM, so the vector loop stays)
         constexpr int VR = BN / 8;                           // 16-byte vectors per row
         asm volatile("bar.sync %0, 128;" ::"r"(1 + q) : "memory");
         const int tq = grp * 32 + lane;
