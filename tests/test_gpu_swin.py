@@ -103,6 +103,13 @@ def test_config3_swin_t_stage1_full_size():
     case(3, B=32, H=56, W=56, C=96, heads=3, window=7, shift=3, mlp_ratio=4, dtype="bf16", images=[0, 31])
 
 
+def test_wide_block_on_cta_pairs_with_a_ragged_last_tile():
+    """B=18, 14x14, C=512: 3528 rows = 27 full row tiles and 72 rows of a 28th, so the GEMMs run on CTA pairs (an even number
+    of row tiles, more than a wave of 256-wide tiles) and the last pair tile ends inside its second CTA's rows: the output
+    boxes of the lean epilogue are clipped by their tensor map, the per-thread stores of the others by the row bound."""
+    case(4, B=18, H=14, W=14, C=512, heads=16, window=7, shift=3, mlp_ratio=4, dtype="bf16", images=[0, 17])
+
+
 def test_config4_swin_b_stage3_block_pair():
     """B=64, 14x14, C=512, 16 heads: a regular block then a shifted block with independent weights."""
     B, H, W, C, heads, ws = 64, 14, 14, 512, 16, 7
